@@ -1,0 +1,309 @@
+"""Pins for the fp64 oracle: every check here compares the oracle with something
+other than itself (published values, closed forms, hand-worked numbers,
+identities the paper states, finite differences, exact summation)."""
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import prsgd_oracle as orc
+from paper_1807_06629_b200 import synth
+
+
+# ---------------------------------------------------------------- the draw
+def test_splitmix64_published_vector(golden_dir):
+    with open(os.path.join(golden_dir, "splitmix64_seed1234567.txt")) as f:
+        want = [int(s) for s in f.read().split("\n") if s and not s.startswith("#")]
+    assert orc.splitmix64_stream(1234567, len(want)) == want
+
+
+def test_draw_block_is_two_nested_streams():
+    # block = (i+1)-th output of the stream keyed by the t-th output of the seed's stream
+    for seed, i, t, nb in [(20180717, 0, 1, 64), (20180717, 3, 17, 64), (5, 63, 256, 32), (2**63 + 11, 7, 1000, 250)]:
+        u = orc.splitmix64_stream(seed, t)[-1]
+        v = orc.splitmix64_stream(u, i + 1)[-1]
+        assert orc.draw_block(seed, i, t, nb) == v % nb
+
+
+def test_draw_block_spreads_and_decorrelates_workers():
+    nb, T, N = 16, 4000, 4
+    d = np.array([[orc.draw_block(99, i, t, nb) for t in range(1, T + 1)] for i in range(N)])
+    assert d.min() == 0 and d.max() == nb - 1
+    for i in range(N):
+        cnt = np.bincount(d[i], minlength=nb)
+        chi2 = ((cnt - T / nb) ** 2 / (T / nb)).sum()
+        assert chi2 < 45.0  # 15 dof, P(chi2 > 45) ~ 8e-5
+    # two workers must not draw the same block more often than chance (1/nb)
+    same = (d[0] == d[1]).mean()
+    assert abs(same - 1.0 / nb) < 0.02
+
+
+# ------------------------------------------------- the gradient of the MLP loss
+def test_loss_hand_worked_single_layer():
+    # W = 0, b = (ln1, ln2, ln3): softmax = (1/6, 2/6, 3/6) for any input
+    dims = (2, 3)
+    x = np.zeros(orc.param_count(dims))
+    x[6:] = np.log([1.0, 2.0, 3.0])
+    Xb = np.array([[0.3, -1.2], [2.0, 0.5]])
+    yb = np.array([2, 0])
+    loss, g = orc.mlp_loss_grad(x, dims, Xb, yb)
+    assert loss == pytest.approx(0.5 * (math.log(2.0) + math.log(6.0)), abs=1e-14)
+    p = np.array([1 / 6, 2 / 6, 3 / 6])
+    d0 = (p - np.array([0, 0, 1.0])) / 2
+    d1 = (p - np.array([1.0, 0, 0])) / 2
+    gW = np.outer(d0, Xb[0]) + np.outer(d1, Xb[1])
+    assert np.allclose(g[:6].reshape(3, 2), gW, atol=1e-15)
+    assert np.allclose(g[6:], d0 + d1, atol=1e-15)
+
+
+def test_grad_hand_worked_two_layers():
+    # x = (1,-2); z1 = (1,-2,-0.5) -> a1 = (1,0,0); z2 = (0, ln3) -> softmax (1/4, 3/4); label 0
+    dims = (2, 3, 2)
+    W1 = np.array([[1.0, 0.0], [0.0, 1.0], [1.0, 1.0]])
+    b1 = np.array([0.0, 0.0, 0.5])
+    W2 = np.array([[0.0, 5.0, -7.0], [math.log(3.0), 2.0, 9.0]])
+    b2 = np.zeros(2)
+    x = np.concatenate([W1.ravel(), b1, W2.ravel(), b2])
+    loss, g = orc.mlp_loss_grad(x, dims, np.array([[1.0, -2.0]]), np.array([0]))
+    assert loss == pytest.approx(math.log(4.0), abs=1e-14)
+    (gW1, gb1), (gW2, gb2) = orc.unpack(g, dims)
+    d1 = 0.75 * math.log(3.0)
+    assert np.allclose(gW2, [[-0.75, 0, 0], [0.75, 0, 0]], atol=1e-15)
+    assert np.allclose(gb2, [-0.75, 0.75], atol=1e-15)
+    assert np.allclose(gW1, [[d1, -2 * d1], [0, 0], [0, 0]], atol=1e-15)
+    assert np.allclose(gb1, [d1, 0, 0], atol=1e-15)
+
+
+def test_uniform_logits_give_ln_C_and_zero_sum_delta():
+    dims = (5, 7, 10)
+    x = np.zeros(orc.param_count(dims))
+    rng = np.random.default_rng(0)
+    Xb = rng.standard_normal((6, 5))
+    yb = rng.integers(0, 10, 6)
+    loss, g = orc.mlp_loss_grad(x, dims, Xb, yb)
+    assert loss == pytest.approx(math.log(10.0), abs=1e-14)
+    gbL = orc.unpack(g, dims)[-1][1]
+    assert abs(gbL.sum()) < 1e-15          # sum_c delta_L[b, c] = 0 for every sample
+    want = np.full(10, 6 / 10 / 6) - np.bincount(yb, minlength=10) / 6
+    assert np.allclose(gbL, want, atol=1e-15)
+
+
+def test_single_layer_is_multinomial_logistic_regression():
+    from scipy.special import log_softmax, softmax
+    dims = (9, 4)
+    rng = np.random.default_rng(1)
+    x = rng.standard_normal(orc.param_count(dims))
+    Xb = rng.standard_normal((11, 9))
+    yb = rng.integers(0, 4, 11)
+    W, b = x[:36].reshape(4, 9), x[36:]
+    Z = Xb @ W.T + b
+    loss, g = orc.mlp_loss_grad(x, dims, Xb, yb)
+    assert loss == pytest.approx(-log_softmax(Z, axis=1)[np.arange(11), yb].mean(), rel=1e-13)
+    R = softmax(Z, axis=1)
+    R[np.arange(11), yb] -= 1
+    assert np.allclose(g[:36].reshape(4, 9), R.T @ Xb / 11, atol=1e-13)
+    assert np.allclose(g[36:], R.sum(0) / 11, atol=1e-13)
+
+
+@pytest.mark.parametrize("dims,B", [((32, 64, 10), 16), ((6, 5, 4, 3), 3)])
+def test_gradient_matches_central_differences(dims, B):
+    rng = np.random.default_rng(7)
+    x = synth.init_params(dims, seed=11).astype(np.float64)
+    x += 0.05 * rng.standard_normal(x.shape)          # non-zero biases too
+    Xb = rng.standard_normal((B, dims[0]))
+    yb = rng.integers(0, dims[-1], B)
+    # stay away from ReLU kinks: every hidden pre-activation at least 1e-4 from 0
+    a = Xb
+    for (W, b) in orc.unpack(x, dims)[:-1]:
+        z = a @ W.T + b
+        assert np.abs(z).min() > 1e-4
+        a = np.maximum(z, 0)
+    _, g = orc.mlp_loss_grad(x, dims, Xb, yb)
+    fd = np.empty_like(g)
+    for j in range(x.size):
+        h = 1e-6 * max(1.0, abs(x[j]))
+        xp, xm = x.copy(), x.copy()
+        xp[j] += h
+        xm[j] -= h
+        fd[j] = (orc.mlp_loss_grad(xp, dims, Xb, yb)[0] - orc.mlp_loss_grad(xm, dims, Xb, yb)[0]) / (2 * h)
+    rel = np.linalg.norm(g - fd) / np.linalg.norm(fd)
+    assert rel < 1e-6
+    assert np.abs(g - fd).max() < 1e-6 * max(1.0, np.abs(fd).max())
+
+
+# --------------------------------------------------------- Algorithm 1 schedule
+def _quad(a, c):
+    return lambda i, t, xi: a[i] * (xi - c[i])
+
+
+def test_brute_force_two_workers_scalar():
+    # F_i(x) = a_i/2 (x - c_i)^2, N=2, m=1, I=2, T=4, worked with scalars
+    a, c, g = [1.0, 3.0], [2.0, -1.0], 0.1
+    x0 = x1 = 0.5
+    for t in range(1, 5):
+        x0 = x0 - g * a[0] * (x0 - c[0])
+        x1 = x1 - g * a[1] * (x1 - c[1])
+        if t % 2 == 0:
+            x0 = x1 = (x0 + x1) / 2
+    out = orc.pr_sgd(np.full((2, 1), 0.5), g, 2, 4, _quad(np.array(a), np.array(c)[:, None]))
+    assert np.allclose(out[:, 0], [x0, x1], atol=1e-15)
+    # and one more step leaves the two workers different again
+    out5 = orc.pr_sgd(out, g, 2, 1, _quad(np.array(a), np.array(c)[:, None]), t0=4)
+    assert out5[0, 0] == pytest.approx(x0 - g * a[0] * (x0 - c[0]), abs=1e-15)
+    assert out5[1, 0] == pytest.approx(x1 - g * a[1] * (x1 - c[1]), abs=1e-15)
+
+
+@pytest.mark.parametrize("I", [1, 3, 5])
+def test_quadratic_closed_form_per_period(I):
+    rng = np.random.default_rng(3)
+    N, m, g = 5, 8, 0.07
+    a = rng.uniform(0.5, 2.0, N)
+    c = rng.standard_normal((N, m))
+    y0 = rng.standard_normal(m)
+    x = orc.pr_sgd(np.tile(y0, (N, 1)), g, I, I, _quad(a, c))
+    want = np.mean([c[i] + (1 - g * a[i]) ** I * (y0 - c[i]) for i in range(N)], axis=0)
+    assert np.allclose(x, want[None, :], atol=1e-13)
+
+
+def test_quadratic_equal_curvature_independent_of_I():
+    rng = np.random.default_rng(4)
+    N, m, g, T = 4, 6, 0.1, 24
+    c = rng.standard_normal((N, m))
+    y0 = rng.standard_normal(m)
+    want = c.mean(0) + (1 - g) ** T * (y0 - c.mean(0))
+    for I in (1, 2, 4, 8, 24):
+        x = orc.pr_sgd(np.tile(y0, (N, 1)), g, I, T, _quad(np.ones(N), c))
+        assert np.allclose(x, want[None, :], atol=1e-13)
+
+
+def _small_mlp_problem(N=3, dims=(6, 5, 4), B=4, P=16, seed=5):
+    w = synth.Workload("t", N, dims, B, 0.05, 2, 8, 0, P, mean_shift=0.5, gumbel=True, seed=seed)
+    X, Y = synth.make_pools(w)
+    x0 = synth.init_params(dims, seed).astype(np.float64)
+    return w, X.astype(np.float64), Y, x0
+
+
+def test_I_equals_1_is_minibatch_sgd_on_the_concatenated_batch():
+    # the third equivalent form of parallel mini-batch SGD (Introduction, footnote 1)
+    w, X, Y, x0 = _small_mlp_problem()
+    T = 6
+    out = orc.pr_sgd(np.tile(x0, (w.N, 1)), w.gamma, 1, T, orc.mlp_grad_fn(w.dims, X, Y, w.B, w.seed))
+
+    def big_batch(i, t, xi):
+        blks = [orc.draw_block(w.seed, k, t, w.n_blocks) for k in range(w.N)]
+        Xc = np.concatenate([X[k, b * w.B:(b + 1) * w.B] for k, b in enumerate(blks)])
+        Yc = np.concatenate([Y[k, b * w.B:(b + 1) * w.B] for k, b in enumerate(blks)])
+        return orc.mlp_loss_grad(xi, w.dims, Xc, Yc)[1]
+
+    single = orc.pr_sgd(x0[None, :], w.gamma, 0, T, big_batch)
+    assert np.allclose(out, single, atol=1e-13)
+    assert np.abs(out - x0).max() > 1e-3
+
+
+def test_one_worker_is_plain_sgd_whatever_I():
+    w, X, Y, x0 = _small_mlp_problem(N=1)
+    fn = orc.mlp_grad_fn(w.dims, X, Y, w.B, w.seed)
+    ref = orc.pr_sgd(x0[None, :], w.gamma, 0, 9, fn)
+    for I in (1, 2, 4, 9):
+        assert np.array_equal(orc.pr_sgd(x0[None, :], w.gamma, I, 9, fn), ref)
+    x = x0.copy()
+    for t in range(1, 10):                                    # SGD written out
+        x = x - w.gamma * fn(0, t, x)
+    assert np.allclose(ref[0], x, atol=1e-15)
+
+
+def test_rows_identical_and_equal_exact_mean_after_average():
+    w, X, Y, x0 = _small_mlp_problem(N=5)
+    fn = orc.mlp_grad_fn(w.dims, X, Y, w.B, w.seed)
+    pre = orc.pr_sgd(np.tile(x0, (w.N, 1)), w.gamma, 0, 3, fn)
+    assert np.abs(pre[0] - pre[1]).max() > 1e-6
+    g4 = np.stack([fn(i, 4, pre[i]) for i in range(w.N)])
+    post = orc.pr_sgd(pre, w.gamma, 4, 1, fn, t0=3)
+    for i in range(1, w.N):
+        assert np.array_equal(post[i], post[0])
+    stepped = pre - w.gamma * g4
+    exact = np.array([math.fsum(stepped[:, j]) / w.N for j in range(stepped.shape[1])])
+    assert np.allclose(post[0], exact, rtol=0, atol=1e-15)
+    assert np.allclose(orc.node_average(stepped), exact, rtol=0, atol=1e-15)
+
+
+@pytest.mark.parametrize("literal", [False, True])
+def test_mean_dynamics_telescoping_and_drift_bound(literal):
+    w, X, Y, x0 = _small_mlp_problem(N=4)
+    I, T = 3, 10
+    fn = orc.mlp_grad_fn(w.dims, X, Y, w.B, w.seed)
+    log = []
+    orc.pr_sgd(np.tile(x0, (w.N, 1)), w.gamma, I, T, fn, literal=literal,
+               on_step=lambda t, b, G, a, avg: log.append((t, b, G, a, avg)))
+    assert [e[4] for e in log] == [t % I == 0 for t in range(1, T + 1)]
+    ybar, acc, gmax, t0 = x0.copy(), np.zeros((w.N, x0.size)), 0.0, 0
+    for (t, before, G, after, avg) in log:
+        # Eq. (overline-x-update): holds on averaging and non-averaging iterations alike
+        assert np.allclose(after.mean(0), before.mean(0) - w.gamma * G.mean(0), atol=1e-14)
+        if literal:
+            continue
+        acc += G
+        gmax = max(gmax, np.linalg.norm(G, axis=1).max())
+        if avg:
+            assert np.allclose(after, (ybar - w.gamma * acc.mean(0))[None, :], atol=1e-13)
+            ybar, acc, gmax, t0 = after[0].copy(), np.zeros_like(acc), 0.0, t
+        else:
+            # proof of Lemma 1: x_i^t = ybar - gamma * sum_{tau=t0+1..t} G_i^tau
+            assert np.allclose(after, ybar[None, :] - w.gamma * acc, atol=1e-13)
+            drift = np.linalg.norm(after - after.mean(0)[None, :], axis=1).max()
+            assert drift <= 2 * w.gamma * (t - t0) * gmax + 1e-12
+
+
+def test_literal_reading_differs_from_restart_reading():
+    w, X, Y, x0 = _small_mlp_problem(N=3)
+    fn = orc.mlp_grad_fn(w.dims, X, Y, w.B, w.seed)
+    a = orc.pr_sgd(np.tile(x0, (w.N, 1)), w.gamma, 2, 4, fn)
+    b = orc.pr_sgd(np.tile(x0, (w.N, 1)), w.gamma, 2, 4, fn, literal=True)
+    assert np.array_equal(a[0], a[1])
+    assert np.abs(b[0] - b[1]).max() > 1e-6          # literal form: workers differ after an averaging iteration
+    # both agree up to the first averaging iteration's gradient point
+    a1 = orc.pr_sgd(np.tile(x0, (w.N, 1)), w.gamma, 2, 1, fn)
+    b1 = orc.pr_sgd(np.tile(x0, (w.N, 1)), w.gamma, 2, 1, fn, literal=True)
+    assert np.array_equal(a1, b1)
+
+
+# ------------------------------------------------ Algorithms 2 and 3 reduce to 1
+def test_alg2_schedule_values():
+    s = orc.alg2_schedule(2, 27)
+    assert s[0] == (1, 2.0)
+    assert s[7][0] == 1 and s[7][1] == pytest.approx(2 / 4)
+    assert s[26][0] == 2 and s[26][1] == pytest.approx(2 / 9)
+    assert orc.alg2_schedule(1, 64)[63] == (4, pytest.approx(1 / 16))
+
+
+def test_alg2_with_constant_schedule_is_alg1():
+    w, X, Y, x0 = _small_mlp_problem(N=3)
+    fn = orc.mlp_grad_fn(w.dims, X, Y, w.B, w.seed)
+    a = orc.pr_sgd_time_varying(np.tile(x0, (w.N, 1)), [(3, w.gamma)] * 3, fn)
+    b = orc.pr_sgd(np.tile(x0, (w.N, 1)), w.gamma, 3, 6, fn)      # two full periods, then 3 free steps
+    b = orc.pr_sgd(b, w.gamma, 0, 3, fn, t0=6)
+    assert np.allclose(a, b, atol=1e-14)
+
+
+def test_alg3_with_equal_lengths_is_alg1_and_slow_workers_stand_still():
+    w, X, Y, x0 = _small_mlp_problem(N=3)
+    fn = orc.mlp_grad_fn(w.dims, X, Y, w.B, w.seed)
+    a = orc.pr_sgd_heterogeneous(np.tile(x0, (w.N, 1)), w.gamma, [2, 2, 2], 2, fn)
+    b = orc.pr_sgd(np.tile(x0, (w.N, 1)), w.gamma, 2, 2, fn)
+    b = orc.pr_sgd(b, w.gamma, 0, 2, fn, t0=2)
+    assert np.allclose(a, b, atol=1e-14)
+    h = orc.pr_sgd_heterogeneous(np.tile(x0, (w.N, 1)), w.gamma, [3, 1, 2], 1, fn)
+    one = orc.pr_sgd(np.tile(x0, (w.N, 1)), w.gamma, 0, 1, fn)
+    assert np.allclose(h[1], one[1], atol=1e-15)                   # worker 1 took exactly one step
+
+
+# ------------------------------------------------------- planted mistakes are caught
+def test_pins_catch_a_planted_mistake(monkeypatch):
+    rng = np.random.default_rng(3)
+    N, m, g, I = 5, 8, 0.07, 3
+    a, c, y0 = rng.uniform(0.5, 2.0, N), rng.standard_normal((N, m)), rng.standard_normal(m)
+    want = np.mean([c[i] + (1 - g * a[i]) ** I * (y0 - c[i]) for i in range(N)], axis=0)
+    monkeypatch.setattr(orc, "node_average", lambda x: x.sum(0) / (x.shape[0] - 1))
+    bad = orc.pr_sgd(np.tile(y0, (N, 1)), g, I, I, _quad(a, c))
+    assert not np.allclose(bad, want[None, :], atol=1e-6)
