@@ -1,0 +1,206 @@
+/*
+ * prsgd.h -- C ABI of the PR-SGD hot path for NVIDIA B200 (sm_100a).
+ *
+ * Parallel Restarted SGD (Yu, Yang, Zhu, AAAI-19, Algorithm 1): N workers hold
+ * N copies x_i of an m-dimensional model.  Every iteration each worker takes a
+ * local SGD step x_i <- x_i - gamma * G_i on its own minibatch; every I
+ * iterations the node average y = (1/N) sum_i x_i replaces every x_i.  Here all
+ * N workers live on one GPU, stacked as the rows of one [N, m_pad] fp32 array,
+ * and F_i is an MLP with ReLU hidden layers and softmax cross-entropy averaged
+ * over the minibatch.
+ *
+ * General rules
+ *  - Every function returns an int status: PRSGD_OK (0) or a negative error
+ *    code.  Nothing throws, aborts or exits across this boundary.
+ *  - "d_" arguments are DEVICE pointers, "h_" arguments are HOST pointers;
+ *    where a pointer may be either, an explicit on_device flag says which.
+ *  - The library allocates NO device memory.  The caller owns the parameter
+ *    store, the bf16 shadow, the scratch area and the data pools, and must keep
+ *    them alive until prsgd_destroy.  The library owns only the host-side
+ *    context.
+ *  - All device work is enqueued on the CUDA stream given to prsgd_create
+ *    (a cudaStream_t passed as void*; NULL = the legacy default stream).  Calls
+ *    that return data to the host synchronise that stream; all others are
+ *    asynchronous.
+ *  - Errors found on the host (bad argument, misalignment, wrong state) are
+ *    returned by the call itself.  Errors found on the device (a bounded wait
+ *    inside a kernel that ran out) are recorded in a status word in the scratch
+ *    area and reported by the next prsgd_sync / prsgd_get_* call.
+ *  - One context may be used by one host thread at a time.
+ *  - Worker i is row i of the store, always.
+ *
+ * Layout of one row of the store (and of the bf16 shadow, in elements):
+ *    W_1 | b_1 | W_2 | b_2 | ... | W_L | b_L
+ *  W_l is row-major [d_l, d_{l-1}].  Every segment starts at a multiple of 32
+ *  elements (128 bytes in the fp32 store); the gap words and the tail up to
+ *  m_pad are zero and stay zero.  prsgd_layout reports the offsets.  The
+ *  "canonical" order used by get/set calls is the same sequence without gaps
+ *  (m floats).
+ */
+#ifndef PRSGD_H_
+#define PRSGD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define PRSGD_OK                  0
+#define PRSGD_ERR_ARG            -1  /* NULL pointer, negative count, value out of range            */
+#define PRSGD_ERR_ALIGN          -2  /* device pointer not 256-byte aligned, or a dimension the
+                                        selected precision cannot tile (see prsgd_model_spec)       */
+#define PRSGD_ERR_SIZE           -3  /* size beyond a stated maximum                                */
+#define PRSGD_ERR_STATE          -4  /* call order: e.g. local_steps before bind_data               */
+#define PRSGD_ERR_CUDA           -5  /* a CUDA runtime/driver call failed; see prsgd_last_error     */
+#define PRSGD_ERR_DEVICE_TIMEOUT -6  /* a bounded wait inside a kernel expired (status word set)    */
+
+#define PRSGD_PRECISION_FP32 0       /* fp32 GEMM operands, fp32 accumulation (CUDA cores)          */
+#define PRSGD_PRECISION_BF16 1       /* bf16 GEMM operands from the shadow, fp32 accumulation in
+                                        TMEM (tcgen05), fp32 master weights updated in place        */
+
+#define PRSGD_X_FP32 0
+#define PRSGD_X_BF16 1
+
+#define PRSGD_MAX_LAYERS 16
+
+typedef struct prsgd_ctx prsgd_ctx;   /* opaque; created by prsgd_create, freed by prsgd_destroy */
+
+/* The model F_i and the sampling of zeta_i^t.  The paper leaves F_i generic
+ * (Introduction, problem statement); this is the F_i of the workloads. */
+typedef struct {
+  int32_t  n_layers;       /* L >= 1, at most PRSGD_MAX_LAYERS                                      */
+  const int32_t* dims;     /* HOST array of L+1 entries d_0..d_L, copied by the callee              */
+  int32_t  batch;          /* B, per-worker minibatch size, 1..256; BF16: 16, 32, 64 or 128         */
+  int32_t  precision;      /* PRSGD_PRECISION_*; BF16 needs d_0..d_{L-1} to be multiples of 64      */
+  int64_t  pool_samples;   /* P, samples in each worker's pool, a positive multiple of B            */
+  uint64_t draw_seed;      /* seed of the minibatch draw, see prsgd_draw_block                      */
+} prsgd_model_spec;
+
+/* Element offsets inside one row.  w_off[l], b_off[l] for layer l+1, l = 0..L-1. */
+typedef struct {
+  int64_t m;               /* parameters per worker, canonical (no gaps)                            */
+  int64_t m_pad;           /* row length in elements, multiple of 32                                */
+  int64_t w_off[PRSGD_MAX_LAYERS];
+  int64_t b_off[PRSGD_MAX_LAYERS];
+} prsgd_layout_t;
+
+/* Row layout of the parameter store for this model (host only, no GPU needed). */
+int prsgd_layout(const prsgd_model_spec* spec, prsgd_layout_t* out);
+
+/* Bytes the caller must provide: params = N*m_pad*4; shadow = N*m_pad*2 for
+ * BF16 precision, else 0; scratch = activations, deltas, logits, losses, the
+ * draw table, one m_pad-float staging row and the status words.  Host only. */
+int prsgd_workspace_bytes(int32_t N, const prsgd_model_spec* spec,
+                          size_t* params_bytes, size_t* shadow_bytes, size_t* scratch_bytes);
+
+/* Algorithm 1, input line: N workers, learning rate gamma > 0, synchronisation
+ * interval I >= 0 (I = 0: never average automatically; I = 1: parallel
+ * mini-batch SGD).  d_params / d_shadow / d_scratch: caller-owned device
+ * memory of at least the sizes above, 256-byte aligned (d_shadow may be NULL
+ * for FP32).  The store and the scratch are zero-filled; the iteration counter
+ * starts at t = 0.  Parameters must then be set with prsgd_set_params. */
+int prsgd_create(int32_t N, const prsgd_model_spec* spec, float gamma, int32_t I,
+                 void* d_params, void* d_shadow, void* d_scratch,
+                 void* cuda_stream, prsgd_ctx** out);
+
+/* Free the host context.  Device memory stays with the caller. */
+int prsgd_destroy(prsgd_ctx* ctx);
+
+/* Per-worker data pools D_i (Introduction: each worker samples zeta_i from its
+ * own distribution).  d_X: [N][P][d_0] row-major, x_dtype PRSGD_X_FP32 for
+ * FP32 precision and PRSGD_X_BF16 for BF16 precision; d_Y: [N][P] int32 class
+ * labels in [0, d_L).  Device pointers, 256-byte aligned, kept by reference. */
+int prsgd_bind_data(prsgd_ctx* ctx, const void* d_X, int32_t x_dtype, const int32_t* d_Y);
+
+/* Copy fresh pool contents from HOST memory (same shapes and dtype as bound)
+ * into the bound device pools, asynchronously on the context's stream.  Pinned
+ * host memory makes the copy overlap-capable; pageable memory also works. */
+int prsgd_upload_data(prsgd_ctx* ctx, const void* h_X, const int32_t* h_Y);
+
+/* x_i^0 (Algorithm 1, input line: every worker starts from the same point).
+ * src holds m floats in canonical order.  worker >= 0: only that row is
+ * written; worker = -1: every row receives the same m floats.  Refreshes the
+ * bf16 shadow.  src_on_device says where src lives. */
+int prsgd_set_params(prsgd_ctx* ctx, const float* src, int32_t worker, int src_on_device);
+
+/* Whole stacked state [N][m] (canonical order per row), e.g. to resume a run. */
+int prsgd_set_params_stacked(prsgd_ctx* ctx, const float* src, int src_on_device);
+int prsgd_get_params_stacked(prsgd_ctx* ctx, float* dst, int dst_on_device);
+
+/* One worker's x_i, m floats, canonical order.  Synchronises the stream. */
+int prsgd_get_params(prsgd_ctx* ctx, float* dst, int32_t worker, int dst_on_device);
+
+/* Iterations t+1 .. t+k of Algorithm 1.  Each iteration: every active worker i
+ * draws its minibatch block prsgd_draw_block(seed, i, t, P/B), evaluates
+ * G_i^t = grad F_i(x_i^{t-1}; block) and updates x_i^t = x_i^{t-1} - gamma G_i^t
+ * in place (Eq. parallel-sgd-x-update); when I > 0 and t mod I == 0 the node
+ * average is formed from the updated models and written to every row, so each
+ * epoch of I iterations starts from a common point (the paragraph after
+ * Algorithm 1; Algorithms 2 and 3 are stated in this form).
+ * local_steps(a) followed by local_steps(b) equals local_steps(a + b).
+ * k >= 0.  Asynchronous. */
+int prsgd_local_steps(prsgd_ctx* ctx, int64_t k);
+
+/* Average and restart now, whatever t is: y = (1/N) sum_i x_i summed in worker
+ * order i = 0..N-1 in fp32, then every row (and the shadow) is overwritten
+ * with y.  After this call all N rows hold identical bits.  Asynchronous. */
+int prsgd_average(prsgd_ctx* ctx);
+
+/* xbar^t = (1/N) sum_i x_i^t (Eq. node-average-x), m floats in canonical
+ * order, WITHOUT modifying the store.  Synchronises the stream when dst is on
+ * the host. */
+int prsgd_get_average(prsgd_ctx* ctx, float* dst, int dst_on_device);
+
+/* Mean minibatch loss F_i(x_i^{t-1}; zeta_i^t) of every worker at the last
+ * iteration run; h_dst holds N floats (HOST).  Synchronises the stream. */
+int prsgd_get_losses(prsgd_ctx* ctx, float* h_dst);
+
+/* Block index every worker drew at the last iteration run (N int32, HOST). */
+int prsgd_get_draws(prsgd_ctx* ctx, int32_t* h_dst);
+
+/* Schedule controls.  set_lr: gamma^s of Algorithm 2.  set_interval: I.
+ * set_active: Algorithm 3 -- h_mask holds N bytes, worker i takes local steps
+ * only while h_mask[i] != 0 (an inactive worker keeps its point, the
+ * zero-gradient convention of the Extensions section); NULL = all active.
+ * get_step / set_step read and write the iteration counter t (resume). */
+int prsgd_set_lr(prsgd_ctx* ctx, float gamma);
+int prsgd_set_interval(prsgd_ctx* ctx, int32_t I);
+int prsgd_set_active(prsgd_ctx* ctx, const uint8_t* h_mask);
+int prsgd_get_step(prsgd_ctx* ctx, int64_t* t);
+int prsgd_set_step(prsgd_ctx* ctx, int64_t t);
+
+/* Options.  PRSGD_OPT_FUSED_AVERAGE (default 1): on an averaging iteration the
+ * update and the average run as one pass over the store instead of an update
+ * pass followed by prsgd_average's pass; both produce identical bits. */
+#define PRSGD_OPT_FUSED_AVERAGE 1
+int prsgd_set_option(prsgd_ctx* ctx, int32_t option, int64_t value);
+
+/* Number of kernels this context has launched so far. */
+int prsgd_get_launch_count(prsgd_ctx* ctx, int64_t* count);
+
+/* Wait for the stream, then report any device-side error recorded so far. */
+int prsgd_sync(prsgd_ctx* ctx);
+
+/* Text of the last error of this context (or of the last context-free call
+ * when ctx is NULL).  Library-owned, valid until the next call. */
+const char* prsgd_last_error(prsgd_ctx* ctx);
+
+/* The averaging step of Algorithm 1 on a bare array: for every column j,
+ * y_j = (1/N) sum_{i=0..N-1} P[i*row_stride + j] (fp32, summed in row order),
+ * then P[i*row_stride + j] = y_j for every i.  d_P is a device pointer,
+ * 16-byte aligned; row_stride >= m in elements and a multiple of 4; N >= 1,
+ * m >= 0.  Asynchronous on cuda_stream.  Uses no scratch memory. */
+int prsgd_average_rows(float* d_P, int64_t N, int64_t m, int64_t row_stride, void* cuda_stream);
+
+/* The minibatch draw zeta_i^t as an integer: the (i+1)-th output of a
+ * SplitMix64 stream keyed by the t-th output of the SplitMix64 stream seeded
+ * with `seed`, modulo n_blocks.  Pure host function; the device code evaluates
+ * the same function.  Returns a value in [0, n_blocks); n_blocks must be > 0. */
+uint64_t prsgd_draw_block(uint64_t seed, int32_t worker, int64_t t, uint64_t n_blocks);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PRSGD_H_ */

@@ -1,0 +1,276 @@
+"""ctypes binding of libprsgd.so: argument marshalling only.
+
+Every function of include/prsgd.h is available under its own name on `lib`
+(e.g. ``lib.prsgd_local_steps``).  The `PRSGD` class wraps a context together
+with the torch tensors that own its device memory; its methods are named after
+the C calls and do no arithmetic of their own.  There is no CPU fallback: if
+the shared library is missing this module raises on import.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+import torch
+
+from ._build import LIB_PATH
+
+PRSGD_OK = 0
+PRECISION_FP32, PRECISION_BF16 = 0, 1
+X_FP32, X_BF16 = 0, 1
+OPT_FUSED_AVERAGE = 1
+MAX_LAYERS = 16
+
+EXPORTS = [
+    "prsgd_layout", "prsgd_workspace_bytes", "prsgd_create", "prsgd_destroy", "prsgd_bind_data",
+    "prsgd_upload_data", "prsgd_set_params", "prsgd_set_params_stacked", "prsgd_get_params_stacked",
+    "prsgd_get_params", "prsgd_local_steps", "prsgd_average", "prsgd_get_average", "prsgd_get_losses",
+    "prsgd_get_draws", "prsgd_set_lr", "prsgd_set_interval", "prsgd_set_active", "prsgd_get_step",
+    "prsgd_set_step", "prsgd_set_option", "prsgd_get_launch_count", "prsgd_sync", "prsgd_last_error",
+    "prsgd_average_rows", "prsgd_draw_block",
+]
+
+
+class ModelSpec(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("dims", C.POINTER(C.c_int32)), ("batch", C.c_int32),
+                ("precision", C.c_int32), ("pool_samples", C.c_int64), ("draw_seed", C.c_uint64)]
+
+
+class Layout(C.Structure):
+    _fields_ = [("m", C.c_int64), ("m_pad", C.c_int64), ("w_off", C.c_int64 * MAX_LAYERS),
+                ("b_off", C.c_int64 * MAX_LAYERS)]
+
+
+def _load() -> C.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it first (python -m paper_1807_06629_b200._build). "
+            "There is no fallback path.")
+    lib = C.CDLL(LIB_PATH)
+    vp, i32, i64, u64 = C.c_void_p, C.c_int32, C.c_int64, C.c_uint64
+    spec_p, szp = C.POINTER(ModelSpec), C.POINTER(C.c_size_t)
+    sig = {
+        "prsgd_layout": (C.c_int, [spec_p, C.POINTER(Layout)]),
+        "prsgd_workspace_bytes": (C.c_int, [i32, spec_p, szp, szp, szp]),
+        "prsgd_create": (C.c_int, [i32, spec_p, C.c_float, i32, vp, vp, vp, vp, C.POINTER(vp)]),
+        "prsgd_destroy": (C.c_int, [vp]),
+        "prsgd_bind_data": (C.c_int, [vp, vp, i32, vp]),
+        "prsgd_upload_data": (C.c_int, [vp, vp, vp]),
+        "prsgd_set_params": (C.c_int, [vp, vp, i32, C.c_int]),
+        "prsgd_set_params_stacked": (C.c_int, [vp, vp, C.c_int]),
+        "prsgd_get_params_stacked": (C.c_int, [vp, vp, C.c_int]),
+        "prsgd_get_params": (C.c_int, [vp, vp, i32, C.c_int]),
+        "prsgd_local_steps": (C.c_int, [vp, i64]),
+        "prsgd_average": (C.c_int, [vp]),
+        "prsgd_get_average": (C.c_int, [vp, vp, C.c_int]),
+        "prsgd_get_losses": (C.c_int, [vp, vp]),
+        "prsgd_get_draws": (C.c_int, [vp, vp]),
+        "prsgd_set_lr": (C.c_int, [vp, C.c_float]),
+        "prsgd_set_interval": (C.c_int, [vp, i32]),
+        "prsgd_set_active": (C.c_int, [vp, vp]),
+        "prsgd_get_step": (C.c_int, [vp, C.POINTER(i64)]),
+        "prsgd_set_step": (C.c_int, [vp, i64]),
+        "prsgd_set_option": (C.c_int, [vp, i32, i64]),
+        "prsgd_get_launch_count": (C.c_int, [vp, C.POINTER(i64)]),
+        "prsgd_sync": (C.c_int, [vp]),
+        "prsgd_last_error": (C.c_char_p, [vp]),
+        "prsgd_average_rows": (C.c_int, [vp, i64, i64, i64, vp]),
+        "prsgd_draw_block": (u64, [u64, i32, i64, u64]),
+    }
+    for name, (res, args) in sig.items():
+        fn = getattr(lib, name)
+        fn.restype, fn.argtypes = res, args
+    return lib
+
+
+lib = _load()
+
+
+class PRSGDError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"prsgd error {code}: {msg}")
+        self.code = code
+
+
+def _check(rc: int, ctx=None) -> None:
+    if rc != PRSGD_OK:
+        raise PRSGDError(rc, (lib.prsgd_last_error(ctx) or b"").decode())
+
+
+def make_spec(dims: Sequence[int], batch: int, precision: int, pool_samples: int, seed: int):
+    arr = (C.c_int32 * len(dims))(*dims)
+    spec = ModelSpec(len(dims) - 1, C.cast(arr, C.POINTER(C.c_int32)), batch, precision, pool_samples, seed)
+    spec._keep = arr
+    return spec
+
+
+def prsgd_layout(dims, batch, precision, pool_samples, seed=0) -> Layout:
+    spec, lay = make_spec(dims, batch, precision, pool_samples, seed), Layout()
+    _check(lib.prsgd_layout(C.byref(spec), C.byref(lay)))
+    return lay
+
+
+def prsgd_workspace_bytes(N, dims, batch, precision, pool_samples, seed=0):
+    spec = make_spec(dims, batch, precision, pool_samples, seed)
+    a, b, c = C.c_size_t(), C.c_size_t(), C.c_size_t()
+    _check(lib.prsgd_workspace_bytes(N, C.byref(spec), C.byref(a), C.byref(b), C.byref(c)))
+    return a.value, b.value, c.value
+
+
+def prsgd_draw_block(seed: int, worker: int, t: int, n_blocks: int) -> int:
+    return int(lib.prsgd_draw_block(seed, worker, t, n_blocks))
+
+
+def prsgd_average_rows(P: torch.Tensor, N: int, m: int, row_stride: Optional[int] = None, stream=None) -> None:
+    """In-place node average + broadcast over the rows of a device fp32 tensor."""
+    assert P.is_cuda and P.dtype == torch.float32
+    s = stream if stream is not None else torch.cuda.current_stream(P.device)
+    with torch.cuda.device(P.device):
+        _check(lib.prsgd_average_rows(P.data_ptr(), N, m, m if row_stride is None else row_stride, s.cuda_stream))
+
+
+def _host_ptr(a: np.ndarray) -> int:
+    assert a.flags["C_CONTIGUOUS"]
+    return a.ctypes.data
+
+
+class PRSGD:
+    """One PR-SGD context plus the device tensors that back it."""
+
+    def __init__(self, N: int, dims: Sequence[int], batch: int, gamma: float, I: int, precision: int,
+                 pool_samples: int, seed: int, device: str = "cuda:0", stream: Optional[torch.cuda.Stream] = None):
+        self.N, self.dims, self.B, self.precision, self.P = N, tuple(dims), batch, precision, pool_samples
+        self.device = torch.device(device)
+        self.stream = stream if stream is not None else torch.cuda.current_stream(self.device)
+        self._spec = make_spec(dims, batch, precision, pool_samples, seed)
+        self.layout = Layout()
+        _check(lib.prsgd_layout(C.byref(self._spec), C.byref(self.layout)))
+        self.m, self.m_pad = self.layout.m, self.layout.m_pad
+        pb, sb, wb = prsgd_workspace_bytes(N, dims, batch, precision, pool_samples, seed)
+        with torch.cuda.device(self.device):
+            self.params = torch.empty(pb // 4, dtype=torch.float32, device=self.device)
+            self.shadow = torch.empty(max(sb // 2, 1), dtype=torch.bfloat16, device=self.device) if sb else None
+            self.scratch = torch.empty(wb, dtype=torch.uint8, device=self.device)
+            ctx = C.c_void_p()
+            _check(lib.prsgd_create(N, C.byref(self._spec), gamma, I, self.params.data_ptr(),
+                                    self.shadow.data_ptr() if self.shadow is not None else None,
+                                    self.scratch.data_ptr(), self.stream.cuda_stream, C.byref(ctx)))
+        self.ctx = ctx
+        self._X = self._Y = None
+
+    def _call(self, fn, *args):
+        with torch.cuda.device(self.device):
+            _check(fn(self.ctx, *args), self.ctx)
+
+    def close(self):
+        if getattr(self, "ctx", None):
+            lib.prsgd_destroy(self.ctx)
+            self.ctx = None
+
+    __del__ = close
+
+    # ---- data -------------------------------------------------------------------
+    def bind_data(self, X: torch.Tensor, Y: torch.Tensor):
+        want = torch.bfloat16 if self.precision == PRECISION_BF16 else torch.float32
+        assert X.is_cuda and Y.is_cuda and X.dtype == want and Y.dtype == torch.int32
+        assert X.is_contiguous() and Y.is_contiguous()
+        assert tuple(X.shape) == (self.N, self.P, self.dims[0]) and tuple(Y.shape) == (self.N, self.P)
+        self._X, self._Y = X, Y
+        self._call(lib.prsgd_bind_data, X.data_ptr(), X_BF16 if want == torch.bfloat16 else X_FP32, Y.data_ptr())
+
+    def upload_data(self, hX: torch.Tensor, hY: torch.Tensor):
+        assert not hX.is_cuda and not hY.is_cuda and hX.is_contiguous() and hY.is_contiguous()
+        self._call(lib.prsgd_upload_data, hX.data_ptr(), hY.data_ptr())
+
+    # ---- parameters -------------------------------------------------------------
+    def set_params(self, x, worker: int = -1):
+        if isinstance(x, torch.Tensor) and x.is_cuda:
+            assert x.dtype == torch.float32 and x.numel() == self.m and x.is_contiguous()
+            self._call(lib.prsgd_set_params, x.data_ptr(), worker, 1)
+        else:
+            a = np.ascontiguousarray(np.asarray(x, dtype=np.float32))
+            assert a.size == self.m
+            self._call(lib.prsgd_set_params, _host_ptr(a), worker, 0)
+
+    def set_params_stacked(self, x):
+        if isinstance(x, torch.Tensor) and x.is_cuda:
+            assert x.dtype == torch.float32 and x.numel() == self.N * self.m and x.is_contiguous()
+            self._call(lib.prsgd_set_params_stacked, x.data_ptr(), 1)
+        else:
+            a = np.ascontiguousarray(np.asarray(x, dtype=np.float32))
+            assert a.size == self.N * self.m
+            self._call(lib.prsgd_set_params_stacked, _host_ptr(a), 0)
+
+    def get_params_stacked(self) -> np.ndarray:
+        out = np.empty((self.N, self.m), dtype=np.float32)
+        self._call(lib.prsgd_get_params_stacked, _host_ptr(out), 0)
+        return out
+
+    def get_params(self, worker: int) -> np.ndarray:
+        out = np.empty(self.m, dtype=np.float32)
+        self._call(lib.prsgd_get_params, _host_ptr(out), worker, 0)
+        return out
+
+    # ---- Algorithm 1 ------------------------------------------------------------
+    def local_steps(self, k: int):
+        self._call(lib.prsgd_local_steps, k)
+
+    def average(self):
+        self._call(lib.prsgd_average)
+
+    def get_average(self, out=None):
+        """Node average; into a host numpy array (default), a pinned host tensor or a device tensor."""
+        if out is None:
+            out = np.empty(self.m, dtype=np.float32)
+        if isinstance(out, np.ndarray):
+            self._call(lib.prsgd_get_average, _host_ptr(out), 0)
+        else:
+            assert out.dtype == torch.float32 and out.numel() == self.m and out.is_contiguous()
+            self._call(lib.prsgd_get_average, out.data_ptr(), 1 if out.is_cuda else 0)
+        return out
+
+    def get_losses(self) -> np.ndarray:
+        out = np.empty(self.N, dtype=np.float32)
+        self._call(lib.prsgd_get_losses, _host_ptr(out))
+        return out
+
+    def get_draws(self) -> np.ndarray:
+        out = np.empty(self.N, dtype=np.int32)
+        self._call(lib.prsgd_get_draws, _host_ptr(out))
+        return out
+
+    # ---- schedule ---------------------------------------------------------------
+    def set_lr(self, gamma: float):
+        self._call(lib.prsgd_set_lr, gamma)
+
+    def set_interval(self, I: int):
+        self._call(lib.prsgd_set_interval, I)
+
+    def set_active(self, mask):
+        if mask is None:
+            self._call(lib.prsgd_set_active, None)
+        else:
+            a = np.ascontiguousarray(np.asarray(mask, dtype=np.uint8))
+            assert a.size == self.N
+            self._call(lib.prsgd_set_active, _host_ptr(a))
+
+    def get_step(self) -> int:
+        t = C.c_int64()
+        self._call(lib.prsgd_get_step, C.byref(t))
+        return t.value
+
+    def set_step(self, t: int):
+        self._call(lib.prsgd_set_step, t)
+
+    def set_option(self, option: int, value: int):
+        self._call(lib.prsgd_set_option, option, value)
+
+    def get_launch_count(self) -> int:
+        n = C.c_int64()
+        self._call(lib.prsgd_get_launch_count, C.byref(n))
+        return n.value
+
+    def sync(self):
+        self._call(lib.prsgd_sync)

@@ -1,0 +1,93 @@
+// Node average over the stacked worker axis (Algorithm 1: y = (1/N) sum_i x_i)
+// with the restart broadcast in the same pass, plus small store utilities.
+// Every column is summed in worker order i = 0..N-1 in fp32 and divided by N
+// once, so the result does not depend on the launch shape.
+#pragma once
+#include "prsgd_common.cuh"
+
+namespace prsgd {
+
+__device__ __forceinline__ float4 ld_stream(const float4* p) { return __ldcs(p); }
+__device__ __forceinline__ void st_stream(float4* p, float4 v) { __stcs(p, v); }
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  uint32_t a = __float_as_uint(lo), b = __float_as_uint(hi);
+  a += 0x7FFFu + ((a >> 16) & 1u);
+  b += 0x7FFFu + ((b >> 16) & 1u);
+  return (a >> 16) | (b & 0xFFFF0000u);
+}
+
+// MODE 0: average + broadcast in place; MODE 1: average only, written to `out` (one row).
+// One thread owns 4 consecutive columns (one 128-bit lane); the tail m % 4 is done by scalar threads.
+template <int MODE, bool SHADOW>
+__global__ void __launch_bounds__(256) average_rows_kernel(float* __restrict__ P, int64_t N, int64_t m,
+                                                           int64_t row_stride, float* __restrict__ out,
+                                                           uint16_t* __restrict__ shadow) {
+  constexpr int U = 8;
+  const int64_t cols4 = m >> 2;
+  const int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const float fN = (float)N;
+  if (c < cols4) {
+    float4* base = reinterpret_cast<float4*>(P) + c;
+    const int64_t s4 = row_stride >> 2;
+    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+    int64_t i = 0;
+    for (; i + U <= N; i += U) {
+      float4 v[U];
+#pragma unroll
+      for (int u = 0; u < U; ++u) v[u] = ld_stream(base + (i + u) * s4);
+#pragma unroll
+      for (int u = 0; u < U; ++u) { s.x += v[u].x; s.y += v[u].y; s.z += v[u].z; s.w += v[u].w; }
+    }
+    for (; i < N; ++i) {
+      float4 v = ld_stream(base + i * s4);
+      s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+    }
+    float4 y = make_float4(__fdiv_rn(s.x, fN), __fdiv_rn(s.y, fN), __fdiv_rn(s.z, fN), __fdiv_rn(s.w, fN));
+    if (MODE == 0) {
+#pragma unroll 8
+      for (int64_t r = 0; r < N; ++r) st_stream(base + r * s4, y);
+      if (SHADOW) {
+        uint2 h = make_uint2(pack_bf16x2(y.x, y.y), pack_bf16x2(y.z, y.w));
+        uint2* sb = reinterpret_cast<uint2*>(shadow) + c;
+        for (int64_t r = 0; r < N; ++r) sb[r * s4] = h;
+      }
+    } else {
+      reinterpret_cast<float4*>(out)[c] = y;
+    }
+  } else if (c < cols4 + (m & 3)) {
+    const int64_t j = (cols4 << 2) + (c - cols4);
+    float s = 0.f;
+    for (int64_t i = 0; i < N; ++i) s += P[i * row_stride + j];
+    float y = __fdiv_rn(s, fN);
+    if (MODE == 0) {
+      for (int64_t r = 0; r < N; ++r) P[r * row_stride + j] = y;
+      if (SHADOW) {
+        for (int64_t r = 0; r < N; ++r) shadow[r * row_stride + j] = (uint16_t)(pack_bf16x2(y, 0.f) & 0xFFFFu);
+      }
+    } else {
+      out[j] = y;
+    }
+  }
+}
+
+// rows 1..N-1 <- row 0 (every worker starts from the same point; Algorithm 1, input line)
+__global__ void __launch_bounds__(256) broadcast_row0_kernel(float* __restrict__ P, int64_t N, int64_t cols4,
+                                                             int64_t stride4) {
+  const int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= cols4) return;
+  float4* base = reinterpret_cast<float4*>(P) + c;
+  float4 v = base[0];
+  for (int64_t r = 1; r < N; ++r) base[r * stride4] = v;
+}
+
+// shadow <- bf16(store), whole [N][m_pad] array
+__global__ void __launch_bounds__(256) refresh_shadow_kernel(const float* __restrict__ P, uint16_t* __restrict__ S,
+                                                             int64_t total4) {
+  const int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= total4) return;
+  float4 v = reinterpret_cast<const float4*>(P)[c];
+  reinterpret_cast<uint2*>(S)[c] = make_uint2(pack_bf16x2(v.x, v.y), pack_bf16x2(v.z, v.w));
+}
+
+}  // namespace prsgd

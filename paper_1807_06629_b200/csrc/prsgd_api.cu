@@ -1,0 +1,550 @@
+// C ABI of the PR-SGD library: host-side context, layout, schedule of
+// Algorithm 1 and the kernel launches.  See include/prsgd.h for the contract.
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "prsgd_common.cuh"
+#include "kernels_f32.cuh"
+#include "kernels_avg.cuh"
+#include "kernels_bf16.cuh"
+
+using namespace prsgd;
+
+namespace {
+
+thread_local std::string g_last_error;
+
+int fail(prsgd_ctx* ctx, int code, const std::string& msg) {
+  if (ctx) ctx->err = msg;
+  g_last_error = msg;
+  return code;
+}
+
+#define CUDA_TRY(ctx, expr)                                                                   \
+  do {                                                                                        \
+    cudaError_t e__ = (expr);                                                                 \
+    if (e__ != cudaSuccess)                                                                   \
+      return fail((ctx), PRSGD_ERR_CUDA, std::string(#expr) + ": " + cudaGetErrorString(e__)); \
+  } while (0)
+
+#define LAUNCH_CHECK(ctx)                                                                      \
+  do {                                                                                         \
+    cudaError_t e__ = cudaGetLastError();                                                      \
+    if (e__ != cudaSuccess)                                                                    \
+      return fail((ctx), PRSGD_ERR_CUDA, std::string("kernel launch: ") + cudaGetErrorString(e__)); \
+    (ctx)->launches++;                                                                         \
+  } while (0)
+
+int check_spec(const prsgd_model_spec* s, std::string* why) {
+  if (!s || !s->dims) { *why = "spec or spec->dims is NULL"; return PRSGD_ERR_ARG; }
+  if (s->n_layers < 1 || s->n_layers > PRSGD_MAX_LAYERS) { *why = "n_layers out of range"; return PRSGD_ERR_ARG; }
+  for (int l = 0; l <= s->n_layers; ++l)
+    if (s->dims[l] < 1 || s->dims[l] > (1 << 20)) { *why = "a layer width is out of range"; return PRSGD_ERR_ARG; }
+  if (s->batch < 1 || s->batch > 256) { *why = "batch must be in 1..256"; return PRSGD_ERR_ARG; }
+  if (s->pool_samples < s->batch || s->pool_samples % s->batch != 0) {
+    *why = "pool_samples must be a positive multiple of batch"; return PRSGD_ERR_ARG;
+  }
+  if (s->pool_samples / s->batch > 0x7fffffffll) { *why = "too many blocks in the pool"; return PRSGD_ERR_SIZE; }
+  if (s->precision != PRSGD_PRECISION_FP32 && s->precision != PRSGD_PRECISION_BF16) {
+    *why = "unknown precision"; return PRSGD_ERR_ARG;
+  }
+  if (s->precision == PRSGD_PRECISION_BF16) {
+    if (s->batch != 16 && s->batch != 32 && s->batch != 64 && s->batch != 128) {
+      *why = "BF16 precision needs batch 16, 32, 64 or 128"; return PRSGD_ERR_ALIGN;
+    }
+    for (int l = 0; l < s->n_layers; ++l)
+      if (s->dims[l] % 64 != 0) { *why = "BF16 precision needs d_0..d_{L-1} to be multiples of 64"; return PRSGD_ERR_ALIGN; }
+  }
+  return PRSGD_OK;
+}
+
+void compute_layout(const prsgd_model_spec* s, prsgd_layout_t* out) {
+  int64_t off = 0, m = 0;
+  for (int l = 0; l < s->n_layers; ++l) {
+    const int64_t din = s->dims[l], dout = s->dims[l + 1];
+    off = round_up(off, kSegAlign);
+    out->w_off[l] = off;
+    off += din * dout;
+    off = round_up(off, kSegAlign);
+    out->b_off[l] = off;
+    off += dout;
+    m += din * dout + dout;
+  }
+  out->m = m;
+  out->m_pad = round_up(off, kSegAlign);
+}
+
+// Carve the scratch area.  With ctx == nullptr only the total is computed.
+size_t carve_scratch(int N, const prsgd_model_spec* s, int64_t m_pad, prsgd_ctx* ctx) {
+  size_t off = 0;
+  unsigned char* base = ctx ? ctx->scratch : nullptr;
+  auto take = [&](size_t bytes) -> unsigned char* {
+    unsigned char* p = base ? base + off : nullptr;
+    off += (size_t)round_up((int64_t)bytes, 256);
+    return p;
+  };
+  const int L = s->n_layers, B = s->batch;
+  auto status = take(sizeof(DeviceStatus));
+  auto draws = take(sizeof(int32_t) * N);
+  auto losses = take(sizeof(float) * N);
+  auto active = take((size_t)N);
+  auto stage = take(sizeof(float) * (size_t)m_pad);
+  if (ctx) {
+    ctx->status = reinterpret_cast<DeviceStatus*>(status);
+    ctx->draws = reinterpret_cast<int32_t*>(draws);
+    ctx->losses = reinterpret_cast<float*>(losses);
+    ctx->active = active;
+    ctx->stage_row = reinterpret_cast<float*>(stage);
+    std::memset(&ctx->buf, 0, sizeof(ctx->buf));
+  }
+  if (s->precision == PRSGD_PRECISION_FP32) {
+    for (int l = 1; l <= L; ++l) {
+      auto a = take(sizeof(float) * (size_t)N * B * s->dims[l]);
+      auto d = take(sizeof(float) * (size_t)N * B * s->dims[l]);
+      if (ctx) {
+        ctx->buf.act_f32[l] = reinterpret_cast<float*>(a);
+        ctx->buf.delta_f32[l] = reinterpret_cast<float*>(d);
+        ctx->buf.ld[l] = s->dims[l];
+      }
+    }
+  } else {
+    for (int l = 1; l <= L; ++l) {
+      const int ld = (int)round_up(s->dims[l], 64);
+      const size_t e = (size_t)N * B * ld;
+      unsigned char *abk = nullptr, *akb = nullptr, *z = nullptr;
+      if (l < L) { abk = take(2 * e); akb = take(2 * e); }
+      else z = take(4 * e);                              // logits, fp32
+      auto dbk = take(2 * e);
+      auto dkb = take(2 * e);
+      if (ctx) {
+        ctx->buf.ld[l] = ld;
+        ctx->buf.act_bk[l] = reinterpret_cast<uint16_t*>(abk);
+        ctx->buf.act_kb[l] = reinterpret_cast<uint16_t*>(akb);
+        ctx->buf.act_f32[l] = reinterpret_cast<float*>(z);
+        ctx->buf.delta_bk[l] = reinterpret_cast<uint16_t*>(dbk);
+        ctx->buf.delta_kb[l] = reinterpret_cast<uint16_t*>(dkb);
+      }
+    }
+  }
+  return off;
+}
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+int grid1d(int64_t n, int block) { return (int)((n + block - 1) / block); }
+
+// ---- copies between the canonical (gap-free) order and the padded rows -----------------
+// rows [row0, row0 + nrows) of the store <-> nrows * m floats at `lin`
+int copy_canonical(prsgd_ctx* c, float* lin, int64_t row0, int64_t nrows, bool to_store) {
+  int64_t pos = 0;
+  for (int l = 0; l < c->L; ++l) {
+    const Layer& ly = c->layer[l];
+    const int64_t seg[2] = {(int64_t)ly.d_in * ly.d_out, (int64_t)ly.d_out};
+    const int64_t offs[2] = {ly.w_off, ly.b_off};
+    for (int k = 0; k < 2; ++k) {
+      float* st = c->params + row0 * c->m_pad + offs[k];
+      float* li = lin + pos;
+      if (to_store)
+        CUDA_TRY(c, cudaMemcpy2DAsync(st, c->m_pad * 4, li, c->m * 4, seg[k] * 4, nrows, cudaMemcpyDefault, c->stream));
+      else
+        CUDA_TRY(c, cudaMemcpy2DAsync(li, c->m * 4, st, c->m_pad * 4, seg[k] * 4, nrows, cudaMemcpyDefault, c->stream));
+      pos += seg[k];
+    }
+  }
+  return PRSGD_OK;
+}
+
+int refresh_shadow(prsgd_ctx* c) {
+  if (c->precision != PRSGD_PRECISION_BF16) return PRSGD_OK;
+  const int64_t total4 = (int64_t)c->N * c->m_pad / 4;
+  refresh_shadow_kernel<<<grid1d(total4, 256), 256, 0, c->stream>>>(c->params, c->shadow, total4);
+  LAUNCH_CHECK(c);
+  return PRSGD_OK;
+}
+
+int check_device_status(prsgd_ctx* c) {
+  DeviceStatus st;
+  CUDA_TRY(c, cudaMemcpyAsync(&st, c->status, 2 * sizeof(unsigned int), cudaMemcpyDeviceToHost, c->stream));
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  if (st.error != 0) {
+    char msg[128];
+    std::snprintf(msg, sizeof msg, "a bounded wait in a kernel expired (code %u, block %u)", st.error, st.where);
+    return fail(c, PRSGD_ERR_DEVICE_TIMEOUT, msg);
+  }
+  return PRSGD_OK;
+}
+
+DrawArgs draw_args(const prsgd_ctx* c, int64_t t) {
+  DrawArgs d;
+  d.seed = c->seed; d.t = t; d.n_blocks = c->n_blocks; d.B = c->B; d.row_elems = c->dims[0];
+  return d;
+}
+
+template <int TM, bool A_PC, bool B_PC, int EPI, bool FUSE>
+void launch_gemm_f32(prsgd_ctx* c, const GemmF32Args& g) {
+  dim3 grid((g.Nn + 63) / 64, (g.M + TM - 1) / TM, FUSE ? 1 : g.N);
+  gemm_f32_kernel<TM, A_PC, B_PC, EPI, FUSE><<<grid, 256, 0, c->stream>>>(g);
+}
+
+// One iteration of Algorithm 1 on the fp32-operand path.
+int step_f32(prsgd_ctx* c, int64_t t, bool averaging) {
+  const int L = c->L, B = c->B, N = c->N;
+  const uint8_t* act_mask = c->has_mask ? c->active : nullptr;
+  const bool fuse = averaging && c->fused_average;
+  const DrawArgs dr = draw_args(c, t);
+  const float* X = static_cast<const float*>(c->X);
+
+  for (int l = 1; l <= L; ++l) {          // forward
+    const Layer& ly = c->layer[l - 1];
+    GemmF32Args g{};
+    if (l == 1) g.A = {X, c->P * (int64_t)c->dims[0], ly.d_in, 1, 1};
+    else        g.A = {c->buf.act_f32[l - 1], (int64_t)B * ly.d_in, ly.d_in, 1, 0};
+    g.Bo = {c->params + ly.w_off, c->m_pad, 1, ly.d_in, 0};
+    g.M = B; g.Nn = ly.d_out; g.K = ly.d_in; g.N = N; g.draw = dr;
+    g.out = c->buf.act_f32[l]; g.out_worker_stride = (int64_t)B * ly.d_out;
+    g.params = c->params; g.params_worker_stride = c->m_pad; g.b_off = ly.b_off;
+    g.active = act_mask;
+    if (l < L) {
+      if (B <= 32) launch_gemm_f32<32, true, true, EPI_FWD_RELU, false>(c, g);
+      else         launch_gemm_f32<64, true, true, EPI_FWD_RELU, false>(c, g);
+    } else {
+      if (B <= 32) launch_gemm_f32<32, true, true, EPI_FWD_LINEAR, false>(c, g);
+      else         launch_gemm_f32<64, true, true, EPI_FWD_LINEAR, false>(c, g);
+    }
+    LAUNCH_CHECK(c);
+  }
+  {
+    SoftmaxArgs a{};
+    a.logits = c->buf.act_f32[L]; a.delta = c->buf.delta_f32[L]; a.ldz = c->dims[L];
+    a.Y = c->Y; a.P = c->P; a.B = B; a.C = c->dims[L]; a.draw = dr;
+    a.losses = c->losses; a.draws = c->draws; a.active = act_mask;
+    softmax_ce_kernel<<<N, 256, 0, c->stream>>>(a);
+    LAUNCH_CHECK(c);
+  }
+  for (int l = L; l >= 1; --l) {          // backward, layer by layer: dX_l reads W_l before it is updated
+    const Layer& ly = c->layer[l - 1];
+    if (l > 1) {
+      GemmF32Args g{};
+      g.A = {c->buf.delta_f32[l], (int64_t)B * ly.d_out, ly.d_out, 1, 0};
+      g.Bo = {c->params + ly.w_off, c->m_pad, ly.d_in, 1, 0};
+      g.M = B; g.Nn = ly.d_in; g.K = ly.d_out; g.N = N; g.draw = dr;
+      g.out = c->buf.delta_f32[l - 1]; g.out_worker_stride = (int64_t)B * ly.d_in;
+      g.mask_src = c->buf.act_f32[l - 1];
+      g.active = act_mask;
+      if (B <= 32) launch_gemm_f32<32, true, false, EPI_DX, false>(c, g);
+      else         launch_gemm_f32<64, true, false, EPI_DX, false>(c, g);
+      LAUNCH_CHECK(c);
+    }
+    GemmF32Args g{};
+    g.A = {c->buf.delta_f32[l], (int64_t)B * ly.d_out, 1, ly.d_out, 0};
+    if (l == 1) g.Bo = {X, c->P * (int64_t)c->dims[0], ly.d_in, 1, 1};
+    else        g.Bo = {c->buf.act_f32[l - 1], (int64_t)B * ly.d_in, ly.d_in, 1, 0};
+    g.M = ly.d_out; g.Nn = ly.d_in; g.K = B; g.N = N; g.draw = dr;
+    g.out = c->params; g.out_worker_stride = c->m_pad; g.w_off = ly.w_off; g.b_off = ly.b_off;
+    g.gamma = c->gamma; g.active = act_mask;
+    if (fuse) launch_gemm_f32<64, false, false, EPI_DW, true>(c, g);
+    else      launch_gemm_f32<64, false, false, EPI_DW, false>(c, g);
+    LAUNCH_CHECK(c);
+  }
+  return PRSGD_OK;
+}
+
+int launch_average(prsgd_ctx* c) {
+  const int64_t threads = c->m_pad / 4;
+  if (c->precision == PRSGD_PRECISION_BF16)
+    average_rows_kernel<0, true><<<grid1d(threads, 256), 256, 0, c->stream>>>(c->params, c->N, c->m_pad, c->m_pad,
+                                                                            nullptr, c->shadow);
+  else
+    average_rows_kernel<0, false><<<grid1d(threads, 256), 256, 0, c->stream>>>(c->params, c->N, c->m_pad, c->m_pad,
+                                                                             nullptr, nullptr);
+  LAUNCH_CHECK(c);
+  return PRSGD_OK;
+}
+
+}  // namespace
+
+// =====================================================================================
+extern "C" {
+
+const char* prsgd_last_error(prsgd_ctx* ctx) { return ctx ? ctx->err.c_str() : g_last_error.c_str(); }
+
+uint64_t prsgd_draw_block(uint64_t seed, int32_t worker, int64_t t, uint64_t n_blocks) {
+  if (n_blocks == 0 || n_blocks > 0xffffffffull) return 0;
+  return draw_block(seed, worker, t, (uint32_t)n_blocks);
+}
+
+int prsgd_layout(const prsgd_model_spec* spec, prsgd_layout_t* out) {
+  std::string why;
+  int rc = check_spec(spec, &why);
+  if (rc != PRSGD_OK) return fail(nullptr, rc, why);
+  if (!out) return fail(nullptr, PRSGD_ERR_ARG, "out is NULL");
+  std::memset(out, 0, sizeof *out);
+  compute_layout(spec, out);
+  return PRSGD_OK;
+}
+
+int prsgd_workspace_bytes(int32_t N, const prsgd_model_spec* spec, size_t* params_bytes, size_t* shadow_bytes,
+                          size_t* scratch_bytes) {
+  std::string why;
+  int rc = check_spec(spec, &why);
+  if (rc != PRSGD_OK) return fail(nullptr, rc, why);
+  if (N < 1 || N > 65536) return fail(nullptr, PRSGD_ERR_ARG, "N must be in 1..65536");
+  prsgd_layout_t lay;
+  compute_layout(spec, &lay);
+  if (params_bytes) *params_bytes = (size_t)N * lay.m_pad * 4;
+  if (shadow_bytes) *shadow_bytes = spec->precision == PRSGD_PRECISION_BF16 ? (size_t)N * lay.m_pad * 2 : 0;
+  if (scratch_bytes) *scratch_bytes = carve_scratch(N, spec, lay.m_pad, nullptr);
+  return PRSGD_OK;
+}
+
+int prsgd_create(int32_t N, const prsgd_model_spec* spec, float gamma, int32_t I, void* d_params, void* d_shadow,
+                 void* d_scratch, void* cuda_stream, prsgd_ctx** out) {
+  std::string why;
+  int rc = check_spec(spec, &why);
+  if (rc != PRSGD_OK) return fail(nullptr, rc, why);
+  if (!out) return fail(nullptr, PRSGD_ERR_ARG, "out is NULL");
+  *out = nullptr;
+  if (N < 1 || N > 65536) return fail(nullptr, PRSGD_ERR_ARG, "N must be in 1..65536");
+  if (!(gamma > 0.f)) return fail(nullptr, PRSGD_ERR_ARG, "gamma must be > 0");
+  if (I < 0) return fail(nullptr, PRSGD_ERR_ARG, "I must be >= 0");
+  if (!d_params || !d_scratch) return fail(nullptr, PRSGD_ERR_ARG, "d_params / d_scratch is NULL");
+  if (spec->precision == PRSGD_PRECISION_BF16 && !d_shadow)
+    return fail(nullptr, PRSGD_ERR_ARG, "BF16 precision needs d_shadow");
+  if (!aligned(d_params, 256) || !aligned(d_scratch, 256) || !aligned(d_shadow, 256))
+    return fail(nullptr, PRSGD_ERR_ALIGN, "device buffers must be 256-byte aligned");
+
+  prsgd_ctx* c = new (std::nothrow) prsgd_ctx();
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "out of host memory");
+  c->N = N; c->L = spec->n_layers; c->B = spec->batch; c->precision = spec->precision;
+  for (int l = 0; l <= c->L; ++l) c->dims[l] = spec->dims[l];
+  c->P = spec->pool_samples; c->n_blocks = (uint32_t)(spec->pool_samples / spec->batch);
+  c->seed = spec->draw_seed; c->gamma = gamma; c->I = I;
+  c->stream = static_cast<cudaStream_t>(cuda_stream);
+  prsgd_layout_t lay;
+  compute_layout(spec, &lay);
+  c->m = lay.m; c->m_pad = lay.m_pad;
+  for (int l = 0; l < c->L; ++l) c->layer[l] = {c->dims[l], c->dims[l + 1], lay.w_off[l], lay.b_off[l]};
+  c->params = static_cast<float*>(d_params);
+  c->shadow = static_cast<uint16_t*>(d_shadow);
+  c->scratch = static_cast<unsigned char*>(d_scratch);
+  c->scratch_bytes = carve_scratch(N, spec, c->m_pad, c);
+
+  auto bail = [&](int code) { delete c; return code; };
+  cudaError_t e = cudaGetDevice(&c->device);
+  if (e == cudaSuccess) e = cudaMemsetAsync(c->params, 0, (size_t)N * c->m_pad * 4, c->stream);
+  if (e == cudaSuccess && c->shadow) e = cudaMemsetAsync(c->shadow, 0, (size_t)N * c->m_pad * 2, c->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(c->scratch, 0, c->scratch_bytes, c->stream);
+  if (e != cudaSuccess) return bail(fail(nullptr, PRSGD_ERR_CUDA, std::string("create: ") + cudaGetErrorString(e)));
+  if (c->precision == PRSGD_PRECISION_BF16) {
+    std::string terr;
+    int trc = tc_create(c, &terr);
+    if (trc != PRSGD_OK) return bail(fail(nullptr, trc, terr));
+  }
+  *out = c;
+  return PRSGD_OK;
+}
+
+int prsgd_destroy(prsgd_ctx* ctx) {
+  if (!ctx) return PRSGD_OK;
+  tc_destroy(ctx);
+  delete ctx;
+  return PRSGD_OK;
+}
+
+int prsgd_bind_data(prsgd_ctx* c, const void* d_X, int32_t x_dtype, const int32_t* d_Y) {
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
+  if (!d_X || !d_Y) return fail(c, PRSGD_ERR_ARG, "d_X / d_Y is NULL");
+  const int want = c->precision == PRSGD_PRECISION_BF16 ? PRSGD_X_BF16 : PRSGD_X_FP32;
+  if (x_dtype != want) return fail(c, PRSGD_ERR_ARG, "x_dtype does not match the context's precision");
+  if (!aligned(d_X, 256) || !aligned(d_Y, 256)) return fail(c, PRSGD_ERR_ALIGN, "pools must be 256-byte aligned");
+  c->X = d_X; c->x_dtype = x_dtype; c->Y = d_Y;
+  if (c->precision == PRSGD_PRECISION_BF16) {
+    std::string terr;
+    int trc = tc_bind_data(c, &terr);
+    if (trc != PRSGD_OK) return fail(c, trc, terr);
+  }
+  return PRSGD_OK;
+}
+
+int prsgd_upload_data(prsgd_ctx* c, const void* h_X, const int32_t* h_Y) {
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
+  if (!c->X) return fail(c, PRSGD_ERR_STATE, "bind_data must come first");
+  if (!h_X || !h_Y) return fail(c, PRSGD_ERR_ARG, "h_X / h_Y is NULL");
+  const size_t esz = c->x_dtype == PRSGD_X_BF16 ? 2 : 4;
+  CUDA_TRY(c, cudaMemcpyAsync(const_cast<void*>(c->X), h_X, (size_t)c->N * c->P * c->dims[0] * esz,
+                              cudaMemcpyHostToDevice, c->stream));
+  CUDA_TRY(c, cudaMemcpyAsync(const_cast<int32_t*>(c->Y), h_Y, (size_t)c->N * c->P * 4, cudaMemcpyHostToDevice,
+                              c->stream));
+  return PRSGD_OK;
+}
+
+int prsgd_set_params(prsgd_ctx* c, const float* src, int32_t worker, int src_on_device) {
+  (void)src_on_device;
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
+  if (!src) return fail(c, PRSGD_ERR_ARG, "src is NULL");
+  if (worker < -1 || worker >= c->N) return fail(c, PRSGD_ERR_ARG, "worker out of range");
+  int rc = copy_canonical(c, const_cast<float*>(src), worker < 0 ? 0 : worker, 1, true);
+  if (rc != PRSGD_OK) return rc;
+  if (worker < 0 && c->N > 1) {
+    broadcast_row0_kernel<<<grid1d(c->m_pad / 4, 256), 256, 0, c->stream>>>(c->params, c->N, c->m_pad / 4, c->m_pad / 4);
+    LAUNCH_CHECK(c);
+  }
+  if (!src_on_device) CUDA_TRY(c, cudaStreamSynchronize(c->stream));   // src may be reused by the caller
+  return refresh_shadow(c);
+}
+
+int prsgd_set_params_stacked(prsgd_ctx* c, const float* src, int src_on_device) {
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
+  if (!src) return fail(c, PRSGD_ERR_ARG, "src is NULL");
+  int rc = copy_canonical(c, const_cast<float*>(src), 0, c->N, true);
+  if (rc != PRSGD_OK) return rc;
+  if (!src_on_device) CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  return refresh_shadow(c);
+}
+
+int prsgd_get_params_stacked(prsgd_ctx* c, float* dst, int dst_on_device) {
+  (void)dst_on_device;
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
+  if (!dst) return fail(c, PRSGD_ERR_ARG, "dst is NULL");
+  int rc = copy_canonical(c, dst, 0, c->N, false);
+  if (rc != PRSGD_OK) return rc;
+  return check_device_status(c);
+}
+
+int prsgd_get_params(prsgd_ctx* c, float* dst, int32_t worker, int dst_on_device) {
+  (void)dst_on_device;
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
+  if (!dst) return fail(c, PRSGD_ERR_ARG, "dst is NULL");
+  if (worker < 0 || worker >= c->N) return fail(c, PRSGD_ERR_ARG, "worker out of range");
+  int rc = copy_canonical(c, dst, worker, 1, false);
+  if (rc != PRSGD_OK) return rc;
+  return check_device_status(c);
+}
+
+int prsgd_local_steps(prsgd_ctx* c, int64_t k) {
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
+  if (k < 0) return fail(c, PRSGD_ERR_ARG, "k must be >= 0");
+  if (!c->X || !c->Y) return fail(c, PRSGD_ERR_STATE, "bind_data must come before local_steps");
+  for (int64_t s = 0; s < k; ++s) {
+    const int64_t t = c->t + 1;
+    const bool averaging = c->I > 0 && (t % c->I) == 0;
+    int rc = c->precision == PRSGD_PRECISION_BF16 ? tc_step(c, t, averaging) : step_f32(c, t, averaging);
+    if (rc != PRSGD_OK) return rc;
+    if (averaging && !c->fused_average) {
+      rc = launch_average(c);
+      if (rc != PRSGD_OK) return rc;
+    }
+    c->t = t;
+  }
+  return PRSGD_OK;
+}
+
+int prsgd_average(prsgd_ctx* c) {
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
+  return launch_average(c);
+}
+
+int prsgd_get_average(prsgd_ctx* c, float* dst, int dst_on_device) {
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
+  if (!dst) return fail(c, PRSGD_ERR_ARG, "dst is NULL");
+  average_rows_kernel<1, false><<<grid1d(c->m_pad / 4, 256), 256, 0, c->stream>>>(c->params, c->N, c->m_pad, c->m_pad,
+                                                                              c->stage_row, nullptr);
+  LAUNCH_CHECK(c);
+  int64_t pos = 0;
+  for (int l = 0; l < c->L; ++l) {
+    const Layer& ly = c->layer[l];
+    const int64_t seg[2] = {(int64_t)ly.d_in * ly.d_out, (int64_t)ly.d_out};
+    const int64_t offs[2] = {ly.w_off, ly.b_off};
+    for (int q = 0; q < 2; ++q) {
+      CUDA_TRY(c, cudaMemcpyAsync(dst + pos, c->stage_row + offs[q], seg[q] * 4, cudaMemcpyDefault, c->stream));
+      pos += seg[q];
+    }
+  }
+  if (!dst_on_device) return check_device_status(c);
+  return PRSGD_OK;
+}
+
+int prsgd_get_losses(prsgd_ctx* c, float* h_dst) {
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
+  if (!h_dst) return fail(c, PRSGD_ERR_ARG, "h_dst is NULL");
+  CUDA_TRY(c, cudaMemcpyAsync(h_dst, c->losses, sizeof(float) * c->N, cudaMemcpyDeviceToHost, c->stream));
+  return check_device_status(c);
+}
+
+int prsgd_get_draws(prsgd_ctx* c, int32_t* h_dst) {
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
+  if (!h_dst) return fail(c, PRSGD_ERR_ARG, "h_dst is NULL");
+  CUDA_TRY(c, cudaMemcpyAsync(h_dst, c->draws, sizeof(int32_t) * c->N, cudaMemcpyDeviceToHost, c->stream));
+  return check_device_status(c);
+}
+
+int prsgd_set_lr(prsgd_ctx* c, float gamma) {
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
+  if (!(gamma > 0.f)) return fail(c, PRSGD_ERR_ARG, "gamma must be > 0");
+  c->gamma = gamma;
+  return PRSGD_OK;
+}
+
+int prsgd_set_interval(prsgd_ctx* c, int32_t I) {
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
+  if (I < 0) return fail(c, PRSGD_ERR_ARG, "I must be >= 0");
+  c->I = I;
+  return PRSGD_OK;
+}
+
+int prsgd_set_active(prsgd_ctx* c, const uint8_t* h_mask) {
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
+  if (!h_mask) { c->has_mask = false; return PRSGD_OK; }
+  CUDA_TRY(c, cudaMemcpyAsync(c->active, h_mask, (size_t)c->N, cudaMemcpyHostToDevice, c->stream));
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  c->has_mask = true;
+  return PRSGD_OK;
+}
+
+int prsgd_get_step(prsgd_ctx* c, int64_t* t) {
+  if (!c || !t) return fail(c, PRSGD_ERR_ARG, "NULL argument");
+  *t = c->t;
+  return PRSGD_OK;
+}
+
+int prsgd_set_step(prsgd_ctx* c, int64_t t) {
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
+  if (t < 0) return fail(c, PRSGD_ERR_ARG, "t must be >= 0");
+  c->t = t;
+  return PRSGD_OK;
+}
+
+int prsgd_set_option(prsgd_ctx* c, int32_t option, int64_t value) {
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
+  if (option == PRSGD_OPT_FUSED_AVERAGE) { c->fused_average = value != 0; return PRSGD_OK; }
+  return fail(c, PRSGD_ERR_ARG, "unknown option");
+}
+
+int prsgd_get_launch_count(prsgd_ctx* c, int64_t* count) {
+  if (!c || !count) return fail(c, PRSGD_ERR_ARG, "NULL argument");
+  *count = c->launches;
+  return PRSGD_OK;
+}
+
+int prsgd_sync(prsgd_ctx* c) {
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
+  return check_device_status(c);
+}
+
+int prsgd_average_rows(float* d_P, int64_t N, int64_t m, int64_t row_stride, void* cuda_stream) {
+  if (!d_P) return fail(nullptr, PRSGD_ERR_ARG, "d_P is NULL");
+  if (N < 1 || m < 0 || row_stride < m) return fail(nullptr, PRSGD_ERR_ARG, "need N >= 1, m >= 0, row_stride >= m");
+  if (!aligned(d_P, 16) || (row_stride % 4) != 0)
+    return fail(nullptr, PRSGD_ERR_ALIGN, "d_P must be 16-byte aligned and row_stride a multiple of 4");
+  if (m == 0) return PRSGD_OK;
+  const int64_t threads = m / 4 + (m & 3);
+  if ((threads + 255) / 256 > 0x7fffffffll) return fail(nullptr, PRSGD_ERR_SIZE, "m too large");
+  average_rows_kernel<0, false><<<grid1d(threads, 256), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+      d_P, N, m, row_stride, nullptr, nullptr);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(nullptr, PRSGD_ERR_CUDA, std::string("average_rows: ") + cudaGetErrorString(e));
+  return PRSGD_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,102 @@
+// Shared declarations of the PR-SGD library: the host context, the row layout
+// and the minibatch draw.  Internal; the public boundary is include/prsgd.h.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda.h>
+#include <stdint.h>
+#include <stddef.h>
+#include <string>
+#include <vector>
+
+#include "prsgd.h"
+
+namespace prsgd {
+
+// ---------------------------------------------------------------------------
+// Minibatch draw zeta_i^t (integer only).  SplitMix64 output function applied
+// twice: first to the t-th state of the stream seeded with `seed`, then to that
+// word advanced by (i + 1) increments.
+// ---------------------------------------------------------------------------
+__host__ __device__ inline uint64_t mix64(uint64_t z) {
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+
+__host__ __device__ inline uint32_t draw_block(uint64_t seed, int worker, int64_t t, uint32_t n_blocks) {
+  const uint64_t inc = 0x9E3779B97F4A7C15ull;
+  uint64_t u = mix64(seed + inc * (uint64_t)t);
+  uint64_t v = mix64(u + inc * (uint64_t)(worker + 1));
+  return (uint32_t)(v % (uint64_t)n_blocks);
+}
+
+// ---------------------------------------------------------------------------
+// Device status words (first 256 bytes of the scratch area)
+// ---------------------------------------------------------------------------
+struct DeviceStatus {
+  unsigned int error;      // 0 = fine; otherwise a code naming the wait that gave up
+  unsigned int where;      // block index that recorded it
+  unsigned int pad[62];
+};
+
+constexpr int64_t kSegAlign = 32;  // every segment of a row starts at a multiple of 32 elements
+
+inline int64_t round_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
+
+struct Layer {
+  int d_in, d_out;
+  int64_t w_off, b_off;    // element offsets inside a row
+};
+
+// Scratch buffers of one precision path.  Index l = 1..L (index 0 unused);
+// act[L] holds the logits on the fp32 path.
+struct Buffers {
+  float* act_f32[PRSGD_MAX_LAYERS + 1];
+  float* delta_f32[PRSGD_MAX_LAYERS + 1];
+  // bf16 path: activations and deltas in both orientations, leading dimension padded
+  uint16_t* act_bk[PRSGD_MAX_LAYERS + 1];   // [N][B][ld]   (batch-major rows, features contiguous)
+  uint16_t* act_kb[PRSGD_MAX_LAYERS + 1];   // [N][ld][B]   (feature-major rows, batch contiguous)
+  uint16_t* delta_bk[PRSGD_MAX_LAYERS + 1];
+  uint16_t* delta_kb[PRSGD_MAX_LAYERS + 1];
+  int ld[PRSGD_MAX_LAYERS + 1];             // padded feature count of layer l's output
+};
+
+}  // namespace prsgd
+
+struct prsgd_ctx {
+  int N = 0, L = 0, B = 0, precision = 0;
+  int dims[PRSGD_MAX_LAYERS + 1] = {0};
+  int64_t P = 0;             // pool samples per worker
+  uint32_t n_blocks = 0;
+  uint64_t seed = 0;
+  float gamma = 0.f;
+  int I = 0;
+  int64_t t = 0;
+  int fused_average = 1;
+  int64_t launches = 0;
+  int64_t m = 0, m_pad = 0;
+  prsgd::Layer layer[PRSGD_MAX_LAYERS];
+  cudaStream_t stream = nullptr;
+  int device = 0;
+
+  float* params = nullptr;       // [N][m_pad] fp32
+  uint16_t* shadow = nullptr;    // [N][m_pad] bf16 bits (BF16 precision only)
+  unsigned char* scratch = nullptr;
+  size_t scratch_bytes = 0;
+
+  prsgd::DeviceStatus* status = nullptr;
+  int32_t* draws = nullptr;      // [N]
+  float* losses = nullptr;       // [N]
+  uint8_t* active = nullptr;     // [N] device copy of the Algorithm-3 mask
+  bool has_mask = false;
+  float* stage_row = nullptr;    // [m_pad] fp32
+  prsgd::Buffers buf;
+
+  const void* X = nullptr;       // [N][P][d0] fp32 or bf16
+  int x_dtype = -1;
+  const int32_t* Y = nullptr;    // [N][P]
+
+  void* tc = nullptr;            // tensor-core path state (tensor maps), owned
+  std::string err;
+};

@@ -1,0 +1,233 @@
+"""GPU parity, fp32-operand path and the averaging kernel, through the C ABI.
+
+Tolerances (relative L2 over the stacked N*m parameter vector, from a state
+synchronised with the oracle): <= 1e-5 after one iteration, <= 1e-4 after one
+full averaging period.  Integer facts (draws, schedule, slot mapping) are exact.
+"""
+import numpy as np
+import pytest
+
+from oracle import prsgd_oracle as orc
+from paper_1807_06629_b200 import synth
+from helpers import make_ctx, make_inputs, oracle_run, rel_l2
+
+pytestmark = pytest.mark.gpu
+
+TOL_STEP, TOL_PERIOD = 1e-5, 1e-4
+TOL_UPDATE = 1e-4          # relative L2 of the *change* x^t - x^{t-1} (a zero update cannot pass)
+
+
+@pytest.fixture(scope="module")
+def torch_cuda():
+    import torch
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    return torch
+
+
+def test_average_rows_matches_fp64_mean(torch_cuda):
+    torch = torch_cuda
+    from paper_1807_06629_b200 import binding
+    for (N, m, stride) in [(8, 1_000_000, 1_000_000), (3, 1027, 1028), (1, 5, 8), (64, 40_003, 40_004), (7, 4, 4),
+                           (256, 5000, 5000)]:
+        V = synth.stacked_vectors(N, stride, seed=N * 7919 + m)
+        P = torch.from_numpy(V).to("cuda:0")
+        binding.prsgd_average_rows(P, N, m, stride)
+        out = P.cpu().numpy()
+        want = orc.node_average(V[:, :m].astype(np.float64))
+        for i in range(1, N):
+            assert np.array_equal(out[i, :m], out[0, :m])          # every slot holds the same bits
+        assert np.array_equal(out[:, m:], V[:, m:])                # columns past m untouched
+        assert np.abs(out[0, :m] - want).max() <= 2.0 ** -22 * np.abs(V[:, :m]).sum(0).max() / N + 1e-12
+        assert rel_l2(out[0, :m], want) < 1e-6
+
+
+def test_average_rows_empty_and_errors(torch_cuda):
+    torch = torch_cuda
+    from paper_1807_06629_b200 import binding
+    P = torch.ones(4, 8, device="cuda:0")
+    binding.prsgd_average_rows(P, 4, 0, 8)                         # m = 0: nothing to do
+    assert torch.equal(P, torch.ones(4, 8, device="cuda:0"))
+    with pytest.raises(binding.PRSGDError):
+        binding.prsgd_average_rows(P, 4, 9, 8)
+
+
+def test_set_get_roundtrip_and_padding_stays_zero(torch_cuda):
+    w = synth.WORKLOADS["cfg1"]
+    X, Y, x0 = make_inputs(w)
+    p = make_ctx(w, X, Y, x0)
+    got = p.get_params_stacked()
+    assert np.array_equal(got, np.tile(x0, (w.N, 1)))
+    x1 = x0 + 1.0
+    p.set_params(x1, worker=2)
+    assert np.array_equal(p.get_params(2), x1) and np.array_equal(p.get_params(1), x0)
+    p.set_params(x0)
+    p.local_steps(9)                                               # includes two averages
+    store = p.params.cpu().numpy().reshape(w.N, p.m_pad)
+    keep = np.zeros(p.m_pad, dtype=bool)
+    for l in range(len(w.dims) - 1):
+        keep[p.layout.w_off[l]:p.layout.w_off[l] + w.dims[l] * w.dims[l + 1]] = True
+        keep[p.layout.b_off[l]:p.layout.b_off[l] + w.dims[l + 1]] = True
+    assert keep.sum() == w.m
+    assert np.all(store[:, ~keep] == 0.0)
+    assert np.array_equal(store[:, keep], p.get_params_stacked())
+
+
+def test_draws_and_schedule_are_bit_exact(torch_cuda):
+    w = synth.WORKLOADS["cfg1"]
+    X, Y, x0 = make_inputs(w)
+    p = make_ctx(w, X, Y, x0)
+    for t in range(1, 13):
+        p.local_steps(1)
+        assert p.get_step() == t
+        want = [orc.draw_block(w.seed, i, t, w.n_blocks) for i in range(w.N)]
+        assert p.get_draws().tolist() == want
+        rows = p.get_params_stacked()
+        identical = all(np.array_equal(rows[i], rows[0]) for i in range(1, w.N))
+        assert identical == (t % w.I == 0)                          # averaged exactly at t = I, 2I, ...
+
+
+@pytest.mark.parametrize("name", ["cfg1", "cfg2"])
+def test_per_step_parity(torch_cuda, name):
+    w = synth.WORKLOADS[name]
+    if name == "cfg2":
+        w = w.with_(pool_samples=32 * 16)
+    X, Y, x0 = make_inputs(w)
+    p = make_ctx(w, X, Y, x0)
+    state = np.tile(x0, (w.N, 1)).astype(np.float64)
+    for t in range(1, w.I + 2):                                     # a whole period and one step beyond
+        losses = {}
+        want = oracle_run(w, X, Y, state, t - 1, 1, losses=losses)
+        p.set_params_stacked(state.astype(np.float32))              # synchronise with the oracle
+        p.set_step(t - 1)
+        p.local_steps(1)
+        got = p.get_params_stacked()
+        s32 = state.astype(np.float32).astype(np.float64)
+        assert rel_l2(got, want) <= TOL_STEP, (t, rel_l2(got, want))
+        assert rel_l2(got - s32, want - s32) <= TOL_UPDATE, (t, rel_l2(got - s32, want - s32))
+        gl = p.get_losses()
+        wl = np.array([losses[(i, t)] for i in range(w.N)])
+        assert np.allclose(gl, wl, rtol=2e-5, atol=1e-6)
+        state = want
+
+
+@pytest.mark.parametrize("name", ["cfg1", "cfg2"])
+def test_full_period_parity(torch_cuda, name):
+    w = synth.WORKLOADS[name]
+    if name == "cfg2":
+        w = w.with_(pool_samples=32 * 16)
+    X, Y, x0 = make_inputs(w)
+    p = make_ctx(w, X, Y, x0)
+    p.local_steps(w.I)
+    got = p.get_params_stacked()
+    want = oracle_run(w, X, Y, np.tile(x0, (w.N, 1)), 0, w.I)
+    assert rel_l2(got, want) <= TOL_PERIOD
+    assert rel_l2(got - x0[None, :], want - x0[None, :]) <= 10 * TOL_UPDATE
+    for i in range(1, w.N):
+        assert np.array_equal(got[i], got[0])
+    # a second period, from the GPU's own state
+    p.local_steps(w.I)
+    want2 = oracle_run(w, X, Y, got, w.I, w.I)
+    assert rel_l2(p.get_params_stacked(), want2) <= TOL_PERIOD
+
+
+def test_fused_average_equals_update_then_average_bit_for_bit(torch_cuda):
+    for name in ("cfg1", "cfg2"):
+        w = synth.WORKLOADS[name]
+        if name == "cfg2":
+            w = w.with_(pool_samples=32 * 16)
+        X, Y, x0 = make_inputs(w)
+        from paper_1807_06629_b200 import binding
+        outs = []
+        for fused in (1, 0):
+            p = make_ctx(w, X, Y, x0)
+            p.set_option(binding.OPT_FUSED_AVERAGE, fused)
+            p.local_steps(2 * w.I)
+            outs.append(p.get_params_stacked())
+        assert np.array_equal(outs[0], outs[1])
+        # and a manual schedule (I = 0 plus explicit average) gives the same bits again
+        p = make_ctx(w, X, Y, x0, I=0)
+        for _ in range(2):
+            p.local_steps(w.I)
+            p.average()
+        assert np.array_equal(p.get_params_stacked(), outs[0])
+
+
+def test_local_steps_compose_and_resume(torch_cuda):
+    w = synth.WORKLOADS["cfg1"]
+    X, Y, x0 = make_inputs(w)
+    a = make_ctx(w, X, Y, x0)
+    a.local_steps(11)
+    b = make_ctx(w, X, Y, x0)
+    b.local_steps(3)
+    b.local_steps(0)
+    b.local_steps(8)
+    assert np.array_equal(a.get_params_stacked(), b.get_params_stacked())
+    # checkpoint / resume: state + step counter reproduce the trajectory bit for bit
+    c = make_ctx(w, X, Y, x0)
+    c.local_steps(5)
+    snap, t = c.get_params_stacked(), c.get_step()
+    d = make_ctx(w, X, Y)
+    d.set_params_stacked(snap)
+    d.set_step(t)
+    d.local_steps(6)
+    assert np.array_equal(d.get_params_stacked(), a.get_params_stacked())
+
+
+def test_get_average_is_the_mean_and_leaves_the_store_alone(torch_cuda):
+    w = synth.WORKLOADS["cfg1"]
+    X, Y, x0 = make_inputs(w)
+    p = make_ctx(w, X, Y, x0)
+    p.local_steps(3)                                                # not an averaging iteration
+    before = p.get_params_stacked()
+    ybar = p.get_average()
+    assert np.array_equal(p.get_params_stacked(), before)
+    assert rel_l2(ybar, orc.node_average(before.astype(np.float64))) < 1e-6
+    # mean dynamics (Eq. overline-x-update): xbar^t = xbar^{t-1} - gamma * mean_i G_i^t, also across an average
+    fn = orc.mlp_grad_fn(w.dims, X.astype(np.float64), Y, w.B, w.seed)
+    G = np.stack([fn(i, 4, before[i].astype(np.float64)) for i in range(w.N)])
+    p.local_steps(1)                                                # t = 4 averages
+    assert np.allclose(p.get_average(), ybar - w.gamma * G.mean(0), rtol=0, atol=2e-6)
+    p.average()
+    rows = p.get_params_stacked()
+    assert all(np.array_equal(rows[i], rows[0]) for i in range(w.N))
+
+
+def test_time_varying_rates_and_heterogeneous_epochs(torch_cuda):
+    w = synth.WORKLOADS["cfg1"]
+    X, Y, x0 = make_inputs(w)
+    fn = orc.mlp_grad_fn(w.dims, X.astype(np.float64), Y, w.B, w.seed)
+    # Algorithm 2 with a short schedule driven through set_lr + explicit averages
+    sched = [(2, 0.08), (1, 0.05), (3, 0.03)]
+    p = make_ctx(w, X, Y, x0, I=0)
+    for (K, g) in sched:
+        p.average()
+        p.set_lr(g)
+        p.local_steps(K)
+    want = orc.pr_sgd_time_varying(np.tile(x0, (w.N, 1)), sched, fn)
+    assert rel_l2(p.get_params_stacked(), want) <= TOL_PERIOD
+    # Algorithm 3: per-worker epoch lengths through the active mask
+    I_i, S = [3, 1, 2, 3], 2
+    q = make_ctx(w, X, Y, x0, I=0)
+    for s in range(S):
+        q.average()
+        for k in range(1, max(I_i) + 1):
+            q.set_active([1 if k <= I_i[i] else 0 for i in range(w.N)])
+            q.local_steps(1)
+    want = orc.pr_sgd_heterogeneous(np.tile(x0, (w.N, 1)), w.gamma, I_i, S, fn)
+    assert rel_l2(q.get_params_stacked(), want) <= TOL_PERIOD
+    q.set_active(None)
+
+
+@pytest.mark.parametrize("N,dims,B", [(1, (5, 3), 1), (3, (7, 5, 3, 2), 5), (2, (130, 70, 33), 48), (5, (16, 300, 11), 100)])
+def test_ragged_shapes(torch_cuda, N, dims, B):
+    w = synth.Workload("ragged", N, dims, B, 0.1, 3, 6, 0, 4 * B, mean_shift=0.3, seed=77)
+    X, Y, x0 = make_inputs(w)
+    p = make_ctx(w, X, Y, x0)
+    p.local_steps(1)
+    want1 = oracle_run(w, X, Y, np.tile(x0, (N, 1)), 0, 1)
+    assert rel_l2(p.get_params_stacked(), want1) <= TOL_STEP
+    p.set_params(x0)
+    p.set_step(0)
+    p.local_steps(w.I)
+    want = oracle_run(w, X, Y, np.tile(x0, (N, 1)), 0, w.I)
+    assert rel_l2(p.get_params_stacked(), want) <= TOL_PERIOD
