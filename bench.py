@@ -1,0 +1,374 @@
+#!/usr/bin/env python
+"""Benchmark of the PR-SGD hot path (Algorithm 1: local SGD steps + periodic node average).
+
+One "step" of this benchmark is one full averaging period of the workload:
+I local iterations of all N workers followed by the node average, i.e.
+prsgd_local_steps(I).  The metric is worker-steps/s = N * I * steps / time.
+
+Prints ONE JSON line.  `value` is timed on the device with inputs resident in
+HBM; `e2e` is the same period driven through the C ABI from pinned HOST
+buffers (pool upload, local steps, read-back of the node average).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config cfg4] [--impl reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+from paper_1807_06629_b200 import synth
+
+DEFAULT_WORKLOAD = "cfg4"
+L2_BYTES = 126 * 1024 * 1024
+METRIC = "worker-steps/s"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1])); power.append(float(f[2]))
+            except ValueError:
+                continue
+            for k, nm in enumerate(names):
+                if f[3 + k].lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------- byte model
+def algorithmic_bytes(w: synth.Workload, m_pad: int) -> dict:
+    """Algorithmic HBM bytes of one local iteration of all N workers, per kernel family.
+
+    bf16 path: forward reads the bf16 shadow (2 B/param); dX reads it again for every layer but
+    the first; the update reads and writes the fp32 master (4 + 4) and writes the shadow (2);
+    activations / deltas are read and written once per use.  fp32 path: 4 B where bf16 has 2, no shadow.
+    The stand-alone average reads and writes the store once (8 B/word, +2 for the shadow).
+    """
+    e = 2 if w.precision == 1 else 4
+    N, B, d = w.N, w.B, w.dims
+    L = len(d) - 1
+    fwd = dx = upd = 0
+    for l in range(1, L + 1):
+        wl = d[l] * d[l - 1]
+        fwd += N * (wl * e + d[l] * 4 + B * d[l - 1] * e + B * d[l] * (e if l < L else 4))
+        if l > 1:
+            dx += N * (wl * e + B * d[l] * e + B * d[l - 1] * 2 * e)
+        upd += N * ((wl + d[l]) * (8 + (2 if w.precision == 1 else 0)) + B * (d[l] + d[l - 1]) * e)
+    avg = N * m_pad * (8 + (2 if w.precision == 1 else 0))
+    return {"forward": fwd, "dx": dx, "update": upd, "update_average": upd, "average": avg,
+            "softmax": N * B * d[L] * (4 + 4 + e)}
+
+
+def flops_per_worker_step(w: synth.Workload) -> int:
+    d, B = w.dims, w.B
+    tot = sum(6 * B * d[l] * d[l - 1] for l in range(1, len(d)))
+    return tot - 2 * B * d[1] * d[0]
+
+
+# ----------------------------------------------------------------------------- oracle (CPU baseline)
+def time_oracle(w: synth.Workload, X, Y, x0, budget_s: float = 15.0):
+    """Times the fp64 oracle, as it stands, on a bounded sample: all N workers for s iterations."""
+    from oracle import prsgd_oracle as orc
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        cores = 1
+    fn = orc.mlp_grad_fn(w.dims, X, Y, w.B, w.seed)
+    state = np.tile(x0.astype(np.float64), (w.N, 1))
+    t0 = time.perf_counter()
+    state = orc.pr_sgd(state, w.gamma, w.I, 1, fn, t0=0)
+    t1 = time.perf_counter() - t0
+    s = int(max(1, min(w.I, budget_s / max(t1, 1e-6))))
+    t0 = time.perf_counter()
+    orc.pr_sgd(state, w.gamma, w.I, s, fn, t0=1)
+    dt = time.perf_counter() - t0
+    return {"value": w.N * s / dt, "unit": METRIC, "cores": cores, "kind": "oracle",
+            "sample": f"all {w.N} workers x {s} consecutive iterations of {w.name} (fp64 numpy), {dt:.1f} s"}
+
+
+def run_reference(args, w):
+    """--impl reference: the oracle on the host cores; each step is one iteration of all N workers."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import prsgd_oracle as orc
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        cores = 1
+    X, Y = synth.make_pools(w)
+    if w.precision == 1:
+        X = synth.bf16_round(X)
+    x0 = synth.init_params(w.dims, w.seed)
+    fn = orc.mlp_grad_fn(w.dims, X, Y, w.B, w.seed)
+    state = np.tile(x0.astype(np.float64), (w.N, 1))
+    t = 0
+    for _ in range(args.warmup):
+        state = orc.pr_sgd(state, w.gamma, w.I, 1, fn, t0=t); t += 1
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        state = orc.pr_sgd(state, w.gamma, w.I, 1, fn, t0=t); t += 1
+    dt = time.perf_counter() - t0
+    val = w.N * args.steps / dt
+    sample = f"each step = 1 iteration of all {w.N} workers of {w.name} (fp64 numpy oracle)"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": METRIC, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(w),
+        "cpu_baseline": {"value": val, "unit": METRIC, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": METRIC, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def workload_config(w, extra=None):
+    c = {"workload": w.name, "N": w.N, "dims": list(w.dims), "B": w.B, "gamma": w.gamma, "I": w.I,
+         "pool_samples": w.pool_samples, "precision": "bf16 operands / fp32 master" if w.precision else "fp32",
+         "step": "one averaging period = prsgd_local_steps(I)"}
+    if extra:
+        c.update(extra)
+    return c
+
+
+# ----------------------------------------------------------------------------- averaging sweep
+def averaging_sweep(torch, binding, peaks, quick=False):
+    """Node-average kernel in isolation on [N, m] fp32: GB/s counting N*m*4 read + N*m*4 written."""
+    out = []
+    for N in synth.SWEEP_N:
+        for m in synth.SWEEP_M:
+            if quick and N * m > 64 * 11_000_000:
+                continue
+            nbytes = N * m * 4
+            copies = max(1, int(np.ceil(2 * L2_BYTES / nbytes))) if nbytes <= 2 * L2_BYTES else 1
+            bufs = [torch.randn(N, m, device="cuda:0", dtype=torch.float32) for _ in range(copies)]
+            reps = 20
+            binding.prsgd_average_rows(bufs[0], N, m)
+            torch.cuda.synchronize()
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+            ev[0].record()
+            for r in range(reps):
+                binding.prsgd_average_rows(bufs[r % copies], N, m)
+            ev[1].record()
+            torch.cuda.synchronize()
+            ms = ev[0].elapsed_time(ev[1]) / reps
+            gbs = 2 * nbytes / ms / 1e6
+            out.append({"N": N, "m": m, "us": round(ms * 1e3, 2), "GBps": round(gbs, 1),
+                        "frac_of_measured_copy": round(gbs / peaks["hbm_gbs"], 4),
+                        "frac_of_8TBps": round(gbs / 8000.0, 4), "rotating_buffers": copies})
+            del bufs
+            torch.cuda.empty_cache()
+    return out
+
+
+# ----------------------------------------------------------------------------- main arm
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=8)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", default=DEFAULT_WORKLOAD, choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--interval", type=int, default=None, help="override the averaging interval I")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the averaging-kernel sweep")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle timing")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    w = synth.WORKLOADS[args.config]
+    if args.interval is not None:
+        w = w.with_(I=args.interval)
+    if args.impl == "reference":
+        return run_reference(args, w)
+
+    import torch
+    import torch.distributed as dist
+    from paper_1807_06629_b200 import _build
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    if rank == 0 or world == 1:
+        _build.build_library()
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+        dist.barrier()
+    from paper_1807_06629_b200 import binding
+    peaks = load_peaks()
+
+    # every rank runs an independent replica of the whole workload on its own seed stream
+    w = w.with_(seed=w.seed + rank)
+    X, Y = synth.make_pools(w)
+    if w.precision == 1:
+        X = synth.bf16_round(X)
+    x0 = synth.init_params(w.dims, w.seed)
+    tdt = torch.bfloat16 if w.precision == 1 else torch.float32
+    hX = torch.from_numpy(X).to(tdt).contiguous().pin_memory()
+    hY = torch.from_numpy(Y).contiguous().pin_memory()
+    p = binding.PRSGD(w.N, w.dims, w.B, w.gamma, w.I, w.precision, w.pool_samples, w.seed, device=dev)
+    p.bind_data(hX.to(dev), hY.to(dev))
+    p.set_params(x0)
+    working_set = p.params.numel() * 4 + (p.shadow.numel() * 2 if p.shadow is not None else 0)
+    need_flush = working_set <= 2 * L2_BYTES
+    flush = torch.empty(3 * L2_BYTES // 4, dtype=torch.float32, device=dev) if need_flush else None
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-timed region: K periods, inputs resident in HBM -------------------------
+    for _ in range(args.warmup):
+        p.local_steps(w.I)
+    p.sync()
+    sampler = ClockSampler(local_rank)
+    barrier()
+    sampler.start()
+    launches0 = p.get_launch_count()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    for k in range(args.steps):
+        if flush is not None:
+            flush.fill_(float(k))
+        evs[k][0].record()
+        p.local_steps(w.I)
+        evs[k][1].record()
+    barrier()
+    clocks = sampler.stop()
+    launches = p.get_launch_count() - launches0
+    ms_total = sum(a.elapsed_time(b) for a, b in evs)
+    tt = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    ms_total = float(tt.item())
+    worker_steps = w.N * w.I * args.steps * world
+    value = worker_steps / (ms_total * 1e-3)
+
+    # ---- per-kernel pass (same region again with an event pair around every launch) ------
+    p.set_option(binding.OPT_PROFILE, 1)
+    p.get_profile()
+    for k in range(args.steps):
+        if flush is not None:
+            flush.fill_(float(k))
+        p.local_steps(w.I)
+    prof = p.get_profile()
+    p.set_option(binding.OPT_PROFILE, 0)
+    bytes_iter = algorithmic_bytes(w, p.m_pad)
+    fams = {k: v for k, v in prof.items() if v[1] > 0 and k in bytes_iter}
+    dom = max(fams, key=lambda k: fams[k][0])
+    L = len(w.dims) - 1
+    per_iter_launches = {"forward": L, "dx": L - 1, "update": L, "update_average": L, "average": 1, "softmax": 1}[dom]
+    dom_ms, dom_launches = fams[dom]
+    iters_seen = dom_launches / max(per_iter_launches, 1)
+    achieved = bytes_iter[dom] * iters_seen / (dom_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"] + " copy bandwidth",
+                "traffic": None,
+                "avg_launch_us": 1e3 * dom_ms / dom_launches,
+                "algorithmic_bytes_per_launch": bytes_iter[dom] / per_iter_launches,
+                "share_of_step_time": {k: round(v[0] / sum(x[0] for x in prof.values()), 4) for k, v in prof.items() if v[1]}}
+    tflops = flops_per_worker_step(w) * value / world / 1e12
+
+    # ---- end to end through the C ABI from pinned host buffers ---------------------------
+    avg_host = torch.empty(p.m, dtype=torch.float32).pin_memory()
+    for _ in range(2):
+        p.upload_data(hX, hY); p.local_steps(w.I); p.get_average(avg_host)
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        p.upload_data(hX, hY)
+        p.local_steps(w.I)
+        p.get_average(avg_host)
+    barrier()
+    e2e_s = time.perf_counter() - t0
+    te = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(te, op=dist.ReduceOp.MAX)
+    e2e = {"value": worker_steps / float(te.item()), "unit": METRIC,
+           "h2d_bytes_per_step": hX.numel() * hX.element_size() + hY.numel() * 4,
+           "d2h_bytes_per_step": p.m * 4}
+
+    out = {
+        "metric": METRIC, "value": value, "unit": METRIC, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.precision else "f32", "data": "synthetic",
+        "config": workload_config(w, {"l2": "L2 flushed between timed steps" if need_flush else
+                                      "parameter store + shadow larger than L2",
+                                      "multi_gpu": "independent replicas, one per rank" if world > 1 else "single GPU"}),
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline,
+        "gemm_tflops": tflops, "gemm_frac_of_bf16_peak": tflops / peaks["bf16_tflops_sustained"],
+    }
+    if rank == 0 and world == 1:
+        if not args.no_sweep:
+            out["averaging_sweep"] = averaging_sweep(torch, binding, peaks)
+        if not args.no_cpu:
+            out["cpu_baseline"] = time_oracle(w, X, Y, x0)
+    if rank == 0:
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -175,7 +175,26 @@ int prsgd_set_step(prsgd_ctx* ctx, int64_t t);
  * update and the average run as one pass over the store instead of an update
  * pass followed by prsgd_average's pass; both produce identical bits. */
 #define PRSGD_OPT_FUSED_AVERAGE 1
+/* PRSGD_OPT_PROFILE (default 0): when 1, every kernel launch is bracketed by a
+ * pair of CUDA events on the context's stream; read the sums with
+ * prsgd_get_profile.  Costs two event records per launch. */
+#define PRSGD_OPT_PROFILE 2
 int prsgd_set_option(prsgd_ctx* ctx, int32_t option, int64_t value);
+
+/* Kernel families of the hot path, for prsgd_get_profile. */
+#define PRSGD_KERNEL_FORWARD        0  /* grouped forward GEMM + bias + ReLU                        */
+#define PRSGD_KERNEL_SOFTMAX        1  /* softmax cross-entropy gradient                            */
+#define PRSGD_KERNEL_DX             2  /* grouped input-gradient GEMM + ReLU mask                   */
+#define PRSGD_KERNEL_UPDATE         3  /* grouped weight-gradient GEMM + in-place SGD update        */
+#define PRSGD_KERNEL_UPDATE_AVERAGE 4  /* the same with the node average fused in                   */
+#define PRSGD_KERNEL_AVERAGE        5  /* stand-alone node average (+ broadcast)                    */
+#define PRSGD_KERNEL_MISC           6  /* broadcast of x^0, shadow refresh                          */
+#define PRSGD_KERNEL_FAMILIES       7
+
+/* Device time (milliseconds, from the event pairs) and launch count of one
+ * kernel family since the previous call for that family; both counters are
+ * then reset.  Synchronises the stream.  Zero unless PRSGD_OPT_PROFILE is on. */
+int prsgd_get_profile(prsgd_ctx* ctx, int32_t family, double* ms_total, int64_t* launches);
 
 /* Number of kernels this context has launched so far. */
 int prsgd_get_launch_count(prsgd_ctx* ctx, int64_t* count);

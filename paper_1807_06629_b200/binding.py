@@ -21,6 +21,8 @@ PRSGD_OK = 0
 PRECISION_FP32, PRECISION_BF16 = 0, 1
 X_FP32, X_BF16 = 0, 1
 OPT_FUSED_AVERAGE = 1
+OPT_PROFILE = 2
+KERNEL_FAMILIES = ("forward", "softmax", "dx", "update", "update_average", "average", "misc")
 MAX_LAYERS = 16
 
 EXPORTS = [
@@ -28,7 +30,7 @@ EXPORTS = [
     "prsgd_upload_data", "prsgd_set_params", "prsgd_set_params_stacked", "prsgd_get_params_stacked",
     "prsgd_get_params", "prsgd_local_steps", "prsgd_average", "prsgd_get_average", "prsgd_get_losses",
     "prsgd_get_draws", "prsgd_set_lr", "prsgd_set_interval", "prsgd_set_active", "prsgd_get_step",
-    "prsgd_set_step", "prsgd_set_option", "prsgd_get_launch_count", "prsgd_sync", "prsgd_last_error",
+    "prsgd_set_step", "prsgd_set_option", "prsgd_get_launch_count", "prsgd_get_profile", "prsgd_sync", "prsgd_last_error",
     "prsgd_average_rows", "prsgd_draw_block",
 ]
 
@@ -74,6 +76,7 @@ def _load() -> C.CDLL:
         "prsgd_set_step": (C.c_int, [vp, i64]),
         "prsgd_set_option": (C.c_int, [vp, i32, i64]),
         "prsgd_get_launch_count": (C.c_int, [vp, C.POINTER(i64)]),
+        "prsgd_get_profile": (C.c_int, [vp, i32, C.POINTER(C.c_double), C.POINTER(i64)]),
         "prsgd_sync": (C.c_int, [vp]),
         "prsgd_last_error": (C.c_char_p, [vp]),
         "prsgd_average_rows": (C.c_int, [vp, i64, i64, i64, vp]),
@@ -271,6 +274,15 @@ class PRSGD:
         n = C.c_int64()
         self._call(lib.prsgd_get_launch_count, C.byref(n))
         return n.value
+
+    def get_profile(self) -> dict:
+        """{family: (ms_total, launches)} since the last call; needs OPT_PROFILE."""
+        out = {}
+        for k, name in enumerate(KERNEL_FAMILIES):
+            ms, n = C.c_double(), C.c_int64()
+            self._call(lib.prsgd_get_profile, k, C.byref(ms), C.byref(n))
+            out[name] = (ms.value, n.value)
+        return out
 
     def sync(self):
         self._call(lib.prsgd_sync)

@@ -34,7 +34,30 @@ int fail(prsgd_ctx* ctx, int code, const std::string& msg) {
     if (e__ != cudaSuccess)                                                                    \
       return fail((ctx), PRSGD_ERR_CUDA, std::string("kernel launch: ") + cudaGetErrorString(e__)); \
     (ctx)->launches++;                                                                         \
+    prof_end(ctx);                                                                             \
   } while (0)
+
+// Optional per-kernel timing: an event pair around every launch of a family.
+void prof_begin(prsgd_ctx* c, int kind) {
+  if (!c->profile) return;
+  cudaEvent_t a, b;
+  if (!c->event_pool.empty()) {
+    a = c->event_pool.back(); c->event_pool.pop_back();
+    b = c->event_pool.back(); c->event_pool.pop_back();
+  } else {
+    if (cudaEventCreate(&a) != cudaSuccess) return;
+    if (cudaEventCreate(&b) != cudaSuccess) { cudaEventDestroy(a); return; }
+  }
+  cudaEventRecord(a, c->stream);
+  c->open_kind = kind; c->open_a = a; c->open_b = b;
+}
+
+void prof_end(prsgd_ctx* c) {
+  if (!c->profile || c->open_kind < 0) return;
+  cudaEventRecord(c->open_b, c->stream);
+  c->pending.push_back({c->open_kind, c->open_a, c->open_b});
+  c->open_kind = -1;
+}
 
 int check_spec(const prsgd_model_spec* s, std::string* why) {
   if (!s || !s->dims) { *why = "spec or spec->dims is NULL"; return PRSGD_ERR_ARG; }
@@ -158,6 +181,7 @@ int copy_canonical(prsgd_ctx* c, float* lin, int64_t row0, int64_t nrows, bool t
 int refresh_shadow(prsgd_ctx* c) {
   if (c->precision != PRSGD_PRECISION_BF16) return PRSGD_OK;
   const int64_t total4 = (int64_t)c->N * c->m_pad / 4;
+  prof_begin(c, PRSGD_KERNEL_MISC);
   refresh_shadow_kernel<<<grid1d(total4, 256), 256, 0, c->stream>>>(c->params, c->shadow, total4);
   LAUNCH_CHECK(c);
   return PRSGD_OK;
@@ -205,6 +229,7 @@ int step_f32(prsgd_ctx* c, int64_t t, bool averaging) {
     g.out = c->buf.act_f32[l]; g.out_worker_stride = (int64_t)B * ly.d_out;
     g.params = c->params; g.params_worker_stride = c->m_pad; g.b_off = ly.b_off;
     g.active = act_mask;
+    prof_begin(c, PRSGD_KERNEL_FORWARD);
     if (l < L) {
       if (B <= 32) launch_gemm_f32<32, true, true, EPI_FWD_RELU, false>(c, g);
       else         launch_gemm_f32<64, true, true, EPI_FWD_RELU, false>(c, g);
@@ -219,6 +244,7 @@ int step_f32(prsgd_ctx* c, int64_t t, bool averaging) {
     a.logits = c->buf.act_f32[L]; a.delta = c->buf.delta_f32[L]; a.ldz = c->dims[L];
     a.Y = c->Y; a.P = c->P; a.B = B; a.C = c->dims[L]; a.draw = dr;
     a.losses = c->losses; a.draws = c->draws; a.active = act_mask;
+    prof_begin(c, PRSGD_KERNEL_SOFTMAX);
     softmax_ce_kernel<<<N, 256, 0, c->stream>>>(a);
     LAUNCH_CHECK(c);
   }
@@ -232,6 +258,7 @@ int step_f32(prsgd_ctx* c, int64_t t, bool averaging) {
       g.out = c->buf.delta_f32[l - 1]; g.out_worker_stride = (int64_t)B * ly.d_in;
       g.mask_src = c->buf.act_f32[l - 1];
       g.active = act_mask;
+      prof_begin(c, PRSGD_KERNEL_DX);
       if (B <= 32) launch_gemm_f32<32, true, false, EPI_DX, false>(c, g);
       else         launch_gemm_f32<64, true, false, EPI_DX, false>(c, g);
       LAUNCH_CHECK(c);
@@ -243,6 +270,7 @@ int step_f32(prsgd_ctx* c, int64_t t, bool averaging) {
     g.M = ly.d_out; g.Nn = ly.d_in; g.K = B; g.N = N; g.draw = dr;
     g.out = c->params; g.out_worker_stride = c->m_pad; g.w_off = ly.w_off; g.b_off = ly.b_off;
     g.gamma = c->gamma; g.active = act_mask;
+    prof_begin(c, fuse ? PRSGD_KERNEL_UPDATE_AVERAGE : PRSGD_KERNEL_UPDATE);
     if (fuse) launch_gemm_f32<64, false, false, EPI_DW, true>(c, g);
     else      launch_gemm_f32<64, false, false, EPI_DW, false>(c, g);
     LAUNCH_CHECK(c);
@@ -252,6 +280,7 @@ int step_f32(prsgd_ctx* c, int64_t t, bool averaging) {
 
 int launch_average(prsgd_ctx* c) {
   const int64_t threads = c->m_pad / 4;
+  prof_begin(c, PRSGD_KERNEL_AVERAGE);
   if (c->precision == PRSGD_PRECISION_BF16)
     average_rows_kernel<0, true><<<grid1d(threads, 256), 256, 0, c->stream>>>(c->params, c->N, c->m_pad, c->m_pad,
                                                                             nullptr, c->shadow);
@@ -348,6 +377,8 @@ int prsgd_create(int32_t N, const prsgd_model_spec* spec, float gamma, int32_t I
 int prsgd_destroy(prsgd_ctx* ctx) {
   if (!ctx) return PRSGD_OK;
   tc_destroy(ctx);
+  for (auto& p : ctx->pending) { cudaEventDestroy(p.a); cudaEventDestroy(p.b); }
+  for (auto e : ctx->event_pool) cudaEventDestroy(e);
   delete ctx;
   return PRSGD_OK;
 }
@@ -387,6 +418,7 @@ int prsgd_set_params(prsgd_ctx* c, const float* src, int32_t worker, int src_on_
   int rc = copy_canonical(c, const_cast<float*>(src), worker < 0 ? 0 : worker, 1, true);
   if (rc != PRSGD_OK) return rc;
   if (worker < 0 && c->N > 1) {
+    prof_begin(c, PRSGD_KERNEL_MISC);
     broadcast_row0_kernel<<<grid1d(c->m_pad / 4, 256), 256, 0, c->stream>>>(c->params, c->N, c->m_pad / 4, c->m_pad / 4);
     LAUNCH_CHECK(c);
   }
@@ -448,6 +480,7 @@ int prsgd_average(prsgd_ctx* c) {
 int prsgd_get_average(prsgd_ctx* c, float* dst, int dst_on_device) {
   if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
   if (!dst) return fail(c, PRSGD_ERR_ARG, "dst is NULL");
+  prof_begin(c, PRSGD_KERNEL_AVERAGE);
   average_rows_kernel<1, false><<<grid1d(c->m_pad / 4, 256), 256, 0, c->stream>>>(c->params, c->N, c->m_pad, c->m_pad,
                                                                               c->stage_row, nullptr);
   LAUNCH_CHECK(c);
@@ -518,12 +551,33 @@ int prsgd_set_step(prsgd_ctx* c, int64_t t) {
 int prsgd_set_option(prsgd_ctx* c, int32_t option, int64_t value) {
   if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
   if (option == PRSGD_OPT_FUSED_AVERAGE) { c->fused_average = value != 0; return PRSGD_OK; }
+  if (option == PRSGD_OPT_PROFILE) { c->profile = value != 0; return PRSGD_OK; }
   return fail(c, PRSGD_ERR_ARG, "unknown option");
 }
 
 int prsgd_get_launch_count(prsgd_ctx* c, int64_t* count) {
   if (!c || !count) return fail(c, PRSGD_ERR_ARG, "NULL argument");
   *count = c->launches;
+  return PRSGD_OK;
+}
+
+int prsgd_get_profile(prsgd_ctx* c, int32_t family, double* ms_total, int64_t* launches) {
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
+  if (family < 0 || family >= PRSGD_KERNEL_FAMILIES) return fail(c, PRSGD_ERR_ARG, "unknown kernel family");
+  if (!c->pending.empty()) {
+    CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+    for (auto& p : c->pending) {
+      float ms = 0.f;
+      if (cudaEventElapsedTime(&ms, p.a, p.b) == cudaSuccess) { c->prof_ms[p.kind] += ms; c->prof_count[p.kind]++; }
+      c->event_pool.push_back(p.a);
+      c->event_pool.push_back(p.b);
+    }
+    c->pending.clear();
+  }
+  if (ms_total) *ms_total = c->prof_ms[family];
+  if (launches) *launches = c->prof_count[family];
+  c->prof_ms[family] = 0.0;
+  c->prof_count[family] = 0;
   return PRSGD_OK;
 }
 

@@ -98,5 +98,15 @@ struct prsgd_ctx {
   const int32_t* Y = nullptr;    // [N][P]
 
   void* tc = nullptr;            // tensor-core path state (tensor maps), owned
+
+  // optional per-kernel timing (PRSGD_OPT_PROFILE)
+  struct Timed { int kind; cudaEvent_t a, b; };
+  bool profile = false;
+  int open_kind = -1;
+  cudaEvent_t open_a = nullptr, open_b = nullptr;
+  std::vector<Timed> pending;
+  std::vector<cudaEvent_t> event_pool;
+  double prof_ms[PRSGD_KERNEL_FAMILIES] = {0};
+  int64_t prof_count[PRSGD_KERNEL_FAMILIES] = {0};
   std::string err;
 };
