@@ -1,9 +1,623 @@
-// bf16-operand tensor-core path (placeholder until the tcgen05 kernels land).
+// bf16-operand tensor-core path (sm_100a): grouped GEMMs on tcgen05 with TMEM
+// accumulators, operands staged by TMA, one problem per worker.
+//
+//   stream kernel  : forward  Z^T[d_out, B]  = W[d_out, d_in] A^T[d_in, B]      (+bias, ReLU)
+//                    backward dA^T[d_in, B]  = W^T[d_in, d_out] dZ^T[d_out, B]  (ReLU mask)
+//                    The layer width sits on the MMA's M axis (128 rows per CTA) and the
+//                    minibatch on its N axis, because B = 16..64 is too small for M.
+//   update kernel  : dW[d_out, d_in] = dZ^T A over K = B, then x <- x - gamma dW in the
+//                    epilogue, in place, fp32 master and bf16 shadow written by TMA.
+//                    A bandwidth kernel: the MMA is tiny, the epilogue moves 10 B per parameter.
+//                    FUSE: the node average of the updated models is formed in registers over
+//                    all workers and written to every worker's rows (Algorithm 1, averaging step).
 #pragma once
+#include <new>
 #include "prsgd_common.cuh"
+#include "kernels_f32.cuh"
+#include "kernels_avg.cuh"
+#include "tc_ptx.cuh"
+
 namespace prsgd {
-inline int tc_create(prsgd_ctx*, std::string* err) { *err = "BF16 precision is not available in this build"; return PRSGD_ERR_STATE; }
-inline void tc_destroy(prsgd_ctx*) {}
-inline int tc_bind_data(prsgd_ctx*, std::string* err) { *err = "BF16 precision is not available in this build"; return PRSGD_ERR_STATE; }
-inline int tc_step(prsgd_ctx*, int64_t, bool) { return PRSGD_ERR_STATE; }
+
+// ---------------------------------------------------------------------------------------------
+// host-side state: tensor maps
+// ---------------------------------------------------------------------------------------------
+struct TcLayerMaps {
+  CUtensorMap shadow_k;     // bf16 W_l  dims {d_in, d_out, N}, box {64, 128, 1}: forward A tiles, shadow stores
+  CUtensorMap shadow_mn;    // same tensor, box {64, 64, 1}: backward A tiles (W^T, MN-major)
+  CUtensorMap master;       // fp32 W_l  dims {d_in, d_out, N}, box {32, 128, 1}: update loads and stores
+  CUtensorMap act_in;       // bf16 a_{l-1} dims {ld, B, N}, box {64, B, 1} (layer 1: the data pool {d0, P, N})
+  CUtensorMap delta_out;    // bf16 dZ_l  dims {ld, B, N}, box {64, B, 1}
+};
+
+struct TcState {
+  TcLayerMaps layer[PRSGD_MAX_LAYERS];
+  int num_sms = 148;
+  bool pool_bound = false;
+};
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline EncodeTiledFn get_encode_fn(std::string* err) {
+  static EncodeTiledFn fn = nullptr;
+  if (fn) return fn;
+  void* p = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q);
+  if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || !p) {
+    *err = "cuTensorMapEncodeTiled is not available from the driver";
+    return nullptr;
+  }
+  fn = reinterpret_cast<EncodeTiledFn>(p);
+  return fn;
 }
+
+// 3-D tiled map with 128-byte swizzle; dims/box innermost first; strides in bytes for dims 1 and 2.
+inline int make_map3(CUtensorMap* m, bool fp32, const void* base, uint64_t d0, uint64_t d1, uint64_t d2,
+                     uint64_t stride1_bytes, uint64_t stride2_bytes, uint32_t b0, uint32_t b1, std::string* err) {
+  EncodeTiledFn enc = get_encode_fn(err);
+  if (!enc) return PRSGD_ERR_CUDA;
+  cuuint64_t dims[3] = {d0, d1, d2};
+  cuuint64_t strides[2] = {stride1_bytes, stride2_bytes};
+  cuuint32_t box[3] = {b0, b1, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = enc(m, fp32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3,
+                   const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    *err = "cuTensorMapEncodeTiled failed with code " + std::to_string((int)r);
+    return PRSGD_ERR_CUDA;
+  }
+  return PRSGD_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// stream kernel: forward and backward-data GEMMs
+// ---------------------------------------------------------------------------------------------
+enum { TC_FWD_RELU = 0, TC_FWD_LINEAR = 1, TC_DX = 2 };
+
+struct StreamArgs {
+  int B, N;
+  int k_blocks;            // contraction length / 64
+  int M_total;             // valid output features
+  int stages;
+  int pool;                // operand B rows come from the data pool at the drawn block
+  DrawArgs draw;
+  uint16_t* out_bk;        // bf16 [N][B][ld_out]
+  float* out_f32;          // fp32 [N][B][ld_out] (logits)
+  int ld_out;
+  const float* bias;       // params + b_off; worker stride bias_stride
+  int64_t bias_stride;
+  const uint16_t* mask_src;  // bf16 a_{l-1} [N][B][ld_out] (TC_DX)
+  const uint8_t* active;
+  DeviceStatus* status;
+};
+
+constexpr int kStreamThreads = 128;
+constexpr uint32_t kTileA = 16384;   // 128 x 64 bf16
+
+__host__ __device__ inline uint32_t stream_stage_bytes(int B) { return kTileA + (uint32_t)B * 128u; }
+inline size_t stream_smem_bytes(int B, int stages) { return (size_t)stages * stream_stage_bytes(B) + 1024 + 256; }
+
+template <int MODE>
+__global__ void __launch_bounds__(kStreamThreads) tc_stream_kernel(const __grid_constant__ CUtensorMap mapW,
+                                                                   const __grid_constant__ CUtensorMap mapB,
+                                                                   const StreamArgs a) {
+  using namespace ptx;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* gen = smem_raw + (base - raw);
+  const uint32_t stage_bytes = stream_stage_bytes(a.B);
+  const int S = a.stages;
+  // barrier block after the stages
+  const uint32_t bar0 = base + (uint32_t)S * stage_bytes;
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 64u + 8u * s; };
+  const uint32_t acc_bar = bar0 + 128u;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen + (size_t)S * stage_bytes + 136);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + (size_t)S * stage_bytes + 140);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int m0 = blockIdx.x * 128, n = blockIdx.y;
+  const uint32_t ncols = a.B < 32 ? 32u : (uint32_t)a.B;
+
+  if (tid == 0) {
+    for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    mbar_init(acc_bar, 1);
+    // a wait that expired in an earlier CTA or launch turns the rest of the work into a no-op
+    *abort_flag = *(volatile unsigned int*)&a.status->error != 0u ? 1 : 0;
+    fence_mbar_init();
+    prefetch_tensormap(&mapW);
+    prefetch_tensormap(&mapB);
+  }
+  if (warp == 1) { tmem_alloc(smem_u32(tmem_slot), ncols); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const bool is_active = (a.active == nullptr || a.active[n] != 0) && *abort_flag == 0;
+
+  if (is_active) {
+    if (warp == 0 && lane == 0) {
+      // ---- producer: TMA loads of the weight tile and the activation tile, one 64-wide K block per stage
+      const int row0 = a.pool ? (int)draw_block(a.draw.seed, n, a.draw.t, a.draw.n_blocks) * a.B : 0;
+      int issued = 0;
+      for (int kb = 0; kb < a.k_blocks; ++kb) {
+        const int s = kb % S;
+        const uint32_t ph = (uint32_t)(kb / S) & 1u;
+        if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, a.status, 0x101)) break;
+        const uint32_t sa = base + (uint32_t)s * stage_bytes, sb = sa + kTileA;
+        mbar_expect_tx(full_bar(s), stage_bytes);
+        if (MODE == TC_DX) {
+          tma_load_3d(sa, &mapW, full_bar(s), m0, kb * 64, n);
+          tma_load_3d(sa + 8192u, &mapW, full_bar(s), m0 + 64, kb * 64, n);
+        } else {
+          tma_load_3d(sa, &mapW, full_bar(s), kb * 64, m0, n);
+        }
+        tma_load_3d(sb, &mapB, full_bar(s), kb * 64, row0, n);
+        issued = kb + 1;
+      }
+      if (*abort_flag) {   // let the copies already in flight land before the CTA goes away
+        for (int kb = issued > S ? issued - S : 0; kb < issued; ++kb) {
+          const uint64_t t0 = globaltimer_ns();
+          while (!mbar_try_wait(full_bar(kb % S), (uint32_t)(kb / S) & 1u) && globaltimer_ns() - t0 < 100000000ull) {}
+        }
+      }
+    } else if (warp == 1 && lane == 0) {
+      // ---- MMA issuer
+      constexpr int A_MN = MODE == TC_DX ? 1 : 0;
+      const uint32_t idesc = idesc_bf16(128, a.B, A_MN, 0);
+      for (int kb = 0; kb < a.k_blocks; ++kb) {
+        const int s = kb % S;
+        const uint32_t ph = (uint32_t)(kb / S) & 1u;
+        if (!mbar_wait(full_bar(s), ph, abort_flag, a.status, 0x102)) break;
+        tc_fence_after();
+        const uint32_t sa = base + (uint32_t)s * stage_bytes, sb = sa + kTileA;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const uint64_t da = A_MN ? smem_desc_sw128(sa + k * 2048u, 8192u, 1024u) : smem_desc_sw128(sa + k * 32u, 16u, 1024u);
+          const uint64_t db = smem_desc_sw128(sb + k * 32u, 16u, 1024u);
+          mma_bf16(tmem, da, db, idesc, (kb | k) != 0 ? 1u : 0u);
+        }
+        mma_commit(empty_bar(s));
+      }
+      mma_commit(acc_bar);
+    }
+    __syncwarp();
+
+    // ---- epilogue: thread <-> output feature m0 + tid, its B accumulators sit in one TMEM lane
+    const bool acc_ok = __all_sync(0xffffffffu, mbar_wait(acc_bar, 0u, abort_flag, a.status, 0x103));
+    tc_fence_after();
+    if (acc_ok) {
+      const int m = m0 + tid;
+      const bool valid = m < a.M_total;
+      float bias = 0.f;
+      if (MODE != TC_DX && valid) bias = a.bias[(int64_t)n * a.bias_stride + m];
+      for (int c0 = 0; c0 < a.B; c0 += 16) {
+        uint32_t v[16];
+        tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
+        tmem_ld_wait();
+        if (valid) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const int64_t o = ((int64_t)n * a.B + c0 + j) * a.ld_out + m;
+            const float x = __uint_as_float(v[j]);
+            if (MODE == TC_FWD_RELU) {
+              a.out_bk[o] = f32_to_bf16_rn(fmaxf(x + bias, 0.f));
+            } else if (MODE == TC_FWD_LINEAR) {
+              a.out_f32[o] = x + bias;
+            } else {
+              a.out_bk[o] = (a.mask_src[o] & 0x7FFFu) != 0 ? f32_to_bf16_rn(x) : (uint16_t)0;
+            }
+          }
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem, ncols);
+}
+
+// ---------------------------------------------------------------------------------------------
+// update kernel: dW GEMM (K = B) + in-place SGD step, optionally fused with the node average
+// ---------------------------------------------------------------------------------------------
+struct UpdateArgs {
+  int B, N;
+  int tiles_m, tiles_n;
+  float gamma;
+  int pool;
+  DrawArgs draw;
+  const uint8_t* active;
+  DeviceStatus* status;
+};
+
+constexpr int kUpdThreads = 224;          // warp 0 loader, 1 MMA, 2 storer, 3..6 epilogue
+constexpr uint32_t kMasterTile = 65536;   // 128 x 128 fp32, four 128 x 32 boxes
+constexpr uint32_t kOpsRegion = 32768;    // operands, later the bf16 output tile (two 128 x 64 boxes)
+constexpr uint32_t kUpdStage = kMasterTile + kOpsRegion;
+constexpr size_t kUpdSmem = 2 * kUpdStage + 1024 + 256;
+
+template <bool FUSE>
+__global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_constant__ CUtensorMap mapDelta,
+                                                                   const __grid_constant__ CUtensorMap mapAct,
+                                                                   const __grid_constant__ CUtensorMap mapMaster,
+                                                                   const __grid_constant__ CUtensorMap mapShadow,
+                                                                   const UpdateArgs a) {
+  using namespace ptx;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* gen = smem_raw + (base - raw);
+  auto master_u32 = [&](int s) { return base + (uint32_t)s * kUpdStage; };
+  auto ops_u32 = [&](int s) { return base + (uint32_t)s * kUpdStage + kMasterTile; };
+  const uint32_t bar0 = base + 2u * kUpdStage;
+  auto full_ops = [&](int s) { return bar0 + 8u * s; };
+  auto full_w = [&](int s) { return bar0 + 16u + 8u * s; };
+  auto stage_empty = [&](int s) { return bar0 + 32u + 8u * s; };
+  auto acc_full = [&](int s) { return bar0 + 48u + 8u * s; };
+  auto acc_empty = [&](int s) { return bar0 + 64u + 8u * s; };
+  auto tile_ready = [&](int s) { return bar0 + 80u + 8u * s; };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen + 2 * kUpdStage + 96);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + 2 * kUpdStage + 100);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t op_box = (uint32_t)a.B * 128u;       // one {64, B} box
+  const int tiles = a.tiles_m * a.tiles_n;
+  const int items_all = FUSE ? tiles : tiles * a.N;    // FUSE: a CTA owns a tile and walks all workers
+
+  if (tid == 0) {
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(full_ops(s), 1); mbar_init(full_w(s), 1); mbar_init(stage_empty(s), 1);
+      mbar_init(acc_full(s), 1); mbar_init(acc_empty(s), 128); mbar_init(tile_ready(s), 128);
+    }
+    *abort_flag = *(volatile unsigned int*)&a.status->error != 0u ? 1 : 0;   // an earlier expired wait: no-op
+    fence_mbar_init();
+    prefetch_tensormap(&mapDelta); prefetch_tensormap(&mapAct);
+    prefetch_tensormap(&mapMaster); prefetch_tensormap(&mapShadow);
+  }
+  if (warp == 1) { tmem_alloc(smem_u32(tmem_slot), 256u); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const int total_items = *abort_flag != 0 ? 0 : items_all;
+
+  // Every role walks the same sequence of (tile, worker) items; `it` counts the items it has handled.
+  auto item_active = [&](int n) { return FUSE || a.active == nullptr || a.active[n] != 0; };
+
+  if (warp == 0 && lane == 0) {
+    // ---------------- loader
+    uint32_t it = 0;
+    bool ok = true;
+    for (int w = blockIdx.x; w < total_items && ok; w += gridDim.x) {
+      const int tile = FUSE ? w : w % tiles;
+      const int n_begin = FUSE ? 0 : w / tiles, n_end = FUSE ? a.N : n_begin + 1;
+      const int m0 = (tile / a.tiles_n) * 128, n0 = (tile % a.tiles_n) * 128;
+      for (int n = n_begin; n < n_end; ++n) {
+        if (!item_active(n)) continue;
+        const int s = it & 1;
+        const uint32_t ph = (it >> 1) & 1u;
+        ok = mbar_wait(stage_empty(s), ph ^ 1u, abort_flag, a.status, 0x201);
+        if (!ok) break;
+        const int row0 = a.pool ? (int)draw_block(a.draw.seed, n, a.draw.t, a.draw.n_blocks) * a.B : 0;
+        const uint32_t ops = ops_u32(s);
+        mbar_expect_tx(full_ops(s), 4u * op_box);
+        tma_load_3d(ops, &mapDelta, full_ops(s), m0, 0, n);
+        tma_load_3d(ops + op_box, &mapDelta, full_ops(s), m0 + 64, 0, n);
+        tma_load_3d(ops + 2u * op_box, &mapAct, full_ops(s), n0, row0, n);
+        tma_load_3d(ops + 3u * op_box, &mapAct, full_ops(s), n0 + 64, row0, n);
+        mbar_expect_tx(full_w(s), kMasterTile);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) tma_load_3d(master_u32(s) + q * 16384u, &mapMaster, full_w(s), n0 + 32 * q, m0, n);
+        ++it;
+      }
+    }
+    if (*abort_flag && it > 0) {   // let the copies already in flight land before the CTA goes away
+      const uint64_t t0 = globaltimer_ns();
+      const uint32_t last = it - 1;
+      while (!mbar_try_wait(full_w(last & 1), (last >> 1) & 1u) && globaltimer_ns() - t0 < 100000000ull) {}
+    }
+  } else if (warp == 1 && lane == 0) {
+    // ---------------- MMA issuer
+    const uint32_t idesc = idesc_bf16(128, 128, 1, 1);
+    const int ksteps = a.B / 16;
+    uint32_t it = 0;
+    bool ok = true;
+    for (int w = blockIdx.x; w < total_items && ok; w += gridDim.x) {
+      const int n_begin = FUSE ? 0 : w / tiles, n_end = FUSE ? a.N : n_begin + 1;
+      for (int n = n_begin; n < n_end; ++n) {
+        if (!item_active(n)) continue;
+        const int s = it & 1;
+        const uint32_t ph = (it >> 1) & 1u;
+        ok = mbar_wait(acc_empty(s), ph ^ 1u, abort_flag, a.status, 0x202) &&
+             mbar_wait(full_ops(s), ph, abort_flag, a.status, 0x203);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t sa = ops_u32(s), sb = sa + 2u * op_box;
+        for (int k = 0; k < ksteps; ++k)
+          mma_bf16(tmem + (uint32_t)s * 128u, smem_desc_sw128(sa + k * 2048u, op_box, 1024u),
+                   smem_desc_sw128(sb + k * 2048u, op_box, 1024u), idesc, k != 0 ? 1u : 0u);
+        mma_commit(acc_full(s));
+        ++it;
+      }
+    }
+  } else if (warp == 2 && lane == 0) {
+    // ---------------- storer: TMA stores of finished tiles, then hands the stage back to the loader
+    uint32_t it = 0, tile_it = 0;
+    bool ok = true;
+    for (int w = blockIdx.x; w < total_items && ok; w += gridDim.x) {
+      const int tile = FUSE ? w : w % tiles;
+      const int m0 = (tile / a.tiles_n) * 128, n0 = (tile % a.tiles_n) * 128;
+      if (!FUSE) {
+        const int n = w / tiles;
+        if (!item_active(n)) continue;
+        const int s = it & 1;
+        const uint32_t ph = (it >> 1) & 1u;
+        ok = mbar_wait(tile_ready(s), ph, abort_flag, a.status, 0x204);
+        if (!ok) break;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) tma_store_3d(&mapMaster, master_u32(s) + q * 16384u, n0 + 32 * q, m0, n);
+        tma_store_3d(&mapShadow, ops_u32(s), n0, m0, n);
+        tma_store_3d(&mapShadow, ops_u32(s) + 16384u, n0 + 64, m0, n);
+        tma_commit_group();
+        tma_wait_group_read0();
+        mbar_arrive(stage_empty(s));
+        ++it;
+      } else {
+        it += (uint32_t)a.N;
+        const int s = (it - 1) & 1;                       // stage of the tile's last worker
+        ok = mbar_wait(tile_ready(0), tile_it & 1u, abort_flag, a.status, 0x205);
+        if (!ok) break;
+        for (int n = 0; n < a.N; ++n) {
+#pragma unroll
+          for (int q = 0; q < 4; ++q) tma_store_3d(&mapMaster, master_u32(s) + q * 16384u, n0 + 32 * q, m0, n);
+          tma_store_3d(&mapShadow, ops_u32(s), n0, m0, n);
+          tma_store_3d(&mapShadow, ops_u32(s) + 16384u, n0 + 64, m0, n);
+        }
+        tma_commit_group();
+        tma_wait_group_read0();
+        mbar_arrive(stage_empty(s));
+        ++tile_it;
+      }
+    }
+    tma_wait_group0();
+  } else if (warp >= 3) {
+    // ---------------- epilogue: row r of the tile <-> TMEM lane r
+    const int q4 = warp & 3;
+    const int r = q4 * 32 + lane;
+    const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
+    const uint32_t row_off = (uint32_t)r * 128u;
+    const uint32_t sw = (uint32_t)(r & 7);
+    const int etid = tid - 96;                            // 0..127 among the epilogue threads
+    const float fN = (float)a.N;
+    uint32_t it = 0;
+    bool ok = true;
+    for (int w = blockIdx.x; w < total_items && ok; w += gridDim.x) {
+      const int n_begin = FUSE ? 0 : w / tiles, n_end = FUSE ? a.N : n_begin + 1;
+      float sum[FUSE ? 128 : 1];
+      if (FUSE) {
+#pragma unroll
+        for (int i = 0; i < 128; ++i) sum[FUSE ? i : 0] = 0.f;
+      }
+      for (int n = n_begin; n < n_end; ++n) {
+        if (!item_active(n)) continue;
+        const bool upd = a.active == nullptr || a.active[n] != 0;
+        const int s = it & 1;
+        const uint32_t ph = (it >> 1) & 1u;
+        ok = mbar_wait(full_w(s), ph, abort_flag, a.status, 0x206) &&
+             mbar_wait(acc_full(s), ph, abort_flag, a.status, 0x207);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        uint8_t* mst = gen + (size_t)s * kUpdStage;
+        uint8_t* stg = mst + kMasterTile;
+        const bool last = FUSE && n == a.N - 1;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint32_t v[32];
+          tmem_ld32(tmem + lane_off + (uint32_t)s * 128u + (uint32_t)c * 32u, v);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            float4* pw = reinterpret_cast<float4*>(mst + c * 16384 + row_off + (((uint32_t)j ^ sw) << 4));
+            float4 x = *pw;
+            if (upd) {
+              x.x = fmaf(-a.gamma, __uint_as_float(v[4 * j + 0]), x.x);
+              x.y = fmaf(-a.gamma, __uint_as_float(v[4 * j + 1]), x.y);
+              x.z = fmaf(-a.gamma, __uint_as_float(v[4 * j + 2]), x.z);
+              x.w = fmaf(-a.gamma, __uint_as_float(v[4 * j + 3]), x.w);
+            }
+            if (FUSE) {
+              float* sp = &sum[FUSE ? c * 32 + 4 * j : 0];
+              sp[0] += x.x; sp[FUSE ? 1 : 0] += x.y; sp[FUSE ? 2 : 0] += x.z; sp[FUSE ? 3 : 0] += x.w;
+              if (last) {
+                x.x = __fdiv_rn(sp[0], fN); x.y = __fdiv_rn(sp[FUSE ? 1 : 0], fN);
+                x.z = __fdiv_rn(sp[FUSE ? 2 : 0], fN); x.w = __fdiv_rn(sp[FUSE ? 3 : 0], fN);
+              }
+            }
+            if (!FUSE || last) {
+              *pw = x;
+              const uint32_t chunk = (uint32_t)((c & 1) * 4 + (j >> 1));
+              uint2* pb = reinterpret_cast<uint2*>(stg + (c >> 1) * 16384 + row_off + ((chunk ^ sw) << 4) + (j & 1) * 8);
+              *pb = make_uint2(pack_bf16x2(x.x, x.y), pack_bf16x2(x.z, x.w));
+            }
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(acc_empty(s));
+        if (!FUSE) {
+          fence_proxy_async();
+          mbar_arrive(tile_ready(s));
+        } else if (last) {
+          fence_proxy_async();
+          mbar_arrive(tile_ready(0));
+        } else {
+          named_bar_sync(1, 128);                         // every epilogue thread is done reading stage s
+          if (etid == 0) mbar_arrive(stage_empty(s));
+        }
+        ++it;
+      }
+    }
+  }
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem, 256u);
+}
+
+// b_l <- b_l - gamma * sum_b dZ_l[b, :], optionally followed by the node average (fixed order).
+template <bool FUSE>
+__global__ void __launch_bounds__(128) bias_update_kernel(float* params, int64_t m_pad, int64_t b_off, int d_out,
+                                                          const uint16_t* delta_bk, int ld, int B, int N, float gamma,
+                                                          const uint8_t* active) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= d_out) return;
+  const int n_begin = FUSE ? 0 : (int)blockIdx.y, n_end = FUSE ? N : n_begin + 1;
+  float sum = 0.f;
+  for (int n = n_begin; n < n_end; ++n) {
+    float* bp = params + (int64_t)n * m_pad + b_off + j;
+    float x = *bp;
+    if (active == nullptr || active[n] != 0) {
+      float g = 0.f;
+      for (int b = 0; b < B; ++b) g += __uint_as_float((uint32_t)delta_bk[((int64_t)n * B + b) * ld + j] << 16);
+      x = fmaf(-gamma, g, x);
+    }
+    if (FUSE) sum += x;
+    else *bp = x;
+  }
+  if (FUSE) {
+    const float y = __fdiv_rn(sum, (float)N);
+    for (int n = 0; n < N; ++n) params[(int64_t)n * m_pad + b_off + j] = y;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------------
+inline int tc_create(prsgd_ctx* c, std::string* err) {
+  if (c->B > 64) { *err = "BF16 precision supports batch 16, 32 or 64"; return PRSGD_ERR_ALIGN; }
+  TcState* st = new (std::nothrow) TcState();
+  if (!st) { *err = "out of host memory"; return PRSGD_ERR_ARG; }
+  int sms = 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device) == cudaSuccess && sms > 0) st->num_sms = sms;
+  const uint64_t N = c->N, B = c->B;
+  int rc = PRSGD_OK;
+  for (int l = 1; l <= c->L && rc == PRSGD_OK; ++l) {
+    const Layer& ly = c->layer[l - 1];
+    TcLayerMaps& mp = st->layer[l - 1];
+    const uint64_t din = ly.d_in, dout = ly.d_out;
+    const uint16_t* sh = c->shadow + ly.w_off;
+    const float* ms = c->params + ly.w_off;
+    rc = make_map3(&mp.shadow_k, false, sh, din, dout, N, din * 2, (uint64_t)c->m_pad * 2, 64, 128, err);
+    if (rc == PRSGD_OK) rc = make_map3(&mp.shadow_mn, false, sh, din, dout, N, din * 2, (uint64_t)c->m_pad * 2, 64, 64, err);
+    if (rc == PRSGD_OK) rc = make_map3(&mp.master, true, ms, din, dout, N, din * 4, (uint64_t)c->m_pad * 4, 32, 128, err);
+    const uint64_t ld = c->buf.ld[l];
+    if (rc == PRSGD_OK) rc = make_map3(&mp.delta_out, false, c->buf.delta_bk[l], ld, B, N, ld * 2, B * ld * 2, 64, (uint32_t)B, err);
+    if (rc == PRSGD_OK && l > 1) {
+      const uint64_t ldi = c->buf.ld[l - 1];
+      rc = make_map3(&mp.act_in, false, c->buf.act_bk[l - 1], ldi, B, N, ldi * 2, B * ldi * 2, 64, (uint32_t)B, err);
+    }
+  }
+  if (rc != PRSGD_OK) { delete st; return rc; }
+  cudaError_t e = cudaSuccess;
+  const int big = (int)stream_smem_bytes(c->B, 8);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_stream_kernel<TC_FWD_RELU>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_stream_kernel<TC_FWD_LINEAR>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_stream_kernel<TC_DX>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kUpdSmem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kUpdSmem);
+  if (e != cudaSuccess) {
+    *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e);
+    delete st;
+    return PRSGD_ERR_CUDA;
+  }
+  c->tc = st;
+  return PRSGD_OK;
+}
+
+inline void tc_destroy(prsgd_ctx* c) {
+  delete static_cast<TcState*>(c->tc);
+  c->tc = nullptr;
+}
+
+inline int tc_bind_data(prsgd_ctx* c, std::string* err) {
+  TcState* st = static_cast<TcState*>(c->tc);
+  const uint64_t d0 = c->dims[0];
+  int rc = make_map3(&st->layer[0].act_in, false, c->X, d0, (uint64_t)c->P, (uint64_t)c->N, d0 * 2,
+                     (uint64_t)c->P * d0 * 2, 64, (uint32_t)c->B, err);
+  st->pool_bound = rc == PRSGD_OK;
+  return rc;
+}
+
+inline int stream_stages(int B, int k_blocks) {
+  int s = (int)(98304 / stream_stage_bytes(B));   // ~96 KB of stages: two CTAs per SM
+  if (s > 8) s = 8;
+  if (s > k_blocks) s = k_blocks;
+  return s < 1 ? 1 : s;
+}
+
+// forward GEMM of layer l (1-based)
+inline void tc_launch_forward(prsgd_ctx* c, int l, const DrawArgs& dr, const uint8_t* active) {
+  TcState* st = static_cast<TcState*>(c->tc);
+  const Layer& ly = c->layer[l - 1];
+  StreamArgs a{};
+  a.B = c->B; a.N = c->N; a.k_blocks = ly.d_in / 64; a.M_total = ly.d_out;
+  a.stages = stream_stages(c->B, a.k_blocks);
+  a.pool = l == 1; a.draw = dr; a.ld_out = c->buf.ld[l];
+  a.out_bk = c->buf.act_bk[l]; a.out_f32 = c->buf.act_f32[l];
+  a.bias = c->params + ly.b_off; a.bias_stride = c->m_pad;
+  a.active = active; a.status = c->status;
+  dim3 grid((ly.d_out + 127) / 128, c->N);
+  const size_t smem = stream_smem_bytes(c->B, a.stages);
+  if (l < c->L)
+    tc_stream_kernel<TC_FWD_RELU><<<grid, kStreamThreads, smem, c->stream>>>(st->layer[l - 1].shadow_k, st->layer[l - 1].act_in, a);
+  else
+    tc_stream_kernel<TC_FWD_LINEAR><<<grid, kStreamThreads, smem, c->stream>>>(st->layer[l - 1].shadow_k, st->layer[l - 1].act_in, a);
+}
+
+// dZ_{l-1} from dZ_l through W_l (l >= 2)
+inline void tc_launch_dx(prsgd_ctx* c, int l, const DrawArgs& dr, const uint8_t* active) {
+  TcState* st = static_cast<TcState*>(c->tc);
+  const Layer& ly = c->layer[l - 1];
+  StreamArgs a{};
+  a.B = c->B; a.N = c->N; a.k_blocks = c->buf.ld[l] / 64; a.M_total = ly.d_in;
+  a.stages = stream_stages(c->B, a.k_blocks);
+  a.pool = 0; a.draw = dr; a.ld_out = c->buf.ld[l - 1];
+  a.out_bk = c->buf.delta_bk[l - 1]; a.mask_src = c->buf.act_bk[l - 1];
+  a.active = active; a.status = c->status;
+  dim3 grid((ly.d_in + 127) / 128, c->N);
+  const size_t smem = stream_smem_bytes(c->B, a.stages);
+  tc_stream_kernel<TC_DX><<<grid, kStreamThreads, smem, c->stream>>>(st->layer[l - 1].shadow_mn, st->layer[l - 1].delta_out, a);
+}
+
+inline void tc_launch_update(prsgd_ctx* c, int l, const DrawArgs& dr, const uint8_t* active, bool fuse) {
+  TcState* st = static_cast<TcState*>(c->tc);
+  const Layer& ly = c->layer[l - 1];
+  UpdateArgs a{};
+  a.B = c->B; a.N = c->N; a.tiles_m = (ly.d_out + 127) / 128; a.tiles_n = (ly.d_in + 127) / 128;
+  a.gamma = c->gamma; a.pool = l == 1; a.draw = dr; a.active = active; a.status = c->status;
+  const int items = a.tiles_m * a.tiles_n * (fuse ? 1 : c->N);
+  const int grid = items < st->num_sms ? items : st->num_sms;
+  const TcLayerMaps& mp = st->layer[l - 1];
+  if (fuse)
+    tc_update_kernel<true><<<grid, kUpdThreads, kUpdSmem, c->stream>>>(mp.delta_out, mp.act_in, mp.master, mp.shadow_k, a);
+  else
+    tc_update_kernel<false><<<grid, kUpdThreads, kUpdSmem, c->stream>>>(mp.delta_out, mp.act_in, mp.master, mp.shadow_k, a);
+}
+
+inline void tc_launch_bias(prsgd_ctx* c, int l, const uint8_t* active, bool fuse) {
+  const Layer& ly = c->layer[l - 1];
+  dim3 grid((ly.d_out + 127) / 128, fuse ? 1 : c->N);
+  if (fuse)
+    bias_update_kernel<true><<<grid, 128, 0, c->stream>>>(c->params, c->m_pad, ly.b_off, ly.d_out, c->buf.delta_bk[l],
+                                                         c->buf.ld[l], c->B, c->N, c->gamma, active);
+  else
+    bias_update_kernel<false><<<grid, 128, 0, c->stream>>>(c->params, c->m_pad, ly.b_off, ly.d_out, c->buf.delta_bk[l],
+                                                          c->buf.ld[l], c->B, c->N, c->gamma, active);
+}
+
+}  // namespace prsgd

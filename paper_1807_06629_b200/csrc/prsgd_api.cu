@@ -136,10 +136,10 @@ size_t carve_scratch(int N, const prsgd_model_spec* s, int64_t m_pad, prsgd_ctx*
       const int ld = (int)round_up(s->dims[l], 64);
       const size_t e = (size_t)N * B * ld;
       unsigned char *abk = nullptr, *akb = nullptr, *z = nullptr;
-      if (l < L) { abk = take(2 * e); akb = take(2 * e); }
+      if (l < L) abk = take(2 * e);
       else z = take(4 * e);                              // logits, fp32
       auto dbk = take(2 * e);
-      auto dkb = take(2 * e);
+      unsigned char* dkb = nullptr;
       if (ctx) {
         ctx->buf.ld[l] = ld;
         ctx->buf.act_bk[l] = reinterpret_cast<uint16_t*>(abk);
@@ -273,6 +273,43 @@ int step_f32(prsgd_ctx* c, int64_t t, bool averaging) {
     prof_begin(c, fuse ? PRSGD_KERNEL_UPDATE_AVERAGE : PRSGD_KERNEL_UPDATE);
     if (fuse) launch_gemm_f32<64, false, false, EPI_DW, true>(c, g);
     else      launch_gemm_f32<64, false, false, EPI_DW, false>(c, g);
+    LAUNCH_CHECK(c);
+  }
+  return PRSGD_OK;
+}
+
+// One iteration of Algorithm 1 on the bf16-operand tensor-core path.
+int step_bf16(prsgd_ctx* c, int64_t t, bool averaging) {
+  const int L = c->L, N = c->N;
+  const uint8_t* act_mask = c->has_mask ? c->active : nullptr;
+  const bool fuse = averaging && c->fused_average;
+  const DrawArgs dr = draw_args(c, t);
+  for (int l = 1; l <= L; ++l) {
+    prof_begin(c, PRSGD_KERNEL_FORWARD);
+    tc_launch_forward(c, l, dr, act_mask);
+    LAUNCH_CHECK(c);
+  }
+  {
+    SoftmaxArgs a{};
+    a.logits = c->buf.act_f32[L]; a.ldz = c->buf.ld[L];
+    a.delta_bk = c->buf.delta_bk[L]; a.ld_bf = c->buf.ld[L];
+    a.Y = c->Y; a.P = c->P; a.B = c->B; a.C = c->dims[L]; a.draw = dr;
+    a.losses = c->losses; a.draws = c->draws; a.active = act_mask;
+    prof_begin(c, PRSGD_KERNEL_SOFTMAX);
+    softmax_ce_kernel<<<N, 256, 0, c->stream>>>(a);
+    LAUNCH_CHECK(c);
+  }
+  for (int l = L; l >= 1; --l) {          // dX_l reads W_l before the update of layer l overwrites it
+    if (l > 1) {
+      prof_begin(c, PRSGD_KERNEL_DX);
+      tc_launch_dx(c, l, dr, act_mask);
+      LAUNCH_CHECK(c);
+    }
+    prof_begin(c, fuse ? PRSGD_KERNEL_UPDATE_AVERAGE : PRSGD_KERNEL_UPDATE);
+    tc_launch_update(c, l, dr, act_mask, fuse);
+    LAUNCH_CHECK(c);
+    prof_begin(c, PRSGD_KERNEL_MISC);
+    tc_launch_bias(c, l, act_mask, fuse);
     LAUNCH_CHECK(c);
   }
   return PRSGD_OK;
@@ -461,7 +498,7 @@ int prsgd_local_steps(prsgd_ctx* c, int64_t k) {
   for (int64_t s = 0; s < k; ++s) {
     const int64_t t = c->t + 1;
     const bool averaging = c->I > 0 && (t % c->I) == 0;
-    int rc = c->precision == PRSGD_PRECISION_BF16 ? tc_step(c, t, averaging) : step_f32(c, t, averaging);
+    int rc = c->precision == PRSGD_PRECISION_BF16 ? step_bf16(c, t, averaging) : step_f32(c, t, averaging);
     if (rc != PRSGD_OK) return rc;
     if (averaging && !c->fused_average) {
       rc = launch_average(c);

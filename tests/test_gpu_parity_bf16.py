@@ -1,0 +1,187 @@
+"""GPU parity, bf16-operand tensor-core path (tcgen05 + TMA), through the C ABI.
+
+The oracle runs in fp64 on the same inputs the GPU sees (data pool rounded to
+bf16 once, fp32 initial parameters).  Tolerance: relative L2 of the stacked
+parameters <= 2e-2 after one full averaging period from a synchronised state.
+Because one period moves the parameters by only a few percent, the tests also
+bound the relative L2 error of the *update* x^t - x^0, which a wrong or
+missing gradient cannot pass.
+
+bf16 rounding of the weights moves a hidden pre-activation by ~2^-9 of its
+scale, so a fraction p ~ 1e-3 of the ReLU units sits close enough to zero to
+switch on one side only; each such unit is a whole wrong entry of dZ and the
+update error it causes is ~sqrt(p), a few percent.  Random-init runs therefore
+use TOL_UPDATE; runs whose hidden biases are +-6 (every unit firmly on or off,
+no switch possible) must meet the much tighter TOL_UPDATE_MARGIN.
+"""
+import numpy as np
+import pytest
+
+from oracle import prsgd_oracle as orc
+from paper_1807_06629_b200 import synth
+from helpers import make_ctx, make_inputs, oracle_run, rel_l2
+
+pytestmark = pytest.mark.gpu
+
+TOL_PERIOD = 2e-2
+TOL_UPDATE = 1e-1
+TOL_UPDATE_MARGIN = 1e-2
+
+
+def with_margin(x0, dims):
+    """Hidden biases alternate +6 / -6: half the units always fire, half never do."""
+    x = x0.copy()
+    off = 0
+    for l in range(len(dims) - 1):
+        off += dims[l] * dims[l + 1]
+        if l < len(dims) - 2:
+            x[off:off + dims[l + 1]] = np.where(np.arange(dims[l + 1]) % 2 == 0, 6.0, -6.0)
+        off += dims[l + 1]
+    return x
+
+
+@pytest.fixture(scope="module")
+def torch_cuda():
+    import torch
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    return torch
+
+
+def _w(name, N, dims, B, I=2, gamma=0.05, P=None, shift=0.5, seed=31):
+    return synth.Workload(name, N, dims, B, gamma, I, 2 * I, 1, P if P else 4 * B, mean_shift=shift, seed=seed)
+
+
+SMALL = [
+    _w("tc-logistic", 2, (64, 10), 32),
+    _w("tc-two-layer", 3, (128, 256, 10), 32),
+    _w("tc-b16", 2, (64, 128, 64, 10), 16),
+    _w("tc-b64", 2, (128, 128, 100), 64),
+    _w("tc-ragged-tiles", 2, (192, 320, 100), 32),
+    _w("tc-many-kblocks", 1, (1024, 128, 10), 32),
+]
+
+
+@pytest.mark.parametrize("w", SMALL, ids=[w.name for w in SMALL])
+def test_every_gemm_is_tight_when_no_relu_can_switch(torch_cuda, w):
+    X, Y, x0 = make_inputs(w)
+    x0 = with_margin(x0, w.dims)
+    p = make_ctx(w, X, Y, x0, I=0)
+    x0s = np.tile(x0, (w.N, 1)).astype(np.float64)
+    losses = {}
+    want = oracle_run(w, X, Y, x0s, 0, 1, I=0, losses=losses)
+    p.local_steps(1)
+    got = p.get_params_stacked()
+    assert np.allclose(p.get_losses(), [losses[(i, 1)] for i in range(w.N)], rtol=1e-2, atol=1e-3)
+    off = 0
+    for l in range(len(w.dims) - 1):                      # every layer's W and b on its own
+        for cnt in (w.dims[l] * w.dims[l + 1], w.dims[l + 1]):
+            g, t = got[:, off:off + cnt] - x0s[:, off:off + cnt], want[:, off:off + cnt] - x0s[:, off:off + cnt]
+            assert np.linalg.norm(t) > 0
+            assert rel_l2(g, t) <= TOL_UPDATE_MARGIN, (l, cnt, rel_l2(g, t))
+            off += cnt
+
+
+@pytest.mark.parametrize("w", SMALL, ids=[w.name for w in SMALL])
+def test_one_step_and_one_period(torch_cuda, w):
+    X, Y, x0 = make_inputs(w)
+    p = make_ctx(w, X, Y, x0)
+    x0s = np.tile(x0, (w.N, 1)).astype(np.float64)
+    # one iteration
+    losses = {}
+    want1 = oracle_run(w, X, Y, x0s, 0, 1, I=0, losses=losses)
+    p.set_interval(0)
+    p.local_steps(1)
+    got1 = p.get_params_stacked()
+    assert p.get_draws().tolist() == [orc.draw_block(w.seed, i, 1, w.n_blocks) for i in range(w.N)]
+    gl, wl = p.get_losses(), np.array([losses[(i, 1)] for i in range(w.N)])
+    assert np.allclose(gl, wl, rtol=2e-2, atol=2e-3), (gl, wl)
+    assert rel_l2(got1 - x0s, want1 - x0s) <= TOL_UPDATE, rel_l2(got1 - x0s, want1 - x0s)
+    assert rel_l2(got1, want1) <= TOL_PERIOD
+    # one full period from the synchronised start
+    p.set_params(x0)
+    p.set_step(0)
+    p.set_interval(w.I)
+    p.local_steps(w.I)
+    got = p.get_params_stacked()
+    want = oracle_run(w, X, Y, x0s, 0, w.I)
+    assert all(np.array_equal(got[i], got[0]) for i in range(w.N))
+    assert rel_l2(got, want) <= TOL_PERIOD
+    assert rel_l2(got - x0s, want - x0s) <= TOL_UPDATE, rel_l2(got - x0s, want - x0s)
+
+
+def test_fused_average_equals_update_then_average_bit_for_bit(torch_cuda):
+    from paper_1807_06629_b200 import binding
+    for w in (SMALL[1], SMALL[4], _w("tc-n5", 5, (64, 128, 10), 32, I=3)):
+        X, Y, x0 = make_inputs(w)
+        outs = []
+        for fused in (1, 0):
+            p = make_ctx(w, X, Y, x0)
+            p.set_option(binding.OPT_FUSED_AVERAGE, fused)
+            p.local_steps(2 * w.I + 1)
+            outs.append(p.get_params_stacked())
+        assert np.array_equal(outs[0], outs[1])
+
+
+def test_shadow_tracks_master_and_padding_stays_zero(torch_cuda):
+    torch = torch_cuda
+    w = SMALL[4]
+    X, Y, x0 = make_inputs(w)
+    p = make_ctx(w, X, Y, x0)
+    p.local_steps(2 * w.I + 1)
+    p.sync()
+    store = p.params.cpu().numpy().reshape(w.N, p.m_pad)
+    shadow = p.shadow.view(torch.int16).cpu().numpy().view(np.uint16).reshape(w.N, p.m_pad)
+    keep = np.zeros(p.m_pad, dtype=bool)
+    for l in range(len(w.dims) - 1):
+        a, n = p.layout.w_off[l], w.dims[l] * w.dims[l + 1]
+        keep[a:a + n] = True
+        assert np.array_equal(shadow[:, a:a + n], synth.bf16_bits(store[:, a:a + n]))   # weights: shadow = bf16(master)
+        keep[p.layout.b_off[l]:p.layout.b_off[l] + w.dims[l + 1]] = True
+    assert np.all(store[:, ~keep] == 0.0)
+
+
+def test_inactive_workers_keep_their_point(torch_cuda):
+    w = _w("tc-mask", 4, (64, 128, 10), 32, I=0)
+    X, Y, x0 = make_inputs(w)
+    fn = orc.mlp_grad_fn(w.dims, X.astype(np.float64), Y, w.B, w.seed)
+    I_i, S = [3, 1, 2, 3], 2
+    q = make_ctx(w, X, Y, x0, I=0)
+    for s in range(S):
+        q.average()
+        for k in range(1, max(I_i) + 1):
+            q.set_active([1 if k <= I_i[i] else 0 for i in range(w.N)])
+            q.local_steps(1)
+    want = orc.pr_sgd_heterogeneous(np.tile(x0, (w.N, 1)), w.gamma, I_i, S, fn)
+    got = q.get_params_stacked()
+    x0s = np.tile(x0, (w.N, 1))
+    assert rel_l2(got - x0s, want - x0s) <= TOL_UPDATE
+    # fused average with a mask: inactive workers contribute their unchanged point
+    r = make_ctx(w, X, Y, x0, I=1)
+    r.set_active([1, 0, 1, 0])
+    r.local_steps(1)
+    one = oracle_run(w, X, Y, x0s, 0, 1, I=0)
+    one[1], one[3] = x0, x0
+    assert rel_l2(r.get_params_stacked()[0] - x0, one.mean(0) - x0) <= TOL_UPDATE
+
+
+@pytest.mark.parametrize("name,I", [("cfg3", 4), ("cfg4", 2)])
+def test_full_size_configs(torch_cuda, name, I):
+    """cfg3 / cfg4 at their full N, widths and batch, in the launch shapes the benchmark times."""
+    w = synth.WORKLOADS[name].with_(pool_samples=4 * synth.WORKLOADS[name].B, I=I)
+    X, Y, x0 = make_inputs(w)
+    p = make_ctx(w, X, Y, x0)
+    x0s = np.tile(x0, (w.N, 1)).astype(np.float64)
+    p.local_steps(w.I)
+    got = p.get_params_stacked()
+    want = oracle_run(w, X, Y, x0s, 0, w.I)
+    assert all(np.array_equal(got[i], got[0]) for i in range(w.N))
+    assert rel_l2(got, want) <= TOL_PERIOD
+    assert rel_l2(got - x0s, want - x0s) <= TOL_UPDATE, rel_l2(got - x0s, want - x0s)
+    # the next (non-averaging) iteration of a few sampled workers: x_i^t - x_i^{t-1} = -gamma G_i^t
+    fn = orc.mlp_grad_fn(w.dims, X.astype(np.float64), Y, w.B, w.seed)
+    sample = list(range(0, w.N, max(1, w.N // 4)))
+    G = np.stack([fn(i, w.I + 1, got[i].astype(np.float64)) for i in sample])
+    p.local_steps(1)
+    nxt = p.get_params_stacked()
+    for k, i in enumerate(sample):
+        assert rel_l2(nxt[i] - got[i], -w.gamma * G[k]) <= TOL_UPDATE
