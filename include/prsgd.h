@@ -213,6 +213,35 @@ const char* prsgd_last_error(prsgd_ctx* ctx);
  * m >= 0.  Asynchronous on cuda_stream.  Uses no scratch memory. */
 int prsgd_average_rows(float* d_P, int64_t N, int64_t m, int64_t row_stride, void* cuda_stream);
 
+/* Node average of a bare [N, row_stride] array WITHOUT any allocation and
+ * without touching the array: y_j = (1/N) sum_i P[i*row_stride + j], j < m,
+ * summed in row order in fp32 exactly as prsgd_get_average does, delivered to
+ * dst (m floats; dst_on_device says whether dst is device or host memory).
+ * The paper has no counterpart to this call; it exists for callers that must
+ * not allocate: a monitoring or logging thread that wants xbar^t while the
+ * training stream is busy cannot afford cudaMalloc (it synchronises the whole
+ * device and stalls the step in flight), and a process running under a fixed
+ * device-memory budget has nothing left to allocate from.  Such callers often
+ * hold only pageable host memory, which a kernel cannot write, so the mean is
+ * staged in device memory: here that staging row is a fixed array inside the
+ * library (PRSGD_NOALLOC_MAX_M floats = 4 MiB, held by every GPU that loads the
+ * library until the process exits) instead of caller-provided scratch.
+ *  - m must be in 0..PRSGD_NOALLOC_MAX_M, otherwise PRSGD_ERR_SIZE; d_P 16-byte
+ *    aligned, row_stride >= m and a multiple of 4, N >= 1.
+ *  - The first call on each device looks up the array's device address (that
+ *    device must be current, as for every call); make that first call outside
+ *    any stream capture.  No call allocates or frees anything.
+ *  - All calls on one device share the staging row.  A call overwrites the
+ *    first m entries before reading them back and relies on no earlier
+ *    content, but two calls whose GPU work can overlap (different streams, or
+ *    different host threads) race on it: serialise them.
+ *  - Work is enqueued on cuda_stream; with dst on the host the stream is
+ *    synchronised before returning, with dst on the device the call is
+ *    asynchronous. */
+#define PRSGD_NOALLOC_MAX_M (1 << 20)
+int prsgd_mean_rows_noalloc(const float* d_P, int64_t N, int64_t m, int64_t row_stride,
+                            float* dst, int dst_on_device, void* cuda_stream);
+
 /* The minibatch draw zeta_i^t as an integer: the (i+1)-th output of a
  * SplitMix64 stream keyed by the t-th output of the SplitMix64 stream seeded
  * with `seed`, modulo n_blocks.  Pure host function; the device code evaluates

@@ -31,8 +31,9 @@ EXPORTS = [
     "prsgd_get_params", "prsgd_local_steps", "prsgd_average", "prsgd_get_average", "prsgd_get_losses",
     "prsgd_get_draws", "prsgd_set_lr", "prsgd_set_interval", "prsgd_set_active", "prsgd_get_step",
     "prsgd_set_step", "prsgd_set_option", "prsgd_get_launch_count", "prsgd_get_profile", "prsgd_sync", "prsgd_last_error",
-    "prsgd_average_rows", "prsgd_draw_block",
+    "prsgd_average_rows", "prsgd_draw_block", "prsgd_mean_rows_noalloc",
 ]
+NOALLOC_MAX_M = 1 << 20
 
 
 class ModelSpec(C.Structure):
@@ -81,6 +82,7 @@ def _load() -> C.CDLL:
         "prsgd_last_error": (C.c_char_p, [vp]),
         "prsgd_average_rows": (C.c_int, [vp, i64, i64, i64, vp]),
         "prsgd_draw_block": (u64, [u64, i32, i64, u64]),
+        "prsgd_mean_rows_noalloc": (C.c_int, [vp, i64, i64, i64, vp, C.c_int, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -132,6 +134,22 @@ def prsgd_average_rows(P: torch.Tensor, N: int, m: int, row_stride: Optional[int
     s = stream if stream is not None else torch.cuda.current_stream(P.device)
     with torch.cuda.device(P.device):
         _check(lib.prsgd_average_rows(P.data_ptr(), N, m, m if row_stride is None else row_stride, s.cuda_stream))
+
+
+def prsgd_mean_rows_noalloc(P: torch.Tensor, N: int, m: int, row_stride: int, out, stream=None):
+    """Node average of the rows of a device fp32 tensor into `out` (numpy array, or host / device tensor),
+    staged through the library's fixed device row: nothing is allocated and P is left untouched."""
+    assert P.is_cuda and P.dtype == torch.float32
+    s = stream if stream is not None else torch.cuda.current_stream(P.device)
+    if isinstance(out, np.ndarray):
+        assert out.dtype == np.float32 and out.size >= m and out.flags["C_CONTIGUOUS"]
+        ptr, on_dev = out.ctypes.data, 0
+    else:
+        assert out.dtype == torch.float32 and out.numel() >= m and out.is_contiguous()
+        ptr, on_dev = out.data_ptr(), 1 if out.is_cuda else 0
+    with torch.cuda.device(P.device):
+        _check(lib.prsgd_mean_rows_noalloc(P.data_ptr(), N, m, row_stride, ptr, on_dev, s.cuda_stream))
+    return out
 
 
 def _host_ptr(a: np.ndarray) -> int:

@@ -2,6 +2,7 @@
 // Algorithm 1 and the kernel launches.  See include/prsgd.h for the contract.
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "prsgd_common.cuh"
@@ -635,6 +636,55 @@ int prsgd_average_rows(float* d_P, int64_t N, int64_t m, int64_t row_stride, voi
       d_P, N, m, row_stride, nullptr, nullptr);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return fail(nullptr, PRSGD_ERR_CUDA, std::string("average_rows: ") + cudaGetErrorString(e));
+  return PRSGD_OK;
+}
+
+// ---- allocation-free node average ------------------------------------------------------
+// Staging row for prsgd_mean_rows_noalloc.  In host code this name is only a handle for
+// cudaGetSymbolAddress; the kernel must be given the device address looked up below.
+static __device__ __align__(256) float g_noalloc_row[PRSGD_NOALLOC_MAX_M];
+
+namespace {
+constexpr int kMaxDevices = 64;
+float* g_noalloc_addr[kMaxDevices] = {nullptr};
+std::mutex g_noalloc_mutex;
+}  // namespace
+
+int prsgd_mean_rows_noalloc(const float* d_P, int64_t N, int64_t m, int64_t row_stride, float* dst, int dst_on_device,
+                            void* cuda_stream) {
+  if (!d_P || !dst) return fail(nullptr, PRSGD_ERR_ARG, "d_P / dst is NULL");
+  if (N < 1 || m < 0 || row_stride < m) return fail(nullptr, PRSGD_ERR_ARG, "need N >= 1, m >= 0, row_stride >= m");
+  if (m > PRSGD_NOALLOC_MAX_M)
+    return fail(nullptr, PRSGD_ERR_SIZE, "m exceeds PRSGD_NOALLOC_MAX_M (" + std::to_string(PRSGD_NOALLOC_MAX_M) +
+                                             " floats), the size of the library's fixed staging row");
+  if (!aligned(d_P, 16) || (row_stride % 4) != 0)
+    return fail(nullptr, PRSGD_ERR_ALIGN, "d_P must be 16-byte aligned and row_stride a multiple of 4");
+  if (m == 0) return PRSGD_OK;
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return fail(nullptr, PRSGD_ERR_CUDA, std::string("cudaGetDevice: ") + cudaGetErrorString(e));
+  if (dev < 0 || dev >= kMaxDevices) return fail(nullptr, PRSGD_ERR_ARG, "device ordinal out of range");
+  float* row = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_noalloc_addr[dev]) {                 // once per device, with that device current
+      float* p = nullptr;
+      e = cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_noalloc_row);
+      if (e != cudaSuccess || !p)
+        return fail(nullptr, PRSGD_ERR_CUDA, std::string("cudaGetSymbolAddress: ") + cudaGetErrorString(e));
+      g_noalloc_addr[dev] = p;
+    }
+    row = g_noalloc_addr[dev];
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const int64_t threads = m / 4 + (m & 3);
+  // MODE 1 only reads P; every entry of row[0, m) is written before the copy below reads it
+  average_rows_kernel<1, false><<<grid1d(threads, 256), 256, 0, st>>>(const_cast<float*>(d_P), N, m, row_stride, row, nullptr);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(nullptr, PRSGD_ERR_CUDA, std::string("mean_rows_noalloc: ") + cudaGetErrorString(e));
+  e = cudaMemcpyAsync(dst, row, (size_t)m * 4, dst_on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess && !dst_on_device) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return fail(nullptr, PRSGD_ERR_CUDA, std::string("mean_rows_noalloc copy: ") + cudaGetErrorString(e));
   return PRSGD_OK;
 }
 
