@@ -229,6 +229,7 @@ def main():
     ap.add_argument("--config", default=DEFAULT_WORKLOAD, choices=sorted(synth.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--interval", type=int, default=None, help="override the averaging interval I")
+    ap.add_argument("--workers", type=int, default=None, help="override N (smaller cases for profiler captures)")
     ap.add_argument("--no-sweep", action="store_true", help="skip the averaging-kernel sweep")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle timing")
     args = ap.parse_args()
@@ -237,6 +238,8 @@ def main():
     w = synth.WORKLOADS[args.config]
     if args.interval is not None:
         w = w.with_(I=args.interval)
+    if args.workers is not None:
+        w = w.with_(N=args.workers, name=f"{w.name}-N{args.workers}")
     if args.impl == "reference":
         return run_reference(args, w)
 
