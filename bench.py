@@ -330,6 +330,7 @@ def main():
                 "traffic": None,
                 "avg_launch_us": 1e3 * dom_ms / dom_launches,
                 "algorithmic_bytes_per_launch": bytes_iter[dom] / per_iter_launches,
+                "family_us_per_iteration": {k: round(1e3 * v[0] / (args.steps * max(w.I, 1)), 2) for k, v in prof.items() if v[1]},
                 "share_of_step_time": {k: round(v[0] / sum(x[0] for x in prof.values()), 4) for k, v in prof.items() if v[1]}}
     tflops = flops_per_worker_step(w) * value / world / 1e12
 

@@ -188,17 +188,31 @@ __global__ void __launch_bounds__(kStreamThreads) tc_stream_kernel(const __grid_
     }
     __syncwarp();
 
-    // ---- epilogue: thread <-> output feature m0 + tid, its B accumulators sit in one TMEM lane
+    // ---- epilogue: thread <-> output feature m0 + tid, its B accumulators sit in one TMEM lane.
+    // Work goes in batches of 16 minibatch columns; the ReLU-mask values a batch needs (TC_DX) are
+    // fetched one batch ahead, the first of them before the accumulator is even ready, so that no
+    // global-load latency sits between the accumulator and the stores.
+    const int m = m0 + tid;
+    const bool valid = m < a.M_total;
+    const int batches = a.B / 16;
+    auto mask_fetch = [&](int bi, uint16_t (&mk)[16]) {
+      if (MODE == TC_DX && bi < batches && valid) {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) mk[j] = __ldg(a.mask_src + ((int64_t)n * a.B + bi * 16 + j) * a.ld_out + m);
+      }
+    };
+    uint16_t mk_cur[16], mk_next[16];
+    mask_fetch(0, mk_cur);
+    float bias = 0.f;
+    if (MODE != TC_DX && valid) bias = a.bias[(int64_t)n * a.bias_stride + m];
     const bool acc_ok = __all_sync(0xffffffffu, mbar_wait(acc_bar, 0u, abort_flag, a.status, 0x103));
     tc_fence_after();
     if (acc_ok) {
-      const int m = m0 + tid;
-      const bool valid = m < a.M_total;
-      float bias = 0.f;
-      if (MODE != TC_DX && valid) bias = a.bias[(int64_t)n * a.bias_stride + m];
-      for (int c0 = 0; c0 < a.B; c0 += 16) {
+      for (int bi = 0; bi < batches; ++bi) {
+        const int c0 = bi * 16;
         uint32_t v[16];
         tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
+        mask_fetch(bi + 1, mk_next);
         tmem_ld_wait();
         if (valid) {
 #pragma unroll
@@ -210,9 +224,13 @@ __global__ void __launch_bounds__(kStreamThreads) tc_stream_kernel(const __grid_
             } else if (MODE == TC_FWD_LINEAR) {
               a.out_f32[o] = x + bias;
             } else {
-              a.out_bk[o] = (a.mask_src[o] & 0x7FFFu) != 0 ? f32_to_bf16_rn(x) : (uint16_t)0;
+              a.out_bk[o] = (mk_cur[j] & 0x7FFFu) != 0 ? f32_to_bf16_rn(x) : (uint16_t)0;
             }
           }
+        }
+        if (MODE == TC_DX) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) mk_cur[j] = mk_next[j];
         }
       }
     }
