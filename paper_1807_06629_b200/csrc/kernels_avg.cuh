@@ -24,6 +24,8 @@ __global__ void __launch_bounds__(256) average_rows_kernel(float* __restrict__ P
                                                            int64_t row_stride, float* __restrict__ out,
                                                            uint16_t* __restrict__ shadow) {
   constexpr int U = 8;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");   // no-op unless launched as a programmatic dependent
   const int64_t cols4 = m >> 2;
   const int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   const float fN = (float)N;

@@ -127,8 +127,7 @@ __global__ void __launch_bounds__(kStreamThreads) tc_stream_kernel(const __grid_
   if (tid == 0) {
     for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     mbar_init(acc_bar, 1);
-    // a wait that expired in an earlier CTA or launch turns the rest of the work into a no-op
-    *abort_flag = *(volatile unsigned int*)&a.status->error != 0u ? 1 : 0;
+    *abort_flag = 0;
     fence_mbar_init();
     prefetch_tensormap(&mapW);
     prefetch_tensormap(&mapB);
@@ -137,7 +136,12 @@ __global__ void __launch_bounds__(kStreamThreads) tc_stream_kernel(const __grid_
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  pdl_trigger();
+  pdl_wait();            // everything above overlapped the previous kernel's tail; memory is touched below
   const uint32_t tmem = *tmem_slot;
+  // a wait that expired in an earlier CTA or launch turns the rest of the work into a no-op
+  if (tid == 0) *abort_flag = *(volatile unsigned int*)&a.status->error != 0u ? 1 : 0;
+  __syncthreads();
   const bool is_active = (a.active == nullptr || a.active[n] != 0) && *abort_flag == 0;
 
   if (is_active) {
@@ -292,7 +296,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
       mbar_init(full_ops(s), 1); mbar_init(full_w(s), 1); mbar_init(stage_empty(s), 1);
       mbar_init(acc_full(s), 1); mbar_init(acc_empty(s), 128); mbar_init(tile_ready(s), 128);
     }
-    *abort_flag = *(volatile unsigned int*)&a.status->error != 0u ? 1 : 0;   // an earlier expired wait: no-op
+    *abort_flag = 0;
     fence_mbar_init();
     prefetch_tensormap(&mapDelta); prefetch_tensormap(&mapAct);
     prefetch_tensormap(&mapMaster); prefetch_tensormap(&mapShadow);
@@ -301,7 +305,11 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  pdl_trigger();
+  pdl_wait();            // set-up above overlapped the previous kernel's tail; memory is touched below
   const uint32_t tmem = *tmem_slot;
+  if (tid == 0) *abort_flag = *(volatile unsigned int*)&a.status->error != 0u ? 1 : 0;   // an earlier expired wait: no-op
+  __syncthreads();
   const int total_items = *abort_flag != 0 ? 0 : items_all;
 
   // Every role walks the same sequence of (tile, worker) items; `it` counts the items it has handled.
@@ -487,30 +495,19 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
   if (warp == 1) tmem_dealloc(tmem, 256u);
 }
 
-// b_l <- b_l - gamma * sum_b dZ_l[b, :], optionally followed by the node average (fixed order).
-template <bool FUSE>
+// b_l <- b_l - gamma * sum_b dZ_l[b, :] (the bias part of Eq. parallel-sgd-x-update), one thread per (worker, j).
 __global__ void __launch_bounds__(128) bias_update_kernel(float* params, int64_t m_pad, int64_t b_off, int d_out,
-                                                          const uint16_t* delta_bk, int ld, int B, int N, float gamma,
+                                                          const uint16_t* delta_bk, int ld, int B, float gamma,
                                                           const uint8_t* active) {
+  ptx::pdl_trigger();
+  ptx::pdl_wait();
   const int j = blockIdx.x * blockDim.x + threadIdx.x;
-  if (j >= d_out) return;
-  const int n_begin = FUSE ? 0 : (int)blockIdx.y, n_end = FUSE ? N : n_begin + 1;
-  float sum = 0.f;
-  for (int n = n_begin; n < n_end; ++n) {
-    float* bp = params + (int64_t)n * m_pad + b_off + j;
-    float x = *bp;
-    if (active == nullptr || active[n] != 0) {
-      float g = 0.f;
-      for (int b = 0; b < B; ++b) g += __uint_as_float((uint32_t)delta_bk[((int64_t)n * B + b) * ld + j] << 16);
-      x = fmaf(-gamma, g, x);
-    }
-    if (FUSE) sum += x;
-    else *bp = x;
-  }
-  if (FUSE) {
-    const float y = __fdiv_rn(sum, (float)N);
-    for (int n = 0; n < N; ++n) params[(int64_t)n * m_pad + b_off + j] = y;
-  }
+  const int n = blockIdx.y;
+  if (j >= d_out || (active != nullptr && active[n] == 0)) return;
+  float g = 0.f;
+  for (int b = 0; b < B; ++b) g += __uint_as_float((uint32_t)__ldg(delta_bk + ((int64_t)n * B + b) * ld + j) << 16);
+  float* bp = params + (int64_t)n * m_pad + b_off + j;
+  *bp = fmaf(-gamma, g, *bp);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -592,9 +589,9 @@ inline void tc_launch_forward(prsgd_ctx* c, int l, const DrawArgs& dr, const uin
   dim3 grid((ly.d_out + 127) / 128, c->N);
   const size_t smem = stream_smem_bytes(c->B, a.stages);
   if (l < c->L)
-    tc_stream_kernel<TC_FWD_RELU><<<grid, kStreamThreads, smem, c->stream>>>(st->layer[l - 1].shadow_k, st->layer[l - 1].act_in, a);
+    launch_pdl(tc_stream_kernel<TC_FWD_RELU>, grid, kStreamThreads, smem, c->stream, st->layer[l - 1].shadow_k, st->layer[l - 1].act_in, a);
   else
-    tc_stream_kernel<TC_FWD_LINEAR><<<grid, kStreamThreads, smem, c->stream>>>(st->layer[l - 1].shadow_k, st->layer[l - 1].act_in, a);
+    launch_pdl(tc_stream_kernel<TC_FWD_LINEAR>, grid, kStreamThreads, smem, c->stream, st->layer[l - 1].shadow_k, st->layer[l - 1].act_in, a);
 }
 
 // dZ_{l-1} from dZ_l through W_l (l >= 2)
@@ -609,7 +606,7 @@ inline void tc_launch_dx(prsgd_ctx* c, int l, const DrawArgs& dr, const uint8_t*
   a.active = active; a.status = c->status;
   dim3 grid((ly.d_in + 127) / 128, c->N);
   const size_t smem = stream_smem_bytes(c->B, a.stages);
-  tc_stream_kernel<TC_DX><<<grid, kStreamThreads, smem, c->stream>>>(st->layer[l - 1].shadow_mn, st->layer[l - 1].delta_out, a);
+  launch_pdl(tc_stream_kernel<TC_DX>, grid, kStreamThreads, smem, c->stream, st->layer[l - 1].shadow_mn, st->layer[l - 1].delta_out, a);
 }
 
 inline void tc_launch_update(prsgd_ctx* c, int l, const DrawArgs& dr, const uint8_t* active, bool fuse) {
@@ -622,20 +619,25 @@ inline void tc_launch_update(prsgd_ctx* c, int l, const DrawArgs& dr, const uint
   const int grid = items < st->num_sms ? items : st->num_sms;
   const TcLayerMaps& mp = st->layer[l - 1];
   if (fuse)
-    tc_update_kernel<true><<<grid, kUpdThreads, kUpdSmem, c->stream>>>(mp.delta_out, mp.act_in, mp.master, mp.shadow_k, a);
+    launch_pdl(tc_update_kernel<true>, dim3(grid), kUpdThreads, kUpdSmem, c->stream, mp.delta_out, mp.act_in, mp.master, mp.shadow_k, a);
   else
-    tc_update_kernel<false><<<grid, kUpdThreads, kUpdSmem, c->stream>>>(mp.delta_out, mp.act_in, mp.master, mp.shadow_k, a);
+    launch_pdl(tc_update_kernel<false>, dim3(grid), kUpdThreads, kUpdSmem, c->stream, mp.delta_out, mp.act_in, mp.master, mp.shadow_k, a);
 }
 
-inline void tc_launch_bias(prsgd_ctx* c, int l, const uint8_t* active, bool fuse) {
+// Bias step of layer l; on an averaging iteration it is followed by the node average of the bias
+// segment alone (same arithmetic as the stand-alone averaging kernel, so the bits agree).
+inline void tc_launch_bias(prsgd_ctx* c, int l, const uint8_t* active) {
   const Layer& ly = c->layer[l - 1];
-  dim3 grid((ly.d_out + 127) / 128, fuse ? 1 : c->N);
-  if (fuse)
-    bias_update_kernel<true><<<grid, 128, 0, c->stream>>>(c->params, c->m_pad, ly.b_off, ly.d_out, c->buf.delta_bk[l],
-                                                         c->buf.ld[l], c->B, c->N, c->gamma, active);
-  else
-    bias_update_kernel<false><<<grid, 128, 0, c->stream>>>(c->params, c->m_pad, ly.b_off, ly.d_out, c->buf.delta_bk[l],
-                                                          c->buf.ld[l], c->B, c->N, c->gamma, active);
+  dim3 grid((ly.d_out + 127) / 128, c->N);
+  launch_pdl(bias_update_kernel, grid, dim3(128), 0, c->stream, c->params, c->m_pad, ly.b_off, ly.d_out,
+             (const uint16_t*)c->buf.delta_bk[l], c->buf.ld[l], c->B, c->gamma, active);
+}
+
+inline void tc_launch_bias_average(prsgd_ctx* c, int l) {
+  const Layer& ly = c->layer[l - 1];
+  const int64_t threads = ly.d_out / 4 + (ly.d_out & 3);
+  launch_pdl(average_rows_kernel<0, false>, dim3((unsigned)((threads + 255) / 256)), dim3(256), 0, c->stream,
+             c->params + ly.b_off, (int64_t)c->N, (int64_t)ly.d_out, c->m_pad, (float*)nullptr, (uint16_t*)nullptr);
 }
 
 }  // namespace prsgd

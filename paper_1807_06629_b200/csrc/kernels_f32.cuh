@@ -227,6 +227,8 @@ __device__ __forceinline__ uint16_t f32_to_bf16_rn(float f) {
 
 __global__ void __launch_bounds__(256) softmax_ce_kernel(const SoftmaxArgs a) {
   __shared__ float row_loss[256];
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");   // no-op unless launched as a programmatic dependent
   const int n = blockIdx.x;
   if (a.active != nullptr && a.active[n] == 0) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;

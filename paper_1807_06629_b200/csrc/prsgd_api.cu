@@ -297,7 +297,7 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging) {
     a.Y = c->Y; a.P = c->P; a.B = c->B; a.C = c->dims[L]; a.draw = dr;
     a.losses = c->losses; a.draws = c->draws; a.active = act_mask;
     prof_begin(c, PRSGD_KERNEL_SOFTMAX);
-    softmax_ce_kernel<<<N, 256, 0, c->stream>>>(a);
+    launch_pdl(softmax_ce_kernel, dim3(N), dim3(256), 0, c->stream, a);
     LAUNCH_CHECK(c);
   }
   for (int l = L; l >= 1; --l) {          // dX_l reads W_l before the update of layer l overwrites it
@@ -310,8 +310,13 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging) {
     tc_launch_update(c, l, dr, act_mask, fuse);
     LAUNCH_CHECK(c);
     prof_begin(c, PRSGD_KERNEL_MISC);
-    tc_launch_bias(c, l, act_mask, fuse);
+    tc_launch_bias(c, l, act_mask);
     LAUNCH_CHECK(c);
+    if (fuse) {
+      prof_begin(c, PRSGD_KERNEL_MISC);
+      tc_launch_bias_average(c, l);
+      LAUNCH_CHECK(c);
+    }
   }
   return PRSGD_OK;
 }

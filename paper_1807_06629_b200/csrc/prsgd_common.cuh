@@ -40,6 +40,20 @@ struct DeviceStatus {
   unsigned int pad[62];
 };
 
+// Launch with the programmatic-stream-serialization attribute: the kernel may start while the
+// previous kernel of the stream drains; it must call griddepcontrol.wait before touching memory.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                              Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 constexpr int64_t kSegAlign = 32;  // every segment of a row starts at a multiple of 32 elements
 
 inline int64_t round_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
