@@ -230,6 +230,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--interval", type=int, default=None, help="override the averaging interval I")
     ap.add_argument("--workers", type=int, default=None, help="override N (smaller cases for profiler captures)")
+    ap.add_argument("--update-tile", type=int, default=None, help="tile width of the update kernel (64 or 128)")
     ap.add_argument("--no-sweep", action="store_true", help="skip the averaging-kernel sweep")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle timing")
     args = ap.parse_args()
@@ -273,6 +274,8 @@ def main():
     p = binding.PRSGD(w.N, w.dims, w.B, w.gamma, w.I, w.precision, w.pool_samples, w.seed, device=dev)
     p.bind_data(hX.to(dev), hY.to(dev))
     p.set_params(x0)
+    if args.update_tile is not None:
+        p.set_option(binding.OPT_UPDATE_TILE, args.update_tile)
     working_set = p.params.numel() * 4 + (p.shadow.numel() * 2 if p.shadow is not None else 0)
     need_flush = working_set <= 2 * L2_BYTES
     flush = torch.empty(3 * L2_BYTES // 4, dtype=torch.float32, device=dev) if need_flush else None

@@ -179,6 +179,10 @@ int prsgd_set_step(prsgd_ctx* ctx, int64_t t);
  * pair of CUDA events on the context's stream; read the sums with
  * prsgd_get_profile.  Costs two event records per launch. */
 #define PRSGD_OPT_PROFILE 2
+/* PRSGD_OPT_UPDATE_TILE (default 0): column width of the 128-row tile the tensor-core update
+ * kernel works on: 64 (four pipeline stages per SM), 128 (two), or 0 = chosen per launch from
+ * the layer size.  A tuning knob only: every setting produces the same bits. */
+#define PRSGD_OPT_UPDATE_TILE 3
 int prsgd_set_option(prsgd_ctx* ctx, int32_t option, int64_t value);
 
 /* Kernel families of the hot path, for prsgd_get_profile. */

@@ -258,33 +258,47 @@ struct UpdateArgs {
 };
 
 constexpr int kUpdThreads = 224;          // warp 0 loader, 1 MMA, 2 storer, 3..6 epilogue
-constexpr uint32_t kMasterTile = 65536;   // 128 x 128 fp32, four 128 x 32 boxes
-constexpr uint32_t kOpsRegion = 32768;    // operands, later the bf16 output tile (two 128 x 64 boxes)
-constexpr uint32_t kUpdStage = kMasterTile + kOpsRegion;
-constexpr size_t kUpdSmem = 2 * kUpdStage + 1024 + 256;
 
-template <bool FUSE>
+// One pipeline stage of the update kernel for a 128 x TN tile: the fp32 master tile (TN/32 boxes of
+// 128 x 32) followed by a region that first holds the operands (two dZ boxes and TN/64 activation
+// boxes of {64, B}) and later, once the MMA has consumed them, the bf16 output tile (TN/64 boxes
+// of 128 x 64).  TN = 64 gives four stages, TN = 128 two.
+template <int TN> struct UpdCfg {
+  static constexpr int kStages = TN == 64 ? 4 : 2;
+  static constexpr uint32_t kMaster = 128u * TN * 4u;
+  static constexpr uint32_t kOut = 128u * TN * 2u;
+  __host__ __device__ static uint32_t ops_bytes(int B) { return (uint32_t)(2 + TN / 64) * (uint32_t)B * 128u; }
+  __host__ __device__ static uint32_t region(int B) { return ops_bytes(B) > kOut ? ops_bytes(B) : kOut; }
+  __host__ __device__ static uint32_t stage(int B) { return kMaster + region(B); }
+  static size_t smem(int B) { return (size_t)kStages * stage(B) + 1024 + 256; }
+};
+
+template <bool FUSE, int TN>
 __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_constant__ CUtensorMap mapDelta,
                                                                    const __grid_constant__ CUtensorMap mapAct,
                                                                    const __grid_constant__ CUtensorMap mapMaster,
                                                                    const __grid_constant__ CUtensorMap mapShadow,
                                                                    const UpdateArgs a) {
   using namespace ptx;
+  using Cfg = UpdCfg<TN>;
+  constexpr int S = Cfg::kStages;
+  constexpr int NB32 = TN / 32, NB64 = TN / 64;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* gen = smem_raw + (base - raw);
-  auto master_u32 = [&](int s) { return base + (uint32_t)s * kUpdStage; };
-  auto ops_u32 = [&](int s) { return base + (uint32_t)s * kUpdStage + kMasterTile; };
-  const uint32_t bar0 = base + 2u * kUpdStage;
+  const uint32_t stage_bytes = Cfg::stage(a.B);
+  auto master_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes; };
+  auto ops_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes + Cfg::kMaster; };
+  const uint32_t bar0 = base + (uint32_t)S * stage_bytes;
   auto full_ops = [&](int s) { return bar0 + 8u * s; };
-  auto full_w = [&](int s) { return bar0 + 16u + 8u * s; };
-  auto stage_empty = [&](int s) { return bar0 + 32u + 8u * s; };
-  auto acc_full = [&](int s) { return bar0 + 48u + 8u * s; };
-  auto acc_empty = [&](int s) { return bar0 + 64u + 8u * s; };
-  auto tile_ready = [&](int s) { return bar0 + 80u + 8u * s; };
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen + 2 * kUpdStage + 96);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + 2 * kUpdStage + 100);
+  auto full_w = [&](int s) { return bar0 + 32u + 8u * s; };
+  auto stage_empty = [&](int s) { return bar0 + 64u + 8u * s; };
+  auto acc_full = [&](int s) { return bar0 + 96u + 8u * s; };
+  auto acc_empty = [&](int s) { return bar0 + 128u + 8u * s; };
+  auto tile_ready = [&](int s) { return bar0 + 160u + 8u * s; };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen + (size_t)S * stage_bytes + 192);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + (size_t)S * stage_bytes + 196);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t op_box = (uint32_t)a.B * 128u;       // one {64, B} box
@@ -292,7 +306,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
   const int items_all = FUSE ? tiles : tiles * a.N;    // FUSE: a CTA owns a tile and walks all workers
 
   if (tid == 0) {
-    for (int s = 0; s < 2; ++s) {
+    for (int s = 0; s < S; ++s) {
       mbar_init(full_ops(s), 1); mbar_init(full_w(s), 1); mbar_init(stage_empty(s), 1);
       mbar_init(acc_full(s), 1); mbar_init(acc_empty(s), 128); mbar_init(tile_ready(s), 128);
     }
@@ -312,7 +326,8 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
   __syncthreads();
   const int total_items = *abort_flag != 0 ? 0 : items_all;
 
-  // Every role walks the same sequence of (tile, worker) items; `it` counts the items it has handled.
+  // Every role walks the same sequence of (tile, worker) items; `it` counts the items it has handled,
+  // item `it` lives in stage it % S and TMEM columns (it % S) * TN.
   auto item_active = [&](int n) { return FUSE || a.active == nullptr || a.active[n] != 0; };
 
   if (warp == 0 && lane == 0) {
@@ -322,34 +337,34 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
     for (int w = blockIdx.x; w < total_items && ok; w += gridDim.x) {
       const int tile = FUSE ? w : w % tiles;
       const int n_begin = FUSE ? 0 : w / tiles, n_end = FUSE ? a.N : n_begin + 1;
-      const int m0 = (tile / a.tiles_n) * 128, n0 = (tile % a.tiles_n) * 128;
+      const int m0 = (tile / a.tiles_n) * 128, n0 = (tile % a.tiles_n) * TN;
       for (int n = n_begin; n < n_end; ++n) {
         if (!item_active(n)) continue;
-        const int s = it & 1;
-        const uint32_t ph = (it >> 1) & 1u;
+        const int s = it % S;
+        const uint32_t ph = (it / S) & 1u;
         ok = mbar_wait(stage_empty(s), ph ^ 1u, abort_flag, a.status, 0x201);
         if (!ok) break;
         const int row0 = a.pool ? (int)draw_block(a.draw.seed, n, a.draw.t, a.draw.n_blocks) * a.B : 0;
         const uint32_t ops = ops_u32(s);
-        mbar_expect_tx(full_ops(s), 4u * op_box);
+        mbar_expect_tx(full_ops(s), (2u + NB64) * op_box);
         tma_load_3d(ops, &mapDelta, full_ops(s), m0, 0, n);
         tma_load_3d(ops + op_box, &mapDelta, full_ops(s), m0 + 64, 0, n);
-        tma_load_3d(ops + 2u * op_box, &mapAct, full_ops(s), n0, row0, n);
-        tma_load_3d(ops + 3u * op_box, &mapAct, full_ops(s), n0 + 64, row0, n);
-        mbar_expect_tx(full_w(s), kMasterTile);
 #pragma unroll
-        for (int q = 0; q < 4; ++q) tma_load_3d(master_u32(s) + q * 16384u, &mapMaster, full_w(s), n0 + 32 * q, m0, n);
+        for (int h = 0; h < NB64; ++h) tma_load_3d(ops + (2u + h) * op_box, &mapAct, full_ops(s), n0 + 64 * h, row0, n);
+        mbar_expect_tx(full_w(s), Cfg::kMaster);
+#pragma unroll
+        for (int q = 0; q < NB32; ++q) tma_load_3d(master_u32(s) + q * 16384u, &mapMaster, full_w(s), n0 + 32 * q, m0, n);
         ++it;
       }
     }
     if (*abort_flag && it > 0) {   // let the copies already in flight land before the CTA goes away
       const uint64_t t0 = globaltimer_ns();
       const uint32_t last = it - 1;
-      while (!mbar_try_wait(full_w(last & 1), (last >> 1) & 1u) && globaltimer_ns() - t0 < 100000000ull) {}
+      while (!mbar_try_wait(full_w(last % S), (last / S) & 1u) && globaltimer_ns() - t0 < 100000000ull) {}
     }
   } else if (warp == 1 && lane == 0) {
     // ---------------- MMA issuer
-    const uint32_t idesc = idesc_bf16(128, 128, 1, 1);
+    const uint32_t idesc = idesc_bf16(128, TN, 1, 1);
     const int ksteps = a.B / 16;
     uint32_t it = 0;
     bool ok = true;
@@ -357,15 +372,15 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
       const int n_begin = FUSE ? 0 : w / tiles, n_end = FUSE ? a.N : n_begin + 1;
       for (int n = n_begin; n < n_end; ++n) {
         if (!item_active(n)) continue;
-        const int s = it & 1;
-        const uint32_t ph = (it >> 1) & 1u;
+        const int s = it % S;
+        const uint32_t ph = (it / S) & 1u;
         ok = mbar_wait(acc_empty(s), ph ^ 1u, abort_flag, a.status, 0x202) &&
              mbar_wait(full_ops(s), ph, abort_flag, a.status, 0x203);
         if (!ok) break;
         tc_fence_after();
         const uint32_t sa = ops_u32(s), sb = sa + 2u * op_box;
         for (int k = 0; k < ksteps; ++k)
-          mma_bf16(tmem + (uint32_t)s * 128u, smem_desc_sw128(sa + k * 2048u, op_box, 1024u),
+          mma_bf16(tmem + (uint32_t)(s * TN), smem_desc_sw128(sa + k * 2048u, op_box, 1024u),
                    smem_desc_sw128(sb + k * 2048u, op_box, 1024u), idesc, k != 0 ? 1u : 0u);
         mma_commit(acc_full(s));
         ++it;
@@ -375,35 +390,33 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
     // ---------------- storer: TMA stores of finished tiles, then hands the stage back to the loader
     uint32_t it = 0, tile_it = 0;
     bool ok = true;
+    auto store_tile = [&](int s, int m0, int n0, int n) {
+#pragma unroll
+      for (int q = 0; q < NB32; ++q) tma_store_3d(&mapMaster, master_u32(s) + q * 16384u, n0 + 32 * q, m0, n);
+#pragma unroll
+      for (int h = 0; h < NB64; ++h) tma_store_3d(&mapShadow, ops_u32(s) + h * 16384u, n0 + 64 * h, m0, n);
+    };
     for (int w = blockIdx.x; w < total_items && ok; w += gridDim.x) {
       const int tile = FUSE ? w : w % tiles;
-      const int m0 = (tile / a.tiles_n) * 128, n0 = (tile % a.tiles_n) * 128;
+      const int m0 = (tile / a.tiles_n) * 128, n0 = (tile % a.tiles_n) * TN;
       if (!FUSE) {
         const int n = w / tiles;
         if (!item_active(n)) continue;
-        const int s = it & 1;
-        const uint32_t ph = (it >> 1) & 1u;
+        const int s = it % S;
+        const uint32_t ph = (it / S) & 1u;
         ok = mbar_wait(tile_ready(s), ph, abort_flag, a.status, 0x204);
         if (!ok) break;
-#pragma unroll
-        for (int q = 0; q < 4; ++q) tma_store_3d(&mapMaster, master_u32(s) + q * 16384u, n0 + 32 * q, m0, n);
-        tma_store_3d(&mapShadow, ops_u32(s), n0, m0, n);
-        tma_store_3d(&mapShadow, ops_u32(s) + 16384u, n0 + 64, m0, n);
+        store_tile(s, m0, n0, n);
         tma_commit_group();
         tma_wait_group_read0();
         mbar_arrive(stage_empty(s));
         ++it;
       } else {
         it += (uint32_t)a.N;
-        const int s = (it - 1) & 1;                       // stage of the tile's last worker
+        const int s = (it - 1) % S;                       // stage of the tile's last worker
         ok = mbar_wait(tile_ready(0), tile_it & 1u, abort_flag, a.status, 0x205);
         if (!ok) break;
-        for (int n = 0; n < a.N; ++n) {
-#pragma unroll
-          for (int q = 0; q < 4; ++q) tma_store_3d(&mapMaster, master_u32(s) + q * 16384u, n0 + 32 * q, m0, n);
-          tma_store_3d(&mapShadow, ops_u32(s), n0, m0, n);
-          tma_store_3d(&mapShadow, ops_u32(s) + 16384u, n0 + 64, m0, n);
-        }
+        for (int n = 0; n < a.N; ++n) store_tile(s, m0, n0, n);
         tma_commit_group();
         tma_wait_group_read0();
         mbar_arrive(stage_empty(s));
@@ -420,32 +433,31 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
     const uint32_t sw = (uint32_t)(r & 7);
     const int etid = tid - 96;                            // 0..127 among the epilogue threads
     const float fN = (float)a.N;
+    constexpr int NSUM = FUSE ? TN : 1;
     uint32_t it = 0;
     bool ok = true;
     for (int w = blockIdx.x; w < total_items && ok; w += gridDim.x) {
       const int n_begin = FUSE ? 0 : w / tiles, n_end = FUSE ? a.N : n_begin + 1;
-      float sum[FUSE ? 128 : 1];
-      if (FUSE) {
+      float sum[NSUM];
 #pragma unroll
-        for (int i = 0; i < 128; ++i) sum[FUSE ? i : 0] = 0.f;
-      }
+      for (int i = 0; i < NSUM; ++i) sum[i] = 0.f;
       for (int n = n_begin; n < n_end; ++n) {
         if (!item_active(n)) continue;
         const bool upd = a.active == nullptr || a.active[n] != 0;
-        const int s = it & 1;
-        const uint32_t ph = (it >> 1) & 1u;
+        const int s = it % S;
+        const uint32_t ph = (it / S) & 1u;
         ok = mbar_wait(full_w(s), ph, abort_flag, a.status, 0x206) &&
              mbar_wait(acc_full(s), ph, abort_flag, a.status, 0x207);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
-        uint8_t* mst = gen + (size_t)s * kUpdStage;
-        uint8_t* stg = mst + kMasterTile;
+        uint8_t* mst = gen + (size_t)s * stage_bytes;
+        uint8_t* stg = mst + Cfg::kMaster;
         const bool last = FUSE && n == a.N - 1;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < NB32; ++c) {
           uint32_t v[32];
-          tmem_ld32(tmem + lane_off + (uint32_t)s * 128u + (uint32_t)c * 32u, v);
+          tmem_ld32(tmem + lane_off + (uint32_t)(s * TN + c * 32), v);
           tmem_ld_wait();
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
@@ -458,11 +470,12 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
               x.w = fmaf(-a.gamma, __uint_as_float(v[4 * j + 3]), x.w);
             }
             if (FUSE) {
-              float* sp = &sum[FUSE ? c * 32 + 4 * j : 0];
-              sp[0] += x.x; sp[FUSE ? 1 : 0] += x.y; sp[FUSE ? 2 : 0] += x.z; sp[FUSE ? 3 : 0] += x.w;
+              constexpr int F = FUSE ? 1 : 0;
+              float* sp = &sum[F * (c * 32 + 4 * j)];
+              sp[0] += x.x; sp[F * 1] += x.y; sp[F * 2] += x.z; sp[F * 3] += x.w;
               if (last) {
-                x.x = __fdiv_rn(sp[0], fN); x.y = __fdiv_rn(sp[FUSE ? 1 : 0], fN);
-                x.z = __fdiv_rn(sp[FUSE ? 2 : 0], fN); x.w = __fdiv_rn(sp[FUSE ? 3 : 0], fN);
+                x.x = __fdiv_rn(sp[0], fN); x.y = __fdiv_rn(sp[F * 1], fN);
+                x.z = __fdiv_rn(sp[F * 2], fN); x.w = __fdiv_rn(sp[F * 3], fN);
               }
             }
             if (!FUSE || last) {
@@ -543,8 +556,10 @@ inline int tc_create(prsgd_ctx* c, std::string* err) {
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_stream_kernel<TC_FWD_RELU>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_stream_kernel<TC_FWD_LINEAR>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_stream_kernel<TC_DX>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kUpdSmem);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kUpdSmem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<false, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<64>::smem(c->B));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<true, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<64>::smem(c->B));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<false, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<128>::smem(c->B));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<true, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<128>::smem(c->B));
   if (e != cudaSuccess) {
     *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e);
     delete st;
@@ -609,19 +624,38 @@ inline void tc_launch_dx(prsgd_ctx* c, int l, const DrawArgs& dr, const uint8_t*
   launch_pdl(tc_stream_kernel<TC_DX>, grid, kStreamThreads, smem, c->stream, st->layer[l - 1].shadow_mn, st->layer[l - 1].delta_out, a);
 }
 
-inline void tc_launch_update(prsgd_ctx* c, int l, const DrawArgs& dr, const uint8_t* active, bool fuse) {
+template <int TN>
+inline void tc_launch_update_tn(prsgd_ctx* c, int l, const DrawArgs& dr, const uint8_t* active, bool fuse) {
   TcState* st = static_cast<TcState*>(c->tc);
   const Layer& ly = c->layer[l - 1];
   UpdateArgs a{};
-  a.B = c->B; a.N = c->N; a.tiles_m = (ly.d_out + 127) / 128; a.tiles_n = (ly.d_in + 127) / 128;
+  a.B = c->B; a.N = c->N; a.tiles_m = (ly.d_out + 127) / 128; a.tiles_n = (ly.d_in + TN - 1) / TN;
   a.gamma = c->gamma; a.pool = l == 1; a.draw = dr; a.active = active; a.status = c->status;
   const int items = a.tiles_m * a.tiles_n * (fuse ? 1 : c->N);
   const int grid = items < st->num_sms ? items : st->num_sms;
   const TcLayerMaps& mp = st->layer[l - 1];
+  const size_t smem = UpdCfg<TN>::smem(c->B);
   if (fuse)
-    launch_pdl(tc_update_kernel<true>, dim3(grid), kUpdThreads, kUpdSmem, c->stream, mp.delta_out, mp.act_in, mp.master, mp.shadow_k, a);
+    launch_pdl(tc_update_kernel<true, TN>, dim3(grid), kUpdThreads, smem, c->stream, mp.delta_out, mp.act_in, mp.master, mp.shadow_k, a);
   else
-    launch_pdl(tc_update_kernel<false>, dim3(grid), kUpdThreads, kUpdSmem, c->stream, mp.delta_out, mp.act_in, mp.master, mp.shadow_k, a);
+    launch_pdl(tc_update_kernel<false, TN>, dim3(grid), kUpdThreads, smem, c->stream, mp.delta_out, mp.act_in, mp.master, mp.shadow_k, a);
+}
+
+// Tile width: forced by PRSGD_OPT_UPDATE_TILE, else chosen per launch.  Wide tiles need fewer TMA
+// operations per byte and win when every SM has a long queue of them; narrow tiles give four
+// pipeline stages and twice as many work items, which wins on small stores and on the fused form,
+// where a launch has only one item per tile.
+inline void tc_launch_update(prsgd_ctx* c, int l, const DrawArgs& dr, const uint8_t* active, bool fuse) {
+  const TcState* st = static_cast<const TcState*>(c->tc);
+  const Layer& ly = c->layer[l - 1];
+  int tile = c->upd_tile;
+  if (tile == 0) {
+    const int64_t tiles128 = (int64_t)((ly.d_out + 127) / 128) * ((ly.d_in + 127) / 128);
+    if (fuse) tile = 2 * tiles128 >= 3 * (int64_t)st->num_sms ? 128 : 64;
+    else tile = (c->B <= 32 && tiles128 * c->N >= 32 * (int64_t)st->num_sms) ? 128 : 64;
+  }
+  if (tile == 128) tc_launch_update_tn<128>(c, l, dr, active, fuse);
+  else tc_launch_update_tn<64>(c, l, dr, active, fuse);
 }
 
 // Bias step of layer l; on an averaging iteration it is followed by the node average of the bias

@@ -595,6 +595,11 @@ int prsgd_set_option(prsgd_ctx* c, int32_t option, int64_t value) {
   if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
   if (option == PRSGD_OPT_FUSED_AVERAGE) { c->fused_average = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_PROFILE) { c->profile = value != 0; return PRSGD_OK; }
+  if (option == PRSGD_OPT_UPDATE_TILE) {
+    if (value != 0 && value != 64 && value != 128) return fail(c, PRSGD_ERR_ARG, "update tile width must be 0, 64 or 128");
+    c->upd_tile = (int)value;
+    return PRSGD_OK;
+  }
   return fail(c, PRSGD_ERR_ARG, "unknown option");
 }
 

@@ -88,6 +88,7 @@ struct prsgd_ctx {
   int I = 0;
   int64_t t = 0;
   int fused_average = 1;
+  int upd_tile = 0;              // column width of the update kernel's tile: 0 = chosen per launch, 64 or 128
   int64_t launches = 0;
   int64_t m = 0, m_pad = 0;
   prsgd::Layer layer[PRSGD_MAX_LAYERS];

@@ -114,12 +114,14 @@ def test_fused_average_equals_update_then_average_bit_for_bit(torch_cuda):
     for w in (SMALL[1], SMALL[4], _w("tc-n5", 5, (64, 128, 10), 32, I=3)):
         X, Y, x0 = make_inputs(w)
         outs = []
-        for fused in (1, 0):
+        for fused, tile in ((1, 0), (0, 0), (1, 64), (0, 64), (1, 128), (0, 128)):   # tile width changes no bit either
             p = make_ctx(w, X, Y, x0)
             p.set_option(binding.OPT_FUSED_AVERAGE, fused)
+            p.set_option(binding.OPT_UPDATE_TILE, tile)
             p.local_steps(2 * w.I + 1)
             outs.append(p.get_params_stacked())
-        assert np.array_equal(outs[0], outs[1])
+        for o in outs[1:]:
+            assert np.array_equal(outs[0], o)
 
 
 def test_shadow_tracks_master_and_padding_stays_zero(torch_cuda):
