@@ -201,20 +201,19 @@ __global__ void __launch_bounds__(256) gemm_f32_kernel(const GemmF32Args g) {
   }
 }
 
-// delta_L = (softmax(z_L) - onehot(y)) / B and the mean minibatch loss.
-// One block per worker; warp w handles rows w, w + 8, ...
+// delta_L = (softmax(z_L) - onehot(y)) / B and the per-sample losses.
+// Grid (N, ceil(B / 8)), 256 threads: one warp per minibatch row.
 struct SoftmaxArgs {
   const float* logits;   // [N][B][ldz]
   float* delta;          // [N][B][ldz]  (fp32), may be nullptr
   uint16_t* delta_bk;    // bf16 [N][B][ld_bf] or nullptr
-  uint16_t* delta_kb;    // bf16 [N][ld_bf][B] or nullptr
   int ld_bf;
   int ldz;
   const int32_t* Y;      // [N][P]
   int64_t P;
   int B, C;
   DrawArgs draw;
-  float* losses;         // [N]
+  float* row_losses;     // [N][B]: logsumexp(z_b) - z_b[y_b]; the caller averages them in row order
   int32_t* draws;        // [N]
   const uint8_t* active;
 };
@@ -226,42 +225,33 @@ __device__ __forceinline__ uint16_t f32_to_bf16_rn(float f) {
 }
 
 __global__ void __launch_bounds__(256) softmax_ce_kernel(const SoftmaxArgs a) {
-  __shared__ float row_loss[256];
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");   // no-op unless launched as a programmatic dependent
   const int n = blockIdx.x;
   if (a.active != nullptr && a.active[n] == 0) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int b = blockIdx.y * 8 + warp;
   const uint32_t blk = draw_block(a.draw.seed, n, a.draw.t, a.draw.n_blocks);
-  if (threadIdx.x == 0) a.draws[n] = (int32_t)blk;
-  const int32_t* y = a.Y + (int64_t)n * a.P + (int64_t)blk * a.B;
+  if (blockIdx.y == 0 && threadIdx.x == 0) a.draws[n] = (int32_t)blk;
+  if (b >= a.B) return;
   const float invB = 1.f / (float)a.B;
-  for (int b = warp; b < a.B; b += 8) {
-    const float* z = a.logits + ((int64_t)n * a.B + b) * a.ldz;
-    float mx = -INFINITY;
-    for (int c = lane; c < a.C; c += 32) mx = fmaxf(mx, z[c]);
+  const float* z = a.logits + ((int64_t)n * a.B + b) * a.ldz;
+  float mx = -INFINITY;
+  for (int c = lane; c < a.C; c += 32) mx = fmaxf(mx, z[c]);
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    float s = 0.f;
-    for (int c = lane; c < a.C; c += 32) s += expf(z[c] - mx);
+  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  float s = 0.f;
+  for (int c = lane; c < a.C; c += 32) s += expf(z[c] - mx);
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-    const float lse = mx + logf(s);
-    const int label = y[b];
-    for (int c = lane; c < a.C; c += 32) {
-      float d = (expf(z[c] - lse) - (c == label ? 1.f : 0.f)) * invB;
-      if (a.delta) a.delta[((int64_t)n * a.B + b) * a.ldz + c] = d;
-      if (a.delta_bk) a.delta_bk[((int64_t)n * a.B + b) * a.ld_bf + c] = f32_to_bf16_rn(d);
-      if (a.delta_kb) a.delta_kb[((int64_t)n * a.ld_bf + c) * a.B + b] = f32_to_bf16_rn(d);
-    }
-    if (lane == 0) row_loss[b] = lse - z[label];
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+  const float lse = mx + logf(s);
+  const int label = a.Y[(int64_t)n * a.P + (int64_t)blk * a.B + b];
+  for (int c = lane; c < a.C; c += 32) {
+    float d = (expf(z[c] - lse) - (c == label ? 1.f : 0.f)) * invB;
+    if (a.delta) a.delta[((int64_t)n * a.B + b) * a.ldz + c] = d;
+    if (a.delta_bk) a.delta_bk[((int64_t)n * a.B + b) * a.ld_bf + c] = f32_to_bf16_rn(d);
   }
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    float s = 0.f;
-    for (int b = 0; b < a.B; ++b) s += row_loss[b];
-    a.losses[n] = s * invB;
-  }
+  if (lane == 0) a.row_losses[(int64_t)n * a.B + b] = lse - z[label];
 }
 
 }  // namespace prsgd

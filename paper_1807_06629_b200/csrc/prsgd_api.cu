@@ -111,7 +111,7 @@ size_t carve_scratch(int N, const prsgd_model_spec* s, int64_t m_pad, prsgd_ctx*
   const int L = s->n_layers, B = s->batch;
   auto status = take(sizeof(DeviceStatus));
   auto draws = take(sizeof(int32_t) * N);
-  auto losses = take(sizeof(float) * N);
+  auto losses = take(sizeof(float) * (size_t)N * B);
   auto active = take((size_t)N);
   auto stage = take(sizeof(float) * (size_t)m_pad);
   if (ctx) {
@@ -244,9 +244,9 @@ int step_f32(prsgd_ctx* c, int64_t t, bool averaging) {
     SoftmaxArgs a{};
     a.logits = c->buf.act_f32[L]; a.delta = c->buf.delta_f32[L]; a.ldz = c->dims[L];
     a.Y = c->Y; a.P = c->P; a.B = B; a.C = c->dims[L]; a.draw = dr;
-    a.losses = c->losses; a.draws = c->draws; a.active = act_mask;
+    a.row_losses = c->losses; a.draws = c->draws; a.active = act_mask;
     prof_begin(c, PRSGD_KERNEL_SOFTMAX);
-    softmax_ce_kernel<<<N, 256, 0, c->stream>>>(a);
+    softmax_ce_kernel<<<dim3(N, (B + 7) / 8), 256, 0, c->stream>>>(a);
     LAUNCH_CHECK(c);
   }
   for (int l = L; l >= 1; --l) {          // backward, layer by layer: dX_l reads W_l before it is updated
@@ -295,9 +295,9 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging) {
     a.logits = c->buf.act_f32[L]; a.ldz = c->buf.ld[L];
     a.delta_bk = c->buf.delta_bk[L]; a.ld_bf = c->buf.ld[L];
     a.Y = c->Y; a.P = c->P; a.B = c->B; a.C = c->dims[L]; a.draw = dr;
-    a.losses = c->losses; a.draws = c->draws; a.active = act_mask;
+    a.row_losses = c->losses; a.draws = c->draws; a.active = act_mask;
     prof_begin(c, PRSGD_KERNEL_SOFTMAX);
-    launch_pdl(softmax_ce_kernel, dim3(N), dim3(256), 0, c->stream, a);
+    launch_pdl(softmax_ce_kernel, dim3(N, (c->B + 7) / 8), dim3(256), 0, c->stream, a);
     LAUNCH_CHECK(c);
   }
   for (int l = L; l >= 1; --l) {          // dX_l reads W_l before the update of layer l overwrites it
@@ -544,8 +544,16 @@ int prsgd_get_average(prsgd_ctx* c, float* dst, int dst_on_device) {
 int prsgd_get_losses(prsgd_ctx* c, float* h_dst) {
   if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
   if (!h_dst) return fail(c, PRSGD_ERR_ARG, "h_dst is NULL");
-  CUDA_TRY(c, cudaMemcpyAsync(h_dst, c->losses, sizeof(float) * c->N, cudaMemcpyDeviceToHost, c->stream));
-  return check_device_status(c);
+  std::vector<float> rows((size_t)c->N * c->B);
+  CUDA_TRY(c, cudaMemcpyAsync(rows.data(), c->losses, sizeof(float) * rows.size(), cudaMemcpyDeviceToHost, c->stream));
+  int rc = check_device_status(c);
+  if (rc != PRSGD_OK) return rc;
+  for (int n = 0; n < c->N; ++n) {          // mean over the minibatch, rows added in order
+    float s = 0.f;
+    for (int b = 0; b < c->B; ++b) s += rows[(size_t)n * c->B + b];
+    h_dst[n] = s / (float)c->B;
+  }
+  return PRSGD_OK;
 }
 
 int prsgd_get_draws(prsgd_ctx* c, int32_t* h_dst) {

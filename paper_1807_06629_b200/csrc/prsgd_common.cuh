@@ -102,7 +102,7 @@ struct prsgd_ctx {
 
   prsgd::DeviceStatus* status = nullptr;
   int32_t* draws = nullptr;      // [N]
-  float* losses = nullptr;       // [N]
+  float* losses = nullptr;       // [N][B] per-sample losses of the last iteration
   uint8_t* active = nullptr;     // [N] device copy of the Algorithm-3 mask
   bool has_mask = false;
   float* stage_row = nullptr;    // [m_pad] fp32
