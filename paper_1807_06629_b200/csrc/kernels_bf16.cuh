@@ -1,7 +1,7 @@
 // bf16-operand tensor-core path (sm_100a): grouped GEMMs on tcgen05 with TMEM
 // accumulators, operands staged by TMA, one problem per worker.
 //
-//   stream kernel  : forward  Z^T[d_out, B]  = W[d_out, d_in] A^T[d_in, B]      (+bias, ReLU)
+//   stream kernel  : forward  Z^T[d_out, B]  = W[d_out, d_in] A^T[d_in, B]      (+bias, ReLU)   (persistent)
 //                    backward dA^T[d_in, B]  = W^T[d_in, d_out] dZ^T[d_out, B]  (ReLU mask)
 //                    The layer width sits on the MMA's M axis (128 rows per CTA) and the
 //                    minibatch on its N axis, because B = 16..64 is too small for M.
@@ -80,7 +80,8 @@ enum { TC_FWD_RELU = 0, TC_FWD_LINEAR = 1, TC_DX = 2 };
 
 struct StreamArgs {
   int B, N;
-  int k_blocks;            // contraction length / 64
+  int k_steps;             // pipeline steps per item: ceil(contraction length / 128)
+  int tiles_m;             // 128-row tiles of the output features
   int M_total;             // valid output features
   int stages;
   int pool;                // operand B rows come from the data pool at the drawn block
@@ -95,38 +96,47 @@ struct StreamArgs {
   DeviceStatus* status;
 };
 
-constexpr int kStreamThreads = 128;
+// Persistent: one CTA per SM walks (tile, worker) items.  Warp 0 issues TMA, warp 1 issues MMAs,
+// warps 2..5 run the epilogue of item i from one TMEM accumulator while the loads and MMAs of
+// item i + 1 fill the other, so the weight stream never pauses at an item boundary.
+// A stage holds TWO 64-wide K blocks (>= 40 KB per barrier phase): a single issuing thread
+// sustains only ~2 barrier phases per microsecond, so small stages would cap the stream.
+constexpr int kStreamThreads = 192;
 constexpr uint32_t kTileA = 16384;   // 128 x 64 bf16
 
-__host__ __device__ inline uint32_t stream_stage_bytes(int B) { return kTileA + (uint32_t)B * 128u; }
-inline size_t stream_smem_bytes(int B, int stages) { return (size_t)stages * stream_stage_bytes(B) + 1024 + 256; }
+__host__ __device__ inline uint32_t stream_stage_bytes(int B) { return 2u * (kTileA + (uint32_t)B * 128u); }
+inline int stream_stages(int B) {
+  int s = (int)(200000u / stream_stage_bytes(B));
+  return s > 6 ? 6 : s;
+}
+inline size_t stream_smem_bytes(int B) { return (size_t)stream_stages(B) * stream_stage_bytes(B) + 1024 + 256; }
 
 template <int MODE>
-__global__ void __launch_bounds__(kStreamThreads) tc_stream_kernel(const __grid_constant__ CUtensorMap mapW,
-                                                                   const __grid_constant__ CUtensorMap mapB,
-                                                                   const StreamArgs a) {
+__global__ void __launch_bounds__(kStreamThreads, 1) tc_stream_kernel(const __grid_constant__ CUtensorMap mapW,
+                                                                      const __grid_constant__ CUtensorMap mapB,
+                                                                      const StreamArgs a) {
   using namespace ptx;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* gen = smem_raw + (base - raw);
   const uint32_t stage_bytes = stream_stage_bytes(a.B);
+  const uint32_t b_box = (uint32_t)a.B * 128u;
   const int S = a.stages;
-  // barrier block after the stages
   const uint32_t bar0 = base + (uint32_t)S * stage_bytes;
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 64u + 8u * s; };
-  const uint32_t acc_bar = bar0 + 128u;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen + (size_t)S * stage_bytes + 136);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + (size_t)S * stage_bytes + 140);
+  auto acc_full = [&](int q) { return bar0 + 128u + 8u * q; };
+  auto acc_empty = [&](int q) { return bar0 + 144u + 8u * q; };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen + (size_t)S * stage_bytes + 160);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + (size_t)S * stage_bytes + 164);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int m0 = blockIdx.x * 128, n = blockIdx.y;
-  const uint32_t ncols = a.B < 32 ? 32u : (uint32_t)a.B;
+  const uint32_t ncols = 2 * a.B < 32 ? 32u : (uint32_t)(2 * a.B);   // two accumulators of B columns
 
   if (tid == 0) {
     for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    mbar_init(acc_bar, 1);
+    for (int q = 0; q < 2; ++q) { mbar_init(acc_full(q), 1); mbar_init(acc_empty(q), 128); }
     *abort_flag = 0;
     fence_mbar_init();
     prefetch_tensormap(&mapW);
@@ -142,80 +152,109 @@ __global__ void __launch_bounds__(kStreamThreads) tc_stream_kernel(const __grid_
   // a wait that expired in an earlier CTA or launch turns the rest of the work into a no-op
   if (tid == 0) *abort_flag = *(volatile unsigned int*)&a.status->error != 0u ? 1 : 0;
   __syncthreads();
-  const bool is_active = (a.active == nullptr || a.active[n] != 0) && *abort_flag == 0;
+  const int total_items = *abort_flag != 0 ? 0 : a.tiles_m * a.N;
+  auto item_active = [&](int n) { return a.active == nullptr || a.active[n] != 0; };
 
-  if (is_active) {
-    if (warp == 0 && lane == 0) {
-      // ---- producer: TMA loads of the weight tile and the activation tile, one 64-wide K block per stage
+  if (warp == 0 && lane == 0) {
+    // ---------------- producer: per step two weight K blocks and two activation K blocks
+    uint32_t g = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
+      const int n = item / a.tiles_m, m0 = (item % a.tiles_m) * 128;
+      if (!item_active(n)) continue;
       const int row0 = a.pool ? (int)draw_block(a.draw.seed, n, a.draw.t, a.draw.n_blocks) * a.B : 0;
-      int issued = 0;
-      for (int kb = 0; kb < a.k_blocks; ++kb) {
-        const int s = kb % S;
-        const uint32_t ph = (uint32_t)(kb / S) & 1u;
-        if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, a.status, 0x101)) break;
-        const uint32_t sa = base + (uint32_t)s * stage_bytes, sb = sa + kTileA;
+      for (int ks = 0; ks < a.k_steps; ++ks, ++g) {
+        const int s = g % S;
+        const uint32_t ph = (g / S) & 1u;
+        ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, a.status, 0x101);
+        if (!ok) break;
+        const uint32_t sa = base + (uint32_t)s * stage_bytes, sb = sa + 2u * kTileA;
         mbar_expect_tx(full_bar(s), stage_bytes);
-        if (MODE == TC_DX) {
-          tma_load_3d(sa, &mapW, full_bar(s), m0, kb * 64, n);
-          tma_load_3d(sa + 8192u, &mapW, full_bar(s), m0 + 64, kb * 64, n);
-        } else {
-          tma_load_3d(sa, &mapW, full_bar(s), kb * 64, m0, n);
-        }
-        tma_load_3d(sb, &mapB, full_bar(s), kb * 64, row0, n);
-        issued = kb + 1;
-      }
-      if (*abort_flag) {   // let the copies already in flight land before the CTA goes away
-        for (int kb = issued > S ? issued - S : 0; kb < issued; ++kb) {
-          const uint64_t t0 = globaltimer_ns();
-          while (!mbar_try_wait(full_bar(kb % S), (uint32_t)(kb / S) & 1u) && globaltimer_ns() - t0 < 100000000ull) {}
-        }
-      }
-    } else if (warp == 1 && lane == 0) {
-      // ---- MMA issuer
-      constexpr int A_MN = MODE == TC_DX ? 1 : 0;
-      const uint32_t idesc = idesc_bf16(128, a.B, A_MN, 0);
-      for (int kb = 0; kb < a.k_blocks; ++kb) {
-        const int s = kb % S;
-        const uint32_t ph = (uint32_t)(kb / S) & 1u;
-        if (!mbar_wait(full_bar(s), ph, abort_flag, a.status, 0x102)) break;
-        tc_fence_after();
-        const uint32_t sa = base + (uint32_t)s * stage_bytes, sb = sa + kTileA;
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const uint64_t da = A_MN ? smem_desc_sw128(sa + k * 2048u, 8192u, 1024u) : smem_desc_sw128(sa + k * 32u, 16u, 1024u);
-          const uint64_t db = smem_desc_sw128(sb + k * 32u, 16u, 1024u);
-          mma_bf16(tmem, da, db, idesc, (kb | k) != 0 ? 1u : 0u);
+        for (int j = 0; j < 2; ++j) {
+          const int k0 = (2 * ks + j) * 64;          // a block past the end of K is zero-filled by TMA
+          if (MODE == TC_DX) {
+            tma_load_3d(sa + j * kTileA, &mapW, full_bar(s), m0, k0, n);
+            tma_load_3d(sa + j * kTileA + 8192u, &mapW, full_bar(s), m0 + 64, k0, n);
+          } else {
+            tma_load_3d(sa + j * kTileA, &mapW, full_bar(s), k0, m0, n);
+          }
+          tma_load_3d(sb + j * b_box, &mapB, full_bar(s), k0, row0, n);
+        }
+      }
+    }
+    if (*abort_flag && g > 0) {   // let the copies already in flight land before the CTA goes away
+      const long long t0 = clock64();
+      const uint32_t last = g - 1;
+      while (!mbar_try_wait(full_bar(last % S), (last / S) & 1u) && clock64() - t0 < 200000000ll) {}
+    }
+  } else if (warp == 1 && lane == 0) {
+    // ---------------- MMA issuer
+    constexpr int A_MN = MODE == TC_DX ? 1 : 0;
+    const uint32_t idesc = idesc_bf16(128, a.B, A_MN, 0);
+    uint32_t g = 0, it = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
+      if (!item_active(item / a.tiles_m)) continue;
+      const int q = it & 1;
+      ok = mbar_wait(acc_empty(q), ((it >> 1) & 1u) ^ 1u, abort_flag, a.status, 0x104);
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t acc = tmem + (uint32_t)(q * a.B);
+      for (int ks = 0; ks < a.k_steps; ++ks, ++g) {
+        const int s = g % S;
+        ok = mbar_wait(full_bar(s), (g / S) & 1u, abort_flag, a.status, 0x102);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t sa = base + (uint32_t)s * stage_bytes, sb = sa + 2u * kTileA;
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const uint32_t aj = sa + j * kTileA, bj = sb + j * b_box;
+            const uint64_t da = A_MN ? smem_desc_sw128(aj + k * 2048u, 8192u, 1024u) : smem_desc_sw128(aj + k * 32u, 16u, 1024u);
+            const uint64_t db = smem_desc_sw128(bj + k * 32u, 16u, 1024u);
+            mma_bf16(acc, da, db, idesc, (ks | j | k) != 0 ? 1u : 0u);
+          }
         }
         mma_commit(empty_bar(s));
       }
-      mma_commit(acc_bar);
+      if (ok) mma_commit(acc_full(q));
+      ++it;
     }
-    __syncwarp();
-
-    // ---- epilogue: thread <-> output feature m0 + tid, its B accumulators sit in one TMEM lane.
+  } else if (warp >= 2) {
+    // ---------------- epilogue: thread <-> output feature, its B accumulators sit in one TMEM lane.
     // Work goes in batches of 16 minibatch columns; the ReLU-mask values a batch needs (TC_DX) are
     // fetched one batch ahead, the first of them before the accumulator is even ready, so that no
     // global-load latency sits between the accumulator and the stores.
-    const int m = m0 + tid;
-    const bool valid = m < a.M_total;
+    const int q4 = warp & 3;
+    const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
     const int batches = a.B / 16;
-    auto mask_fetch = [&](int bi, uint16_t (&mk)[16]) {
-      if (MODE == TC_DX && bi < batches && valid) {
+    uint32_t it = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
+      const int n = item / a.tiles_m;
+      if (!item_active(n)) continue;
+      const int m = (item % a.tiles_m) * 128 + q4 * 32 + lane;
+      const bool valid = m < a.M_total;
+      auto mask_fetch = [&](int bi, uint16_t (&mk)[16]) {
+        if (MODE == TC_DX && bi < batches && valid) {
 #pragma unroll
-        for (int j = 0; j < 16; ++j) mk[j] = __ldg(a.mask_src + ((int64_t)n * a.B + bi * 16 + j) * a.ld_out + m);
-      }
-    };
-    uint16_t mk_cur[16], mk_next[16];
-    mask_fetch(0, mk_cur);
-    float bias = 0.f;
-    if (MODE != TC_DX && valid) bias = a.bias[(int64_t)n * a.bias_stride + m];
-    const bool acc_ok = __all_sync(0xffffffffu, mbar_wait(acc_bar, 0u, abort_flag, a.status, 0x103));
-    tc_fence_after();
-    if (acc_ok) {
+          for (int j = 0; j < 16; ++j) mk[j] = __ldg(a.mask_src + ((int64_t)n * a.B + bi * 16 + j) * a.ld_out + m);
+        }
+      };
+      uint16_t mk_cur[16], mk_next[16];
+      mask_fetch(0, mk_cur);
+      float bias = 0.f;
+      if (MODE != TC_DX && valid) bias = a.bias[(int64_t)n * a.bias_stride + m];
+      const int q = it & 1;
+      ok = __all_sync(0xffffffffu, mbar_wait(acc_full(q), (it >> 1) & 1u, abort_flag, a.status, 0x103));
+      if (!ok) break;
+      tc_fence_after();
       for (int bi = 0; bi < batches; ++bi) {
         const int c0 = bi * 16;
         uint32_t v[16];
-        tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
+        tmem_ld16(tmem + lane_off + (uint32_t)(q * a.B + c0), v);
         mask_fetch(bi + 1, mk_next);
         tmem_ld_wait();
         if (valid) {
@@ -237,8 +276,12 @@ __global__ void __launch_bounds__(kStreamThreads) tc_stream_kernel(const __grid_
           for (int j = 0; j < 16; ++j) mk_cur[j] = mk_next[j];
         }
       }
+      tc_fence_before();
+      mbar_arrive(acc_empty(q));
+      ++it;
     }
   }
+  __syncwarp();
   tc_fence_before();
   __syncthreads();
   if (warp == 1) tmem_dealloc(tmem, ncols);
@@ -552,7 +595,7 @@ inline int tc_create(prsgd_ctx* c, std::string* err) {
   }
   if (rc != PRSGD_OK) { delete st; return rc; }
   cudaError_t e = cudaSuccess;
-  const int big = (int)stream_smem_bytes(c->B, 8);
+  const int big = (int)stream_smem_bytes(c->B);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_stream_kernel<TC_FWD_RELU>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_stream_kernel<TC_FWD_LINEAR>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_stream_kernel<TC_DX>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
@@ -583,26 +626,20 @@ inline int tc_bind_data(prsgd_ctx* c, std::string* err) {
   return rc;
 }
 
-inline int stream_stages(int B, int k_blocks) {
-  int s = (int)(98304 / stream_stage_bytes(B));   // ~96 KB of stages: two CTAs per SM
-  if (s > 8) s = 8;
-  if (s > k_blocks) s = k_blocks;
-  return s < 1 ? 1 : s;
-}
-
 // forward GEMM of layer l (1-based)
 inline void tc_launch_forward(prsgd_ctx* c, int l, const DrawArgs& dr, const uint8_t* active) {
   TcState* st = static_cast<TcState*>(c->tc);
   const Layer& ly = c->layer[l - 1];
   StreamArgs a{};
-  a.B = c->B; a.N = c->N; a.k_blocks = ly.d_in / 64; a.M_total = ly.d_out;
-  a.stages = stream_stages(c->B, a.k_blocks);
+  a.B = c->B; a.N = c->N; a.k_steps = (ly.d_in / 64 + 1) / 2; a.M_total = ly.d_out; a.tiles_m = (ly.d_out + 127) / 128;
+  a.stages = stream_stages(c->B);
   a.pool = l == 1; a.draw = dr; a.ld_out = c->buf.ld[l];
   a.out_bk = c->buf.act_bk[l]; a.out_f32 = c->buf.act_f32[l];
   a.bias = c->params + ly.b_off; a.bias_stride = c->m_pad;
   a.active = active; a.status = c->status;
-  dim3 grid((ly.d_out + 127) / 128, c->N);
-  const size_t smem = stream_smem_bytes(c->B, a.stages);
+  const int items = a.tiles_m * c->N;
+  dim3 grid(items < st->num_sms ? items : st->num_sms);
+  const size_t smem = stream_smem_bytes(c->B);
   if (l < c->L)
     launch_pdl(tc_stream_kernel<TC_FWD_RELU>, grid, kStreamThreads, smem, c->stream, st->layer[l - 1].shadow_k, st->layer[l - 1].act_in, a);
   else
@@ -614,14 +651,15 @@ inline void tc_launch_dx(prsgd_ctx* c, int l, const DrawArgs& dr, const uint8_t*
   TcState* st = static_cast<TcState*>(c->tc);
   const Layer& ly = c->layer[l - 1];
   StreamArgs a{};
-  a.B = c->B; a.N = c->N; a.k_blocks = c->buf.ld[l] / 64; a.M_total = ly.d_in;
-  a.stages = stream_stages(c->B, a.k_blocks);
+  a.B = c->B; a.N = c->N; a.k_steps = (c->buf.ld[l] / 64 + 1) / 2; a.M_total = ly.d_in; a.tiles_m = (ly.d_in + 127) / 128;
+  a.stages = stream_stages(c->B);
   a.pool = 0; a.draw = dr; a.ld_out = c->buf.ld[l - 1];
   a.out_bk = c->buf.delta_bk[l - 1]; a.mask_src = c->buf.act_bk[l - 1];
   a.active = active; a.status = c->status;
-  dim3 grid((ly.d_in + 127) / 128, c->N);
-  const size_t smem = stream_smem_bytes(c->B, a.stages);
-  launch_pdl(tc_stream_kernel<TC_DX>, grid, kStreamThreads, smem, c->stream, st->layer[l - 1].shadow_mn, st->layer[l - 1].delta_out, a);
+  const int items = a.tiles_m * c->N;
+  dim3 grid(items < st->num_sms ? items : st->num_sms);
+  launch_pdl(tc_stream_kernel<TC_DX>, grid, kStreamThreads, stream_smem_bytes(c->B), c->stream, st->layer[l - 1].shadow_mn,
+             st->layer[l - 1].delta_out, a);
 }
 
 template <int TN>

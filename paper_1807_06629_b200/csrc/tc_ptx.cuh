@@ -1,6 +1,6 @@
 // Thin wrappers over the sm_100a instructions the tensor-core path uses:
 // mbarrier, TMA tiled bulk copies, tcgen05 (TMEM allocation, MMA, commit, load).
-// Every wait is bounded: after ~2 s it records an error word and returns false.
+// Every wait is bounded: after about 2 s it records an error word and returns false.
 #pragma once
 #include <cuda.h>
 #include <stdint.h>
@@ -42,19 +42,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
-constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s
+constexpr long long kWaitLimitCycles = 4000000000ll;   // about 2 s at the SM clock (read with clock64: cheap, SM-local)
 
 // Bounded wait.  `abort_flag` lives in shared memory: once any wait of the CTA gives up, all others
 // return quickly.  On expiry the code `what` is recorded in the device status words.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                           DeviceStatus* status, unsigned what) {
   if (mbar_try_wait(bar, parity)) return true;
-  const uint64_t t0 = globaltimer_ns();
+  long long t0 = 0;
   for (uint32_t it = 1;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 255u) == 0u) {
+    if ((it & 63u) == 0u) {
       if (*abort_flag) return false;
-      if (globaltimer_ns() - t0 > kWaitLimitNs) {
+      const long long now = clock64();
+      if (t0 == 0) t0 = now;
+      if (now - t0 > kWaitLimitCycles) {
         *abort_flag = 1;
         if (atomicCAS(&status->error, 0u, what) == 0u) status->where = blockIdx.x;
         return false;
