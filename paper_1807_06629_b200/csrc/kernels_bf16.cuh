@@ -551,19 +551,31 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
   if (warp == 1) tmem_dealloc(tmem, 256u);
 }
 
-// b_l <- b_l - gamma * sum_b dZ_l[b, :] (the bias part of Eq. parallel-sgd-x-update), one thread per (worker, j).
-__global__ void __launch_bounds__(128) bias_update_kernel(float* params, int64_t m_pad, int64_t b_off, int d_out,
-                                                          const uint16_t* delta_bk, int ld, int B, float gamma,
-                                                          const uint8_t* active) {
+// b_l <- b_l - gamma * sum_b dZ_l[b, :] (the bias part of Eq. parallel-sgd-x-update) for every layer in
+// one launch: grid (ceil(max d_l / 128), N, L), one thread per (layer, worker, j).
+struct BiasArgs {
+  float* params;
+  int64_t m_pad;
+  int L, B;
+  float gamma;
+  const uint8_t* active;
+  int64_t b_off[PRSGD_MAX_LAYERS];
+  int d_out[PRSGD_MAX_LAYERS];
+  int ld[PRSGD_MAX_LAYERS];
+  const uint16_t* delta_bk[PRSGD_MAX_LAYERS];
+};
+
+__global__ void __launch_bounds__(128) bias_update_kernel(const BiasArgs a) {
   ptx::pdl_trigger();
   ptx::pdl_wait();
+  const int l = blockIdx.z, n = blockIdx.y;
   const int j = blockIdx.x * blockDim.x + threadIdx.x;
-  const int n = blockIdx.y;
-  if (j >= d_out || (active != nullptr && active[n] == 0)) return;
+  if (j >= a.d_out[l] || (a.active != nullptr && a.active[n] == 0)) return;
+  const uint16_t* d = a.delta_bk[l] + (int64_t)n * a.B * a.ld[l] + j;
   float g = 0.f;
-  for (int b = 0; b < B; ++b) g += __uint_as_float((uint32_t)__ldg(delta_bk + ((int64_t)n * B + b) * ld + j) << 16);
-  float* bp = params + (int64_t)n * m_pad + b_off + j;
-  *bp = fmaf(-gamma, g, *bp);
+  for (int b = 0; b < a.B; ++b) g += __uint_as_float((uint32_t)__ldg(d + (int64_t)b * a.ld[l]) << 16);
+  float* bp = a.params + (int64_t)n * a.m_pad + a.b_off[l] + j;
+  *bp = fmaf(-a.gamma, g, *bp);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -696,13 +708,19 @@ inline void tc_launch_update(prsgd_ctx* c, int l, const DrawArgs& dr, const uint
   else tc_launch_update_tn<64>(c, l, dr, active, fuse);
 }
 
-// Bias step of layer l; on an averaging iteration it is followed by the node average of the bias
-// segment alone (same arithmetic as the stand-alone averaging kernel, so the bits agree).
-inline void tc_launch_bias(prsgd_ctx* c, int l, const uint8_t* active) {
-  const Layer& ly = c->layer[l - 1];
-  dim3 grid((ly.d_out + 127) / 128, c->N);
-  launch_pdl(bias_update_kernel, grid, dim3(128), 0, c->stream, c->params, c->m_pad, ly.b_off, ly.d_out,
-             (const uint16_t*)c->buf.delta_bk[l], c->buf.ld[l], c->B, c->gamma, active);
+// Bias step of all layers (after the last dZ has been formed).  On an averaging iteration it is followed
+// by the node average of each bias segment (same arithmetic as the stand-alone averaging kernel, so
+// the bits agree with update-then-average).
+inline void tc_launch_bias(prsgd_ctx* c, const uint8_t* active) {
+  BiasArgs a{};
+  a.params = c->params; a.m_pad = c->m_pad; a.L = c->L; a.B = c->B; a.gamma = c->gamma; a.active = active;
+  int dmax = 1;
+  for (int l = 1; l <= c->L; ++l) {
+    const Layer& ly = c->layer[l - 1];
+    a.b_off[l - 1] = ly.b_off; a.d_out[l - 1] = ly.d_out; a.ld[l - 1] = c->buf.ld[l]; a.delta_bk[l - 1] = c->buf.delta_bk[l];
+    if (ly.d_out > dmax) dmax = ly.d_out;
+  }
+  launch_pdl(bias_update_kernel, dim3((dmax + 127) / 128, c->N, c->L), dim3(128), 0, c->stream, a);
 }
 
 inline void tc_launch_bias_average(prsgd_ctx* c, int l) {

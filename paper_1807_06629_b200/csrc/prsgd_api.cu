@@ -309,10 +309,12 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging) {
     prof_begin(c, fuse ? PRSGD_KERNEL_UPDATE_AVERAGE : PRSGD_KERNEL_UPDATE);
     tc_launch_update(c, l, dr, act_mask, fuse);
     LAUNCH_CHECK(c);
-    prof_begin(c, PRSGD_KERNEL_MISC);
-    tc_launch_bias(c, l, act_mask);
-    LAUNCH_CHECK(c);
-    if (fuse) {
+  }
+  prof_begin(c, PRSGD_KERNEL_MISC);
+  tc_launch_bias(c, act_mask);
+  LAUNCH_CHECK(c);
+  if (fuse) {
+    for (int l = 1; l <= L; ++l) {
       prof_begin(c, PRSGD_KERNEL_MISC);
       tc_launch_bias_average(c, l);
       LAUNCH_CHECK(c);
