@@ -47,13 +47,16 @@ __device__ __forceinline__ const float* operand_ptr(const OperandF32& o, int n, 
   return p;
 }
 
-// C(i, j) = sum_p A(i, p) B(p, j); tile TM x 64 x 16, 256 threads, (TM/16) x 4 outputs per thread.
+// C(i, j) = sum_p A(i, p) B(p, j); tile TM x 64 x 32, 256 threads, (TM/16) x 4 outputs per thread.
 // A_PC / B_PC: the contraction index p is the contiguous one of that operand.
 template <int TM, bool A_PC, bool B_PC, int EPI, bool FUSE>
 __global__ void __launch_bounds__(256) gemm_f32_kernel(const GemmF32Args g) {
-  constexpr int TN = 64, TK = 16, RM = TM / 16;
-  __shared__ float As[TK][TM + 1];
-  __shared__ __align__(16) float Bs[TK][TN + 4];
+  constexpr int TN = 64, TK = 32, RM = TM / 16;
+  constexpr int LA = TM * TK / 256, LB = TN * TK / 256;   // elements each thread moves per K chunk
+  __shared__ float As[2][TK][TM + 1];
+  __shared__ __align__(16) float Bs[2][TK][TN + 4];
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");   // no-op unless launched as a programmatic dependent
 
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
   const int i0 = blockIdx.y * TM, j0 = blockIdx.x * TN;
@@ -81,32 +84,50 @@ __global__ void __launch_bounds__(256) gemm_f32_kernel(const GemmF32Args g) {
     if (is_active) {
       const float* Ap = operand_ptr(g.A, n, g.draw);
       const float* Bp = operand_ptr(g.Bo, n, g.draw);
+      // software pipeline: the next K chunk travels global -> registers while the current one is
+      // consumed from shared memory; two shared buffers, one barrier per chunk
+      float ra[LA], rb[LB];
+      auto gload = [&](int k0) {
+#pragma unroll
+        for (int r = 0; r < LA; ++r) {
+          const int e = tid + 256 * r;
+          const int i = A_PC ? e / TK : e % TM;
+          const int p = A_PC ? e % TK : e / TM;
+          ra[r] = (i0 + i < g.M && k0 + p < g.K) ? Ap[(int64_t)(i0 + i) * g.A.s0 + (int64_t)(k0 + p) * g.A.s1] : 0.f;
+        }
+#pragma unroll
+        for (int r = 0; r < LB; ++r) {
+          const int e = tid + 256 * r;
+          const int j = B_PC ? e / TK : e % TN;
+          const int p = B_PC ? e % TK : e / TN;
+          rb[r] = (j0 + j < g.Nn && k0 + p < g.K) ? Bp[(int64_t)(k0 + p) * g.Bo.s0 + (int64_t)(j0 + j) * g.Bo.s1] : 0.f;
+        }
+      };
+      auto sstore = [&](int buf) {
+#pragma unroll
+        for (int r = 0; r < LA; ++r) {
+          const int e = tid + 256 * r;
+          As[buf][A_PC ? e % TK : e / TM][A_PC ? e / TK : e % TM] = ra[r];
+        }
+#pragma unroll
+        for (int r = 0; r < LB; ++r) {
+          const int e = tid + 256 * r;
+          Bs[buf][B_PC ? e % TK : e / TN][B_PC ? e / TK : e % TN] = rb[r];
+        }
+      };
+      gload(0);
+      sstore(0);
+      __syncthreads();
+      int buf = 0;
       for (int k0 = 0; k0 < g.K; k0 += TK) {
-#pragma unroll
-        for (int r = 0; r < RM; ++r) {
-          int e = tid + 256 * r;
-          int i = A_PC ? e / TK : e % TM;
-          int p = A_PC ? e % TK : e / TM;
-          float v = 0.f;
-          if (i0 + i < g.M && k0 + p < g.K) v = Ap[(int64_t)(i0 + i) * g.A.s0 + (int64_t)(k0 + p) * g.A.s1];
-          As[p][i] = v;
-        }
-#pragma unroll
-        for (int r = 0; r < 4; ++r) {
-          int e = tid + 256 * r;
-          int j = B_PC ? e / TK : e % TN;
-          int p = B_PC ? e % TK : e / TN;
-          float v = 0.f;
-          if (j0 + j < g.Nn && k0 + p < g.K) v = Bp[(int64_t)(k0 + p) * g.Bo.s0 + (int64_t)(j0 + j) * g.Bo.s1];
-          Bs[p][j] = v;
-        }
-        __syncthreads();
+        const bool more = k0 + TK < g.K;
+        if (more) gload(k0 + TK);
 #pragma unroll
         for (int p = 0; p < TK; ++p) {
           float a[RM];
 #pragma unroll
-          for (int r = 0; r < RM; ++r) a[r] = As[p][ty * RM + r];
-          const float4 b4 = *reinterpret_cast<const float4*>(&Bs[p][tx * 4]);
+          for (int r = 0; r < RM; ++r) a[r] = As[buf][p][ty * RM + r];
+          const float4 b4 = *reinterpret_cast<const float4*>(&Bs[buf][p][tx * 4]);
           const float b[4] = {b4.x, b4.y, b4.z, b4.w};
 #pragma unroll
           for (int r = 0; r < RM; ++r)
@@ -115,9 +136,11 @@ __global__ void __launch_bounds__(256) gemm_f32_kernel(const GemmF32Args g) {
         }
         if (do_bias && tid < TM) {
 #pragma unroll
-          for (int p = 0; p < TK; ++p) bsum += As[p][tid];
+          for (int p = 0; p < TK; ++p) bsum += As[buf][p][tid];
         }
+        if (more) sstore(buf ^ 1);
         __syncthreads();
+        buf ^= 1;
       }
     }
 

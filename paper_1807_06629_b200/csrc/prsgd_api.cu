@@ -209,7 +209,7 @@ DrawArgs draw_args(const prsgd_ctx* c, int64_t t) {
 template <int TM, bool A_PC, bool B_PC, int EPI, bool FUSE>
 void launch_gemm_f32(prsgd_ctx* c, const GemmF32Args& g) {
   dim3 grid((g.Nn + 63) / 64, (g.M + TM - 1) / TM, FUSE ? 1 : g.N);
-  gemm_f32_kernel<TM, A_PC, B_PC, EPI, FUSE><<<grid, 256, 0, c->stream>>>(g);
+  launch_pdl(gemm_f32_kernel<TM, A_PC, B_PC, EPI, FUSE>, grid, dim3(256), 0, c->stream, g);
 }
 
 // One iteration of Algorithm 1 on the fp32-operand path.
@@ -246,7 +246,7 @@ int step_f32(prsgd_ctx* c, int64_t t, bool averaging) {
     a.Y = c->Y; a.P = c->P; a.B = B; a.C = c->dims[L]; a.draw = dr;
     a.row_losses = c->losses; a.draws = c->draws; a.active = act_mask;
     prof_begin(c, PRSGD_KERNEL_SOFTMAX);
-    softmax_ce_kernel<<<dim3(N, (B + 7) / 8), 256, 0, c->stream>>>(a);
+    launch_pdl(softmax_ce_kernel, dim3(N, (B + 7) / 8), dim3(256), 0, c->stream, a);
     LAUNCH_CHECK(c);
   }
   for (int l = L; l >= 1; --l) {          // backward, layer by layer: dX_l reads W_l before it is updated
