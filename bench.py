@@ -93,6 +93,35 @@ class ClockSampler:
                 "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
+# ----------------------------------------------------------------------------- ncu traffic
+# dram__bytes_read.sum + dram__bytes_write.sum per iteration of one kernel family, from the one-pass ncu
+# capture summarised in profiles/; valid only while the kernel's source section is unchanged.
+NCU_TRAFFIC = {
+    ("cfg4", "update"): {"bytes_per_iteration": 2.22e9 + 3.04e9, "launches_per_iteration": 4,
+                         "kernel_sha256": "55348bf6e8fa635419181b8251e478103b95905a972f18c2a2b52dd4ab0479ea"},
+}
+
+
+def kernel_section_sha(family: str) -> str:
+    """Hash of the source text of the kernel a family runs (update: tc_update_kernel and its stage layout)."""
+    import hashlib
+    path = os.path.join(ROOT, "paper_1807_06629_b200", "csrc", "kernels_bf16.cuh")
+    with open(path) as f:
+        src = f.read()
+    marks = {"update": ("template <int TN> struct UpdCfg", "// b_l <- b_l - gamma")}
+    if family not in marks:
+        return ""
+    a, b = src.find(marks[family][0]), src.find(marks[family][1])
+    return hashlib.sha256(src[a:b].encode()).hexdigest() if 0 <= a < b else ""
+
+
+def ncu_traffic_per_launch(workload: str, family: str):
+    rec = NCU_TRAFFIC.get((workload, family))
+    if rec is None or rec["kernel_sha256"] != kernel_section_sha(family):
+        return None
+    return rec["bytes_per_iteration"] / rec["launches_per_iteration"]
+
+
 # ----------------------------------------------------------------------------- byte model
 def algorithmic_bytes(w: synth.Workload, m_pad: int) -> dict:
     """Algorithmic HBM bytes of one local iteration of all N workers, per kernel family.
@@ -330,7 +359,7 @@ def main():
     achieved = bytes_iter[dom] * iters_seen / (dom_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"] + " copy bandwidth",
-                "traffic": None,
+                "traffic": ncu_traffic_per_launch(w.name, dom),
                 "avg_launch_us": 1e3 * dom_ms / dom_launches,
                 "algorithmic_bytes_per_launch": bytes_iter[dom] / per_iter_launches,
                 "family_us_per_iteration": {k: round(1e3 * v[0] / (args.steps * max(w.I, 1)), 2) for k, v in prof.items() if v[1]},
