@@ -206,6 +206,16 @@ int prsgd_get_launch_count(prsgd_ctx* ctx, int64_t* count);
 /* Wait for the stream, then report any device-side error recorded so far. */
 int prsgd_sync(prsgd_ctx* ctx);
 
+/* Failure path, exercised without faulting the GPU.  Every wait inside the tensor-core kernels is
+ * bounded; when one expires the kernel records a code in the scratch status words and returns, later
+ * launches of the context become no-ops, and prsgd_sync / prsgd_get_* return
+ * PRSGD_ERR_DEVICE_TIMEOUT.  prsgd_selftest_wait_expiry launches a one-warp kernel that waits about
+ * limit_us microseconds (1..1000000) on a barrier nothing ever signals, so that exactly this happens;
+ * prsgd_clear_device_error zeroes the status words and makes the context usable again (the
+ * parameters are as the last successful launch left them). */
+int prsgd_selftest_wait_expiry(prsgd_ctx* ctx, int32_t limit_us);
+int prsgd_clear_device_error(prsgd_ctx* ctx);
+
 /* Text of the last error of this context (or of the last context-free call
  * when ctx is NULL).  Library-owned, valid until the next call. */
 const char* prsgd_last_error(prsgd_ctx* ctx);

@@ -32,7 +32,8 @@ EXPORTS = [
     "prsgd_get_params", "prsgd_local_steps", "prsgd_average", "prsgd_get_average", "prsgd_get_losses",
     "prsgd_get_draws", "prsgd_set_lr", "prsgd_set_interval", "prsgd_set_active", "prsgd_get_step",
     "prsgd_set_step", "prsgd_set_option", "prsgd_get_launch_count", "prsgd_get_profile", "prsgd_sync", "prsgd_last_error",
-    "prsgd_average_rows", "prsgd_draw_block", "prsgd_mean_rows_noalloc",
+    "prsgd_average_rows", "prsgd_draw_block", "prsgd_mean_rows_noalloc", "prsgd_selftest_wait_expiry",
+    "prsgd_clear_device_error",
 ]
 NOALLOC_MAX_M = 1 << 20
 
@@ -80,6 +81,8 @@ def _load() -> C.CDLL:
         "prsgd_get_launch_count": (C.c_int, [vp, C.POINTER(i64)]),
         "prsgd_get_profile": (C.c_int, [vp, i32, C.POINTER(C.c_double), C.POINTER(i64)]),
         "prsgd_sync": (C.c_int, [vp]),
+        "prsgd_selftest_wait_expiry": (C.c_int, [vp, i32]),
+        "prsgd_clear_device_error": (C.c_int, [vp]),
         "prsgd_last_error": (C.c_char_p, [vp]),
         "prsgd_average_rows": (C.c_int, [vp, i64, i64, i64, vp]),
         "prsgd_draw_block": (u64, [u64, i32, i64, u64]),
@@ -302,6 +305,12 @@ class PRSGD:
             self._call(lib.prsgd_get_profile, k, C.byref(ms), C.byref(n))
             out[name] = (ms.value, n.value)
         return out
+
+    def selftest_wait_expiry(self, limit_us: int = 1000):
+        self._call(lib.prsgd_selftest_wait_expiry, limit_us)
+
+    def clear_device_error(self):
+        self._call(lib.prsgd_clear_device_error)
 
     def sync(self):
         self._call(lib.prsgd_sync)

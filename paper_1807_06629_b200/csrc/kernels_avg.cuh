@@ -22,10 +22,12 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 template <int MODE, bool SHADOW>
 __global__ void __launch_bounds__(256) average_rows_kernel(float* __restrict__ P, int64_t N, int64_t m,
                                                            int64_t row_stride, float* __restrict__ out,
-                                                           uint16_t* __restrict__ shadow) {
+                                                           uint16_t* __restrict__ shadow,
+                                                           const DeviceStatus* status = nullptr) {
   constexpr int U = 8;
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");   // no-op unless launched as a programmatic dependent
+  if (status != nullptr && status->error != 0u) return;   // a recorded expired wait: leave the store alone
   const int64_t cols4 = m >> 2;
   const int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   const float fN = (float)N;

@@ -563,6 +563,7 @@ struct BiasArgs {
   int d_out[PRSGD_MAX_LAYERS];
   int ld[PRSGD_MAX_LAYERS];
   const uint16_t* delta_bk[PRSGD_MAX_LAYERS];
+  const DeviceStatus* status;
 };
 
 __global__ void __launch_bounds__(128) bias_update_kernel(const BiasArgs a) {
@@ -570,12 +571,25 @@ __global__ void __launch_bounds__(128) bias_update_kernel(const BiasArgs a) {
   ptx::pdl_wait();
   const int l = blockIdx.z, n = blockIdx.y;
   const int j = blockIdx.x * blockDim.x + threadIdx.x;
-  if (j >= a.d_out[l] || (a.active != nullptr && a.active[n] == 0)) return;
+  if (j >= a.d_out[l] || (a.active != nullptr && a.active[n] == 0) || a.status->error != 0u) return;
   const uint16_t* d = a.delta_bk[l] + (int64_t)n * a.B * a.ld[l] + j;
   float g = 0.f;
   for (int b = 0; b < a.B; ++b) g += __uint_as_float((uint32_t)__ldg(d + (int64_t)b * a.ld[l]) << 16);
   float* bp = a.params + (int64_t)n * a.m_pad + a.b_off[l] + j;
   *bp = fmaf(-a.gamma, g, *bp);
+}
+
+// Self-test of the failure path: waits on an mbarrier that nothing ever arrives on, with a short
+// limit, so that the wait expires, the status word is set and the kernel returns normally.
+__global__ void __launch_bounds__(32) wait_expiry_kernel(DeviceStatus* status, long long limit_cycles) {
+  __shared__ __align__(8) unsigned long long bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    ptx::mbar_init(ptx::smem_u32(&bar), 1);
+    ptx::fence_mbar_init();
+    ptx::mbar_wait(ptx::smem_u32(&bar), 0u, &abort_flag, status, 0x301, limit_cycles);
+  }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -714,6 +728,7 @@ inline void tc_launch_update(prsgd_ctx* c, int l, const DrawArgs& dr, const uint
 inline void tc_launch_bias(prsgd_ctx* c, const uint8_t* active) {
   BiasArgs a{};
   a.params = c->params; a.m_pad = c->m_pad; a.L = c->L; a.B = c->B; a.gamma = c->gamma; a.active = active;
+  a.status = c->status;
   int dmax = 1;
   for (int l = 1; l <= c->L; ++l) {
     const Layer& ly = c->layer[l - 1];
@@ -727,7 +742,8 @@ inline void tc_launch_bias_average(prsgd_ctx* c, int l) {
   const Layer& ly = c->layer[l - 1];
   const int64_t threads = ly.d_out / 4 + (ly.d_out & 3);
   launch_pdl(average_rows_kernel<0, false>, dim3((unsigned)((threads + 255) / 256)), dim3(256), 0, c->stream,
-             c->params + ly.b_off, (int64_t)c->N, (int64_t)ly.d_out, c->m_pad, (float*)nullptr, (uint16_t*)nullptr);
+             c->params + ly.b_off, (int64_t)c->N, (int64_t)ly.d_out, c->m_pad, (float*)nullptr, (uint16_t*)nullptr,
+             (const DeviceStatus*)c->status);
 }
 
 }  // namespace prsgd

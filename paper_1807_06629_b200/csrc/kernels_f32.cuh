@@ -239,6 +239,7 @@ struct SoftmaxArgs {
   float* row_losses;     // [N][B]: logsumexp(z_b) - z_b[y_b]; the caller averages them in row order
   int32_t* draws;        // [N]
   const uint8_t* active;
+  const DeviceStatus* status;   // tensor-core path: a recorded expired wait turns the launch into a no-op
 };
 
 __device__ __forceinline__ uint16_t f32_to_bf16_rn(float f) {
@@ -252,6 +253,7 @@ __global__ void __launch_bounds__(256) softmax_ce_kernel(const SoftmaxArgs a) {
   asm volatile("griddepcontrol.wait;" ::: "memory");   // no-op unless launched as a programmatic dependent
   const int n = blockIdx.x;
   if (a.active != nullptr && a.active[n] == 0) return;
+  if (a.status != nullptr && a.status->error != 0u) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int b = blockIdx.y * 8 + warp;
   const uint32_t blk = draw_block(a.draw.seed, n, a.draw.t, a.draw.n_blocks);

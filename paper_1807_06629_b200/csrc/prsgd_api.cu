@@ -295,7 +295,7 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging) {
     a.logits = c->buf.act_f32[L]; a.ldz = c->buf.ld[L];
     a.delta_bk = c->buf.delta_bk[L]; a.ld_bf = c->buf.ld[L];
     a.Y = c->Y; a.P = c->P; a.B = c->B; a.C = c->dims[L]; a.draw = dr;
-    a.row_losses = c->losses; a.draws = c->draws; a.active = act_mask;
+    a.row_losses = c->losses; a.draws = c->draws; a.active = act_mask; a.status = c->status;
     prof_begin(c, PRSGD_KERNEL_SOFTMAX);
     launch_pdl(softmax_ce_kernel, dim3(N, (c->B + 7) / 8), dim3(256), 0, c->stream, a);
     LAUNCH_CHECK(c);
@@ -328,10 +328,10 @@ int launch_average(prsgd_ctx* c) {
   prof_begin(c, PRSGD_KERNEL_AVERAGE);
   if (c->precision == PRSGD_PRECISION_BF16)
     average_rows_kernel<0, true><<<grid1d(threads, 256), 256, 0, c->stream>>>(c->params, c->N, c->m_pad, c->m_pad,
-                                                                            nullptr, c->shadow);
+                                                                            nullptr, c->shadow, c->status);
   else
     average_rows_kernel<0, false><<<grid1d(threads, 256), 256, 0, c->stream>>>(c->params, c->N, c->m_pad, c->m_pad,
-                                                                             nullptr, nullptr);
+                                                                             nullptr, nullptr, c->status);
   LAUNCH_CHECK(c);
   return PRSGD_OK;
 }
@@ -636,6 +636,23 @@ int prsgd_get_profile(prsgd_ctx* c, int32_t family, double* ms_total, int64_t* l
   if (launches) *launches = c->prof_count[family];
   c->prof_ms[family] = 0.0;
   c->prof_count[family] = 0;
+  return PRSGD_OK;
+}
+
+int prsgd_selftest_wait_expiry(prsgd_ctx* c, int32_t limit_us) {
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
+  if (limit_us < 1 || limit_us > 1000000) return fail(c, PRSGD_ERR_ARG, "limit_us must be in 1..1000000");
+  prof_begin(c, PRSGD_KERNEL_MISC);
+  wait_expiry_kernel<<<1, 32, 0, c->stream>>>(c->status, (long long)limit_us * 2000ll);
+  LAUNCH_CHECK(c);
+  return PRSGD_OK;
+}
+
+int prsgd_clear_device_error(prsgd_ctx* c) {
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
+  CUDA_TRY(c, cudaMemsetAsync(c->status, 0, sizeof(DeviceStatus), c->stream));
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  c->err.clear();
   return PRSGD_OK;
 }
 

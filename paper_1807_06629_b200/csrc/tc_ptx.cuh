@@ -47,7 +47,8 @@ constexpr long long kWaitLimitCycles = 4000000000ll;   // about 2 s at the SM cl
 // Bounded wait.  `abort_flag` lives in shared memory: once any wait of the CTA gives up, all others
 // return quickly.  On expiry the code `what` is recorded in the device status words.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          DeviceStatus* status, unsigned what) {
+                                          DeviceStatus* status, unsigned what,
+                                          long long limit_cycles = kWaitLimitCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   long long t0 = 0;
   for (uint32_t it = 1;; ++it) {
@@ -56,7 +57,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       if (*abort_flag) return false;
       const long long now = clock64();
       if (t0 == 0) t0 = now;
-      if (now - t0 > kWaitLimitCycles) {
+      if (now - t0 > limit_cycles) {
         *abort_flag = 1;
         if (atomicCAS(&status->error, 0u, what) == 0u) status->where = blockIdx.x;
         return false;

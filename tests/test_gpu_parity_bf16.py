@@ -187,3 +187,32 @@ def test_full_size_configs(torch_cuda, name, I):
     nxt = p.get_params_stacked()
     for k, i in enumerate(sample):
         assert rel_l2(nxt[i] - got[i], -w.gamma * G[k]) <= TOL_UPDATE
+
+
+def test_expired_wait_is_reported_and_the_context_recovers(torch_cuda):
+    """Failure path without a fault: a bounded wait runs out, the status word is set, later launches do
+    nothing, the host sees PRSGD_ERR_DEVICE_TIMEOUT, and after clearing the context continues bit for bit."""
+    from paper_1807_06629_b200 import binding
+    w = SMALL[1]
+    X, Y, x0 = make_inputs(w)
+    ref = make_ctx(w, X, Y, x0)
+    ref.local_steps(3)
+    want = ref.get_params_stacked()
+    p = make_ctx(w, X, Y, x0)
+    p.local_steps(1)
+    after1 = p.get_params_stacked()
+    p.selftest_wait_expiry(500)                          # ~0.5 ms wait on a barrier nobody signals
+    with pytest.raises(binding.PRSGDError) as e:
+        p.sync()
+    assert e.value.code == -6 and "expired" in str(e.value)
+    p.local_steps(2)                                     # every tensor-core launch now sees the status word: no-ops
+    with pytest.raises(binding.PRSGDError):
+        p.get_params_stacked()
+    p.clear_device_error()
+    assert np.array_equal(p.get_params_stacked(), after1)   # the two skipped iterations changed nothing
+    assert p.get_step() == 3
+    # start over from a clean state: the context is fully usable again
+    p.set_params(x0)
+    p.set_step(0)
+    p.local_steps(3)
+    assert np.array_equal(p.get_params_stacked(), want)
