@@ -20,6 +20,8 @@ What is implemented (all arithmetic in float64):
   beyond the mean-dynamics and telescoping invariants.
 * Algorithm 2 (time-varying rates, epochs of length K^s) and Algorithm 3
   (per-worker epoch lengths I_i) as schedules over the same step.
+* The local step with momentum used in the paper's experiment (heavy-ball form, momentum buffers
+  local by default; what happens to them at a restart is not stated in the paper).
 * The stochastic gradient of the workload: an MLP with ReLU hidden layers and
   softmax cross-entropy averaged over the minibatch.  The paper leaves F_i
   generic; this is the F_i of the workloads.
@@ -188,6 +190,29 @@ def mlp_grad_fn(dims: Sequence[int], X: np.ndarray, Y: np.ndarray, B: int, seed:
         return g
 
     return fn
+
+
+def pr_sgd_momentum(x: np.ndarray, v: np.ndarray, gamma: float, mu: float, I: int, T: int, grad_fn: GradFn,
+                    t0: int = 0, average_velocity: bool = False) -> Tuple[np.ndarray, np.ndarray]:
+    """Algorithm 1 with the local step of the paper's experiment: SGD with momentum mu (Experiment
+    section, figure captions: momentum 0.9).  Per worker, in the form of the library the paper used:
+        v_i <- mu * v_i + G_i ;   x_i <- x_i - gamma * v_i        (v_i starts at 0)
+    On an averaging iteration the models are averaged after the step.  The paper does not say what
+    happens to the momentum buffers at a restart: by default each worker keeps its own v_i;
+    with average_velocity=True they are averaged like the models.  Returns (x, v), copies.
+    """
+    x = np.array(x, dtype=np.float64, copy=True)
+    v = np.array(v, dtype=np.float64, copy=True)
+    N = x.shape[0]
+    for t in range(t0 + 1, t0 + T + 1):
+        G = np.stack([np.asarray(grad_fn(i, t, x[i]), dtype=np.float64) for i in range(N)])
+        v = mu * v + G
+        x = x - gamma * v
+        if I > 0 and t % I == 0:
+            x[:] = node_average(x)[None, :]
+            if average_velocity:
+                v[:] = node_average(v)[None, :]
+    return x, v
 
 
 # --------------------------------------------------------------------------

@@ -298,6 +298,45 @@ def test_alg3_with_equal_lengths_is_alg1_and_slow_workers_stand_still():
     assert np.allclose(h[1], one[1], atol=1e-15)                   # worker 1 took exactly one step
 
 
+# ------------------------------------------------------------- momentum local step
+def test_momentum_zero_is_plain_pr_sgd_and_first_step_is_a_gradient_step():
+    w, X, Y, x0 = _small_mlp_problem(N=3)
+    fn = orc.mlp_grad_fn(w.dims, X, Y, w.B, w.seed)
+    xs = np.tile(x0, (w.N, 1))
+    a, va = orc.pr_sgd_momentum(xs, np.zeros_like(xs), w.gamma, 0.0, 2, 6, fn)
+    assert np.allclose(a, orc.pr_sgd(xs, w.gamma, 2, 6, fn), atol=1e-15)
+    b, vb = orc.pr_sgd_momentum(xs, np.zeros_like(xs), w.gamma, 0.9, 0, 1, fn)
+    assert np.allclose(b, orc.pr_sgd(xs, w.gamma, 0, 1, fn), atol=1e-15)     # v^1 = G^1
+    assert np.allclose(vb, (xs - b) / w.gamma, atol=1e-12)
+
+
+def test_momentum_on_a_quadratic_matches_the_linear_recurrence():
+    # F(x) = a/2 (x - c)^2:  (x, v)_{t} = M (x - c, v)_{t-1},  M = [[1 - gamma a, -gamma mu], [a, mu]]
+    a, c, gam, mu, T = 1.7, 0.4, 0.1, 0.9, 25
+    x, v = orc.pr_sgd_momentum(np.array([[2.0]]), np.zeros((1, 1)), gam, mu, 0, T, lambda i, t, xi: a * (xi - c))
+    M = np.array([[1 - gam * a, -gam * mu], [a, mu]])
+    want = np.linalg.matrix_power(M, T) @ np.array([2.0 - c, 0.0])
+    assert x[0, 0] == pytest.approx(want[0] + c, abs=1e-13) and v[0, 0] == pytest.approx(want[1], abs=1e-13)
+
+
+def test_momentum_brute_force_and_velocity_choices():
+    a, c, g, mu = np.array([1.0, 3.0]), np.array([[2.0], [-1.0]]), 0.1, 0.5
+    x0_, x1_, v0_, v1_ = 0.5, 0.5, 0.0, 0.0
+    for t in range(1, 5):
+        v0_ = mu * v0_ + a[0] * (x0_ - c[0, 0]); x0_ = x0_ - g * v0_
+        v1_ = mu * v1_ + a[1] * (x1_ - c[1, 0]); x1_ = x1_ - g * v1_
+        if t % 2 == 0:
+            x0_ = x1_ = (x0_ + x1_) / 2
+    x, v = orc.pr_sgd_momentum(np.full((2, 1), 0.5), np.zeros((2, 1)), g, mu, 2, 4, _quad(a, c))
+    assert np.allclose(x[:, 0], [x0_, x1_], atol=1e-15) and np.allclose(v[:, 0], [v0_, v1_], atol=1e-15)
+    assert abs(v[0, 0] - v[1, 0]) > 1e-3                         # local momentum: buffers differ after the average
+    x2, v2 = orc.pr_sgd_momentum(np.full((2, 1), 0.5), np.zeros((2, 1)), g, mu, 2, 4, _quad(a, c), average_velocity=True)
+    assert v2[0, 0] == v2[1, 0] and x2[0, 0] == x2[1, 0]
+    # mean dynamics with momentum on a non-averaging iteration: xbar moves by -gamma * mean(v)
+    x3, v3 = orc.pr_sgd_momentum(x, v, g, mu, 2, 1, _quad(a, c), t0=4)
+    assert np.allclose(x3.mean(0), x.mean(0) - g * v3.mean(0), atol=1e-15)
+
+
 # ------------------------------------------------------- planted mistakes are caught
 def test_pins_catch_a_planted_mistake(monkeypatch):
     rng = np.random.default_rng(3)
