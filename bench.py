@@ -123,12 +123,13 @@ def ncu_traffic_per_launch(workload: str, family: str):
 
 
 # ----------------------------------------------------------------------------- byte model
-def algorithmic_bytes(w: synth.Workload, m_pad: int) -> dict:
+def algorithmic_bytes(w: synth.Workload, m_pad: int, momentum: bool = False) -> dict:
     """Algorithmic HBM bytes of one local iteration of all N workers, per kernel family.
 
     bf16 path: forward reads the bf16 shadow (2 B/param); dX reads it again for every layer but
     the first; the update reads and writes the fp32 master (4 + 4) and writes the shadow (2);
     activations / deltas are read and written once per use.  fp32 path: 4 B where bf16 has 2, no shadow.
+    With momentum the update also reads and writes the fp32 momentum buffer (+8 B/param).
     The stand-alone average reads and writes the store once (8 B/word, +2 for the shadow).
     """
     e = 2 if w.precision == 1 else 4
@@ -140,7 +141,7 @@ def algorithmic_bytes(w: synth.Workload, m_pad: int) -> dict:
         fwd += N * (wl * e + d[l] * 4 + B * d[l - 1] * e + B * d[l] * (e if l < L else 4))
         if l > 1:
             dx += N * (wl * e + B * d[l] * e + B * d[l - 1] * 2 * e)
-        upd += N * ((wl + d[l]) * (8 + (2 if w.precision == 1 else 0)) + B * (d[l] + d[l - 1]) * e)
+        upd += N * ((wl + d[l]) * (8 + (2 if w.precision == 1 else 0) + (8 if momentum else 0)) + B * (d[l] + d[l - 1]) * e)
     avg = N * m_pad * (8 + (2 if w.precision == 1 else 0))
     return {"forward": fwd, "dx": dx, "update": upd, "update_average": upd, "average": avg,
             "softmax": N * B * d[L] * (4 + 4 + e)}
@@ -210,10 +211,12 @@ def run_reference(args, w):
     }))
 
 
-def workload_config(w, extra=None):
+def workload_config(w, extra=None, momentum=None):
     c = {"workload": w.name, "N": w.N, "dims": list(w.dims), "B": w.B, "gamma": w.gamma, "I": w.I,
          "pool_samples": w.pool_samples, "precision": "bf16 operands / fp32 master" if w.precision else "fp32",
          "step": "one averaging period = prsgd_local_steps(I)"}
+    if momentum is not None:
+        c["momentum"] = momentum
     if extra:
         c.update(extra)
     return c
@@ -259,6 +262,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--interval", type=int, default=None, help="override the averaging interval I")
     ap.add_argument("--workers", type=int, default=None, help="override N (smaller cases for profiler captures)")
+    ap.add_argument("--momentum", type=float, default=None, help="local step with momentum mu (the paper's experiment used 0.9)")
     ap.add_argument("--update-tile", type=int, default=None, help="tile width of the update kernel (64 or 128)")
     ap.add_argument("--no-sweep", action="store_true", help="skip the averaging-kernel sweep")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle timing")
@@ -305,6 +309,8 @@ def main():
     p.set_params(x0)
     if args.update_tile is not None:
         p.set_option(binding.OPT_UPDATE_TILE, args.update_tile)
+    if args.momentum is not None:
+        p.enable_momentum(args.momentum)
     working_set = p.params.numel() * 4 + (p.shadow.numel() * 2 if p.shadow is not None else 0)
     need_flush = working_set <= 2 * L2_BYTES
     flush = torch.empty(3 * L2_BYTES // 4, dtype=torch.float32, device=dev) if need_flush else None
@@ -349,7 +355,7 @@ def main():
         p.local_steps(w.I)
     prof = p.get_profile()
     p.set_option(binding.OPT_PROFILE, 0)
-    bytes_iter = algorithmic_bytes(w, p.m_pad)
+    bytes_iter = algorithmic_bytes(w, p.m_pad, args.momentum is not None)
     fams = {k: v for k, v in prof.items() if v[1] > 0 and k in bytes_iter}
     dom = max(fams, key=lambda k: fams[k][0])
     L = len(w.dims) - 1
@@ -391,7 +397,8 @@ def main():
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.precision else "f32", "data": "synthetic",
         "config": workload_config(w, {"l2": "L2 flushed between timed steps" if need_flush else
                                       "parameter store + shadow larger than L2",
-                                      "multi_gpu": "independent replicas, one per rank" if world > 1 else "single GPU"}),
+                                      "multi_gpu": "independent replicas, one per rank" if world > 1 else "single GPU"},
+                                  momentum=args.momentum),
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline,
         "gemm_tflops": tflops, "gemm_frac_of_bf16_peak": tflops / peaks["bf16_tflops_sustained"],
     }

@@ -171,6 +171,18 @@ int prsgd_set_active(prsgd_ctx* ctx, const uint8_t* h_mask);
 int prsgd_get_step(prsgd_ctx* ctx, int64_t* t);
 int prsgd_set_step(prsgd_ctx* ctx, int64_t t);
 
+/* Local step with momentum, as in the paper's experiment (Experiment section, figure captions:
+ * momentum 0.9): per worker v_i <- mu v_i + G_i, x_i <- x_i - gamma v_i, v_i starting at 0.
+ * d_velocity: caller-owned device memory of the same size as the parameter store (N*m_pad*4
+ * bytes, 256-byte aligned), zeroed by this call and laid out like the store.  The paper does not
+ * say what happens to the momentum buffers at a restart: with average_velocity = 0 every worker
+ * keeps its own, with 1 they are averaged together with the models.  While momentum is on, an
+ * averaging iteration runs as update followed by the averaging kernel (no fused form).
+ * d_velocity = NULL switches back to plain SGD.  mu in [0, 1). */
+int prsgd_enable_momentum(prsgd_ctx* ctx, float mu, void* d_velocity, int average_velocity);
+/* The momentum buffers, [N][m] in canonical order.  Synchronises the stream. */
+int prsgd_get_velocity_stacked(prsgd_ctx* ctx, float* dst, int dst_on_device);
+
 /* Options.  PRSGD_OPT_FUSED_AVERAGE (default 1): on an averaging iteration the
  * update and the average run as one pass over the store instead of an update
  * pass followed by prsgd_average's pass; both produce identical bits. */

@@ -33,7 +33,7 @@ EXPORTS = [
     "prsgd_get_draws", "prsgd_set_lr", "prsgd_set_interval", "prsgd_set_active", "prsgd_get_step",
     "prsgd_set_step", "prsgd_set_option", "prsgd_get_launch_count", "prsgd_get_profile", "prsgd_sync", "prsgd_last_error",
     "prsgd_average_rows", "prsgd_draw_block", "prsgd_mean_rows_noalloc", "prsgd_selftest_wait_expiry",
-    "prsgd_clear_device_error",
+    "prsgd_clear_device_error", "prsgd_enable_momentum", "prsgd_get_velocity_stacked",
 ]
 NOALLOC_MAX_M = 1 << 20
 
@@ -83,6 +83,8 @@ def _load() -> C.CDLL:
         "prsgd_sync": (C.c_int, [vp]),
         "prsgd_selftest_wait_expiry": (C.c_int, [vp, i32]),
         "prsgd_clear_device_error": (C.c_int, [vp]),
+        "prsgd_enable_momentum": (C.c_int, [vp, C.c_float, vp, C.c_int]),
+        "prsgd_get_velocity_stacked": (C.c_int, [vp, vp, C.c_int]),
         "prsgd_last_error": (C.c_char_p, [vp]),
         "prsgd_average_rows": (C.c_int, [vp, i64, i64, i64, vp]),
         "prsgd_draw_block": (u64, [u64, i32, i64, u64]),
@@ -264,6 +266,17 @@ class PRSGD:
     def get_draws(self) -> np.ndarray:
         out = np.empty(self.N, dtype=np.int32)
         self._call(lib.prsgd_get_draws, _host_ptr(out))
+        return out
+
+    def enable_momentum(self, mu: float, average_velocity: bool = False):
+        """Allocate the momentum buffers (same size as the store) and switch the local step to SGD with momentum."""
+        with torch.cuda.device(self.device):
+            self.velocity = torch.empty(self.N * self.m_pad, dtype=torch.float32, device=self.device)
+        self._call(lib.prsgd_enable_momentum, mu, self.velocity.data_ptr(), 1 if average_velocity else 0)
+
+    def get_velocity_stacked(self) -> np.ndarray:
+        out = np.empty((self.N, self.m), dtype=np.float32)
+        self._call(lib.prsgd_get_velocity_stacked, _host_ptr(out), 0)
         return out
 
     # ---- schedule ---------------------------------------------------------------

@@ -26,6 +26,7 @@ struct TcLayerMaps {
   CUtensorMap shadow_k;     // bf16 W_l  dims {d_in, d_out, N}, box {64, 128, 1}: forward A tiles, shadow stores
   CUtensorMap shadow_mn;    // same tensor, box {64, 64, 1}: backward A tiles (W^T, MN-major)
   CUtensorMap master;       // fp32 W_l  dims {d_in, d_out, N}, box {32, 128, 1}: update loads and stores
+  CUtensorMap velocity;     // fp32 momentum buffer of W_l, same geometry as master (valid once momentum is enabled)
   CUtensorMap act_in;       // bf16 a_{l-1} dims {ld, B, N}, box {64, B, 1} (layer 1: the data pool {d0, P, N})
   CUtensorMap delta_out;    // bf16 dZ_l  dims {ld, B, N}, box {64, B, 1}
 };
@@ -294,6 +295,7 @@ struct UpdateArgs {
   int B, N;
   int tiles_m, tiles_n;
   float gamma;
+  float mu;
   int pool;
   DrawArgs draw;
   const uint8_t* active;
@@ -306,24 +308,29 @@ constexpr int kUpdThreads = 224;          // warp 0 loader, 1 MMA, 2 storer, 3..
 // 128 x 32) followed by a region that first holds the operands (two dZ boxes and TN/64 activation
 // boxes of {64, B}) and later, once the MMA has consumed them, the bf16 output tile (TN/64 boxes
 // of 128 x 64).  TN = 64 gives four stages, TN = 128 two.
-template <int TN> struct UpdCfg {
-  static constexpr int kStages = TN == 64 ? 4 : 2;
+template <int TN, bool MOM> struct UpdCfg {
+  static constexpr int kStages = (TN == 64 && !MOM) ? 4 : 2;
   static constexpr uint32_t kMaster = 128u * TN * 4u;
+  static constexpr uint32_t kVel = MOM ? kMaster : 0u;          // momentum tile right after the master tile
   static constexpr uint32_t kOut = 128u * TN * 2u;
   __host__ __device__ static uint32_t ops_bytes(int B) { return (uint32_t)(2 + TN / 64) * (uint32_t)B * 128u; }
   __host__ __device__ static uint32_t region(int B) { return ops_bytes(B) > kOut ? ops_bytes(B) : kOut; }
-  __host__ __device__ static uint32_t stage(int B) { return kMaster + region(B); }
+  __host__ __device__ static uint32_t stage(int B) { return kMaster + kVel + region(B); }
   static size_t smem(int B) { return (size_t)kStages * stage(B) + 1024 + 256; }
 };
 
-template <bool FUSE, int TN>
+// MOM: the local step of the paper's experiment, v <- mu v + G, x <- x - gamma v; the momentum tile
+// travels with the master tile (loaded, updated in shared memory, stored back).  Not combined with FUSE.
+template <bool FUSE, int TN, bool MOM>
 __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_constant__ CUtensorMap mapDelta,
                                                                    const __grid_constant__ CUtensorMap mapAct,
                                                                    const __grid_constant__ CUtensorMap mapMaster,
                                                                    const __grid_constant__ CUtensorMap mapShadow,
+                                                                   const __grid_constant__ CUtensorMap mapVel,
                                                                    const UpdateArgs a) {
   using namespace ptx;
-  using Cfg = UpdCfg<TN>;
+  static_assert(!(FUSE && MOM), "the fused average is not built for the momentum step");
+  using Cfg = UpdCfg<TN, MOM>;
   constexpr int S = Cfg::kStages;
   constexpr int NB32 = TN / 32, NB64 = TN / 64;
   extern __shared__ uint8_t smem_raw[];
@@ -332,7 +339,8 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
   uint8_t* gen = smem_raw + (base - raw);
   const uint32_t stage_bytes = Cfg::stage(a.B);
   auto master_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes; };
-  auto ops_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes + Cfg::kMaster; };
+  auto vel_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes + Cfg::kMaster; };
+  auto ops_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes + Cfg::kMaster + Cfg::kVel; };
   const uint32_t bar0 = base + (uint32_t)S * stage_bytes;
   auto full_ops = [&](int s) { return bar0 + 8u * s; };
   auto full_w = [&](int s) { return bar0 + 32u + 8u * s; };
@@ -357,6 +365,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
     fence_mbar_init();
     prefetch_tensormap(&mapDelta); prefetch_tensormap(&mapAct);
     prefetch_tensormap(&mapMaster); prefetch_tensormap(&mapShadow);
+    if (MOM) prefetch_tensormap(&mapVel);
   }
   if (warp == 1) { tmem_alloc(smem_u32(tmem_slot), 256u); tmem_relinquish(); }
   tc_fence_before();
@@ -394,9 +403,13 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
         tma_load_3d(ops + op_box, &mapDelta, full_ops(s), m0 + 64, 0, n);
 #pragma unroll
         for (int h = 0; h < NB64; ++h) tma_load_3d(ops + (2u + h) * op_box, &mapAct, full_ops(s), n0 + 64 * h, row0, n);
-        mbar_expect_tx(full_w(s), Cfg::kMaster);
+        mbar_expect_tx(full_w(s), Cfg::kMaster + Cfg::kVel);
 #pragma unroll
         for (int q = 0; q < NB32; ++q) tma_load_3d(master_u32(s) + q * 16384u, &mapMaster, full_w(s), n0 + 32 * q, m0, n);
+        if (MOM) {
+#pragma unroll
+          for (int q = 0; q < NB32; ++q) tma_load_3d(vel_u32(s) + q * 16384u, &mapVel, full_w(s), n0 + 32 * q, m0, n);
+        }
         ++it;
       }
     }
@@ -436,6 +449,10 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
     auto store_tile = [&](int s, int m0, int n0, int n) {
 #pragma unroll
       for (int q = 0; q < NB32; ++q) tma_store_3d(&mapMaster, master_u32(s) + q * 16384u, n0 + 32 * q, m0, n);
+      if (MOM) {
+#pragma unroll
+        for (int q = 0; q < NB32; ++q) tma_store_3d(&mapVel, vel_u32(s) + q * 16384u, n0 + 32 * q, m0, n);
+      }
 #pragma unroll
       for (int h = 0; h < NB64; ++h) tma_store_3d(&mapShadow, ops_u32(s) + h * 16384u, n0 + 64 * h, m0, n);
     };
@@ -495,7 +512,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
         if (!ok) break;
         tc_fence_after();
         uint8_t* mst = gen + (size_t)s * stage_bytes;
-        uint8_t* stg = mst + Cfg::kMaster;
+        uint8_t* stg = mst + Cfg::kMaster + Cfg::kVel;
         const bool last = FUSE && n == a.N - 1;
 #pragma unroll
         for (int c = 0; c < NB32; ++c) {
@@ -506,11 +523,20 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
           for (int j = 0; j < 8; ++j) {
             float4* pw = reinterpret_cast<float4*>(mst + c * 16384 + row_off + (((uint32_t)j ^ sw) << 4));
             float4 x = *pw;
+            float4 g4 = make_float4(__uint_as_float(v[4 * j + 0]), __uint_as_float(v[4 * j + 1]),
+                                    __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+            if (MOM) {                                      // v <- mu v + G, kept in place next to the master tile
+              float4* pv = reinterpret_cast<float4*>(mst + Cfg::kMaster + c * 16384 + row_off + (((uint32_t)j ^ sw) << 4));
+              const float4 vo = *pv;
+              g4.x = fmaf(a.mu, vo.x, g4.x); g4.y = fmaf(a.mu, vo.y, g4.y);
+              g4.z = fmaf(a.mu, vo.z, g4.z); g4.w = fmaf(a.mu, vo.w, g4.w);
+              *pv = g4;
+            }
             if (upd) {
-              x.x = fmaf(-a.gamma, __uint_as_float(v[4 * j + 0]), x.x);
-              x.y = fmaf(-a.gamma, __uint_as_float(v[4 * j + 1]), x.y);
-              x.z = fmaf(-a.gamma, __uint_as_float(v[4 * j + 2]), x.z);
-              x.w = fmaf(-a.gamma, __uint_as_float(v[4 * j + 3]), x.w);
+              x.x = fmaf(-a.gamma, g4.x, x.x);
+              x.y = fmaf(-a.gamma, g4.y, x.y);
+              x.z = fmaf(-a.gamma, g4.z, x.z);
+              x.w = fmaf(-a.gamma, g4.w, x.w);
             }
             if (FUSE) {
               constexpr int F = FUSE ? 1 : 0;
@@ -564,6 +590,8 @@ struct BiasArgs {
   int ld[PRSGD_MAX_LAYERS];
   const uint16_t* delta_bk[PRSGD_MAX_LAYERS];
   const DeviceStatus* status;
+  float* vel;              // momentum buffers laid out like the store, or nullptr
+  float mu;
 };
 
 __global__ void __launch_bounds__(128) bias_update_kernel(const BiasArgs a) {
@@ -576,6 +604,11 @@ __global__ void __launch_bounds__(128) bias_update_kernel(const BiasArgs a) {
   float g = 0.f;
   for (int b = 0; b < a.B; ++b) g += __uint_as_float((uint32_t)__ldg(d + (int64_t)b * a.ld[l]) << 16);
   float* bp = a.params + (int64_t)n * a.m_pad + a.b_off[l] + j;
+  if (a.vel != nullptr) {
+    float* vp = a.vel + (int64_t)n * a.m_pad + a.b_off[l] + j;
+    g = fmaf(a.mu, *vp, g);
+    *vp = g;
+  }
   *bp = fmaf(-a.gamma, g, *bp);
 }
 
@@ -625,10 +658,11 @@ inline int tc_create(prsgd_ctx* c, std::string* err) {
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_stream_kernel<TC_FWD_RELU>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_stream_kernel<TC_FWD_LINEAR>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_stream_kernel<TC_DX>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<false, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<64>::smem(c->B));
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<true, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<64>::smem(c->B));
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<false, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<128>::smem(c->B));
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<true, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<128>::smem(c->B));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<false, 64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<64, false>::smem(c->B));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<true, 64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<64, false>::smem(c->B));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<false, 128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<128, false>::smem(c->B));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<true, 128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<128, false>::smem(c->B));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<false, 64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<64, true>::smem(c->B));
   if (e != cudaSuccess) {
     *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e);
     delete st;
@@ -641,6 +675,18 @@ inline int tc_create(prsgd_ctx* c, std::string* err) {
 inline void tc_destroy(prsgd_ctx* c) {
   delete static_cast<TcState*>(c->tc);
   c->tc = nullptr;
+}
+
+inline int tc_bind_velocity(prsgd_ctx* c, std::string* err) {
+  TcState* st = static_cast<TcState*>(c->tc);
+  for (int l = 1; l <= c->L; ++l) {
+    const Layer& ly = c->layer[l - 1];
+    const uint64_t din = ly.d_in, dout = ly.d_out;
+    int rc = make_map3(&st->layer[l - 1].velocity, true, c->velocity + ly.w_off, din, dout, (uint64_t)c->N, din * 4,
+                       (uint64_t)c->m_pad * 4, 32, 128, err);
+    if (rc != PRSGD_OK) return rc;
+  }
+  return PRSGD_OK;
 }
 
 inline int tc_bind_data(prsgd_ctx* c, std::string* err) {
@@ -688,21 +734,25 @@ inline void tc_launch_dx(prsgd_ctx* c, int l, const DrawArgs& dr, const uint8_t*
              st->layer[l - 1].delta_out, a);
 }
 
-template <int TN>
+template <int TN, bool MOM>
 inline void tc_launch_update_tn(prsgd_ctx* c, int l, const DrawArgs& dr, const uint8_t* active, bool fuse) {
   TcState* st = static_cast<TcState*>(c->tc);
   const Layer& ly = c->layer[l - 1];
   UpdateArgs a{};
   a.B = c->B; a.N = c->N; a.tiles_m = (ly.d_out + 127) / 128; a.tiles_n = (ly.d_in + TN - 1) / TN;
-  a.gamma = c->gamma; a.pool = l == 1; a.draw = dr; a.active = active; a.status = c->status;
+  a.gamma = c->gamma; a.mu = c->mu; a.pool = l == 1; a.draw = dr; a.active = active; a.status = c->status;
   const int items = a.tiles_m * a.tiles_n * (fuse ? 1 : c->N);
   const int grid = items < st->num_sms ? items : st->num_sms;
   const TcLayerMaps& mp = st->layer[l - 1];
-  const size_t smem = UpdCfg<TN>::smem(c->B);
-  if (fuse)
-    launch_pdl(tc_update_kernel<true, TN>, dim3(grid), kUpdThreads, smem, c->stream, mp.delta_out, mp.act_in, mp.master, mp.shadow_k, a);
-  else
-    launch_pdl(tc_update_kernel<false, TN>, dim3(grid), kUpdThreads, smem, c->stream, mp.delta_out, mp.act_in, mp.master, mp.shadow_k, a);
+  const size_t smem = UpdCfg<TN, MOM>::smem(c->B);
+  if constexpr (MOM) {
+    launch_pdl(tc_update_kernel<false, TN, true>, dim3(grid), kUpdThreads, smem, c->stream, mp.delta_out, mp.act_in, mp.master, mp.shadow_k, mp.velocity, a);
+  } else {
+    if (fuse)
+      launch_pdl(tc_update_kernel<true, TN, false>, dim3(grid), kUpdThreads, smem, c->stream, mp.delta_out, mp.act_in, mp.master, mp.shadow_k, mp.master, a);
+    else
+      launch_pdl(tc_update_kernel<false, TN, false>, dim3(grid), kUpdThreads, smem, c->stream, mp.delta_out, mp.act_in, mp.master, mp.shadow_k, mp.master, a);
+  }
 }
 
 // Tile width: forced by PRSGD_OPT_UPDATE_TILE, else chosen per launch.  Wide tiles need fewer TMA
@@ -712,14 +762,18 @@ inline void tc_launch_update_tn(prsgd_ctx* c, int l, const DrawArgs& dr, const u
 inline void tc_launch_update(prsgd_ctx* c, int l, const DrawArgs& dr, const uint8_t* active, bool fuse) {
   const TcState* st = static_cast<const TcState*>(c->tc);
   const Layer& ly = c->layer[l - 1];
+  if (c->velocity != nullptr) {            // momentum step: 64-wide tiles (two stages of master + momentum + output)
+    tc_launch_update_tn<64, true>(c, l, dr, active, false);
+    return;
+  }
   int tile = c->upd_tile;
   if (tile == 0) {
     const int64_t tiles128 = (int64_t)((ly.d_out + 127) / 128) * ((ly.d_in + 127) / 128);
     if (fuse) tile = 2 * tiles128 >= 3 * (int64_t)st->num_sms ? 128 : 64;
     else tile = (c->B <= 32 && tiles128 * c->N >= 32 * (int64_t)st->num_sms) ? 128 : 64;
   }
-  if (tile == 128) tc_launch_update_tn<128>(c, l, dr, active, fuse);
-  else tc_launch_update_tn<64>(c, l, dr, active, fuse);
+  if (tile == 128) tc_launch_update_tn<128, false>(c, l, dr, active, fuse);
+  else tc_launch_update_tn<64, false>(c, l, dr, active, fuse);
 }
 
 // Bias step of all layers (after the last dZ has been formed).  On an averaging iteration it is followed
@@ -728,7 +782,7 @@ inline void tc_launch_update(prsgd_ctx* c, int l, const DrawArgs& dr, const uint
 inline void tc_launch_bias(prsgd_ctx* c, const uint8_t* active) {
   BiasArgs a{};
   a.params = c->params; a.m_pad = c->m_pad; a.L = c->L; a.B = c->B; a.gamma = c->gamma; a.active = active;
-  a.status = c->status;
+  a.status = c->status; a.vel = c->velocity; a.mu = c->mu;
   int dmax = 1;
   for (int l = 1; l <= c->L; ++l) {
     const Layer& ly = c->layer[l - 1];

@@ -39,6 +39,8 @@ struct GemmF32Args {
   const float* mask_src; // DX: a_{l-1} of the same shape as out (ReLU mask: a > 0)
   float gamma;
   const uint8_t* active; // per-worker flag or nullptr
+  float* vel;            // DW: momentum buffers laid out like the store, or nullptr
+  float mu;
 };
 
 __device__ __forceinline__ const float* operand_ptr(const OperandF32& o, int n, const DrawArgs& d) {
@@ -187,14 +189,26 @@ __global__ void __launch_bounds__(256) gemm_f32_kernel(const GemmF32Args g) {
           int j = j0 + tx * 4 + c;
           if (j >= g.Nn) continue;
           float w = W[(int64_t)i * g.Nn + j];
-          float xi = is_active ? fmaf(-g.gamma, acc[r][c], w) : w;
+          float step = acc[r][c];
+          if (g.vel != nullptr && is_active) {             // v <- mu v + G ; x <- x - gamma v
+            float* vp = g.vel + (int64_t)n * g.out_worker_stride + g.w_off + (int64_t)i * g.Nn + j;
+            step = fmaf(g.mu, *vp, step);
+            *vp = step;
+          }
+          float xi = is_active ? fmaf(-g.gamma, step, w) : w;
           if (FUSE) sum[r][c] += xi;
           else W[(int64_t)i * g.Nn + j] = xi;
         }
       }
       if (do_bias && tid < TM && i0 + tid < g.M) {
         float* bp = row + g.b_off + i0 + tid;
-        float xi = is_active ? fmaf(-g.gamma, bsum, *bp) : *bp;
+        float bstep = bsum;
+        if (g.vel != nullptr && is_active) {
+          float* vp = g.vel + (int64_t)n * g.out_worker_stride + g.b_off + i0 + tid;
+          bstep = fmaf(g.mu, *vp, bstep);
+          *vp = bstep;
+        }
+        float xi = is_active ? fmaf(-g.gamma, bstep, *bp) : *bp;
         if (FUSE) bias_sum_all += xi;
         else *bp = xi;
       }

@@ -216,7 +216,7 @@ void launch_gemm_f32(prsgd_ctx* c, const GemmF32Args& g) {
 int step_f32(prsgd_ctx* c, int64_t t, bool averaging) {
   const int L = c->L, B = c->B, N = c->N;
   const uint8_t* act_mask = c->has_mask ? c->active : nullptr;
-  const bool fuse = averaging && c->fused_average;
+  const bool fuse = averaging && c->fused_average && c->velocity == nullptr;   // the momentum step is not fused
   const DrawArgs dr = draw_args(c, t);
   const float* X = static_cast<const float*>(c->X);
 
@@ -270,7 +270,7 @@ int step_f32(prsgd_ctx* c, int64_t t, bool averaging) {
     else        g.Bo = {c->buf.act_f32[l - 1], (int64_t)B * ly.d_in, ly.d_in, 1, 0};
     g.M = ly.d_out; g.Nn = ly.d_in; g.K = B; g.N = N; g.draw = dr;
     g.out = c->params; g.out_worker_stride = c->m_pad; g.w_off = ly.w_off; g.b_off = ly.b_off;
-    g.gamma = c->gamma; g.active = act_mask;
+    g.gamma = c->gamma; g.active = act_mask; g.vel = c->velocity; g.mu = c->mu;
     prof_begin(c, fuse ? PRSGD_KERNEL_UPDATE_AVERAGE : PRSGD_KERNEL_UPDATE);
     if (fuse) launch_gemm_f32<64, false, false, EPI_DW, true>(c, g);
     else      launch_gemm_f32<64, false, false, EPI_DW, false>(c, g);
@@ -283,7 +283,7 @@ int step_f32(prsgd_ctx* c, int64_t t, bool averaging) {
 int step_bf16(prsgd_ctx* c, int64_t t, bool averaging) {
   const int L = c->L, N = c->N;
   const uint8_t* act_mask = c->has_mask ? c->active : nullptr;
-  const bool fuse = averaging && c->fused_average;
+  const bool fuse = averaging && c->fused_average && c->velocity == nullptr;   // the momentum step is not fused
   const DrawArgs dr = draw_args(c, t);
   for (int l = 1; l <= L; ++l) {
     prof_begin(c, PRSGD_KERNEL_FORWARD);
@@ -333,6 +333,12 @@ int launch_average(prsgd_ctx* c) {
     average_rows_kernel<0, false><<<grid1d(threads, 256), 256, 0, c->stream>>>(c->params, c->N, c->m_pad, c->m_pad,
                                                                              nullptr, nullptr, c->status);
   LAUNCH_CHECK(c);
+  if (c->velocity != nullptr && c->average_velocity) {     // momentum buffers averaged like the models
+    prof_begin(c, PRSGD_KERNEL_AVERAGE);
+    average_rows_kernel<0, false><<<grid1d(threads, 256), 256, 0, c->stream>>>(c->velocity, c->N, c->m_pad, c->m_pad,
+                                                                             nullptr, nullptr, c->status);
+    LAUNCH_CHECK(c);
+  }
   return PRSGD_OK;
 }
 
@@ -508,7 +514,7 @@ int prsgd_local_steps(prsgd_ctx* c, int64_t k) {
     const bool averaging = c->I > 0 && (t % c->I) == 0;
     int rc = c->precision == PRSGD_PRECISION_BF16 ? step_bf16(c, t, averaging) : step_f32(c, t, averaging);
     if (rc != PRSGD_OK) return rc;
-    if (averaging && !c->fused_average) {
+    if (averaging && (!c->fused_average || c->velocity != nullptr)) {
       rc = launch_average(c);
       if (rc != PRSGD_OK) return rc;
     }
@@ -541,6 +547,37 @@ int prsgd_get_average(prsgd_ctx* c, float* dst, int dst_on_device) {
   }
   if (!dst_on_device) return check_device_status(c);
   return PRSGD_OK;
+}
+
+int prsgd_enable_momentum(prsgd_ctx* c, float mu, void* d_velocity, int average_velocity) {
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
+  if (d_velocity == nullptr) {                 // back to plain SGD
+    c->velocity = nullptr; c->mu = 0.f; c->average_velocity = 0;
+    return PRSGD_OK;
+  }
+  if (!(mu >= 0.f && mu < 1.f)) return fail(c, PRSGD_ERR_ARG, "mu must be in [0, 1)");
+  if (!aligned(d_velocity, 256)) return fail(c, PRSGD_ERR_ALIGN, "d_velocity must be 256-byte aligned");
+  CUDA_TRY(c, cudaMemsetAsync(d_velocity, 0, (size_t)c->N * c->m_pad * 4, c->stream));
+  c->velocity = static_cast<float*>(d_velocity); c->mu = mu; c->average_velocity = average_velocity != 0;
+  if (c->precision == PRSGD_PRECISION_BF16) {
+    std::string terr;
+    int trc = tc_bind_velocity(c, &terr);
+    if (trc != PRSGD_OK) { c->velocity = nullptr; c->mu = 0.f; return fail(c, trc, terr); }
+  }
+  return PRSGD_OK;
+}
+
+int prsgd_get_velocity_stacked(prsgd_ctx* c, float* dst, int dst_on_device) {
+  (void)dst_on_device;
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
+  if (!dst) return fail(c, PRSGD_ERR_ARG, "dst is NULL");
+  if (!c->velocity) return fail(c, PRSGD_ERR_STATE, "momentum is not enabled");
+  float* keep = c->params;
+  c->params = c->velocity;                     // same row layout: reuse the canonical gather
+  int rc = copy_canonical(c, dst, 0, c->N, false);
+  c->params = keep;
+  if (rc != PRSGD_OK) return rc;
+  return check_device_status(c);
 }
 
 int prsgd_get_losses(prsgd_ctx* c, float* h_dst) {

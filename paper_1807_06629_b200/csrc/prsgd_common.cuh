@@ -88,6 +88,9 @@ struct prsgd_ctx {
   int I = 0;
   int64_t t = 0;
   int fused_average = 1;
+  float mu = 0.f;                // momentum of the local step (0 = plain SGD)
+  float* velocity = nullptr;     // [N][m_pad] fp32 momentum buffers, caller-owned
+  int average_velocity = 0;      // average the buffers together with the models
   int upd_tile = 0;              // column width of the update kernel's tile: 0 = chosen per launch, 64 or 128
   int64_t launches = 0;
   int64_t m = 0, m_pad = 0;

@@ -189,6 +189,32 @@ def test_full_size_configs(torch_cuda, name, I):
         assert rel_l2(nxt[i] - got[i], -w.gamma * G[k]) <= TOL_UPDATE
 
 
+@pytest.mark.parametrize("avg_v", [False, True])
+def test_momentum_step_on_the_tensor_core_path(torch_cuda, avg_v):
+    """v <- mu v + G, x <- x - gamma v in the update kernel's epilogue; hidden biases +-6 so no ReLU can switch."""
+    for w in (SMALL[1], SMALL[3], SMALL[4]):
+        X, Y, x0 = make_inputs(w)
+        x0 = with_margin(x0, w.dims)
+        p = make_ctx(w, X, Y, x0)
+        p.enable_momentum(0.9, average_velocity=avg_v)
+        fn = orc.mlp_grad_fn(w.dims, X.astype(np.float64), Y, w.B, w.seed)
+        xs = np.tile(x0, (w.N, 1)).astype(np.float64)
+        T = 2 * w.I + 1
+        p.local_steps(T)
+        want_x, want_v = orc.pr_sgd_momentum(xs, np.zeros_like(xs), w.gamma, 0.9, w.I, T, fn, average_velocity=avg_v)
+        got_x, got_v = p.get_params_stacked(), p.get_velocity_stacked()
+        assert rel_l2(got_x, want_x) <= TOL_PERIOD
+        assert rel_l2(got_x - xs, want_x - xs) <= 2e-2, rel_l2(got_x - xs, want_x - xs)
+        # averaged buffers keep only the common part of the gradients: smaller norm, same absolute bf16 noise
+        assert rel_l2(got_v, want_v) <= (5e-2 if avg_v else 2e-2), rel_l2(got_v, want_v)
+        # shadow still tracks the master
+        import torch
+        store = p.params.cpu().numpy().reshape(w.N, p.m_pad)
+        shadow = p.shadow.view(torch.int16).cpu().numpy().view(np.uint16).reshape(w.N, p.m_pad)
+        a, n = p.layout.w_off[0], w.dims[0] * w.dims[1]
+        assert np.array_equal(shadow[:, a:a + n], synth.bf16_bits(store[:, a:a + n]))
+
+
 def test_expired_wait_is_reported_and_the_context_recovers(torch_cuda):
     """Failure path without a fault: a bounded wait runs out, the status word is set, later launches do
     nothing, the host sees PRSGD_ERR_DEVICE_TIMEOUT, and after clearing the context continues bit for bit."""

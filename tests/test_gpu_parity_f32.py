@@ -231,3 +231,24 @@ def test_ragged_shapes(torch_cuda, N, dims, B):
     p.local_steps(w.I)
     want = oracle_run(w, X, Y, np.tile(x0, (N, 1)), 0, w.I)
     assert rel_l2(p.get_params_stacked(), want) <= TOL_PERIOD
+
+
+@pytest.mark.parametrize("avg_v", [False, True])
+def test_momentum_step_matches_oracle(torch_cuda, avg_v):
+    """Local step of the paper's experiment (momentum 0.9): parameters and momentum buffers over two periods."""
+    w = synth.WORKLOADS["cfg1"]
+    X, Y, x0 = make_inputs(w)
+    p = make_ctx(w, X, Y, x0)
+    p.enable_momentum(0.9, average_velocity=avg_v)
+    fn = orc.mlp_grad_fn(w.dims, X.astype(np.float64), Y, w.B, w.seed)
+    xs = np.tile(x0, (w.N, 1)).astype(np.float64)
+    p.local_steps(1)
+    x1, v1 = orc.pr_sgd_momentum(xs, np.zeros_like(xs), w.gamma, 0.9, w.I, 1, fn)
+    assert rel_l2(p.get_params_stacked(), x1) <= TOL_STEP
+    assert rel_l2(p.get_velocity_stacked(), v1) <= 1e-5
+    p.local_steps(2 * w.I - 1)
+    x2, v2 = orc.pr_sgd_momentum(xs, np.zeros_like(xs), w.gamma, 0.9, w.I, 2 * w.I, fn, average_velocity=avg_v)
+    got_x, got_v = p.get_params_stacked(), p.get_velocity_stacked()
+    assert rel_l2(got_x, x2) <= TOL_PERIOD and rel_l2(got_v, v2) <= 1e-3
+    assert all(np.array_equal(got_x[i], got_x[0]) for i in range(w.N))
+    assert all(np.array_equal(got_v[i], got_v[0]) for i in range(w.N)) == avg_v
