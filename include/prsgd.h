@@ -171,6 +171,24 @@ int prsgd_set_active(prsgd_ctx* ctx, const uint8_t* h_mask);
 int prsgd_get_step(prsgd_ctx* ctx, int64_t* t);
 int prsgd_set_step(prsgd_ctx* ctx, int64_t t);
 
+/* Workers spread over several GPUs (one context per GPU, each holding a shard of the N workers).
+ * Inside an epoch workers need no synchronisation; the only exchange is the node average, which the
+ * paper suggests to obtain by an all-reduce of the local models (Section 2, "Communication
+ * Reduction").  The library provides the two local halves; the all-reduce of the m_pad-float row
+ * between them belongs to the caller (NCCL).
+ *  - prsgd_set_worker_offset: global index of this context's row 0; the minibatch draw of local
+ *    row i is that of worker first_worker + i.
+ *  - prsgd_partial_sum: d_dst[j] = sum over the local rows of P[i][j], fp32 in row order, for the
+ *    padded columns j in [col0, col0 + ncols); d_dst is a device row of m_pad floats.
+ *  - prsgd_assign_rows: every local row (and the bf16 shadow) gets d_src[j] / divisor on the same
+ *    column range; with divisor = the global N this is the restart at the node average.
+ * col0 and ncols are multiples of 4 (column ranges let the caller pipeline the all-reduce chunk by
+ * chunk); rows are 16-byte aligned device pointers.  With a single context,
+ * partial_sum + assign_rows(divisor = N) leaves the same bits as prsgd_average.  Asynchronous. */
+int prsgd_set_worker_offset(prsgd_ctx* ctx, int32_t first_worker);
+int prsgd_partial_sum(prsgd_ctx* ctx, float* d_dst, int64_t col0, int64_t ncols);
+int prsgd_assign_rows(prsgd_ctx* ctx, const float* d_src, float divisor, int64_t col0, int64_t ncols);
+
 /* Local step with momentum, as in the paper's experiment (Experiment section, figure captions:
  * momentum 0.9): per worker v_i <- mu v_i + G_i, x_i <- x_i - gamma v_i, v_i starting at 0.
  * d_velocity: caller-owned device memory of the same size as the parameter store (N*m_pad*4

@@ -34,6 +34,7 @@ EXPORTS = [
     "prsgd_set_step", "prsgd_set_option", "prsgd_get_launch_count", "prsgd_get_profile", "prsgd_sync", "prsgd_last_error",
     "prsgd_average_rows", "prsgd_draw_block", "prsgd_mean_rows_noalloc", "prsgd_selftest_wait_expiry",
     "prsgd_clear_device_error", "prsgd_enable_momentum", "prsgd_get_velocity_stacked",
+    "prsgd_set_worker_offset", "prsgd_partial_sum", "prsgd_assign_rows",
 ]
 NOALLOC_MAX_M = 1 << 20
 
@@ -85,6 +86,9 @@ def _load() -> C.CDLL:
         "prsgd_clear_device_error": (C.c_int, [vp]),
         "prsgd_enable_momentum": (C.c_int, [vp, C.c_float, vp, C.c_int]),
         "prsgd_get_velocity_stacked": (C.c_int, [vp, vp, C.c_int]),
+        "prsgd_set_worker_offset": (C.c_int, [vp, i32]),
+        "prsgd_partial_sum": (C.c_int, [vp, vp, i64, i64]),
+        "prsgd_assign_rows": (C.c_int, [vp, vp, C.c_float, i64, i64]),
         "prsgd_last_error": (C.c_char_p, [vp]),
         "prsgd_average_rows": (C.c_int, [vp, i64, i64, i64, vp]),
         "prsgd_draw_block": (u64, [u64, i32, i64, u64]),
@@ -267,6 +271,22 @@ class PRSGD:
         out = np.empty(self.N, dtype=np.int32)
         self._call(lib.prsgd_get_draws, _host_ptr(out))
         return out
+
+    # ---- shard of a multi-GPU job ------------------------------------------------
+    def set_worker_offset(self, first_worker: int):
+        self._call(lib.prsgd_set_worker_offset, first_worker)
+
+    def new_row(self) -> torch.Tensor:
+        """A device row of m_pad floats (the buffer an all-reduce works on)."""
+        return torch.zeros(self.m_pad, dtype=torch.float32, device=self.device)
+
+    def partial_sum(self, row: torch.Tensor, col0: int = 0, ncols: Optional[int] = None):
+        assert row.is_cuda and row.dtype == torch.float32 and row.numel() == self.m_pad
+        self._call(lib.prsgd_partial_sum, row.data_ptr(), col0, self.m_pad - col0 if ncols is None else ncols)
+
+    def assign_rows(self, row: torch.Tensor, divisor: float, col0: int = 0, ncols: Optional[int] = None):
+        assert row.is_cuda and row.dtype == torch.float32 and row.numel() == self.m_pad
+        self._call(lib.prsgd_assign_rows, row.data_ptr(), float(divisor), col0, self.m_pad - col0 if ncols is None else ncols)
 
     def enable_momentum(self, mu: float, average_velocity: bool = False):
         """Allocate the momentum buffers (same size as the store) and switch the local step to SGD with momentum."""

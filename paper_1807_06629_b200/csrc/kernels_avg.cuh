@@ -17,7 +17,9 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return (a >> 16) | (b & 0xFFFF0000u);
 }
 
-// MODE 0: average + broadcast in place; MODE 1: average only, written to `out` (one row).
+// MODE 0: average + broadcast in place; MODE 1: average only, written to `out` (one row);
+// MODE 2: plain sum of the rows (no division) written to `out`: the local part of an average whose
+// rows are spread over several GPUs.
 // One thread owns 4 consecutive columns (one 128-bit lane); the tail m % 4 is done by scalar threads.
 template <int MODE, bool SHADOW>
 __global__ void __launch_bounds__(256) average_rows_kernel(float* __restrict__ P, int64_t N, int64_t m,
@@ -47,7 +49,7 @@ __global__ void __launch_bounds__(256) average_rows_kernel(float* __restrict__ P
       float4 v = ld_stream(base + i * s4);
       s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
     }
-    float4 y = make_float4(__fdiv_rn(s.x, fN), __fdiv_rn(s.y, fN), __fdiv_rn(s.z, fN), __fdiv_rn(s.w, fN));
+    float4 y = MODE == 2 ? s : make_float4(__fdiv_rn(s.x, fN), __fdiv_rn(s.y, fN), __fdiv_rn(s.z, fN), __fdiv_rn(s.w, fN));
     if (MODE == 0) {
 #pragma unroll 8
       for (int64_t r = 0; r < N; ++r) st_stream(base + r * s4, y);
@@ -63,7 +65,7 @@ __global__ void __launch_bounds__(256) average_rows_kernel(float* __restrict__ P
     const int64_t j = (cols4 << 2) + (c - cols4);
     float s = 0.f;
     for (int64_t i = 0; i < N; ++i) s += P[i * row_stride + j];
-    float y = __fdiv_rn(s, fN);
+    float y = MODE == 2 ? s : __fdiv_rn(s, fN);
     if (MODE == 0) {
       for (int64_t r = 0; r < N; ++r) P[r * row_stride + j] = y;
       if (SHADOW) {
@@ -72,6 +74,26 @@ __global__ void __launch_bounds__(256) average_rows_kernel(float* __restrict__ P
     } else {
       out[j] = y;
     }
+  }
+}
+
+// every row <- src / divisor on columns [0, 4 * cols4) (and the bf16 shadow): the restart after an
+// average whose sum was formed elsewhere (all-reduce over GPUs)
+template <bool SHADOW>
+__global__ void __launch_bounds__(256) assign_rows_kernel(float* __restrict__ P, uint16_t* __restrict__ shadow,
+                                                          const float* __restrict__ src, float divisor, int64_t N,
+                                                          int64_t cols4, int64_t stride4, const DeviceStatus* status) {
+  if (status != nullptr && status->error != 0u) return;
+  const int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= cols4) return;
+  const float4 s = reinterpret_cast<const float4*>(src)[c];
+  const float4 y = make_float4(__fdiv_rn(s.x, divisor), __fdiv_rn(s.y, divisor), __fdiv_rn(s.z, divisor), __fdiv_rn(s.w, divisor));
+  float4* base = reinterpret_cast<float4*>(P) + c;
+  for (int64_t r = 0; r < N; ++r) st_stream(base + r * stride4, y);
+  if (SHADOW) {
+    const uint2 h = make_uint2(pack_bf16x2(y.x, y.y), pack_bf16x2(y.z, y.w));
+    uint2* sb = reinterpret_cast<uint2*>(shadow) + c;
+    for (int64_t r = 0; r < N; ++r) sb[r * stride4] = h;
   }
 }
 

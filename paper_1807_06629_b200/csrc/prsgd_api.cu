@@ -202,7 +202,7 @@ int check_device_status(prsgd_ctx* c) {
 
 DrawArgs draw_args(const prsgd_ctx* c, int64_t t) {
   DrawArgs d;
-  d.seed = c->seed; d.t = t; d.n_blocks = c->n_blocks; d.B = c->B; d.row_elems = c->dims[0];
+  d.seed = c->seed; d.t = t; d.n_blocks = c->n_blocks; d.B = c->B; d.row_elems = c->dims[0]; d.worker0 = c->worker0;
   return d;
 }
 
@@ -578,6 +578,50 @@ int prsgd_get_velocity_stacked(prsgd_ctx* c, float* dst, int dst_on_device) {
   c->params = keep;
   if (rc != PRSGD_OK) return rc;
   return check_device_status(c);
+}
+
+int prsgd_set_worker_offset(prsgd_ctx* c, int32_t first_worker) {
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
+  if (first_worker < 0) return fail(c, PRSGD_ERR_ARG, "first_worker must be >= 0");
+  c->worker0 = first_worker;
+  return PRSGD_OK;
+}
+
+namespace {
+int check_cols(prsgd_ctx* c, const void* p, int64_t col0, int64_t ncols) {
+  if (!p) return fail(c, PRSGD_ERR_ARG, "NULL row pointer");
+  if (col0 < 0 || ncols < 0 || col0 + ncols > c->m_pad) return fail(c, PRSGD_ERR_ARG, "column range outside [0, m_pad)");
+  if ((col0 % 4) != 0 || (ncols % 4) != 0 || !aligned(p, 16))
+    return fail(c, PRSGD_ERR_ALIGN, "col0 and ncols must be multiples of 4 and the row 16-byte aligned");
+  return PRSGD_OK;
+}
+}  // namespace
+
+int prsgd_partial_sum(prsgd_ctx* c, float* d_dst, int64_t col0, int64_t ncols) {
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
+  int rc = check_cols(c, d_dst, col0, ncols);
+  if (rc != PRSGD_OK || ncols == 0) return rc;
+  prof_begin(c, PRSGD_KERNEL_AVERAGE);
+  average_rows_kernel<2, false><<<grid1d(ncols / 4, 256), 256, 0, c->stream>>>(c->params + col0, c->N, ncols, c->m_pad,
+                                                                            d_dst + col0, nullptr, c->status);
+  LAUNCH_CHECK(c);
+  return PRSGD_OK;
+}
+
+int prsgd_assign_rows(prsgd_ctx* c, const float* d_src, float divisor, int64_t col0, int64_t ncols) {
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
+  int rc = check_cols(c, d_src, col0, ncols);
+  if (rc != PRSGD_OK || ncols == 0) return rc;
+  if (!(divisor > 0.f)) return fail(c, PRSGD_ERR_ARG, "divisor must be > 0");
+  prof_begin(c, PRSGD_KERNEL_AVERAGE);
+  if (c->precision == PRSGD_PRECISION_BF16)
+    assign_rows_kernel<true><<<grid1d(ncols / 4, 256), 256, 0, c->stream>>>(c->params + col0, c->shadow + col0, d_src + col0,
+                                                                         divisor, c->N, ncols / 4, c->m_pad / 4, c->status);
+  else
+    assign_rows_kernel<false><<<grid1d(ncols / 4, 256), 256, 0, c->stream>>>(c->params + col0, nullptr, d_src + col0, divisor,
+                                                                          c->N, ncols / 4, c->m_pad / 4, c->status);
+  LAUNCH_CHECK(c);
+  return PRSGD_OK;
 }
 
 int prsgd_get_losses(prsgd_ctx* c, float* h_dst) {

@@ -87,6 +87,7 @@ struct prsgd_ctx {
   float gamma = 0.f;
   int I = 0;
   int64_t t = 0;
+  int worker0 = 0;               // global index of row 0 when the N workers here are a shard of a larger job
   int fused_average = 1;
   float mu = 0.f;                // momentum of the local step (0 = plain SGD)
   float* velocity = nullptr;     // [N][m_pad] fp32 momentum buffers, caller-owned

@@ -1,0 +1,73 @@
+"""PR-SGD with the N workers sharded over several GPUs, one process per GPU.
+
+Inside an epoch the workers are independent, so each rank runs its own shard with the
+single-GPU library; the only exchange is the node average of Algorithm 1, obtained as the paper
+suggests by an all-reduce of the local models (Section 2, "Communication Reduction"): every rank
+sums its own rows, the m_pad-float row is all-reduced (sum) over ranks, and every rank restarts its
+rows at sum / N.  The row is cut into column chunks so that the all-reduce of chunk c overlaps the
+local sum of chunk c + 1.
+
+This module only orchestrates: the local work is done by an *engine* object with
+    local_steps(k), get_step(), m_pad, new_row(),
+    partial_sum(row, col0, ncols), assign_rows(row, divisor, col0, ncols)
+which `paper_1807_06629_b200.binding.PRSGD` provides on the GPU (created with I = 0 and
+set_worker_offset(first worker of the rank)).  The collective is `torch.distributed.all_reduce`
+on whatever backend the process group uses (NCCL on GPUs).
+"""
+from __future__ import annotations
+
+from typing import List, Optional, Tuple
+
+import torch
+import torch.distributed as dist
+
+
+def shard_bounds(N_global: int, world: int, rank: int) -> Tuple[int, int]:
+    """Workers [first, first + count) owned by `rank`: contiguous, sizes differing by at most one."""
+    base, extra = divmod(N_global, world)
+    first = rank * base + min(rank, extra)
+    return first, base + (1 if rank < extra else 0)
+
+
+def column_chunks(m_pad: int, chunks: int) -> List[Tuple[int, int]]:
+    """Cut [0, m_pad) into at most `chunks` ranges whose bounds are multiples of 4."""
+    chunks = max(1, min(chunks, m_pad // 4))
+    per = -(-(m_pad // 4) // chunks) * 4
+    out, c0 = [], 0
+    while c0 < m_pad:
+        n = min(per, m_pad - c0)
+        out.append((c0, n))
+        c0 += n
+    return out
+
+
+class ShardedPRSGD:
+    """Algorithm 1 over all ranks of `group`; `engine` holds this rank's shard of the workers."""
+
+    def __init__(self, engine, N_global: int, I: int, group: Optional[dist.ProcessGroup] = None, chunks: int = 4):
+        if I < 0:
+            raise ValueError("I must be >= 0")
+        self.engine, self.N_global, self.I, self.group = engine, N_global, I, group
+        self.row = engine.new_row()
+        self.chunks = column_chunks(engine.m_pad, chunks)
+
+    def average(self) -> None:
+        """Node average over every worker of every rank, then restart all local rows at it."""
+        handles = []
+        for (c0, n) in self.chunks:
+            self.engine.partial_sum(self.row, c0, n)
+            handles.append(dist.all_reduce(self.row[c0:c0 + n], op=dist.ReduceOp.SUM, group=self.group, async_op=True))
+        for (c0, n), h in zip(self.chunks, handles):
+            h.wait()
+            self.engine.assign_rows(self.row, float(self.N_global), c0, n)
+
+    def local_steps(self, k: int) -> None:
+        """Iterations t+1 .. t+k; averages whenever I > 0 and t mod I == 0 (local step first, then the average)."""
+        t = self.engine.get_step()
+        end = t + k
+        while t < end:
+            nxt = end if self.I == 0 else min(end, (t // self.I + 1) * self.I)
+            self.engine.local_steps(nxt - t)
+            t = nxt
+            if self.I > 0 and t % self.I == 0:
+                self.average()

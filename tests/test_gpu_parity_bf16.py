@@ -215,6 +215,24 @@ def test_momentum_step_on_the_tensor_core_path(torch_cuda, avg_v):
         assert np.array_equal(shadow[:, a:a + n], synth.bf16_bits(store[:, a:a + n]))
 
 
+def test_partial_sum_and_assign_rows_equal_average_on_the_bf16_store(torch_cuda):
+    torch = torch_cuda
+    w = SMALL[4]
+    X, Y, x0 = make_inputs(w)
+    a = make_ctx(w, X, Y, x0, I=0)
+    b = make_ctx(w, X, Y, x0, I=0)
+    a.local_steps(2); b.local_steps(2)
+    a.average()
+    r = b.new_row()
+    b.partial_sum(r)
+    b.assign_rows(r, float(w.N))
+    b.sync()
+    assert np.array_equal(a.get_params_stacked(), b.get_params_stacked())
+    assert torch.equal(a.shadow.view(torch.int16), b.shadow.view(torch.int16))     # shadow rewritten too
+    a.local_steps(1); b.local_steps(1)
+    assert np.array_equal(a.get_params_stacked(), b.get_params_stacked())
+
+
 def test_expired_wait_is_reported_and_the_context_recovers(torch_cuda):
     """Failure path without a fault: a bounded wait runs out, the status word is set, later launches do
     nothing, the host sees PRSGD_ERR_DEVICE_TIMEOUT, and after clearing the context continues bit for bit."""

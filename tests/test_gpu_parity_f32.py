@@ -252,3 +252,48 @@ def test_momentum_step_matches_oracle(torch_cuda, avg_v):
     assert rel_l2(got_x, x2) <= TOL_PERIOD and rel_l2(got_v, v2) <= 1e-3
     assert all(np.array_equal(got_x[i], got_x[0]) for i in range(w.N))
     assert all(np.array_equal(got_v[i], got_v[0]) for i in range(w.N)) == avg_v
+
+
+def test_two_shards_on_one_gpu_reproduce_the_unsharded_run(torch_cuda):
+    """The local halves of the multi-GPU average: two contexts hold workers 0-1 and 2-3 (worker offset
+    2), their partial sums are added (standing in for the all-reduce) and assigned back."""
+    torch = torch_cuda
+    from paper_1807_06629_b200 import binding
+    w = synth.WORKLOADS["cfg1"]
+    X, Y, x0 = make_inputs(w)
+    whole = make_ctx(w, X, Y, x0)
+    whole.local_steps(2 * w.I)
+    shards = []
+    for first in (0, 2):
+        ws = w.with_(N=2)
+        p = make_ctx(ws, X[first:first + 2], Y[first:first + 2], x0, I=0)
+        p.set_worker_offset(first)
+        shards.append(p)
+    for period in range(2):
+        rows = []
+        for k, p in enumerate(shards):
+            p.local_steps(w.I)
+            assert p.get_draws().tolist() == [orc.draw_block(w.seed, 2 * k + i, (period + 1) * w.I, w.n_blocks) for i in range(2)]
+            r = p.new_row()
+            p.partial_sum(r, 0, 1000)                     # two column chunks, as the pipelined all-reduce does
+            p.partial_sum(r, 1000, p.m_pad - 1000)
+            rows.append(r)
+        total = rows[0] + rows[1]
+        for p in shards:
+            p.assign_rows(total, float(w.N), 0, 1000)
+            p.assign_rows(total, float(w.N), 1000, p.m_pad - 1000)
+    got = np.concatenate([p.get_params_stacked() for p in shards])
+    want = whole.get_params_stacked()
+    assert all(np.array_equal(got[i], got[0]) for i in range(w.N))
+    assert rel_l2(got, want) <= 1e-6
+    # with a single context the two halves leave exactly the bits of prsgd_average
+    a = make_ctx(w, X, Y, x0, I=0)
+    b = make_ctx(w, X, Y, x0, I=0)
+    a.local_steps(3); b.local_steps(3)
+    a.average()
+    r = b.new_row()
+    b.partial_sum(r)
+    b.assign_rows(r, float(w.N))
+    assert np.array_equal(a.get_params_stacked(), b.get_params_stacked())
+    with pytest.raises(binding.PRSGDError):
+        b.partial_sum(r, 2, 8)                            # misaligned column range
