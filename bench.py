@@ -264,6 +264,8 @@ def main():
     ap.add_argument("--workers", type=int, default=None, help="override N (smaller cases for profiler captures)")
     ap.add_argument("--momentum", type=float, default=None, help="local step with momentum mu (the paper's experiment used 0.9)")
     ap.add_argument("--update-tile", type=int, default=None, help="tile width of the update kernel (64 or 128)")
+    ap.add_argument("--force-sharded", action="store_true",
+                    help="run the multi-GPU code path (sharded workers + all-reduce average) even on one GPU")
     ap.add_argument("--no-sweep", action="store_true", help="skip the averaging-kernel sweep")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle timing")
     args = ap.parse_args()
@@ -289,24 +291,39 @@ def main():
         _build.build_library()
     torch.cuda.set_device(local_rank)
     dev = f"cuda:{local_rank}"
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device(dev))
+    sharded_mode = world > 1 or args.force_sharded
+    if sharded_mode:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", "29533")
+        dist.init_process_group("nccl", rank=rank, world_size=world, device_id=torch.device(dev))
         dist.barrier()
-    from paper_1807_06629_b200 import binding
+    from paper_1807_06629_b200 import binding, sharded
     peaks = load_peaks()
 
-    # every rank runs an independent replica of the whole workload on its own seed stream
+    # Weak scaling: every rank holds w.N workers of a job with w.N * world workers.  All ranks start from
+    # the same x^0; each rank's workers have their own data pools (seed stream of the rank).
+    x0 = synth.init_params(w.dims, w.seed)
     w = w.with_(seed=w.seed + rank)
     X, Y = synth.make_pools(w)
     if w.precision == 1:
         X = synth.bf16_round(X)
-    x0 = synth.init_params(w.dims, w.seed)
     tdt = torch.bfloat16 if w.precision == 1 else torch.float32
     hX = torch.from_numpy(X).to(tdt).contiguous().pin_memory()
     hY = torch.from_numpy(Y).contiguous().pin_memory()
-    p = binding.PRSGD(w.N, w.dims, w.B, w.gamma, w.I, w.precision, w.pool_samples, w.seed, device=dev)
+    p = binding.PRSGD(w.N, w.dims, w.B, w.gamma, 0 if sharded_mode else w.I, w.precision, w.pool_samples, w.seed,
+                      device=dev)
     p.bind_data(hX.to(dev), hY.to(dev))
     p.set_params(x0)
+    job = None
+    if sharded_mode:          # local steps on the shard, node average = local sums + NCCL all-reduce + restart
+        p.set_worker_offset(rank * w.N)
+        job = sharded.ShardedPRSGD(p, w.N * world, w.I)
+
+    def run_period():
+        if job is not None:
+            job.local_steps(w.I)
+        else:
+            p.local_steps(w.I)
     if args.update_tile is not None:
         p.set_option(binding.OPT_UPDATE_TILE, args.update_tile)
     if args.momentum is not None:
@@ -322,7 +339,7 @@ def main():
 
     # ---- device-timed region: K periods, inputs resident in HBM -------------------------
     for _ in range(args.warmup):
-        p.local_steps(w.I)
+        run_period()
     p.sync()
     sampler = ClockSampler(local_rank)
     barrier()
@@ -333,7 +350,7 @@ def main():
         if flush is not None:
             flush.fill_(float(k))
         evs[k][0].record()
-        p.local_steps(w.I)
+        run_period()
         evs[k][1].record()
     barrier()
     clocks = sampler.stop()
@@ -352,7 +369,7 @@ def main():
     for k in range(args.steps):
         if flush is not None:
             flush.fill_(float(k))
-        p.local_steps(w.I)
+        run_period()
     prof = p.get_profile()
     p.set_option(binding.OPT_PROFILE, 0)
     bytes_iter = algorithmic_bytes(w, p.m_pad, args.momentum is not None)
@@ -375,12 +392,12 @@ def main():
     # ---- end to end through the C ABI from pinned host buffers ---------------------------
     avg_host = torch.empty(p.m, dtype=torch.float32).pin_memory()
     for _ in range(2):
-        p.upload_data(hX, hY); p.local_steps(w.I); p.get_average(avg_host)
+        p.upload_data(hX, hY); run_period(); p.get_average(avg_host)
     barrier()
     t0 = time.perf_counter()
     for _ in range(args.steps):
         p.upload_data(hX, hY)
-        p.local_steps(w.I)
+        run_period()
         p.get_average(avg_host)
     barrier()
     e2e_s = time.perf_counter() - t0
@@ -397,7 +414,8 @@ def main():
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.precision else "f32", "data": "synthetic",
         "config": workload_config(w, {"l2": "L2 flushed between timed steps" if need_flush else
                                       "parameter store + shadow larger than L2",
-                                      "multi_gpu": "independent replicas, one per rank" if world > 1 else "single GPU"},
+                                      "multi_gpu": (f"{w.N} workers per rank, node average = local row sums + NCCL all-reduce + restart"
+                                                    if sharded_mode else "single GPU")},
                                   momentum=args.momentum),
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline,
         "gemm_tflops": tflops, "gemm_frac_of_bf16_peak": tflops / peaks["bf16_tflops_sustained"],
@@ -409,7 +427,7 @@ def main():
             out["cpu_baseline"] = time_oracle(w, X, Y, x0)
     if rank == 0:
         print(json.dumps(out))
-    if world > 1:
+    if sharded_mode:
         dist.destroy_process_group()
 
 
