@@ -47,12 +47,12 @@ def load_peaks():
 # ----------------------------------------------------------------------------- clocks
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
 
     def __init__(self, index: int):
-        self.index, self.proc, self.lines = index, None, []
+        self.index, self.proc, self.lines, self.t_mark = index, None, [], None
 
     def start(self):
         try:
@@ -68,6 +68,10 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.lines.append(line.strip())
 
+    def mark(self):
+        """Start of the timed region: earlier samples (warm-up) are dropped if later ones exist."""
+        self.t_mark = time.time()
+
     def stop(self) -> dict:
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
@@ -76,29 +80,35 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-        sm, mx, reasons, power = [], [], set(), []
+        import datetime
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        rows = []
         for ln in self.lines:
             f = [x.strip() for x in ln.split(",")]
-            if len(f) < 7:
+            if len(f) < 8:
                 continue
             try:
-                sm.append(float(f[0])); mx.append(float(f[1])); power.append(float(f[2]))
+                ts = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                rows.append((ts, float(f[1]), float(f[2]), float(f[3]), [nm for k, nm in enumerate(names)
+                                                                           if f[4 + k].lower().startswith("active")]))
             except ValueError:
                 continue
-            for k, nm in enumerate(names):
-                if f[3 + k].lower().startswith("active"):
-                    reasons.add(nm)
+        timed = [r for r in rows if self.t_mark is not None and r[0] >= self.t_mark - 0.05]
+        window = "timed region"
+        if not timed:
+            timed, window = rows, "warm-up + timed region (timed region shorter than the sampling period)"
+        sm, mx, power = [r[1] for r in timed], [r[2] for r in timed], [r[3] for r in timed]
+        reasons = sorted({nm for r in timed for nm in r[4]})
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+                "power_w_max": max(power) if power else None, "samples": len(sm), "window": window, "reasons": reasons}
 
 
 # ----------------------------------------------------------------------------- ncu traffic
 # dram__bytes_read.sum + dram__bytes_write.sum per iteration of one kernel family, from the one-pass ncu
 # capture summarised in profiles/; valid only while the kernel's source section is unchanged.
 NCU_TRAFFIC = {
-    ("cfg4", "update"): {"bytes_per_iteration": 2.22e9 + 3.04e9, "launches_per_iteration": 4,
-                         "kernel_sha256": "55348bf6e8fa635419181b8251e478103b95905a972f18c2a2b52dd4ab0479ea"},
+    ("cfg4", "update"): {"bytes_per_iteration": 2.22e9 + 3.04e9, "launches_per_iteration": 4,   # read + written, four launches
+                         "kernel_sha256": "313230a269f1d87cf4cd1280b04fab24b792ac0b4a43d468bc28e5c320eaad4e"},
 }
 
 
@@ -108,7 +118,7 @@ def kernel_section_sha(family: str) -> str:
     path = os.path.join(ROOT, "paper_1807_06629_b200", "csrc", "kernels_bf16.cuh")
     with open(path) as f:
         src = f.read()
-    marks = {"update": ("template <int TN> struct UpdCfg", "// b_l <- b_l - gamma")}
+    marks = {"update": ("template <int TN, bool MOM> struct UpdCfg", "// b_l <- b_l - gamma")}
     if family not in marks:
         return ""
     a, b = src.find(marks[family][0]), src.find(marks[family][1])
@@ -256,7 +266,7 @@ def averaging_sweep(torch, binding, peaks, quick=False):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=8)
+    ap.add_argument("--steps", type=int, default=24)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", default=DEFAULT_WORKLOAD, choices=sorted(synth.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -276,6 +286,9 @@ def main():
         w = w.with_(I=args.interval)
     if args.workers is not None:
         w = w.with_(N=args.workers, name=f"{w.name}-N{args.workers}")
+    # the pool holds one averaging period's worth of fresh samples per worker (I blocks of B; at least 4),
+    # which is what the end-to-end arm uploads from the host before every period
+    w = w.with_(pool_samples=max(w.I, 4) * w.B)
     if args.impl == "reference":
         return run_reference(args, w)
 
@@ -338,12 +351,13 @@ def main():
         torch.cuda.synchronize()
 
     # ---- device-timed region: K periods, inputs resident in HBM -------------------------
+    sampler = ClockSampler(local_rank)
+    sampler.start()
     for _ in range(args.warmup):
         run_period()
     p.sync()
-    sampler = ClockSampler(local_rank)
     barrier()
-    sampler.start()
+    sampler.mark()
     launches0 = p.get_launch_count()
     evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
     for k in range(args.steps):
