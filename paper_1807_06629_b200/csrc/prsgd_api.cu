@@ -136,18 +136,15 @@ size_t carve_scratch(int N, const prsgd_model_spec* s, int64_t m_pad, prsgd_ctx*
     for (int l = 1; l <= L; ++l) {
       const int ld = (int)round_up(s->dims[l], 64);
       const size_t e = (size_t)N * B * ld;
-      unsigned char *abk = nullptr, *akb = nullptr, *z = nullptr;
+      unsigned char *abk = nullptr, *z = nullptr;
       if (l < L) abk = take(2 * e);
       else z = take(4 * e);                              // logits, fp32
       auto dbk = take(2 * e);
-      unsigned char* dkb = nullptr;
       if (ctx) {
         ctx->buf.ld[l] = ld;
         ctx->buf.act_bk[l] = reinterpret_cast<uint16_t*>(abk);
-        ctx->buf.act_kb[l] = reinterpret_cast<uint16_t*>(akb);
         ctx->buf.act_f32[l] = reinterpret_cast<float*>(z);
         ctx->buf.delta_bk[l] = reinterpret_cast<uint16_t*>(dbk);
-        ctx->buf.delta_kb[l] = reinterpret_cast<uint16_t*>(dkb);
       }
     }
   }
@@ -159,15 +156,15 @@ bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) %
 int grid1d(int64_t n, int block) { return (int)((n + block - 1) / block); }
 
 // ---- copies between the canonical (gap-free) order and the padded rows -----------------
-// rows [row0, row0 + nrows) of the store <-> nrows * m floats at `lin`
-int copy_canonical(prsgd_ctx* c, float* lin, int64_t row0, int64_t nrows, bool to_store) {
+// rows [row0, row0 + nrows) of `store` (the parameters or the momentum buffers) <-> nrows * m floats at `lin`
+int copy_canonical(prsgd_ctx* c, float* store, float* lin, int64_t row0, int64_t nrows, bool to_store) {
   int64_t pos = 0;
   for (int l = 0; l < c->L; ++l) {
     const Layer& ly = c->layer[l];
     const int64_t seg[2] = {(int64_t)ly.d_in * ly.d_out, (int64_t)ly.d_out};
     const int64_t offs[2] = {ly.w_off, ly.b_off};
     for (int k = 0; k < 2; ++k) {
-      float* st = c->params + row0 * c->m_pad + offs[k];
+      float* st = store + row0 * c->m_pad + offs[k];
       float* li = lin + pos;
       if (to_store)
         CUDA_TRY(c, cudaMemcpy2DAsync(st, c->m_pad * 4, li, c->m * 4, seg[k] * 4, nrows, cudaMemcpyDefault, c->stream));
@@ -466,7 +463,7 @@ int prsgd_set_params(prsgd_ctx* c, const float* src, int32_t worker, int src_on_
   if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
   if (!src) return fail(c, PRSGD_ERR_ARG, "src is NULL");
   if (worker < -1 || worker >= c->N) return fail(c, PRSGD_ERR_ARG, "worker out of range");
-  int rc = copy_canonical(c, const_cast<float*>(src), worker < 0 ? 0 : worker, 1, true);
+  int rc = copy_canonical(c, c->params, const_cast<float*>(src), worker < 0 ? 0 : worker, 1, true);
   if (rc != PRSGD_OK) return rc;
   if (worker < 0 && c->N > 1) {
     prof_begin(c, PRSGD_KERNEL_MISC);
@@ -480,7 +477,7 @@ int prsgd_set_params(prsgd_ctx* c, const float* src, int32_t worker, int src_on_
 int prsgd_set_params_stacked(prsgd_ctx* c, const float* src, int src_on_device) {
   if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
   if (!src) return fail(c, PRSGD_ERR_ARG, "src is NULL");
-  int rc = copy_canonical(c, const_cast<float*>(src), 0, c->N, true);
+  int rc = copy_canonical(c, c->params, const_cast<float*>(src), 0, c->N, true);
   if (rc != PRSGD_OK) return rc;
   if (!src_on_device) CUDA_TRY(c, cudaStreamSynchronize(c->stream));
   return refresh_shadow(c);
@@ -490,7 +487,7 @@ int prsgd_get_params_stacked(prsgd_ctx* c, float* dst, int dst_on_device) {
   (void)dst_on_device;
   if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
   if (!dst) return fail(c, PRSGD_ERR_ARG, "dst is NULL");
-  int rc = copy_canonical(c, dst, 0, c->N, false);
+  int rc = copy_canonical(c, c->params, dst, 0, c->N, false);
   if (rc != PRSGD_OK) return rc;
   return check_device_status(c);
 }
@@ -500,7 +497,7 @@ int prsgd_get_params(prsgd_ctx* c, float* dst, int32_t worker, int dst_on_device
   if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
   if (!dst) return fail(c, PRSGD_ERR_ARG, "dst is NULL");
   if (worker < 0 || worker >= c->N) return fail(c, PRSGD_ERR_ARG, "worker out of range");
-  int rc = copy_canonical(c, dst, worker, 1, false);
+  int rc = copy_canonical(c, c->params, dst, worker, 1, false);
   if (rc != PRSGD_OK) return rc;
   return check_device_status(c);
 }
@@ -572,10 +569,7 @@ int prsgd_get_velocity_stacked(prsgd_ctx* c, float* dst, int dst_on_device) {
   if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
   if (!dst) return fail(c, PRSGD_ERR_ARG, "dst is NULL");
   if (!c->velocity) return fail(c, PRSGD_ERR_STATE, "momentum is not enabled");
-  float* keep = c->params;
-  c->params = c->velocity;                     // same row layout: reuse the canonical gather
-  int rc = copy_canonical(c, dst, 0, c->N, false);
-  c->params = keep;
+  int rc = copy_canonical(c, c->velocity, dst, 0, c->N, false);   // same row layout as the store
   if (rc != PRSGD_OK) return rc;
   return check_device_status(c);
 }

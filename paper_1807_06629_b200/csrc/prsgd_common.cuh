@@ -68,11 +68,9 @@ struct Layer {
 struct Buffers {
   float* act_f32[PRSGD_MAX_LAYERS + 1];
   float* delta_f32[PRSGD_MAX_LAYERS + 1];
-  // bf16 path: activations and deltas in both orientations, leading dimension padded
-  uint16_t* act_bk[PRSGD_MAX_LAYERS + 1];   // [N][B][ld]   (batch-major rows, features contiguous)
-  uint16_t* act_kb[PRSGD_MAX_LAYERS + 1];   // [N][ld][B]   (feature-major rows, batch contiguous)
+  // bf16 path: activations and deltas, batch-major rows [N][B][ld] with the leading dimension padded to 64
+  uint16_t* act_bk[PRSGD_MAX_LAYERS + 1];
   uint16_t* delta_bk[PRSGD_MAX_LAYERS + 1];
-  uint16_t* delta_kb[PRSGD_MAX_LAYERS + 1];
   int ld[PRSGD_MAX_LAYERS + 1];             // padded feature count of layer l's output
 };
 
