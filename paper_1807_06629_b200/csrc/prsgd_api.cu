@@ -69,7 +69,7 @@ int check_spec(const prsgd_model_spec* s, std::string* why) {
   if (s->pool_samples < s->batch || s->pool_samples % s->batch != 0) {
     *why = "pool_samples must be a positive multiple of batch"; return PRSGD_ERR_ARG;
   }
-  if (s->pool_samples / s->batch > 0x7fffffffll) { *why = "too many blocks in the pool"; return PRSGD_ERR_SIZE; }
+  if (s->pool_samples > 0x7fffffffll) { *why = "pool_samples must be below 2^31"; return PRSGD_ERR_SIZE; }
   if (s->precision != PRSGD_PRECISION_FP32 && s->precision != PRSGD_PRECISION_BF16) {
     *why = "unknown precision"; return PRSGD_ERR_ARG;
   }

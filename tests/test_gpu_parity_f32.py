@@ -297,3 +297,26 @@ def test_two_shards_on_one_gpu_reproduce_the_unsharded_run(torch_cuda):
     assert np.array_equal(a.get_params_stacked(), b.get_params_stacked())
     with pytest.raises(binding.PRSGDError):
         b.partial_sum(r, 2, 8)                            # misaligned column range
+
+
+@pytest.mark.parametrize("N,m", [(64, 11_000_000), (256, 25_000_000)])
+def test_average_rows_at_full_sweep_sizes(torch_cuda, N, m):
+    """The largest points of the averaging sweep (up to 25.6 GB): inputs are drawn on the device from a
+    seed, the oracle checks a strided sample of columns, and every row must hold the same bits."""
+    torch = torch_cuda
+    from paper_1807_06629_b200 import binding
+    g = torch.Generator(device="cuda:0")
+    g.manual_seed(20180717 + N)
+    P = torch.empty(N, m, device="cuda:0", dtype=torch.float32)
+    for i in range(0, N, 16):                                    # fill in slabs: no second 25 GB temporary
+        P[i:i + 16].normal_(generator=g)
+    cols = torch.arange(0, m, 9973, device="cuda:0")
+    cols = torch.cat([cols, torch.tensor([m - 4, m - 3, m - 2, m - 1], device="cuda:0")])
+    before = P[:, cols].cpu().numpy().astype(np.float64)
+    binding.prsgd_average_rows(P, N, m)
+    after = P[:, cols].cpu().numpy()
+    want = orc.node_average(before)
+    assert all(np.array_equal(after[i], after[0]) for i in range(N))
+    assert np.abs(after[0] - want).max() <= 2.0 ** -22 * np.abs(before).sum(0).max() / N + 1e-12
+    for i in range(1, N, max(1, N // 8)):                        # whole rows, compared on the device
+        assert bool(torch.equal(P[i], P[0]))
