@@ -408,16 +408,23 @@ def main():
     tflops = flops_per_worker_step(w) * value / world / 1e12
 
     # ---- end to end through the C ABI from pinned host buffers ---------------------------
+    # Every period: fresh pools come from pinned host memory (staged on a copy stream into the spare
+    # device pools while the previous period computes, then swapped in), the period runs, and the node
+    # average is read back into pinned host memory.
     avg_host = torch.empty(p.m, dtype=torch.float32).pin_memory()
+    copy_stream = torch.cuda.Stream(device=dev)
+    p.stage_data(hX, hY, copy_stream)
     for _ in range(2):
-        p.upload_data(hX, hY); run_period(); p.get_average(avg_host)
+        p.swap_data(); p.stage_data(hX, hY, copy_stream); run_period(); p.get_average(avg_host)
     barrier()
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        p.upload_data(hX, hY)
+        p.swap_data()                          # pools uploaded during the previous period become current
+        p.stage_data(hX, hY, copy_stream)      # H2D of the next period's pools, overlapped with this period
         run_period()
-        p.get_average(avg_host)
+        p.get_average(avg_host)                # D2H of the result, synchronises
     barrier()
+    copy_stream.synchronize()
     e2e_s = time.perf_counter() - t0
     te = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
     if world > 1:

@@ -119,6 +119,18 @@ int prsgd_bind_data(prsgd_ctx* ctx, const void* d_X, int32_t x_dtype, const int3
  * host memory makes the copy overlap-capable; pageable memory also works. */
 int prsgd_upload_data(prsgd_ctx* ctx, const void* h_X, const int32_t* h_Y);
 
+/* Double-buffered variant of prsgd_upload_data, for callers that stream fresh samples every epoch:
+ * prsgd_stage_data copies the NEXT pool contents from host memory into a pair of SPARE device pools
+ * (same shapes as the bound ones, caller-owned, 256-byte aligned) on `copy_stream`, a stream of the
+ * caller's other than the context's, so that the copy overlaps the local steps in flight;
+ * prsgd_swap_data makes the staged pools the bound ones for all work enqueued afterwards (the
+ * context's stream waits for the staged copy), and the previously bound pools become free to be
+ * staged into next (the copy stream waits until the work that read them is done).  Asynchronous;
+ * pinned host memory is needed for the overlap. */
+int prsgd_stage_data(prsgd_ctx* ctx, const void* h_X, const int32_t* h_Y, void* d_X_spare, int32_t* d_Y_spare,
+                     void* copy_stream);
+int prsgd_swap_data(prsgd_ctx* ctx);
+
 /* x_i^0 (Algorithm 1, input line: every worker starts from the same point).
  * src holds m floats in canonical order.  worker >= 0: only that row is
  * written; worker = -1: every row receives the same m floats.  Refreshes the

@@ -34,7 +34,7 @@ EXPORTS = [
     "prsgd_set_step", "prsgd_set_option", "prsgd_get_launch_count", "prsgd_get_profile", "prsgd_sync", "prsgd_last_error",
     "prsgd_average_rows", "prsgd_draw_block", "prsgd_mean_rows_noalloc", "prsgd_selftest_wait_expiry",
     "prsgd_clear_device_error", "prsgd_enable_momentum", "prsgd_get_velocity_stacked",
-    "prsgd_set_worker_offset", "prsgd_partial_sum", "prsgd_assign_rows",
+    "prsgd_set_worker_offset", "prsgd_partial_sum", "prsgd_assign_rows", "prsgd_stage_data", "prsgd_swap_data",
 ]
 NOALLOC_MAX_M = 1 << 20
 
@@ -86,6 +86,8 @@ def _load() -> C.CDLL:
         "prsgd_clear_device_error": (C.c_int, [vp]),
         "prsgd_enable_momentum": (C.c_int, [vp, C.c_float, vp, C.c_int]),
         "prsgd_get_velocity_stacked": (C.c_int, [vp, vp, C.c_int]),
+        "prsgd_stage_data": (C.c_int, [vp, vp, vp, vp, vp, vp]),
+        "prsgd_swap_data": (C.c_int, [vp]),
         "prsgd_set_worker_offset": (C.c_int, [vp, i32]),
         "prsgd_partial_sum": (C.c_int, [vp, vp, i64, i64]),
         "prsgd_assign_rows": (C.c_int, [vp, vp, C.c_float, i64, i64]),
@@ -214,6 +216,19 @@ class PRSGD:
     def upload_data(self, hX: torch.Tensor, hY: torch.Tensor):
         assert not hX.is_cuda and not hY.is_cuda and hX.is_contiguous() and hY.is_contiguous()
         self._call(lib.prsgd_upload_data, hX.data_ptr(), hY.data_ptr())
+
+    def stage_data(self, hX: torch.Tensor, hY: torch.Tensor, copy_stream: torch.cuda.Stream):
+        """Copy the next pools from (pinned) host tensors into the spare device pools on `copy_stream`."""
+        assert not hX.is_cuda and not hY.is_cuda and hX.is_contiguous() and hY.is_contiguous()
+        if getattr(self, "_spare", None) is None:
+            self._spare = (torch.empty_like(self._X), torch.empty_like(self._Y))
+        self._call(lib.prsgd_stage_data, hX.data_ptr(), hY.data_ptr(), self._spare[0].data_ptr(),
+                   self._spare[1].data_ptr(), copy_stream.cuda_stream)
+
+    def swap_data(self):
+        """Make the staged pools current; the previous pools become the spare ones."""
+        self._call(lib.prsgd_swap_data)
+        (self._X, self._Y), self._spare = self._spare, (self._X, self._Y)
 
     # ---- parameters -------------------------------------------------------------
     def set_params(self, x, worker: int = -1):

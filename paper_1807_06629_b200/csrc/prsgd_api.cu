@@ -427,6 +427,8 @@ int prsgd_destroy(prsgd_ctx* ctx) {
   tc_destroy(ctx);
   for (auto& p : ctx->pending) { cudaEventDestroy(p.a); cudaEventDestroy(p.b); }
   for (auto e : ctx->event_pool) cudaEventDestroy(e);
+  if (ctx->staged_event) cudaEventDestroy(ctx->staged_event);
+  if (ctx->free_event) cudaEventDestroy(ctx->free_event);
   delete ctx;
   return PRSGD_OK;
 }
@@ -455,6 +457,40 @@ int prsgd_upload_data(prsgd_ctx* c, const void* h_X, const int32_t* h_Y) {
                               cudaMemcpyHostToDevice, c->stream));
   CUDA_TRY(c, cudaMemcpyAsync(const_cast<int32_t*>(c->Y), h_Y, (size_t)c->N * c->P * 4, cudaMemcpyHostToDevice,
                               c->stream));
+  return PRSGD_OK;
+}
+
+int prsgd_stage_data(prsgd_ctx* c, const void* h_X, const int32_t* h_Y, void* d_X_spare, int32_t* d_Y_spare,
+                     void* copy_stream) {
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
+  if (!c->X) return fail(c, PRSGD_ERR_STATE, "bind_data must come first");
+  if (!h_X || !h_Y || !d_X_spare || !d_Y_spare) return fail(c, PRSGD_ERR_ARG, "NULL pointer");
+  if (d_X_spare == c->X || d_Y_spare == c->Y) return fail(c, PRSGD_ERR_ARG, "the spare pools must not be the bound pools");
+  if (!aligned(d_X_spare, 256) || !aligned(d_Y_spare, 256)) return fail(c, PRSGD_ERR_ALIGN, "pools must be 256-byte aligned");
+  cudaStream_t cs = static_cast<cudaStream_t>(copy_stream);
+  if (!c->staged_event) CUDA_TRY(c, cudaEventCreateWithFlags(&c->staged_event, cudaEventDisableTiming));
+  if (c->free_event) CUDA_TRY(c, cudaStreamWaitEvent(cs, c->free_event, 0));   // the spare pools are no longer read
+  const size_t esz = c->x_dtype == PRSGD_X_BF16 ? 2 : 4;
+  CUDA_TRY(c, cudaMemcpyAsync(d_X_spare, h_X, (size_t)c->N * c->P * c->dims[0] * esz, cudaMemcpyHostToDevice, cs));
+  CUDA_TRY(c, cudaMemcpyAsync(d_Y_spare, h_Y, (size_t)c->N * c->P * 4, cudaMemcpyHostToDevice, cs));
+  CUDA_TRY(c, cudaEventRecord(c->staged_event, cs));
+  c->staged_X = d_X_spare; c->staged_Y = d_Y_spare;
+  return PRSGD_OK;
+}
+
+int prsgd_swap_data(prsgd_ctx* c) {
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
+  if (!c->staged_X) return fail(c, PRSGD_ERR_STATE, "nothing staged: prsgd_stage_data must come first");
+  if (!c->free_event) CUDA_TRY(c, cudaEventCreateWithFlags(&c->free_event, cudaEventDisableTiming));
+  CUDA_TRY(c, cudaEventRecord(c->free_event, c->stream));                 // everything that read the old pools
+  CUDA_TRY(c, cudaStreamWaitEvent(c->stream, c->staged_event, 0));        // later work sees the staged pools
+  c->X = c->staged_X; c->Y = c->staged_Y;
+  c->staged_X = nullptr; c->staged_Y = nullptr;
+  if (c->precision == PRSGD_PRECISION_BF16) {
+    std::string terr;
+    int trc = tc_bind_data(c, &terr);
+    if (trc != PRSGD_OK) return fail(c, trc, terr);
+  }
   return PRSGD_OK;
 }
 

@@ -116,6 +116,12 @@ struct prsgd_ctx {
 
   void* tc = nullptr;            // tensor-core path state (tensor maps), owned
 
+  // double-buffered pool upload (prsgd_stage_data / prsgd_swap_data)
+  void* staged_X = nullptr;
+  int32_t* staged_Y = nullptr;
+  cudaEvent_t staged_event = nullptr;   // staged copy complete (recorded on the caller's copy stream)
+  cudaEvent_t free_event = nullptr;     // work that read the previous pools complete (recorded at swap)
+
   // optional per-kernel timing (PRSGD_OPT_PROFILE)
   struct Timed { int kind; cudaEvent_t a, b; };
   bool profile = false;

@@ -320,3 +320,26 @@ def test_average_rows_at_full_sweep_sizes(torch_cuda, N, m):
     assert np.abs(after[0] - want).max() <= 2.0 ** -22 * np.abs(before).sum(0).max() / N + 1e-12
     for i in range(1, N, max(1, N // 8)):                        # whole rows, compared on the device
         assert bool(torch.equal(P[i], P[0]))
+
+
+def test_staged_pool_upload_equals_direct_upload(torch_cuda):
+    """Double-buffered upload: stage on a copy stream, swap, run -- same bits as uploading in place."""
+    torch = torch_cuda
+    w = synth.WORKLOADS["cfg1"]
+    X, Y, x0 = make_inputs(w)
+    w2 = w.with_(seed=w.seed + 1)
+    X2, Y2 = synth.make_pools(w2)
+    hX = [torch.from_numpy(a).pin_memory() for a in (X, X2)]
+    hY = [torch.from_numpy(a).pin_memory() for a in (Y, Y2)]
+    a = make_ctx(w, X, Y, x0)
+    b = make_ctx(w, X, Y, x0)
+    cs = torch.cuda.Stream()
+    for k in range(4):
+        a.upload_data(hX[k % 2], hY[k % 2])
+        a.local_steps(3)
+        b.stage_data(hX[k % 2], hY[k % 2], cs)
+        b.swap_data()
+        b.local_steps(3)
+    assert np.array_equal(a.get_params_stacked(), b.get_params_stacked())
+    with pytest.raises(Exception):
+        b.swap_data()                                  # nothing staged
