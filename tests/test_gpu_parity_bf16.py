@@ -58,6 +58,7 @@ SMALL = [
     _w("tc-b64", 2, (128, 128, 100), 64),
     _w("tc-ragged-tiles", 2, (192, 320, 100), 32),
     _w("tc-many-kblocks", 1, (1024, 128, 10), 32),
+    _w("tc-deep", 2, (64,) * 7 + (10,), 32),
 ]
 
 
@@ -77,7 +78,9 @@ def test_every_gemm_is_tight_when_no_relu_can_switch(torch_cuda, w):
         for cnt in (w.dims[l] * w.dims[l + 1], w.dims[l + 1]):
             g, t = got[:, off:off + cnt] - x0s[:, off:off + cnt], want[:, off:off + cnt] - x0s[:, off:off + cnt]
             assert np.linalg.norm(t) > 0
-            assert rel_l2(g, t) <= TOL_UPDATE_MARGIN, (l, cnt, rel_l2(g, t))
+            # dZ is rounded to bf16 once per layer on its way down: allow the noise to grow with the depth below
+            depth = len(w.dims) - 1 - l
+            assert rel_l2(g, t) <= TOL_UPDATE_MARGIN * max(1.0, depth / 2), (l, cnt, rel_l2(g, t))
             off += cnt
 
 

@@ -218,7 +218,8 @@ def test_time_varying_rates_and_heterogeneous_epochs(torch_cuda):
     q.set_active(None)
 
 
-@pytest.mark.parametrize("N,dims,B", [(1, (5, 3), 1), (3, (7, 5, 3, 2), 5), (2, (130, 70, 33), 48), (5, (16, 300, 11), 100)])
+@pytest.mark.parametrize("N,dims,B", [(1, (5, 3), 1), (3, (7, 5, 3, 2), 5), (2, (130, 70, 33), 48), (5, (16, 300, 11), 100),
+                                      (2, (12,) + (9,) * 15 + (4,), 256)])      # last: 16 layers, batch 256 (the maxima)
 def test_ragged_shapes(torch_cuda, N, dims, B):
     w = synth.Workload("ragged", N, dims, B, 0.1, 3, 6, 0, 4 * B, mean_shift=0.3, seed=77)
     X, Y, x0 = make_inputs(w)

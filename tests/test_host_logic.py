@@ -90,6 +90,9 @@ def test_bad_specs_are_refused_on_the_host(binding):
     assert rc((32, 60, 10), 16, 1, 1024) == -2         # bf16 needs multiples of 64
     assert rc((64, 64, 10), 24, 1, 1008) == -2         # bf16 batch
     assert b"multiples of 64" in lib.prsgd_last_error(None) or b"batch" in lib.prsgd_last_error(None)
+    assert rc((8,) * 18, 16, 0, 1024) == -1            # more than PRSGD_MAX_LAYERS layers
+    assert rc((8,) * 17, 16, 0, 1024) == 0             # exactly 16 layers
+    assert rc((32, 64, 10), 257, 0, 257 * 4) == -1     # batch above 256
     assert lib.prsgd_layout(None, C.byref(lay)) == -1
     spec = binding.make_spec((32, 64, 10), 16, 0, 1024, 1)
     out = C.c_void_p()
