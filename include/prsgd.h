@@ -183,6 +183,21 @@ int prsgd_set_active(prsgd_ctx* ctx, const uint8_t* h_mask);
 int prsgd_get_step(prsgd_ctx* ctx, int64_t* t);
 int prsgd_set_step(prsgd_ctx* ctx, int64_t t);
 
+/* Algorithm 2 (PR-SGD with time-varying learning rates) as one call: for s = s_begin..s_end the epoch
+ * starts from the node average, then K^s = ceil(s^(1/3) / N) local steps with rate
+ * gamma^s = N / s^(2/3) (Theorem 2) times gamma_scale (1 gives the theorem's constants, which are
+ * far too large for a neural network with unknown L; the scale keeps the shape of the schedule).
+ * The context's own gamma and I are left as they were.  prsgd_alg2_schedule returns K^s and gamma^s
+ * (host only).  The iteration counter advances by sum_s K^s, as in the re-indexing after Algorithm 2. */
+int prsgd_alg2_schedule(int32_t N, int64_t s, int64_t* K_s, float* gamma_s);
+int prsgd_run_time_varying(prsgd_ctx* ctx, int64_t s_begin, int64_t s_end, float gamma_scale);
+
+/* One epoch of Algorithm 3 (heterogeneous workers): all workers start from the node average, worker
+ * i takes h_I_i[i] local steps (HOST array of N entries >= 0), workers that have finished keep their
+ * point (the zero-gradient convention of the Extensions section).  The iteration counter advances
+ * by max_i I_i; the models are left un-averaged, the next epoch (or prsgd_average) averages them. */
+int prsgd_run_heterogeneous_epoch(prsgd_ctx* ctx, const int32_t* h_I_i);
+
 /* Workers spread over several GPUs (one context per GPU, each holding a shard of the N workers).
  * Inside an epoch workers need no synchronisation; the only exchange is the node average, which the
  * paper suggests to obtain by an all-reduce of the local models (Section 2, "Communication

@@ -35,6 +35,7 @@ EXPORTS = [
     "prsgd_average_rows", "prsgd_draw_block", "prsgd_mean_rows_noalloc", "prsgd_selftest_wait_expiry",
     "prsgd_clear_device_error", "prsgd_enable_momentum", "prsgd_get_velocity_stacked",
     "prsgd_set_worker_offset", "prsgd_partial_sum", "prsgd_assign_rows", "prsgd_stage_data", "prsgd_swap_data",
+    "prsgd_alg2_schedule", "prsgd_run_time_varying", "prsgd_run_heterogeneous_epoch",
 ]
 NOALLOC_MAX_M = 1 << 20
 
@@ -86,6 +87,9 @@ def _load() -> C.CDLL:
         "prsgd_clear_device_error": (C.c_int, [vp]),
         "prsgd_enable_momentum": (C.c_int, [vp, C.c_float, vp, C.c_int]),
         "prsgd_get_velocity_stacked": (C.c_int, [vp, vp, C.c_int]),
+        "prsgd_alg2_schedule": (C.c_int, [i32, i64, C.POINTER(i64), C.POINTER(C.c_float)]),
+        "prsgd_run_time_varying": (C.c_int, [vp, i64, i64, C.c_float]),
+        "prsgd_run_heterogeneous_epoch": (C.c_int, [vp, vp]),
         "prsgd_stage_data": (C.c_int, [vp, vp, vp, vp, vp, vp]),
         "prsgd_swap_data": (C.c_int, [vp]),
         "prsgd_set_worker_offset": (C.c_int, [vp, i32]),
@@ -134,6 +138,13 @@ def prsgd_workspace_bytes(N, dims, batch, precision, pool_samples, seed=0):
     a, b, c = C.c_size_t(), C.c_size_t(), C.c_size_t()
     _check(lib.prsgd_workspace_bytes(N, C.byref(spec), C.byref(a), C.byref(b), C.byref(c)))
     return a.value, b.value, c.value
+
+
+def prsgd_alg2_schedule(N: int, s: int):
+    """(K^s, gamma^s) of Theorem 2."""
+    K, g = C.c_int64(), C.c_float()
+    _check(lib.prsgd_alg2_schedule(N, s, C.byref(K), C.byref(g)))
+    return K.value, g.value
 
 
 def prsgd_draw_block(seed: int, worker: int, t: int, n_blocks: int) -> int:
@@ -313,6 +324,15 @@ class PRSGD:
         out = np.empty((self.N, self.m), dtype=np.float32)
         self._call(lib.prsgd_get_velocity_stacked, _host_ptr(out), 0)
         return out
+
+    # ---- Algorithms 2 and 3 ------------------------------------------------------
+    def run_time_varying(self, s_begin: int, s_end: int, gamma_scale: float = 1.0):
+        self._call(lib.prsgd_run_time_varying, s_begin, s_end, gamma_scale)
+
+    def run_heterogeneous_epoch(self, I_i: Sequence[int]):
+        a = np.ascontiguousarray(np.asarray(I_i, dtype=np.int32))
+        assert a.size == self.N
+        self._call(lib.prsgd_run_heterogeneous_epoch, _host_ptr(a))
 
     # ---- schedule ---------------------------------------------------------------
     def set_lr(self, gamma: float):

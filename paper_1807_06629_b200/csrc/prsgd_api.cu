@@ -1,5 +1,6 @@
 // C ABI of the PR-SGD library: host-side context, layout, schedule of
 // Algorithm 1 and the kernel launches.  See include/prsgd.h for the contract.
+#include <cmath>
 #include <cstdio>
 #include <cstring>
 #include <mutex>
@@ -674,6 +675,66 @@ int prsgd_get_draws(prsgd_ctx* c, int32_t* h_dst) {
   if (!h_dst) return fail(c, PRSGD_ERR_ARG, "h_dst is NULL");
   CUDA_TRY(c, cudaMemcpyAsync(h_dst, c->draws, sizeof(int32_t) * c->N, cudaMemcpyDeviceToHost, c->stream));
   return check_device_status(c);
+}
+
+int prsgd_alg2_schedule(int32_t N, int64_t s, int64_t* K_s, float* gamma_s) {
+  if (N < 1 || s < 1) return fail(nullptr, PRSGD_ERR_ARG, "need N >= 1 and s >= 1");
+  // cube root of s, exact at perfect cubes
+  double root = std::cbrt((double)s);
+  const int64_t r = (int64_t)std::llround(root);
+  if (r * r * r == s) root = (double)r;
+  if (K_s) *K_s = (int64_t)std::ceil(root / (double)N);
+  if (gamma_s) *gamma_s = (float)((double)N / (root * root));
+  return PRSGD_OK;
+}
+
+int prsgd_run_time_varying(prsgd_ctx* c, int64_t s_begin, int64_t s_end, float gamma_scale) {
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
+  if (s_begin < 1 || s_end < s_begin) return fail(c, PRSGD_ERR_ARG, "need 1 <= s_begin <= s_end");
+  if (!(gamma_scale > 0.f)) return fail(c, PRSGD_ERR_ARG, "gamma_scale must be > 0");
+  const int I_keep = c->I;
+  const float g_keep = c->gamma;
+  c->I = 0;                                          // epochs are driven here, not by t mod I
+  int rc = PRSGD_OK;
+  for (int64_t s = s_begin; s <= s_end && rc == PRSGD_OK; ++s) {
+    int64_t K = 0; float g = 0.f;
+    prsgd_alg2_schedule(c->N * 1, s, &K, &g);
+    rc = launch_average(c);                          // x_i^{s,0} = node average of the previous epoch's end points
+    if (rc != PRSGD_OK) break;
+    c->gamma = g * gamma_scale;
+    rc = prsgd_local_steps(c, K);
+  }
+  c->I = I_keep;
+  c->gamma = g_keep;
+  return rc;
+}
+
+int prsgd_run_heterogeneous_epoch(prsgd_ctx* c, const int32_t* h_I_i) {
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
+  if (!h_I_i) return fail(c, PRSGD_ERR_ARG, "h_I_i is NULL");
+  int32_t Imax = 0;
+  for (int i = 0; i < c->N; ++i) {
+    if (h_I_i[i] < 0) return fail(c, PRSGD_ERR_ARG, "epoch lengths must be >= 0");
+    if (h_I_i[i] > Imax) Imax = h_I_i[i];
+  }
+  const int I_keep = c->I;
+  const bool mask_keep = c->has_mask;
+  std::vector<uint8_t> mask((size_t)c->N), old_mask((size_t)c->N);
+  if (mask_keep) {
+    CUDA_TRY(c, cudaMemcpyAsync(old_mask.data(), c->active, (size_t)c->N, cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  }
+  c->I = 0;
+  int rc = launch_average(c);                        // x_i^{s,0} = node average
+  for (int32_t k = 1; k <= Imax && rc == PRSGD_OK; ++k) {
+    bool all = true;
+    for (int i = 0; i < c->N; ++i) { mask[i] = k <= h_I_i[i] ? 1 : 0; all = all && mask[i]; }
+    rc = prsgd_set_active(c, all ? nullptr : mask.data());
+    if (rc == PRSGD_OK) rc = prsgd_local_steps(c, 1);
+  }
+  c->I = I_keep;
+  int rc2 = prsgd_set_active(c, mask_keep ? old_mask.data() : nullptr);
+  return rc != PRSGD_OK ? rc : rc2;
 }
 
 int prsgd_set_lr(prsgd_ctx* c, float gamma) {

@@ -344,3 +344,25 @@ def test_staged_pool_upload_equals_direct_upload(torch_cuda):
     assert np.array_equal(a.get_params_stacked(), b.get_params_stacked())
     with pytest.raises(Exception):
         b.swap_data()                                  # nothing staged
+
+
+def test_algorithm_2_and_3_drivers(torch_cuda):
+    """prsgd_run_time_varying / prsgd_run_heterogeneous_epoch against the oracle's Algorithm 2 and 3."""
+    w = synth.WORKLOADS["cfg1"]
+    X, Y, x0 = make_inputs(w)
+    fn = orc.mlp_grad_fn(w.dims, X.astype(np.float64), Y, w.B, w.seed)
+    xs = np.tile(x0, (w.N, 1))
+    scale = 0.02
+    p = make_ctx(w, X, Y, x0)
+    p.run_time_varying(1, 70, scale)                      # K^s goes from 1 to 2 at s = 65 for N = 4
+    sched = [(K, g * scale) for (K, g) in orc.alg2_schedule(w.N, 70)]
+    assert sum(K for K, _ in sched) == p.get_step() and max(K for K, _ in sched) == 2
+    want = orc.pr_sgd_time_varying(xs, sched, fn)
+    assert rel_l2(p.get_params_stacked(), want) <= 2e-4
+    q = make_ctx(w, X, Y, x0)
+    I_i = [3, 1, 0, 2]
+    for _ in range(2):
+        q.run_heterogeneous_epoch(I_i)
+    want = orc.pr_sgd_heterogeneous(xs, w.gamma, I_i, 2, fn)
+    assert rel_l2(q.get_params_stacked(), want) <= TOL_PERIOD
+    assert q.get_step() == 6

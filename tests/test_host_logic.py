@@ -24,7 +24,7 @@ def binding():
 def test_library_exports_every_declared_symbol(binding):
     with open(os.path.join(ROOT, "include", "prsgd.h")) as f:
         src = re.sub(r"/\*.*?\*/", "", f.read(), flags=re.S)
-    declared = set(re.findall(r"\b(prsgd_[a-z_]+)\s*\(", src))
+    declared = set(re.findall(r"\b(prsgd_[a-z0-9_]+)\s*\(", src))
     assert len(declared) >= 25
     for name in declared:
         assert hasattr(binding.lib, name), name
@@ -107,3 +107,11 @@ def test_bad_specs_are_refused_on_the_host(binding):
     assert lib.prsgd_average_rows(260, 4, 16, 16, None) == -2
     assert lib.prsgd_average_rows(256, 4, 16, 18, None) == -2
     assert lib.prsgd_local_steps(None, 1) == -1
+
+
+def test_alg2_schedule_matches_oracle(binding):
+    for N in (1, 2, 8):
+        want = orc.alg2_schedule(N, 130)
+        for s in (1, 2, 7, 8, 9, 26, 27, 28, 64, 125, 130):
+            K, g = binding.prsgd_alg2_schedule(N, s)
+            assert K == want[s - 1][0] and g == pytest.approx(want[s - 1][1], rel=1e-6)
