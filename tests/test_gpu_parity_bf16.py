@@ -236,6 +236,27 @@ def test_partial_sum_and_assign_rows_equal_average_on_the_bf16_store(torch_cuda)
     assert np.array_equal(a.get_params_stacked(), b.get_params_stacked())
 
 
+def test_training_run_tracks_the_oracle_loss_curve(torch_cuda):
+    """48 iterations (12 periods) on the tensor-core path: draws exact, loss curve within bf16 noise of the
+    oracle's, loss going down."""
+    w = synth.Workload("tc-train", 4, (128, 256, 128, 10), 32, 0.1, 4, 48, 1, 32 * 32, mean_shift=0.5, seed=77)
+    X, Y, x0 = make_inputs(w)
+    p = make_ctx(w, X, Y, x0)
+    losses, draws = {}, {}
+    want = oracle_run(w, X, Y, np.tile(x0, (w.N, 1)), 0, w.T, losses=losses, draws=draws)
+    curve = []
+    for t in range(1, w.T + 1):
+        p.local_steps(1)
+        assert p.get_draws().tolist() == [draws[(i, t)] for i in range(w.N)]
+        curve.append(p.get_losses())
+    curve = np.array(curve)
+    ref = np.array([[losses[(i, t)] for i in range(w.N)] for t in range(1, w.T + 1)])
+    assert np.abs(curve - ref).max() <= 5e-2
+    assert np.abs(curve.mean(1) - ref.mean(1)).max() <= 2e-2
+    assert curve[-8:].mean() < curve[:8].mean() - 0.1
+    assert rel_l2(p.get_params_stacked(), want) <= TOL_PERIOD
+
+
 def test_expired_wait_is_reported_and_the_context_recovers(torch_cuda):
     """Failure path without a fault: a bounded wait runs out, the status word is set, later launches do
     nothing, the host sees PRSGD_ERR_DEVICE_TIMEOUT, and after clearing the context continues bit for bit."""

@@ -366,3 +366,25 @@ def test_algorithm_2_and_3_drivers(torch_cuda):
     want = orc.pr_sgd_heterogeneous(xs, w.gamma, I_i, 2, fn)
     assert rel_l2(q.get_params_stacked(), want) <= TOL_PERIOD
     assert q.get_step() == 6
+
+
+def test_cfg1_whole_run_tracks_the_oracle(torch_cuda):
+    """All T = 64 iterations of the tiny configuration (16 averaging periods), GPU against oracle:
+    the same draws every iteration, the same loss curve, and parameters that stay together."""
+    w = synth.WORKLOADS["cfg1"]
+    X, Y, x0 = make_inputs(w)
+    p = make_ctx(w, X, Y, x0)
+    losses, draws = {}, {}
+    want = oracle_run(w, X, Y, np.tile(x0, (w.N, 1)), 0, w.T, losses=losses, draws=draws)
+    curve = []
+    for t in range(1, w.T + 1):
+        p.local_steps(1)
+        assert p.get_draws().tolist() == [draws[(i, t)] for i in range(w.N)]
+        curve.append(p.get_losses())
+    curve = np.array(curve)
+    ref = np.array([[losses[(i, t)] for i in range(w.N)] for t in range(1, w.T + 1)])
+    assert np.abs(curve - ref).max() <= 1e-3
+    assert curve[-8:].mean() < curve[:8].mean() - 0.05            # it trains
+    got = p.get_params_stacked()
+    assert rel_l2(got, want) <= 1e-3
+    assert all(np.array_equal(got[i], got[0]) for i in range(w.N))  # T = 64 is an averaging iteration
