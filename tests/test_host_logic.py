@@ -115,3 +115,17 @@ def test_alg2_schedule_matches_oracle(binding):
         for s in (1, 2, 7, 8, 9, 26, 27, 28, 64, 125, 130):
             K, g = binding.prsgd_alg2_schedule(N, s)
             assert K == want[s - 1][0] and g == pytest.approx(want[s - 1][1], rel=1e-6)
+
+
+def test_reference_arm_of_the_benchmark_prints_its_json_line():
+    """`bench.py --impl reference` times the oracle on the host and needs no GPU."""
+    import json
+    import subprocess
+    import sys
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--config", "cfg1",
+                          "--steps", "2", "--warmup", "3"], capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0, out.stderr[-2000:]
+    line = json.loads(out.stdout.strip().splitlines()[-1])
+    assert line["impl"] == "reference" and line["metric"] == "worker-steps/s" and line["value"] > 0
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] >= 1
+    assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["config"]["workload"] == "cfg1"
