@@ -306,6 +306,9 @@ def main():
         _build.build_library()
     torch.cuda.set_device(local_rank)
     dev = f"cuda:{local_rank}"
+    # everything below (torch copies, the library's kernels, the timing events) runs on one side stream:
+    # the library replays captured periods as CUDA graphs, which the legacy default stream cannot capture
+    torch.cuda.set_stream(torch.cuda.Stream(device=dev))
     sharded_mode = world > 1 or args.force_sharded
     if sharded_mode:
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")

@@ -236,6 +236,12 @@ int prsgd_get_velocity_stacked(prsgd_ctx* ctx, float* dst, int dst_on_device);
  * pair of CUDA events on the context's stream; read the sums with
  * prsgd_get_profile.  Costs two event records per launch. */
 #define PRSGD_OPT_PROFILE 2
+/* PRSGD_OPT_GRAPH (default 1): whole averaging periods (I iterations that begin right after an
+ * average, k >= I, I > 0, profiling off) are captured once as a CUDA graph and replayed; the kernels
+ * read the iteration number from a device counter, so one capture serves every period.  Settings
+ * that change the launches (gamma, I, options, mask on/off, momentum, the bound pools) key separate
+ * captures.  Results are bit-identical to direct launches; 0 switches the replay off. */
+#define PRSGD_OPT_GRAPH 4
 /* PRSGD_OPT_UPDATE_TILE (default 0): column width of the 128-row tile the tensor-core update
  * kernel works on: 64 (four pipeline stages per SM), 128 (two), or 0 = chosen per launch from
  * the layer size.  A tuning knob only: every setting produces the same bits. */

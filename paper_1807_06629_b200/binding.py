@@ -23,6 +23,7 @@ X_FP32, X_BF16 = 0, 1
 OPT_FUSED_AVERAGE = 1
 OPT_PROFILE = 2
 OPT_UPDATE_TILE = 3
+OPT_GRAPH = 4
 KERNEL_FAMILIES = ("forward", "softmax", "dx", "update", "update_average", "average", "misc")
 MAX_LAYERS = 16
 

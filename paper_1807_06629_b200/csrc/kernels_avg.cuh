@@ -97,6 +97,13 @@ __global__ void __launch_bounds__(256) assign_rows_kernel(float* __restrict__ P,
   }
 }
 
+// device-resident iteration counter of a captured period: set before a replay, advanced at its end
+__global__ void counter_set_kernel(int64_t* counter, int64_t value) { *counter = value; }
+__global__ void counter_add_kernel(int64_t* counter, int64_t delta) {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  *counter += delta;
+}
+
 // rows 1..N-1 <- row 0 (every worker starts from the same point; Algorithm 1, input line)
 __global__ void __launch_bounds__(256) broadcast_row0_kernel(float* __restrict__ P, int64_t N, int64_t cols4,
                                                              int64_t stride4) {

@@ -163,7 +163,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) tc_stream_kernel(const __gr
     for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
       const int n = item / a.tiles_m, m0 = (item % a.tiles_m) * 128;
       if (!item_active(n)) continue;
-      const int row0 = a.pool ? (int)draw_block(a.draw.seed, a.draw.worker0 + n, a.draw.t, a.draw.n_blocks) * a.B : 0;
+      const int row0 = a.pool ? (int)draw_block(a.draw.seed, a.draw.worker0 + n, draw_t(a.draw), a.draw.n_blocks) * a.B : 0;
       for (int ks = 0; ks < a.k_steps; ++ks, ++g) {
         const int s = g % S;
         const uint32_t ph = (g / S) & 1u;
@@ -396,7 +396,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
         const uint32_t ph = (it / S) & 1u;
         ok = mbar_wait(stage_empty(s), ph ^ 1u, abort_flag, a.status, 0x201);
         if (!ok) break;
-        const int row0 = a.pool ? (int)draw_block(a.draw.seed, a.draw.worker0 + n, a.draw.t, a.draw.n_blocks) * a.B : 0;
+        const int row0 = a.pool ? (int)draw_block(a.draw.seed, a.draw.worker0 + n, draw_t(a.draw), a.draw.n_blocks) * a.B : 0;
         const uint32_t ops = ops_u32(s);
         mbar_expect_tx(full_ops(s), (2u + NB64) * op_box);
         tma_load_3d(ops, &mapDelta, full_ops(s), m0, 0, n);

@@ -22,7 +22,10 @@ struct DrawArgs {
   int B;                 // rows per block
   int64_t row_elems;     // d_0
   int worker0;           // global index of local row 0 (workers sharded over several GPUs)
+  const int64_t* t_base; // nullptr, or a device counter added to t (a captured period is replayed with a new base)
 };
+
+__device__ __forceinline__ int64_t draw_t(const DrawArgs& d) { return d.t + (d.t_base != nullptr ? *d.t_base : 0); }
 
 enum { EPI_FWD_RELU = 0, EPI_FWD_LINEAR = 1, EPI_DX = 2, EPI_DW = 3 };
 
@@ -46,7 +49,7 @@ struct GemmF32Args {
 
 __device__ __forceinline__ const float* operand_ptr(const OperandF32& o, int n, const DrawArgs& d) {
   const float* p = o.base + (int64_t)n * o.worker_stride;
-  if (o.pool) p += (int64_t)draw_block(d.seed, d.worker0 + n, d.t, d.n_blocks) * d.B * d.row_elems;
+  if (o.pool) p += (int64_t)draw_block(d.seed, d.worker0 + n, draw_t(d), d.n_blocks) * d.B * d.row_elems;
   return p;
 }
 
@@ -271,7 +274,7 @@ __global__ void __launch_bounds__(256) softmax_ce_kernel(const SoftmaxArgs a) {
   if (a.status != nullptr && a.status->error != 0u) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int b = blockIdx.y * 8 + warp;
-  const uint32_t blk = draw_block(a.draw.seed, a.draw.worker0 + n, a.draw.t, a.draw.n_blocks);
+  const uint32_t blk = draw_block(a.draw.seed, a.draw.worker0 + n, draw_t(a.draw), a.draw.n_blocks);
   if (blockIdx.y == 0 && threadIdx.x == 0) a.draws[n] = (int32_t)blk;
   if (b >= a.B) return;
   const float invB = 1.f / (float)a.B;

@@ -115,7 +115,9 @@ size_t carve_scratch(int N, const prsgd_model_spec* s, int64_t m_pad, prsgd_ctx*
   auto losses = take(sizeof(float) * (size_t)N * B);
   auto active = take((size_t)N);
   auto stage = take(sizeof(float) * (size_t)m_pad);
+  auto tdev = take(sizeof(int64_t));
   if (ctx) {
+    ctx->t_dev = reinterpret_cast<int64_t*>(tdev);
     ctx->status = reinterpret_cast<DeviceStatus*>(status);
     ctx->draws = reinterpret_cast<int32_t*>(draws);
     ctx->losses = reinterpret_cast<float*>(losses);
@@ -201,6 +203,7 @@ int check_device_status(prsgd_ctx* c) {
 DrawArgs draw_args(const prsgd_ctx* c, int64_t t) {
   DrawArgs d;
   d.seed = c->seed; d.t = t; d.n_blocks = c->n_blocks; d.B = c->B; d.row_elems = c->dims[0]; d.worker0 = c->worker0;
+  d.t_base = c->capturing ? c->t_dev : nullptr;      // while capturing, t is relative to the period's start
   return d;
 }
 
@@ -428,6 +431,7 @@ int prsgd_destroy(prsgd_ctx* ctx) {
   tc_destroy(ctx);
   for (auto& p : ctx->pending) { cudaEventDestroy(p.a); cudaEventDestroy(p.b); }
   for (auto e : ctx->event_pool) cudaEventDestroy(e);
+  for (auto& g : ctx->graphs) cudaGraphExecDestroy(g.exec);
   if (ctx->staged_event) cudaEventDestroy(ctx->staged_event);
   if (ctx->free_event) cudaEventDestroy(ctx->free_event);
   delete ctx;
@@ -539,12 +543,11 @@ int prsgd_get_params(prsgd_ctx* c, float* dst, int32_t worker, int dst_on_device
   return check_device_status(c);
 }
 
-int prsgd_local_steps(prsgd_ctx* c, int64_t k) {
-  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
-  if (k < 0) return fail(c, PRSGD_ERR_ARG, "k must be >= 0");
-  if (!c->X || !c->Y) return fail(c, PRSGD_ERR_STATE, "bind_data must come before local_steps");
-  for (int64_t s = 0; s < k; ++s) {
-    const int64_t t = c->t + 1;
+namespace {
+
+// iterations t_first .. t_first + count - 1, launched directly
+int run_iterations(prsgd_ctx* c, int64_t t_first, int64_t count) {
+  for (int64_t t = t_first; t < t_first + count; ++t) {
     const bool averaging = c->I > 0 && (t % c->I) == 0;
     int rc = c->precision == PRSGD_PRECISION_BF16 ? step_bf16(c, t, averaging) : step_f32(c, t, averaging);
     if (rc != PRSGD_OK) return rc;
@@ -552,7 +555,94 @@ int prsgd_local_steps(prsgd_ctx* c, int64_t k) {
       rc = launch_average(c);
       if (rc != PRSGD_OK) return rc;
     }
-    c->t = t;
+  }
+  return PRSGD_OK;
+}
+
+void period_key(const prsgd_ctx* c, uint64_t (&key)[12]) {
+  uint32_t gbits, mbits;
+  std::memcpy(&gbits, &c->gamma, 4);
+  std::memcpy(&mbits, &c->mu, 4);
+  key[0] = gbits; key[1] = (uint64_t)c->I; key[2] = (uint64_t)c->fused_average; key[3] = (uint64_t)c->upd_tile;
+  key[4] = c->has_mask ? 1 : 0; key[5] = reinterpret_cast<uint64_t>(c->velocity); key[6] = mbits;
+  key[7] = (uint64_t)c->average_velocity; key[8] = reinterpret_cast<uint64_t>(c->X);
+  key[9] = reinterpret_cast<uint64_t>(c->Y); key[10] = (uint64_t)c->worker0; key[11] = 0;
+}
+
+// One whole averaging period (I iterations starting right after an average) as a CUDA graph: the
+// kernels take the iteration number as device counter + offset, so one capture serves every period.
+// Returns nullptr when capture is not possible (the caller then launches directly).
+prsgd_ctx::PeriodGraph* get_period_graph(prsgd_ctx* c) {
+  uint64_t key[12];
+  period_key(c, key);
+  for (auto& g : c->graphs)
+    if (std::memcmp(g.key, key, sizeof key) == 0) return &g;
+  if (c->graphs.size() >= 8) {                          // settings keep changing: start over
+    for (auto& g : c->graphs) cudaGraphExecDestroy(g.exec);
+    c->graphs.clear();
+  }
+  if (cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+    cudaGetLastError();
+    c->use_graph = 0;
+    return nullptr;
+  }
+  const int64_t launches0 = c->launches;
+  c->capturing = true;
+  int rc = run_iterations(c, 1, c->I);                  // offsets 1..I; offset I is the averaging iteration
+  if (rc == PRSGD_OK) {
+    counter_add_kernel<<<1, 1, 0, c->stream>>>(c->t_dev, (int64_t)c->I);
+    if (cudaGetLastError() != cudaSuccess) rc = PRSGD_ERR_CUDA;
+  }
+  c->capturing = false;
+  const int64_t per_replay = c->launches - launches0;
+  c->launches = launches0;
+  cudaGraph_t graph = nullptr;
+  cudaError_t e = cudaStreamEndCapture(c->stream, &graph);
+  cudaGraphExec_t exec = nullptr;
+  if (rc == PRSGD_OK && e == cudaSuccess && graph != nullptr) e = cudaGraphInstantiate(&exec, graph, 0);
+  if (graph) cudaGraphDestroy(graph);
+  if (rc != PRSGD_OK || e != cudaSuccess || exec == nullptr) {
+    cudaGetLastError();
+    c->use_graph = 0;                                   // do not try again on this context
+    return nullptr;
+  }
+  prsgd_ctx::PeriodGraph g;
+  std::memcpy(g.key, key, sizeof key);
+  g.exec = exec; g.launches = per_replay;
+  c->graphs.push_back(g);
+  return &c->graphs.back();
+}
+
+}  // namespace
+
+int prsgd_local_steps(prsgd_ctx* c, int64_t k) {
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
+  if (k < 0) return fail(c, PRSGD_ERR_ARG, "k must be >= 0");
+  if (!c->X || !c->Y) return fail(c, PRSGD_ERR_STATE, "bind_data must come before local_steps");
+  while (k > 0) {
+    // whole periods that start right after an average are replayed from a captured graph
+    if (c->use_graph && !c->profile && c->I > 0 && k >= c->I && (c->t % c->I) == 0) {
+      prsgd_ctx::PeriodGraph* g = get_period_graph(c);
+      if (g != nullptr) {
+        counter_set_kernel<<<1, 1, 0, c->stream>>>(c->t_dev, c->t);
+        CUDA_TRY(c, cudaGetLastError());
+        CUDA_TRY(c, cudaGraphLaunch(g->exec, c->stream));
+        c->launches += g->launches + 1;
+        c->t += c->I;
+        k -= c->I;
+        continue;
+      }
+    }
+    // otherwise: directly, up to the next period boundary (or the end of the request)
+    int64_t n = k;
+    if (c->I > 0) {
+      const int64_t to_boundary = c->I - (c->t % c->I);
+      if (to_boundary < n) n = to_boundary;
+    }
+    int rc = run_iterations(c, c->t + 1, n);
+    if (rc != PRSGD_OK) return rc;
+    c->t += n;
+    k -= n;
   }
   return PRSGD_OK;
 }
@@ -777,6 +867,7 @@ int prsgd_set_option(prsgd_ctx* c, int32_t option, int64_t value) {
   if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
   if (option == PRSGD_OPT_FUSED_AVERAGE) { c->fused_average = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_PROFILE) { c->profile = value != 0; return PRSGD_OK; }
+  if (option == PRSGD_OPT_GRAPH) { c->use_graph = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_UPDATE_TILE) {
     if (value != 0 && value != 64 && value != 128) return fail(c, PRSGD_ERR_ARG, "update tile width must be 0, 64 or 128");
     c->upd_tile = (int)value;

@@ -122,6 +122,17 @@ struct prsgd_ctx {
   cudaEvent_t staged_event = nullptr;   // staged copy complete (recorded on the caller's copy stream)
   cudaEvent_t free_event = nullptr;     // work that read the previous pools complete (recorded at swap)
 
+  // whole averaging periods captured as CUDA graphs (PRSGD_OPT_GRAPH)
+  struct PeriodGraph {
+    uint64_t key[12];
+    cudaGraphExec_t exec;
+    int64_t launches;            // kernel launches one replay stands for
+  };
+  int use_graph = 1;
+  bool capturing = false;
+  int64_t* t_dev = nullptr;      // device copy of t at the start of the period being replayed
+  std::vector<PeriodGraph> graphs;
+
   // optional per-kernel timing (PRSGD_OPT_PROFILE)
   struct Timed { int kind; cudaEvent_t a, b; };
   bool profile = false;

@@ -257,6 +257,35 @@ def test_training_run_tracks_the_oracle_loss_curve(torch_cuda):
     assert rel_l2(p.get_params_stacked(), want) <= TOL_PERIOD
 
 
+def test_graph_replay_of_whole_periods_is_bit_identical(torch_cuda):
+    """On a non-default stream whole periods are replayed from a captured CUDA graph (iteration number read
+    from a device counter); the bits, the draws and the step counter must equal direct launches."""
+    torch = torch_cuda
+    from paper_1807_06629_b200 import binding
+    for w in (SMALL[1], _w("tc-n5", 5, (64, 128, 10), 32, I=3), synth.WORKLOADS["cfg1"]):
+        X, Y, x0 = make_inputs(w)
+        outs = []
+        for use_graph in (0, 1):
+            with torch.cuda.stream(torch.cuda.Stream()):
+                p = make_ctx(w, X, Y, x0)
+                p.set_option(binding.OPT_GRAPH, use_graph)
+                n0 = p.get_launch_count()
+                p.local_steps(1)                  # partial period: direct
+                p.local_steps(w.I - 1)            # reaches the first average
+                p.local_steps(3 * w.I + 1)        # three whole periods (replayed) and one more iteration
+                p.set_lr(w.gamma * 0.5)           # a new setting keys a new capture
+                p.local_steps(2 * w.I)
+                outs.append((p.get_params_stacked(), p.get_draws().tolist(), p.get_step(), p.get_losses(),
+                             p.get_launch_count() - n0))
+                torch.cuda.current_stream().synchronize()
+        assert np.array_equal(outs[0][0], outs[1][0])
+        assert outs[0][1] == outs[1][1] and outs[0][2] == outs[1][2] == 6 * w.I + 1
+        assert np.array_equal(outs[0][3], outs[1][3])
+        # same kernels, plus one counter-set launch per replayed period (three, then one after the new setting:
+        # the second request first walks to the period boundary with direct launches)
+        assert outs[1][4] == outs[0][4] + 4
+
+
 def test_expired_wait_is_reported_and_the_context_recovers(torch_cuda):
     """Failure path without a fault: a bounded wait runs out, the status word is set, later launches do
     nothing, the host sees PRSGD_ERR_DEVICE_TIMEOUT, and after clearing the context continues bit for bit."""
