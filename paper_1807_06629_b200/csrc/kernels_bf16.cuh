@@ -602,7 +602,13 @@ __global__ void __launch_bounds__(128) bias_update_kernel(const BiasArgs a) {
   if (j >= a.d_out[l] || (a.active != nullptr && a.active[n] == 0) || a.status->error != 0u) return;
   const uint16_t* d = a.delta_bk[l] + (int64_t)n * a.B * a.ld[l] + j;
   float g = 0.f;
-  for (int b = 0; b < a.B; ++b) g += __uint_as_float((uint32_t)__ldg(d + (int64_t)b * a.ld[l]) << 16);
+  for (int b0 = 0; b0 < a.B; b0 += 16) {            // B is a multiple of 16: 16 loads in flight, added in order
+    uint16_t v[16];
+#pragma unroll
+    for (int u = 0; u < 16; ++u) v[u] = __ldg(d + (int64_t)(b0 + u) * a.ld[l]);
+#pragma unroll
+    for (int u = 0; u < 16; ++u) g += __uint_as_float((uint32_t)v[u] << 16);
+  }
   float* bp = a.params + (int64_t)n * a.m_pad + a.b_off[l] + j;
   if (a.vel != nullptr) {
     float* vp = a.vel + (int64_t)n * a.m_pad + a.b_off[l] + j;
