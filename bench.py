@@ -108,7 +108,7 @@ class ClockSampler:
 # capture summarised in profiles/; valid only while the kernel's source section is unchanged.
 NCU_TRAFFIC = {
     ("cfg4", "update"): {"bytes_per_iteration": 2.22e9 + 3.04e9, "launches_per_iteration": 4,   # read + written, four launches
-                         "kernel_sha256": "313230a269f1d87cf4cd1280b04fab24b792ac0b4a43d468bc28e5c320eaad4e"},
+                         "kernel_sha256": "8c0c30587d29142b1db957df042caf0716f231947833abf2cb8d4da688528bcf"},
 }
 
 
