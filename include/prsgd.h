@@ -246,6 +246,11 @@ int prsgd_get_velocity_stacked(prsgd_ctx* ctx, float* dst, int dst_on_device);
  * kernel works on: 64 (four pipeline stages per SM), 128 (two), or 0 = chosen per launch from
  * the layer size.  A tuning knob only: every setting produces the same bits. */
 #define PRSGD_OPT_UPDATE_TILE 3
+/* PRSGD_OPT_FUSED_EPILOGUES (default 1, tensor-core path): the softmax cross-entropy gradient runs
+ * in the epilogue of the last forward GEMM and each bias step in the epilogue that forms that layer's
+ * dZ, when the class count d_L is at most 128.  With 0 (or d_L > 128) they run as kernels of their
+ * own.  The two forms agree to fp32 rounding (the stand-alone bias kernel sums the bf16-rounded dZ). */
+#define PRSGD_OPT_FUSED_EPILOGUES 5
 int prsgd_set_option(prsgd_ctx* ctx, int32_t option, int64_t value);
 
 /* Kernel families of the hot path, for prsgd_get_profile. */

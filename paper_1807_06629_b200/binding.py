@@ -24,6 +24,7 @@ OPT_FUSED_AVERAGE = 1
 OPT_PROFILE = 2
 OPT_UPDATE_TILE = 3
 OPT_GRAPH = 4
+OPT_FUSED_EPILOGUES = 5
 KERNEL_FAMILIES = ("forward", "softmax", "dx", "update", "update_average", "average", "misc")
 MAX_LAYERS = 16
 

@@ -7,7 +7,6 @@
 
 namespace prsgd {
 
-__device__ __forceinline__ float4 ld_stream(const float4* p) { return __ldcs(p); }
 __device__ __forceinline__ void st_stream(float4* p, float4 v) { __stcs(p, v); }
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
@@ -17,52 +16,67 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return (a >> 16) | (b & 0xFFFF0000u);
 }
 
+template <int V> struct LaneVec;
+template <> struct LaneVec<4> { using type = float4; };
+template <> struct LaneVec<2> { using type = float2; };
+
+__device__ __forceinline__ void acc_lane(float4& s, const float4& v) { s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w; }
+__device__ __forceinline__ void acc_lane(float2& s, const float2& v) { s.x += v.x; s.y += v.y; }
+__device__ __forceinline__ float4 div_lane(const float4& s, float n) {
+  return make_float4(__fdiv_rn(s.x, n), __fdiv_rn(s.y, n), __fdiv_rn(s.z, n), __fdiv_rn(s.w, n));
+}
+__device__ __forceinline__ float2 div_lane(const float2& s, float n) { return make_float2(__fdiv_rn(s.x, n), __fdiv_rn(s.y, n)); }
+__device__ __forceinline__ void st_shadow(uint16_t* row, int64_t c, const float4& y) {
+  reinterpret_cast<uint2*>(row)[c] = make_uint2(pack_bf16x2(y.x, y.y), pack_bf16x2(y.z, y.w));
+}
+__device__ __forceinline__ void st_shadow(uint16_t* row, int64_t c, const float2& y) {
+  reinterpret_cast<uint32_t*>(row)[c] = pack_bf16x2(y.x, y.y);
+}
+
 // MODE 0: average + broadcast in place; MODE 1: average only, written to `out` (one row);
 // MODE 2: plain sum of the rows (no division) written to `out`: the local part of an average whose
 // rows are spread over several GPUs.
-// One thread owns 4 consecutive columns (one 128-bit lane); the tail m % 4 is done by scalar threads.
-template <int MODE, bool SHADOW>
+// One thread owns V consecutive columns (a 128-bit lane for V = 4, a 64-bit lane for V = 2); the tail
+// m % V is done by scalar threads.  V = 2 doubles the number of blocks, which evens out the load of
+// the SMs when a row is so short that 128-bit lanes give less than about two waves of blocks.
+template <int MODE, bool SHADOW, int V = 4>
 __global__ void __launch_bounds__(256) average_rows_kernel(float* __restrict__ P, int64_t N, int64_t m,
                                                            int64_t row_stride, float* __restrict__ out,
                                                            uint16_t* __restrict__ shadow,
                                                            const DeviceStatus* status = nullptr) {
+  using Vec = typename LaneVec<V>::type;
   constexpr int U = 8;
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");   // no-op unless launched as a programmatic dependent
   if (status != nullptr && status->error != 0u) return;   // a recorded expired wait: leave the store alone
-  const int64_t cols4 = m >> 2;
+  const int64_t colsV = m / V;
   const int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   const float fN = (float)N;
-  if (c < cols4) {
-    float4* base = reinterpret_cast<float4*>(P) + c;
-    const int64_t s4 = row_stride >> 2;
-    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (c < colsV) {
+    Vec* base = reinterpret_cast<Vec*>(P) + c;
+    const int64_t sV = row_stride / V;
+    Vec s = Vec();
     int64_t i = 0;
     for (; i + U <= N; i += U) {
-      float4 v[U];
+      Vec v[U];
 #pragma unroll
-      for (int u = 0; u < U; ++u) v[u] = ld_stream(base + (i + u) * s4);
+      for (int u = 0; u < U; ++u) v[u] = __ldcs(base + (i + u) * sV);
 #pragma unroll
-      for (int u = 0; u < U; ++u) { s.x += v[u].x; s.y += v[u].y; s.z += v[u].z; s.w += v[u].w; }
+      for (int u = 0; u < U; ++u) acc_lane(s, v[u]);
     }
-    for (; i < N; ++i) {
-      float4 v = ld_stream(base + i * s4);
-      s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
-    }
-    float4 y = MODE == 2 ? s : make_float4(__fdiv_rn(s.x, fN), __fdiv_rn(s.y, fN), __fdiv_rn(s.z, fN), __fdiv_rn(s.w, fN));
+    for (; i < N; ++i) acc_lane(s, __ldcs(base + i * sV));
+    const Vec y = MODE == 2 ? s : div_lane(s, fN);
     if (MODE == 0) {
 #pragma unroll 8
-      for (int64_t r = 0; r < N; ++r) st_stream(base + r * s4, y);
+      for (int64_t r = 0; r < N; ++r) __stcs(base + r * sV, y);
       if (SHADOW) {
-        uint2 h = make_uint2(pack_bf16x2(y.x, y.y), pack_bf16x2(y.z, y.w));
-        uint2* sb = reinterpret_cast<uint2*>(shadow) + c;
-        for (int64_t r = 0; r < N; ++r) sb[r * s4] = h;
+        for (int64_t r = 0; r < N; ++r) st_shadow(shadow + r * row_stride, c, y);
       }
     } else {
-      reinterpret_cast<float4*>(out)[c] = y;
+      reinterpret_cast<Vec*>(out)[c] = y;
     }
-  } else if (c < cols4 + (m & 3)) {
-    const int64_t j = (cols4 << 2) + (c - cols4);
+  } else if (c < colsV + (m % V)) {
+    const int64_t j = colsV * V + (c - colsV);
     float s = 0.f;
     for (int64_t i = 0; i < N; ++i) s += P[i * row_stride + j];
     float y = MODE == 2 ? s : __fdiv_rn(s, fN);
@@ -76,6 +90,9 @@ __global__ void __launch_bounds__(256) average_rows_kernel(float* __restrict__ P
     }
   }
 }
+
+// Rows shorter than this many columns are averaged with 64-bit lanes (see average_rows_kernel).
+constexpr int64_t kAvgNarrowLaneBelow = 8000000;
 
 // every row <- src / divisor on columns [0, 4 * cols4) (and the bf16 shadow): the restart after an
 // average whose sum was formed elsewhere (all-reduce over GPUs)

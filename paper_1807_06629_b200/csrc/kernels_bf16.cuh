@@ -95,6 +95,19 @@ struct StreamArgs {
   const uint16_t* mask_src;  // bf16 a_{l-1} [N][B][ld_out] (TC_DX)
   const uint8_t* active;
   DeviceStatus* status;
+  // Bias step folded into the epilogue that produces dZ of the output layer (TC_DX: the layer below;
+  // TC_FWD_LINEAR with `softmax`: the last layer): b <- b - gamma sum_b dZ[b, :]
+  float* bias_rw;            // params + b_off of that layer (worker stride bias_stride), or nullptr
+  float* bias_vel;           // its momentum segment, or nullptr
+  float gamma, mu;
+  // Softmax cross-entropy gradient in the epilogue of the last forward GEMM (needs tiles_m == 1)
+  int softmax;
+  const int32_t* Y;          // labels [N][P]
+  int64_t P;
+  uint16_t* delta_bk;        // bf16 dZ_L [N][B][ld_delta]
+  int ld_delta;
+  float* row_losses;         // [N][B]
+  int32_t* draws;            // [N]
 };
 
 // Persistent: one CTA per SM walks (tile, worker) items.  Warp 0 issues TMA, warp 1 issues MMAs,
@@ -105,12 +118,17 @@ struct StreamArgs {
 constexpr int kStreamThreads = 192;
 constexpr uint32_t kTileA = 16384;   // 128 x 64 bf16
 
+constexpr int kLogitLd = 129;        // row pitch (floats) of the logits tile the softmax epilogue keeps in shared memory
+
 __host__ __device__ inline uint32_t stream_stage_bytes(int B) { return 2u * (kTileA + (uint32_t)B * 128u); }
-inline int stream_stages(int B) {
-  int s = (int)(200000u / stream_stage_bytes(B));
+__host__ __device__ inline uint32_t stream_logit_bytes(int B, bool softmax) { return softmax ? (uint32_t)B * kLogitLd * 4u : 0u; }
+inline int stream_stages(int B, bool softmax = false) {
+  int s = (int)((200000u - stream_logit_bytes(B, softmax)) / stream_stage_bytes(B));
   return s > 6 ? 6 : s;
 }
-inline size_t stream_smem_bytes(int B) { return (size_t)stream_stages(B) * stream_stage_bytes(B) + 1024 + 256; }
+inline size_t stream_smem_bytes(int B, bool softmax = false) {
+  return (size_t)stream_stages(B, softmax) * stream_stage_bytes(B) + 1024 + 256 + stream_logit_bytes(B, softmax);
+}
 
 template <int MODE>
 __global__ void __launch_bounds__(kStreamThreads, 1) tc_stream_kernel(const __grid_constant__ CUtensorMap mapW,
@@ -131,6 +149,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) tc_stream_kernel(const __gr
   auto acc_empty = [&](int q) { return bar0 + 144u + 8u * q; };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen + (size_t)S * stage_bytes + 160);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + (size_t)S * stage_bytes + 164);
+  float* zs = reinterpret_cast<float*>(gen + (size_t)S * stage_bytes + 256);   // [B][kLogitLd], softmax epilogue only
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t ncols = 2 * a.B < 32 ? 32u : (uint32_t)(2 * a.B);   // two accumulators of B columns
@@ -248,6 +267,15 @@ __global__ void __launch_bounds__(kStreamThreads, 1) tc_stream_kernel(const __gr
       mask_fetch(0, mk_cur);
       float bias = 0.f;
       if (MODE != TC_DX && valid) bias = a.bias[(int64_t)n * a.bias_stride + m];
+      const bool smx = MODE == TC_FWD_LINEAR && a.softmax != 0;
+      float gsum = 0.f;                                   // sum over the minibatch of this feature's dZ
+      const int etid = tid - 64;                          // 0..127 among the epilogue threads
+      uint32_t blk = 0;
+      int label = 0;
+      if (MODE == TC_FWD_LINEAR && smx) {                 // the label of this thread's row, fetched ahead of the wait
+        blk = draw_block(a.draw.seed, a.draw.worker0 + n, draw_t(a.draw), a.draw.n_blocks);
+        label = a.Y[(int64_t)n * a.P + (int64_t)blk * a.B + etid / (128 / a.B)];
+      }
       const int q = it & 1;
       ok = __all_sync(0xffffffffu, mbar_wait(acc_full(q), (it >> 1) & 1u, abort_flag, a.status, 0x103));
       if (!ok) break;
@@ -266,9 +294,12 @@ __global__ void __launch_bounds__(kStreamThreads, 1) tc_stream_kernel(const __gr
             if (MODE == TC_FWD_RELU) {
               a.out_bk[o] = f32_to_bf16_rn(fmaxf(x + bias, 0.f));
             } else if (MODE == TC_FWD_LINEAR) {
-              a.out_f32[o] = x + bias;
+              if (smx) zs[(c0 + j) * kLogitLd + m] = x + bias;
+              else a.out_f32[o] = x + bias;
             } else {
-              a.out_bk[o] = (mk_cur[j] & 0x7FFFu) != 0 ? f32_to_bf16_rn(x) : (uint16_t)0;
+              const float d = (mk_cur[j] & 0x7FFFu) != 0 ? x : 0.f;
+              gsum += d;
+              a.out_bk[o] = f32_to_bf16_rn(d);
             }
           }
         }
@@ -280,6 +311,47 @@ __global__ void __launch_bounds__(kStreamThreads, 1) tc_stream_kernel(const __gr
       tc_fence_before();
       mbar_arrive(acc_empty(q));
       ++it;
+      if (MODE == TC_FWD_LINEAR && smx) {
+        // Softmax cross-entropy gradient dZ_L = (softmax(z) - onehot(y)) / B and the per-sample loss.
+        // The logits of the whole minibatch sit in shared memory; row b belongs to the T = 128 / B
+        // neighbouring threads etid = b T .. b T + T - 1, each of which takes every T-th class.
+        named_bar_sync(1, 128);
+        const int C = a.M_total;
+        const int T = 128 / a.B, sub = etid % T, b = etid / T;
+        const float invB = 1.f / (float)a.B;
+        float* z = zs + b * kLogitLd;
+        float mx = -INFINITY;
+        for (int cc = sub; cc < C; cc += T) mx = fmaxf(mx, z[cc]);
+        for (int o = T >> 1; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        float se = 0.f;
+        for (int cc = sub; cc < C; cc += T) se += expf(z[cc] - mx);
+        for (int o = T >> 1; o > 0; o >>= 1) se += __shfl_xor_sync(0xffffffffu, se, o);
+        const float lse = mx + logf(se);
+        const float zl = z[label];
+        __syncwarp();
+        for (int cc = sub; cc < C; cc += T) z[cc] = (expf(z[cc] - lse) - (cc == label ? 1.f : 0.f)) * invB;
+        if (sub == 0) a.row_losses[(int64_t)n * a.B + b] = lse - zl;
+        if (etid == 0) a.draws[n] = (int32_t)blk;
+        named_bar_sync(1, 128);
+        if (valid) {
+          for (int bb = 0; bb < a.B; ++bb) gsum += zs[bb * kLogitLd + m];
+        }
+        uint16_t* dn = a.delta_bk + (int64_t)n * a.B * a.ld_delta;
+        for (int idx = etid; idx < a.B * C; idx += 128) {
+          const int bb = idx / C, cc = idx - bb * C;
+          dn[bb * a.ld_delta + cc] = f32_to_bf16_rn(zs[bb * kLogitLd + cc]);
+        }
+        named_bar_sync(1, 128);                           // the tile is free for the next item
+      }
+      if ((MODE == TC_DX || smx) && a.bias_rw != nullptr && valid) {
+        float* bp = a.bias_rw + (int64_t)n * a.bias_stride + m;
+        if (a.bias_vel != nullptr) {                      // momentum form of the local step
+          float* vp = a.bias_vel + (int64_t)n * a.bias_stride + m;
+          gsum = fmaf(a.mu, *vp, gsum);
+          *vp = gsum;
+        }
+        *bp = fmaf(-a.gamma, gsum, *bp);
+      }
     }
   }
   __syncwarp();
@@ -662,7 +734,8 @@ inline int tc_create(prsgd_ctx* c, std::string* err) {
   cudaError_t e = cudaSuccess;
   const int big = (int)stream_smem_bytes(c->B);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_stream_kernel<TC_FWD_RELU>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_stream_kernel<TC_FWD_LINEAR>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+  const int big_sm = (int)stream_smem_bytes(c->B, true);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_stream_kernel<TC_FWD_LINEAR>, cudaFuncAttributeMaxDynamicSharedMemorySize, big > big_sm ? big : big_sm);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_stream_kernel<TC_DX>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<false, 64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<64, false>::smem(c->B));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<true, 64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<64, false>::smem(c->B));
@@ -704,6 +777,10 @@ inline int tc_bind_data(prsgd_ctx* c, std::string* err) {
   return rc;
 }
 
+// The softmax cross-entropy gradient and every bias step run inside GEMM epilogues when the class
+// count fits one 128-row tile (and PRSGD_OPT_FUSED_EPILOGUES is on); otherwise as kernels of their own.
+inline bool tc_epilogues_fused(const prsgd_ctx* c) { return c->fused_epilogues != 0 && c->dims[c->L] <= 128; }
+
 // forward GEMM of layer l (1-based)
 inline void tc_launch_forward(prsgd_ctx* c, int l, const DrawArgs& dr, const uint8_t* active) {
   TcState* st = static_cast<TcState*>(c->tc);
@@ -715,9 +792,17 @@ inline void tc_launch_forward(prsgd_ctx* c, int l, const DrawArgs& dr, const uin
   a.out_bk = c->buf.act_bk[l]; a.out_f32 = c->buf.act_f32[l];
   a.bias = c->params + ly.b_off; a.bias_stride = c->m_pad;
   a.active = active; a.status = c->status;
+  const bool softmax = l == c->L && tc_epilogues_fused(c);
+  if (softmax) {        // the softmax-CE gradient, the loss and the step of b_L happen in this launch's epilogue
+    a.softmax = 1; a.stages = stream_stages(c->B, true);
+    a.Y = c->Y; a.P = c->P; a.delta_bk = c->buf.delta_bk[l]; a.ld_delta = c->buf.ld[l];
+    a.row_losses = c->losses; a.draws = c->draws;
+    a.bias_rw = c->params + ly.b_off; a.gamma = c->gamma; a.mu = c->mu;
+    a.bias_vel = c->velocity != nullptr ? c->velocity + ly.b_off : nullptr;
+  }
   const int items = a.tiles_m * c->N;
   dim3 grid(items < st->num_sms ? items : st->num_sms);
-  const size_t smem = stream_smem_bytes(c->B);
+  const size_t smem = stream_smem_bytes(c->B, softmax);
   if (l < c->L)
     launch_pdl(tc_stream_kernel<TC_FWD_RELU>, grid, kStreamThreads, smem, c->stream, st->layer[l - 1].shadow_k, st->layer[l - 1].act_in, a);
   else
@@ -734,6 +819,10 @@ inline void tc_launch_dx(prsgd_ctx* c, int l, const DrawArgs& dr, const uint8_t*
   a.pool = 0; a.draw = dr; a.ld_out = c->buf.ld[l - 1];
   a.out_bk = c->buf.delta_bk[l - 1]; a.mask_src = c->buf.act_bk[l - 1];
   a.active = active; a.status = c->status;
+  if (tc_epilogues_fused(c)) {      // the step of b_{l-1} rides on the epilogue that forms dZ_{l-1}
+    a.bias_rw = c->params + c->layer[l - 2].b_off; a.bias_stride = c->m_pad; a.gamma = c->gamma; a.mu = c->mu;
+    a.bias_vel = c->velocity != nullptr ? c->velocity + c->layer[l - 2].b_off : nullptr;
+  }
   const int items = a.tiles_m * c->N;
   dim3 grid(items < st->num_sms ? items : st->num_sms);
   launch_pdl(tc_stream_kernel<TC_DX>, grid, kStreamThreads, stream_smem_bytes(c->B), c->stream, st->layer[l - 1].shadow_mn,

@@ -291,7 +291,8 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging) {
     tc_launch_forward(c, l, dr, act_mask);
     LAUNCH_CHECK(c);
   }
-  {
+  const bool epi = tc_epilogues_fused(c);
+  if (!epi) {
     SoftmaxArgs a{};
     a.logits = c->buf.act_f32[L]; a.ldz = c->buf.ld[L];
     a.delta_bk = c->buf.delta_bk[L]; a.ld_bf = c->buf.ld[L];
@@ -311,9 +312,11 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging) {
     tc_launch_update(c, l, dr, act_mask, fuse);
     LAUNCH_CHECK(c);
   }
-  prof_begin(c, PRSGD_KERNEL_MISC);
-  tc_launch_bias(c, act_mask);
-  LAUNCH_CHECK(c);
+  if (!epi) {
+    prof_begin(c, PRSGD_KERNEL_MISC);
+    tc_launch_bias(c, act_mask);
+    LAUNCH_CHECK(c);
+  }
   if (fuse) {
     for (int l = 1; l <= L; ++l) {
       prof_begin(c, PRSGD_KERNEL_MISC);
@@ -325,14 +328,24 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging) {
 }
 
 int launch_average(prsgd_ctx* c) {
-  const int64_t threads = c->m_pad / 4;
+  const bool narrow = c->m_pad < kAvgNarrowLaneBelow;      // m_pad is a multiple of 32: no scalar tail either way
+  const int64_t threads = narrow ? c->m_pad / 2 : c->m_pad / 4;
   prof_begin(c, PRSGD_KERNEL_AVERAGE);
-  if (c->precision == PRSGD_PRECISION_BF16)
-    average_rows_kernel<0, true><<<grid1d(threads, 256), 256, 0, c->stream>>>(c->params, c->N, c->m_pad, c->m_pad,
-                                                                            nullptr, c->shadow, c->status);
-  else
-    average_rows_kernel<0, false><<<grid1d(threads, 256), 256, 0, c->stream>>>(c->params, c->N, c->m_pad, c->m_pad,
-                                                                             nullptr, nullptr, c->status);
+  if (c->precision == PRSGD_PRECISION_BF16) {
+    if (narrow)
+      average_rows_kernel<0, true, 2><<<grid1d(threads, 256), 256, 0, c->stream>>>(c->params, c->N, c->m_pad, c->m_pad,
+                                                                                 nullptr, c->shadow, c->status);
+    else
+      average_rows_kernel<0, true><<<grid1d(threads, 256), 256, 0, c->stream>>>(c->params, c->N, c->m_pad, c->m_pad,
+                                                                              nullptr, c->shadow, c->status);
+  } else {
+    if (narrow)
+      average_rows_kernel<0, false, 2><<<grid1d(threads, 256), 256, 0, c->stream>>>(c->params, c->N, c->m_pad, c->m_pad,
+                                                                                  nullptr, nullptr, c->status);
+    else
+      average_rows_kernel<0, false><<<grid1d(threads, 256), 256, 0, c->stream>>>(c->params, c->N, c->m_pad, c->m_pad,
+                                                                               nullptr, nullptr, c->status);
+  }
   LAUNCH_CHECK(c);
   if (c->velocity != nullptr && c->average_velocity) {     // momentum buffers averaged like the models
     prof_begin(c, PRSGD_KERNEL_AVERAGE);
@@ -566,7 +579,7 @@ void period_key(const prsgd_ctx* c, uint64_t (&key)[12]) {
   key[0] = gbits; key[1] = (uint64_t)c->I; key[2] = (uint64_t)c->fused_average; key[3] = (uint64_t)c->upd_tile;
   key[4] = c->has_mask ? 1 : 0; key[5] = reinterpret_cast<uint64_t>(c->velocity); key[6] = mbits;
   key[7] = (uint64_t)c->average_velocity; key[8] = reinterpret_cast<uint64_t>(c->X);
-  key[9] = reinterpret_cast<uint64_t>(c->Y); key[10] = (uint64_t)c->worker0; key[11] = 0;
+  key[9] = reinterpret_cast<uint64_t>(c->Y); key[10] = (uint64_t)c->worker0; key[11] = (uint64_t)c->fused_epilogues;
 }
 
 // One whole averaging period (I iterations starting right after an average) as a CUDA graph: the
@@ -868,6 +881,7 @@ int prsgd_set_option(prsgd_ctx* c, int32_t option, int64_t value) {
   if (option == PRSGD_OPT_FUSED_AVERAGE) { c->fused_average = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_PROFILE) { c->profile = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_GRAPH) { c->use_graph = value != 0; return PRSGD_OK; }
+  if (option == PRSGD_OPT_FUSED_EPILOGUES) { c->fused_epilogues = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_UPDATE_TILE) {
     if (value != 0 && value != 64 && value != 128) return fail(c, PRSGD_ERR_ARG, "update tile width must be 0, 64 or 128");
     c->upd_tile = (int)value;
@@ -930,10 +944,16 @@ int prsgd_average_rows(float* d_P, int64_t N, int64_t m, int64_t row_stride, voi
   if (!aligned(d_P, 16) || (row_stride % 4) != 0)
     return fail(nullptr, PRSGD_ERR_ALIGN, "d_P must be 16-byte aligned and row_stride a multiple of 4");
   if (m == 0) return PRSGD_OK;
-  const int64_t threads = m / 4 + (m & 3);
-  if ((threads + 255) / 256 > 0x7fffffffll) return fail(nullptr, PRSGD_ERR_SIZE, "m too large");
-  average_rows_kernel<0, false><<<grid1d(threads, 256), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
-      d_P, N, m, row_stride, nullptr, nullptr);
+  if (m < kAvgNarrowLaneBelow) {
+    const int64_t threads = m / 2 + (m & 1);
+    average_rows_kernel<0, false, 2><<<grid1d(threads, 256), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+        d_P, N, m, row_stride, nullptr, nullptr);
+  } else {
+    const int64_t threads = m / 4 + (m & 3);
+    if ((threads + 255) / 256 > 0x7fffffffll) return fail(nullptr, PRSGD_ERR_SIZE, "m too large");
+    average_rows_kernel<0, false><<<grid1d(threads, 256), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+        d_P, N, m, row_stride, nullptr, nullptr);
+  }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return fail(nullptr, PRSGD_ERR_CUDA, std::string("average_rows: ") + cudaGetErrorString(e));
   return PRSGD_OK;

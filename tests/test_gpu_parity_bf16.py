@@ -127,6 +127,63 @@ def test_fused_average_equals_update_then_average_bit_for_bit(torch_cuda):
             assert np.array_equal(outs[0], o)
 
 
+def _segments(dims):
+    """[(is_weight, start, stop)] of a canonical parameter vector."""
+    out, off = [], 0
+    for l in range(len(dims) - 1):
+        for is_w, cnt in ((True, dims[l] * dims[l + 1]), (False, dims[l + 1])):
+            out.append((is_w, off, off + cnt))
+            off += cnt
+    return out
+
+
+@pytest.mark.parametrize("w", [SMALL[0], SMALL[3], SMALL[4], SMALL[6]], ids=lambda w: w.name)
+def test_epilogue_softmax_and_bias_steps_equal_the_standalone_kernels(torch_cuda, w):
+    """Softmax-CE gradient in the last forward GEMM's epilogue and bias steps in the dZ epilogues against the
+    same work done by kernels of their own: identical dZ, so identical weights after one iteration; the bias
+    steps differ only in summing dZ before instead of after its rounding to bf16."""
+    from paper_1807_06629_b200 import binding
+    X, Y, x0 = make_inputs(w)
+    outs = []
+    for fused in (1, 0):
+        p = make_ctx(w, X, Y, x0, I=0)
+        p.set_option(binding.OPT_FUSED_EPILOGUES, fused)
+        n0 = p.get_launch_count()
+        p.local_steps(1)
+        outs.append((p.get_params_stacked(), p.get_losses(), p.get_draws().tolist(), p.get_launch_count() - n0))
+    (a, la, da, na), (b, lb, db, nb) = outs
+    assert nb == na + 2                                   # the softmax kernel and the bias kernel
+    assert da == db and np.array_equal(la, lb)
+    x0s = np.tile(x0, (w.N, 1))
+    for is_w, lo, hi in _segments(w.dims):
+        if is_w:
+            assert np.array_equal(a[:, lo:hi], b[:, lo:hi])
+        else:
+            assert rel_l2(a[:, lo:hi] - x0s[:, lo:hi], b[:, lo:hi] - x0s[:, lo:hi]) <= 5e-3
+
+
+@pytest.mark.parametrize("fused", [1, 0])
+def test_standalone_softmax_and_bias_kernels_against_the_oracle(torch_cuda, fused):
+    """More than 128 classes do not fit one tile of the last GEMM, so the stand-alone kernels run whatever the
+    option says; a 10-class net with the option off takes the same route."""
+    from paper_1807_06629_b200 import binding
+    for w in (_w("tc-200-classes", 2, (64, 128, 200), 32), SMALL[1]):
+        X, Y, x0 = make_inputs(w)
+        p = make_ctx(w, X, Y, x0)
+        p.set_option(binding.OPT_FUSED_EPILOGUES, fused)
+        if w.dims[-1] <= 128 and fused:
+            continue                                      # that combination is every other test of this file
+        x0s = np.tile(x0, (w.N, 1)).astype(np.float64)
+        losses = {}
+        want = oracle_run(w, X, Y, x0s, 0, w.I, losses=losses)
+        p.local_steps(w.I)
+        got = p.get_params_stacked()
+        assert np.allclose(p.get_losses(), [losses[(i, w.I)] for i in range(w.N)], rtol=2e-2, atol=2e-3)
+        assert all(np.array_equal(got[i], got[0]) for i in range(w.N))
+        assert rel_l2(got, want) <= TOL_PERIOD
+        assert rel_l2(got - x0s, want - x0s) <= TOL_UPDATE, rel_l2(got - x0s, want - x0s)
+
+
 def test_shadow_tracks_master_and_padding_stays_zero(torch_cuda):
     torch = torch_cuda
     w = SMALL[4]
@@ -199,6 +256,9 @@ def test_momentum_step_on_the_tensor_core_path(torch_cuda, avg_v):
         X, Y, x0 = make_inputs(w)
         x0 = with_margin(x0, w.dims)
         p = make_ctx(w, X, Y, x0)
+        if w is SMALL[3]:                                 # one workload takes the stand-alone bias kernel
+            from paper_1807_06629_b200 import binding
+            p.set_option(binding.OPT_FUSED_EPILOGUES, 0)
         p.enable_momentum(0.9, average_velocity=avg_v)
         fn = orc.mlp_grad_fn(w.dims, X.astype(np.float64), Y, w.B, w.seed)
         xs = np.tile(x0, (w.N, 1)).astype(np.float64)
