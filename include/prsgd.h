@@ -251,6 +251,11 @@ int prsgd_get_velocity_stacked(prsgd_ctx* ctx, float* dst, int dst_on_device);
  * dZ, when the class count d_L is at most 128.  With 0 (or d_L > 128) they run as kernels of their
  * own.  The two forms agree to fp32 rounding (the stand-alone bias kernel sums the bf16-rounded dZ). */
 #define PRSGD_OPT_FUSED_EPILOGUES 5
+/* PRSGD_OPT_EARLY_LOADS (default 1, tensor-core path): a kernel requests the weight tiles of its first
+ * pipeline stages before it waits for the previous launch to complete, when that launch cannot be
+ * writing them (every layer's forward GEMM but the first, every dX GEMM, the master tiles of every
+ * update; never while a worker mask is set).  Same bits either way. */
+#define PRSGD_OPT_EARLY_LOADS 6
 int prsgd_set_option(prsgd_ctx* ctx, int32_t option, int64_t value);
 
 /* Kernel families of the hot path, for prsgd_get_profile. */

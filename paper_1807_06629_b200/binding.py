@@ -25,6 +25,7 @@ OPT_PROFILE = 2
 OPT_UPDATE_TILE = 3
 OPT_GRAPH = 4
 OPT_FUSED_EPILOGUES = 5
+OPT_EARLY_LOADS = 6
 KERNEL_FAMILIES = ("forward", "softmax", "dx", "update", "update_average", "average", "misc")
 MAX_LAYERS = 16
 

@@ -46,8 +46,8 @@ __global__ void __launch_bounds__(256) average_rows_kernel(float* __restrict__ P
                                                            const DeviceStatus* status = nullptr) {
   using Vec = typename LaneVec<V>::type;
   constexpr int U = 8;
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");   // no-op unless launched as a programmatic dependent
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // after the wait, like every kernel of the tensor-core path
   if (status != nullptr && status->error != 0u) return;   // a recorded expired wait: leave the store alone
   const int64_t colsV = m / V;
   const int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;

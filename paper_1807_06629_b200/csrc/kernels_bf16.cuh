@@ -101,6 +101,7 @@ struct StreamArgs {
   float* bias_vel;           // its momentum segment, or nullptr
   float gamma, mu;
   // Softmax cross-entropy gradient in the epilogue of the last forward GEMM (needs tiles_m == 1)
+  int prefetch;              // 1: the weight tiles may be requested before the previous launch has completed
   int softmax;
   const int32_t* Y;          // labels [N][P]
   int64_t P;
@@ -166,8 +167,38 @@ __global__ void __launch_bounds__(kStreamThreads, 1) tc_stream_kernel(const __gr
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  pdl_trigger();
-  pdl_wait();            // everything above overlapped the previous kernel's tail; memory is touched below
+  // Weight tiles of a pipeline step (two 64-wide K blocks of the 128-row tile of worker n).
+  auto load_weights = [&](int s, int ks, int m0, int n) {
+    const uint32_t sa = base + (uint32_t)s * stage_bytes;
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      const int k0 = (2 * ks + j) * 64;              // a block past the end of K is zero-filled by TMA
+      if (MODE == TC_DX) {
+        tma_load_3d(sa + j * kTileA, &mapW, full_bar(s), m0, k0, n);
+        tma_load_3d(sa + j * kTileA + 8192u, &mapW, full_bar(s), m0 + 64, k0, n);
+      } else {
+        tma_load_3d(sa + j * kTileA, &mapW, full_bar(s), k0, m0, n);
+      }
+    }
+  };
+  auto load_operand = [&](int s, int ks, int row0, int n) {
+    const uint32_t sb = base + (uint32_t)s * stage_bytes + 2u * kTileA;
+#pragma unroll
+    for (int j = 0; j < 2; ++j) tma_load_3d(sb + j * b_box, &mapB, full_bar(s), (2 * ks + j) * 64, row0, n);
+  };
+  // The weights this launch reads were last written before the previous launch began (the host sets
+  // `prefetch` only then), so the first stages' weight tiles are requested while that launch drains.
+  uint32_t pre = 0;
+  if (warp == 0 && lane == 0 && a.prefetch != 0 && (int)blockIdx.x < a.tiles_m * a.N) {
+    const int n = (int)blockIdx.x / a.tiles_m, m0 = ((int)blockIdx.x % a.tiles_m) * 128;
+    pre = (uint32_t)(a.k_steps < S ? a.k_steps : S);
+    for (uint32_t ks = 0; ks < pre; ++ks) {
+      mbar_expect_tx(full_bar(ks), stage_bytes);
+      load_weights((int)ks, (int)ks, m0, n);
+    }
+  }
+  pdl_wait();            // everything above overlapped the previous kernel's tail; dependent memory is touched below
+  pdl_trigger();         // only now: the next launch's early loads may overlap this launch, never an older one
   const uint32_t tmem = *tmem_slot;
   // a wait that expired in an earlier CTA or launch turns the rest of the work into a no-op
   if (tid == 0) *abort_flag = *(volatile unsigned int*)&a.status->error != 0u ? 1 : 0;
@@ -186,27 +217,25 @@ __global__ void __launch_bounds__(kStreamThreads, 1) tc_stream_kernel(const __gr
       for (int ks = 0; ks < a.k_steps; ++ks, ++g) {
         const int s = g % S;
         const uint32_t ph = (g / S) & 1u;
-        ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, a.status, 0x101);
-        if (!ok) break;
-        const uint32_t sa = base + (uint32_t)s * stage_bytes, sb = sa + 2u * kTileA;
-        mbar_expect_tx(full_bar(s), stage_bytes);
-#pragma unroll
-        for (int j = 0; j < 2; ++j) {
-          const int k0 = (2 * ks + j) * 64;          // a block past the end of K is zero-filled by TMA
-          if (MODE == TC_DX) {
-            tma_load_3d(sa + j * kTileA, &mapW, full_bar(s), m0, k0, n);
-            tma_load_3d(sa + j * kTileA + 8192u, &mapW, full_bar(s), m0 + 64, k0, n);
-          } else {
-            tma_load_3d(sa + j * kTileA, &mapW, full_bar(s), k0, m0, n);
-          }
-          tma_load_3d(sb + j * b_box, &mapB, full_bar(s), k0, row0, n);
+        if (g >= pre) {                               // (the early steps already have their weights under way)
+          ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, a.status, 0x101);
+          if (!ok) break;
+          mbar_expect_tx(full_bar(s), stage_bytes);
+          load_weights(s, ks, m0, n);
         }
+        load_operand(s, ks, row0, n);
       }
     }
+    if (total_items == 0 && pre > 0) {   // nothing will consume the early tiles: complete their stages
+      for (uint32_t ks = 0; ks < pre; ++ks) load_operand((int)ks, (int)ks, 0, (int)blockIdx.x / a.tiles_m);
+      g = pre;
+    }
     if (*abort_flag && g > 0) {   // let the copies already in flight land before the CTA goes away
-      const long long t0 = clock64();
-      const uint32_t last = g - 1;
-      while (!mbar_try_wait(full_bar(last % S), (last / S) & 1u) && clock64() - t0 < 200000000ll) {}
+      const uint32_t first = g > (uint32_t)S ? g - (uint32_t)S : 0u;
+      for (uint32_t q = first; q < g; ++q) {
+        const long long t0 = clock64();
+        while (!mbar_try_wait(full_bar(q % S), (q / S) & 1u) && clock64() - t0 < 200000000ll) {}
+      }
     }
   } else if (warp == 1 && lane == 0) {
     // ---------------- MMA issuer
@@ -372,6 +401,7 @@ struct UpdateArgs {
   DrawArgs draw;
   const uint8_t* active;
   DeviceStatus* status;
+  int prefetch;            // 1: master tiles may be requested before the previous launch has completed
 };
 
 constexpr int kUpdThreads = 224;          // warp 0 loader, 1 MMA, 2 storer, 3..6 epilogue
@@ -443,8 +473,31 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  pdl_trigger();
-  pdl_wait();            // set-up above overlapped the previous kernel's tail; memory is touched below
+  auto load_master = [&](int s, int m0, int n0, int n) {
+    mbar_expect_tx(full_w(s), Cfg::kMaster + Cfg::kVel);
+#pragma unroll
+    for (int q = 0; q < NB32; ++q) tma_load_3d(master_u32(s) + q * 16384u, &mapMaster, full_w(s), n0 + 32 * q, m0, n);
+    if (MOM) {
+#pragma unroll
+      for (int q = 0; q < NB32; ++q) tma_load_3d(vel_u32(s) + q * 16384u, &mapVel, full_w(s), n0 + 32 * q, m0, n);
+    }
+  };
+  // The master (and momentum) tiles were last written an iteration ago, so those of the first items
+  // are requested while the previous launch (which only reads the bf16 shadow) drains; `prefetch` is
+  // set by the host when no worker mask is in use, so item k of this CTA is known without reading memory.
+  uint32_t pre = 0;
+  if (warp == 0 && lane == 0 && a.prefetch != 0) {
+    for (int k = 0; k < S; ++k) {
+      const int w = FUSE ? (int)blockIdx.x : (int)blockIdx.x + k * (int)gridDim.x;
+      const int n = FUSE ? k : w / tiles;
+      if (w >= items_all || n >= a.N) break;
+      const int tile = FUSE ? w : w % tiles;
+      load_master(k, (tile / a.tiles_n) * 128, (tile % a.tiles_n) * TN, n);
+      ++pre;
+    }
+  }
+  pdl_wait();            // set-up above overlapped the previous kernel's tail; dependent memory is touched below
+  pdl_trigger();         // only now: the next launch's early loads may overlap this launch, never an older one
   const uint32_t tmem = *tmem_slot;
   if (tid == 0) *abort_flag = *(volatile unsigned int*)&a.status->error != 0u ? 1 : 0;   // an earlier expired wait: no-op
   __syncthreads();
@@ -466,8 +519,10 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
         if (!item_active(n)) continue;
         const int s = it % S;
         const uint32_t ph = (it / S) & 1u;
-        ok = mbar_wait(stage_empty(s), ph ^ 1u, abort_flag, a.status, 0x201);
-        if (!ok) break;
+        if (it >= pre) {                                  // (the early items already have their master tiles under way)
+          ok = mbar_wait(stage_empty(s), ph ^ 1u, abort_flag, a.status, 0x201);
+          if (!ok) break;
+        }
         const int row0 = a.pool ? (int)draw_block(a.draw.seed, a.draw.worker0 + n, draw_t(a.draw), a.draw.n_blocks) * a.B : 0;
         const uint32_t ops = ops_u32(s);
         mbar_expect_tx(full_ops(s), (2u + NB64) * op_box);
@@ -475,20 +530,17 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
         tma_load_3d(ops + op_box, &mapDelta, full_ops(s), m0 + 64, 0, n);
 #pragma unroll
         for (int h = 0; h < NB64; ++h) tma_load_3d(ops + (2u + h) * op_box, &mapAct, full_ops(s), n0 + 64 * h, row0, n);
-        mbar_expect_tx(full_w(s), Cfg::kMaster + Cfg::kVel);
-#pragma unroll
-        for (int q = 0; q < NB32; ++q) tma_load_3d(master_u32(s) + q * 16384u, &mapMaster, full_w(s), n0 + 32 * q, m0, n);
-        if (MOM) {
-#pragma unroll
-          for (int q = 0; q < NB32; ++q) tma_load_3d(vel_u32(s) + q * 16384u, &mapVel, full_w(s), n0 + 32 * q, m0, n);
-        }
+        if (it >= pre) load_master(s, m0, n0, n);
         ++it;
       }
     }
+    if (it < pre) it = pre;        // early tiles that nothing will consume (the launch turned into a no-op)
     if (*abort_flag && it > 0) {   // let the copies already in flight land before the CTA goes away
-      const uint64_t t0 = globaltimer_ns();
-      const uint32_t last = it - 1;
-      while (!mbar_try_wait(full_w(last % S), (last / S) & 1u) && globaltimer_ns() - t0 < 100000000ull) {}
+      const uint32_t first = it > (uint32_t)S ? it - (uint32_t)S : 0u;
+      for (uint32_t q = first; q < it; ++q) {
+        const uint64_t t0 = globaltimer_ns();
+        while (!mbar_try_wait(full_w(q % S), (q / S) & 1u) && globaltimer_ns() - t0 < 100000000ull) {}
+      }
     }
   } else if (warp == 1 && lane == 0) {
     // ---------------- MMA issuer
@@ -667,8 +719,8 @@ struct BiasArgs {
 };
 
 __global__ void __launch_bounds__(128) bias_update_kernel(const BiasArgs a) {
-  ptx::pdl_trigger();
   ptx::pdl_wait();
+  ptx::pdl_trigger();     // after the wait: a later launch's early loads overlap this launch only
   const int l = blockIdx.z, n = blockIdx.y;
   const int j = blockIdx.x * blockDim.x + threadIdx.x;
   if (j >= a.d_out[l] || (a.active != nullptr && a.active[n] == 0) || a.status->error != 0u) return;
@@ -688,6 +740,39 @@ __global__ void __launch_bounds__(128) bias_update_kernel(const BiasArgs a) {
     *vp = g;
   }
   *bp = fmaf(-a.gamma, g, *bp);
+}
+
+// Node average of every layer's bias segment in one launch (averaging iteration of the fused form):
+// grid (ceil(max d_l / 128), L), one thread per bias entry, the same arithmetic as average_rows_kernel
+// (fp32 sum in worker order, one division), so the bits equal update-then-average.
+struct BiasAverageArgs {
+  float* params;
+  int64_t m_pad;
+  int N;
+  int64_t b_off[PRSGD_MAX_LAYERS];
+  int d_out[PRSGD_MAX_LAYERS];
+  const DeviceStatus* status;
+};
+
+__global__ void __launch_bounds__(128) bias_average_kernel(const BiasAverageArgs a) {
+  ptx::pdl_wait();
+  ptx::pdl_trigger();     // after the wait: a later launch's early loads overlap this launch only
+  const int l = blockIdx.y;
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= a.d_out[l] || a.status->error != 0u) return;
+  float* p = a.params + a.b_off[l] + j;
+  float s = 0.f;
+  int i = 0;
+  for (; i + 8 <= a.N; i += 8) {
+    float v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) v[u] = p[(int64_t)(i + u) * a.m_pad];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) s += v[u];
+  }
+  for (; i < a.N; ++i) s += p[(int64_t)i * a.m_pad];
+  const float y = __fdiv_rn(s, (float)a.N);
+  for (int r = 0; r < a.N; ++r) p[(int64_t)r * a.m_pad] = y;
 }
 
 // Self-test of the failure path: waits on an mbarrier that nothing ever arrives on, with a short
@@ -792,6 +877,7 @@ inline void tc_launch_forward(prsgd_ctx* c, int l, const DrawArgs& dr, const uin
   a.out_bk = c->buf.act_bk[l]; a.out_f32 = c->buf.act_f32[l];
   a.bias = c->params + ly.b_off; a.bias_stride = c->m_pad;
   a.active = active; a.status = c->status;
+  a.prefetch = (l > 1 && active == nullptr && c->early_loads) ? 1 : 0;   // W_1 was written by the launch just before
   const bool softmax = l == c->L && tc_epilogues_fused(c);
   if (softmax) {        // the softmax-CE gradient, the loss and the step of b_L happen in this launch's epilogue
     a.softmax = 1; a.stages = stream_stages(c->B, true);
@@ -819,6 +905,7 @@ inline void tc_launch_dx(prsgd_ctx* c, int l, const DrawArgs& dr, const uint8_t*
   a.pool = 0; a.draw = dr; a.ld_out = c->buf.ld[l - 1];
   a.out_bk = c->buf.delta_bk[l - 1]; a.mask_src = c->buf.act_bk[l - 1];
   a.active = active; a.status = c->status;
+  a.prefetch = (active == nullptr && c->early_loads) ? 1 : 0;
   if (tc_epilogues_fused(c)) {      // the step of b_{l-1} rides on the epilogue that forms dZ_{l-1}
     a.bias_rw = c->params + c->layer[l - 2].b_off; a.bias_stride = c->m_pad; a.gamma = c->gamma; a.mu = c->mu;
     a.bias_vel = c->velocity != nullptr ? c->velocity + c->layer[l - 2].b_off : nullptr;
@@ -836,6 +923,7 @@ inline void tc_launch_update_tn(prsgd_ctx* c, int l, const DrawArgs& dr, const u
   UpdateArgs a{};
   a.B = c->B; a.N = c->N; a.tiles_m = (ly.d_out + 127) / 128; a.tiles_n = (ly.d_in + TN - 1) / TN;
   a.gamma = c->gamma; a.mu = c->mu; a.pool = l == 1; a.draw = dr; a.active = active; a.status = c->status;
+  a.prefetch = (active == nullptr && c->early_loads) ? 1 : 0;
   const int items = a.tiles_m * a.tiles_n * (fuse ? 1 : c->N);
   const int grid = items < st->num_sms ? items : st->num_sms;
   const TcLayerMaps& mp = st->layer[l - 1];
@@ -887,12 +975,32 @@ inline void tc_launch_bias(prsgd_ctx* c, const uint8_t* active) {
   launch_pdl(bias_update_kernel, dim3((dmax + 127) / 128, c->N, c->L), dim3(128), 0, c->stream, a);
 }
 
-inline void tc_launch_bias_average(prsgd_ctx* c, int l) {
+// A layer with few tiles gives the fused update + average too few CTAs (each walks all N workers of
+// its tile), so such a layer takes the plain update followed by the node average of its weight segment.
+inline bool tc_layer_fuses_average(const prsgd_ctx* c, int l) {
+  const TcState* st = static_cast<const TcState*>(c->tc);
   const Layer& ly = c->layer[l - 1];
-  const int64_t threads = ly.d_out / 4 + (ly.d_out & 3);
-  launch_pdl(average_rows_kernel<0, false>, dim3((unsigned)((threads + 255) / 256)), dim3(256), 0, c->stream,
-             c->params + ly.b_off, (int64_t)c->N, (int64_t)ly.d_out, c->m_pad, (float*)nullptr, (uint16_t*)nullptr,
+  const int64_t tiles64 = (int64_t)((ly.d_out + 127) / 128) * ((ly.d_in + 63) / 64);
+  return 2 * tiles64 >= (int64_t)st->num_sms;
+}
+
+inline void tc_launch_weight_average(prsgd_ctx* c, int l) {
+  const Layer& ly = c->layer[l - 1];
+  const int64_t cols = (int64_t)ly.d_out * ly.d_in;          // a multiple of 64, like every input width of this path
+  launch_pdl(average_rows_kernel<0, true, 2>, dim3((unsigned)((cols / 2 + (cols & 1) + 255) / 256)), dim3(256), 0, c->stream,
+             c->params + ly.w_off, (int64_t)c->N, cols, c->m_pad, (float*)nullptr, c->shadow + ly.w_off,
              (const DeviceStatus*)c->status);
+}
+
+inline void tc_launch_bias_average(prsgd_ctx* c) {
+  BiasAverageArgs a{};
+  a.params = c->params; a.m_pad = c->m_pad; a.N = c->N; a.status = c->status;
+  int dmax = 1;
+  for (int l = 1; l <= c->L; ++l) {
+    a.b_off[l - 1] = c->layer[l - 1].b_off; a.d_out[l - 1] = c->layer[l - 1].d_out;
+    if (a.d_out[l - 1] > dmax) dmax = a.d_out[l - 1];
+  }
+  launch_pdl(bias_average_kernel, dim3((dmax + 127) / 128, c->L), dim3(128), 0, c->stream, a);
 }
 
 }  // namespace prsgd

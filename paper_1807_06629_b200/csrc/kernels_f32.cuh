@@ -267,8 +267,8 @@ __device__ __forceinline__ uint16_t f32_to_bf16_rn(float f) {
 }
 
 __global__ void __launch_bounds__(256) softmax_ce_kernel(const SoftmaxArgs a) {
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");   // no-op unless launched as a programmatic dependent
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // after the wait: see tc_stream_kernel
   const int n = blockIdx.x;
   if (a.active != nullptr && a.active[n] == 0) return;
   if (a.status != nullptr && a.status->error != 0u) return;

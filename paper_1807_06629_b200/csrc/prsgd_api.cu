@@ -308,9 +308,15 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging) {
       tc_launch_dx(c, l, dr, act_mask);
       LAUNCH_CHECK(c);
     }
-    prof_begin(c, fuse ? PRSGD_KERNEL_UPDATE_AVERAGE : PRSGD_KERNEL_UPDATE);
-    tc_launch_update(c, l, dr, act_mask, fuse);
+    const bool fuse_l = fuse && tc_layer_fuses_average(c, l);
+    prof_begin(c, fuse_l ? PRSGD_KERNEL_UPDATE_AVERAGE : PRSGD_KERNEL_UPDATE);
+    tc_launch_update(c, l, dr, act_mask, fuse_l);
     LAUNCH_CHECK(c);
+    if (fuse && !fuse_l) {
+      prof_begin(c, PRSGD_KERNEL_AVERAGE);
+      tc_launch_weight_average(c, l);
+      LAUNCH_CHECK(c);
+    }
   }
   if (!epi) {
     prof_begin(c, PRSGD_KERNEL_MISC);
@@ -318,11 +324,9 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging) {
     LAUNCH_CHECK(c);
   }
   if (fuse) {
-    for (int l = 1; l <= L; ++l) {
-      prof_begin(c, PRSGD_KERNEL_MISC);
-      tc_launch_bias_average(c, l);
-      LAUNCH_CHECK(c);
-    }
+    prof_begin(c, PRSGD_KERNEL_MISC);
+    tc_launch_bias_average(c);
+    LAUNCH_CHECK(c);
   }
   return PRSGD_OK;
 }
@@ -579,7 +583,7 @@ void period_key(const prsgd_ctx* c, uint64_t (&key)[12]) {
   key[0] = gbits; key[1] = (uint64_t)c->I; key[2] = (uint64_t)c->fused_average; key[3] = (uint64_t)c->upd_tile;
   key[4] = c->has_mask ? 1 : 0; key[5] = reinterpret_cast<uint64_t>(c->velocity); key[6] = mbits;
   key[7] = (uint64_t)c->average_velocity; key[8] = reinterpret_cast<uint64_t>(c->X);
-  key[9] = reinterpret_cast<uint64_t>(c->Y); key[10] = (uint64_t)c->worker0; key[11] = (uint64_t)c->fused_epilogues;
+  key[9] = reinterpret_cast<uint64_t>(c->Y); key[10] = (uint64_t)c->worker0; key[11] = (uint64_t)c->fused_epilogues | ((uint64_t)c->early_loads << 1);
 }
 
 // One whole averaging period (I iterations starting right after an average) as a CUDA graph: the
@@ -882,6 +886,7 @@ int prsgd_set_option(prsgd_ctx* c, int32_t option, int64_t value) {
   if (option == PRSGD_OPT_PROFILE) { c->profile = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_GRAPH) { c->use_graph = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_FUSED_EPILOGUES) { c->fused_epilogues = value != 0; return PRSGD_OK; }
+  if (option == PRSGD_OPT_EARLY_LOADS) { c->early_loads = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_UPDATE_TILE) {
     if (value != 0 && value != 64 && value != 128) return fail(c, PRSGD_ERR_ARG, "update tile width must be 0, 64 or 128");
     c->upd_tile = (int)value;

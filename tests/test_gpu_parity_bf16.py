@@ -127,6 +127,26 @@ def test_fused_average_equals_update_then_average_bit_for_bit(torch_cuda):
             assert np.array_equal(outs[0], o)
 
 
+def test_early_weight_loads_change_no_bit(torch_cuda):
+    """Tiles requested ahead of a kernel's dependency wait (weights nobody is writing at that time) against
+    the same run with every load after the wait: identical bits over several periods, direct and replayed."""
+    torch = torch_cuda
+    from paper_1807_06629_b200 import binding
+    for w in (SMALL[1], SMALL[4], SMALL[6], _w("tc-n5", 5, (64, 128, 10), 32, I=3)):
+        X, Y, x0 = make_inputs(w)
+        outs = []
+        for early, graph in ((1, 0), (0, 0), (1, 1), (0, 1)):
+            with torch.cuda.stream(torch.cuda.Stream()):
+                p = make_ctx(w, X, Y, x0)
+                p.set_option(binding.OPT_EARLY_LOADS, early)
+                p.set_option(binding.OPT_GRAPH, graph)
+                p.local_steps(3 * w.I + 1)
+                outs.append((p.get_params_stacked(), p.get_losses()))
+                torch.cuda.current_stream().synchronize()
+        for o in outs[1:]:
+            assert np.array_equal(outs[0][0], o[0]) and np.array_equal(outs[0][1], o[1])
+
+
 def _segments(dims):
     """[(is_weight, start, stop)] of a canonical parameter vector."""
     out, off = [], 0
