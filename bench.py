@@ -107,8 +107,8 @@ class ClockSampler:
 # dram__bytes_read.sum + dram__bytes_write.sum per iteration of one kernel family, from the one-pass ncu
 # capture summarised in profiles/; valid only while the kernel's source section is unchanged.
 NCU_TRAFFIC = {
-    ("cfg4", "update"): {"bytes_per_iteration": 2.22e9 + 3.04e9, "launches_per_iteration": 4,   # read + written, four launches
-                         "kernel_sha256": "8c0c30587d29142b1db957df042caf0716f231947833abf2cb8d4da688528bcf"},
+    ("cfg4", "update"): {"bytes_per_iteration": 2.229e9 + 3.035e9, "launches_per_iteration": 4,   # read + written, four launches
+                         "kernel_sha256": "20c3a8a2a487e4f915bc302e408ff116e624e98895c886832c53b20c2bbc6d68"},
 }
 
 
