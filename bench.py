@@ -278,6 +278,8 @@ def main():
                     help="averaging iterations run as update + stand-alone averaging kernel instead of the fused pass")
     ap.add_argument("--no-fused-epilogues", action="store_true",
                     help="softmax-CE gradient and bias steps as kernels of their own instead of GEMM epilogues")
+    ap.add_argument("--no-next-forward", action="store_true",
+                    help="layer 1's update does not form the next iteration's a_1")
     ap.add_argument("--no-early-loads", action="store_true",
                     help="no tile requests ahead of a kernel's dependency wait")
     ap.add_argument("--force-sharded", action="store_true",
@@ -352,6 +354,8 @@ def main():
         p.enable_momentum(args.momentum)
     if args.no_fuse:
         p.set_option(binding.OPT_FUSED_AVERAGE, 0)
+    if args.no_next_forward:
+        p.set_option(binding.OPT_NEXT_FORWARD, 0)
     if args.no_early_loads:
         p.set_option(binding.OPT_EARLY_LOADS, 0)
     if args.no_fused_epilogues:

@@ -256,6 +256,13 @@ int prsgd_get_velocity_stacked(prsgd_ctx* ctx, float* dst, int dst_on_device);
  * writing them (every layer's forward GEMM but the first, every dX GEMM, the master tiles of every
  * update; never while a worker mask is set).  Same bits either way. */
 #define PRSGD_OPT_EARLY_LOADS 6
+/* PRSGD_OPT_NEXT_FORWARD (default 1, tensor-core path, more than one layer): on a plain SGD iteration
+ * that is not an averaging one and is followed by another iteration of the same prsgd_local_steps call,
+ * the update of layer 1 also multiplies each freshly stepped tile of W_1 with the next minibatch, so that
+ * the next iteration starts with a_1 in place: its first forward launch is skipped and the bf16 copy of
+ * W_1, which only that launch reads, is not written on such iterations (it is valid whenever a call
+ * returns).  Same bits as the separate launches. */
+#define PRSGD_OPT_NEXT_FORWARD 7
 int prsgd_set_option(prsgd_ctx* ctx, int32_t option, int64_t value);
 
 /* Kernel families of the hot path, for prsgd_get_profile. */

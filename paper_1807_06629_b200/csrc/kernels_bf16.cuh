@@ -701,6 +701,291 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
   if (warp == 1) tmem_dealloc(tmem, 256u);
 }
 
+// ---------------------------------------------------------------------------------------------
+// update of layer 1 with the next iteration's first forward GEMM folded in
+// ---------------------------------------------------------------------------------------------
+// The first layer's input is the data pool, so once a tile of W_1 has taken its step the product of
+// that tile with the NEXT minibatch can be formed straight from the bf16 tile the epilogue has just
+// written to shared memory.  A CTA therefore owns whole row blocks (128 output features of one
+// worker), walks their column tiles left to right, accumulates z_1 = W_1 x' over them in a second
+// TMEM accumulator and finishes the row block with the forward epilogue (bias, ReLU, bf16 a_1).
+// The forward launch of layer 1 in the next iteration is then skipped, and W_1's bf16 shadow, which
+// only that launch reads, need not be written (the host asks for it on the last iteration of a call
+// so that the shadow is valid whenever control returns to the caller).
+struct UpdateNextArgs {
+  int B, N;
+  int tiles_m, tiles_n;
+  float gamma;
+  DrawArgs draw;             // iteration t; the next minibatch is the draw of t + 1
+  DeviceStatus* status;
+  int stages;
+  int write_shadow;
+  uint16_t* next_out;        // bf16 a_1 [N][B][next_ld]
+  int next_ld;
+  const float* bias;         // params + b_off of layer 1 (already stepped by this iteration's dX epilogue)
+  int64_t bias_stride;
+  int M_total;               // d_1
+};
+
+template <int TN> struct UpdNextCfg {
+  static constexpr uint32_t kMaster = 128u * TN * 4u;
+  static constexpr uint32_t kOut = 128u * TN * 2u;
+  __host__ __device__ static uint32_t ops_bytes(int B) { return (uint32_t)(2 + TN / 64) * (uint32_t)B * 128u; }
+  __host__ __device__ static uint32_t region(int B) { return ops_bytes(B) > kOut ? ops_bytes(B) : kOut; }
+  __host__ __device__ static uint32_t next_bytes(int B) { return (uint32_t)(TN / 64) * (uint32_t)B * 128u; }
+  __host__ __device__ static uint32_t stage(int B) { return kMaster + region(B) + next_bytes(B); }
+  static int stages(int B) {
+    int s = (int)((227u * 1024u - 2048u) / stage(B));
+    return s > 4 ? 4 : s;
+  }
+  static size_t smem(int B) { return (size_t)stages(B) * stage(B) + 1024 + 512; }
+};
+
+template <int TN>
+__global__ void __launch_bounds__(kUpdThreads, 1) tc_update_next_kernel(const __grid_constant__ CUtensorMap mapDelta,
+                                                                        const __grid_constant__ CUtensorMap mapPool,
+                                                                        const __grid_constant__ CUtensorMap mapMaster,
+                                                                        const __grid_constant__ CUtensorMap mapShadow,
+                                                                        const UpdateNextArgs a) {
+  using namespace ptx;
+  using Cfg = UpdNextCfg<TN>;
+  constexpr int NB32 = TN / 32, NB64 = TN / 64;
+  constexpr uint32_t kFwdCol = 256u;                    // TMEM: dW accumulators in columns [0, 256), forward ones behind
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* gen = smem_raw + (base - raw);
+  const int S = a.stages;
+  const uint32_t stage_bytes = Cfg::stage(a.B);
+  const uint32_t op_box = (uint32_t)a.B * 128u;         // one {64, B} box
+  auto master_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes; };
+  auto ops_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes + Cfg::kMaster; };
+  auto next_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes + Cfg::kMaster + Cfg::region(a.B); };
+  const uint32_t bar0 = base + (uint32_t)S * stage_bytes;
+  auto full_ops = [&](int s) { return bar0 + 8u * s; };
+  auto full_w = [&](int s) { return bar0 + 32u + 8u * s; };
+  auto stage_empty = [&](int s) { return bar0 + 64u + 8u * s; };
+  auto acc_full = [&](int s) { return bar0 + 96u + 8u * s; };
+  auto acc_empty = [&](int s) { return bar0 + 128u + 8u * s; };
+  auto tile_ready = [&](int s) { return bar0 + 160u + 8u * s; };
+  auto fwd_done = [&](int s) { return bar0 + 192u + 8u * s; };      // forward MMAs have read the stage's bf16 tile
+  auto facc_full = [&](int q) { return bar0 + 224u + 8u * q; };
+  auto facc_empty = [&](int q) { return bar0 + 240u + 8u * q; };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen + (size_t)S * stage_bytes + 256);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + (size_t)S * stage_bytes + 260);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int row_blocks = a.tiles_m * a.N;
+
+  if (tid == 0) {
+    for (int s = 0; s < S; ++s) {
+      mbar_init(full_ops(s), 1); mbar_init(full_w(s), 1); mbar_init(stage_empty(s), 1);
+      mbar_init(acc_full(s), 1); mbar_init(acc_empty(s), 128); mbar_init(tile_ready(s), 128);
+      mbar_init(fwd_done(s), 1);
+    }
+    for (int q = 0; q < 2; ++q) { mbar_init(facc_full(q), 1); mbar_init(facc_empty(q), 128); }
+    *abort_flag = 0;
+    fence_mbar_init();
+    prefetch_tensormap(&mapDelta); prefetch_tensormap(&mapPool);
+    prefetch_tensormap(&mapMaster); prefetch_tensormap(&mapShadow);
+  }
+  if (warp == 1) { tmem_alloc(smem_u32(tmem_slot), 512u); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  pdl_wait();
+  pdl_trigger();
+  const uint32_t tmem = *tmem_slot;
+  if (tid == 0) *abort_flag = *(volatile unsigned int*)&a.status->error != 0u ? 1 : 0;   // an earlier expired wait: no-op
+  __syncthreads();
+  const int total_rb = *abort_flag != 0 ? 0 : row_blocks;
+
+  // Every role walks the same sequence of tiles: row blocks rb = blockIdx.x, + gridDim.x, ..., and inside a
+  // row block the column tiles kb = 0 .. tiles_n - 1; `it` counts tiles, tile `it` lives in stage it % S.
+  if (warp == 0 && lane == 0) {
+    // ---------------- loader
+    uint32_t it = 0;
+    bool ok = true;
+    for (int rb = blockIdx.x; rb < total_rb && ok; rb += gridDim.x) {
+      const int n = rb / a.tiles_m, m0 = (rb % a.tiles_m) * 128;
+      const int64_t t = draw_t(a.draw);
+      const int row0 = (int)draw_block(a.draw.seed, a.draw.worker0 + n, t, a.draw.n_blocks) * a.B;
+      const int row1 = (int)draw_block(a.draw.seed, a.draw.worker0 + n, t + 1, a.draw.n_blocks) * a.B;
+      for (int kb = 0; kb < a.tiles_n; ++kb, ++it) {
+        const int s = it % S;
+        const uint32_t ph = (it / S) & 1u;
+        ok = mbar_wait(stage_empty(s), ph ^ 1u, abort_flag, a.status, 0x401);
+        if (!ok) break;
+        const int n0 = kb * TN;
+        const uint32_t ops = ops_u32(s), nx = next_u32(s);
+        mbar_expect_tx(full_ops(s), (2u + 2u * NB64) * op_box);
+        tma_load_3d(ops, &mapDelta, full_ops(s), m0, 0, n);
+        tma_load_3d(ops + op_box, &mapDelta, full_ops(s), m0 + 64, 0, n);
+#pragma unroll
+        for (int h = 0; h < NB64; ++h) {
+          tma_load_3d(ops + (2u + h) * op_box, &mapPool, full_ops(s), n0 + 64 * h, row0, n);
+          tma_load_3d(nx + h * op_box, &mapPool, full_ops(s), n0 + 64 * h, row1, n);
+        }
+        mbar_expect_tx(full_w(s), Cfg::kMaster);
+#pragma unroll
+        for (int q = 0; q < NB32; ++q) tma_load_3d(master_u32(s) + q * 16384u, &mapMaster, full_w(s), n0 + 32 * q, m0, n);
+      }
+    }
+    if (*abort_flag && it > 0) {   // let the copies already in flight land before the CTA goes away
+      const uint32_t first = it > (uint32_t)S ? it - (uint32_t)S : 0u;
+      for (uint32_t q = first; q < it; ++q) {
+        const uint64_t t0 = globaltimer_ns();
+        while (!(mbar_try_wait(full_w(q % S), (q / S) & 1u) && mbar_try_wait(full_ops(q % S), (q / S) & 1u)) &&
+               globaltimer_ns() - t0 < 100000000ull) {}
+      }
+    }
+  } else if (warp == 1 && lane == 0) {
+    // ---------------- MMA issuer: dW of tile `it`, then the forward product of tile it - 1 (whose
+    // stepped bf16 tile the epilogue has finished meanwhile)
+    const uint32_t idesc_dw = idesc_bf16(128, TN, 1, 1);
+    const uint32_t idesc_fw = idesc_bf16(128, a.B, 0, 0);
+    const int ksteps = a.B / 16;
+    uint32_t it = 0, rbi = 0;
+    bool ok = true;
+    bool have_prev = false;
+    uint32_t p_it = 0, p_rbi = 0;
+    int p_kb = 0;
+    auto forward_of = [&](uint32_t j, int kb, uint32_t rj) -> bool {
+      const int s = j % S, q = rj & 1;
+      if (kb == 0 && !mbar_wait(facc_empty(q), ((rj >> 1) & 1u) ^ 1u, abort_flag, a.status, 0x402)) return false;
+      if (!mbar_wait(tile_ready(s), (j / S) & 1u, abort_flag, a.status, 0x403)) return false;
+      tc_fence_after();
+      const uint32_t acc = tmem + kFwdCol + (uint32_t)(q * a.B);
+#pragma unroll
+      for (int h = 0; h < NB64; ++h) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          mma_bf16(acc, smem_desc_sw128(ops_u32(s) + h * 16384u + k * 32u, 16u, 1024u),
+                   smem_desc_sw128(next_u32(s) + h * op_box + k * 32u, 16u, 1024u), idesc_fw, (kb | h | k) != 0 ? 1u : 0u);
+      }
+      mma_commit(fwd_done(s));
+      if (kb == a.tiles_n - 1) mma_commit(facc_full(q));
+      return true;
+    };
+    for (int rb = blockIdx.x; rb < total_rb && ok; rb += gridDim.x, ++rbi) {
+      for (int kb = 0; kb < a.tiles_n && ok; ++kb, ++it) {
+        const int s = it % S;
+        const uint32_t ph = (it / S) & 1u;
+        ok = mbar_wait(acc_empty(s), ph ^ 1u, abort_flag, a.status, 0x404) &&
+             mbar_wait(full_ops(s), ph, abort_flag, a.status, 0x405);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t sa = ops_u32(s), sb = sa + 2u * op_box;
+        for (int k = 0; k < ksteps; ++k)
+          mma_bf16(tmem + (uint32_t)(s * TN), smem_desc_sw128(sa + k * 2048u, op_box, 1024u),
+                   smem_desc_sw128(sb + k * 2048u, op_box, 1024u), idesc_dw, k != 0 ? 1u : 0u);
+        mma_commit(acc_full(s));
+        if (have_prev) ok = forward_of(p_it, p_kb, p_rbi);
+        p_it = it; p_kb = kb; p_rbi = rbi; have_prev = true;
+      }
+    }
+    if (ok && have_prev) forward_of(p_it, p_kb, p_rbi);
+  } else if (warp == 2 && lane == 0) {
+    // ---------------- storer: TMA stores of finished tiles; the stage goes back to the loader once the
+    // forward MMAs have consumed its bf16 tile too
+    uint32_t it = 0;
+    bool ok = true;
+    for (int rb = blockIdx.x; rb < total_rb && ok; rb += gridDim.x) {
+      const int n = rb / a.tiles_m, m0 = (rb % a.tiles_m) * 128;
+      for (int kb = 0; kb < a.tiles_n; ++kb, ++it) {
+        const int s = it % S;
+        const uint32_t ph = (it / S) & 1u;
+        const int n0 = kb * TN;
+        ok = mbar_wait(tile_ready(s), ph, abort_flag, a.status, 0x406);
+        if (!ok) break;
+#pragma unroll
+        for (int q = 0; q < NB32; ++q) tma_store_3d(&mapMaster, master_u32(s) + q * 16384u, n0 + 32 * q, m0, n);
+        if (a.write_shadow) {
+#pragma unroll
+          for (int h = 0; h < NB64; ++h) tma_store_3d(&mapShadow, ops_u32(s) + h * 16384u, n0 + 64 * h, m0, n);
+        }
+        tma_commit_group();
+        tma_wait_group_read0();
+        ok = mbar_wait(fwd_done(s), ph, abort_flag, a.status, 0x407);
+        if (!ok) break;
+        mbar_arrive(stage_empty(s));
+      }
+    }
+    tma_wait_group0();
+  } else if (warp >= 3) {
+    // ---------------- epilogue: row r of the tile <-> TMEM lane r
+    const int q4 = warp & 3;
+    const int r = q4 * 32 + lane;
+    const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
+    const uint32_t row_off = (uint32_t)r * 128u;
+    const uint32_t sw = (uint32_t)(r & 7);
+    const int batches = a.B / 16;
+    uint32_t it = 0, rbi = 0;
+    bool ok = true;
+    for (int rb = blockIdx.x; rb < total_rb && ok; rb += gridDim.x, ++rbi) {
+      const int n = rb / a.tiles_m, m = (rb % a.tiles_m) * 128 + r;
+      for (int kb = 0; kb < a.tiles_n; ++kb, ++it) {
+        const int s = it % S;
+        const uint32_t ph = (it / S) & 1u;
+        ok = mbar_wait(full_w(s), ph, abort_flag, a.status, 0x408) &&
+             mbar_wait(acc_full(s), ph, abort_flag, a.status, 0x409);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        uint8_t* mst = gen + (size_t)s * stage_bytes;
+        uint8_t* stg = mst + Cfg::kMaster;
+#pragma unroll
+        for (int c = 0; c < NB32; ++c) {
+          uint32_t v[32];
+          tmem_ld32(tmem + lane_off + (uint32_t)(s * TN + c * 32), v);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            float4* pw = reinterpret_cast<float4*>(mst + c * 16384 + row_off + (((uint32_t)j ^ sw) << 4));
+            float4 x = *pw;
+            x.x = fmaf(-a.gamma, __uint_as_float(v[4 * j + 0]), x.x);
+            x.y = fmaf(-a.gamma, __uint_as_float(v[4 * j + 1]), x.y);
+            x.z = fmaf(-a.gamma, __uint_as_float(v[4 * j + 2]), x.z);
+            x.w = fmaf(-a.gamma, __uint_as_float(v[4 * j + 3]), x.w);
+            *pw = x;
+            const uint32_t chunk = (uint32_t)((c & 1) * 4 + (j >> 1));
+            uint2* pb = reinterpret_cast<uint2*>(stg + (c >> 1) * 16384 + row_off + ((chunk ^ sw) << 4) + (j & 1) * 8);
+            *pb = make_uint2(pack_bf16x2(x.x, x.y), pack_bf16x2(x.z, x.w));
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(acc_empty(s));
+        fence_proxy_async();
+        mbar_arrive(tile_ready(s));
+      }
+      if (!ok) break;
+      // forward epilogue of the row block: a_1[., m] = relu(z + b_1[m]) for the next iteration
+      const int q = rbi & 1;
+      const bool valid = m < a.M_total;
+      const float bias = valid ? a.bias[(int64_t)n * a.bias_stride + m] : 0.f;
+      ok = __all_sync(0xffffffffu, mbar_wait(facc_full(q), (rbi >> 1) & 1u, abort_flag, a.status, 0x40A));
+      if (!ok) break;
+      tc_fence_after();
+      for (int bi = 0; bi < batches; ++bi) {
+        uint32_t v[16];
+        tmem_ld16(tmem + lane_off + kFwdCol + (uint32_t)(q * a.B + bi * 16), v);
+        tmem_ld_wait();
+        if (valid) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            a.next_out[((int64_t)n * a.B + bi * 16 + j) * a.next_ld + m] = f32_to_bf16_rn(fmaxf(__uint_as_float(v[j]) + bias, 0.f));
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(facc_empty(q));
+    }
+  }
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem, 512u);
+}
+
 // b_l <- b_l - gamma * sum_b dZ_l[b, :] (the bias part of Eq. parallel-sgd-x-update) for every layer in
 // one launch: grid (ceil(max d_l / 128), N, L), one thread per (layer, worker, j).
 struct BiasArgs {
@@ -827,6 +1112,8 @@ inline int tc_create(prsgd_ctx* c, std::string* err) {
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<false, 128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<128, false>::smem(c->B));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<true, 128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<128, false>::smem(c->B));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<false, 64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<64, true>::smem(c->B));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_next_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdNextCfg<64>::smem(c->B));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_next_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdNextCfg<128>::smem(c->B));
   if (e != cudaSuccess) {
     *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e);
     delete st;
@@ -936,6 +1223,36 @@ inline void tc_launch_update_tn(prsgd_ctx* c, int l, const DrawArgs& dr, const u
     else
       launch_pdl(tc_update_kernel<false, TN, false>, dim3(grid), kUpdThreads, smem, c->stream, mp.delta_out, mp.act_in, mp.master, mp.shadow_k, mp.master, a);
   }
+}
+
+// Update of layer 1 that also forms a_1 of the next iteration (tc_update_next_kernel).
+template <int TN>
+inline void tc_launch_update_next_tn(prsgd_ctx* c, const DrawArgs& dr, bool write_shadow) {
+  TcState* st = static_cast<TcState*>(c->tc);
+  const Layer& ly = c->layer[0];
+  UpdateNextArgs a{};
+  a.B = c->B; a.N = c->N; a.tiles_m = (ly.d_out + 127) / 128; a.tiles_n = (ly.d_in + TN - 1) / TN;
+  a.gamma = c->gamma; a.draw = dr; a.status = c->status;
+  a.stages = UpdNextCfg<TN>::stages(c->B); a.write_shadow = write_shadow ? 1 : 0;
+  a.next_out = c->buf.act_bk[1]; a.next_ld = c->buf.ld[1];
+  a.bias = c->params + ly.b_off; a.bias_stride = c->m_pad; a.M_total = ly.d_out;
+  const int items = a.tiles_m * c->N;
+  const int grid = items < st->num_sms ? items : st->num_sms;
+  const TcLayerMaps& mp = st->layer[0];
+  launch_pdl(tc_update_next_kernel<TN>, dim3(grid), kUpdThreads, UpdNextCfg<TN>::smem(c->B), c->stream, mp.delta_out, mp.act_in,
+             mp.master, mp.shadow_k, a);
+}
+
+inline void tc_launch_update_next(prsgd_ctx* c, const DrawArgs& dr, bool write_shadow) {
+  const TcState* st = static_cast<const TcState*>(c->tc);
+  const Layer& ly = c->layer[0];
+  int tile = c->upd_tile;
+  if (tile == 0) {
+    const int64_t tiles128 = (int64_t)((ly.d_out + 127) / 128) * ((ly.d_in + 127) / 128);
+    tile = (c->B <= 32 && tiles128 * c->N >= 32 * (int64_t)st->num_sms) ? 128 : 64;
+  }
+  if (tile == 128) tc_launch_update_next_tn<128>(c, dr, write_shadow);
+  else tc_launch_update_next_tn<64>(c, dr, write_shadow);
 }
 
 // Tile width: forced by PRSGD_OPT_UPDATE_TILE, else chosen per launch.  Wide tiles need fewer TMA

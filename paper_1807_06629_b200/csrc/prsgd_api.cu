@@ -281,12 +281,20 @@ int step_f32(prsgd_ctx* c, int64_t t, bool averaging) {
 }
 
 // One iteration of Algorithm 1 on the bf16-operand tensor-core path.
-int step_bf16(prsgd_ctx* c, int64_t t, bool averaging) {
+// `more_follow`: the caller runs iteration t + 1 right after this one (same call, nothing in between).
+int step_bf16(prsgd_ctx* c, int64_t t, bool averaging, bool more_follow) {
   const int L = c->L, N = c->N;
   const uint8_t* act_mask = c->has_mask ? c->active : nullptr;
   const bool fuse = averaging && c->fused_average && c->velocity == nullptr;   // the momentum step is not fused
   const DrawArgs dr = draw_args(c, t);
-  for (int l = 1; l <= L; ++l) {
+  // Layer 1's update can form a_1 of iteration t + 1 as well (its input is the data pool), which saves that
+  // iteration's first forward launch and the write of W_1's shadow: only on a plain SGD iteration that is
+  // not an averaging one and is followed by another one of the same call.
+  const bool next_fwd = c->next_forward && more_follow && !averaging && L > 1 && act_mask == nullptr &&
+                        c->velocity == nullptr && tc_epilogues_fused(c);
+  const bool skip_f1 = c->a1_ready;
+  c->a1_ready = false;
+  for (int l = skip_f1 ? 2 : 1; l <= L; ++l) {
     prof_begin(c, PRSGD_KERNEL_FORWARD);
     tc_launch_forward(c, l, dr, act_mask);
     LAUNCH_CHECK(c);
@@ -310,7 +318,12 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging) {
     }
     const bool fuse_l = fuse && tc_layer_fuses_average(c, l);
     prof_begin(c, fuse_l ? PRSGD_KERNEL_UPDATE_AVERAGE : PRSGD_KERNEL_UPDATE);
-    tc_launch_update(c, l, dr, act_mask, fuse_l);
+    if (l == 1 && next_fwd) {
+      tc_launch_update_next(c, dr, false);
+      c->a1_ready = true;
+    } else {
+      tc_launch_update(c, l, dr, act_mask, fuse_l);
+    }
     LAUNCH_CHECK(c);
     if (fuse && !fuse_l) {
       prof_begin(c, PRSGD_KERNEL_AVERAGE);
@@ -566,7 +579,8 @@ namespace {
 int run_iterations(prsgd_ctx* c, int64_t t_first, int64_t count) {
   for (int64_t t = t_first; t < t_first + count; ++t) {
     const bool averaging = c->I > 0 && (t % c->I) == 0;
-    int rc = c->precision == PRSGD_PRECISION_BF16 ? step_bf16(c, t, averaging) : step_f32(c, t, averaging);
+    const bool more_follow = t + 1 < t_first + count;
+    int rc = c->precision == PRSGD_PRECISION_BF16 ? step_bf16(c, t, averaging, more_follow) : step_f32(c, t, averaging);
     if (rc != PRSGD_OK) return rc;
     if (averaging && (!c->fused_average || c->velocity != nullptr)) {
       rc = launch_average(c);
@@ -583,7 +597,7 @@ void period_key(const prsgd_ctx* c, uint64_t (&key)[12]) {
   key[0] = gbits; key[1] = (uint64_t)c->I; key[2] = (uint64_t)c->fused_average; key[3] = (uint64_t)c->upd_tile;
   key[4] = c->has_mask ? 1 : 0; key[5] = reinterpret_cast<uint64_t>(c->velocity); key[6] = mbits;
   key[7] = (uint64_t)c->average_velocity; key[8] = reinterpret_cast<uint64_t>(c->X);
-  key[9] = reinterpret_cast<uint64_t>(c->Y); key[10] = (uint64_t)c->worker0; key[11] = (uint64_t)c->fused_epilogues | ((uint64_t)c->early_loads << 1);
+  key[9] = reinterpret_cast<uint64_t>(c->Y); key[10] = (uint64_t)c->worker0; key[11] = (uint64_t)c->fused_epilogues | ((uint64_t)c->early_loads << 1) | ((uint64_t)c->next_forward << 2);
 }
 
 // One whole averaging period (I iterations starting right after an average) as a CUDA graph: the
@@ -887,6 +901,7 @@ int prsgd_set_option(prsgd_ctx* c, int32_t option, int64_t value) {
   if (option == PRSGD_OPT_GRAPH) { c->use_graph = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_FUSED_EPILOGUES) { c->fused_epilogues = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_EARLY_LOADS) { c->early_loads = value != 0; return PRSGD_OK; }
+  if (option == PRSGD_OPT_NEXT_FORWARD) { c->next_forward = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_UPDATE_TILE) {
     if (value != 0 && value != 64 && value != 128) return fail(c, PRSGD_ERR_ARG, "update tile width must be 0, 64 or 128");
     c->upd_tile = (int)value;

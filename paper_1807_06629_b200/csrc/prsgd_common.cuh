@@ -91,6 +91,8 @@ struct prsgd_ctx {
   float* velocity = nullptr;     // [N][m_pad] fp32 momentum buffers, caller-owned
   int average_velocity = 0;      // average the buffers together with the models
   int upd_tile = 0;              // column width of the update kernel's tile: 0 = chosen per launch, 64 or 128
+  int next_forward = 1;          // layer 1's update also forms a_1 of the next iteration (tensor-core path)
+  bool a1_ready = false;         // a_1 of the coming iteration has already been formed by the previous update
   int early_loads = 1;           // tensor-core kernels request tiles nobody is writing before their dependency wait
   int fused_epilogues = 1;       // softmax-CE gradient and bias steps inside the GEMM epilogues (tensor-core path)
   int64_t launches = 0;

@@ -147,6 +147,42 @@ def test_early_weight_loads_change_no_bit(torch_cuda):
             assert np.array_equal(outs[0][0], o[0]) and np.array_equal(outs[0][1], o[1])
 
 
+def test_next_forward_folded_into_the_first_layers_update_changes_no_bit(torch_cuda):
+    """The update of layer 1 also forms a_1 of the following iteration from its freshly stepped tiles (and leaves
+    W_1's bf16 copy unwritten meanwhile) against the separate forward launch: identical parameters, losses and
+    draws, direct and replayed, for both tile widths, ragged tiles and calls that end in the middle of a period;
+    the bf16 copy of every layer equals bf16(master) whenever a call has returned."""
+    torch = torch_cuda
+    from paper_1807_06629_b200 import binding
+    cases = (SMALL[1], SMALL[2], SMALL[3], SMALL[4], SMALL[5], SMALL[6], _w("tc-n5-I5", 5, (192, 128, 10), 32, I=5),
+             _w("tc-wide-in", 3, (448, 256, 10), 16, I=4))
+    for w in cases:
+        X, Y, x0 = make_inputs(w)
+        outs = []
+        for nxt, graph, tile in ((0, 0, 0), (1, 0, 0), (1, 1, 0), (1, 0, 64), (1, 1, 128)):
+            with torch.cuda.stream(torch.cuda.Stream()):
+                p = make_ctx(w, X, Y, x0)
+                p.set_option(binding.OPT_NEXT_FORWARD, nxt)
+                p.set_option(binding.OPT_GRAPH, graph)
+                p.set_option(binding.OPT_UPDATE_TILE, tile)
+                n0 = p.get_launch_count()
+                p.local_steps(2)                       # ends inside a period
+                p.local_steps(2 * w.I + 1)             # crosses two averages
+                launches = p.get_launch_count() - n0
+                p.sync()
+                store = p.params.cpu().numpy().reshape(w.N, p.m_pad)
+                shadow = p.shadow.view(torch.int16).cpu().numpy().view(np.uint16).reshape(w.N, p.m_pad)
+                for l in range(len(w.dims) - 1):
+                    a, n = p.layout.w_off[l], w.dims[l] * w.dims[l + 1]
+                    assert np.array_equal(shadow[:, a:a + n], synth.bf16_bits(store[:, a:a + n])), (w.name, l)
+                outs.append((p.get_params_stacked(), p.get_losses(), p.get_draws().tolist(), launches))
+                torch.cuda.current_stream().synchronize()
+        for o in outs[1:]:
+            assert np.array_equal(outs[0][0], o[0]), w.name
+            assert np.array_equal(outs[0][1], o[1]) and outs[0][2] == o[2]
+        assert outs[1][3] < outs[0][3]                 # forward launches were saved
+
+
 def _segments(dims):
     """[(is_weight, start, stop)] of a canonical parameter vector."""
     out, off = [], 0
