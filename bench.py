@@ -133,7 +133,7 @@ def ncu_traffic_per_launch(workload: str, family: str):
 
 
 # ----------------------------------------------------------------------------- byte model
-def algorithmic_bytes(w: synth.Workload, m_pad: int, momentum: bool = False) -> dict:
+def algorithmic_bytes(w: synth.Workload, m_pad: int, momentum: bool = False, next_forward: bool = False) -> dict:
     """Algorithmic HBM bytes of one local iteration of all N workers, per kernel family.
 
     bf16 path: forward reads the bf16 shadow (2 B/param); dX reads it again for every layer but
@@ -141,6 +141,8 @@ def algorithmic_bytes(w: synth.Workload, m_pad: int, momentum: bool = False) -> 
     activations / deltas are read and written once per use.  fp32 path: 4 B where bf16 has 2, no shadow.
     With momentum the update also reads and writes the fp32 momentum buffer (+8 B/param).
     The stand-alone average reads and writes the store once (8 B/word, +2 for the shadow).
+    next_forward: layer 1's update also forms the next a_1, so it does not write W_1's shadow (-2 B/param) but
+    reads a second minibatch and writes a_1; the forward family then has no layer-1 launch.
     """
     e = 2 if w.precision == 1 else 4
     N, B, d = w.N, w.B, w.dims
@@ -153,7 +155,11 @@ def algorithmic_bytes(w: synth.Workload, m_pad: int, momentum: bool = False) -> 
             dx += N * (wl * e + B * d[l] * e + B * d[l - 1] * 2 * e)
         upd += N * ((wl + d[l]) * (8 + (2 if w.precision == 1 else 0) + (8 if momentum else 0)) + B * (d[l] + d[l - 1]) * e)
     avg = N * m_pad * (8 + (2 if w.precision == 1 else 0))
-    return {"forward": fwd, "dx": dx, "update": upd, "update_average": upd, "average": avg,
+    upd_plain = upd
+    if next_forward:
+        upd += N * (-d[1] * d[0] * 2 + B * d[0] * e + B * d[1] * e + d[1] * 4)
+        fwd -= N * (d[1] * d[0] * e + d[1] * 4 + B * d[0] * e + B * d[1] * e)
+    return {"forward": fwd, "dx": dx, "update": upd, "update_average": upd_plain, "average": avg,
             "softmax": N * B * d[L] * (4 + 4 + e)}
 
 
@@ -405,11 +411,15 @@ def main():
         run_period()
     prof = p.get_profile()
     p.set_option(binding.OPT_PROFILE, 0)
-    bytes_iter = algorithmic_bytes(w, p.m_pad, args.momentum is not None)
+    L = len(w.dims) - 1
+    # iterations 1..I-1 of a period run layer 1's update with the next forward folded in (tensor-core path)
+    next_fwd = (w.precision == 1 and L > 1 and w.I > 1 and w.dims[L] <= 128 and args.momentum is None
+                and not args.no_next_forward and not args.no_fused_epilogues)
+    bytes_iter = algorithmic_bytes(w, p.m_pad, args.momentum is not None, next_fwd)
     fams = {k: v for k, v in prof.items() if v[1] > 0 and k in bytes_iter}
     dom = max(fams, key=lambda k: fams[k][0])
-    L = len(w.dims) - 1
-    per_iter_launches = {"forward": L, "dx": L - 1, "update": L, "update_average": L, "average": 1, "softmax": 1}[dom]
+    per_iter_launches = {"forward": L - 1 if next_fwd else L, "dx": L - 1, "update": L, "update_average": L,
+                         "average": 1, "softmax": 1}[dom]
     dom_ms, dom_launches = fams[dom]
     iters_seen = dom_launches / max(per_iter_launches, 1)
     achieved = bytes_iter[dom] * iters_seen / (dom_ms * 1e-3) / 1e9

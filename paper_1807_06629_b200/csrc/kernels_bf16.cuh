@@ -158,7 +158,10 @@ __global__ void __launch_bounds__(kStreamThreads, 1) tc_stream_kernel(const __gr
   if (tid == 0) {
     for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int q = 0; q < 2; ++q) { mbar_init(acc_full(q), 1); mbar_init(acc_empty(q), 128); }
-    *abort_flag = 0;
+    // A wait that expired in an earlier launch turns this one into a no-op.  The word is read here, off
+    // the critical path: a launch whose set-up overlapped the failing one may miss it and run (its own
+    // waits are bounded too); every launch after that sees it.
+    *abort_flag = *(volatile unsigned int*)&a.status->error != 0u ? 1 : 0;
     fence_mbar_init();
     prefetch_tensormap(&mapW);
     prefetch_tensormap(&mapB);
@@ -200,9 +203,6 @@ __global__ void __launch_bounds__(kStreamThreads, 1) tc_stream_kernel(const __gr
   pdl_wait();            // everything above overlapped the previous kernel's tail; dependent memory is touched below
   pdl_trigger();         // only now: the next launch's early loads may overlap this launch, never an older one
   const uint32_t tmem = *tmem_slot;
-  // a wait that expired in an earlier CTA or launch turns the rest of the work into a no-op
-  if (tid == 0) *abort_flag = *(volatile unsigned int*)&a.status->error != 0u ? 1 : 0;
-  __syncthreads();
   const int total_items = *abort_flag != 0 ? 0 : a.tiles_m * a.N;
   auto item_active = [&](int n) { return a.active == nullptr || a.active[n] != 0; };
 
@@ -463,7 +463,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
       mbar_init(full_ops(s), 1); mbar_init(full_w(s), 1); mbar_init(stage_empty(s), 1);
       mbar_init(acc_full(s), 1); mbar_init(acc_empty(s), 128); mbar_init(tile_ready(s), 128);
     }
-    *abort_flag = 0;
+    *abort_flag = *(volatile unsigned int*)&a.status->error != 0u ? 1 : 0;   // an earlier expired wait: no-op (see tc_stream_kernel)
     fence_mbar_init();
     prefetch_tensormap(&mapDelta); prefetch_tensormap(&mapAct);
     prefetch_tensormap(&mapMaster); prefetch_tensormap(&mapShadow);
@@ -499,8 +499,6 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
   pdl_wait();            // set-up above overlapped the previous kernel's tail; dependent memory is touched below
   pdl_trigger();         // only now: the next launch's early loads may overlap this launch, never an older one
   const uint32_t tmem = *tmem_slot;
-  if (tid == 0) *abort_flag = *(volatile unsigned int*)&a.status->error != 0u ? 1 : 0;   // an earlier expired wait: no-op
-  __syncthreads();
   const int total_items = *abort_flag != 0 ? 0 : items_all;
 
   // Every role walks the same sequence of (tile, worker) items; `it` counts the items it has handled,
@@ -784,7 +782,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_next_kernel(const __
       mbar_init(fwd_done(s), 1);
     }
     for (int q = 0; q < 2; ++q) { mbar_init(facc_full(q), 1); mbar_init(facc_empty(q), 128); }
-    *abort_flag = 0;
+    *abort_flag = *(volatile unsigned int*)&a.status->error != 0u ? 1 : 0;   // an earlier expired wait: no-op (see tc_stream_kernel)
     fence_mbar_init();
     prefetch_tensormap(&mapDelta); prefetch_tensormap(&mapPool);
     prefetch_tensormap(&mapMaster); prefetch_tensormap(&mapShadow);
@@ -796,8 +794,6 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_next_kernel(const __
   pdl_wait();
   pdl_trigger();
   const uint32_t tmem = *tmem_slot;
-  if (tid == 0) *abort_flag = *(volatile unsigned int*)&a.status->error != 0u ? 1 : 0;   // an earlier expired wait: no-op
-  __syncthreads();
   const int total_rb = *abort_flag != 0 ? 0 : row_blocks;
 
   // Every role walks the same sequence of tiles: row blocks rb = blockIdx.x, + gridDim.x, ..., and inside a
