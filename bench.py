@@ -133,7 +133,8 @@ def ncu_traffic_per_launch(workload: str, family: str):
 
 
 # ----------------------------------------------------------------------------- byte model
-def algorithmic_bytes(w: synth.Workload, m_pad: int, momentum: bool = False, next_forward: bool = False) -> dict:
+def algorithmic_bytes(w: synth.Workload, m_pad: int, momentum: bool = False, next_forward: bool = False,
+                      dx_in_update: bool = False, sms: int = 148) -> dict:
     """Algorithmic HBM bytes of one local iteration of all N workers, per kernel family.
 
     bf16 path: forward reads the bf16 shadow (2 B/param); dX reads it again for every layer but
@@ -143,6 +144,8 @@ def algorithmic_bytes(w: synth.Workload, m_pad: int, momentum: bool = False, nex
     The stand-alone average reads and writes the store once (8 B/word, +2 for the shadow).
     next_forward: layer 1's update also forms the next a_1, so it does not write W_1's shadow (-2 B/param) but
     reads a second minibatch and writes a_1; the forward family then has no layer-1 launch.
+    dx_in_update: layers >= 2 with enough column blocks form dZ of the layer below inside the update launch
+    (no second read of the bf16 weights; the mask read and the dZ write move to the update family).
     """
     e = 2 if w.precision == 1 else 4
     N, B, d = w.N, w.B, w.dims
@@ -151,7 +154,9 @@ def algorithmic_bytes(w: synth.Workload, m_pad: int, momentum: bool = False, nex
     for l in range(1, L + 1):
         wl = d[l] * d[l - 1]
         fwd += N * (wl * e + d[l] * 4 + B * d[l - 1] * e + B * d[l] * (e if l < L else 4))
-        if l > 1:
+        if l > 1 and dx_in_update and ((d[l - 1] + 63) // 64) * N >= 3 * sms:
+            upd += N * B * d[l - 1] * 2 * e
+        elif l > 1:
             dx += N * (wl * e + B * d[l] * e + B * d[l - 1] * 2 * e)
         upd += N * ((wl + d[l]) * (8 + (2 if w.precision == 1 else 0) + (8 if momentum else 0)) + B * (d[l] + d[l - 1]) * e)
     avg = N * m_pad * (8 + (2 if w.precision == 1 else 0))
@@ -284,6 +289,8 @@ def main():
                     help="averaging iterations run as update + stand-alone averaging kernel instead of the fused pass")
     ap.add_argument("--no-fused-epilogues", action="store_true",
                     help="softmax-CE gradient and bias steps as kernels of their own instead of GEMM epilogues")
+    ap.add_argument("--no-dx-in-update", action="store_true",
+                    help="separate dX launches instead of forming dZ of the layer below inside the update launch")
     ap.add_argument("--no-next-forward", action="store_true",
                     help="layer 1's update does not form the next iteration's a_1")
     ap.add_argument("--no-early-loads", action="store_true",
@@ -360,6 +367,8 @@ def main():
         p.enable_momentum(args.momentum)
     if args.no_fuse:
         p.set_option(binding.OPT_FUSED_AVERAGE, 0)
+    if args.no_dx_in_update:
+        p.set_option(binding.OPT_DX_IN_UPDATE, 0)
     if args.no_next_forward:
         p.set_option(binding.OPT_NEXT_FORWARD, 0)
     if args.no_early_loads:
@@ -415,7 +424,10 @@ def main():
     # iterations 1..I-1 of a period run layer 1's update with the next forward folded in (tensor-core path)
     next_fwd = (w.precision == 1 and L > 1 and w.I > 1 and w.dims[L] <= 128 and args.momentum is None
                 and not args.no_next_forward and not args.no_fused_epilogues)
-    bytes_iter = algorithmic_bytes(w, p.m_pad, args.momentum is not None, next_fwd)
+    dx_in_upd = (w.precision == 1 and w.dims[L] <= 128 and args.momentum is None and not args.no_dx_in_update
+                 and not args.no_fused_epilogues)
+    bytes_iter = algorithmic_bytes(w, p.m_pad, args.momentum is not None, next_fwd, dx_in_upd,
+                                   torch.cuda.get_device_properties(dev).multi_processor_count)
     fams = {k: v for k, v in prof.items() if v[1] > 0 and k in bytes_iter}
     dom = max(fams, key=lambda k: fams[k][0])
     per_iter_launches = {"forward": L - 1 if next_fwd else L, "dx": L - 1, "update": L, "update_average": L,

@@ -263,6 +263,13 @@ int prsgd_get_velocity_stacked(prsgd_ctx* ctx, float* dst, int dst_on_device);
  * W_1, which only that launch reads, is not written on such iterations (it is valid whenever a call
  * returns).  Same bits as the separate launches. */
 #define PRSGD_OPT_NEXT_FORWARD 7
+/* PRSGD_OPT_DX_IN_UPDATE (default 1, tensor-core path): on a plain SGD iteration the update launch of a
+ * layer l >= 2 also forms dZ_{l-1} from the bf16 values its weights had before the step, which it
+ * derives from the fp32 tiles it holds, so the separate dX launch and its second read of the layer's
+ * bf16 weights are saved.  1 = for layers with at least three 64-wide column blocks per SM over all
+ * workers (fewer do not balance), 2 = for every layer, 0 = never.  Not on fused update + average
+ * iterations, with a worker mask or with momentum.  Same bits as the separate launches. */
+#define PRSGD_OPT_DX_IN_UPDATE 8
 int prsgd_set_option(prsgd_ctx* ctx, int32_t option, int64_t value);
 
 /* Kernel families of the hot path, for prsgd_get_profile. */

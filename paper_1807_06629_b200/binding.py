@@ -27,6 +27,7 @@ OPT_GRAPH = 4
 OPT_FUSED_EPILOGUES = 5
 OPT_EARLY_LOADS = 6
 OPT_NEXT_FORWARD = 7
+OPT_DX_IN_UPDATE = 8
 KERNEL_FAMILIES = ("forward", "softmax", "dx", "update", "update_average", "average", "misc")
 MAX_LAYERS = 16
 

@@ -982,6 +982,296 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_next_kernel(const __
   if (warp == 1) tmem_dealloc(tmem, 512u);
 }
 
+// ---------------------------------------------------------------------------------------------
+// update of a layer l >= 2 with its input-gradient GEMM folded in
+// ---------------------------------------------------------------------------------------------
+// dZ_{l-1} = (dZ_l W_l) (.) relu' needs the bf16 value of every weight BEFORE its step, and the update
+// kernel has the fp32 master tile of exactly those weights in shared memory.  Its epilogue therefore
+// writes two bf16 tiles, the old values and the stepped ones; the old tile (MN-major A operand, the
+// layer's input features on the MMA's M axis) and the dZ_l boxes already loaded for dW (K-major B
+// operand) feed a second accumulator dZ_{l-1}^T[64, B].  A CTA owns a 64-wide column block of one
+// worker, walks its row tiles top to bottom so that the contraction over d_l completes in TMEM, and
+// ends the block with the dX epilogue (ReLU mask, bf16 dZ_{l-1}, bias step of layer l-1).  That saves
+// the separate dX launch and its second read of the layer's bf16 weights.
+// The accumulator has 128 lanes but the block only 64 features: the descriptor's second 64-row
+// half points at other shared memory of the stage and lanes 64..127 are never read.
+struct UpdateDxArgs {
+  int B, N;
+  int tiles_m, tiles_n;      // 128-row tiles of d_l, 64-column tiles of d_{l-1}
+  float gamma;
+  DeviceStatus* status;
+  int stages;
+  uint16_t* out_bk;          // bf16 dZ_{l-1} [N][B][ld_out]
+  const uint16_t* mask_src;  // bf16 a_{l-1}  [N][B][ld_out]
+  int ld_out;
+  int M_total;               // d_{l-1}
+  float* bias_rw;            // params + b_off of layer l-1 (worker stride bias_stride), or nullptr
+  int64_t bias_stride;
+};
+
+struct UpdDxCfg {
+  static constexpr uint32_t kMaster = 128u * 64u * 4u;     // fp32 master tile
+  static constexpr uint32_t kOld = 128u * 64u * 2u;        // bf16 of the weights before the step
+  static constexpr uint32_t kNew = 128u * 64u * 2u;        // first the a_{l-1} box, then bf16 of the stepped weights
+  __host__ __device__ static uint32_t delta_bytes(int B) { return 2u * (uint32_t)B * 128u; }
+  __host__ __device__ static uint32_t stage(int B) { return kMaster + kOld + kNew + delta_bytes(B); }
+  static int stages(int B) {
+    int s = (int)((227u * 1024u - 2048u) / stage(B));
+    return s > 4 ? 4 : s;
+  }
+  static size_t smem(int B) { return (size_t)stages(B) * stage(B) + 1024 + 512; }
+};
+
+__global__ void __launch_bounds__(kUpdThreads, 1) tc_update_dx_kernel(const __grid_constant__ CUtensorMap mapDelta,
+                                                                      const __grid_constant__ CUtensorMap mapAct,
+                                                                      const __grid_constant__ CUtensorMap mapMaster,
+                                                                      const __grid_constant__ CUtensorMap mapShadow,
+                                                                      const UpdateDxArgs a) {
+  using namespace ptx;
+  using Cfg = UpdDxCfg;
+  constexpr int TN = 64;
+  constexpr uint32_t kDxCol = 256u;                     // TMEM: dW accumulators in columns [0, 256), dX ones behind
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* gen = smem_raw + (base - raw);
+  const int S = a.stages;
+  const uint32_t stage_bytes = Cfg::stage(a.B);
+  const uint32_t op_box = (uint32_t)a.B * 128u;         // one {64, B} box
+  auto master_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes; };
+  auto old_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes + Cfg::kMaster; };
+  auto new_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes + Cfg::kMaster + Cfg::kOld; };
+  auto delta_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes + Cfg::kMaster + Cfg::kOld + Cfg::kNew; };
+  const uint32_t bar0 = base + (uint32_t)S * stage_bytes;
+  auto full_ops = [&](int s) { return bar0 + 8u * s; };
+  auto full_w = [&](int s) { return bar0 + 32u + 8u * s; };
+  auto stage_empty = [&](int s) { return bar0 + 64u + 8u * s; };
+  auto acc_full = [&](int s) { return bar0 + 96u + 8u * s; };
+  auto acc_empty = [&](int s) { return bar0 + 128u + 8u * s; };
+  auto tile_ready = [&](int s) { return bar0 + 160u + 8u * s; };
+  auto dx_done = [&](int s) { return bar0 + 192u + 8u * s; };       // the dX MMAs have read the stage's old tile and dZ boxes
+  auto dacc_full = [&](int q) { return bar0 + 224u + 8u * q; };
+  auto dacc_empty = [&](int q) { return bar0 + 240u + 8u * q; };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen + (size_t)S * stage_bytes + 256);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + (size_t)S * stage_bytes + 260);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int col_blocks = a.tiles_n * a.N;
+
+  if (tid == 0) {
+    for (int s = 0; s < S; ++s) {
+      mbar_init(full_ops(s), 1); mbar_init(full_w(s), 1); mbar_init(stage_empty(s), 1);
+      mbar_init(acc_full(s), 1); mbar_init(acc_empty(s), 128); mbar_init(tile_ready(s), 128);
+      mbar_init(dx_done(s), 1);
+    }
+    for (int q = 0; q < 2; ++q) { mbar_init(dacc_full(q), 1); mbar_init(dacc_empty(q), 128); }
+    *abort_flag = *(volatile unsigned int*)&a.status->error != 0u ? 1 : 0;   // an earlier expired wait: no-op (see tc_stream_kernel)
+    fence_mbar_init();
+    prefetch_tensormap(&mapDelta); prefetch_tensormap(&mapAct);
+    prefetch_tensormap(&mapMaster); prefetch_tensormap(&mapShadow);
+  }
+  if (warp == 1) { tmem_alloc(smem_u32(tmem_slot), 512u); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  pdl_wait();
+  pdl_trigger();
+  const uint32_t tmem = *tmem_slot;
+  const int total_cb = *abort_flag != 0 ? 0 : col_blocks;
+
+  // Every role walks the same sequence of tiles: column blocks cb = blockIdx.x, + gridDim.x, ..., and inside
+  // a column block the row tiles mb = 0 .. tiles_m - 1; `it` counts tiles, tile `it` lives in stage it % S.
+  if (warp == 0 && lane == 0) {
+    // ---------------- loader
+    uint32_t it = 0;
+    bool ok = true;
+    for (int cb = blockIdx.x; cb < total_cb && ok; cb += gridDim.x) {
+      const int n = cb / a.tiles_n, n0 = (cb % a.tiles_n) * TN;
+      for (int mb = 0; mb < a.tiles_m; ++mb, ++it) {
+        const int s = it % S;
+        const uint32_t ph = (it / S) & 1u;
+        ok = mbar_wait(stage_empty(s), ph ^ 1u, abort_flag, a.status, 0x501);
+        if (!ok) break;
+        const int m0 = mb * 128;
+        mbar_expect_tx(full_ops(s), 3u * op_box);
+        tma_load_3d(delta_u32(s), &mapDelta, full_ops(s), m0, 0, n);
+        tma_load_3d(delta_u32(s) + op_box, &mapDelta, full_ops(s), m0 + 64, 0, n);
+        tma_load_3d(new_u32(s), &mapAct, full_ops(s), n0, 0, n);
+        mbar_expect_tx(full_w(s), Cfg::kMaster);
+        tma_load_3d(master_u32(s), &mapMaster, full_w(s), n0, m0, n);
+        tma_load_3d(master_u32(s) + 16384u, &mapMaster, full_w(s), n0 + 32, m0, n);
+      }
+    }
+    if (*abort_flag && it > 0) {   // let the copies already in flight land before the CTA goes away
+      const uint32_t first = it > (uint32_t)S ? it - (uint32_t)S : 0u;
+      for (uint32_t q = first; q < it; ++q) {
+        const uint64_t t0 = globaltimer_ns();
+        while (!(mbar_try_wait(full_w(q % S), (q / S) & 1u) && mbar_try_wait(full_ops(q % S), (q / S) & 1u)) &&
+               globaltimer_ns() - t0 < 100000000ull) {}
+      }
+    }
+  } else if (warp == 1 && lane == 0) {
+    // ---------------- MMA issuer: dW of tile `it`, then the dX contribution of tile it - 1 (whose bf16
+    // tiles the epilogue has finished meanwhile)
+    const uint32_t idesc_dw = idesc_bf16(128, TN, 1, 1);
+    const uint32_t idesc_dx = idesc_bf16(128, a.B, 1, 0);
+    const int ksteps = a.B / 16;
+    uint32_t it = 0, cbi = 0;
+    bool ok = true;
+    bool have_prev = false;
+    uint32_t p_it = 0, p_cbi = 0;
+    int p_mb = 0;
+    auto dx_of = [&](uint32_t j, int mb, uint32_t cj) -> bool {
+      const int s = j % S, q = cj & 1;
+      if (mb == 0 && !mbar_wait(dacc_empty(q), ((cj >> 1) & 1u) ^ 1u, abort_flag, a.status, 0x502)) return false;
+      if (!mbar_wait(tile_ready(s), (j / S) & 1u, abort_flag, a.status, 0x503)) return false;
+      tc_fence_after();
+      const uint32_t acc = tmem + kDxCol + (uint32_t)(q * a.B);
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {                       // the tile's two 64-row halves = the two dZ_l boxes
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          mma_bf16(acc, smem_desc_sw128(old_u32(s) + (uint32_t)(h * 4 + k) * 2048u, Cfg::kOld, 1024u),
+                   smem_desc_sw128(delta_u32(s) + h * op_box + k * 32u, 16u, 1024u), idesc_dx, (mb | h | k) != 0 ? 1u : 0u);
+      }
+      mma_commit(dx_done(s));
+      if (mb == a.tiles_m - 1) mma_commit(dacc_full(q));
+      return true;
+    };
+    for (int cb = blockIdx.x; cb < total_cb && ok; cb += gridDim.x, ++cbi) {
+      for (int mb = 0; mb < a.tiles_m && ok; ++mb, ++it) {
+        const int s = it % S;
+        const uint32_t ph = (it / S) & 1u;
+        ok = mbar_wait(acc_empty(s), ph ^ 1u, abort_flag, a.status, 0x504) &&
+             mbar_wait(full_ops(s), ph, abort_flag, a.status, 0x505);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t sa = delta_u32(s), sb = new_u32(s);
+        for (int k = 0; k < ksteps; ++k)
+          mma_bf16(tmem + (uint32_t)(s * TN), smem_desc_sw128(sa + k * 2048u, op_box, 1024u),
+                   smem_desc_sw128(sb + k * 2048u, op_box, 1024u), idesc_dw, k != 0 ? 1u : 0u);
+        mma_commit(acc_full(s));
+        if (have_prev) ok = dx_of(p_it, p_mb, p_cbi);
+        p_it = it; p_mb = mb; p_cbi = cbi; have_prev = true;
+      }
+    }
+    if (ok && have_prev) dx_of(p_it, p_mb, p_cbi);
+  } else if (warp == 2 && lane == 0) {
+    // ---------------- storer
+    uint32_t it = 0;
+    bool ok = true;
+    for (int cb = blockIdx.x; cb < total_cb && ok; cb += gridDim.x) {
+      const int n = cb / a.tiles_n, n0 = (cb % a.tiles_n) * TN;
+      for (int mb = 0; mb < a.tiles_m; ++mb, ++it) {
+        const int s = it % S;
+        const uint32_t ph = (it / S) & 1u;
+        const int m0 = mb * 128;
+        ok = mbar_wait(tile_ready(s), ph, abort_flag, a.status, 0x506);
+        if (!ok) break;
+        tma_store_3d(&mapMaster, master_u32(s), n0, m0, n);
+        tma_store_3d(&mapMaster, master_u32(s) + 16384u, n0 + 32, m0, n);
+        tma_store_3d(&mapShadow, new_u32(s), n0, m0, n);
+        tma_commit_group();
+        tma_wait_group_read0();
+        ok = mbar_wait(dx_done(s), ph, abort_flag, a.status, 0x507);
+        if (!ok) break;
+        mbar_arrive(stage_empty(s));
+      }
+    }
+    tma_wait_group0();
+  } else if (warp >= 3) {
+    // ---------------- epilogue: row r of the tile <-> TMEM lane r
+    const int q4 = warp & 3;
+    const int r = q4 * 32 + lane;
+    const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
+    const uint32_t row_off = (uint32_t)r * 128u;
+    const uint32_t sw = (uint32_t)(r & 7);
+    const int batches = a.B / 16;
+    uint32_t it = 0, cbi = 0;
+    bool ok = true;
+    for (int cb = blockIdx.x; cb < total_cb && ok; cb += gridDim.x, ++cbi) {
+      const int n = cb / a.tiles_n, n0 = (cb % a.tiles_n) * TN;
+      for (int mb = 0; mb < a.tiles_m; ++mb, ++it) {
+        const int s = it % S;
+        const uint32_t ph = (it / S) & 1u;
+        ok = mbar_wait(full_w(s), ph, abort_flag, a.status, 0x508) &&
+             mbar_wait(acc_full(s), ph, abort_flag, a.status, 0x509);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        uint8_t* mst = gen + (size_t)s * stage_bytes;
+        uint8_t* old = mst + Cfg::kMaster;
+        uint8_t* stg = old + Cfg::kOld;
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          uint32_t v[32];
+          tmem_ld32(tmem + lane_off + (uint32_t)(s * TN + c * 32), v);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            float4* pw = reinterpret_cast<float4*>(mst + c * 16384 + row_off + (((uint32_t)j ^ sw) << 4));
+            float4 x = *pw;
+            const uint32_t chunk = (uint32_t)(c * 4 + (j >> 1));
+            const uint32_t boff = row_off + ((chunk ^ sw) << 4) + (uint32_t)(j & 1) * 8u;
+            *reinterpret_cast<uint2*>(old + boff) = make_uint2(pack_bf16x2(x.x, x.y), pack_bf16x2(x.z, x.w));
+            x.x = fmaf(-a.gamma, __uint_as_float(v[4 * j + 0]), x.x);
+            x.y = fmaf(-a.gamma, __uint_as_float(v[4 * j + 1]), x.y);
+            x.z = fmaf(-a.gamma, __uint_as_float(v[4 * j + 2]), x.z);
+            x.w = fmaf(-a.gamma, __uint_as_float(v[4 * j + 3]), x.w);
+            *pw = x;
+            *reinterpret_cast<uint2*>(stg + boff) = make_uint2(pack_bf16x2(x.x, x.y), pack_bf16x2(x.z, x.w));
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(acc_empty(s));
+        fence_proxy_async();
+        mbar_arrive(tile_ready(s));
+      }
+      if (!ok) break;
+      // dX epilogue of the column block: feature c = n0 + r (lanes 0..63 only)
+      const int q = cbi & 1;
+      const int cfeat = n0 + r;
+      const bool valid = r < TN && cfeat < a.M_total;
+      uint16_t mk[16];
+      auto mask_fetch = [&](int bi) {
+        if (bi < batches && valid) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) mk[j] = __ldg(a.mask_src + ((int64_t)n * a.B + bi * 16 + j) * a.ld_out + cfeat);
+        }
+      };
+      mask_fetch(0);
+      ok = __all_sync(0xffffffffu, mbar_wait(dacc_full(q), (cbi >> 1) & 1u, abort_flag, a.status, 0x50A));
+      if (!ok) break;
+      tc_fence_after();
+      float gsum = 0.f;
+      for (int bi = 0; bi < batches; ++bi) {
+        uint32_t v[16];
+        tmem_ld16(tmem + lane_off + kDxCol + (uint32_t)(q * a.B + bi * 16), v);
+        tmem_ld_wait();
+        if (valid) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const float d = (mk[j] & 0x7FFFu) != 0 ? __uint_as_float(v[j]) : 0.f;
+            gsum += d;
+            a.out_bk[((int64_t)n * a.B + bi * 16 + j) * a.ld_out + cfeat] = f32_to_bf16_rn(d);
+          }
+        }
+        mask_fetch(bi + 1);
+      }
+      tc_fence_before();
+      mbar_arrive(dacc_empty(q));
+      if (valid && a.bias_rw != nullptr) {
+        float* bp = a.bias_rw + (int64_t)n * a.bias_stride + cfeat;
+        *bp = fmaf(-a.gamma, gsum, *bp);
+      }
+    }
+  }
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem, 512u);
+}
+
 // b_l <- b_l - gamma * sum_b dZ_l[b, :] (the bias part of Eq. parallel-sgd-x-update) for every layer in
 // one launch: grid (ceil(max d_l / 128), N, L), one thread per (layer, worker, j).
 struct BiasArgs {
@@ -1108,6 +1398,7 @@ inline int tc_create(prsgd_ctx* c, std::string* err) {
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<false, 128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<128, false>::smem(c->B));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<true, 128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<128, false>::smem(c->B));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<false, 64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<64, true>::smem(c->B));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_dx_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdDxCfg::smem(c->B));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_next_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdNextCfg<64>::smem(c->B));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_next_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdNextCfg<128>::smem(c->B));
   if (e != cudaSuccess) {
@@ -1219,6 +1510,31 @@ inline void tc_launch_update_tn(prsgd_ctx* c, int l, const DrawArgs& dr, const u
     else
       launch_pdl(tc_update_kernel<false, TN, false>, dim3(grid), kUpdThreads, smem, c->stream, mp.delta_out, mp.act_in, mp.master, mp.shadow_k, mp.master, a);
   }
+}
+
+// The folded form gives a CTA whole 64-wide column blocks of one worker (all row tiles of the block), so it
+// needs several blocks per SM to balance; with fewer the separate dX and update launches (one tile per
+// item) are faster.
+inline bool tc_layer_folds_dx(const prsgd_ctx* c, int l) {
+  const TcState* st = static_cast<const TcState*>(c->tc);
+  const int64_t blocks = (int64_t)((c->layer[l - 1].d_in + 63) / 64) * c->N;
+  return blocks >= 3 * (int64_t)st->num_sms;
+}
+
+// Update of layer l >= 2 that also forms dZ_{l-1} (tc_update_dx_kernel): replaces dX_l + update_l.
+inline void tc_launch_update_dx(prsgd_ctx* c, int l) {
+  TcState* st = static_cast<TcState*>(c->tc);
+  const Layer& ly = c->layer[l - 1];
+  UpdateDxArgs a{};
+  a.B = c->B; a.N = c->N; a.tiles_m = (ly.d_out + 127) / 128; a.tiles_n = (ly.d_in + 63) / 64;
+  a.gamma = c->gamma; a.status = c->status; a.stages = UpdDxCfg::stages(c->B);
+  a.out_bk = c->buf.delta_bk[l - 1]; a.mask_src = c->buf.act_bk[l - 1]; a.ld_out = c->buf.ld[l - 1]; a.M_total = ly.d_in;
+  a.bias_rw = c->params + c->layer[l - 2].b_off; a.bias_stride = c->m_pad;
+  const int items = a.tiles_n * c->N;
+  const int grid = items < st->num_sms ? items : st->num_sms;
+  const TcLayerMaps& mp = st->layer[l - 1];
+  launch_pdl(tc_update_dx_kernel, dim3(grid), kUpdThreads, UpdDxCfg::smem(c->B), c->stream, mp.delta_out, mp.act_in, mp.master,
+             mp.shadow_k, a);
 }
 
 // Update of layer 1 that also forms a_1 of the next iteration (tc_update_next_kernel).

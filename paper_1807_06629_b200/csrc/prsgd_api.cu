@@ -310,7 +310,16 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging, bool more_follow) {
     launch_pdl(softmax_ce_kernel, dim3(N, (c->B + 7) / 8), dim3(256), 0, c->stream, a);
     LAUNCH_CHECK(c);
   }
+  // Layers >= 2 on a plain SGD iteration: one launch forms dZ_{l-1} and applies the step of W_l (the fused
+  // update + average of an averaging iteration owns a tile across workers instead and keeps dX separate).
+  const bool dx_in_upd = c->dx_in_update && !fuse && act_mask == nullptr && c->velocity == nullptr && tc_epilogues_fused(c);
   for (int l = L; l >= 1; --l) {          // dX_l reads W_l before the update of layer l overwrites it
+    if (l > 1 && dx_in_upd && (c->dx_in_update == 2 || tc_layer_folds_dx(c, l))) {
+      prof_begin(c, PRSGD_KERNEL_UPDATE);
+      tc_launch_update_dx(c, l);
+      LAUNCH_CHECK(c);
+      continue;
+    }
     if (l > 1) {
       prof_begin(c, PRSGD_KERNEL_DX);
       tc_launch_dx(c, l, dr, act_mask);
@@ -597,7 +606,7 @@ void period_key(const prsgd_ctx* c, uint64_t (&key)[12]) {
   key[0] = gbits; key[1] = (uint64_t)c->I; key[2] = (uint64_t)c->fused_average; key[3] = (uint64_t)c->upd_tile;
   key[4] = c->has_mask ? 1 : 0; key[5] = reinterpret_cast<uint64_t>(c->velocity); key[6] = mbits;
   key[7] = (uint64_t)c->average_velocity; key[8] = reinterpret_cast<uint64_t>(c->X);
-  key[9] = reinterpret_cast<uint64_t>(c->Y); key[10] = (uint64_t)c->worker0; key[11] = (uint64_t)c->fused_epilogues | ((uint64_t)c->early_loads << 1) | ((uint64_t)c->next_forward << 2);
+  key[9] = reinterpret_cast<uint64_t>(c->Y); key[10] = (uint64_t)c->worker0; key[11] = (uint64_t)c->fused_epilogues | ((uint64_t)c->early_loads << 1) | ((uint64_t)c->next_forward << 2) | ((uint64_t)c->dx_in_update << 3);
 }
 
 // One whole averaging period (I iterations starting right after an average) as a CUDA graph: the
@@ -902,6 +911,11 @@ int prsgd_set_option(prsgd_ctx* c, int32_t option, int64_t value) {
   if (option == PRSGD_OPT_FUSED_EPILOGUES) { c->fused_epilogues = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_EARLY_LOADS) { c->early_loads = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_NEXT_FORWARD) { c->next_forward = value != 0; return PRSGD_OK; }
+  if (option == PRSGD_OPT_DX_IN_UPDATE) {
+    if (value < 0 || value > 2) return fail(c, PRSGD_ERR_ARG, "PRSGD_OPT_DX_IN_UPDATE takes 0, 1 or 2");
+    c->dx_in_update = (int)value;
+    return PRSGD_OK;
+  }
   if (option == PRSGD_OPT_UPDATE_TILE) {
     if (value != 0 && value != 64 && value != 128) return fail(c, PRSGD_ERR_ARG, "update tile width must be 0, 64 or 128");
     c->upd_tile = (int)value;

@@ -183,6 +183,34 @@ def test_next_forward_folded_into_the_first_layers_update_changes_no_bit(torch_c
         assert outs[1][3] < outs[0][3]                 # forward launches were saved
 
 
+def test_dx_folded_into_the_update_changes_no_bit(torch_cuda):
+    """dZ of the layer below formed inside the update launch (from the bf16 values the weights had before the
+    step) against the separate dX launch: identical parameters, losses and bias steps over several periods,
+    direct and replayed, with and without the folded next forward."""
+    torch = torch_cuda
+    from paper_1807_06629_b200 import binding
+    cases = (SMALL[1], SMALL[2], SMALL[3], SMALL[4], SMALL[6], _w("tc-n5-I5", 5, (192, 128, 10), 32, I=5),
+             _w("tc-wide-hidden", 3, (64, 448, 320, 10), 16, I=4))
+    for w in cases:
+        X, Y, x0 = make_inputs(w)
+        outs = []
+        for dxu, nxt, graph in ((0, 0, 0), (2, 0, 0), (2, 1, 0), (2, 1, 1), (2, 0, 1)):      # 2 = every layer, whatever its size
+            with torch.cuda.stream(torch.cuda.Stream()):
+                p = make_ctx(w, X, Y, x0)
+                p.set_option(binding.OPT_DX_IN_UPDATE, dxu)
+                p.set_option(binding.OPT_NEXT_FORWARD, nxt)
+                p.set_option(binding.OPT_GRAPH, graph)
+                n0 = p.get_launch_count()
+                p.local_steps(2)
+                p.local_steps(2 * w.I + 1)
+                outs.append((p.get_params_stacked(), p.get_losses(), p.get_launch_count() - n0))
+                torch.cuda.current_stream().synchronize()
+        for o in outs[1:]:
+            assert np.array_equal(outs[0][0], o[0]), w.name
+            assert np.array_equal(outs[0][1], o[1])
+        assert outs[1][2] < outs[0][2]
+
+
 def _segments(dims):
     """[(is_weight, start, stop)] of a canonical parameter vector."""
     out, off = [], 0
@@ -204,6 +232,7 @@ def test_epilogue_softmax_and_bias_steps_equal_the_standalone_kernels(torch_cuda
     for fused in (1, 0):
         p = make_ctx(w, X, Y, x0, I=0)
         p.set_option(binding.OPT_FUSED_EPILOGUES, fused)
+        p.set_option(binding.OPT_DX_IN_UPDATE, 0)         # (needs the epilogue form; off in both arms)
         n0 = p.get_launch_count()
         p.local_steps(1)
         outs.append((p.get_params_stacked(), p.get_losses(), p.get_draws().tolist(), p.get_launch_count() - n0))
