@@ -332,6 +332,8 @@ def main():
     if sharded_mode:
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         os.environ.setdefault("MASTER_PORT", "29533")
+        if os.environ.get("NCCL_DEBUG", "").upper() == "VERSION":   # its banner would share stdout with the JSON line
+            os.environ["NCCL_DEBUG"] = "WARN"
         dist.init_process_group("nccl", rank=rank, world_size=world, device_id=torch.device(dev))
         dist.barrier()
     from paper_1807_06629_b200 import binding, sharded

@@ -295,8 +295,9 @@ int prsgd_sync(prsgd_ctx* ctx);
 
 /* Failure path, exercised without faulting the GPU.  Every wait inside the tensor-core kernels is
  * bounded; when one expires the kernel records a code in the scratch status words and returns, later
- * launches of the context become no-ops, and prsgd_sync / prsgd_get_* return
- * PRSGD_ERR_DEVICE_TIMEOUT.  prsgd_selftest_wait_expiry launches a one-warp kernel that waits about
+ * launches of the context become no-ops (a kernel reads the word while it sets up, so the one launch
+ * whose set-up overlapped the failing kernel may still run; the parameters are to be set again after
+ * a timeout in any case), and prsgd_sync / prsgd_get_* return PRSGD_ERR_DEVICE_TIMEOUT.  prsgd_selftest_wait_expiry launches a one-warp kernel that waits about
  * limit_us microseconds (1..1000000) on a barrier nothing ever signals, so that exactly this happens;
  * prsgd_clear_device_error zeroes the status words and makes the context usable again (the
  * parameters are as the last successful launch left them). */

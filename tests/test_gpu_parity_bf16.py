@@ -194,16 +194,25 @@ def test_dx_folded_into_the_update_changes_no_bit(torch_cuda):
     for w in cases:
         X, Y, x0 = make_inputs(w)
         outs = []
-        for dxu, nxt, graph in ((0, 0, 0), (2, 0, 0), (2, 1, 0), (2, 1, 1), (2, 0, 1)):      # 2 = every layer, whatever its size
+        # dxu 2 = every layer, whatever its size; the tile width only concerns layer 1's update here
+        for dxu, nxt, graph, tile in ((0, 0, 0, 0), (2, 0, 0, 64), (2, 1, 0, 128), (2, 1, 1, 64), (2, 0, 1, 128)):
             with torch.cuda.stream(torch.cuda.Stream()):
                 p = make_ctx(w, X, Y, x0)
                 p.set_option(binding.OPT_DX_IN_UPDATE, dxu)
                 p.set_option(binding.OPT_NEXT_FORWARD, nxt)
                 p.set_option(binding.OPT_GRAPH, graph)
+                p.set_option(binding.OPT_UPDATE_TILE, tile)
                 n0 = p.get_launch_count()
                 p.local_steps(2)
                 p.local_steps(2 * w.I + 1)
-                outs.append((p.get_params_stacked(), p.get_losses(), p.get_launch_count() - n0))
+                launches = p.get_launch_count() - n0
+                p.sync()
+                store = p.params.cpu().numpy().reshape(w.N, p.m_pad)
+                shadow = p.shadow.view(torch.int16).cpu().numpy().view(np.uint16).reshape(w.N, p.m_pad)
+                for l in range(len(w.dims) - 1):          # the bf16 copy follows the master through either store path
+                    a, n = p.layout.w_off[l], w.dims[l] * w.dims[l + 1]
+                    assert np.array_equal(shadow[:, a:a + n], synth.bf16_bits(store[:, a:a + n])), (w.name, l, tile)
+                outs.append((p.get_params_stacked(), p.get_losses(), launches))
                 torch.cuda.current_stream().synchronize()
         for o in outs[1:]:
             assert np.array_equal(outs[0][0], o[0]), w.name
