@@ -107,8 +107,8 @@ class ClockSampler:
 # dram__bytes_read.sum + dram__bytes_write.sum per iteration of one kernel family, from the one-pass ncu
 # capture summarised in profiles/; valid only while the kernel's source section is unchanged.
 NCU_TRAFFIC = {
-    ("cfg4", "update"): {"bytes_per_iteration": 2.229e9 + 3.035e9, "launches_per_iteration": 4,   # read + written, four launches
-                         "kernel_sha256": "20c3a8a2a487e4f915bc302e408ff116e624e98895c886832c53b20c2bbc6d68"},
+    ("cfg4", "update"): {"bytes_per_iteration": 2.229e9 + 2.795e9, "launches_per_iteration": 4,   # read + written, four launches
+                         "kernel_sha256": "8cc569b9ddeba64fbde7ec602239fe0f95a469eecf0f1d1b48647a906608ffe3"},
 }
 
 
@@ -154,7 +154,7 @@ def algorithmic_bytes(w: synth.Workload, m_pad: int, momentum: bool = False, nex
     for l in range(1, L + 1):
         wl = d[l] * d[l - 1]
         fwd += N * (wl * e + d[l] * 4 + B * d[l - 1] * e + B * d[l] * (e if l < L else 4))
-        if l > 1 and dx_in_update and ((d[l - 1] + 63) // 64) * N >= 3 * sms:
+        if l > 1 and dx_in_update and (((d[l - 1] + 63) // 64) * N >= 3 * sms or d[l] <= 128):
             upd += N * B * d[l - 1] * 2 * e
         elif l > 1:
             dx += N * (wl * e + B * d[l] * e + B * d[l - 1] * 2 * e)

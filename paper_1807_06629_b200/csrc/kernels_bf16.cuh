@@ -1514,11 +1514,12 @@ inline void tc_launch_update_tn(prsgd_ctx* c, int l, const DrawArgs& dr, const u
 
 // The folded form gives a CTA whole 64-wide column blocks of one worker (all row tiles of the block), so it
 // needs several blocks per SM to balance; with fewer the separate dX and update launches (one tile per
-// item) are faster.
+// item) are faster.  A layer of a single row tile (the class layer) has one tile per block anyway and is
+// latency-bound: there one launch instead of two always wins.
 inline bool tc_layer_folds_dx(const prsgd_ctx* c, int l) {
   const TcState* st = static_cast<const TcState*>(c->tc);
   const int64_t blocks = (int64_t)((c->layer[l - 1].d_in + 63) / 64) * c->N;
-  return blocks >= 3 * (int64_t)st->num_sms;
+  return blocks >= 3 * (int64_t)st->num_sms || c->layer[l - 1].d_out <= 128;
 }
 
 // Update of layer l >= 2 that also forms dZ_{l-1} (tc_update_dx_kernel): replaces dX_l + update_l.
