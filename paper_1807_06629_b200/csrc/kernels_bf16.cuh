@@ -936,17 +936,22 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_next_kernel(const __
           tmem_ld32(tmem + lane_off + (uint32_t)(s * TN + c * 32), v);
           tmem_ld_wait();
 #pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            float4* pw = reinterpret_cast<float4*>(mst + c * 16384 + row_off + (((uint32_t)j ^ sw) << 4));
-            float4 x = *pw;
-            x.x = fmaf(-a.gamma, __uint_as_float(v[4 * j + 0]), x.x);
-            x.y = fmaf(-a.gamma, __uint_as_float(v[4 * j + 1]), x.y);
-            x.z = fmaf(-a.gamma, __uint_as_float(v[4 * j + 2]), x.z);
-            x.w = fmaf(-a.gamma, __uint_as_float(v[4 * j + 3]), x.w);
-            *pw = x;
-            const uint32_t chunk = (uint32_t)((c & 1) * 4 + (j >> 1));
-            uint2* pb = reinterpret_cast<uint2*>(stg + (c >> 1) * 16384 + row_off + ((chunk ^ sw) << 4) + (j & 1) * 8);
-            *pb = make_uint2(pack_bf16x2(x.x, x.y), pack_bf16x2(x.z, x.w));
+          for (int jp = 0; jp < 4; ++jp) {                  // two 16-byte fp32 chunks = one 16-byte bf16 chunk
+            float4* p0 = reinterpret_cast<float4*>(mst + c * 16384 + row_off + (((uint32_t)(2 * jp) ^ sw) << 4));
+            float4* p1 = reinterpret_cast<float4*>(mst + c * 16384 + row_off + (((uint32_t)(2 * jp + 1) ^ sw) << 4));
+            float4 x = *p0, y = *p1;
+            x.x = fmaf(-a.gamma, __uint_as_float(v[8 * jp + 0]), x.x);
+            x.y = fmaf(-a.gamma, __uint_as_float(v[8 * jp + 1]), x.y);
+            x.z = fmaf(-a.gamma, __uint_as_float(v[8 * jp + 2]), x.z);
+            x.w = fmaf(-a.gamma, __uint_as_float(v[8 * jp + 3]), x.w);
+            y.x = fmaf(-a.gamma, __uint_as_float(v[8 * jp + 4]), y.x);
+            y.y = fmaf(-a.gamma, __uint_as_float(v[8 * jp + 5]), y.y);
+            y.z = fmaf(-a.gamma, __uint_as_float(v[8 * jp + 6]), y.z);
+            y.w = fmaf(-a.gamma, __uint_as_float(v[8 * jp + 7]), y.w);
+            *p0 = x; *p1 = y;
+            const uint32_t chunk = (uint32_t)((c & 1) * 4 + jp);
+            *reinterpret_cast<uint4*>(stg + (c >> 1) * 16384 + row_off + ((chunk ^ sw) << 4)) =
+                make_uint4(pack_bf16x2(x.x, x.y), pack_bf16x2(x.z, x.w), pack_bf16x2(y.x, y.y), pack_bf16x2(y.z, y.w));
           }
         }
         tc_fence_before();
@@ -1208,18 +1213,24 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_dx_kernel(const __gr
           tmem_ld32(tmem + lane_off + (uint32_t)(s * TN + c * 32), v);
           tmem_ld_wait();
 #pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            float4* pw = reinterpret_cast<float4*>(mst + c * 16384 + row_off + (((uint32_t)j ^ sw) << 4));
-            float4 x = *pw;
-            const uint32_t chunk = (uint32_t)(c * 4 + (j >> 1));
-            const uint32_t boff = row_off + ((chunk ^ sw) << 4) + (uint32_t)(j & 1) * 8u;
-            *reinterpret_cast<uint2*>(old + boff) = make_uint2(pack_bf16x2(x.x, x.y), pack_bf16x2(x.z, x.w));
-            x.x = fmaf(-a.gamma, __uint_as_float(v[4 * j + 0]), x.x);
-            x.y = fmaf(-a.gamma, __uint_as_float(v[4 * j + 1]), x.y);
-            x.z = fmaf(-a.gamma, __uint_as_float(v[4 * j + 2]), x.z);
-            x.w = fmaf(-a.gamma, __uint_as_float(v[4 * j + 3]), x.w);
-            *pw = x;
-            *reinterpret_cast<uint2*>(stg + boff) = make_uint2(pack_bf16x2(x.x, x.y), pack_bf16x2(x.z, x.w));
+          for (int jp = 0; jp < 4; ++jp) {                  // two 16-byte fp32 chunks = one 16-byte bf16 chunk
+            float4* p0 = reinterpret_cast<float4*>(mst + c * 16384 + row_off + (((uint32_t)(2 * jp) ^ sw) << 4));
+            float4* p1 = reinterpret_cast<float4*>(mst + c * 16384 + row_off + (((uint32_t)(2 * jp + 1) ^ sw) << 4));
+            float4 x = *p0, y = *p1;
+            const uint32_t boff = row_off + (((uint32_t)(c * 4 + jp) ^ sw) << 4);
+            *reinterpret_cast<uint4*>(old + boff) = make_uint4(pack_bf16x2(x.x, x.y), pack_bf16x2(x.z, x.w),
+                                                               pack_bf16x2(y.x, y.y), pack_bf16x2(y.z, y.w));
+            x.x = fmaf(-a.gamma, __uint_as_float(v[8 * jp + 0]), x.x);
+            x.y = fmaf(-a.gamma, __uint_as_float(v[8 * jp + 1]), x.y);
+            x.z = fmaf(-a.gamma, __uint_as_float(v[8 * jp + 2]), x.z);
+            x.w = fmaf(-a.gamma, __uint_as_float(v[8 * jp + 3]), x.w);
+            y.x = fmaf(-a.gamma, __uint_as_float(v[8 * jp + 4]), y.x);
+            y.y = fmaf(-a.gamma, __uint_as_float(v[8 * jp + 5]), y.y);
+            y.z = fmaf(-a.gamma, __uint_as_float(v[8 * jp + 6]), y.z);
+            y.w = fmaf(-a.gamma, __uint_as_float(v[8 * jp + 7]), y.w);
+            *p0 = x; *p1 = y;
+            *reinterpret_cast<uint4*>(stg + boff) = make_uint4(pack_bf16x2(x.x, x.y), pack_bf16x2(x.z, x.w),
+                                                               pack_bf16x2(y.x, y.y), pack_bf16x2(y.z, y.w));
           }
         }
         tc_fence_before();
