@@ -108,7 +108,7 @@ class ClockSampler:
 # capture summarised in profiles/; valid only while the kernel's source section is unchanged.
 NCU_TRAFFIC = {
     ("cfg4", "update"): {"bytes_per_iteration": 2.229e9 + 2.795e9, "launches_per_iteration": 4,   # read + written, four launches
-                         "kernel_sha256": "8cc569b9ddeba64fbde7ec602239fe0f95a469eecf0f1d1b48647a906608ffe3"},
+                         "kernel_sha256": "c4a779b798958f0d7598e1b80f5f3c23f8874727a33142956d97076ae4443bb2"},
 }
 
 
