@@ -641,6 +641,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
           uint32_t v[32];
           tmem_ld32(tmem + lane_off + (uint32_t)(s * TN + c * 32), v);
           tmem_ld_wait();
+          uint2 lo = make_uint2(0u, 0u);
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
             float4* pw = reinterpret_cast<float4*>(mst + c * 16384 + row_off + (((uint32_t)j ^ sw) << 4));
@@ -671,9 +672,14 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
             }
             if (!FUSE || last) {
               *pw = x;
-              const uint32_t chunk = (uint32_t)((c & 1) * 4 + (j >> 1));
-              uint2* pb = reinterpret_cast<uint2*>(stg + (c >> 1) * 16384 + row_off + ((chunk ^ sw) << 4) + (j & 1) * 8);
-              *pb = make_uint2(pack_bf16x2(x.x, x.y), pack_bf16x2(x.z, x.w));
+              // two neighbouring fp32 chunks make one 16-byte bf16 chunk: a single conflict-free store
+              if ((j & 1) == 0) {
+                lo = make_uint2(pack_bf16x2(x.x, x.y), pack_bf16x2(x.z, x.w));
+              } else {
+                const uint32_t chunk = (uint32_t)((c & 1) * 4 + (j >> 1));
+                *reinterpret_cast<uint4*>(stg + (c >> 1) * 16384 + row_off + ((chunk ^ sw) << 4)) =
+                    make_uint4(lo.x, lo.y, pack_bf16x2(x.x, x.y), pack_bf16x2(x.z, x.w));
+              }
             }
           }
         }
@@ -708,8 +714,8 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
 // worker), walks their column tiles left to right, accumulates z_1 = W_1 x' over them in a second
 // TMEM accumulator and finishes the row block with the forward epilogue (bias, ReLU, bf16 a_1).
 // The forward launch of layer 1 in the next iteration is then skipped, and W_1's bf16 shadow, which
-// only that launch reads, need not be written (the host asks for it on the last iteration of a call
-// so that the shadow is valid whenever control returns to the caller).
+// only that launch reads, is not written (the host uses the ordinary update on the last iteration of
+// a call, so the shadow is valid whenever control returns to the caller).
 struct UpdateNextArgs {
   int B, N;
   int tiles_m, tiles_n;
@@ -717,7 +723,6 @@ struct UpdateNextArgs {
   DrawArgs draw;             // iteration t; the next minibatch is the draw of t + 1
   DeviceStatus* status;
   int stages;
-  int write_shadow;
   uint16_t* next_out;        // bf16 a_1 [N][B][next_ld]
   int next_ld;
   const float* bias;         // params + b_off of layer 1 (already stepped by this iteration's dX epilogue)
@@ -743,7 +748,6 @@ template <int TN>
 __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_next_kernel(const __grid_constant__ CUtensorMap mapDelta,
                                                                         const __grid_constant__ CUtensorMap mapPool,
                                                                         const __grid_constant__ CUtensorMap mapMaster,
-                                                                        const __grid_constant__ CUtensorMap mapShadow,
                                                                         const UpdateNextArgs a) {
   using namespace ptx;
   using Cfg = UpdNextCfg<TN>;
@@ -785,7 +789,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_next_kernel(const __
     *abort_flag = *(volatile unsigned int*)&a.status->error != 0u ? 1 : 0;   // an earlier expired wait: no-op (see tc_stream_kernel)
     fence_mbar_init();
     prefetch_tensormap(&mapDelta); prefetch_tensormap(&mapPool);
-    prefetch_tensormap(&mapMaster); prefetch_tensormap(&mapShadow);
+    prefetch_tensormap(&mapMaster);
   }
   if (warp == 1) { tmem_alloc(smem_u32(tmem_slot), 512u); tmem_relinquish(); }
   tc_fence_before();
@@ -896,10 +900,6 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_next_kernel(const __
         if (!ok) break;
 #pragma unroll
         for (int q = 0; q < NB32; ++q) tma_store_3d(&mapMaster, master_u32(s) + q * 16384u, n0 + 32 * q, m0, n);
-        if (a.write_shadow) {
-#pragma unroll
-          for (int h = 0; h < NB64; ++h) tma_store_3d(&mapShadow, ops_u32(s) + h * 16384u, n0 + 64 * h, m0, n);
-        }
         tma_commit_group();
         tma_wait_group_read0();
         ok = mbar_wait(fwd_done(s), ph, abort_flag, a.status, 0x407);
@@ -1551,23 +1551,23 @@ inline void tc_launch_update_dx(prsgd_ctx* c, int l) {
 
 // Update of layer 1 that also forms a_1 of the next iteration (tc_update_next_kernel).
 template <int TN>
-inline void tc_launch_update_next_tn(prsgd_ctx* c, const DrawArgs& dr, bool write_shadow) {
+inline void tc_launch_update_next_tn(prsgd_ctx* c, const DrawArgs& dr) {
   TcState* st = static_cast<TcState*>(c->tc);
   const Layer& ly = c->layer[0];
   UpdateNextArgs a{};
   a.B = c->B; a.N = c->N; a.tiles_m = (ly.d_out + 127) / 128; a.tiles_n = (ly.d_in + TN - 1) / TN;
   a.gamma = c->gamma; a.draw = dr; a.status = c->status;
-  a.stages = UpdNextCfg<TN>::stages(c->B); a.write_shadow = write_shadow ? 1 : 0;
+  a.stages = UpdNextCfg<TN>::stages(c->B);
   a.next_out = c->buf.act_bk[1]; a.next_ld = c->buf.ld[1];
   a.bias = c->params + ly.b_off; a.bias_stride = c->m_pad; a.M_total = ly.d_out;
   const int items = a.tiles_m * c->N;
   const int grid = items < st->num_sms ? items : st->num_sms;
   const TcLayerMaps& mp = st->layer[0];
   launch_pdl(tc_update_next_kernel<TN>, dim3(grid), kUpdThreads, UpdNextCfg<TN>::smem(c->B), c->stream, mp.delta_out, mp.act_in,
-             mp.master, mp.shadow_k, a);
+             mp.master, a);
 }
 
-inline void tc_launch_update_next(prsgd_ctx* c, const DrawArgs& dr, bool write_shadow) {
+inline void tc_launch_update_next(prsgd_ctx* c, const DrawArgs& dr) {
   const TcState* st = static_cast<const TcState*>(c->tc);
   const Layer& ly = c->layer[0];
   int tile = c->upd_tile;
@@ -1575,8 +1575,8 @@ inline void tc_launch_update_next(prsgd_ctx* c, const DrawArgs& dr, bool write_s
     const int64_t tiles128 = (int64_t)((ly.d_out + 127) / 128) * ((ly.d_in + 127) / 128);
     tile = (c->B <= 32 && tiles128 * c->N >= 32 * (int64_t)st->num_sms) ? 128 : 64;
   }
-  if (tile == 128) tc_launch_update_next_tn<128>(c, dr, write_shadow);
-  else tc_launch_update_next_tn<64>(c, dr, write_shadow);
+  if (tile == 128) tc_launch_update_next_tn<128>(c, dr);
+  else tc_launch_update_next_tn<64>(c, dr);
 }
 
 // Tile width: forced by PRSGD_OPT_UPDATE_TILE, else chosen per launch.  Wide tiles need fewer TMA

@@ -328,7 +328,7 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging, bool more_follow) {
     const bool fuse_l = fuse && tc_layer_fuses_average(c, l);
     prof_begin(c, fuse_l ? PRSGD_KERNEL_UPDATE_AVERAGE : PRSGD_KERNEL_UPDATE);
     if (l == 1 && next_fwd) {
-      tc_launch_update_next(c, dr, false);
+      tc_launch_update_next(c, dr);
       c->a1_ready = true;
     } else {
       tc_launch_update(c, l, dr, act_mask, fuse_l);
