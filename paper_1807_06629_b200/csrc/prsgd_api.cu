@@ -310,30 +310,30 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging, bool more_follow) {
     launch_pdl(softmax_ce_kernel, dim3(N, (c->B + 7) / 8), dim3(256), 0, c->stream, a);
     LAUNCH_CHECK(c);
   }
-  // Layers >= 2 on a plain SGD iteration: one launch forms dZ_{l-1} and applies the step of W_l (the fused
-  // update + average of an averaging iteration owns a tile across workers instead and keeps dX separate).
-  const bool dx_in_upd = c->dx_in_update && !fuse && act_mask == nullptr && c->velocity == nullptr && tc_epilogues_fused(c);
+  // Layers >= 2 whose update is the plain SGD step: one launch forms dZ_{l-1} and applies the step of W_l (the
+  // fused update + average of an averaging iteration owns a tile across workers instead and keeps dX separate).
+  const bool dx_in_upd = c->dx_in_update && act_mask == nullptr && c->velocity == nullptr && tc_epilogues_fused(c);
   for (int l = L; l >= 1; --l) {          // dX_l reads W_l before the update of layer l overwrites it
-    if (l > 1 && dx_in_upd && (c->dx_in_update == 2 || tc_layer_folds_dx(c, l))) {
+    const bool fuse_l = fuse && tc_layer_fuses_average(c, l);
+    if (l > 1 && dx_in_upd && !fuse_l && (c->dx_in_update == 2 || tc_layer_folds_dx(c, l))) {
       prof_begin(c, PRSGD_KERNEL_UPDATE);
       tc_launch_update_dx(c, l);
       LAUNCH_CHECK(c);
-      continue;
-    }
-    if (l > 1) {
-      prof_begin(c, PRSGD_KERNEL_DX);
-      tc_launch_dx(c, l, dr, act_mask);
+    } else {
+      if (l > 1) {
+        prof_begin(c, PRSGD_KERNEL_DX);
+        tc_launch_dx(c, l, dr, act_mask);
+        LAUNCH_CHECK(c);
+      }
+      prof_begin(c, fuse_l ? PRSGD_KERNEL_UPDATE_AVERAGE : PRSGD_KERNEL_UPDATE);
+      if (l == 1 && next_fwd) {
+        tc_launch_update_next(c, dr);
+        c->a1_ready = true;
+      } else {
+        tc_launch_update(c, l, dr, act_mask, fuse_l);
+      }
       LAUNCH_CHECK(c);
     }
-    const bool fuse_l = fuse && tc_layer_fuses_average(c, l);
-    prof_begin(c, fuse_l ? PRSGD_KERNEL_UPDATE_AVERAGE : PRSGD_KERNEL_UPDATE);
-    if (l == 1 && next_fwd) {
-      tc_launch_update_next(c, dr);
-      c->a1_ready = true;
-    } else {
-      tc_launch_update(c, l, dr, act_mask, fuse_l);
-    }
-    LAUNCH_CHECK(c);
     if (fuse && !fuse_l) {
       prof_begin(c, PRSGD_KERNEL_AVERAGE);
       tc_launch_weight_average(c, l);
