@@ -978,15 +978,19 @@ int prsgd_average_rows(float* d_P, int64_t N, int64_t m, int64_t row_stride, voi
   if (!aligned(d_P, 16) || (row_stride % 4) != 0)
     return fail(nullptr, PRSGD_ERR_ALIGN, "d_P must be 16-byte aligned and row_stride a multiple of 4");
   if (m == 0) return PRSGD_OK;
+  // Launched as a programmatic dependent: its blocks may become resident while the kernel before it in
+  // the stream drains (they touch no memory before griddepcontrol.wait), which hides the launch latency
+  // of back-to-back calls on short rows.
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   if (m < kAvgNarrowLaneBelow) {
     const int64_t threads = m / 2 + (m & 1);
-    average_rows_kernel<0, false, 2><<<grid1d(threads, 256), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
-        d_P, N, m, row_stride, nullptr, nullptr);
+    launch_pdl(average_rows_kernel<0, false, 2>, grid1d(threads, 256), dim3(256), 0, st, d_P, N, m, row_stride,
+               (float*)nullptr, (uint16_t*)nullptr, (const DeviceStatus*)nullptr);
   } else {
     const int64_t threads = m / 4 + (m & 3);
     if ((threads + 255) / 256 > 0x7fffffffll) return fail(nullptr, PRSGD_ERR_SIZE, "m too large");
-    average_rows_kernel<0, false><<<grid1d(threads, 256), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
-        d_P, N, m, row_stride, nullptr, nullptr);
+    launch_pdl(average_rows_kernel<0, false>, grid1d(threads, 256), dim3(256), 0, st, d_P, N, m, row_stride,
+               (float*)nullptr, (uint16_t*)nullptr, (const DeviceStatus*)nullptr);
   }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return fail(nullptr, PRSGD_ERR_CUDA, std::string("average_rows: ") + cudaGetErrorString(e));
