@@ -424,9 +424,9 @@ def main():
     p.set_option(binding.OPT_PROFILE, 0)
     L = len(w.dims) - 1
     # iterations 1..I-1 of a period run layer 1's update with the next forward folded in (tensor-core path)
-    next_fwd = (w.precision == 1 and L > 1 and w.I > 1 and w.dims[L] <= 128 and args.momentum is None
+    next_fwd = (w.precision == 1 and L > 1 and w.I > 1 and w.dims[L] <= 128
                 and not args.no_next_forward and not args.no_fused_epilogues)
-    dx_in_upd = (w.precision == 1 and w.dims[L] <= 128 and args.momentum is None and not args.no_dx_in_update
+    dx_in_upd = (w.precision == 1 and w.dims[L] <= 128 and not args.no_dx_in_update
                  and not args.no_fused_epilogues)
     bytes_iter = algorithmic_bytes(w, p.m_pad, args.momentum is not None, next_fwd, dx_in_upd,
                                    torch.cuda.get_device_properties(dev).multi_processor_count)

@@ -705,6 +705,17 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
   if (warp == 1) tmem_dealloc(tmem, 256u);
 }
 
+// v <- mu v + G on two neighbouring 16-byte chunks (j, j + 1) of a 128-byte-swizzled fp32 row of the momentum
+// tile, in place; G is replaced by the new v, which the caller then applies as the step direction.
+__device__ __forceinline__ void momentum_pair(uint8_t* vrow, uint32_t j, uint32_t sw, float mu, float4& gx, float4& gy) {
+  float4* q0 = reinterpret_cast<float4*>(vrow + ((j ^ sw) << 4));
+  float4* q1 = reinterpret_cast<float4*>(vrow + (((j + 1u) ^ sw) << 4));
+  const float4 v0 = *q0, v1 = *q1;
+  gx.x = fmaf(mu, v0.x, gx.x); gx.y = fmaf(mu, v0.y, gx.y); gx.z = fmaf(mu, v0.z, gx.z); gx.w = fmaf(mu, v0.w, gx.w);
+  gy.x = fmaf(mu, v1.x, gy.x); gy.y = fmaf(mu, v1.y, gy.y); gy.z = fmaf(mu, v1.z, gy.z); gy.w = fmaf(mu, v1.w, gy.w);
+  *q0 = gx; *q1 = gy;
+}
+
 // ---------------------------------------------------------------------------------------------
 // update of layer 1 with the next iteration's first forward GEMM folded in
 // ---------------------------------------------------------------------------------------------
@@ -728,15 +739,17 @@ struct UpdateNextArgs {
   const float* bias;         // params + b_off of layer 1 (already stepped by this iteration's dX epilogue)
   int64_t bias_stride;
   int M_total;               // d_1
+  float mu;                  // momentum form: v <- mu v + G, x <- x - gamma v
 };
 
-template <int TN> struct UpdNextCfg {
+template <int TN, bool MOM> struct UpdNextCfg {
   static constexpr uint32_t kMaster = 128u * TN * 4u;
+  static constexpr uint32_t kVel = MOM ? kMaster : 0u;          // momentum tile right after the master tile
   static constexpr uint32_t kOut = 128u * TN * 2u;
   __host__ __device__ static uint32_t ops_bytes(int B) { return (uint32_t)(2 + TN / 64) * (uint32_t)B * 128u; }
   __host__ __device__ static uint32_t region(int B) { return ops_bytes(B) > kOut ? ops_bytes(B) : kOut; }
   __host__ __device__ static uint32_t next_bytes(int B) { return (uint32_t)(TN / 64) * (uint32_t)B * 128u; }
-  __host__ __device__ static uint32_t stage(int B) { return kMaster + region(B) + next_bytes(B); }
+  __host__ __device__ static uint32_t stage(int B) { return kMaster + kVel + region(B) + next_bytes(B); }
   static int stages(int B) {
     int s = (int)((227u * 1024u - 2048u) / stage(B));
     return s > 4 ? 4 : s;
@@ -744,13 +757,14 @@ template <int TN> struct UpdNextCfg {
   static size_t smem(int B) { return (size_t)stages(B) * stage(B) + 1024 + 512; }
 };
 
-template <int TN>
+template <int TN, bool MOM>
 __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_next_kernel(const __grid_constant__ CUtensorMap mapDelta,
                                                                         const __grid_constant__ CUtensorMap mapPool,
                                                                         const __grid_constant__ CUtensorMap mapMaster,
+                                                                        const __grid_constant__ CUtensorMap mapVel,
                                                                         const UpdateNextArgs a) {
   using namespace ptx;
-  using Cfg = UpdNextCfg<TN>;
+  using Cfg = UpdNextCfg<TN, MOM>;
   constexpr int NB32 = TN / 32, NB64 = TN / 64;
   constexpr uint32_t kFwdCol = 256u;                    // TMEM: dW accumulators in columns [0, 256), forward ones behind
   extern __shared__ uint8_t smem_raw[];
@@ -761,8 +775,9 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_next_kernel(const __
   const uint32_t stage_bytes = Cfg::stage(a.B);
   const uint32_t op_box = (uint32_t)a.B * 128u;         // one {64, B} box
   auto master_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes; };
-  auto ops_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes + Cfg::kMaster; };
-  auto next_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes + Cfg::kMaster + Cfg::region(a.B); };
+  auto vel_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes + Cfg::kMaster; };
+  auto ops_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes + Cfg::kMaster + Cfg::kVel; };
+  auto next_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes + Cfg::kMaster + Cfg::kVel + Cfg::region(a.B); };
   const uint32_t bar0 = base + (uint32_t)S * stage_bytes;
   auto full_ops = [&](int s) { return bar0 + 8u * s; };
   auto full_w = [&](int s) { return bar0 + 32u + 8u * s; };
@@ -790,6 +805,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_next_kernel(const __
     fence_mbar_init();
     prefetch_tensormap(&mapDelta); prefetch_tensormap(&mapPool);
     prefetch_tensormap(&mapMaster);
+    if (MOM) prefetch_tensormap(&mapVel);
   }
   if (warp == 1) { tmem_alloc(smem_u32(tmem_slot), 512u); tmem_relinquish(); }
   tc_fence_before();
@@ -826,9 +842,13 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_next_kernel(const __
           tma_load_3d(ops + (2u + h) * op_box, &mapPool, full_ops(s), n0 + 64 * h, row0, n);
           tma_load_3d(nx + h * op_box, &mapPool, full_ops(s), n0 + 64 * h, row1, n);
         }
-        mbar_expect_tx(full_w(s), Cfg::kMaster);
+        mbar_expect_tx(full_w(s), Cfg::kMaster + Cfg::kVel);
 #pragma unroll
         for (int q = 0; q < NB32; ++q) tma_load_3d(master_u32(s) + q * 16384u, &mapMaster, full_w(s), n0 + 32 * q, m0, n);
+        if (MOM) {
+#pragma unroll
+          for (int q = 0; q < NB32; ++q) tma_load_3d(vel_u32(s) + q * 16384u, &mapVel, full_w(s), n0 + 32 * q, m0, n);
+        }
       }
     }
     if (*abort_flag && it > 0) {   // let the copies already in flight land before the CTA goes away
@@ -900,6 +920,10 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_next_kernel(const __
         if (!ok) break;
 #pragma unroll
         for (int q = 0; q < NB32; ++q) tma_store_3d(&mapMaster, master_u32(s) + q * 16384u, n0 + 32 * q, m0, n);
+        if (MOM) {
+#pragma unroll
+          for (int q = 0; q < NB32; ++q) tma_store_3d(&mapVel, vel_u32(s) + q * 16384u, n0 + 32 * q, m0, n);
+        }
         tma_commit_group();
         tma_wait_group_read0();
         ok = mbar_wait(fwd_done(s), ph, abort_flag, a.status, 0x407);
@@ -929,7 +953,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_next_kernel(const __
         if (!ok) break;
         tc_fence_after();
         uint8_t* mst = gen + (size_t)s * stage_bytes;
-        uint8_t* stg = mst + Cfg::kMaster;
+        uint8_t* stg = mst + Cfg::kMaster + Cfg::kVel;
 #pragma unroll
         for (int c = 0; c < NB32; ++c) {
           uint32_t v[32];
@@ -940,14 +964,15 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_next_kernel(const __
             float4* p0 = reinterpret_cast<float4*>(mst + c * 16384 + row_off + (((uint32_t)(2 * jp) ^ sw) << 4));
             float4* p1 = reinterpret_cast<float4*>(mst + c * 16384 + row_off + (((uint32_t)(2 * jp + 1) ^ sw) << 4));
             float4 x = *p0, y = *p1;
-            x.x = fmaf(-a.gamma, __uint_as_float(v[8 * jp + 0]), x.x);
-            x.y = fmaf(-a.gamma, __uint_as_float(v[8 * jp + 1]), x.y);
-            x.z = fmaf(-a.gamma, __uint_as_float(v[8 * jp + 2]), x.z);
-            x.w = fmaf(-a.gamma, __uint_as_float(v[8 * jp + 3]), x.w);
-            y.x = fmaf(-a.gamma, __uint_as_float(v[8 * jp + 4]), y.x);
-            y.y = fmaf(-a.gamma, __uint_as_float(v[8 * jp + 5]), y.y);
-            y.z = fmaf(-a.gamma, __uint_as_float(v[8 * jp + 6]), y.z);
-            y.w = fmaf(-a.gamma, __uint_as_float(v[8 * jp + 7]), y.w);
+            float4 gx = make_float4(__uint_as_float(v[8 * jp + 0]), __uint_as_float(v[8 * jp + 1]),
+                                    __uint_as_float(v[8 * jp + 2]), __uint_as_float(v[8 * jp + 3]));
+            float4 gy = make_float4(__uint_as_float(v[8 * jp + 4]), __uint_as_float(v[8 * jp + 5]),
+                                    __uint_as_float(v[8 * jp + 6]), __uint_as_float(v[8 * jp + 7]));
+            if (MOM) momentum_pair(mst + Cfg::kMaster + c * 16384 + row_off, (uint32_t)(2 * jp), sw, a.mu, gx, gy);
+            x.x = fmaf(-a.gamma, gx.x, x.x); x.y = fmaf(-a.gamma, gx.y, x.y);
+            x.z = fmaf(-a.gamma, gx.z, x.z); x.w = fmaf(-a.gamma, gx.w, x.w);
+            y.x = fmaf(-a.gamma, gy.x, y.x); y.y = fmaf(-a.gamma, gy.y, y.y);
+            y.z = fmaf(-a.gamma, gy.z, y.z); y.w = fmaf(-a.gamma, gy.w, y.w);
             *p0 = x; *p1 = y;
             const uint32_t chunk = (uint32_t)((c & 1) * 4 + jp);
             *reinterpret_cast<uint4*>(stg + (c >> 1) * 16384 + row_off + ((chunk ^ sw) << 4)) =
@@ -1012,14 +1037,17 @@ struct UpdateDxArgs {
   int M_total;               // d_{l-1}
   float* bias_rw;            // params + b_off of layer l-1 (worker stride bias_stride), or nullptr
   int64_t bias_stride;
+  float mu;                  // momentum form: v <- mu v + G, x <- x - gamma v
+  float* bias_vel;           // momentum segment of b_{l-1}, or nullptr
 };
 
-struct UpdDxCfg {
+template <bool MOM> struct UpdDxCfg {
   static constexpr uint32_t kMaster = 128u * 64u * 4u;     // fp32 master tile
+  static constexpr uint32_t kVel = MOM ? kMaster : 0u;     // fp32 momentum tile right behind it
   static constexpr uint32_t kOld = 128u * 64u * 2u;        // bf16 of the weights before the step
   static constexpr uint32_t kNew = 128u * 64u * 2u;        // first the a_{l-1} box, then bf16 of the stepped weights
   __host__ __device__ static uint32_t delta_bytes(int B) { return 2u * (uint32_t)B * 128u; }
-  __host__ __device__ static uint32_t stage(int B) { return kMaster + kOld + kNew + delta_bytes(B); }
+  __host__ __device__ static uint32_t stage(int B) { return kMaster + kVel + kOld + kNew + delta_bytes(B); }
   static int stages(int B) {
     int s = (int)((227u * 1024u - 2048u) / stage(B));
     return s > 4 ? 4 : s;
@@ -1027,13 +1055,15 @@ struct UpdDxCfg {
   static size_t smem(int B) { return (size_t)stages(B) * stage(B) + 1024 + 512; }
 };
 
+template <bool MOM>
 __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_dx_kernel(const __grid_constant__ CUtensorMap mapDelta,
                                                                       const __grid_constant__ CUtensorMap mapAct,
                                                                       const __grid_constant__ CUtensorMap mapMaster,
                                                                       const __grid_constant__ CUtensorMap mapShadow,
+                                                                      const __grid_constant__ CUtensorMap mapVel,
                                                                       const UpdateDxArgs a) {
   using namespace ptx;
-  using Cfg = UpdDxCfg;
+  using Cfg = UpdDxCfg<MOM>;
   constexpr int TN = 64;
   constexpr uint32_t kDxCol = 256u;                     // TMEM: dW accumulators in columns [0, 256), dX ones behind
   extern __shared__ uint8_t smem_raw[];
@@ -1044,9 +1074,10 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_dx_kernel(const __gr
   const uint32_t stage_bytes = Cfg::stage(a.B);
   const uint32_t op_box = (uint32_t)a.B * 128u;         // one {64, B} box
   auto master_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes; };
-  auto old_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes + Cfg::kMaster; };
-  auto new_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes + Cfg::kMaster + Cfg::kOld; };
-  auto delta_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes + Cfg::kMaster + Cfg::kOld + Cfg::kNew; };
+  auto vel_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes + Cfg::kMaster; };
+  auto old_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes + Cfg::kMaster + Cfg::kVel; };
+  auto new_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes + Cfg::kMaster + Cfg::kVel + Cfg::kOld; };
+  auto delta_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes + Cfg::kMaster + Cfg::kVel + Cfg::kOld + Cfg::kNew; };
   const uint32_t bar0 = base + (uint32_t)S * stage_bytes;
   auto full_ops = [&](int s) { return bar0 + 8u * s; };
   auto full_w = [&](int s) { return bar0 + 32u + 8u * s; };
@@ -1074,6 +1105,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_dx_kernel(const __gr
     fence_mbar_init();
     prefetch_tensormap(&mapDelta); prefetch_tensormap(&mapAct);
     prefetch_tensormap(&mapMaster); prefetch_tensormap(&mapShadow);
+    if (MOM) prefetch_tensormap(&mapVel);
   }
   if (warp == 1) { tmem_alloc(smem_u32(tmem_slot), 512u); tmem_relinquish(); }
   tc_fence_before();
@@ -1102,9 +1134,13 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_dx_kernel(const __gr
         tma_load_3d(delta_u32(s), &mapDelta, full_ops(s), m0, 0, n);
         tma_load_3d(delta_u32(s) + op_box, &mapDelta, full_ops(s), m0 + 64, 0, n);
         tma_load_3d(new_u32(s), &mapAct, full_ops(s), n0, 0, n);
-        mbar_expect_tx(full_w(s), Cfg::kMaster);
+        mbar_expect_tx(full_w(s), Cfg::kMaster + Cfg::kVel);
         tma_load_3d(master_u32(s), &mapMaster, full_w(s), n0, m0, n);
         tma_load_3d(master_u32(s) + 16384u, &mapMaster, full_w(s), n0 + 32, m0, n);
+        if (MOM) {
+          tma_load_3d(vel_u32(s), &mapVel, full_w(s), n0, m0, n);
+          tma_load_3d(vel_u32(s) + 16384u, &mapVel, full_w(s), n0 + 32, m0, n);
+        }
       }
     }
     if (*abort_flag && it > 0) {   // let the copies already in flight land before the CTA goes away
@@ -1175,6 +1211,10 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_dx_kernel(const __gr
         if (!ok) break;
         tma_store_3d(&mapMaster, master_u32(s), n0, m0, n);
         tma_store_3d(&mapMaster, master_u32(s) + 16384u, n0 + 32, m0, n);
+        if (MOM) {
+          tma_store_3d(&mapVel, vel_u32(s), n0, m0, n);
+          tma_store_3d(&mapVel, vel_u32(s) + 16384u, n0 + 32, m0, n);
+        }
         tma_store_3d(&mapShadow, new_u32(s), n0, m0, n);
         tma_commit_group();
         tma_wait_group_read0();
@@ -1205,7 +1245,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_dx_kernel(const __gr
         if (!ok) break;
         tc_fence_after();
         uint8_t* mst = gen + (size_t)s * stage_bytes;
-        uint8_t* old = mst + Cfg::kMaster;
+        uint8_t* old = mst + Cfg::kMaster + Cfg::kVel;
         uint8_t* stg = old + Cfg::kOld;
 #pragma unroll
         for (int c = 0; c < 2; ++c) {
@@ -1220,14 +1260,15 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_dx_kernel(const __gr
             const uint32_t boff = row_off + (((uint32_t)(c * 4 + jp) ^ sw) << 4);
             *reinterpret_cast<uint4*>(old + boff) = make_uint4(pack_bf16x2(x.x, x.y), pack_bf16x2(x.z, x.w),
                                                                pack_bf16x2(y.x, y.y), pack_bf16x2(y.z, y.w));
-            x.x = fmaf(-a.gamma, __uint_as_float(v[8 * jp + 0]), x.x);
-            x.y = fmaf(-a.gamma, __uint_as_float(v[8 * jp + 1]), x.y);
-            x.z = fmaf(-a.gamma, __uint_as_float(v[8 * jp + 2]), x.z);
-            x.w = fmaf(-a.gamma, __uint_as_float(v[8 * jp + 3]), x.w);
-            y.x = fmaf(-a.gamma, __uint_as_float(v[8 * jp + 4]), y.x);
-            y.y = fmaf(-a.gamma, __uint_as_float(v[8 * jp + 5]), y.y);
-            y.z = fmaf(-a.gamma, __uint_as_float(v[8 * jp + 6]), y.z);
-            y.w = fmaf(-a.gamma, __uint_as_float(v[8 * jp + 7]), y.w);
+            float4 gx = make_float4(__uint_as_float(v[8 * jp + 0]), __uint_as_float(v[8 * jp + 1]),
+                                    __uint_as_float(v[8 * jp + 2]), __uint_as_float(v[8 * jp + 3]));
+            float4 gy = make_float4(__uint_as_float(v[8 * jp + 4]), __uint_as_float(v[8 * jp + 5]),
+                                    __uint_as_float(v[8 * jp + 6]), __uint_as_float(v[8 * jp + 7]));
+            if (MOM) momentum_pair(mst + Cfg::kMaster + c * 16384 + row_off, (uint32_t)(2 * jp), sw, a.mu, gx, gy);
+            x.x = fmaf(-a.gamma, gx.x, x.x); x.y = fmaf(-a.gamma, gx.y, x.y);
+            x.z = fmaf(-a.gamma, gx.z, x.z); x.w = fmaf(-a.gamma, gx.w, x.w);
+            y.x = fmaf(-a.gamma, gy.x, y.x); y.y = fmaf(-a.gamma, gy.y, y.y);
+            y.z = fmaf(-a.gamma, gy.z, y.z); y.w = fmaf(-a.gamma, gy.w, y.w);
             *p0 = x; *p1 = y;
             *reinterpret_cast<uint4*>(stg + boff) = make_uint4(pack_bf16x2(x.x, x.y), pack_bf16x2(x.z, x.w),
                                                                pack_bf16x2(y.x, y.y), pack_bf16x2(y.z, y.w));
@@ -1273,6 +1314,11 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_dx_kernel(const __gr
       mbar_arrive(dacc_empty(q));
       if (valid && a.bias_rw != nullptr) {
         float* bp = a.bias_rw + (int64_t)n * a.bias_stride + cfeat;
+        if (a.bias_vel != nullptr) {                      // momentum form of the bias step
+          float* vp = a.bias_vel + (int64_t)n * a.bias_stride + cfeat;
+          gsum = fmaf(a.mu, *vp, gsum);
+          *vp = gsum;
+        }
         *bp = fmaf(-a.gamma, gsum, *bp);
       }
     }
@@ -1409,9 +1455,11 @@ inline int tc_create(prsgd_ctx* c, std::string* err) {
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<false, 128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<128, false>::smem(c->B));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<true, 128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<128, false>::smem(c->B));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<false, 64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<64, true>::smem(c->B));
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_dx_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdDxCfg::smem(c->B));
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_next_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdNextCfg<64>::smem(c->B));
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_next_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdNextCfg<128>::smem(c->B));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_dx_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdDxCfg<false>::smem(c->B));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_dx_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdDxCfg<true>::smem(c->B));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_next_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdNextCfg<64, false>::smem(c->B));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_next_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdNextCfg<128, false>::smem(c->B));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_next_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdNextCfg<64, true>::smem(c->B));
   if (e != cudaSuccess) {
     *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e);
     delete st;
@@ -1534,49 +1582,60 @@ inline bool tc_layer_folds_dx(const prsgd_ctx* c, int l) {
 }
 
 // Update of layer l >= 2 that also forms dZ_{l-1} (tc_update_dx_kernel): replaces dX_l + update_l.
-inline void tc_launch_update_dx(prsgd_ctx* c, int l) {
+template <bool MOM>
+inline void tc_launch_update_dx_m(prsgd_ctx* c, int l) {
   TcState* st = static_cast<TcState*>(c->tc);
   const Layer& ly = c->layer[l - 1];
   UpdateDxArgs a{};
   a.B = c->B; a.N = c->N; a.tiles_m = (ly.d_out + 127) / 128; a.tiles_n = (ly.d_in + 63) / 64;
-  a.gamma = c->gamma; a.status = c->status; a.stages = UpdDxCfg::stages(c->B);
+  a.gamma = c->gamma; a.status = c->status; a.stages = UpdDxCfg<MOM>::stages(c->B);
   a.out_bk = c->buf.delta_bk[l - 1]; a.mask_src = c->buf.act_bk[l - 1]; a.ld_out = c->buf.ld[l - 1]; a.M_total = ly.d_in;
   a.bias_rw = c->params + c->layer[l - 2].b_off; a.bias_stride = c->m_pad;
+  a.mu = c->mu; a.bias_vel = MOM ? c->velocity + c->layer[l - 2].b_off : nullptr;
   const int items = a.tiles_n * c->N;
   const int grid = items < st->num_sms ? items : st->num_sms;
   const TcLayerMaps& mp = st->layer[l - 1];
-  launch_pdl(tc_update_dx_kernel, dim3(grid), kUpdThreads, UpdDxCfg::smem(c->B), c->stream, mp.delta_out, mp.act_in, mp.master,
-             mp.shadow_k, a);
+  launch_pdl(tc_update_dx_kernel<MOM>, dim3(grid), kUpdThreads, UpdDxCfg<MOM>::smem(c->B), c->stream, mp.delta_out, mp.act_in,
+             mp.master, mp.shadow_k, MOM ? mp.velocity : mp.master, a);
+}
+
+inline void tc_launch_update_dx(prsgd_ctx* c, int l) {
+  if (c->velocity != nullptr) tc_launch_update_dx_m<true>(c, l);
+  else tc_launch_update_dx_m<false>(c, l);
 }
 
 // Update of layer 1 that also forms a_1 of the next iteration (tc_update_next_kernel).
-template <int TN>
+template <int TN, bool MOM>
 inline void tc_launch_update_next_tn(prsgd_ctx* c, const DrawArgs& dr) {
   TcState* st = static_cast<TcState*>(c->tc);
   const Layer& ly = c->layer[0];
   UpdateNextArgs a{};
   a.B = c->B; a.N = c->N; a.tiles_m = (ly.d_out + 127) / 128; a.tiles_n = (ly.d_in + TN - 1) / TN;
-  a.gamma = c->gamma; a.draw = dr; a.status = c->status;
-  a.stages = UpdNextCfg<TN>::stages(c->B);
+  a.gamma = c->gamma; a.mu = c->mu; a.draw = dr; a.status = c->status;
+  a.stages = UpdNextCfg<TN, MOM>::stages(c->B);
   a.next_out = c->buf.act_bk[1]; a.next_ld = c->buf.ld[1];
   a.bias = c->params + ly.b_off; a.bias_stride = c->m_pad; a.M_total = ly.d_out;
   const int items = a.tiles_m * c->N;
   const int grid = items < st->num_sms ? items : st->num_sms;
   const TcLayerMaps& mp = st->layer[0];
-  launch_pdl(tc_update_next_kernel<TN>, dim3(grid), kUpdThreads, UpdNextCfg<TN>::smem(c->B), c->stream, mp.delta_out, mp.act_in,
-             mp.master, a);
+  launch_pdl(tc_update_next_kernel<TN, MOM>, dim3(grid), kUpdThreads, UpdNextCfg<TN, MOM>::smem(c->B), c->stream, mp.delta_out,
+             mp.act_in, mp.master, MOM ? mp.velocity : mp.master, a);
 }
 
 inline void tc_launch_update_next(prsgd_ctx* c, const DrawArgs& dr) {
   const TcState* st = static_cast<const TcState*>(c->tc);
   const Layer& ly = c->layer[0];
+  if (c->velocity != nullptr) {            // momentum step: 64-wide tiles (two stages of master + momentum tiles)
+    tc_launch_update_next_tn<64, true>(c, dr);
+    return;
+  }
   int tile = c->upd_tile;
   if (tile == 0) {
     const int64_t tiles128 = (int64_t)((ly.d_out + 127) / 128) * ((ly.d_in + 127) / 128);
     tile = (c->B <= 32 && tiles128 * c->N >= 32 * (int64_t)st->num_sms) ? 128 : 64;
   }
-  if (tile == 128) tc_launch_update_next_tn<128>(c, dr);
-  else tc_launch_update_next_tn<64>(c, dr);
+  if (tile == 128) tc_launch_update_next_tn<128, false>(c, dr);
+  else tc_launch_update_next_tn<64, false>(c, dr);
 }
 
 // Tile width: forced by PRSGD_OPT_UPDATE_TILE, else chosen per launch.  Wide tiles need fewer TMA

@@ -220,6 +220,32 @@ def test_dx_folded_into_the_update_changes_no_bit(torch_cuda):
         assert outs[1][2] < outs[0][2]
 
 
+@pytest.mark.parametrize("avg_v", [False, True])
+def test_folded_kernels_with_momentum_change_no_bit(torch_cuda, avg_v):
+    """The momentum step inside the two folded update kernels (dZ of the layer below, next forward of layer 1)
+    against the separate launches: identical parameters, momentum buffers and losses across averages."""
+    torch = torch_cuda
+    from paper_1807_06629_b200 import binding
+    for w in (SMALL[1], SMALL[3], SMALL[4], SMALL[6], _w("tc-wide-hidden", 3, (64, 448, 320, 10), 16, I=4)):
+        X, Y, x0 = make_inputs(w)
+        outs = []
+        for dxu, nxt, graph in ((0, 0, 0), (2, 1, 0), (2, 0, 1), (0, 1, 1)):
+            with torch.cuda.stream(torch.cuda.Stream()):
+                p = make_ctx(w, X, Y, x0)
+                p.enable_momentum(0.9, average_velocity=avg_v)
+                p.set_option(binding.OPT_DX_IN_UPDATE, dxu)
+                p.set_option(binding.OPT_NEXT_FORWARD, nxt)
+                p.set_option(binding.OPT_GRAPH, graph)
+                p.local_steps(2)
+                p.local_steps(2 * w.I + 1)
+                outs.append((p.get_params_stacked(), p.get_velocity_stacked(), p.get_losses()))
+                torch.cuda.current_stream().synchronize()
+        for o in outs[1:]:
+            assert np.array_equal(outs[0][0], o[0]), w.name
+            assert np.array_equal(outs[0][1], o[1]), w.name
+            assert np.array_equal(outs[0][2], o[2])
+
+
 def _segments(dims):
     """[(is_weight, start, stop)] of a canonical parameter vector."""
     out, off = [], 0
