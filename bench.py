@@ -108,7 +108,7 @@ class ClockSampler:
 # capture summarised in profiles/; valid only while the kernel's source section is unchanged.
 NCU_TRAFFIC = {
     ("cfg4", "update"): {"bytes_per_iteration": 2.229e9 + 2.795e9, "launches_per_iteration": 4,   # read + written, four launches
-                         "kernel_sha256": "eb4fe72e64d1d896b4655458366723239d4647bb81c69bf5fc9082c9e5018fa9"},
+                         "kernel_sha256": "b9fc54fcc8ad427eb76bce90a245d12a1202090221ca892906cdf33294b529ae"},
 }
 
 
