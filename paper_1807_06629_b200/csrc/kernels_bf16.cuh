@@ -1041,21 +1041,33 @@ struct UpdateDxArgs {
   float* bias_vel;           // momentum segment of b_{l-1}, or nullptr
 };
 
-template <bool MOM> struct UpdDxCfg {
-  static constexpr uint32_t kMaster = 128u * 64u * 4u;     // fp32 master tile
+// TN = 64: every stage holds fp32 master | momentum | bf16 old | bf16 new (first the a_{l-1} box) | two dZ_l boxes.
+// TN = 128 (512-byte rows, which the memory system serves ~7 % faster than 256-byte ones): the two bf16 tiles
+// do not fit twice, so only master | dZ_l boxes | a_{l-1} boxes are staged (two stages) and ONE pair of bf16
+// tiles behind the stages is shared: the epilogue of a tile waits until the pair of the tile before it has been
+// read by its TMA store and its dX MMAs.  No momentum form at this width.
+template <int TN, bool MOM> struct UpdDxCfg {
+  static_assert(TN == 64 || !MOM, "the momentum form uses 64-wide tiles");
+  static constexpr bool kSharedPair = TN == 128;
+  static constexpr uint32_t kMaster = 128u * TN * 4u;      // fp32 master tile
   static constexpr uint32_t kVel = MOM ? kMaster : 0u;     // fp32 momentum tile right behind it
-  static constexpr uint32_t kOld = 128u * 64u * 2u;        // bf16 of the weights before the step
-  static constexpr uint32_t kNew = 128u * 64u * 2u;        // first the a_{l-1} box, then bf16 of the stepped weights
+  static constexpr uint32_t kOld = 128u * TN * 2u;         // bf16 of the weights before the step
+  static constexpr uint32_t kNew = 128u * TN * 2u;         // bf16 of the stepped weights
   __host__ __device__ static uint32_t delta_bytes(int B) { return 2u * (uint32_t)B * 128u; }
-  __host__ __device__ static uint32_t stage(int B) { return kMaster + kVel + kOld + kNew + delta_bytes(B); }
+  __host__ __device__ static uint32_t act_bytes(int B) { return (uint32_t)(TN / 64) * (uint32_t)B * 128u; }
+  __host__ __device__ static uint32_t stage(int B) {
+    return kSharedPair ? kMaster + delta_bytes(B) + act_bytes(B) : kMaster + kVel + kOld + kNew + delta_bytes(B);
+  }
+  __host__ __device__ static uint32_t shared_bytes() { return kSharedPair ? kOld + kNew : 0u; }
   static int stages(int B) {
+    if (kSharedPair) return (2u * stage(B) + shared_bytes() + 2048u <= 227u * 1024u) ? 2 : 0;
     int s = (int)((227u * 1024u - 2048u) / stage(B));
     return s > 4 ? 4 : s;
   }
-  static size_t smem(int B) { return (size_t)stages(B) * stage(B) + 1024 + 512; }
+  static size_t smem(int B) { return (size_t)stages(B) * stage(B) + shared_bytes() + 1024 + 512; }
 };
 
-template <bool MOM>
+template <int TN, bool MOM>
 __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_dx_kernel(const __grid_constant__ CUtensorMap mapDelta,
                                                                       const __grid_constant__ CUtensorMap mapAct,
                                                                       const __grid_constant__ CUtensorMap mapMaster,
@@ -1063,8 +1075,9 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_dx_kernel(const __gr
                                                                       const __grid_constant__ CUtensorMap mapVel,
                                                                       const UpdateDxArgs a) {
   using namespace ptx;
-  using Cfg = UpdDxCfg<MOM>;
-  constexpr int TN = 64;
+  using Cfg = UpdDxCfg<TN, MOM>;
+  constexpr int NB32 = TN / 32, NB64 = TN / 64;
+  constexpr bool kSharedPair = Cfg::kSharedPair;
   constexpr uint32_t kDxCol = 256u;                     // TMEM: dW accumulators in columns [0, 256), dX ones behind
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -1075,10 +1088,14 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_dx_kernel(const __gr
   const uint32_t op_box = (uint32_t)a.B * 128u;         // one {64, B} box
   auto master_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes; };
   auto vel_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes + Cfg::kMaster; };
-  auto old_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes + Cfg::kMaster + Cfg::kVel; };
-  auto new_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes + Cfg::kMaster + Cfg::kVel + Cfg::kOld; };
-  auto delta_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes + Cfg::kMaster + Cfg::kVel + Cfg::kOld + Cfg::kNew; };
-  const uint32_t bar0 = base + (uint32_t)S * stage_bytes;
+  const uint32_t pair0 = base + (uint32_t)S * stage_bytes;            // the shared bf16 pair (TN = 128)
+  auto old_u32 = [&](int s) { return kSharedPair ? pair0 : base + (uint32_t)s * stage_bytes + Cfg::kMaster + Cfg::kVel; };
+  auto new_u32 = [&](int s) { return old_u32(s) + Cfg::kOld; };
+  auto delta_u32 = [&](int s) {
+    return base + (uint32_t)s * stage_bytes + (kSharedPair ? Cfg::kMaster : Cfg::kMaster + Cfg::kVel + Cfg::kOld + Cfg::kNew);
+  };
+  auto act_u32 = [&](int s) { return kSharedPair ? delta_u32(s) + 2u * op_box : new_u32(s); };
+  const uint32_t bar0 = pair0 + Cfg::shared_bytes();
   auto full_ops = [&](int s) { return bar0 + 8u * s; };
   auto full_w = [&](int s) { return bar0 + 32u + 8u * s; };
   auto stage_empty = [&](int s) { return bar0 + 64u + 8u * s; };
@@ -1088,8 +1105,10 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_dx_kernel(const __gr
   auto dx_done = [&](int s) { return bar0 + 192u + 8u * s; };       // the dX MMAs have read the stage's old tile and dZ boxes
   auto dacc_full = [&](int q) { return bar0 + 224u + 8u * q; };
   auto dacc_empty = [&](int q) { return bar0 + 240u + 8u * q; };
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen + (size_t)S * stage_bytes + 256);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + (size_t)S * stage_bytes + 260);
+  uint8_t* tail = gen + (size_t)S * stage_bytes + Cfg::shared_bytes();
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 256);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 260);
+  const uint32_t pair_free = bar0 + 264u;      // shared pair: the store of the tile's new half and its dX MMAs are done
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int col_blocks = a.tiles_n * a.N;
@@ -1101,6 +1120,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_dx_kernel(const __gr
       mbar_init(dx_done(s), 1);
     }
     for (int q = 0; q < 2; ++q) { mbar_init(dacc_full(q), 1); mbar_init(dacc_empty(q), 128); }
+    mbar_init(pair_free, 2);
     *abort_flag = *(volatile unsigned int*)&a.status->error != 0u ? 1 : 0;   // an earlier expired wait: no-op (see tc_stream_kernel)
     fence_mbar_init();
     prefetch_tensormap(&mapDelta); prefetch_tensormap(&mapAct);
@@ -1130,13 +1150,14 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_dx_kernel(const __gr
         ok = mbar_wait(stage_empty(s), ph ^ 1u, abort_flag, a.status, 0x501);
         if (!ok) break;
         const int m0 = mb * 128;
-        mbar_expect_tx(full_ops(s), 3u * op_box);
+        mbar_expect_tx(full_ops(s), (2u + NB64) * op_box);
         tma_load_3d(delta_u32(s), &mapDelta, full_ops(s), m0, 0, n);
         tma_load_3d(delta_u32(s) + op_box, &mapDelta, full_ops(s), m0 + 64, 0, n);
-        tma_load_3d(new_u32(s), &mapAct, full_ops(s), n0, 0, n);
+#pragma unroll
+        for (int h = 0; h < NB64; ++h) tma_load_3d(act_u32(s) + h * op_box, &mapAct, full_ops(s), n0 + 64 * h, 0, n);
         mbar_expect_tx(full_w(s), Cfg::kMaster + Cfg::kVel);
-        tma_load_3d(master_u32(s), &mapMaster, full_w(s), n0, m0, n);
-        tma_load_3d(master_u32(s) + 16384u, &mapMaster, full_w(s), n0 + 32, m0, n);
+#pragma unroll
+        for (int q = 0; q < NB32; ++q) tma_load_3d(master_u32(s) + q * 16384u, &mapMaster, full_w(s), n0 + 32 * q, m0, n);
         if (MOM) {
           tma_load_3d(vel_u32(s), &mapVel, full_w(s), n0, m0, n);
           tma_load_3d(vel_u32(s) + 16384u, &mapVel, full_w(s), n0 + 32, m0, n);
@@ -1172,10 +1193,11 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_dx_kernel(const __gr
       for (int h = 0; h < 2; ++h) {                       // the tile's two 64-row halves = the two dZ_l boxes
 #pragma unroll
         for (int k = 0; k < 4; ++k)
-          mma_bf16(acc, smem_desc_sw128(old_u32(s) + (uint32_t)(h * 4 + k) * 2048u, Cfg::kOld, 1024u),
+          mma_bf16(acc, smem_desc_sw128(old_u32(s) + (uint32_t)(h * 4 + k) * 2048u, 16384u, 1024u),
                    smem_desc_sw128(delta_u32(s) + h * op_box + k * 32u, 16u, 1024u), idesc_dx, (mb | h | k) != 0 ? 1u : 0u);
       }
       mma_commit(dx_done(s));
+      if (kSharedPair) mma_commit(pair_free);
       if (mb == a.tiles_m - 1) mma_commit(dacc_full(q));
       return true;
     };
@@ -1187,7 +1209,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_dx_kernel(const __gr
              mbar_wait(full_ops(s), ph, abort_flag, a.status, 0x505);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t sa = delta_u32(s), sb = new_u32(s);
+        const uint32_t sa = delta_u32(s), sb = act_u32(s);
         for (int k = 0; k < ksteps; ++k)
           mma_bf16(tmem + (uint32_t)(s * TN), smem_desc_sw128(sa + k * 2048u, op_box, 1024u),
                    smem_desc_sw128(sb + k * 2048u, op_box, 1024u), idesc_dw, k != 0 ? 1u : 0u);
@@ -1209,14 +1231,20 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_dx_kernel(const __gr
         const int m0 = mb * 128;
         ok = mbar_wait(tile_ready(s), ph, abort_flag, a.status, 0x506);
         if (!ok) break;
-        tma_store_3d(&mapMaster, master_u32(s), n0, m0, n);
-        tma_store_3d(&mapMaster, master_u32(s) + 16384u, n0 + 32, m0, n);
+#pragma unroll
+        for (int h = 0; h < NB64; ++h) tma_store_3d(&mapShadow, new_u32(s) + h * 16384u, n0 + 64 * h, m0, n);
+        if (kSharedPair) tma_commit_group();              // a group of its own: the shared pair is released first
+#pragma unroll
+        for (int q = 0; q < NB32; ++q) tma_store_3d(&mapMaster, master_u32(s) + q * 16384u, n0 + 32 * q, m0, n);
         if (MOM) {
           tma_store_3d(&mapVel, vel_u32(s), n0, m0, n);
           tma_store_3d(&mapVel, vel_u32(s) + 16384u, n0 + 32, m0, n);
         }
-        tma_store_3d(&mapShadow, new_u32(s), n0, m0, n);
         tma_commit_group();
+        if (kSharedPair) {
+          tma_wait_group_read1();
+          mbar_arrive(pair_free);
+        }
         tma_wait_group_read0();
         ok = mbar_wait(dx_done(s), ph, abort_flag, a.status, 0x507);
         if (!ok) break;
@@ -1244,11 +1272,15 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_dx_kernel(const __gr
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
+        if (kSharedPair && it > 0) {            // the one bf16 pair is free once the tile before has let go of it
+          ok = __all_sync(0xffffffffu, mbar_wait(pair_free, (it - 1) & 1u, abort_flag, a.status, 0x50B));
+          if (!ok) break;
+        }
         uint8_t* mst = gen + (size_t)s * stage_bytes;
-        uint8_t* old = mst + Cfg::kMaster + Cfg::kVel;
+        uint8_t* old = kSharedPair ? gen + (size_t)S * stage_bytes : mst + Cfg::kMaster + Cfg::kVel;
         uint8_t* stg = old + Cfg::kOld;
 #pragma unroll
-        for (int c = 0; c < 2; ++c) {
+        for (int c = 0; c < NB32; ++c) {
           uint32_t v[32];
           tmem_ld32(tmem + lane_off + (uint32_t)(s * TN + c * 32), v);
           tmem_ld_wait();
@@ -1257,7 +1289,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_dx_kernel(const __gr
             float4* p0 = reinterpret_cast<float4*>(mst + c * 16384 + row_off + (((uint32_t)(2 * jp) ^ sw) << 4));
             float4* p1 = reinterpret_cast<float4*>(mst + c * 16384 + row_off + (((uint32_t)(2 * jp + 1) ^ sw) << 4));
             float4 x = *p0, y = *p1;
-            const uint32_t boff = row_off + (((uint32_t)(c * 4 + jp) ^ sw) << 4);
+            const uint32_t boff = (uint32_t)(c >> 1) * 16384u + row_off + (((uint32_t)((c & 1) * 4 + jp) ^ sw) << 4);
             *reinterpret_cast<uint4*>(old + boff) = make_uint4(pack_bf16x2(x.x, x.y), pack_bf16x2(x.z, x.w),
                                                                pack_bf16x2(y.x, y.y), pack_bf16x2(y.z, y.w));
             float4 gx = make_float4(__uint_as_float(v[8 * jp + 0]), __uint_as_float(v[8 * jp + 1]),
@@ -1455,8 +1487,10 @@ inline int tc_create(prsgd_ctx* c, std::string* err) {
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<false, 128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<128, false>::smem(c->B));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<true, 128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<128, false>::smem(c->B));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<false, 64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<64, true>::smem(c->B));
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_dx_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdDxCfg<false>::smem(c->B));
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_dx_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdDxCfg<true>::smem(c->B));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_dx_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdDxCfg<64, false>::smem(c->B));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_dx_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdDxCfg<64, true>::smem(c->B));
+  if (e == cudaSuccess && UpdDxCfg<128, false>::stages(c->B) == 2)
+    e = cudaFuncSetAttribute(tc_update_dx_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdDxCfg<128, false>::smem(c->B));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_next_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdNextCfg<64, false>::smem(c->B));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_next_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdNextCfg<128, false>::smem(c->B));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_next_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdNextCfg<64, true>::smem(c->B));
@@ -1582,26 +1616,36 @@ inline bool tc_layer_folds_dx(const prsgd_ctx* c, int l) {
 }
 
 // Update of layer l >= 2 that also forms dZ_{l-1} (tc_update_dx_kernel): replaces dX_l + update_l.
-template <bool MOM>
+template <int TN, bool MOM>
 inline void tc_launch_update_dx_m(prsgd_ctx* c, int l) {
   TcState* st = static_cast<TcState*>(c->tc);
   const Layer& ly = c->layer[l - 1];
   UpdateDxArgs a{};
-  a.B = c->B; a.N = c->N; a.tiles_m = (ly.d_out + 127) / 128; a.tiles_n = (ly.d_in + 63) / 64;
-  a.gamma = c->gamma; a.status = c->status; a.stages = UpdDxCfg<MOM>::stages(c->B);
+  a.B = c->B; a.N = c->N; a.tiles_m = (ly.d_out + 127) / 128; a.tiles_n = (ly.d_in + TN - 1) / TN;
+  a.gamma = c->gamma; a.status = c->status; a.stages = UpdDxCfg<TN, MOM>::stages(c->B);
   a.out_bk = c->buf.delta_bk[l - 1]; a.mask_src = c->buf.act_bk[l - 1]; a.ld_out = c->buf.ld[l - 1]; a.M_total = ly.d_in;
   a.bias_rw = c->params + c->layer[l - 2].b_off; a.bias_stride = c->m_pad;
   a.mu = c->mu; a.bias_vel = MOM ? c->velocity + c->layer[l - 2].b_off : nullptr;
   const int items = a.tiles_n * c->N;
   const int grid = items < st->num_sms ? items : st->num_sms;
   const TcLayerMaps& mp = st->layer[l - 1];
-  launch_pdl(tc_update_dx_kernel<MOM>, dim3(grid), kUpdThreads, UpdDxCfg<MOM>::smem(c->B), c->stream, mp.delta_out, mp.act_in,
-             mp.master, mp.shadow_k, MOM ? mp.velocity : mp.master, a);
+  launch_pdl(tc_update_dx_kernel<TN, MOM>, dim3(grid), kUpdThreads, UpdDxCfg<TN, MOM>::smem(c->B), c->stream, mp.delta_out,
+             mp.act_in, mp.master, mp.shadow_k, MOM ? mp.velocity : mp.master, a);
 }
 
+// 128-wide column blocks when every SM has a long queue of them and the operand boxes leave room for two
+// stages (B <= 32); 64-wide ones otherwise and for the momentum form.
 inline void tc_launch_update_dx(prsgd_ctx* c, int l) {
-  if (c->velocity != nullptr) tc_launch_update_dx_m<true>(c, l);
-  else tc_launch_update_dx_m<false>(c, l);
+  if (c->velocity != nullptr) { tc_launch_update_dx_m<64, true>(c, l); return; }
+  const TcState* st = static_cast<const TcState*>(c->tc);
+  const Layer& ly = c->layer[l - 1];
+  int tile = c->upd_tile;
+  if (tile == 0) {
+    const int64_t blocks128 = (int64_t)((ly.d_in + 127) / 128) * c->N;
+    tile = (blocks128 >= 4 * (int64_t)st->num_sms && ly.d_out > 128) ? 128 : 64;
+  }
+  if (tile == 128 && UpdDxCfg<128, false>::stages(c->B) == 2) tc_launch_update_dx_m<128, false>(c, l);
+  else tc_launch_update_dx_m<64, false>(c, l);
 }
 
 // Update of layer 1 that also forms a_1 of the next iteration (tc_update_next_kernel).
