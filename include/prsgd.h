@@ -268,8 +268,8 @@ int prsgd_get_velocity_stacked(prsgd_ctx* ctx, float* dst, int dst_on_device);
  * derives from the fp32 tiles it holds, so the separate dX launch and its second read of the layer's
  * bf16 weights are saved.  1 = for layers with at least three 64-wide column blocks per SM over all
  * workers (fewer do not balance) and for single-row-tile layers, 2 = for every layer, 0 = never.  Not
- * for a layer that takes the fused update + average on an averaging iteration, nor with a worker mask.
- * Same bits as the separate launches. */
+ * for a layer that takes the fused update + average on an averaging iteration.  Same bits as the
+ * separate launches (also with momentum and with a worker mask). */
 #define PRSGD_OPT_DX_IN_UPDATE 8
 int prsgd_set_option(prsgd_ctx* ctx, int32_t option, int64_t value);
 

@@ -740,6 +740,7 @@ struct UpdateNextArgs {
   int64_t bias_stride;
   int M_total;               // d_1
   float mu;                  // momentum form: v <- mu v + G, x <- x - gamma v
+  const uint8_t* active;     // per-worker flag or nullptr: an inactive worker's row blocks are skipped
 };
 
 template <int TN, bool MOM> struct UpdNextCfg {
@@ -815,6 +816,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_next_kernel(const __
   pdl_trigger();
   const uint32_t tmem = *tmem_slot;
   const int total_rb = *abort_flag != 0 ? 0 : row_blocks;
+  auto item_active = [&](int n) { return a.active == nullptr || a.active[n] != 0; };
 
   // Every role walks the same sequence of tiles: row blocks rb = blockIdx.x, + gridDim.x, ..., and inside a
   // row block the column tiles kb = 0 .. tiles_n - 1; `it` counts tiles, tile `it` lives in stage it % S.
@@ -824,6 +826,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_next_kernel(const __
     bool ok = true;
     for (int rb = blockIdx.x; rb < total_rb && ok; rb += gridDim.x) {
       const int n = rb / a.tiles_m, m0 = (rb % a.tiles_m) * 128;
+      if (!item_active(n)) continue;
       const int64_t t = draw_t(a.draw);
       const int row0 = (int)draw_block(a.draw.seed, a.draw.worker0 + n, t, a.draw.n_blocks) * a.B;
       const int row1 = (int)draw_block(a.draw.seed, a.draw.worker0 + n, t + 1, a.draw.n_blocks) * a.B;
@@ -887,7 +890,8 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_next_kernel(const __
       if (kb == a.tiles_n - 1) mma_commit(facc_full(q));
       return true;
     };
-    for (int rb = blockIdx.x; rb < total_rb && ok; rb += gridDim.x, ++rbi) {
+    for (int rb = blockIdx.x; rb < total_rb && ok; rb += gridDim.x) {
+      if (!item_active(rb / a.tiles_m)) continue;
       for (int kb = 0; kb < a.tiles_n && ok; ++kb, ++it) {
         const int s = it % S;
         const uint32_t ph = (it / S) & 1u;
@@ -903,6 +907,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_next_kernel(const __
         if (have_prev) ok = forward_of(p_it, p_kb, p_rbi);
         p_it = it; p_kb = kb; p_rbi = rbi; have_prev = true;
       }
+      ++rbi;                                              // counts the row blocks actually walked
     }
     if (ok && have_prev) forward_of(p_it, p_kb, p_rbi);
   } else if (warp == 2 && lane == 0) {
@@ -912,6 +917,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_next_kernel(const __
     bool ok = true;
     for (int rb = blockIdx.x; rb < total_rb && ok; rb += gridDim.x) {
       const int n = rb / a.tiles_m, m0 = (rb % a.tiles_m) * 128;
+      if (!item_active(n)) continue;
       for (int kb = 0; kb < a.tiles_n; ++kb, ++it) {
         const int s = it % S;
         const uint32_t ph = (it / S) & 1u;
@@ -942,8 +948,9 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_next_kernel(const __
     const int batches = a.B / 16;
     uint32_t it = 0, rbi = 0;
     bool ok = true;
-    for (int rb = blockIdx.x; rb < total_rb && ok; rb += gridDim.x, ++rbi) {
+    for (int rb = blockIdx.x; rb < total_rb && ok; rb += gridDim.x) {
       const int n = rb / a.tiles_m, m = (rb % a.tiles_m) * 128 + r;
+      if (!item_active(n)) continue;
       for (int kb = 0; kb < a.tiles_n; ++kb, ++it) {
         const int s = it % S;
         const uint32_t ph = (it / S) & 1u;
@@ -1004,6 +1011,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_next_kernel(const __
       }
       tc_fence_before();
       mbar_arrive(facc_empty(q));
+      ++rbi;
     }
   }
   __syncwarp();
@@ -1039,6 +1047,7 @@ struct UpdateDxArgs {
   int64_t bias_stride;
   float mu;                  // momentum form: v <- mu v + G, x <- x - gamma v
   float* bias_vel;           // momentum segment of b_{l-1}, or nullptr
+  const uint8_t* active;     // per-worker flag or nullptr: an inactive worker's column blocks are skipped
 };
 
 // TN = 64: every stage holds fp32 master | momentum | bf16 old | bf16 new (first the a_{l-1} box) | two dZ_l boxes.
@@ -1135,6 +1144,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_dx_kernel(const __gr
   pdl_trigger();
   const uint32_t tmem = *tmem_slot;
   const int total_cb = *abort_flag != 0 ? 0 : col_blocks;
+  auto item_active = [&](int n) { return a.active == nullptr || a.active[n] != 0; };
 
   // Every role walks the same sequence of tiles: column blocks cb = blockIdx.x, + gridDim.x, ..., and inside
   // a column block the row tiles mb = 0 .. tiles_m - 1; `it` counts tiles, tile `it` lives in stage it % S.
@@ -1144,6 +1154,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_dx_kernel(const __gr
     bool ok = true;
     for (int cb = blockIdx.x; cb < total_cb && ok; cb += gridDim.x) {
       const int n = cb / a.tiles_n, n0 = (cb % a.tiles_n) * TN;
+      if (!item_active(n)) continue;
       for (int mb = 0; mb < a.tiles_m; ++mb, ++it) {
         const int s = it % S;
         const uint32_t ph = (it / S) & 1u;
@@ -1201,7 +1212,8 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_dx_kernel(const __gr
       if (mb == a.tiles_m - 1) mma_commit(dacc_full(q));
       return true;
     };
-    for (int cb = blockIdx.x; cb < total_cb && ok; cb += gridDim.x, ++cbi) {
+    for (int cb = blockIdx.x; cb < total_cb && ok; cb += gridDim.x) {
+      if (!item_active(cb / a.tiles_n)) continue;
       for (int mb = 0; mb < a.tiles_m && ok; ++mb, ++it) {
         const int s = it % S;
         const uint32_t ph = (it / S) & 1u;
@@ -1217,6 +1229,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_dx_kernel(const __gr
         if (have_prev) ok = dx_of(p_it, p_mb, p_cbi);
         p_it = it; p_mb = mb; p_cbi = cbi; have_prev = true;
       }
+      ++cbi;                                              // counts the column blocks actually walked
     }
     if (ok && have_prev) dx_of(p_it, p_mb, p_cbi);
   } else if (warp == 2 && lane == 0) {
@@ -1225,6 +1238,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_dx_kernel(const __gr
     bool ok = true;
     for (int cb = blockIdx.x; cb < total_cb && ok; cb += gridDim.x) {
       const int n = cb / a.tiles_n, n0 = (cb % a.tiles_n) * TN;
+      if (!item_active(n)) continue;
       for (int mb = 0; mb < a.tiles_m; ++mb, ++it) {
         const int s = it % S;
         const uint32_t ph = (it / S) & 1u;
@@ -1262,8 +1276,9 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_dx_kernel(const __gr
     const int batches = a.B / 16;
     uint32_t it = 0, cbi = 0;
     bool ok = true;
-    for (int cb = blockIdx.x; cb < total_cb && ok; cb += gridDim.x, ++cbi) {
+    for (int cb = blockIdx.x; cb < total_cb && ok; cb += gridDim.x) {
       const int n = cb / a.tiles_n, n0 = (cb % a.tiles_n) * TN;
+      if (!item_active(n)) continue;
       for (int mb = 0; mb < a.tiles_m; ++mb, ++it) {
         const int s = it % S;
         const uint32_t ph = (it / S) & 1u;
@@ -1353,6 +1368,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_dx_kernel(const __gr
         }
         *bp = fmaf(-a.gamma, gsum, *bp);
       }
+      ++cbi;
     }
   }
   __syncwarp();
@@ -1626,6 +1642,7 @@ inline void tc_launch_update_dx_m(prsgd_ctx* c, int l) {
   a.out_bk = c->buf.delta_bk[l - 1]; a.mask_src = c->buf.act_bk[l - 1]; a.ld_out = c->buf.ld[l - 1]; a.M_total = ly.d_in;
   a.bias_rw = c->params + c->layer[l - 2].b_off; a.bias_stride = c->m_pad;
   a.mu = c->mu; a.bias_vel = MOM ? c->velocity + c->layer[l - 2].b_off : nullptr;
+  a.active = c->has_mask ? c->active : nullptr;
   const int items = a.tiles_n * c->N;
   const int grid = items < st->num_sms ? items : st->num_sms;
   const TcLayerMaps& mp = st->layer[l - 1];
@@ -1656,6 +1673,7 @@ inline void tc_launch_update_next_tn(prsgd_ctx* c, const DrawArgs& dr) {
   UpdateNextArgs a{};
   a.B = c->B; a.N = c->N; a.tiles_m = (ly.d_out + 127) / 128; a.tiles_n = (ly.d_in + TN - 1) / TN;
   a.gamma = c->gamma; a.mu = c->mu; a.draw = dr; a.status = c->status;
+  a.active = c->has_mask ? c->active : nullptr;
   a.stages = UpdNextCfg<TN, MOM>::stages(c->B);
   a.next_out = c->buf.act_bk[1]; a.next_ld = c->buf.ld[1];
   a.bias = c->params + ly.b_off; a.bias_stride = c->m_pad; a.M_total = ly.d_out;

@@ -290,8 +290,7 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging, bool more_follow) {
   // Layer 1's update can form a_1 of iteration t + 1 as well (its input is the data pool), which saves that
   // iteration's first forward launch and the write of W_1's shadow: only on a plain SGD iteration that is
   // not an averaging one and is followed by another one of the same call.
-  const bool next_fwd = c->next_forward && more_follow && !averaging && L > 1 && act_mask == nullptr &&
-                        tc_epilogues_fused(c);
+  const bool next_fwd = c->next_forward && more_follow && !averaging && L > 1 && tc_epilogues_fused(c);
   const bool skip_f1 = c->a1_ready;
   c->a1_ready = false;
   for (int l = skip_f1 ? 2 : 1; l <= L; ++l) {
@@ -312,7 +311,7 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging, bool more_follow) {
   }
   // Layers >= 2 whose update is the plain SGD step: one launch forms dZ_{l-1} and applies the step of W_l (the
   // fused update + average of an averaging iteration owns a tile across workers instead and keeps dX separate).
-  const bool dx_in_upd = c->dx_in_update && act_mask == nullptr && tc_epilogues_fused(c);
+  const bool dx_in_upd = c->dx_in_update && tc_epilogues_fused(c);
   for (int l = L; l >= 1; --l) {          // dX_l reads W_l before the update of layer l overwrites it
     const bool fuse_l = fuse && tc_layer_fuses_average(c, l);
     if (l > 1 && dx_in_upd && !fuse_l && (c->dx_in_update == 2 || tc_layer_folds_dx(c, l))) {

@@ -246,6 +246,41 @@ def test_folded_kernels_with_momentum_change_no_bit(torch_cuda, avg_v):
             assert np.array_equal(outs[0][2], o[2])
 
 
+def test_folded_kernels_with_a_worker_mask_change_no_bit(torch_cuda):
+    """Algorithm 3's worker mask inside the folded update kernels (an inactive worker's blocks are skipped by
+    every role of the kernel) against the separate launches, several iterations per call so that the folded
+    next forward runs too; the inactive workers' rows must not move between averages."""
+    torch = torch_cuda
+    from paper_1807_06629_b200 import binding
+    for w in (_w("tc-mask5", 5, (192, 128, 10), 32, I=3), _w("tc-mask-deep", 4, (64, 448, 320, 10), 16, I=4), SMALL[3]):
+        X, Y, x0 = make_inputs(w)
+        mask = [1 if i % 2 == 0 else 0 for i in range(w.N)]
+        outs = []
+        for dxu, nxt, graph, tile in ((0, 0, 0, 0), (2, 1, 0, 64), (2, 1, 1, 128), (2, 0, 0, 128)):
+            with torch.cuda.stream(torch.cuda.Stream()):
+                p = make_ctx(w, X, Y, x0)
+                p.set_option(binding.OPT_DX_IN_UPDATE, dxu)
+                p.set_option(binding.OPT_NEXT_FORWARD, nxt)
+                p.set_option(binding.OPT_GRAPH, graph)
+                p.set_option(binding.OPT_UPDATE_TILE, tile)
+                p.set_active(mask)
+                p.local_steps(w.I - 1)                     # stops just before the first average
+                before = p.get_params_stacked()
+                p.local_steps(2 * w.I + 2)
+                outs.append((before, p.get_params_stacked(), p.get_losses()))
+                torch.cuda.current_stream().synchronize()
+        x0s = np.tile(x0, (w.N, 1))
+        for i in range(w.N):
+            if not mask[i]:
+                assert np.array_equal(outs[0][0][i], x0s[i])           # an inactive worker has not moved
+            else:
+                assert not np.array_equal(outs[0][0][i], x0s[i])
+        for o in outs[1:]:
+            assert np.array_equal(outs[0][0], o[0]) and np.array_equal(outs[0][1], o[1]), w.name
+            active = [i for i in range(w.N) if mask[i]]
+            assert np.array_equal(outs[0][2][active], o[2][active])
+
+
 def _segments(dims):
     """[(is_weight, start, stop)] of a canonical parameter vector."""
     out, off = [], 0
