@@ -108,7 +108,7 @@ class ClockSampler:
 # capture summarised in profiles/; valid only while the kernel's source section is unchanged.
 NCU_TRAFFIC = {
     ("cfg4", "update"): {"bytes_per_iteration": 2.230e9 + 2.795e9, "launches_per_iteration": 4,   # read + written, four launches
-                         "kernel_sha256": "63039ea6b84a3a2fb52a2d91df2b362254a316e9bf4de42c1c5c1e27fec451e9"},
+                         "kernel_sha256": "190478fcda273dd3a048434f4502704d04d08aa81d379573c362e8cdfd2f91d4"},
 }
 
 
