@@ -404,6 +404,40 @@ def test_full_size_configs(torch_cuda, name, I):
         assert rel_l2(nxt[i] - got[i], -w.gamma * G[k]) <= TOL_UPDATE
 
 
+@pytest.mark.parametrize("name,T", [("cfg3", 64), ("cfg4", 64)])
+def test_full_size_runs_of_whole_periods_keep_the_invariants(torch_cuda, name, T):
+    """cfg3 / cfg4 at full size over several whole periods in one call (graph replay, folded kernels): after the
+    last average every row holds the same bits, the bf16 copy equals bf16(master), the padding is still zero,
+    and the loss has gone down."""
+    torch = torch_cuda
+    w = synth.WORKLOADS[name]
+    w = w.with_(pool_samples=max(w.I, 4) * w.B)
+    X, Y, x0 = make_inputs(w)
+    with torch.cuda.stream(torch.cuda.Stream()):
+        p = make_ctx(w, X, Y, x0)
+        p.local_steps(1)
+        first = p.get_losses().mean()
+        p.local_steps(T - 1)
+        assert p.get_step() == T and T % w.I == 0
+        p.sync()
+        rows = p.params.view(w.N, p.m_pad)
+        assert bool((rows == rows[0:1]).all())             # the run ended on an average: one point, N copies
+        p.local_steps(1)                                   # one more iteration for a loss at the averaged point
+        last = p.get_losses().mean()
+        p.sync()
+        assert np.isfinite(last) and last < first - 0.05, (first, last)
+        store = p.params.cpu().numpy().reshape(w.N, p.m_pad)
+        shadow = p.shadow.view(torch.int16).cpu().numpy().view(np.uint16).reshape(w.N, p.m_pad)
+        keep = np.zeros(p.m_pad, dtype=bool)
+        for l in range(len(w.dims) - 1):
+            a, n = p.layout.w_off[l], w.dims[l] * w.dims[l + 1]
+            keep[a:a + n] = True
+            keep[p.layout.b_off[l]:p.layout.b_off[l] + w.dims[l + 1]] = True
+            assert np.array_equal(shadow[:, a:a + n], synth.bf16_bits(store[:, a:a + n])), l
+        assert np.all(store[:, ~keep] == 0.0)
+        torch.cuda.current_stream().synchronize()
+
+
 @pytest.mark.parametrize("avg_v", [False, True])
 def test_momentum_step_on_the_tensor_core_path(torch_cuda, avg_v):
     """v <- mu v + G, x <- x - gamma v in the update kernel's epilogue; hidden biases +-6 so no ReLU can switch."""
