@@ -165,6 +165,14 @@ int prsgd_average(prsgd_ctx* ctx);
  * the host. */
 int prsgd_get_average(prsgd_ctx* ctx, float* dst, int dst_on_device);
 
+/* The same read-out without stopping the training stream: the mean (Eq. node-average-x) is formed into
+ * the context's staging row on the context's stream, and its copy to h_dst (m floats, HOST memory,
+ * page-locked for the copy to be asynchronous) runs on copy_stream, which must be a different stream.
+ * The call returns at once; h_dst is valid once copy_stream has been synchronised by the caller.
+ * Later prsgd_local_steps calls may run while the copy is in flight (they do not touch the staging
+ * row); the next read-out waits for it.  Device errors surface at the next prsgd_sync. */
+int prsgd_get_average_async(prsgd_ctx* ctx, float* h_dst, void* copy_stream);
+
 /* Mean minibatch loss F_i(x_i^{t-1}; zeta_i^t) of every worker at the last
  * iteration run; h_dst holds N floats (HOST).  Synchronises the stream. */
 int prsgd_get_losses(prsgd_ctx* ctx, float* h_dst);

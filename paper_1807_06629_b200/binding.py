@@ -34,7 +34,7 @@ MAX_LAYERS = 16
 EXPORTS = [
     "prsgd_layout", "prsgd_workspace_bytes", "prsgd_create", "prsgd_destroy", "prsgd_bind_data",
     "prsgd_upload_data", "prsgd_set_params", "prsgd_set_params_stacked", "prsgd_get_params_stacked",
-    "prsgd_get_params", "prsgd_local_steps", "prsgd_average", "prsgd_get_average", "prsgd_get_losses",
+    "prsgd_get_params", "prsgd_local_steps", "prsgd_average", "prsgd_get_average", "prsgd_get_average_async", "prsgd_get_losses",
     "prsgd_get_draws", "prsgd_set_lr", "prsgd_set_interval", "prsgd_set_active", "prsgd_get_step",
     "prsgd_set_step", "prsgd_set_option", "prsgd_get_launch_count", "prsgd_get_profile", "prsgd_sync", "prsgd_last_error",
     "prsgd_average_rows", "prsgd_draw_block", "prsgd_mean_rows_noalloc", "prsgd_selftest_wait_expiry",
@@ -77,6 +77,7 @@ def _load() -> C.CDLL:
         "prsgd_local_steps": (C.c_int, [vp, i64]),
         "prsgd_average": (C.c_int, [vp]),
         "prsgd_get_average": (C.c_int, [vp, vp, C.c_int]),
+        "prsgd_get_average_async": (C.c_int, [vp, vp, vp]),
         "prsgd_get_losses": (C.c_int, [vp, vp]),
         "prsgd_get_draws": (C.c_int, [vp, vp]),
         "prsgd_set_lr": (C.c_int, [vp, C.c_float]),
@@ -291,6 +292,12 @@ class PRSGD:
         else:
             assert out.dtype == torch.float32 and out.numel() == self.m and out.is_contiguous()
             self._call(lib.prsgd_get_average, out.data_ptr(), 1 if out.is_cuda else 0)
+        return out
+
+    def get_average_async(self, out, copy_stream):
+        """Node average into a pinned host tensor through `copy_stream`; valid once that stream is synchronised."""
+        assert out.dtype == torch.float32 and out.numel() == self.m and out.is_contiguous() and out.is_pinned()
+        self._call(lib.prsgd_get_average_async, out.data_ptr(), copy_stream.cuda_stream)
         return out
 
     def get_losses(self) -> np.ndarray:

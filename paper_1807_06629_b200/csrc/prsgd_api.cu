@@ -470,6 +470,8 @@ int prsgd_destroy(prsgd_ctx* ctx) {
   for (auto& p : ctx->pending) { cudaEventDestroy(p.a); cudaEventDestroy(p.b); }
   for (auto e : ctx->event_pool) cudaEventDestroy(e);
   for (auto& g : ctx->graphs) cudaGraphExecDestroy(g.exec);
+  if (ctx->mean_ready_event) cudaEventDestroy(ctx->mean_ready_event);
+  if (ctx->readout_event) cudaEventDestroy(ctx->readout_event);
   if (ctx->staged_event) cudaEventDestroy(ctx->staged_event);
   if (ctx->free_event) cudaEventDestroy(ctx->free_event);
   delete ctx;
@@ -691,9 +693,40 @@ int prsgd_average(prsgd_ctx* c) {
   return launch_average(c);
 }
 
+int prsgd_get_average_async(prsgd_ctx* c, float* h_dst, void* copy_stream) {
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
+  if (!h_dst) return fail(c, PRSGD_ERR_ARG, "h_dst is NULL");
+  cudaStream_t cs = static_cast<cudaStream_t>(copy_stream);
+  if (cs == c->stream) return fail(c, PRSGD_ERR_ARG, "copy_stream must differ from the context's stream");
+  if (!c->mean_ready_event) CUDA_TRY(c, cudaEventCreateWithFlags(&c->mean_ready_event, cudaEventDisableTiming));
+  if (!c->readout_event) CUDA_TRY(c, cudaEventCreateWithFlags(&c->readout_event, cudaEventDisableTiming));
+  // the staging row is free again once the previous asynchronous read-out has left it
+  if (c->readout_pending) CUDA_TRY(c, cudaStreamWaitEvent(c->stream, c->readout_event, 0));
+  prof_begin(c, PRSGD_KERNEL_AVERAGE);
+  average_rows_kernel<1, false><<<grid1d(c->m_pad / 4, 256), 256, 0, c->stream>>>(c->params, c->N, c->m_pad, c->m_pad,
+                                                                              c->stage_row, nullptr);
+  LAUNCH_CHECK(c);
+  CUDA_TRY(c, cudaEventRecord(c->mean_ready_event, c->stream));
+  CUDA_TRY(c, cudaStreamWaitEvent(cs, c->mean_ready_event, 0));
+  int64_t pos = 0;
+  for (int l = 0; l < c->L; ++l) {
+    const Layer& ly = c->layer[l];
+    const int64_t seg[2] = {(int64_t)ly.d_in * ly.d_out, (int64_t)ly.d_out};
+    const int64_t offs[2] = {ly.w_off, ly.b_off};
+    for (int q = 0; q < 2; ++q) {
+      CUDA_TRY(c, cudaMemcpyAsync(h_dst + pos, c->stage_row + offs[q], seg[q] * 4, cudaMemcpyDeviceToHost, cs));
+      pos += seg[q];
+    }
+  }
+  CUDA_TRY(c, cudaEventRecord(c->readout_event, cs));
+  c->readout_pending = true;
+  return PRSGD_OK;
+}
+
 int prsgd_get_average(prsgd_ctx* c, float* dst, int dst_on_device) {
   if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
   if (!dst) return fail(c, PRSGD_ERR_ARG, "dst is NULL");
+  if (c->readout_pending) CUDA_TRY(c, cudaStreamWaitEvent(c->stream, c->readout_event, 0));   // staging row in use
   prof_begin(c, PRSGD_KERNEL_AVERAGE);
   average_rows_kernel<1, false><<<grid1d(c->m_pad / 4, 256), 256, 0, c->stream>>>(c->params, c->N, c->m_pad, c->m_pad,
                                                                               c->stage_row, nullptr);

@@ -127,6 +127,11 @@ struct prsgd_ctx {
   cudaEvent_t staged_event = nullptr;   // staged copy complete (recorded on the caller's copy stream)
   cudaEvent_t free_event = nullptr;     // work that read the previous pools complete (recorded at swap)
 
+  // asynchronous read-out of the node average (prsgd_get_average_async)
+  cudaEvent_t mean_ready_event = nullptr;   // the mean sits in the staging row (recorded on the compute stream)
+  cudaEvent_t readout_event = nullptr;      // its copy to the host has been issued / completed (caller's copy stream)
+  bool readout_pending = false;
+
   // whole averaging periods captured as CUDA graphs (PRSGD_OPT_GRAPH)
   struct PeriodGraph {
     uint64_t key[12];

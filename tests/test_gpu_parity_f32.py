@@ -192,6 +192,35 @@ def test_get_average_is_the_mean_and_leaves_the_store_alone(torch_cuda):
     assert all(np.array_equal(rows[i], rows[0]) for i in range(w.N))
 
 
+def test_asynchronous_read_out_equals_get_average_while_training_goes_on(torch_cuda):
+    """prsgd_get_average_async: the mean is snapshotted on the training stream and copied on another one; training
+    that is queued right behind it must not leak into the snapshot, and back-to-back read-outs must not overwrite
+    each other's staging row."""
+    torch = torch_cuda
+    w = synth.WORKLOADS["cfg2"].with_(pool_samples=8 * 32, I=3)
+    X, Y, x0 = make_inputs(w)
+    with torch.cuda.stream(torch.cuda.Stream()):
+        ref = make_ctx(w, X, Y, x0)
+        p = make_ctx(w, X, Y, x0)
+        rs = torch.cuda.Stream()
+        outs = [torch.empty(p.m, dtype=torch.float32).pin_memory() for _ in range(3)]
+        want = []
+        for k in range(3):
+            ref.local_steps(2 + k)
+            want.append(ref.get_average().copy())
+            p.local_steps(2 + k)
+            p.get_average_async(outs[k], rs)               # returns at once; more work follows immediately
+        p.local_steps(4)
+        rs.synchronize()
+        for k in range(3):
+            assert np.array_equal(outs[k].numpy(), want[k]), k
+        ref.local_steps(4)
+        assert np.array_equal(p.get_average(), ref.get_average())
+        with pytest.raises(Exception):
+            p.get_average_async(outs[0], torch.cuda.current_stream())   # needs a stream of its own
+        torch.cuda.current_stream().synchronize()
+
+
 def test_time_varying_rates_and_heterogeneous_epochs(torch_cuda):
     w = synth.WORKLOADS["cfg1"]
     X, Y, x0 = make_inputs(w)
