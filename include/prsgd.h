@@ -55,6 +55,8 @@ extern "C" {
 #define PRSGD_ERR_STATE          -4  /* call order: e.g. local_steps before bind_data               */
 #define PRSGD_ERR_CUDA           -5  /* a CUDA runtime/driver call failed; see prsgd_last_error     */
 #define PRSGD_ERR_DEVICE_TIMEOUT -6  /* a bounded wait inside a kernel expired (status word set)    */
+#define PRSGD_ERR_NONFINITE      -7  /* the parameter store holds a NaN or an infinity (found by the
+                                        finite check, see prsgd_check_finite)                       */
 
 #define PRSGD_PRECISION_FP32 0       /* fp32 GEMM operands, fp32 accumulation (CUDA cores)          */
 #define PRSGD_PRECISION_BF16 1       /* bf16 GEMM operands from the shadow, fp32 accumulation in
@@ -72,7 +74,7 @@ typedef struct prsgd_ctx prsgd_ctx;   /* opaque; created by prsgd_create, freed 
 typedef struct {
   int32_t  n_layers;       /* L >= 1, at most PRSGD_MAX_LAYERS                                      */
   const int32_t* dims;     /* HOST array of L+1 entries d_0..d_L, copied by the callee              */
-  int32_t  batch;          /* B, per-worker minibatch size, 1..256; BF16: 16, 32, 64 or 128         */
+  int32_t  batch;          /* B, per-worker minibatch size, 1..256; BF16: 16, 32 or 64              */
   int32_t  precision;      /* PRSGD_PRECISION_*; BF16 needs d_0..d_{L-1} to be multiples of 64      */
   int64_t  pool_samples;   /* P, samples in each worker's pool, a positive multiple of B            */
   uint64_t draw_seed;      /* seed of the minibatch draw, see prsgd_draw_block                      */
@@ -213,6 +215,12 @@ int prsgd_run_heterogeneous_epoch(prsgd_ctx* ctx, const int32_t* h_I_i);
  * between them belongs to the caller (NCCL).
  *  - prsgd_set_worker_offset: global index of this context's row 0; the minibatch draw of local
  *    row i is that of worker first_worker + i.
+ *  - prsgd_set_global_workers: the N of the whole job (all contexts together, >= first_worker + the
+ *    context's own N; 0 = this context is the whole job).  Theorem 2's K^s and gamma^s are functions
+ *    of that N, so prsgd_run_time_varying takes its schedule from it; on a context that holds only a
+ *    shard that call returns PRSGD_ERR_STATE, because the epoch's starting average needs every GPU:
+ *    the caller drives the epochs with prsgd_alg2_schedule(N_global, s), prsgd_set_lr,
+ *    prsgd_local_steps and its all-reduce.
  *  - prsgd_partial_sum: d_dst[j] = sum over the local rows of P[i][j], fp32 in row order, for the
  *    padded columns j in [col0, col0 + ncols); d_dst is a device row of m_pad floats.
  *  - prsgd_assign_rows: every local row (and the bf16 shadow) gets d_src[j] / divisor on the same
@@ -221,6 +229,7 @@ int prsgd_run_heterogeneous_epoch(prsgd_ctx* ctx, const int32_t* h_I_i);
  * chunk); rows are 16-byte aligned device pointers.  With a single context,
  * partial_sum + assign_rows(divisor = N) leaves the same bits as prsgd_average.  Asynchronous. */
 int prsgd_set_worker_offset(prsgd_ctx* ctx, int32_t first_worker);
+int prsgd_set_global_workers(prsgd_ctx* ctx, int32_t N_global);
 int prsgd_partial_sum(prsgd_ctx* ctx, float* d_dst, int64_t col0, int64_t ncols);
 int prsgd_assign_rows(prsgd_ctx* ctx, const float* d_src, float divisor, int64_t col0, int64_t ncols);
 
@@ -279,6 +288,8 @@ int prsgd_get_velocity_stacked(prsgd_ctx* ctx, float* dst, int dst_on_device);
  * for a layer that takes the fused update + average on an averaging iteration.  Same bits as the
  * separate launches (also with momentum and with a worker mask). */
 #define PRSGD_OPT_DX_IN_UPDATE 8
+/* PRSGD_OPT_CHECK_FINITE (default 0): when 1, prsgd_sync also runs prsgd_check_finite. */
+#define PRSGD_OPT_CHECK_FINITE 9
 int prsgd_set_option(prsgd_ctx* ctx, int32_t option, int64_t value);
 
 /* Kernel families of the hot path, for prsgd_get_profile. */
@@ -302,11 +313,21 @@ int prsgd_get_launch_count(prsgd_ctx* ctx, int64_t* count);
 /* Wait for the stream, then report any device-side error recorded so far. */
 int prsgd_sync(prsgd_ctx* ctx);
 
+/* Finite check of the whole parameter store (and of the momentum buffers when momentum is on): one
+ * pass that reads every word and counts those whose exponent field is all ones (NaN, +-infinity).
+ * Algorithm 1's averaging step spreads a single worker's NaN to all N workers, so a caller that
+ * wants to stop a diverged run checks before it averages or checkpoints.  Returns PRSGD_OK when
+ * every value is finite, PRSGD_ERR_NONFINITE otherwise; *count (may be NULL) receives the number of
+ * non-finite words, *first_worker (may be NULL) the lowest row that holds one (-1 if none).  Nothing
+ * traps and the store is not modified.  Synchronises the stream. */
+int prsgd_check_finite(prsgd_ctx* ctx, int64_t* count, int32_t* first_worker);
+
 /* Failure path, exercised without faulting the GPU.  Every wait inside the tensor-core kernels is
  * bounded; when one expires the kernel records a code in the scratch status words and returns, later
- * launches of the context become no-ops (a kernel reads the word while it sets up, so the one launch
- * whose set-up overlapped the failing kernel may still run; the parameters are to be set again after
- * a timeout in any case), and prsgd_sync / prsgd_get_* return PRSGD_ERR_DEVICE_TIMEOUT.  prsgd_selftest_wait_expiry launches a one-warp kernel that waits about
+ * local-step and averaging launches of the context (both precisions) become no-ops (a kernel reads the
+ * word while it sets up, so the one launch whose set-up overlapped the failing kernel may still run;
+ * the parameters are to be set again after a timeout in any case: prsgd_set_params* keep working),
+ * and prsgd_sync / prsgd_get_* return PRSGD_ERR_DEVICE_TIMEOUT.  prsgd_selftest_wait_expiry launches a one-warp kernel that waits about
  * limit_us microseconds (1..1000000) on a barrier nothing ever signals, so that exactly this happens;
  * prsgd_clear_device_error zeroes the status words and makes the context usable again (the
  * parameters are as the last successful launch left them). */

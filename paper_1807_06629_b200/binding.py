@@ -28,6 +28,8 @@ OPT_FUSED_EPILOGUES = 5
 OPT_EARLY_LOADS = 6
 OPT_NEXT_FORWARD = 7
 OPT_DX_IN_UPDATE = 8
+OPT_CHECK_FINITE = 9
+ERR_DEVICE_TIMEOUT, ERR_NONFINITE = -6, -7
 KERNEL_FAMILIES = ("forward", "softmax", "dx", "update", "update_average", "average", "misc")
 MAX_LAYERS = 16
 
@@ -41,6 +43,7 @@ EXPORTS = [
     "prsgd_clear_device_error", "prsgd_enable_momentum", "prsgd_get_velocity_stacked",
     "prsgd_set_worker_offset", "prsgd_partial_sum", "prsgd_assign_rows", "prsgd_stage_data", "prsgd_swap_data",
     "prsgd_alg2_schedule", "prsgd_run_time_varying", "prsgd_run_heterogeneous_epoch",
+    "prsgd_set_global_workers", "prsgd_check_finite",
 ]
 NOALLOC_MAX_M = 1 << 20
 
@@ -99,6 +102,8 @@ def _load() -> C.CDLL:
         "prsgd_stage_data": (C.c_int, [vp, vp, vp, vp, vp, vp]),
         "prsgd_swap_data": (C.c_int, [vp]),
         "prsgd_set_worker_offset": (C.c_int, [vp, i32]),
+        "prsgd_set_global_workers": (C.c_int, [vp, i32]),
+        "prsgd_check_finite": (C.c_int, [vp, C.POINTER(i64), C.POINTER(i32)]),
         "prsgd_partial_sum": (C.c_int, [vp, vp, i64, i64]),
         "prsgd_assign_rows": (C.c_int, [vp, vp, C.c_float, i64, i64]),
         "prsgd_last_error": (C.c_char_p, [vp]),
@@ -314,6 +319,9 @@ class PRSGD:
     def set_worker_offset(self, first_worker: int):
         self._call(lib.prsgd_set_worker_offset, first_worker)
 
+    def set_global_workers(self, N_global: int):
+        self._call(lib.prsgd_set_global_workers, N_global)
+
     def new_row(self) -> torch.Tensor:
         """A device row of m_pad floats (the buffer an all-reduce works on)."""
         return torch.zeros(self.m_pad, dtype=torch.float32, device=self.device)
@@ -394,3 +402,10 @@ class PRSGD:
 
     def sync(self):
         self._call(lib.prsgd_sync)
+
+    def check_finite(self):
+        """(return code, count of non-finite words, lowest worker that holds one or -1); does not raise."""
+        n, first = C.c_int64(), C.c_int32()
+        with torch.cuda.device(self.device):
+            rc = lib.prsgd_check_finite(self.ctx, C.byref(n), C.byref(first))
+        return rc, n.value, first.value

@@ -114,6 +114,28 @@ __global__ void __launch_bounds__(256) assign_rows_kernel(float* __restrict__ P,
   }
 }
 
+// Finite check: counts the words of `P` (total4 float4 lanes, rows of row4 lanes) whose exponent field is
+// all ones (NaN or +-infinity) and records the lowest row that holds one.  Reads only.
+__global__ void __launch_bounds__(256) finite_check_kernel(const float* __restrict__ P, int64_t total4, int64_t row4,
+                                                           DeviceStatus* status) {
+  unsigned int bad = 0u, row = 0xFFFFFFFFu;
+  for (int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; c < total4; c += (int64_t)gridDim.x * blockDim.x) {
+    const uint4 v = __ldcs(reinterpret_cast<const uint4*>(P) + c);
+    const unsigned int k = ((v.x & 0x7F800000u) == 0x7F800000u) + ((v.y & 0x7F800000u) == 0x7F800000u) +
+                           ((v.z & 0x7F800000u) == 0x7F800000u) + ((v.w & 0x7F800000u) == 0x7F800000u);
+    if (k != 0u) {
+      bad += k;
+      const unsigned int r = (unsigned int)(c / row4);
+      row = r < row ? r : row;
+    }
+  }
+  if (bad != 0u) {                       // rare: the atomics cost nothing on a healthy store
+    const unsigned int old = atomicAdd(&status->nonfinite, bad);
+    if (old + bad < old) atomicExch(&status->nonfinite, 0xFFFFFFFFu);   // saturate instead of wrapping
+    atomicMin(&status->nonfinite_row, row);
+  }
+}
+
 // device-resident iteration counter of a captured period: set before a replay, advanced at its end
 __global__ void counter_set_kernel(int64_t* counter, int64_t value) { *counter = value; }
 __global__ void counter_add_kernel(int64_t* counter, int64_t delta) {

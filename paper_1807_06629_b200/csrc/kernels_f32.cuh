@@ -45,6 +45,7 @@ struct GemmF32Args {
   const uint8_t* active; // per-worker flag or nullptr
   float* vel;            // DW: momentum buffers laid out like the store, or nullptr
   float mu;
+  const DeviceStatus* status;   // a recorded expired wait turns the launch into a no-op
 };
 
 __device__ __forceinline__ const float* operand_ptr(const OperandF32& o, int n, const DrawArgs& d) {
@@ -63,6 +64,7 @@ __global__ void __launch_bounds__(256) gemm_f32_kernel(const GemmF32Args g) {
   __shared__ __align__(16) float Bs[2][TK][TN + 4];
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");   // no-op unless launched as a programmatic dependent
+  if (g.status != nullptr && g.status->error != 0u) return;   // uniform over the grid: leave everything alone
 
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
   const int i0 = blockIdx.y * TM, j0 = blockIdx.x * TN;

@@ -1,5 +1,6 @@
 // C ABI of the PR-SGD library: host-side context, layout, schedule of
 // Algorithm 1 and the kernel launches.  See include/prsgd.h for the contract.
+#include <algorithm>
 #include <cmath>
 #include <cstdio>
 #include <cstring>
@@ -75,8 +76,8 @@ int check_spec(const prsgd_model_spec* s, std::string* why) {
     *why = "unknown precision"; return PRSGD_ERR_ARG;
   }
   if (s->precision == PRSGD_PRECISION_BF16) {
-    if (s->batch != 16 && s->batch != 32 && s->batch != 64 && s->batch != 128) {
-      *why = "BF16 precision needs batch 16, 32, 64 or 128"; return PRSGD_ERR_ALIGN;
+    if (s->batch != 16 && s->batch != 32 && s->batch != 64) {
+      *why = "BF16 precision needs batch 16, 32 or 64"; return PRSGD_ERR_ALIGN;
     }
     for (int l = 0; l < s->n_layers; ++l)
       if (s->dims[l] % 64 != 0) { *why = "BF16 precision needs d_0..d_{L-1} to be multiples of 64"; return PRSGD_ERR_ALIGN; }
@@ -190,7 +191,7 @@ int refresh_shadow(prsgd_ctx* c) {
 
 int check_device_status(prsgd_ctx* c) {
   DeviceStatus st;
-  CUDA_TRY(c, cudaMemcpyAsync(&st, c->status, 2 * sizeof(unsigned int), cudaMemcpyDeviceToHost, c->stream));
+  CUDA_TRY(c, cudaMemcpyAsync(&st, c->status, 4 * sizeof(unsigned int), cudaMemcpyDeviceToHost, c->stream));
   CUDA_TRY(c, cudaStreamSynchronize(c->stream));
   if (st.error != 0) {
     char msg[128];
@@ -230,7 +231,7 @@ int step_f32(prsgd_ctx* c, int64_t t, bool averaging) {
     g.M = B; g.Nn = ly.d_out; g.K = ly.d_in; g.N = N; g.draw = dr;
     g.out = c->buf.act_f32[l]; g.out_worker_stride = (int64_t)B * ly.d_out;
     g.params = c->params; g.params_worker_stride = c->m_pad; g.b_off = ly.b_off;
-    g.active = act_mask;
+    g.active = act_mask; g.status = c->status;
     prof_begin(c, PRSGD_KERNEL_FORWARD);
     if (l < L) {
       if (B <= 32) launch_gemm_f32<32, true, true, EPI_FWD_RELU, false>(c, g);
@@ -245,7 +246,7 @@ int step_f32(prsgd_ctx* c, int64_t t, bool averaging) {
     SoftmaxArgs a{};
     a.logits = c->buf.act_f32[L]; a.delta = c->buf.delta_f32[L]; a.ldz = c->dims[L];
     a.Y = c->Y; a.P = c->P; a.B = B; a.C = c->dims[L]; a.draw = dr;
-    a.row_losses = c->losses; a.draws = c->draws; a.active = act_mask;
+    a.row_losses = c->losses; a.draws = c->draws; a.active = act_mask; a.status = c->status;
     prof_begin(c, PRSGD_KERNEL_SOFTMAX);
     launch_pdl(softmax_ce_kernel, dim3(N, (B + 7) / 8), dim3(256), 0, c->stream, a);
     LAUNCH_CHECK(c);
@@ -259,7 +260,7 @@ int step_f32(prsgd_ctx* c, int64_t t, bool averaging) {
       g.M = B; g.Nn = ly.d_in; g.K = ly.d_out; g.N = N; g.draw = dr;
       g.out = c->buf.delta_f32[l - 1]; g.out_worker_stride = (int64_t)B * ly.d_in;
       g.mask_src = c->buf.act_f32[l - 1];
-      g.active = act_mask;
+      g.active = act_mask; g.status = c->status;
       prof_begin(c, PRSGD_KERNEL_DX);
       if (B <= 32) launch_gemm_f32<32, true, false, EPI_DX, false>(c, g);
       else         launch_gemm_f32<64, true, false, EPI_DX, false>(c, g);
@@ -271,7 +272,7 @@ int step_f32(prsgd_ctx* c, int64_t t, bool averaging) {
     else        g.Bo = {c->buf.act_f32[l - 1], (int64_t)B * ly.d_in, ly.d_in, 1, 0};
     g.M = ly.d_out; g.Nn = ly.d_in; g.K = B; g.N = N; g.draw = dr;
     g.out = c->params; g.out_worker_stride = c->m_pad; g.w_off = ly.w_off; g.b_off = ly.b_off;
-    g.gamma = c->gamma; g.active = act_mask; g.vel = c->velocity; g.mu = c->mu;
+    g.gamma = c->gamma; g.active = act_mask; g.vel = c->velocity; g.mu = c->mu; g.status = c->status;
     prof_begin(c, fuse ? PRSGD_KERNEL_UPDATE_AVERAGE : PRSGD_KERNEL_UPDATE);
     if (fuse) launch_gemm_f32<64, false, false, EPI_DW, true>(c, g);
     else      launch_gemm_f32<64, false, false, EPI_DW, false>(c, g);
@@ -591,10 +592,10 @@ int run_iterations(prsgd_ctx* c, int64_t t_first, int64_t count) {
     const bool averaging = c->I > 0 && (t % c->I) == 0;
     const bool more_follow = t + 1 < t_first + count;
     int rc = c->precision == PRSGD_PRECISION_BF16 ? step_bf16(c, t, averaging, more_follow) : step_f32(c, t, averaging);
-    if (rc != PRSGD_OK) return rc;
-    if (averaging && (!c->fused_average || c->velocity != nullptr)) {
-      rc = launch_average(c);
-      if (rc != PRSGD_OK) return rc;
+    if (rc == PRSGD_OK && averaging && (!c->fused_average || c->velocity != nullptr)) rc = launch_average(c);
+    if (rc != PRSGD_OK) {
+      c->a1_ready = false;      // a launch failed: the next iteration must not count on an a_1 formed ahead
+      return rc;
     }
   }
   return PRSGD_OK;
@@ -642,6 +643,7 @@ prsgd_ctx::PeriodGraph* get_period_graph(prsgd_ctx* c) {
   cudaGraphExec_t exec = nullptr;
   if (rc == PRSGD_OK && e == cudaSuccess && graph != nullptr) e = cudaGraphInstantiate(&exec, graph, 0);
   if (graph) cudaGraphDestroy(graph);
+  c->a1_ready = false;     // launches recorded into a capture have not run: no a_1 has been formed ahead
   if (rc != PRSGD_OK || e != cudaSuccess || exec == nullptr) {
     cudaGetLastError();
     c->use_graph = 0;                                   // do not try again on this context
@@ -780,6 +782,14 @@ int prsgd_set_worker_offset(prsgd_ctx* c, int32_t first_worker) {
   return PRSGD_OK;
 }
 
+int prsgd_set_global_workers(prsgd_ctx* c, int32_t N_global) {
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
+  if (N_global != 0 && N_global < c->worker0 + c->N)
+    return fail(c, PRSGD_ERR_ARG, "N_global must be 0 or at least first_worker + the context's own N");
+  c->N_global = N_global;
+  return PRSGD_OK;
+}
+
 namespace {
 int check_cols(prsgd_ctx* c, const void* p, int64_t col0, int64_t ncols) {
   if (!p) return fail(c, PRSGD_ERR_ARG, "NULL row pointer");
@@ -854,13 +864,16 @@ int prsgd_run_time_varying(prsgd_ctx* c, int64_t s_begin, int64_t s_end, float g
   if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
   if (s_begin < 1 || s_end < s_begin) return fail(c, PRSGD_ERR_ARG, "need 1 <= s_begin <= s_end");
   if (!(gamma_scale > 0.f)) return fail(c, PRSGD_ERR_ARG, "gamma_scale must be > 0");
+  if (c->N_global > c->N)
+    return fail(c, PRSGD_ERR_STATE, "this context holds a shard of the workers: the epoch's starting average needs "
+                                    "every shard; drive the epochs with prsgd_alg2_schedule(N_global, s)");
   const int I_keep = c->I;
   const float g_keep = c->gamma;
   c->I = 0;                                          // epochs are driven here, not by t mod I
   int rc = PRSGD_OK;
   for (int64_t s = s_begin; s <= s_end && rc == PRSGD_OK; ++s) {
     int64_t K = 0; float g = 0.f;
-    prsgd_alg2_schedule(c->N * 1, s, &K, &g);
+    prsgd_alg2_schedule(c->N_global > 0 ? c->N_global : c->N, s, &K, &g);   // Theorem 2's N counts every worker
     rc = launch_average(c);                          // x_i^{s,0} = node average of the previous epoch's end points
     if (rc != PRSGD_OK) break;
     c->gamma = g * gamma_scale;
@@ -943,6 +956,7 @@ int prsgd_set_option(prsgd_ctx* c, int32_t option, int64_t value) {
   if (option == PRSGD_OPT_FUSED_EPILOGUES) { c->fused_epilogues = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_EARLY_LOADS) { c->early_loads = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_NEXT_FORWARD) { c->next_forward = value != 0; return PRSGD_OK; }
+  if (option == PRSGD_OPT_CHECK_FINITE) { c->check_finite = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_DX_IN_UPDATE) {
     if (value < 0 || value > 2) return fail(c, PRSGD_ERR_ARG, "PRSGD_OPT_DX_IN_UPDATE takes 0, 1 or 2");
     c->dx_in_update = (int)value;
@@ -999,9 +1013,38 @@ int prsgd_clear_device_error(prsgd_ctx* c) {
   return PRSGD_OK;
 }
 
+int prsgd_check_finite(prsgd_ctx* c, int64_t* count, int32_t* first_worker) {
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
+  CUDA_TRY(c, cudaMemsetAsync(&c->status->nonfinite, 0, sizeof(unsigned int), c->stream));
+  CUDA_TRY(c, cudaMemsetAsync(&c->status->nonfinite_row, 0xFF, sizeof(unsigned int), c->stream));
+  const int64_t row4 = c->m_pad / 4;
+  const int64_t total4 = (int64_t)c->N * row4;
+  const int grid = (int)std::min<int64_t>((total4 + 1023) / 1024, 148 * 16);
+  for (const float* store : {(const float*)c->params, (const float*)c->velocity}) {
+    if (store == nullptr) continue;
+    prof_begin(c, PRSGD_KERNEL_MISC);
+    finite_check_kernel<<<grid, 256, 0, c->stream>>>(store, total4, row4, c->status);
+    LAUNCH_CHECK(c);
+  }
+  DeviceStatus st;
+  CUDA_TRY(c, cudaMemcpyAsync(&st, c->status, 4 * sizeof(unsigned int), cudaMemcpyDeviceToHost, c->stream));
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  if (count) *count = (int64_t)st.nonfinite;
+  if (first_worker) *first_worker = st.nonfinite != 0u ? (int32_t)st.nonfinite_row : -1;
+  if (st.nonfinite != 0u) {
+    char msg[160];
+    std::snprintf(msg, sizeof msg, "%u non-finite value(s) in the parameter store, the first in worker %u's row",
+                  st.nonfinite, st.nonfinite_row);
+    return fail(c, PRSGD_ERR_NONFINITE, msg);
+  }
+  return PRSGD_OK;
+}
+
 int prsgd_sync(prsgd_ctx* c) {
   if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
-  return check_device_status(c);
+  int rc = check_device_status(c);
+  if (rc == PRSGD_OK && c->check_finite) rc = prsgd_check_finite(c, nullptr, nullptr);
+  return rc;
 }
 
 int prsgd_average_rows(float* d_P, int64_t N, int64_t m, int64_t row_stride, void* cuda_stream) {

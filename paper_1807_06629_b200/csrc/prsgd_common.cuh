@@ -37,7 +37,9 @@ __host__ __device__ inline uint32_t draw_block(uint64_t seed, int worker, int64_
 struct DeviceStatus {
   unsigned int error;      // 0 = fine; otherwise a code naming the wait that gave up
   unsigned int where;      // block index that recorded it
-  unsigned int pad[62];
+  unsigned int nonfinite;      // finite check: number of NaN / infinite words found (saturating)
+  unsigned int nonfinite_row;  // finite check: lowest row that holds one
+  unsigned int pad[60];
 };
 
 // Launch with the programmatic-stream-serialization attribute: the kernel may start while the
@@ -86,6 +88,8 @@ struct prsgd_ctx {
   int I = 0;
   int64_t t = 0;
   int worker0 = 0;               // global index of row 0 when the N workers here are a shard of a larger job
+  int N_global = 0;              // workers of the whole job (0: this context is the whole job)
+  int check_finite = 0;          // prsgd_sync also runs the finite check
   int fused_average = 1;
   float mu = 0.f;                // momentum of the local step (0 = plain SGD)
   float* velocity = nullptr;     // [N][m_pad] fp32 momentum buffers, caller-owned

@@ -397,6 +397,80 @@ def test_algorithm_2_and_3_drivers(torch_cuda):
     assert q.get_step() == 6
 
 
+def test_non_finite_parameters_are_reported_not_trapped(torch_cuda):
+    """A NaN (or an infinity) put into ONE worker's row through prsgd_set_params is found by the finite check
+    before the average, and after the average, which spreads it to every row (Algorithm 1's averaging step),
+    in all N rows; with PRSGD_OPT_CHECK_FINITE prsgd_sync reports it too.  Both precisions."""
+    from paper_1807_06629_b200 import binding
+    cases = [(synth.WORKLOADS["cfg1"], float("nan")), (synth.WORKLOADS["cfg1"], float("-inf")),
+             (synth.Workload("tc-nonfinite", 3, (64, 128, 10), 32, 0.05, 2, 4, 1, 128, mean_shift=0.5, seed=5), float("nan"))]
+    for w, poison in cases:
+        X, Y, x0 = make_inputs(w)
+        p = make_ctx(w, X, Y, x0, I=0)
+        p.local_steps(1)
+        assert p.check_finite() == (0, 0, -1)
+        bad = p.get_params(w.N - 2)
+        bad[[7, x0.size - 1]] = poison                   # a weight of the first layer and the last bias
+        p.set_params(bad, worker=w.N - 2)
+        rc, count, first = p.check_finite()
+        assert (rc, count, first) == (binding.ERR_NONFINITE, 2, w.N - 2)
+        assert b"non-finite" in binding.lib.prsgd_last_error(p.ctx)
+        p.sync()                                         # the plain sync does not look for it ...
+        p.set_option(binding.OPT_CHECK_FINITE, 1)
+        with pytest.raises(binding.PRSGDError) as e:     # ... unless asked to
+            p.sync()
+        assert e.value.code == binding.ERR_NONFINITE
+        p.set_option(binding.OPT_CHECK_FINITE, 0)
+        p.average()
+        rc, count, first = p.check_finite()
+        assert (rc, count, first) == (binding.ERR_NONFINITE, 2 * w.N, 0)
+        p.set_params(x0)                                 # a clean state again: the context is usable
+        assert p.check_finite() == (0, 0, -1)
+        p.enable_momentum(0.9)
+        p.local_steps(1)
+        assert p.check_finite() == (0, 0, -1)            # (the momentum buffers are read as well)
+
+
+def test_expired_wait_stops_the_fp32_path_too(torch_cuda):
+    """After a bounded wait has run out, the local-step kernels of an FP32 context leave the store alone."""
+    from paper_1807_06629_b200 import binding
+    w = synth.WORKLOADS["cfg1"]
+    X, Y, x0 = make_inputs(w)
+    p = make_ctx(w, X, Y, x0)
+    p.local_steps(1)
+    after1 = p.get_params_stacked()
+    p.selftest_wait_expiry(300)
+    with pytest.raises(binding.PRSGDError) as e:
+        p.sync()
+    assert e.value.code == binding.ERR_DEVICE_TIMEOUT
+    p.local_steps(2 * w.I)                               # forward, dX, update and averaging launches: all no-ops
+    p.clear_device_error()
+    assert np.array_equal(p.get_params_stacked(), after1)
+    q = make_ctx(w, X, Y, x0)                            # and the context carries on like a fresh one
+    q.local_steps(1 + 2 * w.I)
+    p.set_step(1)
+    p.local_steps(2 * w.I)
+    assert np.array_equal(p.get_params_stacked(), q.get_params_stacked())
+
+
+def test_time_varying_schedule_uses_the_global_worker_count(torch_cuda):
+    """Theorem 2's K^s and gamma^s are functions of the N of the whole job: a context that is told it holds all
+    of a larger job's rows is refused (its average would be a shard's), one that is the whole job runs."""
+    from paper_1807_06629_b200 import binding
+    w = synth.WORKLOADS["cfg1"]
+    X, Y, x0 = make_inputs(w)
+    p = make_ctx(w, X, Y, x0)
+    with pytest.raises(binding.PRSGDError):
+        p.set_global_workers(w.N - 1)
+    p.set_global_workers(2 * w.N)
+    with pytest.raises(binding.PRSGDError) as e:
+        p.run_time_varying(1, 3, 0.02)
+    assert e.value.code == -4
+    p.set_global_workers(0)
+    p.run_time_varying(1, 3, 0.02)
+    assert p.get_step() == sum(K for K, _ in orc.alg2_schedule(w.N, 3))
+
+
 def test_cfg1_whole_run_tracks_the_oracle(torch_cuda):
     """All T = 64 iterations of the tiny configuration (16 averaging periods), GPU against oracle:
     the same draws every iteration, the same loss curve, and parameters that stay together."""

@@ -89,6 +89,8 @@ def test_bad_specs_are_refused_on_the_host(binding):
     assert rc((32, 64, 10), 16, 7, 1024) == -1         # precision
     assert rc((32, 60, 10), 16, 1, 1024) == -2         # bf16 needs multiples of 64
     assert rc((64, 64, 10), 24, 1, 1008) == -2         # bf16 batch
+    assert rc((64, 64, 10), 128, 1, 1024) == -2        # bf16 batch above 64: refused before any buffer is sized
+    assert rc((64, 64, 10), 128, 0, 1024) == 0         # (fp32 takes it)
     assert b"multiples of 64" in lib.prsgd_last_error(None) or b"batch" in lib.prsgd_last_error(None)
     assert rc((8,) * 18, 16, 0, 1024) == -1            # more than PRSGD_MAX_LAYERS layers
     assert rc((8,) * 17, 16, 0, 1024) == 0             # exactly 16 layers
