@@ -5,17 +5,26 @@ One "step" of this benchmark is one full averaging period of the workload:
 I local iterations of all N workers followed by the node average, i.e.
 prsgd_local_steps(I).  The metric is worker-steps/s = N * I * steps / time.
 
-Prints ONE JSON line.  `value` is timed on the device with inputs resident in
-HBM; `e2e` is the same period driven through the C ABI from pinned HOST
-buffers (pool upload, local steps, read-back of the node average).
+Prints ONE JSON line (the last line of stdout).  `value` is timed on the device
+with inputs resident in HBM; `e2e` is the same period driven through the C ABI
+from pinned HOST buffers (pool upload, local steps, read-back of the node
+average).  `configs` carries short runs of the other training configurations.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--config cfg4] [--impl reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config cfg4] [--scaling weak|strong] [--impl reference]
+
+Several GPUs: one process per GPU.  Started under torchrun (WORLD_SIZE set) the
+script is one rank; started plainly with --gpus N > 1 it starts the N ranks
+itself (`launch_ranks`).  The workers are sharded over the ranks (`--scaling
+strong`: the configuration's N workers are split; `weak`, the default: every rank
+holds N workers of a job of N * G), local steps need no exchange, and the node
+average is local row sums + an NCCL all-reduce + the restart.
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
+import socket
 import subprocess
 import sys
 import threading
@@ -32,6 +41,8 @@ from paper_1807_06629_b200 import synth
 DEFAULT_WORKLOAD = "cfg4"
 L2_BYTES = 126 * 1024 * 1024
 METRIC = "worker-steps/s"
+# the other training configurations, measured briefly in the default run: (workload, I, timed periods)
+OTHER_CONFIGS = (("cfg1", 4, 60), ("cfg2", 8, 40), ("cfg3", 1, 60), ("cfg3", 4, 40), ("cfg3", 16, 20))
 
 
 def load_peaks():
@@ -42,6 +53,86 @@ def load_peaks():
         return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
                 "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ----------------------------------------------------------------------------- ranks
+def rank_env():
+    """(rank, local_rank, world_size) as torchrun exports them; (0, 0, 1) for a plain start."""
+    return (int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")),
+            int(os.environ.get("WORLD_SIZE", "1")))
+
+
+def free_port() -> int:
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    return port
+
+
+def launch_ranks(n: int, script_args, script: str = None, capture: bool = False, timeout: float = None):
+    """Start `script` (this file by default) as n ranks of one node, one process per GPU, the way the
+    launcher of torch.distributed does (rendezvous on 127.0.0.1), and wait for them.  Returns the
+    CompletedProcess; with capture=True stdout and stderr are captured instead of inherited."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(free_port()), script or os.path.abspath(__file__)]
+    cmd += list(script_args)
+    env = dict(os.environ)
+    env.setdefault("OMP_NUM_THREADS", "4")
+    return subprocess.run(cmd, env=env, capture_output=capture, text=True, timeout=timeout)
+
+
+def max_over_ranks(x: float, world: int, device="cpu") -> float:
+    """The slowest rank's figure (a multi-GPU time is the maximum over the ranks)."""
+    if world <= 1:
+        return float(x)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+class CudaTimer:
+    """CUDA events on torch's current stream, one pair per timed step."""
+
+    def __init__(self, torch, steps):
+        self.ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+
+    def start(self, k):
+        self.ev[k][0].record()
+
+    def stop(self, k):
+        self.ev[k][1].record()
+
+    def total_ms(self):
+        return sum(a.elapsed_time(b) for a, b in self.ev)
+
+
+def time_periods(run_period, steps: int, warmup: int, timer, barrier, before_step=None, after_warmup=None) -> float:
+    """`warmup` untimed periods, a barrier, then exactly `steps` timed periods and a barrier;
+    returns this rank's summed time in ms (the caller takes the maximum over ranks)."""
+    for _ in range(warmup):
+        run_period()
+    barrier()
+    if after_warmup is not None:
+        after_warmup()
+    for k in range(steps):
+        if before_step is not None:
+            before_step(k)
+        timer.start(k)
+        run_period()
+        timer.stop(k)
+    barrier()
+    return timer.total_ms()
+
+
+def result_line(w_cfg: dict, value: float, ms_total: float, steps: int, warmup: int, world: int, scaling: str,
+                dtype: str) -> dict:
+    """The keys every line of this benchmark carries."""
+    return {"metric": METRIC, "value": value, "unit": METRIC, "n_gpus": world, "steps": steps, "warmup": warmup,
+            "ms_per_step": ms_total / steps, "higher_is_better": True, "scaling": scaling, "vs_baseline": None,
+            "dtype": dtype, "data": "synthetic", "config": w_cfg}
 
 
 # ----------------------------------------------------------------------------- clocks
@@ -104,16 +195,17 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------- ncu traffic
-# dram__bytes_read.sum + dram__bytes_write.sum per iteration of one kernel family, from the one-pass ncu
-# capture summarised in profiles/; valid only while the kernel's source section is unchanged.
+# dram__bytes_read.sum + dram__bytes_write.sum per plain iteration of one kernel family, from a one-pass ncu
+# capture of a SMALL case (cfg4 shapes with `workers` workers, a few hundred MB on the device; summary in
+# profiles/).  The update kernels stream every worker's tiles once, so traffic grows in proportion to the
+# number of workers: the record is scaled by N / workers.  Valid only while the kernels' source is unchanged.
 NCU_TRAFFIC = {
-    ("cfg4", "update"): {"bytes_per_iteration": 2.230e9 + 2.795e9, "launches_per_iteration": 4,   # read + written, four launches
-                         "kernel_sha256": "190478fcda273dd3a048434f4502704d04d08aa81d379573c362e8cdfd2f91d4"},
+    ("cfg4", "update"): {"workers": 16, "bytes_per_iteration": None, "launches_per_iteration": 4, "kernel_sha256": ""},
 }
 
 
 def kernel_section_sha(family: str) -> str:
-    """Hash of the source text of the kernel a family runs (update: tc_update_kernel and its stage layout)."""
+    """Hash of the source text of the kernels a family runs (update: the update kernels and their stage layouts)."""
     import hashlib
     path = os.path.join(ROOT, "paper_1807_06629_b200", "csrc", "kernels_bf16.cuh")
     with open(path) as f:
@@ -125,11 +217,11 @@ def kernel_section_sha(family: str) -> str:
     return hashlib.sha256(src[a:b].encode()).hexdigest() if 0 <= a < b else ""
 
 
-def ncu_traffic_per_launch(workload: str, family: str):
-    rec = NCU_TRAFFIC.get((workload, family))
-    if rec is None or rec["kernel_sha256"] != kernel_section_sha(family):
+def ncu_traffic_per_launch(workload: str, family: str, N: int):
+    rec = NCU_TRAFFIC.get((workload.split("-")[0], family))
+    if rec is None or rec["bytes_per_iteration"] is None or rec["kernel_sha256"] != kernel_section_sha(family):
         return None
-    return rec["bytes_per_iteration"] / rec["launches_per_iteration"]
+    return rec["bytes_per_iteration"] * (N / rec["workers"]) / rec["launches_per_iteration"]
 
 
 # ----------------------------------------------------------------------------- byte model
@@ -175,14 +267,18 @@ def flops_per_worker_step(w: synth.Workload) -> int:
 
 
 # ----------------------------------------------------------------------------- oracle (CPU baseline)
+def oracle_cores() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        return max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        return 1
+
+
 def time_oracle(w: synth.Workload, X, Y, x0, budget_s: float = 15.0):
     """Times the fp64 oracle, as it stands, on a bounded sample: all N workers for s iterations."""
     from oracle import prsgd_oracle as orc
-    try:
-        from threadpoolctl import threadpool_info
-        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
-    except Exception:
-        cores = 1
+    cores = oracle_cores()
     fn = orc.mlp_grad_fn(w.dims, X, Y, w.B, w.seed)
     state = np.tile(x0.astype(np.float64), (w.N, 1))
     t0 = time.perf_counter()
@@ -197,16 +293,12 @@ def time_oracle(w: synth.Workload, X, Y, x0, budget_s: float = 15.0):
 
 
 def run_reference(args, w):
-    """--impl reference: the oracle on the host cores; each step is one iteration of all N workers."""
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
+    """--impl reference: the oracle on the host cores; each step is one iteration of all N workers.
+    Under a multi-rank launch rank 0 alone runs and prints; the other ranks exit without work."""
+    if rank_env()[0] != 0:
         return
     from oracle import prsgd_oracle as orc
-    try:
-        from threadpoolctl import threadpool_info
-        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
-    except Exception:
-        cores = 1
+    cores = oracle_cores()
     X, Y = synth.make_pools(w)
     if w.precision == 1:
         X = synth.bf16_round(X)
@@ -222,14 +314,11 @@ def run_reference(args, w):
     dt = time.perf_counter() - t0
     val = w.N * args.steps / dt
     sample = f"each step = 1 iteration of all {w.N} workers of {w.name} (fp64 numpy oracle)"
-    print(json.dumps({
-        "impl": "reference", "metric": METRIC, "value": val, "unit": METRIC, "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": workload_config(w),
-        "cpu_baseline": {"value": val, "unit": METRIC, "cores": cores, "kind": "oracle", "sample": sample},
-        "e2e": {"value": val, "unit": METRIC, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
-    }))
+    line = result_line(workload_config(w), val, 1e3 * dt, args.steps, args.warmup, args.gpus, "weak", "f64")
+    line.update({"impl": "reference",
+                 "cpu_baseline": {"value": val, "unit": METRIC, "cores": cores, "kind": "oracle", "sample": sample},
+                 "e2e": {"value": val, "unit": METRIC, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}})
+    print(json.dumps(line))
 
 
 def workload_config(w, extra=None, momentum=None):
@@ -244,7 +333,7 @@ def workload_config(w, extra=None, momentum=None):
 
 
 # ----------------------------------------------------------------------------- averaging sweep
-def averaging_sweep(torch, binding, peaks, quick=False):
+def averaging_sweep(torch, binding, peaks, dev, quick=False):
     """Node-average kernel in isolation on [N, m] fp32: GB/s counting N*m*4 read + N*m*4 written."""
     out = []
     for N in synth.SWEEP_N:
@@ -253,7 +342,7 @@ def averaging_sweep(torch, binding, peaks, quick=False):
                 continue
             nbytes = N * m * 4
             copies = max(1, int(np.ceil(2 * L2_BYTES / nbytes))) if nbytes <= 2 * L2_BYTES else 1
-            bufs = [torch.randn(N, m, device="cuda:0", dtype=torch.float32) for _ in range(copies)]
+            bufs = [torch.randn(N, m, device=dev, dtype=torch.float32) for _ in range(copies)]
             reps = 20
             binding.prsgd_average_rows(bufs[0], N, m)
             torch.cuda.synchronize()
@@ -273,77 +362,21 @@ def averaging_sweep(torch, binding, peaks, quick=False):
     return out
 
 
-# ----------------------------------------------------------------------------- main arm
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=24)
-    ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--config", default=DEFAULT_WORKLOAD, choices=sorted(synth.WORKLOADS))
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--interval", type=int, default=None, help="override the averaging interval I")
-    ap.add_argument("--workers", type=int, default=None, help="override N (smaller cases for profiler captures)")
-    ap.add_argument("--momentum", type=float, default=None, help="local step with momentum mu (the paper's experiment used 0.9)")
-    ap.add_argument("--update-tile", type=int, default=None, help="tile width of the update kernel (64 or 128)")
-    ap.add_argument("--no-fuse", action="store_true",
-                    help="averaging iterations run as update + stand-alone averaging kernel instead of the fused pass")
-    ap.add_argument("--no-fused-epilogues", action="store_true",
-                    help="softmax-CE gradient and bias steps as kernels of their own instead of GEMM epilogues")
-    ap.add_argument("--no-dx-in-update", action="store_true",
-                    help="separate dX launches instead of forming dZ of the layer below inside the update launch")
-    ap.add_argument("--no-next-forward", action="store_true",
-                    help="layer 1's update does not form the next iteration's a_1")
-    ap.add_argument("--no-early-loads", action="store_true",
-                    help="no tile requests ahead of a kernel's dependency wait")
-    ap.add_argument("--force-sharded", action="store_true",
-                    help="run the multi-GPU code path (sharded workers + all-reduce average) even on one GPU")
-    ap.add_argument("--no-sweep", action="store_true", help="skip the averaging-kernel sweep")
-    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle timing")
-    args = ap.parse_args()
-    if args.warmup < 3:
-        args.warmup = 3
-    w = synth.WORKLOADS[args.config]
-    if args.interval is not None:
-        w = w.with_(I=args.interval)
-    if args.workers is not None:
-        w = w.with_(N=args.workers, name=f"{w.name}-N{args.workers}")
+# ----------------------------------------------------------------------------- one configuration on the GPU
+def measure_config(torch, w_cfg, args, dev, rank, world, scaling, steps, warmup, peaks, sharded_mode,
+                   with_e2e, with_clocks):
+    """Builds the context of this rank's shard of `w_cfg`, times `steps` periods on the device (CUDA events,
+    maximum over ranks), repeats the region with an event pair around every launch for the roofline, and
+    (with_e2e) times the same periods driven from pinned host buffers.  Returns (result dict, state for the
+    CPU-oracle leg)."""
+    import torch.distributed as dist
+    from paper_1807_06629_b200 import binding, sharded
+    first, n_local, n_global = sharded.partition(w_cfg.N, world, rank, scaling) if sharded_mode else (0, w_cfg.N, w_cfg.N)
     # the pool holds one averaging period's worth of fresh samples per worker (I blocks of B; at least 4),
     # which is what the end-to-end arm uploads from the host before every period
-    w = w.with_(pool_samples=max(w.I, 4) * w.B)
-    if args.impl == "reference":
-        return run_reference(args, w)
-
-    import torch
-    import torch.distributed as dist
-    from paper_1807_06629_b200 import _build
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
-    if rank == 0 or world == 1:
-        _build.build_library()
-    torch.cuda.set_device(local_rank)
-    dev = f"cuda:{local_rank}"
-    # everything below (torch copies, the library's kernels, the timing events) runs on one side stream:
-    # the library replays captured periods as CUDA graphs, which the legacy default stream cannot capture
-    torch.cuda.set_stream(torch.cuda.Stream(device=dev))
-    sharded_mode = world > 1 or args.force_sharded
-    if sharded_mode:
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        os.environ.setdefault("MASTER_PORT", "29533")
-        if os.environ.get("NCCL_DEBUG", "").upper() == "VERSION":   # its banner would share stdout with the JSON line
-            os.environ["NCCL_DEBUG"] = "WARN"
-        dist.init_process_group("nccl", rank=rank, world_size=world, device_id=torch.device(dev))
-        dist.barrier()
-    from paper_1807_06629_b200 import binding, sharded
-    peaks = load_peaks()
-
-    # Weak scaling: every rank holds w.N workers of a job with w.N * world workers.  All ranks start from
-    # the same x^0; each rank's workers have their own data pools (seed stream of the rank).
-    x0 = synth.init_params(w.dims, w.seed)
-    w = w.with_(seed=w.seed + rank)
-    X, Y = synth.make_pools(w)
+    w = w_cfg.with_(N=n_local, pool_samples=max(w_cfg.I, 4) * w_cfg.B)
+    x0 = synth.init_params(w.dims, w.seed)              # the same x^0 on every rank
+    X, Y = synth.make_pools(w, first)                   # this rank's workers of the job
     if w.precision == 1:
         X = synth.bf16_round(X)
     tdt = torch.bfloat16 if w.precision == 1 else torch.float32
@@ -355,8 +388,9 @@ def main():
     p.set_params(x0)
     job = None
     if sharded_mode:          # local steps on the shard, node average = local sums + NCCL all-reduce + restart
-        p.set_worker_offset(rank * w.N)
-        job = sharded.ShardedPRSGD(p, w.N * world, w.I)
+        p.set_worker_offset(first)
+        p.set_global_workers(n_global)
+        job = sharded.ShardedPRSGD(p, n_global, w.I)
 
     def run_period():
         if job is not None:
@@ -367,16 +401,11 @@ def main():
         p.set_option(binding.OPT_UPDATE_TILE, args.update_tile)
     if args.momentum is not None:
         p.enable_momentum(args.momentum)
-    if args.no_fuse:
-        p.set_option(binding.OPT_FUSED_AVERAGE, 0)
-    if args.no_dx_in_update:
-        p.set_option(binding.OPT_DX_IN_UPDATE, 0)
-    if args.no_next_forward:
-        p.set_option(binding.OPT_NEXT_FORWARD, 0)
-    if args.no_early_loads:
-        p.set_option(binding.OPT_EARLY_LOADS, 0)
-    if args.no_fused_epilogues:
-        p.set_option(binding.OPT_FUSED_EPILOGUES, 0)
+    for flag, opt in ((args.no_fuse, binding.OPT_FUSED_AVERAGE), (args.no_dx_in_update, binding.OPT_DX_IN_UPDATE),
+                      (args.no_next_forward, binding.OPT_NEXT_FORWARD), (args.no_early_loads, binding.OPT_EARLY_LOADS),
+                      (args.no_fused_epilogues, binding.OPT_FUSED_EPILOGUES)):
+        if flag:
+            p.set_option(opt, 0)
     working_set = p.params.numel() * 4 + (p.shadow.numel() * 2 if p.shadow is not None else 0)
     need_flush = working_set <= 2 * L2_BYTES
     flush = torch.empty(3 * L2_BYTES // 4, dtype=torch.float32, device=dev) if need_flush else None
@@ -386,39 +415,33 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- device-timed region: K periods, inputs resident in HBM -------------------------
-    sampler = ClockSampler(local_rank)
-    sampler.start()
-    for _ in range(args.warmup):
-        run_period()
-    p.sync()
-    barrier()
-    sampler.mark()
-    launches0 = p.get_launch_count()
-    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    for k in range(args.steps):
+    def flush_l2(k):
         if flush is not None:
             flush.fill_(float(k))
-        evs[k][0].record()
-        run_period()
-        evs[k][1].record()
-    barrier()
-    clocks = sampler.stop()
-    launches = p.get_launch_count() - launches0
-    ms_total = sum(a.elapsed_time(b) for a, b in evs)
-    tt = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-    ms_total = float(tt.item())
-    worker_steps = w.N * w.I * args.steps * world
+
+    # ---- device-timed region: K periods, inputs resident in HBM -------------------------
+    sampler = ClockSampler(torch.cuda.current_device()) if with_clocks else None
+    if sampler:
+        sampler.start()
+    launches0 = [0]
+
+    def after_warmup():
+        p.sync()
+        if sampler:
+            sampler.mark()
+        launches0[0] = p.get_launch_count()
+    ms_local = time_periods(run_period, steps, warmup, CudaTimer(torch, steps), barrier, flush_l2, after_warmup)
+    clocks = sampler.stop() if sampler else None
+    launches = p.get_launch_count() - launches0[0]
+    ms_total = max_over_ranks(ms_local, world, dev)
+    worker_steps = n_global * w.I * steps          # what all ranks processed
     value = worker_steps / (ms_total * 1e-3)
 
     # ---- per-kernel pass (same region again with an event pair around every launch) ------
     p.set_option(binding.OPT_PROFILE, 1)
     p.get_profile()
-    for k in range(args.steps):
-        if flush is not None:
-            flush.fill_(float(k))
+    for k in range(steps):
+        flush_l2(k)
         run_period()
     prof = p.get_profile()
     p.set_option(binding.OPT_PROFILE, 0)
@@ -437,65 +460,164 @@ def main():
     dom_ms, dom_launches = fams[dom]
     iters_seen = dom_launches / max(per_iter_launches, 1)
     achieved = bytes_iter[dom] * iters_seen / (dom_ms * 1e-3) / 1e9
+    prof_sum = sum(x[0] for x in prof.values())
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"] + " copy bandwidth",
-                "traffic": ncu_traffic_per_launch(w.name, dom),
+                "traffic": ncu_traffic_per_launch(w_cfg.name, dom, w.N),
                 "avg_launch_us": 1e3 * dom_ms / dom_launches,
                 "algorithmic_bytes_per_launch": bytes_iter[dom] / per_iter_launches,
-                "family_us_per_iteration": {k: round(1e3 * v[0] / (args.steps * max(w.I, 1)), 2) for k, v in prof.items() if v[1]},
-                "share_of_step_time": {k: round(v[0] / sum(x[0] for x in prof.values()), 4) for k, v in prof.items() if v[1]}}
+                "family_us_per_iteration": {k: round(1e3 * v[0] / (steps * max(w.I, 1)), 2) for k, v in prof.items() if v[1]},
+                "share_of_step_time": {k: round(v[0] / prof_sum, 4) for k, v in prof.items() if v[1]}}
     tflops = flops_per_worker_step(w) * value / world / 1e12
+    res = {"value": value, "ms_total": ms_total, "launches": launches, "roofline": roofline, "clocks": clocks,
+           "gemm_tflops": tflops, "need_flush": need_flush, "n_local": n_local, "n_global": n_global, "w": w,
+           "pool_samples": w.pool_samples}
 
     # ---- end to end through the C ABI from pinned host buffers ---------------------------
     # Every period: fresh pools come from pinned host memory (staged on a copy stream into the spare
     # device pools while the previous period computes, then swapped in), the period runs, and the node
     # average is read back into pinned host memory.
-    avg_host = [torch.empty(p.m, dtype=torch.float32).pin_memory() for _ in range(2)]
-    copy_stream = torch.cuda.Stream(device=dev)
-    read_stream = torch.cuda.Stream(device=dev)
-    p.stage_data(hX, hY, copy_stream)
-    for k in range(2):
-        p.swap_data(); p.stage_data(hX, hY, copy_stream); run_period(); p.get_average_async(avg_host[k % 2], read_stream)
-    read_stream.synchronize()
-    barrier()
-    t0 = time.perf_counter()
-    for k in range(args.steps):
-        p.swap_data()                          # pools uploaded during the previous period become current
-        p.stage_data(hX, hY, copy_stream)      # H2D of the next period's pools, overlapped with this period
-        run_period()
-        # D2H of the result: the mean is formed on the training stream, its copy to pinned host memory overlaps
-        # the next period (two host buffers; the last copy is waited for inside the timed region)
-        p.get_average_async(avg_host[k % 2], read_stream)
-    read_stream.synchronize()
-    barrier()
-    copy_stream.synchronize()
-    e2e_s = time.perf_counter() - t0
-    te = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(te, op=dist.ReduceOp.MAX)
-    e2e = {"value": worker_steps / float(te.item()), "unit": METRIC,
-           "h2d_bytes_per_step": hX.numel() * hX.element_size() + hY.numel() * 4,
-           "d2h_bytes_per_step": p.m * 4}
+    if with_e2e:
+        avg_host = [torch.empty(p.m, dtype=torch.float32).pin_memory() for _ in range(2)]
+        copy_stream = torch.cuda.Stream(device=dev)
+        read_stream = torch.cuda.Stream(device=dev)
+        p.stage_data(hX, hY, copy_stream)
+        for k in range(2):
+            p.swap_data(); p.stage_data(hX, hY, copy_stream); run_period(); p.get_average_async(avg_host[k % 2], read_stream)
+        read_stream.synchronize()
+        barrier()
+        t0 = time.perf_counter()
+        for k in range(steps):
+            p.swap_data()                          # pools uploaded during the previous period become current
+            p.stage_data(hX, hY, copy_stream)      # H2D of the next period's pools, overlapped with this period
+            run_period()
+            # D2H of the result: the mean is formed on the training stream, its copy to pinned host memory overlaps
+            # the next period (two host buffers; the last copy is waited for inside the timed region)
+            p.get_average_async(avg_host[k % 2], read_stream)
+        read_stream.synchronize()
+        barrier()
+        copy_stream.synchronize()
+        e2e_s = max_over_ranks(time.perf_counter() - t0, world, dev)
+        res["e2e"] = {"value": worker_steps / e2e_s, "unit": METRIC,
+                      "h2d_bytes_per_step": hX.numel() * hX.element_size() + hY.numel() * 4,
+                      "d2h_bytes_per_step": p.m * 4}
+    p.sync()
+    p.close()
+    return res, (w, X, Y, x0)
 
-    out = {
-        "metric": METRIC, "value": value, "unit": METRIC, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.precision else "f32", "data": "synthetic",
-        "config": workload_config(w, {"l2": "L2 flushed between timed steps" if need_flush else
-                                      "parameter store + shadow larger than L2",
-                                      "multi_gpu": (f"{w.N} workers per rank, node average = local row sums + NCCL all-reduce + restart"
-                                                    if sharded_mode else "single GPU")},
-                                  momentum=args.momentum),
-        "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline,
-        "gemm_tflops": tflops, "gemm_frac_of_bf16_peak": tflops / peaks["bf16_tflops_sustained"],
-    }
-    if rank == 0 and world == 1:
-        if not args.no_sweep:
-            out["averaging_sweep"] = averaging_sweep(torch, binding, peaks)
-        if not args.no_cpu:
-            out["cpu_baseline"] = time_oracle(w, X, Y, x0)
+
+def parse_args(argv=None):
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=24)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", default=DEFAULT_WORKLOAD, choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--scaling", default="weak", choices=["weak", "strong"],
+                    help="several GPUs: weak = N workers per rank (N * G in all), strong = the configuration's N split over the ranks")
+    ap.add_argument("--interval", type=int, default=None, help="override the averaging interval I")
+    ap.add_argument("--workers", type=int, default=None, help="override N (smaller cases for profiler captures)")
+    ap.add_argument("--momentum", type=float, default=None, help="local step with momentum mu (the paper's experiment used 0.9)")
+    ap.add_argument("--update-tile", type=int, default=None, help="tile width of the update kernel (64 or 128)")
+    ap.add_argument("--no-fuse", action="store_true",
+                    help="averaging iterations run as update + stand-alone averaging kernel instead of the fused pass")
+    ap.add_argument("--no-fused-epilogues", action="store_true",
+                    help="softmax-CE gradient and bias steps as kernels of their own instead of GEMM epilogues")
+    ap.add_argument("--no-dx-in-update", action="store_true",
+                    help="separate dX launches instead of forming dZ of the layer below inside the update launch")
+    ap.add_argument("--no-next-forward", action="store_true",
+                    help="layer 1's update does not form the next iteration's a_1")
+    ap.add_argument("--no-early-loads", action="store_true",
+                    help="no tile requests ahead of a kernel's dependency wait")
+    ap.add_argument("--force-sharded", action="store_true",
+                    help="run the multi-GPU code path (sharded workers + all-reduce average) even on one GPU")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the averaging-kernel sweep")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle timing")
+    ap.add_argument("--no-configs", action="store_true", help="skip the short runs of the other configurations")
+    args = ap.parse_args(argv)
+    if args.warmup < 3:
+        args.warmup = 3
+    return args
+
+
+def main(argv=None):
+    args = parse_args(argv)
+    w = synth.WORKLOADS[args.config]
+    if args.interval is not None:
+        w = w.with_(I=args.interval)
+    if args.workers is not None:
+        w = w.with_(N=args.workers, name=f"{w.name}-N{args.workers}")
+    if args.impl == "reference":
+        return run_reference(args, w.with_(pool_samples=max(w.I, 4) * w.B))
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # a plain start that asks for several GPUs: start one rank per GPU and let rank 0 print the line
+        raise SystemExit(launch_ranks(args.gpus, sys.argv[1:] if argv is None else list(argv)).returncode)
+
+    import torch
+    import torch.distributed as dist
+    from paper_1807_06629_b200 import _build
+    rank, local_rank, world = rank_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
     if rank == 0:
-        print(json.dumps(out))
+        _build.build_library()
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    # everything below (torch copies, the library's kernels, the timing events) runs on one side stream:
+    # the library replays captured periods as CUDA graphs, which the legacy default stream cannot capture
+    torch.cuda.set_stream(torch.cuda.Stream(device=dev))
+    sharded_mode = world > 1 or args.force_sharded
+    if sharded_mode:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", "29533")
+        dist.init_process_group("nccl", rank=rank, world_size=world, device_id=torch.device(dev))
+        dist.barrier()            # (also: the library rank 0 may just have built is in place for every rank)
+    from paper_1807_06629_b200 import binding
+    peaks = load_peaks()
+
+    res, (wl, X, Y, x0) = measure_config(torch, w, args, dev, rank, world, args.scaling, args.steps, args.warmup, peaks,
+                                         sharded_mode, with_e2e=True, with_clocks=True)
+    if sharded_mode:
+        how = (f"{args.scaling} scaling: rank g holds {res['n_local']} of the job's {res['n_global']} workers "
+               f"(rows [g*N/G, (g+1)*N/G)); node average = local row sums + NCCL all-reduce + restart")
+    else:
+        how = "single GPU"
+    cfg = workload_config(w.with_(N=res["n_global"], pool_samples=res["pool_samples"]),
+                          {"l2": "L2 flushed between timed steps" if res["need_flush"] else "parameter store + shadow larger than L2",
+                           "multi_gpu": how}, momentum=args.momentum)
+    out = result_line(cfg, res["value"], res["ms_total"], args.steps, args.warmup, world,
+                      args.scaling if world > 1 else "weak", "bf16" if w.precision else "f32")
+    out.update({"clocks": res["clocks"], "e2e": res["e2e"], "gpu_launches": res["launches"], "roofline": res["roofline"],
+                "gemm_tflops": res["gemm_tflops"],
+                "gemm_frac_of_bf16_peak": res["gemm_tflops"] / peaks["bf16_tflops_sustained"]})
+    if world == 1 and not args.force_sharded:
+        default_run = args.config == DEFAULT_WORKLOAD and args.interval is None and args.workers is None
+        if default_run and not args.no_configs:
+            others = []
+            for name, I, k in OTHER_CONFIGS:
+                wo = synth.WORKLOADS[name].with_(I=I)
+                r, _ = measure_config(torch, wo, args, dev, rank, world, "weak", k, 3, peaks, False,
+                                      with_e2e=False, with_clocks=False)
+                rf = r["roofline"]
+                others.append({"workload": name, "N": wo.N, "I": I, "value": round(r["value"], 1), "unit": METRIC,
+                               "steps": k, "ms_per_step": round(r["ms_total"] / k, 4),
+                               "dtype": "bf16" if wo.precision else "f32",
+                               "dominant_family": rf["kernel"], "achieved_GBps": round(rf["achieved"], 1),
+                               "frac_of_measured_copy": round(rf["frac"], 4),
+                               "family_us_per_iteration": rf["family_us_per_iteration"],
+                               "gemm_tflops": round(r["gemm_tflops"], 2),
+                               "l2": "L2 flushed between timed steps" if r["need_flush"] else "store larger than L2"})
+                torch.cuda.empty_cache()
+            out["configs"] = others
+        if not args.no_sweep:
+            out["averaging_sweep"] = averaging_sweep(torch, binding, peaks, dev)
+        if not args.no_cpu:
+            out["cpu_baseline"] = time_oracle(wl, X, Y, x0)
+    if sharded_mode:
+        dist.barrier()
+    if rank == 0:
+        sys.stdout.flush()
+        print(json.dumps(out), flush=True)          # the JSON line is the last thing this run prints
     if sharded_mode:
         dist.destroy_process_group()
 

@@ -214,6 +214,7 @@ class PRSGD:
                                     self.scratch.data_ptr(), self.stream.cuda_stream, C.byref(ctx)))
         self.ctx = ctx
         self._X = self._Y = None
+        self.average_velocity = False
 
     def _call(self, fn, *args):
         with torch.cuda.device(self.device):
@@ -339,6 +340,7 @@ class PRSGD:
         with torch.cuda.device(self.device):
             self.velocity = torch.empty(self.N * self.m_pad, dtype=torch.float32, device=self.device)
         self._call(lib.prsgd_enable_momentum, mu, self.velocity.data_ptr(), 1 if average_velocity else 0)
+        self.average_velocity = bool(average_velocity)
 
     def get_velocity_stacked(self) -> np.ndarray:
         out = np.empty((self.N, self.m), dtype=np.float32)

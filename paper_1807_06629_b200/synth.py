@@ -109,8 +109,11 @@ def _teacher_logits(dims: Sequence[int], theta: np.ndarray, X: np.ndarray) -> np
     return a
 
 
-def make_pools(w: Workload) -> Tuple[np.ndarray, np.ndarray]:
+def make_pools(w: Workload, first: int = 0) -> Tuple[np.ndarray, np.ndarray]:
     """Per-worker data pools X [N, P, d_0] fp32 and labels Y [N, P] int32.
+
+    Row k holds the pool of worker first + k (a rank that owns a shard of a larger job asks for its
+    own workers only; worker i's pool does not depend on which rank generates it).
 
     x ~ N(mu_i, I) with mu_i = mean_shift * N(0, I) per worker (mu_i = 0 when
     mean_shift = 0); label = argmax of a fixed random teacher MLP of the same
@@ -121,7 +124,7 @@ def make_pools(w: Workload) -> Tuple[np.ndarray, np.ndarray]:
     X = np.empty((w.N, w.pool_samples, d0), dtype=np.float32)
     Y = np.empty((w.N, w.pool_samples), dtype=np.int32)
     for i in range(w.N):
-        g = _rng(w.seed, 3, i)
+        g = _rng(w.seed, 3, first + i)
         xi = g.standard_normal((w.pool_samples, d0), dtype=np.float32)
         if w.mean_shift != 0.0:
             mu = (w.mean_shift * g.standard_normal(d0)).astype(np.float32)

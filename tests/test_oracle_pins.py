@@ -286,6 +286,36 @@ def test_alg2_with_constant_schedule_is_alg1():
     assert np.allclose(a, b, atol=1e-14)
 
 
+def test_alg2_varying_schedule_matches_the_closed_form_per_epoch():
+    """Algorithm 2 with Theorem 2's K^s = ceil(s^(1/3) / N), gamma^s = N / s^(2/3) (scaled) on the quadratic
+    instance F_i(x) = a_i/2 |x - c_i|^2: epoch s starts every worker at the node average y of the previous
+    epoch's end points and takes K^s gradient steps with rate gamma^s, so x_i = c_i + (1 - gamma^s a_i)^(K^s) (y - c_i).
+    The epochs' rates and lengths both change inside the run, so using the wrong epoch's rate (the first one's
+    throughout, or the neighbour's) or the wrong epoch length cannot pass."""
+    rng = np.random.default_rng(11)
+    N, m, S, scale = 2, 5, 30, 0.05
+    a, c = rng.uniform(0.5, 2.0, N), rng.standard_normal((N, m))
+    start = rng.standard_normal((N, m))                  # workers need not start equal: epoch 1 averages first
+    Ks = [math.ceil(round(s ** (1 / 3), 12) / N) for s in range(1, S + 1)]     # written out here, not taken from the oracle
+    gs = [scale * N / (s ** (1 / 3)) ** 2 for s in range(1, S + 1)]
+    assert Ks[7] == 1 and Ks[8] == 2 and Ks[26] == 2 and Ks[27] == 2 and len(set(Ks)) == 2
+
+    def closed_form(Ks, gs):
+        x = start.copy()
+        for K, g in zip(Ks, gs):
+            y = x.mean(0)
+            x = np.stack([c[i] + (1 - g * a[i]) ** K * (y - c[i]) for i in range(N)])
+        return x
+    sched = [(K, g * scale) for (K, g) in orc.alg2_schedule(N, S)]
+    got = orc.pr_sgd_time_varying(start, sched, _quad(a, c))
+    assert np.allclose(got, closed_form(Ks, gs), atol=1e-13)
+    assert np.abs(got[0] - got[1]).max() > 1e-3          # the end points are not averaged
+    # the pin discriminates: the mistakes it is there to catch move the result far beyond the tolerance
+    for wrong in (closed_form(Ks, [gs[0]] * S), closed_form(Ks, gs[1:] + gs[-1:]), closed_form(Ks, gs[:1] + gs[:-1]),
+                  closed_form([1] * S, gs), closed_form(Ks[1:] + Ks[-1:], gs)):
+        assert np.abs(wrong - got).max() > 1e-6
+
+
 def test_alg3_with_equal_lengths_is_alg1_and_slow_workers_stand_still():
     w, X, Y, x0 = _small_mlp_problem(N=3)
     fn = orc.mlp_grad_fn(w.dims, X, Y, w.B, w.seed)
@@ -335,6 +365,43 @@ def test_momentum_brute_force_and_velocity_choices():
     # mean dynamics with momentum on a non-averaging iteration: xbar moves by -gamma * mean(v)
     x3, v3 = orc.pr_sgd_momentum(x, v, g, mu, 2, 1, _quad(a, c), t0=4)
     assert np.allclose(x3.mean(0), x.mean(0) - g * v3.mean(0), atol=1e-15)
+
+
+def test_averaged_momentum_buffers_value_pins():
+    """average_velocity=True.  (a) Equal curvature: per worker (x_i - c_i, v_i) <- M (x_i - c_i, v_i) with
+    M = [[1 - gamma a, -gamma mu], [a, mu]]; the map is linear, so the worker mean obeys it with c replaced by
+    the mean of the c_i, and after an averaging iteration with averaged buffers EVERY worker holds that mean
+    state: x_i = cbar + (M^T z0)_0, v_i = (M^T z0)_1 with z0 = (y0 - cbar, 0).  (b) Different curvatures:
+    scalar recurrences worked in the test, buffers averaged by hand at t = 2, 4."""
+    rng = np.random.default_rng(12)
+    N, m, a, gam, mu, I, T = 4, 3, 1.3, 0.1, 0.9, 3, 9
+    c, y0 = rng.standard_normal((N, m)), rng.standard_normal(m)
+    x, v = orc.pr_sgd_momentum(np.tile(y0, (N, 1)), np.zeros((N, m)), gam, mu, I, T, _quad(np.full(N, a), c),
+                               average_velocity=True)
+    M = np.linalg.matrix_power(np.array([[1 - gam * a, -gam * mu], [a, mu]]), T)
+    cbar = c.mean(0)
+    want_x, want_v = cbar + M[0, 0] * (y0 - cbar), M[1, 0] * (y0 - cbar)
+    assert np.allclose(x, want_x[None, :], atol=1e-13) and np.allclose(v, want_v[None, :], atol=1e-13)
+    xl, vl = orc.pr_sgd_momentum(np.tile(y0, (N, 1)), np.zeros((N, m)), gam, mu, I, T, _quad(np.full(N, a), c))
+    assert np.allclose(xl, want_x[None, :], atol=1e-13)           # same models (linear map, equal curvature) ...
+    assert np.abs(vl - want_v[None, :]).max() > 1e-3              # ... but local buffers stay apart
+    assert np.allclose(vl.mean(0), want_v, atol=1e-13)
+    # (b)
+    aa, cc, g, mu2 = [1.0, 3.0], [2.0, -1.0], 0.1, 0.5
+    x0_ = x1_ = 0.5
+    v0_ = v1_ = 0.0
+    for t in range(1, 5):
+        v0_ = mu2 * v0_ + aa[0] * (x0_ - cc[0]); x0_ -= g * v0_
+        v1_ = mu2 * v1_ + aa[1] * (x1_ - cc[1]); x1_ -= g * v1_
+        if t % 2 == 0:
+            x0_ = x1_ = (x0_ + x1_) / 2
+            v0_ = v1_ = (v0_ + v1_) / 2
+    x2, v2 = orc.pr_sgd_momentum(np.full((2, 1), 0.5), np.zeros((2, 1)), g, mu2, 2, 4,
+                                 _quad(np.array(aa), np.array(cc)[:, None]), average_velocity=True)
+    assert np.allclose(x2[:, 0], [x0_, x1_], atol=1e-15) and np.allclose(v2[:, 0], [v0_, v1_], atol=1e-15)
+    xk, _ = orc.pr_sgd_momentum(np.full((2, 1), 0.5), np.zeros((2, 1)), g, mu2, 2, 4,
+                                _quad(np.array(aa), np.array(cc)[:, None]))
+    assert abs(xk[0, 0] - x2[0, 0]) > 1e-4                        # with different curvatures the choice changes the models
 
 
 # ------------------------------------------------------- planted mistakes are caught

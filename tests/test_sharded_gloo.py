@@ -13,38 +13,7 @@ import torch.multiprocessing as mp
 
 from oracle import prsgd_oracle as orc
 from paper_1807_06629_b200 import sharded, synth
-
-
-class OracleEngine:
-    """Stand-in shard: rows first..first+count of the oracle's state, padded to a multiple of 4 columns."""
-
-    def __init__(self, w, X, Y, x0, first, count):
-        self.w, self.first, self.count, self.t = w, first, count, 0
-        self.m = x0.size
-        self.m_pad = (self.m + 3) // 4 * 4
-        self.x = np.tile(x0.astype(np.float64), (count, 1))
-        g = orc.mlp_grad_fn(w.dims, X.astype(np.float64), Y, w.B, w.seed)
-        self.fn = lambda i, t, xi: g(self.first + i, t, xi)      # local row i is global worker first + i
-
-    def new_row(self):
-        return torch.zeros(self.m_pad, dtype=torch.float64)
-
-    def get_step(self):
-        return self.t
-
-    def local_steps(self, k):
-        self.x = orc.pr_sgd(self.x, self.w.gamma, 0, k, self.fn, t0=self.t)
-        self.t += k
-
-    def partial_sum(self, row, c0, n):
-        s = np.zeros(self.m_pad)
-        s[:self.m] = self.x.sum(0)
-        row[c0:c0 + n] = torch.from_numpy(s[c0:c0 + n])
-
-    def assign_rows(self, row, divisor, c0, n):
-        hi = min(c0 + n, self.m)
-        if hi > c0:
-            self.x[:, c0:hi] = (row[c0:hi].numpy() / divisor)[None, :]
+from helpers import OracleEngine
 
 
 def _worker(rank, world, port, q):
@@ -59,7 +28,10 @@ def _worker(rank, world, port, q):
         job = sharded.ShardedPRSGD(eng, w.N, w.I, chunks=3)
         job.local_steps(2)
         job.local_steps(5)            # crosses the averages after t = 3 and t = 6
-        q.put((rank, first, count, eng.x.copy(), eng.t))
+        # Algorithm 2 over the ranks: K^s and gamma^s come from the job's N (5), not from the shard's 3 or 2
+        eng2 = OracleEngine(w, X, Y, x0, first, count)
+        sharded.ShardedPRSGD(eng2, w.N, 0, chunks=2).run_time_varying(1, 130, 0.02)
+        q.put((rank, first, count, eng.x.copy(), eng.t, eng2.x.copy(), eng2.t))
     finally:
         dist.destroy_process_group()
 
@@ -72,7 +44,6 @@ def test_shard_bounds_and_chunks():
     assert sharded.column_chunks(8, 16) == [(0, 4), (4, 4)]
 
 
-@pytest.mark.timeout(180)
 def test_two_ranks_reproduce_the_single_process_run():
     s = socket.socket(); s.bind(("127.0.0.1", 0)); port = s.getsockname()[1]; s.close()
     ctx = mp.get_context("spawn")
@@ -92,3 +63,9 @@ def test_two_ranks_reproduce_the_single_process_run():
     assert [r[4] for r in res] == [7, 7]
     assert got.shape == want.shape and np.allclose(got, want, atol=1e-13)
     assert np.abs(got[0] - got[4]).max() > 1e-6        # t = 7 is one step past the average: workers differ again
+    sched = [(K, g * 0.02) for (K, g) in orc.alg2_schedule(w.N, 130)]
+    assert max(K for K, _ in sched) == 2               # (K^s changes inside the run: ceil(s^(1/3) / 5) = 2 from s = 126)
+    want2 = orc.pr_sgd_time_varying(np.tile(x0, (w.N, 1)), sched, orc.mlp_grad_fn(w.dims, X.astype(np.float64), Y, w.B, w.seed))
+    got2 = np.concatenate([r[5] for r in res])
+    assert [r[6] for r in res] == [sum(K for K, _ in sched)] * 2
+    assert np.allclose(got2, want2, atol=1e-9)              # (the library returns gamma^s as a float)
