@@ -225,39 +225,68 @@ def ncu_traffic_per_launch(workload: str, family: str, N: int):
 
 
 # ----------------------------------------------------------------------------- byte model
-def algorithmic_bytes(w: synth.Workload, m_pad: int, momentum: bool = False, next_forward: bool = False,
-                      dx_in_update: bool = False, sms: int = 148) -> dict:
-    """Algorithmic HBM bytes of one local iteration of all N workers, per kernel family.
+def period_bytes(w: synth.Workload, m_pad: int, sms: int = 148, momentum: bool = False, fused_average: bool = True,
+                 fused_epilogues: bool = True, next_forward: bool = True, dx_in_update: bool = True) -> dict:
+    """Algorithmic HBM bytes and launch counts of ONE averaging period (prsgd_local_steps(I) from a period
+    boundary) of all N workers, per kernel family: {family: [bytes, launches]}.
 
-    bf16 path: forward reads the bf16 shadow (2 B/param); dX reads it again for every layer but
-    the first; the update reads and writes the fp32 master (4 + 4) and writes the shadow (2);
-    activations / deltas are read and written once per use.  fp32 path: 4 B where bf16 has 2, no shadow.
-    With momentum the update also reads and writes the fp32 momentum buffer (+8 B/param).
-    The stand-alone average reads and writes the store once (8 B/word, +2 for the shadow).
-    next_forward: layer 1's update also forms the next a_1, so it does not write W_1's shadow (-2 B/param) but
-    reads a second minibatch and writes a_1; the forward family then has no layer-1 launch.
-    dx_in_update: layers >= 2 with enough column blocks form dZ of the layer below inside the update launch
-    (no second read of the bf16 weights; the mask read and the dZ write move to the update family).
+    The unit is one parameter of one worker.  bf16 path: a forward GEMM reads the bf16 copy (2 B/param), a dX
+    GEMM reads it again (layers >= 2), an update reads and writes the fp32 master (4 + 4) and writes the bf16
+    copy (2) (+ 4 + 4 for the momentum buffer); activations, deltas and biases are charged once per use.  fp32
+    path: 4 B where bf16 has 2, no bf16 copy.  The launches follow the library's own rules: on a plain
+    iteration the update of a layer >= 2 also forms dZ of the layer below when the layer has enough column
+    blocks (no dX launch: the mask read and the dZ write move to the update family), and layer 1's update also
+    forms the next a_1 when another iteration follows (no write of W_1's bf16 copy, a second minibatch read,
+    a_1 written; the next iteration has no layer-1 forward launch); on the averaging iteration a layer with
+    enough tiles takes the fused update + average (same bytes as a plain update, dX a launch of its own),
+    a smaller one the plain update followed by the node average of its weight segment (8 + 2 B/param).
+    Without the fused form the stand-alone average reads and writes the whole store (8 B/word, + 2 B bf16 copy).
     """
-    e = 2 if w.precision == 1 else 4
-    N, B, d = w.N, w.B, w.dims
+    bf = w.precision == 1
+    e = 2 if bf else 4
+    N, B, d, I = w.N, w.B, w.dims, max(w.I, 1)
     L = len(d) - 1
-    fwd = dx = upd = 0
-    for l in range(1, L + 1):
-        wl = d[l] * d[l - 1]
-        fwd += N * (wl * e + d[l] * 4 + B * d[l - 1] * e + B * d[l] * (e if l < L else 4))
-        if l > 1 and dx_in_update and (((d[l - 1] + 63) // 64) * N >= 3 * sms or d[l] <= 128):
-            upd += N * B * d[l - 1] * 2 * e
-        elif l > 1:
-            dx += N * (wl * e + B * d[l] * e + B * d[l - 1] * 2 * e)
-        upd += N * ((wl + d[l]) * (8 + (2 if w.precision == 1 else 0) + (8 if momentum else 0)) + B * (d[l] + d[l - 1]) * e)
-    avg = N * m_pad * (8 + (2 if w.precision == 1 else 0))
-    upd_plain = upd
-    if next_forward:
-        upd += N * (-d[1] * d[0] * 2 + B * d[0] * e + B * d[1] * e + d[1] * 4)
-        fwd -= N * (d[1] * d[0] * e + d[1] * 4 + B * d[0] * e + B * d[1] * e)
-    return {"forward": fwd, "dx": dx, "update": upd, "update_average": upd_plain, "average": avg,
-            "softmax": N * B * d[L] * (4 + 4 + e)}
+    upd_b = 8 + (2 if bf else 0) + (8 if momentum else 0)
+    epi = bf and fused_epilogues and d[L] <= 128
+    fam = {k: [0, 0] for k in ("forward", "softmax", "dx", "update", "update_average", "average", "misc")}
+
+    def add(name, nbytes):
+        fam[name][0] += nbytes
+        fam[name][1] += 1
+    a1_ready = False
+    for j in range(1, I + 1):
+        averaging = w.I > 0 and j == I
+        fuse = averaging and fused_average and not momentum
+        nxt = bf and next_forward and j < I and not averaging and L > 1 and epi
+        for l in range(2 if a1_ready else 1, L + 1):
+            add("forward", N * (d[l] * d[l - 1] * e + d[l] * 4 + B * d[l - 1] * e + B * d[l] * (e if l < L else 4)))
+        a1_ready = False
+        if not epi:
+            add("softmax", N * B * d[L] * (4 + 4 + e))
+        for l in range(L, 0, -1):
+            wl = d[l] * d[l - 1]
+            tiles64 = ((d[l] + 127) // 128) * ((d[l - 1] + 63) // 64)
+            fuse_l = fuse and (not bf or 2 * tiles64 >= sms)
+            folds = bf and epi and dx_in_update and (((d[l - 1] + 63) // 64) * N >= 3 * sms or d[l] <= 128)
+            upd = N * ((wl + d[l]) * upd_b + B * (d[l] + d[l - 1]) * e)
+            if l > 1 and folds and not fuse_l:
+                add("update", upd + N * B * d[l - 1] * 2 * e)
+            else:
+                if l > 1:
+                    add("dx", N * (wl * e + B * d[l] * e + B * d[l - 1] * 2 * e))
+                if l == 1 and nxt:
+                    upd += N * (-wl * 2 + B * d[0] * e + B * d[1] * e + d[1] * 4)
+                    a1_ready = True
+                add("update_average" if fuse_l else "update", upd)
+            if bf and fuse and not fuse_l:
+                add("average", N * wl * 10)
+        if not epi and bf:
+            add("misc", 0)
+        if bf and fuse:
+            add("misc", 0)
+        if averaging and not fuse:
+            add("average", N * m_pad * (8 + (2 if bf else 0)))
+    return fam
 
 
 def flops_per_worker_step(w: synth.Workload) -> int:
@@ -445,27 +474,28 @@ def measure_config(torch, w_cfg, args, dev, rank, world, scaling, steps, warmup,
         run_period()
     prof = p.get_profile()
     p.set_option(binding.OPT_PROFILE, 0)
-    L = len(w.dims) - 1
-    # iterations 1..I-1 of a period run layer 1's update with the next forward folded in (tensor-core path)
-    next_fwd = (w.precision == 1 and L > 1 and w.I > 1 and w.dims[L] <= 128
-                and not args.no_next_forward and not args.no_fused_epilogues)
-    dx_in_upd = (w.precision == 1 and w.dims[L] <= 128 and not args.no_dx_in_update
-                 and not args.no_fused_epilogues)
-    bytes_iter = algorithmic_bytes(w, p.m_pad, args.momentum is not None, next_fwd, dx_in_upd,
-                                   torch.cuda.get_device_properties(dev).multi_processor_count)
-    fams = {k: v for k, v in prof.items() if v[1] > 0 and k in bytes_iter}
+    fam_model = period_bytes(w, p.m_pad, torch.cuda.get_device_properties(dev).multi_processor_count,
+                             momentum=args.momentum is not None, fused_average=not args.no_fuse,
+                             fused_epilogues=not args.no_fused_epilogues, next_forward=not args.no_next_forward,
+                             dx_in_update=not args.no_dx_in_update)
+    if sharded_mode:          # a shard's period: I plain iterations, then the average as passes of their own
+        fam_model = period_bytes(w.with_(I=0), p.m_pad, torch.cuda.get_device_properties(dev).multi_processor_count,
+                                 momentum=args.momentum is not None, fused_epilogues=not args.no_fused_epilogues,
+                                 next_forward=not args.no_next_forward, dx_in_update=not args.no_dx_in_update)
+        fam_model = {k: [v[0] * w.I, v[1] * w.I] for k, v in fam_model.items()}
+        fam_model["average"] = [w.N * p.m_pad * (4 + 4 + (2 if w.precision == 1 else 0)), 8]
+    fams = {k: v for k, v in prof.items() if v[1] > 0 and fam_model.get(k, [0, 0])[0] > 0}
     dom = max(fams, key=lambda k: fams[k][0])
-    per_iter_launches = {"forward": L - 1 if next_fwd else L, "dx": L - 1, "update": L, "update_average": L,
-                         "average": 1, "softmax": 1}[dom]
     dom_ms, dom_launches = fams[dom]
-    iters_seen = dom_launches / max(per_iter_launches, 1)
-    achieved = bytes_iter[dom] * iters_seen / (dom_ms * 1e-3) / 1e9
+    dom_bytes, dom_per_period = fam_model[dom]
+    achieved = dom_bytes * steps / (dom_ms * 1e-3) / 1e9
     prof_sum = sum(x[0] for x in prof.values())
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"] + " copy bandwidth",
                 "traffic": ncu_traffic_per_launch(w_cfg.name, dom, w.N),
                 "avg_launch_us": 1e3 * dom_ms / dom_launches,
-                "algorithmic_bytes_per_launch": bytes_iter[dom] / per_iter_launches,
+                "algorithmic_bytes_per_launch": dom_bytes / max(dom_per_period, 1),
+                "launches_per_period": {"counted": dom_launches / steps, "model": dom_per_period},
                 "family_us_per_iteration": {k: round(1e3 * v[0] / (steps * max(w.I, 1)), 2) for k, v in prof.items() if v[1]},
                 "share_of_step_time": {k: round(v[0] / prof_sum, 4) for k, v in prof.items() if v[1]}}
     tflops = flops_per_worker_step(w) * value / world / 1e12

@@ -405,6 +405,10 @@ struct UpdateArgs {
 };
 
 constexpr int kUpdThreads = 224;          // warp 0 loader, 1 MMA, 2 storer, 3..6 epilogue
+// The two folded update kernels end every block of tiles (a column block's dX, a row block's next forward)
+// with an epilogue of its own; four more warps (7..10) run it, so that the tile epilogue warps go straight
+// on to the next block's tiles and the weight stream does not pause at a block boundary.
+constexpr int kUpdBlkThreads = 352;
 
 // One pipeline stage of the update kernel for a 128 x TN tile: the fp32 master tile (TN/32 boxes of
 // 128 x 32) followed by a region that first holds the operands (two dZ boxes and TN/64 activation
@@ -759,7 +763,7 @@ template <int TN, bool MOM> struct UpdNextCfg {
 };
 
 template <int TN, bool MOM>
-__global__ void __launch_bounds__(kUpdThreads, 1) tc_update_next_kernel(const __grid_constant__ CUtensorMap mapDelta,
+__global__ void __launch_bounds__(kUpdBlkThreads, 1) tc_update_next_kernel(const __grid_constant__ CUtensorMap mapDelta,
                                                                         const __grid_constant__ CUtensorMap mapPool,
                                                                         const __grid_constant__ CUtensorMap mapMaster,
                                                                         const __grid_constant__ CUtensorMap mapVel,
@@ -938,19 +942,17 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_next_kernel(const __
       }
     }
     tma_wait_group0();
-  } else if (warp >= 3) {
-    // ---------------- epilogue: row r of the tile <-> TMEM lane r
+  } else if (warp >= 3 && warp < 7) {
+    // ---------------- tile epilogue: row r of the tile <-> TMEM lane r
     const int q4 = warp & 3;
     const int r = q4 * 32 + lane;
     const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
     const uint32_t row_off = (uint32_t)r * 128u;
     const uint32_t sw = (uint32_t)(r & 7);
-    const int batches = a.B / 16;
-    uint32_t it = 0, rbi = 0;
+    uint32_t it = 0;
     bool ok = true;
     for (int rb = blockIdx.x; rb < total_rb && ok; rb += gridDim.x) {
-      const int n = rb / a.tiles_m, m = (rb % a.tiles_m) * 128 + r;
-      if (!item_active(n)) continue;
+      if (!item_active(rb / a.tiles_m)) continue;
       for (int kb = 0; kb < a.tiles_n; ++kb, ++it) {
         const int s = it % S;
         const uint32_t ph = (it / S) & 1u;
@@ -991,8 +993,19 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_next_kernel(const __
         fence_proxy_async();
         mbar_arrive(tile_ready(s));
       }
-      if (!ok) break;
-      // forward epilogue of the row block: a_1[., m] = relu(z + b_1[m]) for the next iteration
+    }
+  } else if (warp >= 7) {
+    // ---------------- block epilogue: forward epilogue of every row block, a_1[., m] = relu(z + b_1[m]) for
+    // the next iteration, while the tile epilogue warps are already on the next row block
+    const int q4 = warp & 3;
+    const int r = q4 * 32 + lane;
+    const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
+    const int batches = a.B / 16;
+    uint32_t rbi = 0;
+    bool ok = true;
+    for (int rb = blockIdx.x; rb < total_rb && ok; rb += gridDim.x) {
+      const int n = rb / a.tiles_m, m = (rb % a.tiles_m) * 128 + r;
+      if (!item_active(n)) continue;
       const int q = rbi & 1;
       const bool valid = m < a.M_total;
       const float bias = valid ? a.bias[(int64_t)n * a.bias_stride + m] : 0.f;
@@ -1077,7 +1090,7 @@ template <int TN, bool MOM> struct UpdDxCfg {
 };
 
 template <int TN, bool MOM>
-__global__ void __launch_bounds__(kUpdThreads, 1) tc_update_dx_kernel(const __grid_constant__ CUtensorMap mapDelta,
+__global__ void __launch_bounds__(kUpdBlkThreads, 1) tc_update_dx_kernel(const __grid_constant__ CUtensorMap mapDelta,
                                                                       const __grid_constant__ CUtensorMap mapAct,
                                                                       const __grid_constant__ CUtensorMap mapMaster,
                                                                       const __grid_constant__ CUtensorMap mapShadow,
@@ -1266,19 +1279,17 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_dx_kernel(const __gr
       }
     }
     tma_wait_group0();
-  } else if (warp >= 3) {
-    // ---------------- epilogue: row r of the tile <-> TMEM lane r
+  } else if (warp >= 3 && warp < 7) {
+    // ---------------- tile epilogue: row r of the tile <-> TMEM lane r
     const int q4 = warp & 3;
     const int r = q4 * 32 + lane;
     const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
     const uint32_t row_off = (uint32_t)r * 128u;
     const uint32_t sw = (uint32_t)(r & 7);
-    const int batches = a.B / 16;
-    uint32_t it = 0, cbi = 0;
+    uint32_t it = 0;
     bool ok = true;
     for (int cb = blockIdx.x; cb < total_cb && ok; cb += gridDim.x) {
-      const int n = cb / a.tiles_n, n0 = (cb % a.tiles_n) * TN;
-      if (!item_active(n)) continue;
+      if (!item_active(cb / a.tiles_n)) continue;
       for (int mb = 0; mb < a.tiles_m; ++mb, ++it) {
         const int s = it % S;
         const uint32_t ph = (it / S) & 1u;
@@ -1326,8 +1337,20 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_dx_kernel(const __gr
         fence_proxy_async();
         mbar_arrive(tile_ready(s));
       }
-      if (!ok) break;
-      // dX epilogue of the column block: feature c = n0 + r (lanes 0..63 only)
+    }
+  } else if (warp >= 7) {
+    // ---------------- block epilogue: dX epilogue of every column block (ReLU mask, bf16 dZ_{l-1}, bias step of
+    // layer l-1), feature c = n0 + r (lanes 0..TN-1 only), while the tile epilogue warps are already on the
+    // next column block
+    const int q4 = warp & 3;
+    const int r = q4 * 32 + lane;
+    const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
+    const int batches = a.B / 16;
+    uint32_t cbi = 0;
+    bool ok = true;
+    for (int cb = blockIdx.x; cb < total_cb && ok; cb += gridDim.x) {
+      const int n = cb / a.tiles_n, n0 = (cb % a.tiles_n) * TN;
+      if (!item_active(n)) continue;
       const int q = cbi & 1;
       const int cfeat = n0 + r;
       const bool valid = r < TN && cfeat < a.M_total;
@@ -1646,7 +1669,7 @@ inline void tc_launch_update_dx_m(prsgd_ctx* c, int l) {
   const int items = a.tiles_n * c->N;
   const int grid = items < st->num_sms ? items : st->num_sms;
   const TcLayerMaps& mp = st->layer[l - 1];
-  launch_pdl(tc_update_dx_kernel<TN, MOM>, dim3(grid), kUpdThreads, UpdDxCfg<TN, MOM>::smem(c->B), c->stream, mp.delta_out,
+  launch_pdl(tc_update_dx_kernel<TN, MOM>, dim3(grid), kUpdBlkThreads, UpdDxCfg<TN, MOM>::smem(c->B), c->stream, mp.delta_out,
              mp.act_in, mp.master, mp.shadow_k, MOM ? mp.velocity : mp.master, a);
 }
 
@@ -1680,7 +1703,7 @@ inline void tc_launch_update_next_tn(prsgd_ctx* c, const DrawArgs& dr) {
   const int items = a.tiles_m * c->N;
   const int grid = items < st->num_sms ? items : st->num_sms;
   const TcLayerMaps& mp = st->layer[0];
-  launch_pdl(tc_update_next_kernel<TN, MOM>, dim3(grid), kUpdThreads, UpdNextCfg<TN, MOM>::smem(c->B), c->stream, mp.delta_out,
+  launch_pdl(tc_update_next_kernel<TN, MOM>, dim3(grid), kUpdBlkThreads, UpdNextCfg<TN, MOM>::smem(c->B), c->stream, mp.delta_out,
              mp.act_in, mp.master, MOM ? mp.velocity : mp.master, a);
 }
 
