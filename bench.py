@@ -226,7 +226,8 @@ def ncu_traffic_per_launch(workload: str, family: str, N: int):
 
 # ----------------------------------------------------------------------------- byte model
 def period_bytes(w: synth.Workload, m_pad: int, sms: int = 148, momentum: bool = False, fused_average: bool = True,
-                 fused_epilogues: bool = True, next_forward: bool = True, dx_in_update: bool = True) -> dict:
+                 fused_epilogues: bool = True, next_forward: bool = True, dx_in_update=True,
+                 shared_restart: bool = True) -> dict:
     """Algorithmic HBM bytes and launch counts of ONE averaging period (prsgd_local_steps(I) from a period
     boundary) of all N workers, per kernel family: {family: [bytes, launches]}.
 
@@ -258,8 +259,11 @@ def period_bytes(w: synth.Workload, m_pad: int, sms: int = 148, momentum: bool =
         averaging = w.I > 0 and j == I
         fuse = averaging and fused_average and not momentum
         nxt = bf and next_forward and j < I and not averaging and L > 1 and epi
+        # the first iteration of a period starts from N equal rows: launches that only read the weights (and the
+        # fused update + average) read one copy for all workers
+        wr = 1 if (bf and shared_restart and j == 1 and w.I > 0) else N
         for l in range(2 if a1_ready else 1, L + 1):
-            add("forward", N * (d[l] * d[l - 1] * e + d[l] * 4 + B * d[l - 1] * e + B * d[l] * (e if l < L else 4)))
+            add("forward", wr * d[l] * d[l - 1] * e + N * (d[l] * 4 + B * d[l - 1] * e + B * d[l] * (e if l < L else 4)))
         a1_ready = False
         if not epi:
             add("softmax", N * B * d[L] * (4 + 4 + e))
@@ -267,16 +271,18 @@ def period_bytes(w: synth.Workload, m_pad: int, sms: int = 148, momentum: bool =
             wl = d[l] * d[l - 1]
             tiles64 = ((d[l] + 127) // 128) * ((d[l - 1] + 63) // 64)
             fuse_l = fuse and (not bf or 2 * tiles64 >= sms)
-            folds = bf and epi and dx_in_update and (((d[l - 1] + 63) // 64) * N >= 3 * sms or d[l] <= 128)
+            folds = bf and epi and dx_in_update and (dx_in_update == 2 or ((d[l - 1] + 63) // 64) * N >= 3 * sms or d[l] <= 128)
             upd = N * ((wl + d[l]) * upd_b + B * (d[l] + d[l - 1]) * e)
             if l > 1 and folds and not fuse_l:
                 add("update", upd + N * B * d[l - 1] * 2 * e)
             else:
                 if l > 1:
-                    add("dx", N * (wl * e + B * d[l] * e + B * d[l - 1] * 2 * e))
+                    add("dx", wr * wl * e + N * (B * d[l] * e + B * d[l - 1] * 2 * e))
                 if l == 1 and nxt:
                     upd += N * (-wl * 2 + B * d[0] * e + B * d[1] * e + d[1] * 4)
                     a1_ready = True
+                if fuse_l:
+                    upd -= (N - wr) * wl * 4
                 add("update_average" if fuse_l else "update", upd)
             if bf and fuse and not fuse_l:
                 add("average", N * wl * 10)
@@ -432,9 +438,12 @@ def measure_config(torch, w_cfg, args, dev, rank, world, scaling, steps, warmup,
         p.enable_momentum(args.momentum)
     for flag, opt in ((args.no_fuse, binding.OPT_FUSED_AVERAGE), (args.no_dx_in_update, binding.OPT_DX_IN_UPDATE),
                       (args.no_next_forward, binding.OPT_NEXT_FORWARD), (args.no_early_loads, binding.OPT_EARLY_LOADS),
-                      (args.no_fused_epilogues, binding.OPT_FUSED_EPILOGUES)):
+                      (args.no_fused_epilogues, binding.OPT_FUSED_EPILOGUES),
+                      (args.no_shared_restart, binding.OPT_SHARED_RESTART)):
         if flag:
             p.set_option(opt, 0)
+    if args.fold_all_dx:
+        p.set_option(binding.OPT_DX_IN_UPDATE, 2)
     working_set = p.params.numel() * 4 + (p.shadow.numel() * 2 if p.shadow is not None else 0)
     need_flush = working_set <= 2 * L2_BYTES
     flush = torch.empty(3 * L2_BYTES // 4, dtype=torch.float32, device=dev) if need_flush else None
@@ -477,7 +486,8 @@ def measure_config(torch, w_cfg, args, dev, rank, world, scaling, steps, warmup,
     fam_model = period_bytes(w, p.m_pad, torch.cuda.get_device_properties(dev).multi_processor_count,
                              momentum=args.momentum is not None, fused_average=not args.no_fuse,
                              fused_epilogues=not args.no_fused_epilogues, next_forward=not args.no_next_forward,
-                             dx_in_update=not args.no_dx_in_update)
+                             dx_in_update=0 if args.no_dx_in_update else (2 if args.fold_all_dx else 1),
+                             shared_restart=not args.no_shared_restart)
     if sharded_mode:          # a shard's period: I plain iterations, then the average as passes of their own
         fam_model = period_bytes(w.with_(I=0), p.m_pad, torch.cuda.get_device_properties(dev).multi_processor_count,
                                  momentum=args.momentum is not None, fused_epilogues=not args.no_fused_epilogues,
@@ -555,6 +565,10 @@ def parse_args(argv=None):
                     help="softmax-CE gradient and bias steps as kernels of their own instead of GEMM epilogues")
     ap.add_argument("--no-dx-in-update", action="store_true",
                     help="separate dX launches instead of forming dZ of the layer below inside the update launch")
+    ap.add_argument("--fold-all-dx", action="store_true",
+                    help="form dZ of the layer below inside the update launch for every layer, whatever its size")
+    ap.add_argument("--no-shared-restart", action="store_true",
+                    help="the iteration after an average reads every worker's own copy of the common point")
     ap.add_argument("--no-next-forward", action="store_true",
                     help="layer 1's update does not form the next iteration's a_1")
     ap.add_argument("--no-early-loads", action="store_true",

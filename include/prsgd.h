@@ -288,6 +288,14 @@ int prsgd_get_velocity_stacked(prsgd_ctx* ctx, float* dst, int dst_on_device);
  * for a layer that takes the fused update + average on an averaging iteration.  Same bits as the
  * separate launches (also with momentum and with a worker mask). */
 #define PRSGD_OPT_DX_IN_UPDATE 8
+/* PRSGD_OPT_SHARED_RESTART (default 1, tensor-core path): right after a node average every worker holds the
+ * same point (the restart of Algorithm 1), so the iteration that follows reads worker 0's weights for every
+ * worker wherever a launch only reads them (forward, dX) or reads all N copies of a tile before it writes any
+ * (the fused update + average): one HBM read serves all N workers.  The library keeps track of whether the
+ * rows are equal (after prsgd_average, an averaging iteration, prsgd_set_params for all workers, or
+ * prsgd_assign_rows calls that cover the row in ascending order); a caller that writes into the store
+ * through its own pointer instead of these calls must switch the option off.  Same bits either way. */
+#define PRSGD_OPT_SHARED_RESTART 10
 /* PRSGD_OPT_CHECK_FINITE (default 0): when 1, prsgd_sync also runs prsgd_check_finite. */
 #define PRSGD_OPT_CHECK_FINITE 9
 int prsgd_set_option(prsgd_ctx* ctx, int32_t option, int64_t value);

@@ -29,6 +29,7 @@ OPT_EARLY_LOADS = 6
 OPT_NEXT_FORWARD = 7
 OPT_DX_IN_UPDATE = 8
 OPT_CHECK_FINITE = 9
+OPT_SHARED_RESTART = 10
 ERR_DEVICE_TIMEOUT, ERR_NONFINITE = -6, -7
 KERNEL_FAMILIES = ("forward", "softmax", "dx", "update", "update_average", "average", "misc")
 MAX_LAYERS = 16

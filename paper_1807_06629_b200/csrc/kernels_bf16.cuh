@@ -102,6 +102,8 @@ struct StreamArgs {
   float gamma, mu;
   // Softmax cross-entropy gradient in the epilogue of the last forward GEMM (needs tiles_m == 1)
   int prefetch;              // 1: the weight tiles may be requested before the previous launch has completed
+  int shared_w;              // 1: every worker's weights hold the same bits (the launch follows a node average with
+                             // nothing in between), so every item reads worker 0's tiles: one HBM read serves all N
   int softmax;
   const int32_t* Y;          // labels [N][P]
   int64_t P;
@@ -191,9 +193,13 @@ __global__ void __launch_bounds__(kStreamThreads, 1) tc_stream_kernel(const __gr
   };
   // The weights this launch reads were last written before the previous launch began (the host sets
   // `prefetch` only then), so the first stages' weight tiles are requested while that launch drains.
+  // Item -> (worker, row tile).  Worker-major as a rule; with shared weights tile-major, so that the N items
+  // that read the same tile run at about the same time and all but the first find it in L2.
+  auto item_worker = [&](int item) { return a.shared_w ? item % a.N : item / a.tiles_m; };
+  auto item_row0 = [&](int item) { return (a.shared_w ? item / a.N : item % a.tiles_m) * 128; };
   uint32_t pre = 0;
   if (warp == 0 && lane == 0 && a.prefetch != 0 && (int)blockIdx.x < a.tiles_m * a.N) {
-    const int n = (int)blockIdx.x / a.tiles_m, m0 = ((int)blockIdx.x % a.tiles_m) * 128;
+    const int n = a.shared_w ? 0 : item_worker((int)blockIdx.x), m0 = item_row0((int)blockIdx.x);
     pre = (uint32_t)(a.k_steps < S ? a.k_steps : S);
     for (uint32_t ks = 0; ks < pre; ++ks) {
       mbar_expect_tx(full_bar(ks), stage_bytes);
@@ -211,7 +217,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) tc_stream_kernel(const __gr
     uint32_t g = 0;
     bool ok = true;
     for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
-      const int n = item / a.tiles_m, m0 = (item % a.tiles_m) * 128;
+      const int n = item_worker(item), m0 = item_row0(item);
       if (!item_active(n)) continue;
       const int row0 = a.pool ? (int)draw_block(a.draw.seed, a.draw.worker0 + n, draw_t(a.draw), a.draw.n_blocks) * a.B : 0;
       for (int ks = 0; ks < a.k_steps; ++ks, ++g) {
@@ -221,13 +227,13 @@ __global__ void __launch_bounds__(kStreamThreads, 1) tc_stream_kernel(const __gr
           ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, a.status, 0x101);
           if (!ok) break;
           mbar_expect_tx(full_bar(s), stage_bytes);
-          load_weights(s, ks, m0, n);
+          load_weights(s, ks, m0, a.shared_w ? 0 : n);
         }
         load_operand(s, ks, row0, n);
       }
     }
     if (total_items == 0 && pre > 0) {   // nothing will consume the early tiles: complete their stages
-      for (uint32_t ks = 0; ks < pre; ++ks) load_operand((int)ks, (int)ks, 0, (int)blockIdx.x / a.tiles_m);
+      for (uint32_t ks = 0; ks < pre; ++ks) load_operand((int)ks, (int)ks, 0, item_worker((int)blockIdx.x));
       g = pre;
     }
     if (*abort_flag && g > 0) {   // let the copies already in flight land before the CTA goes away
@@ -244,7 +250,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) tc_stream_kernel(const __gr
     uint32_t g = 0, it = 0;
     bool ok = true;
     for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
-      if (!item_active(item / a.tiles_m)) continue;
+      if (!item_active(item_worker(item))) continue;
       const int q = it & 1;
       ok = mbar_wait(acc_empty(q), ((it >> 1) & 1u) ^ 1u, abort_flag, a.status, 0x104);
       if (!ok) break;
@@ -282,9 +288,9 @@ __global__ void __launch_bounds__(kStreamThreads, 1) tc_stream_kernel(const __gr
     uint32_t it = 0;
     bool ok = true;
     for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
-      const int n = item / a.tiles_m;
+      const int n = item_worker(item);
       if (!item_active(n)) continue;
-      const int m = (item % a.tiles_m) * 128 + q4 * 32 + lane;
+      const int m = item_row0(item) + q4 * 32 + lane;
       const bool valid = m < a.M_total;
       auto mask_fetch = [&](int bi, uint16_t (&mk)[16]) {
         if (MODE == TC_DX && bi < batches && valid) {
@@ -402,6 +408,9 @@ struct UpdateArgs {
   const uint8_t* active;
   DeviceStatus* status;
   int prefetch;            // 1: master tiles may be requested before the previous launch has completed
+  int shared_w;            // fused form only, 1: every worker's master tile holds the same bits (the launch follows a
+                           // node average with nothing in between): all N loads of a tile read worker 0's copy, which
+                           // nobody overwrites before the CTA that owns the tile has summed all N workers
 };
 
 constexpr int kUpdThreads = 224;          // warp 0 loader, 1 MMA, 2 storer, 3..6 epilogue
@@ -496,7 +505,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
       const int n = FUSE ? k : w / tiles;
       if (w >= items_all || n >= a.N) break;
       const int tile = FUSE ? w : w % tiles;
-      load_master(k, (tile / a.tiles_n) * 128, (tile % a.tiles_n) * TN, n);
+      load_master(k, (tile / a.tiles_n) * 128, (tile % a.tiles_n) * TN, (FUSE && a.shared_w) ? 0 : n);
       ++pre;
     }
   }
@@ -532,7 +541,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
         tma_load_3d(ops + op_box, &mapDelta, full_ops(s), m0 + 64, 0, n);
 #pragma unroll
         for (int h = 0; h < NB64; ++h) tma_load_3d(ops + (2u + h) * op_box, &mapAct, full_ops(s), n0 + 64 * h, row0, n);
-        if (it >= pre) load_master(s, m0, n0, n);
+        if (it >= pre) load_master(s, m0, n0, (FUSE && a.shared_w) ? 0 : n);
         ++it;
       }
     }
@@ -1572,6 +1581,15 @@ inline int tc_bind_data(prsgd_ctx* c, std::string* err) {
 // count fits one 128-row tile (and PRSGD_OPT_FUSED_EPILOGUES is on); otherwise as kernels of their own.
 inline bool tc_epilogues_fused(const prsgd_ctx* c) { return c->fused_epilogues != 0 && c->dims[c->L] <= 128; }
 
+// Right after a node average every worker's row holds the same bits (Algorithm 1: all workers restart from y),
+// so the launches of the iteration that follows may read worker 0's weights for every worker.  Safe for
+// launches that only read the weights (forward, dX) and for the fused update + average, whose CTA has read all
+// N copies of a tile before it writes any; NOT for the plain in-place update, where worker 0's row changes
+// while other workers' items are still to come.
+inline bool tc_shared_restart(const prsgd_ctx* c, const uint8_t* active) {
+  return c->shared_restart != 0 && c->rows_identical && active == nullptr && c->N > 1;
+}
+
 // forward GEMM of layer l (1-based)
 inline void tc_launch_forward(prsgd_ctx* c, int l, const DrawArgs& dr, const uint8_t* active) {
   TcState* st = static_cast<TcState*>(c->tc);
@@ -1584,6 +1602,7 @@ inline void tc_launch_forward(prsgd_ctx* c, int l, const DrawArgs& dr, const uin
   a.bias = c->params + ly.b_off; a.bias_stride = c->m_pad;
   a.active = active; a.status = c->status;
   a.prefetch = (l > 1 && active == nullptr && c->early_loads) ? 1 : 0;   // W_1 was written by the launch just before
+  a.shared_w = tc_shared_restart(c, active) ? 1 : 0;
   const bool softmax = l == c->L && tc_epilogues_fused(c);
   if (softmax) {        // the softmax-CE gradient, the loss and the step of b_L happen in this launch's epilogue
     a.softmax = 1; a.stages = stream_stages(c->B, true);
@@ -1612,6 +1631,7 @@ inline void tc_launch_dx(prsgd_ctx* c, int l, const DrawArgs& dr, const uint8_t*
   a.out_bk = c->buf.delta_bk[l - 1]; a.mask_src = c->buf.act_bk[l - 1];
   a.active = active; a.status = c->status;
   a.prefetch = (active == nullptr && c->early_loads) ? 1 : 0;
+  a.shared_w = tc_shared_restart(c, active) ? 1 : 0;
   if (tc_epilogues_fused(c)) {      // the step of b_{l-1} rides on the epilogue that forms dZ_{l-1}
     a.bias_rw = c->params + c->layer[l - 2].b_off; a.bias_stride = c->m_pad; a.gamma = c->gamma; a.mu = c->mu;
     a.bias_vel = c->velocity != nullptr ? c->velocity + c->layer[l - 2].b_off : nullptr;
@@ -1630,6 +1650,7 @@ inline void tc_launch_update_tn(prsgd_ctx* c, int l, const DrawArgs& dr, const u
   a.B = c->B; a.N = c->N; a.tiles_m = (ly.d_out + 127) / 128; a.tiles_n = (ly.d_in + TN - 1) / TN;
   a.gamma = c->gamma; a.mu = c->mu; a.pool = l == 1; a.draw = dr; a.active = active; a.status = c->status;
   a.prefetch = (active == nullptr && c->early_loads) ? 1 : 0;
+  a.shared_w = (fuse && tc_shared_restart(c, active)) ? 1 : 0;
   const int items = a.tiles_m * a.tiles_n * (fuse ? 1 : c->N);
   const int grid = items < st->num_sms ? items : st->num_sms;
   const TcLayerMaps& mp = st->layer[l - 1];

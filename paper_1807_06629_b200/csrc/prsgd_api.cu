@@ -379,6 +379,7 @@ int launch_average(prsgd_ctx* c) {
                                                                              nullptr, nullptr, c->status);
     LAUNCH_CHECK(c);
   }
+  c->rows_identical = true;      // N copies of y
   return PRSGD_OK;
 }
 
@@ -553,6 +554,8 @@ int prsgd_set_params(prsgd_ctx* c, const float* src, int32_t worker, int src_on_
     LAUNCH_CHECK(c);
   }
   if (!src_on_device) CUDA_TRY(c, cudaStreamSynchronize(c->stream));   // src may be reused by the caller
+  c->rows_identical = worker < 0 || c->N == 1;
+  c->a1_ready = false;
   return refresh_shadow(c);
 }
 
@@ -562,6 +565,8 @@ int prsgd_set_params_stacked(prsgd_ctx* c, const float* src, int src_on_device) 
   int rc = copy_canonical(c, c->params, const_cast<float*>(src), 0, c->N, true);
   if (rc != PRSGD_OK) return rc;
   if (!src_on_device) CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  c->rows_identical = c->N == 1;
+  c->a1_ready = false;
   return refresh_shadow(c);
 }
 
@@ -595,13 +600,16 @@ int run_iterations(prsgd_ctx* c, int64_t t_first, int64_t count) {
     if (rc == PRSGD_OK && averaging && (!c->fused_average || c->velocity != nullptr)) rc = launch_average(c);
     if (rc != PRSGD_OK) {
       c->a1_ready = false;      // a launch failed: the next iteration must not count on an a_1 formed ahead
+      c->rows_identical = false;
       return rc;
     }
+    c->rows_identical = averaging;     // an averaging iteration leaves N copies of y, any other one N different points
+    c->assigned_upto = -1;
   }
   return PRSGD_OK;
 }
 
-void period_key(const prsgd_ctx* c, uint64_t (&key)[12]) {
+void period_key(const prsgd_ctx* c, uint64_t (&key)[13]) {
   uint32_t gbits, mbits;
   std::memcpy(&gbits, &c->gamma, 4);
   std::memcpy(&mbits, &c->mu, 4);
@@ -609,13 +617,14 @@ void period_key(const prsgd_ctx* c, uint64_t (&key)[12]) {
   key[4] = c->has_mask ? 1 : 0; key[5] = reinterpret_cast<uint64_t>(c->velocity); key[6] = mbits;
   key[7] = (uint64_t)c->average_velocity; key[8] = reinterpret_cast<uint64_t>(c->X);
   key[9] = reinterpret_cast<uint64_t>(c->Y); key[10] = (uint64_t)c->worker0; key[11] = (uint64_t)c->fused_epilogues | ((uint64_t)c->early_loads << 1) | ((uint64_t)c->next_forward << 2) | ((uint64_t)c->dx_in_update << 3);
+  key[12] = (c->rows_identical ? 1u : 0u) | ((uint64_t)c->shared_restart << 1);   // the period's first iteration may share reads
 }
 
 // One whole averaging period (I iterations starting right after an average) as a CUDA graph: the
 // kernels take the iteration number as device counter + offset, so one capture serves every period.
 // Returns nullptr when capture is not possible (the caller then launches directly).
 prsgd_ctx::PeriodGraph* get_period_graph(prsgd_ctx* c) {
-  uint64_t key[12];
+  uint64_t key[13];
   period_key(c, key);
   for (auto& g : c->graphs)
     if (std::memcmp(g.key, key, sizeof key) == 0) return &g;
@@ -629,6 +638,7 @@ prsgd_ctx::PeriodGraph* get_period_graph(prsgd_ctx* c) {
     return nullptr;
   }
   const int64_t launches0 = c->launches;
+  const bool identical0 = c->rows_identical;
   c->capturing = true;
   int rc = run_iterations(c, 1, c->I);                  // offsets 1..I; offset I is the averaging iteration
   if (rc == PRSGD_OK) {
@@ -644,6 +654,7 @@ prsgd_ctx::PeriodGraph* get_period_graph(prsgd_ctx* c) {
   if (rc == PRSGD_OK && e == cudaSuccess && graph != nullptr) e = cudaGraphInstantiate(&exec, graph, 0);
   if (graph) cudaGraphDestroy(graph);
   c->a1_ready = false;     // launches recorded into a capture have not run: no a_1 has been formed ahead
+  c->rows_identical = identical0;
   if (rc != PRSGD_OK || e != cudaSuccess || exec == nullptr) {
     cudaGetLastError();
     c->use_graph = 0;                                   // do not try again on this context
@@ -670,6 +681,7 @@ int prsgd_local_steps(prsgd_ctx* c, int64_t k) {
         counter_set_kernel<<<1, 1, 0, c->stream>>>(c->t_dev, c->t);
         CUDA_TRY(c, cudaGetLastError());
         CUDA_TRY(c, cudaGraphLaunch(g->exec, c->stream));
+        c->rows_identical = true;                      // a period ends with the node average
         c->launches += g->launches + 1;
         c->t += c->I;
         k -= c->I;
@@ -824,6 +836,11 @@ int prsgd_assign_rows(prsgd_ctx* c, const float* d_src, float divisor, int64_t c
     assign_rows_kernel<false><<<grid1d(ncols / 4, 256), 256, 0, c->stream>>>(c->params + col0, nullptr, d_src + col0, divisor,
                                                                           c->N, ncols / 4, c->m_pad / 4, c->status);
   LAUNCH_CHECK(c);
+  // chunks assigned in ascending order since the last local step: once they cover the row, all rows are equal
+  if (col0 == 0) c->assigned_upto = ncols;
+  else if (col0 == c->assigned_upto) c->assigned_upto += ncols;
+  else c->assigned_upto = -1;
+  if (c->assigned_upto == c->m_pad) c->rows_identical = true;
   return PRSGD_OK;
 }
 
@@ -957,6 +974,7 @@ int prsgd_set_option(prsgd_ctx* c, int32_t option, int64_t value) {
   if (option == PRSGD_OPT_EARLY_LOADS) { c->early_loads = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_NEXT_FORWARD) { c->next_forward = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_CHECK_FINITE) { c->check_finite = value != 0; return PRSGD_OK; }
+  if (option == PRSGD_OPT_SHARED_RESTART) { c->shared_restart = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_DX_IN_UPDATE) {
     if (value < 0 || value > 2) return fail(c, PRSGD_ERR_ARG, "PRSGD_OPT_DX_IN_UPDATE takes 0, 1 or 2");
     c->dx_in_update = (int)value;
@@ -1010,6 +1028,8 @@ int prsgd_clear_device_error(prsgd_ctx* c) {
   CUDA_TRY(c, cudaMemsetAsync(c->status, 0, sizeof(DeviceStatus), c->stream));
   CUDA_TRY(c, cudaStreamSynchronize(c->stream));
   c->err.clear();
+  c->rows_identical = false;     // whatever the interrupted launches left
+  c->a1_ready = false;
   return PRSGD_OK;
 }
 

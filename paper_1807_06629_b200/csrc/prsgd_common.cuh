@@ -100,6 +100,9 @@ struct prsgd_ctx {
   bool a1_ready = false;         // a_1 of the coming iteration has already been formed by the previous update
   int early_loads = 1;           // tensor-core kernels request tiles nobody is writing before their dependency wait
   int fused_epilogues = 1;       // softmax-CE gradient and bias steps inside the GEMM epilogues (tensor-core path)
+  int shared_restart = 1;        // the iteration after a node average reads worker 0's weights for every worker
+  bool rows_identical = false;   // every row of the store (and of the bf16 copy) holds the same bits right now
+  int64_t assigned_upto = -1;    // prsgd_assign_rows calls since the last local step have covered columns [0, assigned_upto)
   int64_t launches = 0;
   int64_t m = 0, m_pad = 0;
   prsgd::Layer layer[PRSGD_MAX_LAYERS];
@@ -138,7 +141,7 @@ struct prsgd_ctx {
 
   // whole averaging periods captured as CUDA graphs (PRSGD_OPT_GRAPH)
   struct PeriodGraph {
-    uint64_t key[12];
+    uint64_t key[13];
     cudaGraphExec_t exec;
     int64_t launches;            // kernel launches one replay stands for
   };

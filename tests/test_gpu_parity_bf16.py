@@ -281,6 +281,52 @@ def test_folded_kernels_with_a_worker_mask_change_no_bit(torch_cuda):
             assert np.array_equal(outs[0][2][active], o[2][active])
 
 
+def test_reading_the_common_restart_point_once_changes_no_bit(torch_cuda):
+    """After a node average all N rows hold the same bits, so the following iteration's forward, dX and fused
+    update + average launches read worker 0's weights for every worker (PRSGD_OPT_SHARED_RESTART).  Against
+    the same runs with the option off: identical parameters, losses and momentum buffers for I = 1 (every
+    iteration follows an average), I = 3, replayed periods, a start from N different points (nothing may be
+    shared before the first average), momentum, and the two halves of the multi-GPU average."""
+    torch = torch_cuda
+    from paper_1807_06629_b200 import binding
+    cases = [(_w("tc-share-I1", 5, (192, 320, 100), 32, I=1), None), (_w("tc-share-I3", 4, (64, 448, 320, 10), 16, I=3), None),
+             (SMALL[3].with_(I=1), None), (_w("tc-share-mom", 3, (128, 256, 10), 32, I=1), 0.9), (SMALL[6], None)]
+    for w, mu in cases:
+        X, Y, x0 = make_inputs(w)
+        rng = np.random.default_rng(1)
+        apart = np.tile(x0, (w.N, 1)) * (1.0 + 0.01 * rng.standard_normal((w.N, 1))).astype(np.float32)
+        outs = []
+        for share, graph, start in ((0, 0, "same"), (1, 0, "same"), (1, 1, "same"), (0, 0, "apart"), (1, 1, "apart")):
+            with torch.cuda.stream(torch.cuda.Stream()):
+                p = make_ctx(w, X, Y, x0)
+                p.set_option(binding.OPT_SHARED_RESTART, share)
+                p.set_option(binding.OPT_GRAPH, graph)
+                if mu is not None:
+                    p.enable_momentum(mu)
+                if start == "apart":
+                    p.set_params_stacked(apart)
+                p.local_steps(2 * w.I + 1)
+                p.local_steps(3 * w.I)
+                # the multi-GPU halves leave N equal rows too: the iteration after them shares its reads
+                row = p.new_row()
+                half = (p.m_pad // 8) * 4
+                p.partial_sum(row)
+                p.assign_rows(row, float(w.N), 0, half)
+                p.assign_rows(row, float(w.N), half, p.m_pad - half)
+                p.local_steps(2)
+                outs.append((start, p.get_params_stacked(), p.get_losses(),
+                             p.get_velocity_stacked() if mu is not None else None))
+                torch.cuda.current_stream().synchronize()
+                p.close()
+        for start in ("same", "apart"):
+            grp = [o for o in outs if o[0] == start]
+            for o in grp[1:]:
+                assert np.array_equal(grp[0][1], o[1]), (w.name, start)
+                assert np.array_equal(grp[0][2], o[2])
+                if mu is not None:
+                    assert np.array_equal(grp[0][3], o[3])
+
+
 def _segments(dims):
     """[(is_weight, start, stop)] of a canonical parameter vector."""
     out, off = [], 0
