@@ -238,9 +238,10 @@ int prsgd_assign_rows(prsgd_ctx* ctx, const float* d_src, float divisor, int64_t
  * d_velocity: caller-owned device memory of the same size as the parameter store (N*m_pad*4
  * bytes, 256-byte aligned), zeroed by this call and laid out like the store.  The paper does not
  * say what happens to the momentum buffers at a restart: with average_velocity = 0 every worker
- * keeps its own, with 1 they are averaged together with the models.  While momentum is on, an
- * averaging iteration runs as update followed by the averaging kernel (no fused form).
- * d_velocity = NULL switches back to plain SGD.  mu in [0, 1). */
+ * keeps its own, with 1 they are averaged together with the models.  On the tensor-core path an
+ * averaging iteration takes the fused update + average with momentum too (every worker's new buffer
+ * tile goes back to its own row, or the averaged tile to every row); on the FP32 path it runs as
+ * update followed by the averaging kernel.  d_velocity = NULL switches back to plain SGD.  mu in [0, 1). */
 int prsgd_enable_momentum(prsgd_ctx* ctx, float mu, void* d_velocity, int average_velocity);
 /* The momentum buffers, [N][m] in canonical order.  Synchronises the stream. */
 int prsgd_get_velocity_stacked(prsgd_ctx* ctx, float* dst, int dst_on_device);

@@ -408,6 +408,7 @@ struct UpdateArgs {
   const uint8_t* active;
   DeviceStatus* status;
   int prefetch;            // 1: master tiles may be requested before the previous launch has completed
+  int avg_vel;             // fused form with momentum, 1: the momentum buffers are averaged like the models
   int shared_w;            // fused form only, 1: every worker's master tile holds the same bits (the launch follows a
                            // node average with nothing in between): all N loads of a tile read worker 0's copy, which
                            // nobody overwrites before the CTA that owns the tile has summed all N workers
@@ -435,7 +436,9 @@ template <int TN, bool MOM> struct UpdCfg {
 };
 
 // MOM: the local step of the paper's experiment, v <- mu v + G, x <- x - gamma v; the momentum tile
-// travels with the master tile (loaded, updated in shared memory, stored back).  Not combined with FUSE.
+// travels with the master tile (loaded, updated in shared memory, stored back).  FUSE with MOM: every worker's
+// new momentum tile goes back to its own row as the CTA walks the workers (avg_vel = 0), or a second set of
+// running sums averages the momentum tiles as well and the mean goes to every row with the models (avg_vel = 1).
 template <bool FUSE, int TN, bool MOM>
 __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_constant__ CUtensorMap mapDelta,
                                                                    const __grid_constant__ CUtensorMap mapAct,
@@ -444,10 +447,13 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
                                                                    const __grid_constant__ CUtensorMap mapVel,
                                                                    const UpdateArgs a) {
   using namespace ptx;
-  static_assert(!(FUSE && MOM), "the fused average is not built for the momentum step");
   using Cfg = UpdCfg<TN, MOM>;
   constexpr int S = Cfg::kStages;
   constexpr int NB32 = TN / 32, NB64 = TN / 64;
+  // Fused form on shared weights (every worker's master tile holds the same bits): all loads of a tile read
+  // worker 0's copy; with 64-wide tiles and the plain step the tile is loaded ONCE, by its first worker, and
+  // kept in registers while the CTA walks the other workers (wider tiles and the momentum step reload it from L2).
+  constexpr bool kShareOnce = FUSE && !MOM && TN == 64;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -486,10 +492,12 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  // (with shared weights the master tile comes from worker 0's row; the momentum tile is always the worker's own)
   auto load_master = [&](int s, int m0, int n0, int n) {
     mbar_expect_tx(full_w(s), Cfg::kMaster + Cfg::kVel);
+    const int nm = (FUSE && a.shared_w) ? 0 : n;
 #pragma unroll
-    for (int q = 0; q < NB32; ++q) tma_load_3d(master_u32(s) + q * 16384u, &mapMaster, full_w(s), n0 + 32 * q, m0, n);
+    for (int q = 0; q < NB32; ++q) tma_load_3d(master_u32(s) + q * 16384u, &mapMaster, full_w(s), n0 + 32 * q, m0, nm);
     if (MOM) {
 #pragma unroll
       for (int q = 0; q < NB32; ++q) tma_load_3d(vel_u32(s) + q * 16384u, &mapVel, full_w(s), n0 + 32 * q, m0, n);
@@ -505,7 +513,8 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
       const int n = FUSE ? k : w / tiles;
       if (w >= items_all || n >= a.N) break;
       const int tile = FUSE ? w : w % tiles;
-      load_master(k, (tile / a.tiles_n) * 128, (tile % a.tiles_n) * TN, (FUSE && a.shared_w) ? 0 : n);
+      if (kShareOnce && a.shared_w && n > 0) mbar_arrive(full_w(k));     // the common master tile is read once per tile
+      else load_master(k, (tile / a.tiles_n) * 128, (tile % a.tiles_n) * TN, n);
       ++pre;
     }
   }
@@ -541,7 +550,10 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
         tma_load_3d(ops + op_box, &mapDelta, full_ops(s), m0 + 64, 0, n);
 #pragma unroll
         for (int h = 0; h < NB64; ++h) tma_load_3d(ops + (2u + h) * op_box, &mapAct, full_ops(s), n0 + 64 * h, row0, n);
-        if (it >= pre) load_master(s, m0, n0, (FUSE && a.shared_w) ? 0 : n);
+        if (it >= pre) {
+          if (kShareOnce && a.shared_w && n > n_begin) mbar_arrive(full_w(s));   // (its first worker has brought it)
+          else load_master(s, m0, n0, n);
+        }
         ++it;
       }
     }
@@ -606,6 +618,28 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
         tma_wait_group_read0();
         mbar_arrive(stage_empty(s));
         ++it;
+      } else if (MOM && a.avg_vel == 0) {
+        // every worker's new momentum tile goes back to its own row; the last worker's stage also holds the
+        // averaged models, which go to every row
+        for (int n = 0; n < a.N && ok; ++n, ++it) {
+          const int s = it % S;
+          const uint32_t ph = (it / S) & 1u;
+          ok = mbar_wait(tile_ready(s), ph, abort_flag, a.status, 0x208);
+          if (!ok) break;
+          if (n == a.N - 1) {
+            for (int rr = 0; rr < a.N; ++rr) {
+#pragma unroll
+              for (int q = 0; q < NB32; ++q) tma_store_3d(&mapMaster, master_u32(s) + q * 16384u, n0 + 32 * q, m0, rr);
+#pragma unroll
+              for (int h = 0; h < NB64; ++h) tma_store_3d(&mapShadow, ops_u32(s) + h * 16384u, n0 + 64 * h, m0, rr);
+            }
+          }
+#pragma unroll
+          for (int q = 0; q < NB32; ++q) tma_store_3d(&mapVel, vel_u32(s) + q * 16384u, n0 + 32 * q, m0, n);
+          tma_commit_group();
+          tma_wait_group_read0();
+          mbar_arrive(stage_empty(s));
+        }
       } else {
         it += (uint32_t)a.N;
         const int s = (it - 1) % S;                       // stage of the tile's last worker
@@ -629,13 +663,21 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
     const int etid = tid - 96;                            // 0..127 among the epilogue threads
     const float fN = (float)a.N;
     constexpr int NSUM = FUSE ? TN : 1;
+    constexpr int NVSUM = (FUSE && MOM) ? TN : 1;
+    constexpr int NXR = kShareOnce ? TN : 1;
+    const bool shared_x = kShareOnce && a.shared_w != 0;
+    const bool avg_vel = FUSE && MOM && a.avg_vel != 0;
+    const bool vel_per_worker = FUSE && MOM && a.avg_vel == 0;      // the storer takes every worker's momentum tile
     uint32_t it = 0;
     bool ok = true;
     for (int w = blockIdx.x; w < total_items && ok; w += gridDim.x) {
       const int n_begin = FUSE ? 0 : w / tiles, n_end = FUSE ? a.N : n_begin + 1;
-      float sum[NSUM];
+      float sum[NSUM], vsum[NVSUM];
+      float xr[NXR];                                        // shared weights: the tile every worker starts from
 #pragma unroll
       for (int i = 0; i < NSUM; ++i) sum[i] = 0.f;
+#pragma unroll
+      for (int i = 0; i < NVSUM; ++i) vsum[i] = 0.f;
       for (int n = n_begin; n < n_end; ++n) {
         if (!item_active(n)) continue;
         const bool upd = a.active == nullptr || a.active[n] != 0;
@@ -658,15 +700,37 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
             float4* pw = reinterpret_cast<float4*>(mst + c * 16384 + row_off + (((uint32_t)j ^ sw) << 4));
-            float4 x = *pw;
+            float4 x;
+            if (kShareOnce && shared_x) {                   // worker 0's load brought the common tile: keep it in registers
+              constexpr int F = kShareOnce ? 1 : 0;
+              float* xp = &xr[F * (c * 32 + 4 * j)];
+              if (n == 0) { x = *pw; xp[0] = x.x; xp[F * 1] = x.y; xp[F * 2] = x.z; xp[F * 3] = x.w; }
+              else x = make_float4(xp[0], xp[F * 1], xp[F * 2], xp[F * 3]);
+            } else {
+              x = *pw;
+            }
             float4 g4 = make_float4(__uint_as_float(v[4 * j + 0]), __uint_as_float(v[4 * j + 1]),
                                     __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
             if (MOM) {                                      // v <- mu v + G, kept in place next to the master tile
               float4* pv = reinterpret_cast<float4*>(mst + Cfg::kMaster + c * 16384 + row_off + (((uint32_t)j ^ sw) << 4));
               const float4 vo = *pv;
-              g4.x = fmaf(a.mu, vo.x, g4.x); g4.y = fmaf(a.mu, vo.y, g4.y);
-              g4.z = fmaf(a.mu, vo.z, g4.z); g4.w = fmaf(a.mu, vo.w, g4.w);
-              *pv = g4;
+              if (!FUSE || upd) {
+                g4.x = fmaf(a.mu, vo.x, g4.x); g4.y = fmaf(a.mu, vo.y, g4.y);
+                g4.z = fmaf(a.mu, vo.z, g4.z); g4.w = fmaf(a.mu, vo.w, g4.w);
+              } else {
+                g4 = vo;                                    // an inactive worker keeps its momentum (and its point)
+              }
+              float4 vst = g4;
+              if (FUSE && MOM && avg_vel) {                 // running sums of the momentum tiles, worker order
+                constexpr int F = (FUSE && MOM) ? 1 : 0;
+                float* vp = &vsum[F * (c * 32 + 4 * j)];
+                vp[0] += g4.x; vp[F * 1] += g4.y; vp[F * 2] += g4.z; vp[F * 3] += g4.w;
+                if (last) {
+                  vst.x = __fdiv_rn(vp[0], fN); vst.y = __fdiv_rn(vp[F * 1], fN);
+                  vst.z = __fdiv_rn(vp[F * 2], fN); vst.w = __fdiv_rn(vp[F * 3], fN);
+                }
+              }
+              if (!avg_vel || last) *pv = vst;
             }
             if (upd) {
               x.x = fmaf(-a.gamma, g4.x, x.x);
@@ -698,7 +762,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
         }
         tc_fence_before();
         mbar_arrive(acc_empty(s));
-        if (!FUSE) {
+        if (!FUSE || vel_per_worker) {
           fence_proxy_async();
           mbar_arrive(tile_ready(s));
         } else if (last) {
@@ -1454,7 +1518,7 @@ __global__ void __launch_bounds__(128) bias_update_kernel(const BiasArgs a) {
 // grid (ceil(max d_l / 128), L), one thread per bias entry, the same arithmetic as average_rows_kernel
 // (fp32 sum in worker order, one division), so the bits equal update-then-average.
 struct BiasAverageArgs {
-  float* params;
+  float* params;             // the store, or the momentum buffers (same layout)
   int64_t m_pad;
   int N;
   int64_t b_off[PRSGD_MAX_LAYERS];
@@ -1535,6 +1599,7 @@ inline int tc_create(prsgd_ctx* c, std::string* err) {
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<false, 128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<128, false>::smem(c->B));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<true, 128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<128, false>::smem(c->B));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<false, 64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<64, true>::smem(c->B));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<true, 64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<64, true>::smem(c->B));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_dx_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdDxCfg<64, false>::smem(c->B));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_dx_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdDxCfg<64, true>::smem(c->B));
   if (e == cudaSuccess && UpdDxCfg<128, false>::stages(c->B) == 2)
@@ -1651,12 +1716,16 @@ inline void tc_launch_update_tn(prsgd_ctx* c, int l, const DrawArgs& dr, const u
   a.gamma = c->gamma; a.mu = c->mu; a.pool = l == 1; a.draw = dr; a.active = active; a.status = c->status;
   a.prefetch = (active == nullptr && c->early_loads) ? 1 : 0;
   a.shared_w = (fuse && tc_shared_restart(c, active)) ? 1 : 0;
+  a.avg_vel = c->average_velocity ? 1 : 0;
   const int items = a.tiles_m * a.tiles_n * (fuse ? 1 : c->N);
   const int grid = items < st->num_sms ? items : st->num_sms;
   const TcLayerMaps& mp = st->layer[l - 1];
   const size_t smem = UpdCfg<TN, MOM>::smem(c->B);
   if constexpr (MOM) {
-    launch_pdl(tc_update_kernel<false, TN, true>, dim3(grid), kUpdThreads, smem, c->stream, mp.delta_out, mp.act_in, mp.master, mp.shadow_k, mp.velocity, a);
+    if (fuse)
+      launch_pdl(tc_update_kernel<true, TN, true>, dim3(grid), kUpdThreads, smem, c->stream, mp.delta_out, mp.act_in, mp.master, mp.shadow_k, mp.velocity, a);
+    else
+      launch_pdl(tc_update_kernel<false, TN, true>, dim3(grid), kUpdThreads, smem, c->stream, mp.delta_out, mp.act_in, mp.master, mp.shadow_k, mp.velocity, a);
   } else {
     if (fuse)
       launch_pdl(tc_update_kernel<true, TN, false>, dim3(grid), kUpdThreads, smem, c->stream, mp.delta_out, mp.act_in, mp.master, mp.shadow_k, mp.master, a);
@@ -1752,7 +1821,7 @@ inline void tc_launch_update(prsgd_ctx* c, int l, const DrawArgs& dr, const uint
   const TcState* st = static_cast<const TcState*>(c->tc);
   const Layer& ly = c->layer[l - 1];
   if (c->velocity != nullptr) {            // momentum step: 64-wide tiles (two stages of master + momentum + output)
-    tc_launch_update_tn<64, true>(c, l, dr, active, false);
+    tc_launch_update_tn<64, true>(c, l, dr, active, fuse);
     return;
   }
   int tile = c->upd_tile;
@@ -1798,9 +1867,18 @@ inline void tc_launch_weight_average(prsgd_ctx* c, int l) {
              (const DeviceStatus*)c->status);
 }
 
-inline void tc_launch_bias_average(prsgd_ctx* c) {
+// the same segment of the momentum buffers, when they are averaged with the models
+inline void tc_launch_velocity_segment_average(prsgd_ctx* c, int l) {
+  const Layer& ly = c->layer[l - 1];
+  const int64_t cols = (int64_t)ly.d_out * ly.d_in;
+  launch_pdl(average_rows_kernel<0, false, 2>, dim3((unsigned)((cols / 2 + (cols & 1) + 255) / 256)), dim3(256), 0, c->stream,
+             c->velocity + ly.w_off, (int64_t)c->N, cols, c->m_pad, (float*)nullptr, (uint16_t*)nullptr,
+             (const DeviceStatus*)c->status);
+}
+
+inline void tc_launch_bias_average(prsgd_ctx* c, float* store) {
   BiasAverageArgs a{};
-  a.params = c->params; a.m_pad = c->m_pad; a.N = c->N; a.status = c->status;
+  a.params = store; a.m_pad = c->m_pad; a.N = c->N; a.status = c->status;
   int dmax = 1;
   for (int l = 1; l <= c->L; ++l) {
     a.b_off[l - 1] = c->layer[l - 1].b_off; a.d_out[l - 1] = c->layer[l - 1].d_out;

@@ -286,7 +286,8 @@ int step_f32(prsgd_ctx* c, int64_t t, bool averaging) {
 int step_bf16(prsgd_ctx* c, int64_t t, bool averaging, bool more_follow) {
   const int L = c->L, N = c->N;
   const uint8_t* act_mask = c->has_mask ? c->active : nullptr;
-  const bool fuse = averaging && c->fused_average && c->velocity == nullptr;   // the momentum step is not fused
+  const bool fuse = averaging && c->fused_average;
+  const bool avg_vel = c->velocity != nullptr && c->average_velocity;
   const DrawArgs dr = draw_args(c, t);
   // Layer 1's update can form a_1 of iteration t + 1 as well (its input is the data pool), which saves that
   // iteration's first forward launch and the write of W_1's shadow: only on a plain SGD iteration that is
@@ -338,6 +339,11 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging, bool more_follow) {
       prof_begin(c, PRSGD_KERNEL_AVERAGE);
       tc_launch_weight_average(c, l);
       LAUNCH_CHECK(c);
+      if (avg_vel) {
+        prof_begin(c, PRSGD_KERNEL_AVERAGE);
+        tc_launch_velocity_segment_average(c, l);
+        LAUNCH_CHECK(c);
+      }
     }
   }
   if (!epi) {
@@ -347,8 +353,13 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging, bool more_follow) {
   }
   if (fuse) {
     prof_begin(c, PRSGD_KERNEL_MISC);
-    tc_launch_bias_average(c);
+    tc_launch_bias_average(c, c->params);
     LAUNCH_CHECK(c);
+    if (avg_vel) {
+      prof_begin(c, PRSGD_KERNEL_MISC);
+      tc_launch_bias_average(c, c->velocity);
+      LAUNCH_CHECK(c);
+    }
   }
   return PRSGD_OK;
 }
@@ -597,7 +608,9 @@ int run_iterations(prsgd_ctx* c, int64_t t_first, int64_t count) {
     const bool averaging = c->I > 0 && (t % c->I) == 0;
     const bool more_follow = t + 1 < t_first + count;
     int rc = c->precision == PRSGD_PRECISION_BF16 ? step_bf16(c, t, averaging, more_follow) : step_f32(c, t, averaging);
-    if (rc == PRSGD_OK && averaging && (!c->fused_average || c->velocity != nullptr)) rc = launch_average(c);
+    // (the fp32 path has no fused form for the momentum step)
+    const bool separate_average = !c->fused_average || (c->velocity != nullptr && c->precision == PRSGD_PRECISION_FP32);
+    if (rc == PRSGD_OK && averaging && separate_average) rc = launch_average(c);
     if (rc != PRSGD_OK) {
       c->a1_ready = false;      // a launch failed: the next iteration must not count on an a_1 formed ahead
       c->rows_identical = false;

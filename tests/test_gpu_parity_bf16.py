@@ -127,6 +127,38 @@ def test_fused_average_equals_update_then_average_bit_for_bit(torch_cuda):
             assert np.array_equal(outs[0], o)
 
 
+@pytest.mark.parametrize("avg_v", [False, True])
+def test_fused_average_with_momentum_equals_update_then_average_bit_for_bit(torch_cuda, avg_v):
+    """The momentum step inside the fused update + average (every worker's new buffer tile written back to its
+    own row, or a second set of running sums when the buffers are averaged too) against the momentum update
+    followed by the stand-alone average: identical parameters and momentum buffers, also with a worker mask
+    (an inactive worker contributes its unchanged point and keeps its buffer) and replayed periods."""
+    torch = torch_cuda
+    from paper_1807_06629_b200 import binding
+    for w in (SMALL[1], SMALL[4], _w("tc-n5", 5, (64, 128, 10), 32, I=3), _w("tc-mom-I1", 4, (192, 320, 100), 16, I=1)):
+        X, Y, x0 = make_inputs(w)
+        for mask in (None, [1 if i != 1 else 0 for i in range(w.N)]):
+            outs = []
+            for fused, graph in ((0, 0), (1, 0), (1, 1)):
+                with torch.cuda.stream(torch.cuda.Stream()):
+                    p = make_ctx(w, X, Y, x0)
+                    p.enable_momentum(0.9, average_velocity=avg_v)
+                    p.set_option(binding.OPT_FUSED_AVERAGE, fused)
+                    p.set_option(binding.OPT_GRAPH, graph)
+                    if mask is not None:
+                        p.set_active(mask)
+                    n0 = p.get_launch_count()
+                    p.local_steps(3 * w.I + 1)
+                    outs.append((p.get_params_stacked(), p.get_velocity_stacked(), p.get_launch_count() - n0))
+                    torch.cuda.current_stream().synchronize()
+                    p.close()
+            for o in outs[1:]:
+                assert np.array_equal(outs[0][0], o[0]), (w.name, mask)
+                assert np.array_equal(outs[0][1], o[1]), (w.name, mask)
+            if not avg_v:
+                assert len({tuple(v) for v in outs[0][1][:, :8]}) > 1      # local buffers stay apart
+
+
 def test_early_weight_loads_change_no_bit(torch_cuda):
     """Tiles requested ahead of a kernel's dependency wait (weights nobody is writing at that time) against
     the same run with every load after the wait: identical bits over several periods, direct and replayed."""
