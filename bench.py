@@ -227,7 +227,7 @@ def ncu_traffic_per_launch(workload: str, family: str, N: int):
 # ----------------------------------------------------------------------------- byte model
 def period_bytes(w: synth.Workload, m_pad: int, sms: int = 148, momentum: bool = False, fused_average: bool = True,
                  fused_epilogues: bool = True, next_forward: bool = True, dx_in_update=True,
-                 shared_restart: bool = True) -> dict:
+                 shared_restart: bool = True, forward_chain: bool = True) -> dict:
     """Algorithmic HBM bytes and launch counts of ONE averaging period (prsgd_local_steps(I) from a period
     boundary) of all N workers, per kernel family: {family: [bytes, launches]}.
 
@@ -262,8 +262,12 @@ def period_bytes(w: synth.Workload, m_pad: int, sms: int = 148, momentum: bool =
         # the first iteration of a period starts from N equal rows: launches that only read the weights (and the
         # fused update + average) read one copy for all workers
         wr = 1 if (bf and shared_restart and j == 1 and w.I > 0) else N
-        for l in range(2 if a1_ready else 1, L + 1):
+        l_first = 2 if a1_ready else 1
+        chained = bf and forward_chain and 2 <= L - l_first + 1 <= 8      # all layers' forward GEMMs in one launch
+        for l in range(l_first, L + 1):
             add("forward", wr * d[l] * d[l - 1] * e + N * (d[l] * 4 + B * d[l - 1] * e + B * d[l] * (e if l < L else 4)))
+            if chained and l > l_first:
+                fam["forward"][1] -= 1
         a1_ready = False
         if not epi:
             add("softmax", N * B * d[L] * (4 + 4 + e))
@@ -439,7 +443,8 @@ def measure_config(torch, w_cfg, args, dev, rank, world, scaling, steps, warmup,
     for flag, opt in ((args.no_fuse, binding.OPT_FUSED_AVERAGE), (args.no_dx_in_update, binding.OPT_DX_IN_UPDATE),
                       (args.no_next_forward, binding.OPT_NEXT_FORWARD), (args.no_early_loads, binding.OPT_EARLY_LOADS),
                       (args.no_fused_epilogues, binding.OPT_FUSED_EPILOGUES),
-                      (args.no_shared_restart, binding.OPT_SHARED_RESTART)):
+                      (args.no_shared_restart, binding.OPT_SHARED_RESTART),
+                      (args.no_forward_chain, binding.OPT_FORWARD_CHAIN)):
         if flag:
             p.set_option(opt, 0)
     if args.fold_all_dx:
@@ -487,7 +492,7 @@ def measure_config(torch, w_cfg, args, dev, rank, world, scaling, steps, warmup,
                              momentum=args.momentum is not None, fused_average=not args.no_fuse,
                              fused_epilogues=not args.no_fused_epilogues, next_forward=not args.no_next_forward,
                              dx_in_update=0 if args.no_dx_in_update else (2 if args.fold_all_dx else 1),
-                             shared_restart=not args.no_shared_restart)
+                             shared_restart=not args.no_shared_restart, forward_chain=not args.no_forward_chain)
     if sharded_mode:          # a shard's period: I plain iterations, then the average as passes of their own
         fam_model = period_bytes(w.with_(I=0), p.m_pad, torch.cuda.get_device_properties(dev).multi_processor_count,
                                  momentum=args.momentum is not None, fused_epilogues=not args.no_fused_epilogues,
@@ -569,6 +574,8 @@ def parse_args(argv=None):
                     help="form dZ of the layer below inside the update launch for every layer, whatever its size")
     ap.add_argument("--no-shared-restart", action="store_true",
                     help="the iteration after an average reads every worker's own copy of the common point")
+    ap.add_argument("--no-forward-chain", action="store_true",
+                    help="one forward launch per layer instead of one launch for all layers")
     ap.add_argument("--no-next-forward", action="store_true",
                     help="layer 1's update does not form the next iteration's a_1")
     ap.add_argument("--no-early-loads", action="store_true",

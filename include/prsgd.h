@@ -297,6 +297,12 @@ int prsgd_get_velocity_stacked(prsgd_ctx* ctx, float* dst, int dst_on_device);
  * prsgd_assign_rows calls that cover the row in ascending order); a caller that writes into the store
  * through its own pointer instead of these calls must switch the option off.  Same bits either way. */
 #define PRSGD_OPT_SHARED_RESTART 10
+/* PRSGD_OPT_FORWARD_CHAIN (default 1, tensor-core path, 2 to 8 layers left to run): the forward GEMMs of an
+ * iteration run as ONE launch whose CTAs walk the items of all layers without draining in between; an item
+ * of layer l waits (bounded, status word on expiry) only for a_{l-1} of its own worker, counted per
+ * (layer, worker) in the scratch area, since workers do not depend on one another inside an iteration.
+ * With 0 every layer is a launch of its own.  Same bits either way. */
+#define PRSGD_OPT_FORWARD_CHAIN 11
 /* PRSGD_OPT_CHECK_FINITE (default 0): when 1, prsgd_sync also runs prsgd_check_finite. */
 #define PRSGD_OPT_CHECK_FINITE 9
 int prsgd_set_option(prsgd_ctx* ctx, int32_t option, int64_t value);

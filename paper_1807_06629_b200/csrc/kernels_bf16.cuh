@@ -396,6 +396,301 @@ __global__ void __launch_bounds__(kStreamThreads, 1) tc_stream_kernel(const __gr
 }
 
 // ---------------------------------------------------------------------------------------------
+// forward chain: the forward GEMMs of consecutive layers l_first..L in ONE launch
+// ---------------------------------------------------------------------------------------------
+// The items of all layers form one list (layer by layer); a CTA walks its share of the list with the same
+// TMA / MMA / epilogue pipeline as tc_stream_kernel and never drains between layers.  Workers are independent
+// inside an iteration, so an item of layer l only needs a_{l-1} of ITS worker: a counter per (layer, worker)
+// counts the finished row tiles, the epilogue adds to it once an item's activations are in global memory,
+// and the loader waits for it (bounded) before it requests the activation tiles; the weight tiles, which do
+// not depend on this launch, are requested first.  Items are walked in list order and every grid has at
+// most one CTA per SM, all resident, so the oldest unfinished item can always run: no wait can be circular.
+// The last CTA to finish zeroes the counters for the next launch.
+constexpr int kChainMax = 8;
+
+struct ChainSeg {
+  int k_steps, tiles_m, M_total, ld_out;
+  int linear;                // 0: bias + ReLU, bf16 out; 1: the last layer (fp32 logits, or the softmax epilogue)
+  int pool;                  // operand B rows come from the data pool at the drawn block (layer 1)
+  int prefetch;              // the weight tiles may be requested before the previous launch has completed
+  int item0;                 // index of the layer's first item in the list
+  uint16_t* out_bk;          // bf16 [N][B][ld_out]
+  float* out_f32;            // fp32 [N][B][ld_out] (logits without the softmax epilogue)
+  const float* bias;         // params + b_off; worker stride ChainArgs::bias_stride
+};
+
+struct ChainMaps {
+  CUtensorMap w[kChainMax];  // bf16 W_l, box {64, 128, 1}
+  CUtensorMap b[kChainMax];  // bf16 a_{l-1} (the data pool for layer 1), box {64, B, 1}
+};
+
+struct ChainArgs {
+  int B, N, stages, n_seg, total_items;
+  int shared_w;              // every worker's weights hold the same bits: read worker 0's tiles (see StreamArgs)
+  int softmax;               // the last layer's epilogue forms the softmax cross-entropy gradient
+  DrawArgs draw;
+  const uint8_t* active;
+  DeviceStatus* status;
+  int64_t bias_stride;
+  unsigned int* ready;       // [n_seg][N] finished row tiles of (layer, worker); zero between launches
+  unsigned int* done;        // CTAs that have finished; zero between launches
+  float* bias_rw; float* bias_vel; float gamma, mu;     // step of b_L in the softmax epilogue
+  const int32_t* Y; int64_t P; uint16_t* delta_bk; int ld_delta; float* row_losses; int32_t* draws;
+  ChainSeg seg[kChainMax];
+};
+
+__global__ void __launch_bounds__(kStreamThreads, 1) tc_forward_chain_kernel(const __grid_constant__ ChainMaps maps,
+                                                                             const __grid_constant__ ChainArgs a) {
+  using namespace ptx;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* gen = smem_raw + (base - raw);
+  const uint32_t stage_bytes = stream_stage_bytes(a.B);
+  const uint32_t b_box = (uint32_t)a.B * 128u;
+  const int S = a.stages;
+  const uint32_t bar0 = base + (uint32_t)S * stage_bytes;
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 64u + 8u * s; };
+  auto acc_full = [&](int q) { return bar0 + 128u + 8u * q; };
+  auto acc_empty = [&](int q) { return bar0 + 144u + 8u * q; };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen + (size_t)S * stage_bytes + 160);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + (size_t)S * stage_bytes + 164);
+  float* zs = reinterpret_cast<float*>(gen + (size_t)S * stage_bytes + 256);   // [B][kLogitLd], softmax epilogue only
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t ncols = 2 * a.B < 32 ? 32u : (uint32_t)(2 * a.B);   // two accumulators of B columns
+
+  if (tid == 0) {
+    for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int q = 0; q < 2; ++q) { mbar_init(acc_full(q), 1); mbar_init(acc_empty(q), 128); }
+    *abort_flag = *(volatile unsigned int*)&a.status->error != 0u ? 1 : 0;   // an earlier expired wait: no-op (see tc_stream_kernel)
+    fence_mbar_init();
+    for (int i = 0; i < a.n_seg; ++i) { prefetch_tensormap(&maps.w[i]); prefetch_tensormap(&maps.b[i]); }
+  }
+  if (warp == 1) { tmem_alloc(smem_u32(tmem_slot), ncols); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+
+  auto seg_of = [&](int item) { int si = 0; while (si + 1 < a.n_seg && item >= a.seg[si + 1].item0) ++si; return si; };
+  // worker-major inside a layer as a rule; tile-major with shared weights (see tc_stream_kernel)
+  auto item_worker = [&](const ChainSeg& g, int item) { const int r = item - g.item0; return a.shared_w ? r % a.N : r / g.tiles_m; };
+  auto item_row0 = [&](const ChainSeg& g, int item) { const int r = item - g.item0; return (a.shared_w ? r / a.N : r % g.tiles_m) * 128; };
+  auto load_weights = [&](int si, int s, int ks, int m0, int n) {
+    const uint32_t sa = base + (uint32_t)s * stage_bytes;
+#pragma unroll
+    for (int j = 0; j < 2; ++j) tma_load_3d(sa + j * kTileA, &maps.w[si], full_bar(s), (2 * ks + j) * 64, m0, n);
+  };
+  auto load_operand = [&](int si, int s, int ks, int row0, int n) {
+    const uint32_t sb = base + (uint32_t)s * stage_bytes + 2u * kTileA;
+#pragma unroll
+    for (int j = 0; j < 2; ++j) tma_load_3d(sb + j * b_box, &maps.b[si], full_bar(s), (2 * ks + j) * 64, row0, n);
+  };
+  // early weight loads of this CTA's first item (see tc_stream_kernel), when its layer allows them
+  uint32_t pre = 0;
+  if (warp == 0 && lane == 0 && (int)blockIdx.x < a.total_items) {
+    const int si = seg_of((int)blockIdx.x);
+    const ChainSeg& g = a.seg[si];
+    if (g.prefetch != 0) {
+      const int n = a.shared_w ? 0 : item_worker(g, (int)blockIdx.x), m0 = item_row0(g, (int)blockIdx.x);
+      pre = (uint32_t)(g.k_steps < S ? g.k_steps : S);
+      for (uint32_t ks = 0; ks < pre; ++ks) {
+        mbar_expect_tx(full_bar(ks), stage_bytes);
+        load_weights(si, (int)ks, (int)ks, m0, n);
+      }
+    }
+  }
+  pdl_wait();
+  pdl_trigger();
+  const uint32_t tmem = *tmem_slot;
+  const int total_items = *abort_flag != 0 ? 0 : a.total_items;
+  auto item_active = [&](int n) { return a.active == nullptr || a.active[n] != 0; };
+
+  if (warp == 0 && lane == 0) {
+    // ---------------- producer
+    uint32_t g = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
+      const int si = seg_of(item);
+      const ChainSeg& sg = a.seg[si];
+      const int n = item_worker(sg, item), m0 = item_row0(sg, item);
+      if (!item_active(n)) continue;
+      const int row0 = sg.pool ? (int)draw_block(a.draw.seed, a.draw.worker0 + n, draw_t(a.draw), a.draw.n_blocks) * a.B : 0;
+      for (int ks = 0; ks < sg.k_steps; ++ks, ++g) {
+        const int s = g % S;
+        const uint32_t ph = (g / S) & 1u;
+        if (g >= pre) {
+          ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, a.status, 0x601);
+          if (!ok) break;
+          mbar_expect_tx(full_bar(s), stage_bytes);
+          load_weights(si, s, ks, m0, a.shared_w ? 0 : n);
+        }
+        if (ks == 0 && si > 0) {
+          // a_{l-1} of this worker: every row tile of the layer below must be in global memory
+          ok = flag_wait(a.ready + (size_t)(si - 1) * a.N + n, (unsigned)a.seg[si - 1].tiles_m, abort_flag, a.status, 0x605);
+          if (!ok) break;
+          fence_proxy_async_all();                      // written by other CTAs' plain stores, read below by TMA
+        }
+        load_operand(si, s, ks, row0, n);
+      }
+    }
+    if (total_items == 0 && pre > 0) {   // nothing will consume the early tiles: complete their stages
+      const int si = seg_of((int)blockIdx.x);
+      for (uint32_t ks = 0; ks < pre; ++ks) load_operand(si, (int)ks, (int)ks, 0, 0);
+      g = pre;
+    }
+    if (*abort_flag && g > 0) {   // let the copies already in flight land before the CTA goes away
+      const uint32_t first = g > (uint32_t)S ? g - (uint32_t)S : 0u;
+      for (uint32_t q = first; q < g; ++q) {
+        const long long t0 = clock64();
+        while (!mbar_try_wait(full_bar(q % S), (q / S) & 1u) && clock64() - t0 < 200000000ll) {}
+      }
+    }
+  } else if (warp == 1 && lane == 0) {
+    // ---------------- MMA issuer
+    const uint32_t idesc = idesc_bf16(128, a.B, 0, 0);
+    uint32_t g = 0, it = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
+      const ChainSeg& sg = a.seg[seg_of(item)];
+      if (!item_active(item_worker(sg, item))) continue;
+      const int q = it & 1;
+      ok = mbar_wait(acc_empty(q), ((it >> 1) & 1u) ^ 1u, abort_flag, a.status, 0x604);
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t acc = tmem + (uint32_t)(q * a.B);
+      for (int ks = 0; ks < sg.k_steps; ++ks, ++g) {
+        const int s = g % S;
+        ok = mbar_wait(full_bar(s), (g / S) & 1u, abort_flag, a.status, 0x602);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t sa = base + (uint32_t)s * stage_bytes, sb = sa + 2u * kTileA;
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const uint32_t aj = sa + j * kTileA, bj = sb + j * b_box;
+            mma_bf16(acc, smem_desc_sw128(aj + k * 32u, 16u, 1024u), smem_desc_sw128(bj + k * 32u, 16u, 1024u), idesc,
+                     (ks | j | k) != 0 ? 1u : 0u);
+          }
+        }
+        mma_commit(empty_bar(s));
+      }
+      if (ok) mma_commit(acc_full(q));
+      ++it;
+    }
+  } else if (warp >= 2) {
+    // ---------------- epilogue: thread <-> output feature (see tc_stream_kernel)
+    const int q4 = warp & 3;
+    const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
+    const int batches = a.B / 16;
+    const int etid = tid - 64;                            // 0..127 among the epilogue threads
+    uint32_t it = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
+      const int si = seg_of(item);
+      const ChainSeg& sg = a.seg[si];
+      const int n = item_worker(sg, item);
+      if (!item_active(n)) continue;
+      const int m = item_row0(sg, item) + q4 * 32 + lane;
+      const bool valid = m < sg.M_total;
+      const float bias = valid ? sg.bias[(int64_t)n * a.bias_stride + m] : 0.f;
+      const bool smx = sg.linear != 0 && a.softmax != 0;
+      float gsum = 0.f;                                   // sum over the minibatch of this feature's dZ
+      uint32_t blk = 0;
+      int label = 0;
+      if (smx) {                                          // the label of this thread's row, fetched ahead of the wait
+        blk = draw_block(a.draw.seed, a.draw.worker0 + n, draw_t(a.draw), a.draw.n_blocks);
+        label = a.Y[(int64_t)n * a.P + (int64_t)blk * a.B + etid / (128 / a.B)];
+      }
+      const int q = it & 1;
+      ok = __all_sync(0xffffffffu, mbar_wait(acc_full(q), (it >> 1) & 1u, abort_flag, a.status, 0x603));
+      if (!ok) break;
+      tc_fence_after();
+      for (int bi = 0; bi < batches; ++bi) {
+        const int c0 = bi * 16;
+        uint32_t v[16];
+        tmem_ld16(tmem + lane_off + (uint32_t)(q * a.B + c0), v);
+        tmem_ld_wait();
+        if (valid) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const int64_t o = ((int64_t)n * a.B + c0 + j) * sg.ld_out + m;
+            const float x = __uint_as_float(v[j]) + bias;
+            if (sg.linear == 0) sg.out_bk[o] = f32_to_bf16_rn(fmaxf(x, 0.f));
+            else if (smx) zs[(c0 + j) * kLogitLd + m] = x;
+            else sg.out_f32[o] = x;
+          }
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(acc_empty(q));
+      ++it;
+      if (si + 1 < a.n_seg) {
+        // this row tile of a_l is in global memory: count it for the items of layer l + 1 of this worker
+        __threadfence();
+        named_bar_sync(2, 128);
+        if (etid == 0) red_release_add(a.ready + (size_t)si * a.N + n, 1u);
+      }
+      if (smx) {
+        // softmax cross-entropy gradient and the step of b_L (see tc_stream_kernel)
+        named_bar_sync(1, 128);
+        const int C = sg.M_total;
+        const int T = 128 / a.B, sub = etid % T, b = etid / T;
+        const float invB = 1.f / (float)a.B;
+        float* z = zs + b * kLogitLd;
+        float mx = -INFINITY;
+        for (int cc = sub; cc < C; cc += T) mx = fmaxf(mx, z[cc]);
+        for (int o = T >> 1; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        float se = 0.f;
+        for (int cc = sub; cc < C; cc += T) se += expf(z[cc] - mx);
+        for (int o = T >> 1; o > 0; o >>= 1) se += __shfl_xor_sync(0xffffffffu, se, o);
+        const float lse = mx + logf(se);
+        const float zl = z[label];
+        __syncwarp();
+        for (int cc = sub; cc < C; cc += T) z[cc] = (expf(z[cc] - lse) - (cc == label ? 1.f : 0.f)) * invB;
+        if (sub == 0) a.row_losses[(int64_t)n * a.B + b] = lse - zl;
+        if (etid == 0) a.draws[n] = (int32_t)blk;
+        named_bar_sync(1, 128);
+        if (valid) {
+          for (int bb = 0; bb < a.B; ++bb) gsum += zs[bb * kLogitLd + m];
+        }
+        uint16_t* dn = a.delta_bk + (int64_t)n * a.B * a.ld_delta;
+        for (int idx = etid; idx < a.B * C; idx += 128) {
+          const int bb = idx / C, cc = idx - bb * C;
+          dn[bb * a.ld_delta + cc] = f32_to_bf16_rn(zs[bb * kLogitLd + cc]);
+        }
+        named_bar_sync(1, 128);                           // the tile is free for the next item
+        if (a.bias_rw != nullptr && valid) {
+          float* bp = a.bias_rw + (int64_t)n * a.bias_stride + m;
+          if (a.bias_vel != nullptr) {                    // momentum form of the local step
+            float* vp = a.bias_vel + (int64_t)n * a.bias_stride + m;
+            gsum = fmaf(a.mu, *vp, gsum);
+            *vp = gsum;
+          }
+          *bp = fmaf(-a.gamma, gsum, *bp);
+        }
+      }
+    }
+  }
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem, ncols);
+  if (tid == 0) {
+    // the last CTA to get here has seen every other CTA finish all its waits: zero the counters for the next launch
+    __threadfence();
+    const unsigned int before = atomicAdd(a.done, 1u);
+    if (before == gridDim.x - 1) {
+      for (int i = 0; i < a.n_seg * a.N; ++i) a.ready[i] = 0u;
+      *a.done = 0u;
+      __threadfence();
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
 // update kernel: dW GEMM (K = B) + in-place SGD step, optionally fused with the node average
 // ---------------------------------------------------------------------------------------------
 struct UpdateArgs {
@@ -448,7 +743,12 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
                                                                    const UpdateArgs a) {
   using namespace ptx;
   using Cfg = UpdCfg<TN, MOM>;
-  constexpr int S = Cfg::kStages;
+  // Fused form, plain step, 64-wide tiles: the averaged tile (fp32 + bf16, 48 KB) is written to a buffer of its
+  // own that takes the place of the fourth pipeline stage.  Its N row stores last ~17 us at one SM's share of
+  // the HBM bandwidth; from a stage they would stall the loader for that long, from the buffer the three
+  // remaining stages keep cycling through the next tile's workers meanwhile.
+  constexpr bool kOutBuf = FUSE && !MOM && TN == 64;
+  constexpr int S = kOutBuf ? Cfg::kStages - 1 : Cfg::kStages;
   constexpr int NB32 = TN / 32, NB64 = TN / 64;
   // Fused form on shared weights (every worker's master tile holds the same bits): all loads of a tile read
   // worker 0's copy; with 64-wide tiles and the plain step the tile is loaded ONCE, by its first worker, and
@@ -462,15 +762,17 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
   auto master_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes; };
   auto vel_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes + Cfg::kMaster; };
   auto ops_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes + Cfg::kMaster + Cfg::kVel; };
-  const uint32_t bar0 = base + (uint32_t)S * stage_bytes;
+  const uint32_t bar0 = base + (uint32_t)Cfg::kStages * stage_bytes;
   auto full_ops = [&](int s) { return bar0 + 8u * s; };
   auto full_w = [&](int s) { return bar0 + 32u + 8u * s; };
   auto stage_empty = [&](int s) { return bar0 + 64u + 8u * s; };
   auto acc_full = [&](int s) { return bar0 + 96u + 8u * s; };
   auto acc_empty = [&](int s) { return bar0 + 128u + 8u * s; };
   auto tile_ready = [&](int s) { return bar0 + 160u + 8u * s; };
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen + (size_t)S * stage_bytes + 192);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + (size_t)S * stage_bytes + 196);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen + (size_t)Cfg::kStages * stage_bytes + 192);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + (size_t)Cfg::kStages * stage_bytes + 196);
+  const uint32_t out_free = bar0 + 200u;               // kOutBuf: the row stores have read the output buffer
+  const uint32_t out_u32 = base + (uint32_t)S * stage_bytes;     // kOutBuf: fp32 tile, then the bf16 tile
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t op_box = (uint32_t)a.B * 128u;       // one {64, B} box
@@ -482,6 +784,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
       mbar_init(full_ops(s), 1); mbar_init(full_w(s), 1); mbar_init(stage_empty(s), 1);
       mbar_init(acc_full(s), 1); mbar_init(acc_empty(s), 128); mbar_init(tile_ready(s), 128);
     }
+    mbar_init(out_free, 1);
     *abort_flag = *(volatile unsigned int*)&a.status->error != 0u ? 1 : 0;   // an earlier expired wait: no-op (see tc_stream_kernel)
     fence_mbar_init();
     prefetch_tensormap(&mapDelta); prefetch_tensormap(&mapAct);
@@ -618,6 +921,21 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
         tma_wait_group_read0();
         mbar_arrive(stage_empty(s));
         ++it;
+      } else if (kOutBuf) {
+        ok = mbar_wait(tile_ready(0), tile_it & 1u, abort_flag, a.status, 0x209);
+        if (!ok) break;
+        // one row at a time: a burst of all N rows would sit in the copy engine's queue ahead of the next
+        // tile's operand loads for as long as the memory system takes to absorb it
+        for (int n = 0; n < a.N; ++n) {
+#pragma unroll
+          for (int q = 0; q < NB32; ++q) tma_store_3d(&mapMaster, out_u32 + q * 16384u, n0 + 32 * q, m0, n);
+#pragma unroll
+          for (int h = 0; h < NB64; ++h) tma_store_3d(&mapShadow, out_u32 + Cfg::kMaster + h * 16384u, n0 + 64 * h, m0, n);
+          tma_commit_group();
+          tma_wait_group_read0();
+        }
+        mbar_arrive(out_free);
+        ++tile_it;
       } else if (MOM && a.avg_vel == 0) {
         // every worker's new momentum tile goes back to its own row; the last worker's stage also holds the
         // averaged models, which go to every row
@@ -668,9 +986,9 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
     const bool shared_x = kShareOnce && a.shared_w != 0;
     const bool avg_vel = FUSE && MOM && a.avg_vel != 0;
     const bool vel_per_worker = FUSE && MOM && a.avg_vel == 0;      // the storer takes every worker's momentum tile
-    uint32_t it = 0;
+    uint32_t it = 0, tile_it = 0;
     bool ok = true;
-    for (int w = blockIdx.x; w < total_items && ok; w += gridDim.x) {
+    for (int w = blockIdx.x; w < total_items && ok; w += gridDim.x, ++tile_it) {
       const int n_begin = FUSE ? 0 : w / tiles, n_end = FUSE ? a.N : n_begin + 1;
       float sum[NSUM], vsum[NVSUM];
       float xr[NXR];                                        // shared weights: the tile every worker starts from
@@ -691,6 +1009,15 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
         uint8_t* mst = gen + (size_t)s * stage_bytes;
         uint8_t* stg = mst + Cfg::kMaster + Cfg::kVel;
         const bool last = FUSE && n == a.N - 1;
+        uint8_t* dst_w = mst;                               // where the tile to be stored is written
+        if (kOutBuf && last) {
+          dst_w = gen + (size_t)S * stage_bytes;
+          stg = dst_w + Cfg::kMaster;
+          if (tile_it > 0) {                                // the previous tile's row stores have read the buffer
+            ok = __all_sync(0xffffffffu, mbar_wait(out_free, (tile_it - 1) & 1u, abort_flag, a.status, 0x20A));
+            if (!ok) break;
+          }
+        }
 #pragma unroll
         for (int c = 0; c < NB32; ++c) {
           uint32_t v[32];
@@ -748,7 +1075,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
               }
             }
             if (!FUSE || last) {
-              *pw = x;
+              *reinterpret_cast<float4*>(dst_w + c * 16384 + row_off + (((uint32_t)j ^ sw) << 4)) = x;
               // two neighbouring fp32 chunks make one 16-byte bf16 chunk: a single conflict-free store
               if ((j & 1) == 0) {
                 lo = make_uint2(pack_bf16x2(x.x, x.y), pack_bf16x2(x.z, x.w));
@@ -765,10 +1092,14 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
         if (!FUSE || vel_per_worker) {
           fence_proxy_async();
           mbar_arrive(tile_ready(s));
-        } else if (last) {
+        } else if (last && !kOutBuf) {
           fence_proxy_async();
           mbar_arrive(tile_ready(0));
         } else {
+          if (kOutBuf && last) {                            // the averaged tile sits in its own buffer: hand it over
+            fence_proxy_async();
+            mbar_arrive(tile_ready(0));
+          }
           named_bar_sync(1, 128);                         // every epilogue thread is done reading stage s
           if (etid == 0) mbar_arrive(stage_empty(s));
         }
@@ -1594,6 +1925,7 @@ inline int tc_create(prsgd_ctx* c, std::string* err) {
   const int big_sm = (int)stream_smem_bytes(c->B, true);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_stream_kernel<TC_FWD_LINEAR>, cudaFuncAttributeMaxDynamicSharedMemorySize, big > big_sm ? big : big_sm);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_stream_kernel<TC_DX>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_forward_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, big > big_sm ? big : big_sm);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<false, 64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<64, false>::smem(c->B));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<true, 64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<64, false>::smem(c->B));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<false, 128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<128, false>::smem(c->B));
@@ -1683,6 +2015,48 @@ inline void tc_launch_forward(prsgd_ctx* c, int l, const DrawArgs& dr, const uin
     launch_pdl(tc_stream_kernel<TC_FWD_RELU>, grid, kStreamThreads, smem, c->stream, st->layer[l - 1].shadow_k, st->layer[l - 1].act_in, a);
   else
     launch_pdl(tc_stream_kernel<TC_FWD_LINEAR>, grid, kStreamThreads, smem, c->stream, st->layer[l - 1].shadow_k, st->layer[l - 1].act_in, a);
+}
+
+// forward GEMMs of layers l_first..L as one launch (tc_forward_chain_kernel)
+inline bool tc_chain_applies(const prsgd_ctx* c, int l_first) {
+  const int n_seg = c->L - l_first + 1;
+  return c->forward_chain != 0 && n_seg >= 2 && n_seg <= kChainMax;
+}
+
+inline void tc_launch_forward_chain(prsgd_ctx* c, int l_first, const DrawArgs& dr, const uint8_t* active) {
+  TcState* st = static_cast<TcState*>(c->tc);
+  ChainMaps maps;
+  ChainArgs a{};
+  a.B = c->B; a.N = c->N; a.n_seg = c->L - l_first + 1;
+  a.shared_w = tc_shared_restart(c, active) ? 1 : 0;
+  a.softmax = tc_epilogues_fused(c) ? 1 : 0;
+  a.stages = stream_stages(c->B, a.softmax != 0);
+  a.draw = dr; a.active = active; a.status = c->status; a.bias_stride = c->m_pad;
+  a.ready = c->chain_ready; a.done = c->chain_ready + (size_t)kChainMax * c->N;
+  int items = 0;
+  for (int l = l_first; l <= c->L; ++l) {
+    const Layer& ly = c->layer[l - 1];
+    ChainSeg& g = a.seg[l - l_first];
+    g.k_steps = (ly.d_in / 64 + 1) / 2; g.tiles_m = (ly.d_out + 127) / 128; g.M_total = ly.d_out; g.ld_out = c->buf.ld[l];
+    g.linear = l == c->L ? 1 : 0; g.pool = l == 1 ? 1 : 0;
+    g.prefetch = (l > 1 && active == nullptr && c->early_loads) ? 1 : 0;   // W_1 was written by the launch just before
+    g.item0 = items;
+    g.out_bk = c->buf.act_bk[l]; g.out_f32 = c->buf.act_f32[l]; g.bias = c->params + ly.b_off;
+    items += g.tiles_m * c->N;
+    maps.w[l - l_first] = st->layer[l - 1].shadow_k;
+    maps.b[l - l_first] = st->layer[l - 1].act_in;
+  }
+  for (int i = a.n_seg; i < kChainMax; ++i) { maps.w[i] = maps.w[0]; maps.b[i] = maps.b[0]; }
+  a.total_items = items;
+  if (a.softmax) {
+    const Layer& ly = c->layer[c->L - 1];
+    a.Y = c->Y; a.P = c->P; a.delta_bk = c->buf.delta_bk[c->L]; a.ld_delta = c->buf.ld[c->L];
+    a.row_losses = c->losses; a.draws = c->draws;
+    a.bias_rw = c->params + ly.b_off; a.gamma = c->gamma; a.mu = c->mu;
+    a.bias_vel = c->velocity != nullptr ? c->velocity + ly.b_off : nullptr;
+  }
+  dim3 grid(items < st->num_sms ? items : st->num_sms);
+  launch_pdl(tc_forward_chain_kernel, grid, kStreamThreads, stream_smem_bytes(c->B, a.softmax != 0), c->stream, maps, a);
 }
 
 // dZ_{l-1} from dZ_l through W_l (l >= 2)

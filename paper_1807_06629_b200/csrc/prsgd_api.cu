@@ -117,7 +117,9 @@ size_t carve_scratch(int N, const prsgd_model_spec* s, int64_t m_pad, prsgd_ctx*
   auto active = take((size_t)N);
   auto stage = take(sizeof(float) * (size_t)m_pad);
   auto tdev = take(sizeof(int64_t));
+  auto chain = take(sizeof(unsigned int) * ((size_t)kChainMax * N + 1));
   if (ctx) {
+    ctx->chain_ready = reinterpret_cast<unsigned int*>(chain);
     ctx->t_dev = reinterpret_cast<int64_t*>(tdev);
     ctx->status = reinterpret_cast<DeviceStatus*>(status);
     ctx->draws = reinterpret_cast<int32_t*>(draws);
@@ -295,10 +297,16 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging, bool more_follow) {
   const bool next_fwd = c->next_forward && more_follow && !averaging && L > 1 && tc_epilogues_fused(c);
   const bool skip_f1 = c->a1_ready;
   c->a1_ready = false;
-  for (int l = skip_f1 ? 2 : 1; l <= L; ++l) {
+  if (tc_chain_applies(c, skip_f1 ? 2 : 1)) {          // every remaining layer's forward GEMM in one launch
     prof_begin(c, PRSGD_KERNEL_FORWARD);
-    tc_launch_forward(c, l, dr, act_mask);
+    tc_launch_forward_chain(c, skip_f1 ? 2 : 1, dr, act_mask);
     LAUNCH_CHECK(c);
+  } else {
+    for (int l = skip_f1 ? 2 : 1; l <= L; ++l) {
+      prof_begin(c, PRSGD_KERNEL_FORWARD);
+      tc_launch_forward(c, l, dr, act_mask);
+      LAUNCH_CHECK(c);
+    }
   }
   const bool epi = tc_epilogues_fused(c);
   if (!epi) {
@@ -630,7 +638,7 @@ void period_key(const prsgd_ctx* c, uint64_t (&key)[13]) {
   key[4] = c->has_mask ? 1 : 0; key[5] = reinterpret_cast<uint64_t>(c->velocity); key[6] = mbits;
   key[7] = (uint64_t)c->average_velocity; key[8] = reinterpret_cast<uint64_t>(c->X);
   key[9] = reinterpret_cast<uint64_t>(c->Y); key[10] = (uint64_t)c->worker0; key[11] = (uint64_t)c->fused_epilogues | ((uint64_t)c->early_loads << 1) | ((uint64_t)c->next_forward << 2) | ((uint64_t)c->dx_in_update << 3);
-  key[12] = (c->rows_identical ? 1u : 0u) | ((uint64_t)c->shared_restart << 1);   // the period's first iteration may share reads
+  key[12] = (c->rows_identical ? 1u : 0u) | ((uint64_t)c->shared_restart << 1) | ((uint64_t)c->forward_chain << 2);   // the period's first iteration may share reads
 }
 
 // One whole averaging period (I iterations starting right after an average) as a CUDA graph: the
@@ -988,6 +996,7 @@ int prsgd_set_option(prsgd_ctx* c, int32_t option, int64_t value) {
   if (option == PRSGD_OPT_NEXT_FORWARD) { c->next_forward = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_CHECK_FINITE) { c->check_finite = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_SHARED_RESTART) { c->shared_restart = value != 0; return PRSGD_OK; }
+  if (option == PRSGD_OPT_FORWARD_CHAIN) { c->forward_chain = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_DX_IN_UPDATE) {
     if (value < 0 || value > 2) return fail(c, PRSGD_ERR_ARG, "PRSGD_OPT_DX_IN_UPDATE takes 0, 1 or 2");
     c->dx_in_update = (int)value;
@@ -1039,6 +1048,8 @@ int prsgd_selftest_wait_expiry(prsgd_ctx* c, int32_t limit_us) {
 int prsgd_clear_device_error(prsgd_ctx* c) {
   if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
   CUDA_TRY(c, cudaMemsetAsync(c->status, 0, sizeof(DeviceStatus), c->stream));
+  // an interrupted forward chain may have left its counters half way
+  CUDA_TRY(c, cudaMemsetAsync(c->chain_ready, 0, sizeof(unsigned int) * ((size_t)kChainMax * c->N + 1), c->stream));
   CUDA_TRY(c, cudaStreamSynchronize(c->stream));
   c->err.clear();
   c->rows_identical = false;     // whatever the interrupted launches left

@@ -66,6 +66,39 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
 }
 
+// ---- counters in global memory that one CTA raises and another waits for ------------------------------
+__device__ __forceinline__ void red_release_add(unsigned int* p, unsigned int v) {
+  asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ unsigned int ld_acquire(const unsigned int* p) {
+  unsigned int v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+// orders earlier generic-proxy accesses (the acquire above) before later async-proxy ones (TMA loads) in every space
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
+// Bounded wait until *counter >= target; same limit and error reporting as mbar_wait.
+__device__ __forceinline__ bool flag_wait(const unsigned int* counter, unsigned int target, volatile int* abort_flag,
+                                          DeviceStatus* status, unsigned what,
+                                          long long limit_cycles = kWaitLimitCycles) {
+  if (ld_acquire(counter) >= target) return true;
+  long long t0 = 0;
+  for (uint32_t it = 1;; ++it) {
+    if (ld_acquire(counter) >= target) return true;
+    if ((it & 63u) == 0u) {
+      if (*abort_flag) return false;
+      const long long now = clock64();
+      if (t0 == 0) t0 = now;
+      if (now - t0 > limit_cycles) {
+        *abort_flag = 1;
+        if (atomicCAS(&status->error, 0u, what) == 0u) status->where = blockIdx.x;
+        return false;
+      }
+    }
+  }
+}
+
 // ---- TMA (tiled; every load targets this CTA's own shared memory) -------------------------
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
   asm volatile(

@@ -313,6 +313,41 @@ def test_folded_kernels_with_a_worker_mask_change_no_bit(torch_cuda):
             assert np.array_equal(outs[0][2][active], o[2][active])
 
 
+def test_forward_chain_in_one_launch_changes_no_bit(torch_cuda):
+    """The forward GEMMs of all layers as one launch whose items wait per (layer, worker) for the activations
+    below them, against one launch per layer: identical parameters, losses and draws over several periods,
+    direct and replayed, with a worker mask, with momentum, for deep and ragged nets; fewer launches."""
+    torch = torch_cuda
+    from paper_1807_06629_b200 import binding
+    cases = (SMALL[1], SMALL[2], SMALL[3], SMALL[4], SMALL[6], _w("tc-chain-n7", 7, (192, 128, 256, 10), 32, I=3),
+             _w("tc-chain-200", 2, (64, 128, 200), 32), _w("tc-chain-wide", 3, (64, 448, 320, 10), 16, I=4))
+    for w in cases:
+        X, Y, x0 = make_inputs(w)
+        for variant in ("plain", "mask", "momentum"):
+            outs = []
+            for chain, graph in ((0, 0), (1, 0), (1, 1)):
+                with torch.cuda.stream(torch.cuda.Stream()):
+                    p = make_ctx(w, X, Y, x0)
+                    p.set_option(binding.OPT_FORWARD_CHAIN, chain)
+                    p.set_option(binding.OPT_GRAPH, graph)
+                    if variant == "mask":
+                        p.set_active([1 if i % 2 == 0 else 0 for i in range(w.N)])
+                    if variant == "momentum":
+                        p.enable_momentum(0.9)
+                    n0 = p.get_launch_count()
+                    p.local_steps(2)
+                    p.local_steps(3 * w.I + 1)
+                    outs.append((p.get_params_stacked(), p.get_losses(), p.get_draws().tolist(), p.get_launch_count() - n0))
+                    torch.cuda.current_stream().synchronize()
+                    p.close()
+            keep = [i for i in range(w.N) if variant != "mask" or i % 2 == 0]
+            for o in outs[1:]:
+                assert np.array_equal(outs[0][0], o[0]), (w.name, variant)
+                assert np.array_equal(outs[0][1][keep], o[1][keep])
+                assert [outs[0][2][i] for i in keep] == [o[2][i] for i in keep]
+            assert outs[1][3] < outs[0][3]
+
+
 def test_reading_the_common_restart_point_once_changes_no_bit(torch_cuda):
     """After a node average all N rows hold the same bits, so the following iteration's forward, dX and fused
     update + average launches read worker 0's weights for every worker (PRSGD_OPT_SHARED_RESTART).  Against
