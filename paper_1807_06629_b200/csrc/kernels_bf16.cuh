@@ -2039,7 +2039,9 @@ inline void tc_launch_forward_chain(prsgd_ctx* c, int l_first, const DrawArgs& d
     ChainSeg& g = a.seg[l - l_first];
     g.k_steps = (ly.d_in / 64 + 1) / 2; g.tiles_m = (ly.d_out + 127) / 128; g.M_total = ly.d_out; g.ld_out = c->buf.ld[l];
     g.linear = l == c->L ? 1 : 0; g.pool = l == 1 ? 1 : 0;
-    g.prefetch = (l > 1 && active == nullptr && c->early_loads) ? 1 : 0;   // W_1 was written by the launch just before
+    // early weight loads overlap whatever launch precedes the whole forward pass: only when that launch is known
+    // to leave the weights of layers >= 2 alone (the layer-1 update or a bias launch that ended the iteration before)
+    g.prefetch = (l > 1 && active == nullptr && c->early_loads && c->upper_weights_quiet) ? 1 : 0;
     g.item0 = items;
     g.out_bk = c->buf.act_bk[l]; g.out_f32 = c->buf.act_f32[l]; g.bias = c->params + ly.b_off;
     items += g.tiles_m * c->N;

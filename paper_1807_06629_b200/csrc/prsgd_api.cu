@@ -37,6 +37,7 @@ int fail(prsgd_ctx* ctx, int code, const std::string& msg) {
     if (e__ != cudaSuccess)                                                                    \
       return fail((ctx), PRSGD_ERR_CUDA, std::string("kernel launch: ") + cudaGetErrorString(e__)); \
     (ctx)->launches++;                                                                         \
+    (ctx)->upper_weights_quiet = false;                                                        \
     prof_end(ctx);                                                                             \
   } while (0)
 
@@ -369,6 +370,8 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging, bool more_follow) {
       LAUNCH_CHECK(c);
     }
   }
+  // the iteration ends with layer 1's update (or a bias launch after it): nothing in flight writes W_2..W_L
+  c->upper_weights_quiet = true;
   return PRSGD_OK;
 }
 

@@ -101,7 +101,8 @@ struct prsgd_ctx {
   int early_loads = 1;           // tensor-core kernels request tiles nobody is writing before their dependency wait
   int fused_epilogues = 1;       // softmax-CE gradient and bias steps inside the GEMM epilogues (tensor-core path)
   int shared_restart = 1;        // the iteration after a node average reads worker 0's weights for every worker
-  int forward_chain = 1;         // the forward GEMMs of consecutive layers run as one launch (tensor-core path)
+  int forward_chain = 0;         // the forward GEMMs of consecutive layers run as one launch (tensor-core path)
+  bool upper_weights_quiet = false;      // the launch enqueued last does not write the weights of any layer >= 2
   unsigned int* chain_ready = nullptr;   // [8][N] row-tile counters of the forward chain + one word, zero between launches
   bool rows_identical = false;   // every row of the store (and of the bf16 copy) holds the same bits right now
   int64_t assigned_upto = -1;    // prsgd_assign_rows calls since the last local step have covered columns [0, assigned_upto)
