@@ -372,13 +372,13 @@ def workload_config(w, extra=None, momentum=None):
 
 
 # ----------------------------------------------------------------------------- averaging sweep
-def averaging_sweep(torch, binding, peaks, dev, quick=False):
+def averaging_sweep(torch, binding, peaks, dev, points=None):
     """Node-average kernel in isolation on [N, m] fp32: GB/s counting N*m*4 read + N*m*4 written."""
     out = []
-    for N in synth.SWEEP_N:
-        for m in synth.SWEEP_M:
-            if quick and N * m > 64 * 11_000_000:
-                continue
+    if points is None:
+        points = [(N, m) for N in synth.SWEEP_N for m in synth.SWEEP_M]
+    for (N, m) in points:
+        if True:
             nbytes = N * m * 4
             copies = max(1, int(np.ceil(2 * L2_BYTES / nbytes))) if nbytes <= 2 * L2_BYTES else 1
             bufs = [torch.randn(N, m, device=dev, dtype=torch.float32) for _ in range(copies)]
@@ -583,6 +583,8 @@ def parse_args(argv=None):
     ap.add_argument("--force-sharded", action="store_true",
                     help="run the multi-GPU code path (sharded workers + all-reduce average) even on one GPU")
     ap.add_argument("--no-sweep", action="store_true", help="skip the averaging-kernel sweep")
+    ap.add_argument("--sweep-only", default=None, metavar="NxM[,NxM...]",
+                    help="run only the averaging kernel on these [N, m] shapes (small cases for profiler captures) and print their line")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle timing")
     ap.add_argument("--no-configs", action="store_true", help="skip the short runs of the other configurations")
     args = ap.parse_args(argv)
@@ -625,6 +627,10 @@ def main(argv=None):
         dist.barrier()            # (also: the library rank 0 may just have built is in place for every rank)
     from paper_1807_06629_b200 import binding
     peaks = load_peaks()
+    if args.sweep_only:
+        pts = [tuple(int(v) for v in p.lower().split("x")) for p in args.sweep_only.split(",")]
+        print(json.dumps({"averaging_sweep": averaging_sweep(torch, binding, peaks, dev, pts)}), flush=True)
+        return
 
     res, (wl, X, Y, x0) = measure_config(torch, w, args, dev, rank, world, args.scaling, args.steps, args.warmup, peaks,
                                          sharded_mode, with_e2e=True, with_clocks=True)

@@ -963,9 +963,11 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
         const int s = (it - 1) % S;                       // stage of the tile's last worker
         ok = mbar_wait(tile_ready(0), tile_it & 1u, abort_flag, a.status, 0x205);
         if (!ok) break;
-        for (int n = 0; n < a.N; ++n) store_tile(s, m0, n0, n);
-        tma_commit_group();
-        tma_wait_group_read0();
+        for (int n = 0; n < a.N; ++n) {                   // one row at a time (see the buffered form above)
+          store_tile(s, m0, n0, n);
+          tma_commit_group();
+          tma_wait_group_read0();
+        }
         mbar_arrive(stage_empty(s));
         ++tile_it;
       }
