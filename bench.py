@@ -227,7 +227,7 @@ def ncu_traffic_per_launch(workload: str, family: str, N: int):
 # ----------------------------------------------------------------------------- byte model
 def period_bytes(w: synth.Workload, m_pad: int, sms: int = 148, momentum: bool = False, fused_average: bool = True,
                  fused_epilogues: bool = True, next_forward: bool = True, dx_in_update=True,
-                 shared_restart: bool = True, forward_chain: bool = True) -> dict:
+                 shared_restart: bool = True, forward_chain: bool = False) -> dict:
     """Algorithmic HBM bytes and launch counts of ONE averaging period (prsgd_local_steps(I) from a period
     boundary) of all N workers, per kernel family: {family: [bytes, launches]}.
 
@@ -449,6 +449,10 @@ def measure_config(torch, w_cfg, args, dev, rank, world, scaling, steps, warmup,
             p.set_option(opt, 0)
     if args.fold_all_dx:
         p.set_option(binding.OPT_DX_IN_UPDATE, 2)
+    if args.forward_chain:
+        p.set_option(binding.OPT_FORWARD_CHAIN, 1)
+    if args.worker_groups is not None:
+        p.set_option(binding.OPT_WORKER_GROUPS, args.worker_groups)
     working_set = p.params.numel() * 4 + (p.shadow.numel() * 2 if p.shadow is not None else 0)
     need_flush = working_set <= 2 * L2_BYTES
     flush = torch.empty(3 * L2_BYTES // 4, dtype=torch.float32, device=dev) if need_flush else None
@@ -492,7 +496,7 @@ def measure_config(torch, w_cfg, args, dev, rank, world, scaling, steps, warmup,
                              momentum=args.momentum is not None, fused_average=not args.no_fuse,
                              fused_epilogues=not args.no_fused_epilogues, next_forward=not args.no_next_forward,
                              dx_in_update=0 if args.no_dx_in_update else (2 if args.fold_all_dx else 1),
-                             shared_restart=not args.no_shared_restart, forward_chain=not args.no_forward_chain)
+                             shared_restart=not args.no_shared_restart, forward_chain=args.forward_chain)
     if sharded_mode:          # a shard's period: I plain iterations, then the average as passes of their own
         fam_model = period_bytes(w.with_(I=0), p.m_pad, torch.cuda.get_device_properties(dev).multi_processor_count,
                                  momentum=args.momentum is not None, fused_epilogues=not args.no_fused_epilogues,
@@ -574,6 +578,9 @@ def parse_args(argv=None):
                     help="form dZ of the layer below inside the update launch for every layer, whatever its size")
     ap.add_argument("--no-shared-restart", action="store_true",
                     help="the iteration after an average reads every worker's own copy of the common point")
+    ap.add_argument("--worker-groups", type=int, default=None,
+                    help="plain iterations as this many independent launch chains (one per group of workers) on streams of their own")
+    ap.add_argument("--forward-chain", action="store_true", help="one forward launch for all layers")
     ap.add_argument("--no-forward-chain", action="store_true",
                     help="one forward launch per layer instead of one launch for all layers")
     ap.add_argument("--no-next-forward", action="store_true",

@@ -303,6 +303,13 @@ int prsgd_get_velocity_stacked(prsgd_ctx* ctx, float* dst, int dst_on_device);
  * (layer, worker) in the scratch area, since workers do not depend on one another inside an iteration.
  * With 0 every layer is a launch of its own.  Same bits either way. */
 #define PRSGD_OPT_FORWARD_CHAIN 11
+/* PRSGD_OPT_WORKER_GROUPS (default 1 = off; 2..4, tensor-core path): inside an epoch the workers need no
+ * synchronisation (the text after Algorithm 1), so the plain iterations between two averages are enqueued as
+ * G independent chains of launches, one per contiguous group of N/G workers, on G streams the library creates
+ * for itself; they fork from the context's stream and join it again before the averaging iteration.  While
+ * one group's long update kernels run, another group's short launches find free SMs.  Not while a worker
+ * mask or profiling is on.  Same bits as one chain for all workers. */
+#define PRSGD_OPT_WORKER_GROUPS 12
 /* PRSGD_OPT_CHECK_FINITE (default 0): when 1, prsgd_sync also runs prsgd_check_finite. */
 #define PRSGD_OPT_CHECK_FINITE 9
 int prsgd_set_option(prsgd_ctx* ctx, int32_t option, int64_t value);

@@ -2019,10 +2019,16 @@ inline void tc_launch_forward(prsgd_ctx* c, int l, const DrawArgs& dr, const uin
     launch_pdl(tc_stream_kernel<TC_FWD_LINEAR>, grid, kStreamThreads, smem, c->stream, st->layer[l - 1].shadow_k, st->layer[l - 1].act_in, a);
 }
 
+// The per-worker flags the launches being enqueued honour: Algorithm 3's mask, or the mask of a worker group.
+inline const uint8_t* worker_mask(const prsgd_ctx* c) {
+  if (c->group_active != nullptr) return c->group_active;
+  return c->has_mask ? c->active : nullptr;
+}
+
 // forward GEMMs of layers l_first..L as one launch (tc_forward_chain_kernel)
 inline bool tc_chain_applies(const prsgd_ctx* c, int l_first) {
   const int n_seg = c->L - l_first + 1;
-  return c->forward_chain != 0 && n_seg >= 2 && n_seg <= kChainMax;
+  return c->forward_chain != 0 && n_seg >= 2 && n_seg <= kChainMax && c->group_active == nullptr;   // (its counters serve one chain at a time)
 }
 
 inline void tc_launch_forward_chain(prsgd_ctx* c, int l_first, const DrawArgs& dr, const uint8_t* active) {
@@ -2133,7 +2139,7 @@ inline void tc_launch_update_dx_m(prsgd_ctx* c, int l) {
   a.out_bk = c->buf.delta_bk[l - 1]; a.mask_src = c->buf.act_bk[l - 1]; a.ld_out = c->buf.ld[l - 1]; a.M_total = ly.d_in;
   a.bias_rw = c->params + c->layer[l - 2].b_off; a.bias_stride = c->m_pad;
   a.mu = c->mu; a.bias_vel = MOM ? c->velocity + c->layer[l - 2].b_off : nullptr;
-  a.active = c->has_mask ? c->active : nullptr;
+  a.active = worker_mask(c);
   const int items = a.tiles_n * c->N;
   const int grid = items < st->num_sms ? items : st->num_sms;
   const TcLayerMaps& mp = st->layer[l - 1];
@@ -2164,7 +2170,7 @@ inline void tc_launch_update_next_tn(prsgd_ctx* c, const DrawArgs& dr) {
   UpdateNextArgs a{};
   a.B = c->B; a.N = c->N; a.tiles_m = (ly.d_out + 127) / 128; a.tiles_n = (ly.d_in + TN - 1) / TN;
   a.gamma = c->gamma; a.mu = c->mu; a.draw = dr; a.status = c->status;
-  a.active = c->has_mask ? c->active : nullptr;
+  a.active = worker_mask(c);
   a.stages = UpdNextCfg<TN, MOM>::stages(c->B);
   a.next_out = c->buf.act_bk[1]; a.next_ld = c->buf.ld[1];
   a.bias = c->params + ly.b_off; a.bias_stride = c->m_pad; a.M_total = ly.d_out;

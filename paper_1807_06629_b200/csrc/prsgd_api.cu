@@ -119,7 +119,9 @@ size_t carve_scratch(int N, const prsgd_model_spec* s, int64_t m_pad, prsgd_ctx*
   auto stage = take(sizeof(float) * (size_t)m_pad);
   auto tdev = take(sizeof(int64_t));
   auto chain = take(sizeof(unsigned int) * ((size_t)kChainMax * N + 1));
+  auto gmasks = take((size_t)kMaxGroups * N);
   if (ctx) {
+    ctx->group_masks = gmasks;
     ctx->chain_ready = reinterpret_cast<unsigned int*>(chain);
     ctx->t_dev = reinterpret_cast<int64_t*>(tdev);
     ctx->status = reinterpret_cast<DeviceStatus*>(status);
@@ -288,7 +290,7 @@ int step_f32(prsgd_ctx* c, int64_t t, bool averaging) {
 // `more_follow`: the caller runs iteration t + 1 right after this one (same call, nothing in between).
 int step_bf16(prsgd_ctx* c, int64_t t, bool averaging, bool more_follow) {
   const int L = c->L, N = c->N;
-  const uint8_t* act_mask = c->has_mask ? c->active : nullptr;
+  const uint8_t* act_mask = worker_mask(c);
   const bool fuse = averaging && c->fused_average;
   const bool avg_vel = c->velocity != nullptr && c->average_velocity;
   const DrawArgs dr = draw_args(c, t);
@@ -308,6 +310,10 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging, bool more_follow) {
       tc_launch_forward(c, l, dr, act_mask);
       LAUNCH_CHECK(c);
     }
+  }
+  if (c->record_after_forward != nullptr) {             // the next worker group starts once this one's forward pass is enqueued
+    cudaEventRecord(c->record_after_forward, c->stream);
+    c->record_after_forward = nullptr;
   }
   const bool epi = tc_epilogues_fused(c);
   if (!epi) {
@@ -498,6 +504,12 @@ int prsgd_destroy(prsgd_ctx* ctx) {
   if (ctx->readout_event) cudaEventDestroy(ctx->readout_event);
   if (ctx->staged_event) cudaEventDestroy(ctx->staged_event);
   if (ctx->free_event) cudaEventDestroy(ctx->free_event);
+  if (ctx->group_fork) cudaEventDestroy(ctx->group_fork);
+  for (int g = 0; g < kMaxGroups; ++g) {
+    if (ctx->group_join[g]) cudaEventDestroy(ctx->group_join[g]);
+    if (ctx->group_stagger[g]) cudaEventDestroy(ctx->group_stagger[g]);
+    if (ctx->group_stream[g]) cudaStreamDestroy(ctx->group_stream[g]);
+  }
   delete ctx;
   return PRSGD_OK;
 }
@@ -614,10 +626,10 @@ int prsgd_get_params(prsgd_ctx* c, float* dst, int32_t worker, int dst_on_device
 namespace {
 
 // iterations t_first .. t_first + count - 1, launched directly
-int run_iterations(prsgd_ctx* c, int64_t t_first, int64_t count) {
+int run_iterations_on_stream(prsgd_ctx* c, int64_t t_first, int64_t count, int64_t t_call_end) {
   for (int64_t t = t_first; t < t_first + count; ++t) {
     const bool averaging = c->I > 0 && (t % c->I) == 0;
-    const bool more_follow = t + 1 < t_first + count;
+    const bool more_follow = t + 1 < t_call_end;
     int rc = c->precision == PRSGD_PRECISION_BF16 ? step_bf16(c, t, averaging, more_follow) : step_f32(c, t, averaging);
     // (the fp32 path has no fused form for the momentum step)
     const bool separate_average = !c->fused_average || (c->velocity != nullptr && c->precision == PRSGD_PRECISION_FP32);
@@ -633,6 +645,65 @@ int run_iterations(prsgd_ctx* c, int64_t t_first, int64_t count) {
   return PRSGD_OK;
 }
 
+// Worker groups: inside an epoch the workers need no synchronisation (the text after Algorithm 1), so a run of
+// plain iterations can be enqueued as G independent chains of launches, one per group of workers, each on a
+// stream of its own; the launches of a chain skip the other groups' workers (the per-worker flags of Algorithm
+// 3's mask).  While one group's long update kernels run, another group's short, latency-bound launches find
+// free SMs.  The chains fork from the context's stream and join it again before the next averaging iteration.
+int ensure_group_resources(prsgd_ctx* c) {
+  for (int g = 0; g < c->worker_groups; ++g) {
+    if (!c->group_stream[g]) CUDA_TRY(c, cudaStreamCreateWithFlags(&c->group_stream[g], cudaStreamNonBlocking));
+    if (!c->group_join[g]) CUDA_TRY(c, cudaEventCreateWithFlags(&c->group_join[g], cudaEventDisableTiming));
+    if (!c->group_stagger[g]) CUDA_TRY(c, cudaEventCreateWithFlags(&c->group_stagger[g], cudaEventDisableTiming));
+  }
+  if (!c->group_fork) CUDA_TRY(c, cudaEventCreateWithFlags(&c->group_fork, cudaEventDisableTiming));
+  return PRSGD_OK;
+}
+
+int run_iterations(prsgd_ctx* c, int64_t t_first, int64_t count) {
+  const int64_t t_end = t_first + count;
+  int64_t t = t_first;
+  while (t < t_end) {
+    // the run of plain iterations that starts here
+    int64_t plain = 0;
+    while (t + plain < t_end && !(c->I > 0 && ((t + plain) % c->I) == 0)) ++plain;
+    const bool grouped = c->worker_groups > 1 && c->precision == PRSGD_PRECISION_BF16 && !c->has_mask && !c->profile &&
+                         plain >= 2 && c->N >= 2 * c->worker_groups;
+    if (!grouped) {
+      const int64_t n = plain > 0 ? plain : 1;           // the plain run, or the averaging iteration it ends at
+      int rc = run_iterations_on_stream(c, t, n, t_end);
+      if (rc != PRSGD_OK) return rc;
+      t += n;
+      continue;
+    }
+    int rc = ensure_group_resources(c);
+    if (rc != PRSGD_OK) return rc;
+    cudaStream_t main_stream = c->stream;
+    const bool a1_0 = c->a1_ready, ident_0 = c->rows_identical, quiet_0 = c->upper_weights_quiet;
+    CUDA_TRY(c, cudaEventRecord(c->group_fork, main_stream));
+    for (int g = 0; g < c->worker_groups && rc == PRSGD_OK; ++g) {
+      cudaStream_t gs = c->group_stream[g];
+      CUDA_TRY(c, cudaStreamWaitEvent(gs, c->group_fork, 0));
+      if (g > 0) CUDA_TRY(c, cudaStreamWaitEvent(gs, c->group_stagger[g - 1], 0));   // half a step behind the group before
+      c->stream = gs;
+      c->group_active = c->group_masks + (size_t)g * c->N;
+      c->a1_ready = a1_0; c->rows_identical = ident_0; c->upper_weights_quiet = quiet_0;
+      c->record_after_forward = g + 1 < c->worker_groups ? c->group_stagger[g] : nullptr;
+      rc = run_iterations_on_stream(c, t, plain, t_end);
+      c->stream = main_stream;
+      c->group_active = nullptr;
+      c->record_after_forward = nullptr;
+      if (rc == PRSGD_OK) {
+        CUDA_TRY(c, cudaEventRecord(c->group_join[g], gs));
+        CUDA_TRY(c, cudaStreamWaitEvent(main_stream, c->group_join[g], 0));
+      }
+    }
+    if (rc != PRSGD_OK) return rc;
+    t += plain;
+  }
+  return PRSGD_OK;
+}
+
 void period_key(const prsgd_ctx* c, uint64_t (&key)[13]) {
   uint32_t gbits, mbits;
   std::memcpy(&gbits, &c->gamma, 4);
@@ -641,7 +712,8 @@ void period_key(const prsgd_ctx* c, uint64_t (&key)[13]) {
   key[4] = c->has_mask ? 1 : 0; key[5] = reinterpret_cast<uint64_t>(c->velocity); key[6] = mbits;
   key[7] = (uint64_t)c->average_velocity; key[8] = reinterpret_cast<uint64_t>(c->X);
   key[9] = reinterpret_cast<uint64_t>(c->Y); key[10] = (uint64_t)c->worker0; key[11] = (uint64_t)c->fused_epilogues | ((uint64_t)c->early_loads << 1) | ((uint64_t)c->next_forward << 2) | ((uint64_t)c->dx_in_update << 3);
-  key[12] = (c->rows_identical ? 1u : 0u) | ((uint64_t)c->shared_restart << 1) | ((uint64_t)c->forward_chain << 2);   // the period's first iteration may share reads
+  key[12] = (c->rows_identical ? 1u : 0u) | ((uint64_t)c->shared_restart << 1) | ((uint64_t)c->forward_chain << 2) |
+            ((uint64_t)c->worker_groups << 3);   // the period's first iteration may share reads
 }
 
 // One whole averaging period (I iterations starting right after an average) as a CUDA graph: the
@@ -1000,6 +1072,16 @@ int prsgd_set_option(prsgd_ctx* c, int32_t option, int64_t value) {
   if (option == PRSGD_OPT_CHECK_FINITE) { c->check_finite = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_SHARED_RESTART) { c->shared_restart = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_FORWARD_CHAIN) { c->forward_chain = value != 0; return PRSGD_OK; }
+  if (option == PRSGD_OPT_WORKER_GROUPS) {
+    if (value < 1 || value > kMaxGroups) return fail(c, PRSGD_ERR_ARG, "PRSGD_OPT_WORKER_GROUPS takes 1..4");
+    // group g holds the contiguous workers [g N / G, (g + 1) N / G)
+    std::vector<uint8_t> m((size_t)kMaxGroups * c->N, 0);
+    for (int i = 0; i < c->N; ++i) m[(size_t)((int64_t)i * value / c->N) * c->N + i] = 1;
+    CUDA_TRY(c, cudaMemcpyAsync(c->group_masks, m.data(), m.size(), cudaMemcpyHostToDevice, c->stream));
+    CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+    c->worker_groups = (int)value;
+    return PRSGD_OK;
+  }
   if (option == PRSGD_OPT_DX_IN_UPDATE) {
     if (value < 0 || value > 2) return fail(c, PRSGD_ERR_ARG, "PRSGD_OPT_DX_IN_UPDATE takes 0, 1 or 2");
     c->dx_in_update = (int)value;

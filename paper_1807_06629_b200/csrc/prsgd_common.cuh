@@ -56,6 +56,7 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
+constexpr int kMaxGroups = 4;
 constexpr int64_t kSegAlign = 32;  // every segment of a row starts at a multiple of 32 elements
 
 inline int64_t round_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
@@ -102,6 +103,15 @@ struct prsgd_ctx {
   int fused_epilogues = 1;       // softmax-CE gradient and bias steps inside the GEMM epilogues (tensor-core path)
   int shared_restart = 1;        // the iteration after a node average reads worker 0's weights for every worker
   int forward_chain = 0;         // the forward GEMMs of consecutive layers run as one launch (tensor-core path)
+  // Worker groups (PRSGD_OPT_WORKER_GROUPS): the plain iterations of a period run as G independent launch chains,
+  // one per contiguous group of workers, on G streams of the library's own
+  int worker_groups = 1;
+  uint8_t* group_masks = nullptr;        // [kMaxGroups][N] device: 1 where the worker belongs to the group
+  const uint8_t* group_active = nullptr; // mask of the group whose launches are being enqueued (nullptr: none)
+  cudaStream_t group_stream[4] = {nullptr, nullptr, nullptr, nullptr};
+  cudaEvent_t group_fork = nullptr, group_join[4] = {nullptr, nullptr, nullptr, nullptr};
+  cudaEvent_t group_stagger[4] = {nullptr, nullptr, nullptr, nullptr};
+  cudaEvent_t record_after_forward = nullptr;   // recorded once after the next forward pass (staggers the groups)
   bool upper_weights_quiet = false;      // the launch enqueued last does not write the weights of any layer >= 2
   unsigned int* chain_ready = nullptr;   // [8][N] row-tile counters of the forward chain + one word, zero between launches
   bool rows_identical = false;   // every row of the store (and of the bf16 copy) holds the same bits right now

@@ -348,6 +348,42 @@ def test_forward_chain_in_one_launch_changes_no_bit(torch_cuda):
             assert outs[1][3] < outs[0][3]
 
 
+def test_worker_groups_on_their_own_streams_change_no_bit(torch_cuda):
+    """The plain iterations of a period as 2, 3 or 4 independent launch chains (one per group of workers, each on
+    a stream of the library's own, forked from and joined to the context's stream) against one chain for all
+    workers: identical parameters, losses, draws and momentum buffers over several periods, direct and replayed,
+    with calls that end in the middle of a period and group sizes that do not divide N."""
+    torch = torch_cuda
+    from paper_1807_06629_b200 import binding
+    cases = (_w("tc-groups-n8", 8, (128, 256, 10), 32, I=4), _w("tc-groups-n7", 7, (192, 128, 256, 10), 32, I=5),
+             _w("tc-groups-wide", 9, (64, 448, 320, 10), 16, I=3), _w("tc-groups-b64", 8, (128, 128, 100), 64, I=4))
+    for w in cases:
+        X, Y, x0 = make_inputs(w)
+        for mu in (None, 0.9):
+            outs = []
+            for groups, graph in ((1, 0), (2, 0), (2, 1), (3, 1), (4, 0)):
+                with torch.cuda.stream(torch.cuda.Stream()):
+                    p = make_ctx(w, X, Y, x0)
+                    p.set_option(binding.OPT_WORKER_GROUPS, groups)
+                    p.set_option(binding.OPT_GRAPH, graph)
+                    if mu is not None:
+                        p.enable_momentum(mu)
+                    p.local_steps(2)                       # ends inside a period
+                    p.local_steps(3 * w.I + 2)             # crosses three averages, ends inside a period again
+                    p.local_steps(w.I - 1)
+                    outs.append((p.get_params_stacked(), p.get_losses(), p.get_draws().tolist(), p.get_step(),
+                                 p.get_velocity_stacked() if mu is not None else None))
+                    torch.cuda.current_stream().synchronize()
+                    p.close()
+            for o in outs[1:]:
+                assert np.array_equal(outs[0][0], o[0]), (w.name, mu)
+                assert np.array_equal(outs[0][1], o[1]) and outs[0][2] == o[2] and outs[0][3] == o[3]
+                if mu is not None:
+                    assert np.array_equal(outs[0][4], o[4])
+    with pytest.raises(binding.PRSGDError):
+        make_ctx(cases[0], *make_inputs(cases[0])).set_option(binding.OPT_WORKER_GROUPS, 5)
+
+
 def test_reading_the_common_restart_point_once_changes_no_bit(torch_cuda):
     """After a node average all N rows hold the same bits, so the following iteration's forward, dX and fused
     update + average launches read worker 0's weights for every worker (PRSGD_OPT_SHARED_RESTART).  Against
