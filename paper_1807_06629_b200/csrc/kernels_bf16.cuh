@@ -1157,15 +1157,19 @@ template <int TN, bool MOM> struct UpdNextCfg {
   static constexpr uint32_t kMaster = 128u * TN * 4u;
   static constexpr uint32_t kVel = MOM ? kMaster : 0u;          // momentum tile right after the master tile
   static constexpr uint32_t kOut = 128u * TN * 2u;
-  __host__ __device__ static uint32_t ops_bytes(int B) { return (uint32_t)(2 + TN / 64) * (uint32_t)B * 128u; }
+  // per stage: the minibatch boxes of the tile's columns (later the bf16 output tile), then the next minibatch's
+  __host__ __device__ static uint32_t ops_bytes(int B) { return (uint32_t)(TN / 64) * (uint32_t)B * 128u; }
   __host__ __device__ static uint32_t region(int B) { return ops_bytes(B) > kOut ? ops_bytes(B) : kOut; }
   __host__ __device__ static uint32_t next_bytes(int B) { return (uint32_t)(TN / 64) * (uint32_t)B * 128u; }
   __host__ __device__ static uint32_t stage(int B) { return kMaster + kVel + region(B) + next_bytes(B); }
+  // behind the stages: the two dZ boxes of a row block, which every column tile of the block uses, loaded once
+  // per block (two buffers, so that the next block's boxes arrive while this block's last tiles are multiplied)
+  __host__ __device__ static uint32_t dz_bytes(int B) { return 4u * (uint32_t)B * 128u; }
   static int stages(int B) {
-    int s = (int)((227u * 1024u - 2048u) / stage(B));
+    int s = (int)((227u * 1024u - 2048u - dz_bytes(B)) / stage(B));
     return s > 4 ? 4 : s;
   }
-  static size_t smem(int B) { return (size_t)stages(B) * stage(B) + 1024 + 512; }
+  static size_t smem(int B) { return (size_t)stages(B) * stage(B) + dz_bytes(B) + 1024 + 512; }
 };
 
 template <int TN, bool MOM>
@@ -1189,7 +1193,8 @@ __global__ void __launch_bounds__(kUpdBlkThreads, 1) tc_update_next_kernel(const
   auto vel_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes + Cfg::kMaster; };
   auto ops_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes + Cfg::kMaster + Cfg::kVel; };
   auto next_u32 = [&](int s) { return base + (uint32_t)s * stage_bytes + Cfg::kMaster + Cfg::kVel + Cfg::region(a.B); };
-  const uint32_t bar0 = base + (uint32_t)S * stage_bytes;
+  auto dz_u32 = [&](int q) { return base + (uint32_t)S * stage_bytes + (uint32_t)q * 2u * op_box; };
+  const uint32_t bar0 = base + (uint32_t)S * stage_bytes + Cfg::dz_bytes(a.B);
   auto full_ops = [&](int s) { return bar0 + 8u * s; };
   auto full_w = [&](int s) { return bar0 + 32u + 8u * s; };
   auto stage_empty = [&](int s) { return bar0 + 64u + 8u * s; };
@@ -1199,8 +1204,10 @@ __global__ void __launch_bounds__(kUpdBlkThreads, 1) tc_update_next_kernel(const
   auto fwd_done = [&](int s) { return bar0 + 192u + 8u * s; };      // forward MMAs have read the stage's bf16 tile
   auto facc_full = [&](int q) { return bar0 + 224u + 8u * q; };
   auto facc_empty = [&](int q) { return bar0 + 240u + 8u * q; };
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen + (size_t)S * stage_bytes + 256);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + (size_t)S * stage_bytes + 260);
+  auto dz_full = [&](int q) { return bar0 + 272u + 8u * q; };       // the row block's dZ boxes have arrived
+  auto dz_empty = [&](int q) { return bar0 + 288u + 8u * q; };      // every dW product of the block has read them
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen + (bar0 - base) + 256);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + (bar0 - base) + 260);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int row_blocks = a.tiles_m * a.N;
@@ -1211,7 +1218,10 @@ __global__ void __launch_bounds__(kUpdBlkThreads, 1) tc_update_next_kernel(const
       mbar_init(acc_full(s), 1); mbar_init(acc_empty(s), 128); mbar_init(tile_ready(s), 128);
       mbar_init(fwd_done(s), 1);
     }
-    for (int q = 0; q < 2; ++q) { mbar_init(facc_full(q), 1); mbar_init(facc_empty(q), 128); }
+    for (int q = 0; q < 2; ++q) {
+      mbar_init(facc_full(q), 1); mbar_init(facc_empty(q), 128);
+      mbar_init(dz_full(q), 1); mbar_init(dz_empty(q), 1);
+    }
     *abort_flag = *(volatile unsigned int*)&a.status->error != 0u ? 1 : 0;   // an earlier expired wait: no-op (see tc_stream_kernel)
     fence_mbar_init();
     prefetch_tensormap(&mapDelta); prefetch_tensormap(&mapPool);
@@ -1232,7 +1242,7 @@ __global__ void __launch_bounds__(kUpdBlkThreads, 1) tc_update_next_kernel(const
   // row block the column tiles kb = 0 .. tiles_n - 1; `it` counts tiles, tile `it` lives in stage it % S.
   if (warp == 0 && lane == 0) {
     // ---------------- loader
-    uint32_t it = 0;
+    uint32_t it = 0, rbi = 0;
     bool ok = true;
     for (int rb = blockIdx.x; rb < total_rb && ok; rb += gridDim.x) {
       const int n = rb / a.tiles_m, m0 = (rb % a.tiles_m) * 128;
@@ -1240,6 +1250,15 @@ __global__ void __launch_bounds__(kUpdBlkThreads, 1) tc_update_next_kernel(const
       const int64_t t = draw_t(a.draw);
       const int row0 = (int)draw_block(a.draw.seed, a.draw.worker0 + n, t, a.draw.n_blocks) * a.B;
       const int row1 = (int)draw_block(a.draw.seed, a.draw.worker0 + n, t + 1, a.draw.n_blocks) * a.B;
+      {   // the block's two dZ boxes, once for all its column tiles
+        const int q = rbi & 1;
+        ok = mbar_wait(dz_empty(q), ((rbi >> 1) & 1u) ^ 1u, abort_flag, a.status, 0x40B);
+        if (!ok) break;
+        mbar_expect_tx(dz_full(q), 2u * op_box);
+        tma_load_3d(dz_u32(q), &mapDelta, dz_full(q), m0, 0, n);
+        tma_load_3d(dz_u32(q) + op_box, &mapDelta, dz_full(q), m0 + 64, 0, n);
+        ++rbi;
+      }
       for (int kb = 0; kb < a.tiles_n; ++kb, ++it) {
         const int s = it % S;
         const uint32_t ph = (it / S) & 1u;
@@ -1247,12 +1266,10 @@ __global__ void __launch_bounds__(kUpdBlkThreads, 1) tc_update_next_kernel(const
         if (!ok) break;
         const int n0 = kb * TN;
         const uint32_t ops = ops_u32(s), nx = next_u32(s);
-        mbar_expect_tx(full_ops(s), (2u + 2u * NB64) * op_box);
-        tma_load_3d(ops, &mapDelta, full_ops(s), m0, 0, n);
-        tma_load_3d(ops + op_box, &mapDelta, full_ops(s), m0 + 64, 0, n);
+        mbar_expect_tx(full_ops(s), 2u * NB64 * op_box);
 #pragma unroll
         for (int h = 0; h < NB64; ++h) {
-          tma_load_3d(ops + (2u + h) * op_box, &mapPool, full_ops(s), n0 + 64 * h, row0, n);
+          tma_load_3d(ops + h * op_box, &mapPool, full_ops(s), n0 + 64 * h, row0, n);
           tma_load_3d(nx + h * op_box, &mapPool, full_ops(s), n0 + 64 * h, row1, n);
         }
         mbar_expect_tx(full_w(s), Cfg::kMaster + Cfg::kVel);
@@ -1271,6 +1288,10 @@ __global__ void __launch_bounds__(kUpdBlkThreads, 1) tc_update_next_kernel(const
         while (!(mbar_try_wait(full_w(q % S), (q / S) & 1u) && mbar_try_wait(full_ops(q % S), (q / S) & 1u)) &&
                globaltimer_ns() - t0 < 100000000ull) {}
       }
+    }
+    if (*abort_flag && rbi > 0) {
+      const uint64_t t0 = globaltimer_ns();
+      while (!mbar_try_wait(dz_full((rbi - 1) & 1), ((rbi - 1) >> 1) & 1u) && globaltimer_ns() - t0 < 100000000ull) {}
     }
   } else if (warp == 1 && lane == 0) {
     // ---------------- MMA issuer: dW of tile `it`, then the forward product of tile it - 1 (whose
@@ -1305,15 +1326,21 @@ __global__ void __launch_bounds__(kUpdBlkThreads, 1) tc_update_next_kernel(const
       for (int kb = 0; kb < a.tiles_n && ok; ++kb, ++it) {
         const int s = it % S;
         const uint32_t ph = (it / S) & 1u;
+        const int dq = rbi & 1;
+        if (kb == 0) {
+          ok = mbar_wait(dz_full(dq), (rbi >> 1) & 1u, abort_flag, a.status, 0x40C);
+          if (!ok) break;
+        }
         ok = mbar_wait(acc_empty(s), ph ^ 1u, abort_flag, a.status, 0x404) &&
              mbar_wait(full_ops(s), ph, abort_flag, a.status, 0x405);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t sa = ops_u32(s), sb = sa + 2u * op_box;
+        const uint32_t sa = dz_u32(dq), sb = ops_u32(s);
         for (int k = 0; k < ksteps; ++k)
           mma_bf16(tmem + (uint32_t)(s * TN), smem_desc_sw128(sa + k * 2048u, op_box, 1024u),
                    smem_desc_sw128(sb + k * 2048u, op_box, 1024u), idesc_dw, k != 0 ? 1u : 0u);
         mma_commit(acc_full(s));
+        if (kb == a.tiles_n - 1) mma_commit(dz_empty(dq));      // the block's dZ boxes are free once these products are done
         if (have_prev) ok = forward_of(p_it, p_kb, p_rbi);
         p_it = it; p_kb = kb; p_rbi = rbi; have_prev = true;
       }
@@ -2193,7 +2220,7 @@ inline void tc_launch_update_next(prsgd_ctx* c, const DrawArgs& dr) {
     const int64_t tiles128 = (int64_t)((ly.d_out + 127) / 128) * ((ly.d_in + 127) / 128);
     tile = (c->B <= 32 && tiles128 * c->N >= 32 * (int64_t)st->num_sms) ? 128 : 64;
   }
-  if (tile == 128) tc_launch_update_next_tn<128, false>(c, dr);
+  if (tile == 128 && UpdNextCfg<128, false>::stages(c->B) >= 2) tc_launch_update_next_tn<128, false>(c, dr);
   else tc_launch_update_next_tn<64, false>(c, dr);
 }
 
