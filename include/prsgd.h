@@ -225,12 +225,20 @@ int prsgd_run_heterogeneous_epoch(prsgd_ctx* ctx, const int32_t* h_I_i);
  *    padded columns j in [col0, col0 + ncols); d_dst is a device row of m_pad floats.
  *  - prsgd_assign_rows: every local row (and the bf16 shadow) gets d_src[j] / divisor on the same
  *    column range; with divisor = the global N this is the restart at the node average.
+ *  - prsgd_local_steps_sum: iterations t+1 .. t+k like prsgd_local_steps (needs I = 0), except that the
+ *    k-th one runs in the fused update + average form with the division left out: afterwards EVERY local
+ *    row holds sum_i x_i^{t+k} over the local rows (what prsgd_partial_sum would have computed from the
+ *    updated rows, without that extra pass over the store).  Row 0 of the store (m_pad floats at d_params) is
+ *    then the buffer to all-reduce, and prsgd_assign_rows(d_params, N_global, ...) completes the average; until
+ *    it has covered the whole row the store holds sums, not models.  Same bits as prsgd_local_steps(k) +
+ *    prsgd_partial_sum + prsgd_assign_rows.  Not with averaged momentum buffers.
  * col0 and ncols are multiples of 4 (column ranges let the caller pipeline the all-reduce chunk by
  * chunk); rows are 16-byte aligned device pointers.  With a single context,
  * partial_sum + assign_rows(divisor = N) leaves the same bits as prsgd_average.  Asynchronous. */
 int prsgd_set_worker_offset(prsgd_ctx* ctx, int32_t first_worker);
 int prsgd_set_global_workers(prsgd_ctx* ctx, int32_t N_global);
 int prsgd_partial_sum(prsgd_ctx* ctx, float* d_dst, int64_t col0, int64_t ncols);
+int prsgd_local_steps_sum(prsgd_ctx* ctx, int64_t k);
 int prsgd_assign_rows(prsgd_ctx* ctx, const float* d_src, float divisor, int64_t col0, int64_t ncols);
 
 /* Local step with momentum, as in the paper's experiment (Experiment section, figure captions:

@@ -46,7 +46,7 @@ EXPORTS = [
     "prsgd_clear_device_error", "prsgd_enable_momentum", "prsgd_get_velocity_stacked",
     "prsgd_set_worker_offset", "prsgd_partial_sum", "prsgd_assign_rows", "prsgd_stage_data", "prsgd_swap_data",
     "prsgd_alg2_schedule", "prsgd_run_time_varying", "prsgd_run_heterogeneous_epoch",
-    "prsgd_set_global_workers", "prsgd_check_finite",
+    "prsgd_set_global_workers", "prsgd_check_finite", "prsgd_local_steps_sum",
 ]
 NOALLOC_MAX_M = 1 << 20
 
@@ -81,6 +81,7 @@ def _load() -> C.CDLL:
         "prsgd_get_params_stacked": (C.c_int, [vp, vp, C.c_int]),
         "prsgd_get_params": (C.c_int, [vp, vp, i32, C.c_int]),
         "prsgd_local_steps": (C.c_int, [vp, i64]),
+        "prsgd_local_steps_sum": (C.c_int, [vp, i64]),
         "prsgd_average": (C.c_int, [vp]),
         "prsgd_get_average": (C.c_int, [vp, vp, C.c_int]),
         "prsgd_get_average_async": (C.c_int, [vp, vp, vp]),
@@ -288,6 +289,14 @@ class PRSGD:
     # ---- Algorithm 1 ------------------------------------------------------------
     def local_steps(self, k: int):
         self._call(lib.prsgd_local_steps, k)
+
+    def local_steps_sum(self, k: int):
+        """k iterations, the last one leaving the SUM of the updated local rows in every row (see prsgd.h)."""
+        self._call(lib.prsgd_local_steps_sum, k)
+
+    def row0(self) -> torch.Tensor:
+        """Row 0 of the store as a tensor of m_pad floats (the all-reduce buffer after local_steps_sum)."""
+        return self.params[:self.m_pad]
 
     def average(self):
         self._call(lib.prsgd_average)

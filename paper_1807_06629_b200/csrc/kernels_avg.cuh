@@ -43,7 +43,7 @@ template <int MODE, bool SHADOW, int V = 4>
 __global__ void __launch_bounds__(256) average_rows_kernel(float* __restrict__ P, int64_t N, int64_t m,
                                                            int64_t row_stride, float* __restrict__ out,
                                                            uint16_t* __restrict__ shadow,
-                                                           const DeviceStatus* status = nullptr) {
+                                                           const DeviceStatus* status = nullptr, float divisor = 0.f) {
   using Vec = typename LaneVec<V>::type;
   constexpr int U = 8;
   asm volatile("griddepcontrol.wait;" ::: "memory");   // no-op unless launched as a programmatic dependent
@@ -51,7 +51,7 @@ __global__ void __launch_bounds__(256) average_rows_kernel(float* __restrict__ P
   if (status != nullptr && status->error != 0u) return;   // a recorded expired wait: leave the store alone
   const int64_t colsV = m / V;
   const int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  const float fN = (float)N;
+  const float fN = divisor > 0.f ? divisor : (float)N;      // (divisor 1: every row receives the row SUM)
   if (c < colsV) {
     Vec* base = reinterpret_cast<Vec*>(P) + c;
     const int64_t sV = row_stride / V;

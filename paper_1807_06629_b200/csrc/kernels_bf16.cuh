@@ -703,6 +703,8 @@ struct UpdateArgs {
   const uint8_t* active;
   DeviceStatus* status;
   int prefetch;            // 1: master tiles may be requested before the previous launch has completed
+  float divisor;           // fused form: the summed models are divided by this (N; 1 leaves the local row SUM in every
+                           // row, the first half of an average whose other rows live on other GPUs)
   int avg_vel;             // fused form with momentum, 1: the momentum buffers are averaged like the models
   int shared_w;            // fused form only, 1: every worker's master tile holds the same bits (the launch follows a
                            // node average with nothing in between): all N loads of a tile read worker 0's copy, which
@@ -982,6 +984,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
     const uint32_t sw = (uint32_t)(r & 7);
     const int etid = tid - 96;                            // 0..127 among the epilogue threads
     const float fN = (float)a.N;
+    const float fD = a.divisor;
     constexpr int NSUM = FUSE ? TN : 1;
     constexpr int NVSUM = (FUSE && MOM) ? TN : 1;
     constexpr int NXR = kShareOnce ? TN : 1;
@@ -1072,8 +1075,8 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
               float* sp = &sum[F * (c * 32 + 4 * j)];
               sp[0] += x.x; sp[F * 1] += x.y; sp[F * 2] += x.z; sp[F * 3] += x.w;
               if (last) {
-                x.x = __fdiv_rn(sp[0], fN); x.y = __fdiv_rn(sp[F * 1], fN);
-                x.z = __fdiv_rn(sp[F * 2], fN); x.w = __fdiv_rn(sp[F * 3], fN);
+                x.x = __fdiv_rn(sp[0], fD); x.y = __fdiv_rn(sp[F * 1], fD);
+                x.z = __fdiv_rn(sp[F * 2], fD); x.w = __fdiv_rn(sp[F * 3], fD);
               }
             }
             if (!FUSE || last) {
@@ -1884,6 +1887,7 @@ struct BiasAverageArgs {
   int64_t b_off[PRSGD_MAX_LAYERS];
   int d_out[PRSGD_MAX_LAYERS];
   const DeviceStatus* status;
+  float divisor;             // N, or 1 to leave the row sum
 };
 
 __global__ void __launch_bounds__(128) bias_average_kernel(const BiasAverageArgs a) {
@@ -1903,7 +1907,7 @@ __global__ void __launch_bounds__(128) bias_average_kernel(const BiasAverageArgs
     for (int u = 0; u < 8; ++u) s += v[u];
   }
   for (; i < a.N; ++i) s += p[(int64_t)i * a.m_pad];
-  const float y = __fdiv_rn(s, (float)a.N);
+  const float y = __fdiv_rn(s, a.divisor);
   for (int r = 0; r < a.N; ++r) p[(int64_t)r * a.m_pad] = y;
 }
 
@@ -2128,6 +2132,7 @@ inline void tc_launch_update_tn(prsgd_ctx* c, int l, const DrawArgs& dr, const u
   a.prefetch = (active == nullptr && c->early_loads) ? 1 : 0;
   a.shared_w = (fuse && tc_shared_restart(c, active)) ? 1 : 0;
   a.avg_vel = c->average_velocity ? 1 : 0;
+  a.divisor = c->avg_divisor > 0.f ? c->avg_divisor : (float)c->N;
   const int items = a.tiles_m * a.tiles_n * (fuse ? 1 : c->N);
   const int grid = items < st->num_sms ? items : st->num_sms;
   const TcLayerMaps& mp = st->layer[l - 1];
@@ -2275,7 +2280,7 @@ inline void tc_launch_weight_average(prsgd_ctx* c, int l) {
   const int64_t cols = (int64_t)ly.d_out * ly.d_in;          // a multiple of 64, like every input width of this path
   launch_pdl(average_rows_kernel<0, true, 2>, dim3((unsigned)((cols / 2 + (cols & 1) + 255) / 256)), dim3(256), 0, c->stream,
              c->params + ly.w_off, (int64_t)c->N, cols, c->m_pad, (float*)nullptr, c->shadow + ly.w_off,
-             (const DeviceStatus*)c->status);
+             (const DeviceStatus*)c->status, c->avg_divisor);
 }
 
 // the same segment of the momentum buffers, when they are averaged with the models
@@ -2284,12 +2289,13 @@ inline void tc_launch_velocity_segment_average(prsgd_ctx* c, int l) {
   const int64_t cols = (int64_t)ly.d_out * ly.d_in;
   launch_pdl(average_rows_kernel<0, false, 2>, dim3((unsigned)((cols / 2 + (cols & 1) + 255) / 256)), dim3(256), 0, c->stream,
              c->velocity + ly.w_off, (int64_t)c->N, cols, c->m_pad, (float*)nullptr, (uint16_t*)nullptr,
-             (const DeviceStatus*)c->status);
+             (const DeviceStatus*)c->status, 0.f);
 }
 
 inline void tc_launch_bias_average(prsgd_ctx* c, float* store) {
   BiasAverageArgs a{};
   a.params = store; a.m_pad = c->m_pad; a.N = c->N; a.status = c->status;
+  a.divisor = (store == c->params && c->avg_divisor > 0.f) ? c->avg_divisor : (float)c->N;
   int dmax = 1;
   for (int l = 1; l <= c->L; ++l) {
     a.b_off[l - 1] = c->layer[l - 1].b_off; a.d_out[l - 1] = c->layer[l - 1].d_out;

@@ -803,6 +803,42 @@ int prsgd_average(prsgd_ctx* c) {
   return launch_average(c);
 }
 
+int prsgd_local_steps_sum(prsgd_ctx* c, int64_t k) {
+  if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
+  if (k < 1) return fail(c, PRSGD_ERR_ARG, "k must be >= 1");
+  if (c->I != 0) return fail(c, PRSGD_ERR_STATE, "prsgd_local_steps_sum needs I = 0: the caller drives the averages");
+  if (!c->X || !c->Y) return fail(c, PRSGD_ERR_STATE, "bind_data must come before local steps");
+  if (c->velocity != nullptr && c->average_velocity)
+    return fail(c, PRSGD_ERR_STATE, "averaged momentum buffers have no row-sum form");
+  const int64_t t_end = c->t + k + 1;                  // (exclusive) so that iteration t + k - 1 knows another one follows
+  int rc = k > 1 ? run_iterations_on_stream(c, c->t + 1, k - 1, t_end) : PRSGD_OK;
+  if (rc != PRSGD_OK) return rc;
+  // iteration t + k: the local step in its fused form, with the summed rows divided by 1 instead of N
+  c->avg_divisor = 1.f;
+  const int fused_keep = c->fused_average;
+  if (c->precision == PRSGD_PRECISION_BF16) {
+    c->fused_average = 1;
+    rc = step_bf16(c, c->t + k, /*averaging=*/true, /*more_follow=*/false);
+  } else {
+    rc = step_f32(c, c->t + k, /*averaging=*/false);   // plain step, then every row <- sum of the rows
+    if (rc == PRSGD_OK) {
+      const int64_t threads = c->m_pad / 4;
+      prof_begin(c, PRSGD_KERNEL_AVERAGE);
+      average_rows_kernel<0, false><<<grid1d(threads, 256), 256, 0, c->stream>>>(c->params, c->N, c->m_pad, c->m_pad, nullptr,
+                                                                               nullptr, c->status, 1.f);
+      LAUNCH_CHECK(c);
+    }
+  }
+  c->fused_average = fused_keep;
+  c->avg_divisor = 0.f;
+  c->a1_ready = false;
+  c->rows_identical = rc == PRSGD_OK;                  // every row holds the same bits: the row sum
+  c->assigned_upto = -1;
+  if (rc != PRSGD_OK) return rc;
+  c->t += k;
+  return PRSGD_OK;
+}
+
 int prsgd_get_average_async(prsgd_ctx* c, float* h_dst, void* copy_stream) {
   if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
   if (!h_dst) return fail(c, PRSGD_ERR_ARG, "h_dst is NULL");
@@ -1189,12 +1225,12 @@ int prsgd_average_rows(float* d_P, int64_t N, int64_t m, int64_t row_stride, voi
   if (m < kAvgNarrowLaneBelow) {
     const int64_t threads = m / 2 + (m & 1);
     launch_pdl(average_rows_kernel<0, false, 2>, grid1d(threads, 256), dim3(256), 0, st, d_P, N, m, row_stride,
-               (float*)nullptr, (uint16_t*)nullptr, (const DeviceStatus*)nullptr);
+               (float*)nullptr, (uint16_t*)nullptr, (const DeviceStatus*)nullptr, 0.f);
   } else {
     const int64_t threads = m / 4 + (m & 3);
     if ((threads + 255) / 256 > 0x7fffffffll) return fail(nullptr, PRSGD_ERR_SIZE, "m too large");
     launch_pdl(average_rows_kernel<0, false>, grid1d(threads, 256), dim3(256), 0, st, d_P, N, m, row_stride,
-               (float*)nullptr, (uint16_t*)nullptr, (const DeviceStatus*)nullptr);
+               (float*)nullptr, (uint16_t*)nullptr, (const DeviceStatus*)nullptr, 0.f);
   }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return fail(nullptr, PRSGD_ERR_CUDA, std::string("average_rows: ") + cudaGetErrorString(e));

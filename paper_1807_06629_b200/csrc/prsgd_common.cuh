@@ -112,6 +112,7 @@ struct prsgd_ctx {
   cudaEvent_t group_fork = nullptr, group_join[4] = {nullptr, nullptr, nullptr, nullptr};
   cudaEvent_t group_stagger[4] = {nullptr, nullptr, nullptr, nullptr};
   cudaEvent_t record_after_forward = nullptr;   // recorded once after the next forward pass (staggers the groups)
+  float avg_divisor = 0.f;               // > 0: an averaging iteration divides the summed rows by this instead of N
   bool upper_weights_quiet = false;      // the launch enqueued last does not write the weights of any layer >= 2
   unsigned int* chain_ready = nullptr;   // [8][N] row-tile counters of the forward chain + one word, zero between launches
   bool rows_identical = false;   // every row of the store (and of the bf16 copy) holds the same bits right now

@@ -15,6 +15,8 @@ Two partitions of a job over G ranks are provided by `partition`:
 This module only orchestrates: the local work is done by an *engine* object with
     local_steps(k), get_step(), m_pad, new_row(), set_lr(gamma),
     partial_sum(row, col0, ncols), assign_rows(row, divisor, col0, ncols)
+and optionally local_steps_sum(k) + row0() (the last local step of a period leaves the local row sums in
+every row, so the separate row-sum pass is saved)
 which `paper_1807_06629_b200.binding.PRSGD` provides on the GPU (created with I = 0,
 set_worker_offset(first worker of the rank) and set_global_workers(N of the job)).  The collective
 is `torch.distributed.all_reduce` on whatever backend the process group uses (NCCL on GPUs).
@@ -65,13 +67,15 @@ def column_chunks(m_pad: int, chunks: int) -> List[Tuple[int, int]]:
 class ShardedPRSGD:
     """Algorithm 1 over all ranks of `group`; `engine` holds this rank's shard of the workers."""
 
-    def __init__(self, engine, N_global: int, I: int, group: Optional[dist.ProcessGroup] = None, chunks: int = 4):
+    def __init__(self, engine, N_global: int, I: int, group: Optional[dist.ProcessGroup] = None, chunks: int = 4,
+                 fuse_row_sums: bool = True):
         if I < 0:
             raise ValueError("I must be >= 0")
         if getattr(engine, "average_velocity", False):
             raise ValueError("averaged momentum buffers are not supported on a sharded job: "
                              "enable momentum with average_velocity=False")
         self.engine, self.N_global, self.I, self.group = engine, N_global, I, group
+        self.fuse_row_sums = fuse_row_sums     # use the engine's local_steps_sum (if it has one) instead of a row-sum pass
         self.stream = getattr(engine, "stream", None)
         with self._on_engine_stream():
             self.row = engine.new_row()
@@ -94,16 +98,34 @@ class ShardedPRSGD:
                 h.wait()
                 self.engine.assign_rows(self.row, float(self.N_global), c0, n)
 
+    def average_from_row_sums(self) -> None:
+        """Second half of an average whose first half the engine has fused into the last local step
+        (`local_steps_sum`: every local row holds the local row sum): all-reduce row 0 in place, chunk by
+        chunk, and restart all local rows at sum / N."""
+        with self._on_engine_stream():
+            row = self.engine.row0()
+            handles = [dist.all_reduce(row[c0:c0 + n], op=dist.ReduceOp.SUM, group=self.group, async_op=True)
+                       for (c0, n) in self.chunks]
+            for (c0, n), h in zip(self.chunks, handles):
+                h.wait()
+                self.engine.assign_rows(row, float(self.N_global), c0, n)
+
     def local_steps(self, k: int) -> None:
         """Iterations t+1 .. t+k; averages whenever I > 0 and t mod I == 0 (local step first, then the average)."""
         t = self.engine.get_step()
         end = t + k
+        fused = self.fuse_row_sums and hasattr(self.engine, "local_steps_sum")
         while t < end:
             nxt = end if self.I == 0 else min(end, (t // self.I + 1) * self.I)
-            self.engine.local_steps(nxt - t)
+            averaging = self.I > 0 and nxt % self.I == 0
+            if averaging and fused:           # the last local step of the period also forms the local row sums
+                self.engine.local_steps_sum(nxt - t)
+                self.average_from_row_sums()
+            else:
+                self.engine.local_steps(nxt - t)
+                if averaging:
+                    self.average()
             t = nxt
-            if self.I > 0 and t % self.I == 0:
-                self.average()
 
     def run_time_varying(self, s_begin: int, s_end: int, gamma_scale: float = 1.0) -> None:
         """Algorithm 2 over all ranks: epoch s starts from the node average of the whole job and takes

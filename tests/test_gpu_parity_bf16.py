@@ -655,6 +655,50 @@ def test_partial_sum_and_assign_rows_equal_average_on_the_bf16_store(torch_cuda)
     assert np.array_equal(a.get_params_stacked(), b.get_params_stacked())
 
 
+def test_row_sums_fused_into_the_last_local_step_equal_the_separate_pass(torch_cuda):
+    """prsgd_local_steps_sum (the period's last step in fused form with the division left out, every row = the
+    local row sum) followed by prsgd_assign_rows(row 0, N) against the fused update + average, and against
+    local steps + prsgd_partial_sum + prsgd_assign_rows: identical parameters and bf16 copy, plain and momentum
+    step; the next period's iterations agree too (the restart point is flagged as common in all three)."""
+    torch = torch_cuda
+    from paper_1807_06629_b200 import binding
+    for w in (SMALL[1], SMALL[4], _w("tc-sum-n5", 5, (64, 128, 10), 32, I=3), _w("tc-sum-wide", 3, (64, 448, 320, 10), 16, I=4)):
+        X, Y, x0 = make_inputs(w)
+        for mu in (None, 0.9):
+            outs = []
+            for how in ("fused average", "row sums in the last step", "separate row-sum pass"):
+                p = make_ctx(w, X, Y, x0, I=w.I if how == "fused average" else 0)
+                if mu is not None:
+                    p.enable_momentum(mu)
+                for period in range(2):
+                    if how == "fused average":
+                        p.local_steps(w.I)
+                    elif how == "row sums in the last step":
+                        p.local_steps_sum(w.I)
+                        half = (p.m_pad // 8) * 4
+                        p.assign_rows(p.row0(), float(w.N), 0, half)
+                        p.assign_rows(p.row0(), float(w.N), half, p.m_pad - half)
+                    else:
+                        p.local_steps(w.I)
+                        r = p.new_row()
+                        p.partial_sum(r)
+                        p.assign_rows(r, float(w.N))
+                p.set_interval(0)
+                p.local_steps(1)
+                p.sync()
+                outs.append((p.get_params_stacked(), p.shadow.view(torch.int16).cpu().numpy().copy(), p.get_step(),
+                             p.get_velocity_stacked() if mu is not None else None))
+                p.close()
+            for o in outs[1:]:
+                assert np.array_equal(outs[0][0], o[0]), (w.name, mu)
+                assert np.array_equal(outs[0][1], o[1]) and outs[0][2] == o[2] == 2 * w.I + 1
+                if mu is not None:
+                    assert np.array_equal(outs[0][3], o[3])
+    q = make_ctx(SMALL[1], *make_inputs(SMALL[1]))              # I = 2: the library averages by itself
+    with pytest.raises(binding.PRSGDError):
+        q.local_steps_sum(2)
+
+
 def test_training_run_tracks_the_oracle_loss_curve(torch_cuda):
     """48 iterations (12 periods) on the tensor-core path: draws exact, loss curve within bf16 noise of the
     oracle's, loss going down."""

@@ -316,6 +316,27 @@ def test_two_shards_on_one_gpu_reproduce_the_unsharded_run(torch_cuda):
     want = whole.get_params_stacked()
     assert all(np.array_equal(got[i], got[0]) for i in range(w.N))
     assert rel_l2(got, want) <= 1e-6
+    # the same job with the row sums formed by the period's last local step (prsgd_local_steps_sum): row 0 of each
+    # shard is the buffer the all-reduce would work on
+    fused = []
+    for first in (0, 2):
+        p = make_ctx(w.with_(N=2), X[first:first + 2], Y[first:first + 2], x0, I=0)
+        p.set_worker_offset(first)
+        p.set_global_workers(w.N)
+        fused.append(p)
+    for period in range(2):
+        for p in fused:
+            p.local_steps_sum(w.I)
+        total = fused[0].row0() + fused[1].row0()
+        for p in fused:
+            p.assign_rows(total, float(w.N))
+    got2 = np.concatenate([p.get_params_stacked() for p in fused])
+    assert np.array_equal(got2, got)
+    one = make_ctx(w, X, Y, x0, I=0)                      # one context: sums in place, then the division
+    for period in range(2):
+        one.local_steps_sum(w.I)
+        one.assign_rows(one.row0(), float(w.N))
+    assert np.array_equal(one.get_params_stacked(), want)
     # with a single context the two halves leave exactly the bits of prsgd_average
     a = make_ctx(w, X, Y, x0, I=0)
     b = make_ctx(w, X, Y, x0, I=0)
