@@ -259,7 +259,7 @@ def period_bytes(w: synth.Workload, m_pad: int, sms: int = 148, momentum: bool =
     a1_ready = False
     for j in range(1, I + 1):
         averaging = w.I > 0 and j == I
-        fuse = averaging and fused_average and not momentum
+        fuse = averaging and fused_average and (bf or not momentum)     # (the fp32 path has no fused momentum form)
         nxt = bf and next_forward and j < I and not averaging and L > 1 and epi
         # the first iteration of a period starts from N equal rows: launches that only read the weights (and the
         # fused update + average) read one copy for all workers
