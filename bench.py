@@ -499,12 +499,9 @@ def measure_config(torch, w_cfg, args, dev, rank, world, scaling, steps, warmup,
                              fused_epilogues=not args.no_fused_epilogues, next_forward=not args.no_next_forward,
                              dx_in_update=0 if args.no_dx_in_update else (2 if args.fold_all_dx else 1),
                              shared_restart=not args.no_shared_restart, forward_chain=args.forward_chain)
-    if sharded_mode:          # a shard's period: I plain iterations, then the average as passes of their own
-        fam_model = period_bytes(w.with_(I=0), p.m_pad, torch.cuda.get_device_properties(dev).multi_processor_count,
-                                 momentum=args.momentum is not None, fused_epilogues=not args.no_fused_epilogues,
-                                 next_forward=not args.no_next_forward, dx_in_update=not args.no_dx_in_update)
-        fam_model = {k: [v[0] * w.I, v[1] * w.I] for k, v in fam_model.items()}
-        fam_model["average"] = [w.N * p.m_pad * (4 + 4 + (2 if w.precision == 1 else 0)), 8]
+    if sharded_mode:          # a shard's period ends with row sums fused into the last step; the restart is a pass of its own
+        fam_model["average"] = [fam_model["average"][0] + p.m_pad * 4 + w.N * p.m_pad * (4 + (2 if w.precision == 1 else 0)),
+                                fam_model["average"][1] + 4]
     fams = {k: v for k, v in prof.items() if v[1] > 0 and fam_model.get(k, [0, 0])[0] > 0}
     dom = max(fams, key=lambda k: fams[k][0])
     dom_ms, dom_launches = fams[dom]

@@ -1790,42 +1790,55 @@ __global__ void __launch_bounds__(kUpdBlkThreads, 1) tc_update_dx_kernel(const _
       const int q = cbi & 1;
       const int cfeat = n0 + r;
       const bool valid = r < TN && cfeat < a.M_total;
-      uint16_t mk[16];
-      auto mask_fetch = [&](int bi) {
-        if (bi < batches && valid) {
+      // Everything this epilogue reads from global memory (the ReLU-mask values of the whole minibatch, the bias
+      // and its momentum) is requested before the accumulator wait: a layer of one row tile per block (the class
+      // layer) runs at the pace of this epilogue, and three dependent load latencies per block were most of it.
+      uint16_t mk[4][16];                                 // B <= 64: at most four batches of 16
+      if (valid) {
 #pragma unroll
-          for (int j = 0; j < 16; ++j) mk[j] = __ldg(a.mask_src + ((int64_t)n * a.B + bi * 16 + j) * a.ld_out + cfeat);
+        for (int bi = 0; bi < 4; ++bi) {
+          if (bi < batches) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) mk[bi][j] = __ldg(a.mask_src + ((int64_t)n * a.B + bi * 16 + j) * a.ld_out + cfeat);
+          }
         }
-      };
-      mask_fetch(0);
+      }
+      const bool step_bias = valid && a.bias_rw != nullptr;
+      float* bp = a.bias_rw + (int64_t)n * a.bias_stride + cfeat;
+      float* vp = a.bias_vel + (int64_t)n * a.bias_stride + cfeat;
+      float b_old = 0.f, v_old = 0.f;
+      if (step_bias) {
+        b_old = *bp;
+        if (a.bias_vel != nullptr) v_old = *vp;
+      }
       ok = __all_sync(0xffffffffu, mbar_wait(dacc_full(q), (cbi >> 1) & 1u, abort_flag, a.status, 0x50A));
       if (!ok) break;
       tc_fence_after();
       float gsum = 0.f;
-      for (int bi = 0; bi < batches; ++bi) {
-        uint32_t v[16];
-        tmem_ld16(tmem + lane_off + kDxCol + (uint32_t)(q * a.B + bi * 16), v);
-        tmem_ld_wait();
-        if (valid) {
 #pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const float d = (mk[j] & 0x7FFFu) != 0 ? __uint_as_float(v[j]) : 0.f;
-            gsum += d;
-            a.out_bk[((int64_t)n * a.B + bi * 16 + j) * a.ld_out + cfeat] = f32_to_bf16_rn(d);
+      for (int bi = 0; bi < 4; ++bi) {
+        if (bi < batches) {
+          uint32_t v[16];
+          tmem_ld16(tmem + lane_off + kDxCol + (uint32_t)(q * a.B + bi * 16), v);
+          tmem_ld_wait();
+          if (valid) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const float d = (mk[bi][j] & 0x7FFFu) != 0 ? __uint_as_float(v[j]) : 0.f;
+              gsum += d;
+              a.out_bk[((int64_t)n * a.B + bi * 16 + j) * a.ld_out + cfeat] = f32_to_bf16_rn(d);
+            }
           }
         }
-        mask_fetch(bi + 1);
       }
       tc_fence_before();
       mbar_arrive(dacc_empty(q));
-      if (valid && a.bias_rw != nullptr) {
-        float* bp = a.bias_rw + (int64_t)n * a.bias_stride + cfeat;
+      if (step_bias) {
         if (a.bias_vel != nullptr) {                      // momentum form of the bias step
-          float* vp = a.bias_vel + (int64_t)n * a.bias_stride + cfeat;
-          gsum = fmaf(a.mu, *vp, gsum);
+          gsum = fmaf(a.mu, v_old, gsum);
           *vp = gsum;
         }
-        *bp = fmaf(-a.gamma, gsum, *bp);
+        *bp = fmaf(-a.gamma, gsum, b_old);
       }
       ++cbi;
     }
