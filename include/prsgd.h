@@ -163,8 +163,10 @@ int prsgd_local_steps(prsgd_ctx* ctx, int64_t k);
 int prsgd_average(prsgd_ctx* ctx);
 
 /* xbar^t = (1/N) sum_i x_i^t (Eq. node-average-x), m floats in canonical
- * order, WITHOUT modifying the store.  Synchronises the stream when dst is on
- * the host. */
+ * order, WITHOUT modifying the store.  When the library knows that all rows hold
+ * the same bits (right after an average, see PRSGD_OPT_SHARED_RESTART) that row
+ * is returned as it stands instead of summing N copies of it.  Synchronises the
+ * stream when dst is on the host. */
 int prsgd_get_average(prsgd_ctx* ctx, float* dst, int dst_on_device);
 
 /* The same read-out without stopping the training stream: the mean (Eq. node-average-x) is formed into

@@ -848,10 +848,15 @@ int prsgd_get_average_async(prsgd_ctx* c, float* h_dst, void* copy_stream) {
   if (!c->readout_event) CUDA_TRY(c, cudaEventCreateWithFlags(&c->readout_event, cudaEventDisableTiming));
   // the staging row is free again once the previous asynchronous read-out has left it
   if (c->readout_pending) CUDA_TRY(c, cudaStreamWaitEvent(c->stream, c->readout_event, 0));
-  prof_begin(c, PRSGD_KERNEL_AVERAGE);
-  average_rows_kernel<1, false><<<grid1d(c->m_pad / 4, 256), 256, 0, c->stream>>>(c->params, c->N, c->m_pad, c->m_pad,
-                                                                              c->stage_row, nullptr);
-  LAUNCH_CHECK(c);
+  if (c->rows_identical) {
+    // right after an average every row IS the node average: snapshot row 0 instead of summing N equal rows
+    CUDA_TRY(c, cudaMemcpyAsync(c->stage_row, c->params, (size_t)c->m_pad * 4, cudaMemcpyDeviceToDevice, c->stream));
+  } else {
+    prof_begin(c, PRSGD_KERNEL_AVERAGE);
+    average_rows_kernel<1, false><<<grid1d(c->m_pad / 4, 256), 256, 0, c->stream>>>(c->params, c->N, c->m_pad, c->m_pad,
+                                                                                c->stage_row, nullptr);
+    LAUNCH_CHECK(c);
+  }
   CUDA_TRY(c, cudaEventRecord(c->mean_ready_event, c->stream));
   CUDA_TRY(c, cudaStreamWaitEvent(cs, c->mean_ready_event, 0));
   int64_t pos = 0;
@@ -873,17 +878,22 @@ int prsgd_get_average(prsgd_ctx* c, float* dst, int dst_on_device) {
   if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
   if (!dst) return fail(c, PRSGD_ERR_ARG, "dst is NULL");
   if (c->readout_pending) CUDA_TRY(c, cudaStreamWaitEvent(c->stream, c->readout_event, 0));   // staging row in use
-  prof_begin(c, PRSGD_KERNEL_AVERAGE);
-  average_rows_kernel<1, false><<<grid1d(c->m_pad / 4, 256), 256, 0, c->stream>>>(c->params, c->N, c->m_pad, c->m_pad,
-                                                                              c->stage_row, nullptr);
-  LAUNCH_CHECK(c);
+  const float* mean = c->stage_row;
+  if (c->rows_identical) {
+    mean = c->params;            // right after an average every row IS the node average: row 0, as it stands
+  } else {
+    prof_begin(c, PRSGD_KERNEL_AVERAGE);
+    average_rows_kernel<1, false><<<grid1d(c->m_pad / 4, 256), 256, 0, c->stream>>>(c->params, c->N, c->m_pad, c->m_pad,
+                                                                                c->stage_row, nullptr);
+    LAUNCH_CHECK(c);
+  }
   int64_t pos = 0;
   for (int l = 0; l < c->L; ++l) {
     const Layer& ly = c->layer[l];
     const int64_t seg[2] = {(int64_t)ly.d_in * ly.d_out, (int64_t)ly.d_out};
     const int64_t offs[2] = {ly.w_off, ly.b_off};
     for (int q = 0; q < 2; ++q) {
-      CUDA_TRY(c, cudaMemcpyAsync(dst + pos, c->stage_row + offs[q], seg[q] * 4, cudaMemcpyDefault, c->stream));
+      CUDA_TRY(c, cudaMemcpyAsync(dst + pos, mean + offs[q], seg[q] * 4, cudaMemcpyDefault, c->stream));
       pos += seg[q];
     }
   }

@@ -190,6 +190,17 @@ def test_get_average_is_the_mean_and_leaves_the_store_alone(torch_cuda):
     p.average()
     rows = p.get_params_stacked()
     assert all(np.array_equal(rows[i], rows[0]) for i in range(w.N))
+    # right after an average the node average IS every row: returned as it stands, also for a worker count
+    # that is no power of two (summing N copies and dividing would round)
+    assert np.array_equal(p.get_average(), rows[0])
+    w3 = w.with_(N=3)
+    q = make_ctx(w3, X[:3], Y[:3], x0)
+    q.local_steps(w3.I)                                             # ends on an averaging iteration
+    assert np.array_equal(q.get_average(), q.get_params(0))
+    q.local_steps(1)
+    after = q.get_params_stacked().astype(np.float64)
+    assert not np.array_equal(q.get_average(), q.get_params(0))     # workers differ again: the mean is formed
+    assert rel_l2(q.get_average(), orc.node_average(after)) < 1e-6
 
 
 def test_asynchronous_read_out_equals_get_average_while_training_goes_on(torch_cuda):
