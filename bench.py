@@ -451,6 +451,8 @@ def measure_config(torch, w_cfg, args, dev, rank, world, scaling, steps, warmup,
             p.set_option(opt, 0)
     if args.fold_all_dx:
         p.set_option(binding.OPT_DX_IN_UPDATE, 2)
+    if args.dx_own_pairs:
+        p.set_option(binding.OPT_DX_SHARED_PAIR, 0)
     if args.forward_chain:
         p.set_option(binding.OPT_FORWARD_CHAIN, 1)
     if args.worker_groups is not None:
@@ -573,6 +575,8 @@ def parse_args(argv=None):
                     help="softmax-CE gradient and bias steps as kernels of their own instead of GEMM epilogues")
     ap.add_argument("--no-dx-in-update", action="store_true",
                     help="separate dX launches instead of forming dZ of the layer below inside the update launch")
+    ap.add_argument("--dx-own-pairs", action="store_true",
+                    help="64-wide update + dX with a pair of bf16 tiles per stage instead of one shared pair")
     ap.add_argument("--fold-all-dx", action="store_true",
                     help="form dZ of the layer below inside the update launch for every layer, whatever its size")
     ap.add_argument("--no-shared-restart", action="store_true",

@@ -320,6 +320,11 @@ int prsgd_get_velocity_stacked(prsgd_ctx* ctx, float* dst, int dst_on_device);
  * one group's long update kernels run, another group's short launches find free SMs.  Not while a worker
  * mask or profiling is on.  Same bits as one chain for all workers. */
 #define PRSGD_OPT_WORKER_GROUPS 12
+/* PRSGD_OPT_DX_SHARED_PAIR (default 1, tensor-core path): stage layout of the 64-wide update + dX launch.  1: the
+ * two bf16 tiles (old and stepped weights) exist once, behind the stages, and a stage holds only the fp32 tile
+ * and the operand boxes, which makes room for a deeper pipeline; 0: every stage has its own pair.  A tuning knob:
+ * same bits either way. */
+#define PRSGD_OPT_DX_SHARED_PAIR 13
 /* PRSGD_OPT_CHECK_FINITE (default 0): when 1, prsgd_sync also runs prsgd_check_finite. */
 #define PRSGD_OPT_CHECK_FINITE 9
 int prsgd_set_option(prsgd_ctx* ctx, int32_t option, int64_t value);

@@ -32,6 +32,7 @@ OPT_CHECK_FINITE = 9
 OPT_SHARED_RESTART = 10
 OPT_FORWARD_CHAIN = 11
 OPT_WORKER_GROUPS = 12
+OPT_DX_SHARED_PAIR = 13
 ERR_DEVICE_TIMEOUT, ERR_NONFINITE = -6, -7
 KERNEL_FAMILIES = ("forward", "softmax", "dx", "update", "update_average", "average", "misc")
 MAX_LAYERS = 16

@@ -1499,14 +1499,18 @@ struct UpdateDxArgs {
   const uint8_t* active;     // per-worker flag or nullptr: an inactive worker's column blocks are skipped
 };
 
-// TN = 64: every stage holds fp32 master | momentum | bf16 old | bf16 new (first the a_{l-1} box) | two dZ_l boxes.
-// TN = 128 (512-byte rows, which the memory system serves ~7 % faster than 256-byte ones): the two bf16 tiles
-// do not fit twice, so only master | dZ_l boxes | a_{l-1} boxes are staged (two stages) and ONE pair of bf16
-// tiles behind the stages is shared: the epilogue of a tile waits until the pair of the tile before it has been
-// read by its TMA store and its dX MMAs.  No momentum form at this width.
-template <int TN, bool MOM> struct UpdDxCfg {
+// Two stage layouts.  Own pair (SP = false): every stage holds fp32 master | momentum | bf16 old | bf16 new (first
+// the a_{l-1} box) | two dZ_l boxes.  Shared pair (SP = true): only what has a long latency is staged (master |
+// dZ_l boxes | a_{l-1} boxes) and ONE pair of bf16 tiles behind the stages is shared: the epilogue of a tile
+// waits until the pair of the tile before it has been read by its TMA store and its dX MMAs.  The shared pair
+// makes room for more stages (64-wide: four instead of three at B = 32, three instead of two at B = 64), and it
+// is the only way 128-wide tiles fit at all (512-byte rows, which the memory system serves ~7 % faster than
+// 256-byte ones; two stages, B <= 32).  The momentum form keeps its own pairs.
+template <int TN, bool MOM, bool SP = (TN == 128)> struct UpdDxCfg {
   static_assert(TN == 64 || !MOM, "the momentum form uses 64-wide tiles");
-  static constexpr bool kSharedPair = TN == 128;
+  static_assert(!(SP && MOM), "the momentum form keeps a pair of bf16 tiles per stage");
+  static_assert(TN == 64 || SP, "128-wide tiles need the shared pair");
+  static constexpr bool kSharedPair = SP;
   static constexpr uint32_t kMaster = 128u * TN * 4u;      // fp32 master tile
   static constexpr uint32_t kVel = MOM ? kMaster : 0u;     // fp32 momentum tile right behind it
   static constexpr uint32_t kOld = 128u * TN * 2u;         // bf16 of the weights before the step
@@ -1518,14 +1522,14 @@ template <int TN, bool MOM> struct UpdDxCfg {
   }
   __host__ __device__ static uint32_t shared_bytes() { return kSharedPair ? kOld + kNew : 0u; }
   static int stages(int B) {
-    if (kSharedPair) return (2u * stage(B) + shared_bytes() + 2048u <= 227u * 1024u) ? 2 : 0;
-    int s = (int)((227u * 1024u - 2048u) / stage(B));
+    int s = (int)((227u * 1024u - 2048u - shared_bytes()) / stage(B));
+    if (s < 2) return 0;                       // (a tile's dX product is issued after the next tile's dW: two stages at least)
     return s > 4 ? 4 : s;
   }
   static size_t smem(int B) { return (size_t)stages(B) * stage(B) + shared_bytes() + 1024 + 512; }
 };
 
-template <int TN, bool MOM>
+template <int TN, bool MOM, bool SP = (TN == 128)>
 __global__ void __launch_bounds__(kUpdBlkThreads, 1) tc_update_dx_kernel(const __grid_constant__ CUtensorMap mapDelta,
                                                                       const __grid_constant__ CUtensorMap mapAct,
                                                                       const __grid_constant__ CUtensorMap mapMaster,
@@ -1533,7 +1537,7 @@ __global__ void __launch_bounds__(kUpdBlkThreads, 1) tc_update_dx_kernel(const _
                                                                       const __grid_constant__ CUtensorMap mapVel,
                                                                       const UpdateDxArgs a) {
   using namespace ptx;
-  using Cfg = UpdDxCfg<TN, MOM>;
+  using Cfg = UpdDxCfg<TN, MOM, SP>;
   constexpr int NB32 = TN / 32, NB64 = TN / 64;
   constexpr bool kSharedPair = Cfg::kSharedPair;
   constexpr uint32_t kDxCol = 256u;                     // TMEM: dW accumulators in columns [0, 256), dX ones behind
@@ -1980,8 +1984,10 @@ inline int tc_create(prsgd_ctx* c, std::string* err) {
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_kernel<true, 64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCfg<64, true>::smem(c->B));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_dx_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdDxCfg<64, false>::smem(c->B));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_dx_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdDxCfg<64, true>::smem(c->B));
-  if (e == cudaSuccess && UpdDxCfg<128, false>::stages(c->B) == 2)
+  if (e == cudaSuccess && UpdDxCfg<128, false>::stages(c->B) >= 2)
     e = cudaFuncSetAttribute(tc_update_dx_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdDxCfg<128, false>::smem(c->B));
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(tc_update_dx_kernel<64, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdDxCfg<64, false, true>::smem(c->B));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_next_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdNextCfg<64, false>::smem(c->B));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_next_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdNextCfg<128, false>::smem(c->B));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_next_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdNextCfg<64, true>::smem(c->B));
@@ -2174,13 +2180,13 @@ inline bool tc_layer_folds_dx(const prsgd_ctx* c, int l) {
 }
 
 // Update of layer l >= 2 that also forms dZ_{l-1} (tc_update_dx_kernel): replaces dX_l + update_l.
-template <int TN, bool MOM>
+template <int TN, bool MOM, bool SP = (TN == 128)>
 inline void tc_launch_update_dx_m(prsgd_ctx* c, int l) {
   TcState* st = static_cast<TcState*>(c->tc);
   const Layer& ly = c->layer[l - 1];
   UpdateDxArgs a{};
   a.B = c->B; a.N = c->N; a.tiles_m = (ly.d_out + 127) / 128; a.tiles_n = (ly.d_in + TN - 1) / TN;
-  a.gamma = c->gamma; a.status = c->status; a.stages = UpdDxCfg<TN, MOM>::stages(c->B);
+  a.gamma = c->gamma; a.status = c->status; a.stages = UpdDxCfg<TN, MOM, SP>::stages(c->B);
   a.out_bk = c->buf.delta_bk[l - 1]; a.mask_src = c->buf.act_bk[l - 1]; a.ld_out = c->buf.ld[l - 1]; a.M_total = ly.d_in;
   a.bias_rw = c->params + c->layer[l - 2].b_off; a.bias_stride = c->m_pad;
   a.mu = c->mu; a.bias_vel = MOM ? c->velocity + c->layer[l - 2].b_off : nullptr;
@@ -2188,7 +2194,7 @@ inline void tc_launch_update_dx_m(prsgd_ctx* c, int l) {
   const int items = a.tiles_n * c->N;
   const int grid = items < st->num_sms ? items : st->num_sms;
   const TcLayerMaps& mp = st->layer[l - 1];
-  launch_pdl(tc_update_dx_kernel<TN, MOM>, dim3(grid), kUpdBlkThreads, UpdDxCfg<TN, MOM>::smem(c->B), c->stream, mp.delta_out,
+  launch_pdl(tc_update_dx_kernel<TN, MOM, SP>, dim3(grid), kUpdBlkThreads, UpdDxCfg<TN, MOM, SP>::smem(c->B), c->stream, mp.delta_out,
              mp.act_in, mp.master, mp.shadow_k, MOM ? mp.velocity : mp.master, a);
 }
 
@@ -2203,8 +2209,9 @@ inline void tc_launch_update_dx(prsgd_ctx* c, int l) {
     const int64_t blocks128 = (int64_t)((ly.d_in + 127) / 128) * c->N;
     tile = (blocks128 >= 4 * (int64_t)st->num_sms && ly.d_out > 128) ? 128 : 64;
   }
-  if (tile == 128 && UpdDxCfg<128, false>::stages(c->B) == 2) tc_launch_update_dx_m<128, false>(c, l);
-  else tc_launch_update_dx_m<64, false>(c, l);
+  if (tile == 128 && UpdDxCfg<128, false>::stages(c->B) >= 2) tc_launch_update_dx_m<128, false>(c, l);
+  else if (c->dx_shared_pair) tc_launch_update_dx_m<64, false, true>(c, l);      // more stages (see UpdDxCfg)
+  else tc_launch_update_dx_m<64, false, false>(c, l);
 }
 
 // Update of layer 1 that also forms a_1 of the next iteration (tc_update_next_kernel).

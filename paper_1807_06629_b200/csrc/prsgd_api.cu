@@ -713,7 +713,7 @@ void period_key(const prsgd_ctx* c, uint64_t (&key)[13]) {
   key[7] = (uint64_t)c->average_velocity; key[8] = reinterpret_cast<uint64_t>(c->X);
   key[9] = reinterpret_cast<uint64_t>(c->Y); key[10] = (uint64_t)c->worker0; key[11] = (uint64_t)c->fused_epilogues | ((uint64_t)c->early_loads << 1) | ((uint64_t)c->next_forward << 2) | ((uint64_t)c->dx_in_update << 3);
   key[12] = (c->rows_identical ? 1u : 0u) | ((uint64_t)c->shared_restart << 1) | ((uint64_t)c->forward_chain << 2) |
-            ((uint64_t)c->worker_groups << 3);   // the period's first iteration may share reads
+            ((uint64_t)c->worker_groups << 3) | ((uint64_t)c->dx_shared_pair << 6);   // the period's first iteration may share reads
 }
 
 // One whole averaging period (I iterations starting right after an average) as a CUDA graph: the
@@ -1118,6 +1118,7 @@ int prsgd_set_option(prsgd_ctx* c, int32_t option, int64_t value) {
   if (option == PRSGD_OPT_CHECK_FINITE) { c->check_finite = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_SHARED_RESTART) { c->shared_restart = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_FORWARD_CHAIN) { c->forward_chain = value != 0; return PRSGD_OK; }
+  if (option == PRSGD_OPT_DX_SHARED_PAIR) { c->dx_shared_pair = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_WORKER_GROUPS) {
     if (value < 1 || value > kMaxGroups) return fail(c, PRSGD_ERR_ARG, "PRSGD_OPT_WORKER_GROUPS takes 1..4");
     // group g holds the contiguous workers [g N / G, (g + 1) N / G)

@@ -96,6 +96,7 @@ struct prsgd_ctx {
   float* velocity = nullptr;     // [N][m_pad] fp32 momentum buffers, caller-owned
   int average_velocity = 0;      // average the buffers together with the models
   int upd_tile = 0;              // column width of the update kernel's tile: 0 = chosen per launch, 64 or 128
+  int dx_shared_pair = 1;        // 64-wide update + dX: one pair of bf16 tiles behind the stages (more stages) instead of one per stage
   int dx_in_update = 1;          // layers >= 2: the update launch also forms dZ of the layer below (tensor-core path)
   int next_forward = 1;          // layer 1's update also forms a_1 of the next iteration (tensor-core path)
   bool a1_ready = false;         // a_1 of the coming iteration has already been formed by the previous update

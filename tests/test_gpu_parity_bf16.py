@@ -252,6 +252,39 @@ def test_dx_folded_into_the_update_changes_no_bit(torch_cuda):
         assert outs[1][2] < outs[0][2]
 
 
+def test_stage_layouts_of_the_update_dx_kernel_change_no_bit(torch_cuda):
+    """64-wide update + dX with one shared pair of bf16 tiles behind a deeper pipeline against a pair per stage:
+    identical parameters, losses and bf16 copies for B = 16, 32, 64, single- and multi-tile column blocks, ragged
+    widths, a worker mask, direct and replayed."""
+    torch = torch_cuda
+    from paper_1807_06629_b200 import binding
+    cases = (SMALL[1], SMALL[2], SMALL[3], SMALL[4], SMALL[6], _w("tc-pair-b64", 3, (128, 320, 192, 10), 64, I=3),
+             _w("tc-pair-wide", 3, (64, 448, 320, 10), 16, I=4))
+    for w in cases:
+        X, Y, x0 = make_inputs(w)
+        for mask in (None, [1 if i != 1 else 0 for i in range(w.N)]):
+            outs = []
+            for shared, graph in ((0, 0), (1, 0), (1, 1)):
+                with torch.cuda.stream(torch.cuda.Stream()):
+                    p = make_ctx(w, X, Y, x0)
+                    p.set_option(binding.OPT_DX_IN_UPDATE, 2)          # every layer >= 2 takes the folded kernel
+                    p.set_option(binding.OPT_UPDATE_TILE, 64)
+                    p.set_option(binding.OPT_DX_SHARED_PAIR, shared)
+                    p.set_option(binding.OPT_GRAPH, graph)
+                    if mask is not None:
+                        p.set_active(mask)
+                    p.local_steps(2)
+                    p.local_steps(2 * w.I + 1)
+                    p.sync()
+                    outs.append((p.get_params_stacked(), p.get_losses(), p.shadow.view(torch.int16).cpu().numpy().copy()))
+                    torch.cuda.current_stream().synchronize()
+                    p.close()
+            keep = [i for i in range(w.N) if mask is None or mask[i]]
+            for o in outs[1:]:
+                assert np.array_equal(outs[0][0], o[0]), (w.name, mask)
+                assert np.array_equal(outs[0][1][keep], o[1][keep]) and np.array_equal(outs[0][2], o[2])
+
+
 @pytest.mark.parametrize("avg_v", [False, True])
 def test_folded_kernels_with_momentum_change_no_bit(torch_cuda, avg_v):
     """The momentum step inside the two folded update kernels (dZ of the layer below, next forward of layer 1)
