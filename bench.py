@@ -229,7 +229,7 @@ def ncu_traffic_per_launch(workload: str, family: str, N: int):
 # ----------------------------------------------------------------------------- byte model
 def period_bytes(w: synth.Workload, m_pad: int, sms: int = 148, momentum: bool = False, fused_average: bool = True,
                  fused_epilogues: bool = True, next_forward: bool = True, dx_in_update=True,
-                 shared_restart: bool = True, forward_chain: bool = False) -> dict:
+                 shared_restart: bool = True, forward_chain: bool = False, head_kernel=1) -> dict:
     """Algorithmic HBM bytes and launch counts of ONE averaging period (prsgd_local_steps(I) from a period
     boundary) of all N workers, per kernel family: {family: [bytes, launches]}.
 
@@ -244,6 +244,9 @@ def period_bytes(w: synth.Workload, m_pad: int, sms: int = 148, momentum: bool =
     enough tiles takes the fused update + average (same bytes as a plain update, dX a launch of its own),
     a smaller one the plain update followed by the node average of its weight segment (8 + 2 B/param).
     Without the fused form the stand-alone average reads and writes the whole store (8 B/word, + 2 B bf16 copy).
+    The class layer (at most 128 classes, last hidden width 128..1024, plain step) is one launch of its own
+    family ("head"): its forward read of the bf16 copy, its update (10 B/param) and the mask read and dZ write
+    of the layer below; a_{L-1} is read once for both products.
     """
     bf = w.precision == 1
     e = 2 if bf else 4
@@ -251,7 +254,9 @@ def period_bytes(w: synth.Workload, m_pad: int, sms: int = 148, momentum: bool =
     L = len(d) - 1
     upd_b = 8 + (2 if bf else 0) + (8 if momentum else 0)
     epi = bf and fused_epilogues and d[L] <= 128
-    fam = {k: [0, 0] for k in ("forward", "softmax", "dx", "update", "update_average", "average", "misc")}
+    fam = {k: [0, 0] for k in ("forward", "softmax", "dx", "update", "update_average", "average", "misc", "head")}
+    head_ok = (bf and epi and head_kernel and dx_in_update == 1 and L >= 2 and not momentum
+               and d[L - 1] in (128, 256, 512, 1024) and (head_kernel == 2 or N * (d[L - 1] // 128) <= sms))
 
     def add(name, nbytes):
         fam[name][0] += nbytes
@@ -265,16 +270,24 @@ def period_bytes(w: synth.Workload, m_pad: int, sms: int = 148, momentum: bool =
         # fused update + average) read one copy for all workers
         wr = 1 if (bf and shared_restart and j == 1 and w.I > 0) else N
         l_first = 2 if a1_ready else 1
-        chained = bf and forward_chain and 2 <= L - l_first + 1 <= 8      # all layers' forward GEMMs in one launch
-        for l in range(l_first, L + 1):
+        head = head_ok and not (fuse and 2 * ((d[L] + 127) // 128) * ((d[L - 1] + 63) // 64) >= sms)
+        l_last = L - 1 if head else L
+        chained = bf and forward_chain and 2 <= l_last - l_first + 1 <= 8      # all layers' forward GEMMs in one launch
+        for l in range(l_first, l_last + 1):
             add("forward", wr * d[l] * d[l - 1] * e + N * (d[l] * 4 + B * d[l - 1] * e + B * d[l] * (e if l < L else 4)))
             if chained and l > l_first:
                 fam["forward"][1] -= 1
         a1_ready = False
         if not epi:
             add("softmax", N * B * d[L] * (4 + 4 + e))
+        if head:
+            add("head", N * (d[L] * d[L - 1] * e + B * d[L - 1] * e + (d[L] * d[L - 1] + d[L]) * upd_b + B * d[L - 1] * 2 * e))
         for l in range(L, 0, -1):
             wl = d[l] * d[l - 1]
+            if l == L and head:
+                if bf and fuse:
+                    add("average", N * wl * 10)
+                continue
             tiles64 = ((d[l] + 127) // 128) * ((d[l - 1] + 63) // 64)
             fuse_l = fuse and (not bf or 2 * tiles64 >= sms)
             folds = bf and epi and dx_in_update and (dx_in_update == 2 or ((d[l - 1] + 63) // 64) * N >= 3 * sms or d[l] <= 128)
@@ -446,9 +459,12 @@ def measure_config(torch, w_cfg, args, dev, rank, world, scaling, steps, warmup,
                       (args.no_next_forward, binding.OPT_NEXT_FORWARD), (args.no_early_loads, binding.OPT_EARLY_LOADS),
                       (args.no_fused_epilogues, binding.OPT_FUSED_EPILOGUES),
                       (args.no_shared_restart, binding.OPT_SHARED_RESTART),
-                      (args.no_forward_chain, binding.OPT_FORWARD_CHAIN)):
+                      (args.no_forward_chain, binding.OPT_FORWARD_CHAIN),
+                      (args.no_head_kernel, binding.OPT_HEAD_KERNEL)):
         if flag:
             p.set_option(opt, 0)
+    if args.head_kernel_always:
+        p.set_option(binding.OPT_HEAD_KERNEL, 2)
     if args.fold_all_dx:
         p.set_option(binding.OPT_DX_IN_UPDATE, 2)
     if args.dx_own_pairs:
@@ -500,7 +516,8 @@ def measure_config(torch, w_cfg, args, dev, rank, world, scaling, steps, warmup,
                              momentum=args.momentum is not None, fused_average=not args.no_fuse,
                              fused_epilogues=not args.no_fused_epilogues, next_forward=not args.no_next_forward,
                              dx_in_update=0 if args.no_dx_in_update else (2 if args.fold_all_dx else 1),
-                             shared_restart=not args.no_shared_restart, forward_chain=args.forward_chain)
+                             shared_restart=not args.no_shared_restart, forward_chain=args.forward_chain,
+                             head_kernel=0 if args.no_head_kernel else (2 if args.head_kernel_always else 1))
     if sharded_mode:          # a shard's period ends with row sums fused into the last step; the restart is a pass of its own
         fam_model["average"] = [fam_model["average"][0] + p.m_pad * 4 + w.N * p.m_pad * (4 + (2 if w.precision == 1 else 0)),
                                 fam_model["average"][1] + 4]
@@ -586,6 +603,10 @@ def parse_args(argv=None):
     ap.add_argument("--forward-chain", action="store_true", help="one forward launch for all layers")
     ap.add_argument("--no-forward-chain", action="store_true",
                     help="one forward launch per layer instead of one launch for all layers")
+    ap.add_argument("--head-kernel-always", action="store_true",
+                    help="the class layer as one launch of clusters even when its CTAs need more than one wave")
+    ap.add_argument("--no-head-kernel", action="store_true",
+                    help="the class layer's forward GEMM and update as launches of their own instead of one launch of clusters")
     ap.add_argument("--no-next-forward", action="store_true",
                     help="layer 1's update does not form the next iteration's a_1")
     ap.add_argument("--no-early-loads", action="store_true",

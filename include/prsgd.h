@@ -325,6 +325,24 @@ int prsgd_get_velocity_stacked(prsgd_ctx* ctx, float* dst, int dst_on_device);
  * and the operand boxes, which makes room for a deeper pipeline; 0: every stage has its own pair.  A tuning knob:
  * same bits either way. */
 #define PRSGD_OPT_DX_SHARED_PAIR 13
+/* PRSGD_OPT_HEAD_KERNEL (default 1, tensor-core path, at least two layers, at most 128 classes, width of the last
+ * hidden layer 128, 256, 512 or 1024, plain SGD step, PRSGD_OPT_DX_IN_UPDATE and PRSGD_OPT_FUSED_EPILOGUES at
+ * their defaults): everything an iteration does with the class layer -- logits, softmax cross-entropy gradient
+ * and loss, the step of W_L and b_L (Eq. parallel-sgd-x-update), dZ of the layer below and the step of its
+ * bias -- is one launch in which a thread-block cluster per worker splits the last hidden layer's features among
+ * its CTAs (128 each) and sums the logit shares in a fixed order.  1: when all those CTAs fit on the GPU at once
+ * (workers x width / 128 <= SM count); 2: always; 0: never, the last forward GEMM and the class layer's update are
+ * launches of their own.  The two forms agree to fp32 rounding of the logits (different summation order, fast
+ * exponential), not bit for bit; each is deterministic. */
+#define PRSGD_OPT_HEAD_KERNEL 14
+/* PRSGD_OPT_COMMON_POINT (default 1, tensor-core path, plain SGD step, fused average, PRSGD_OPT_SHARED_RESTART on):
+ * an averaging iteration that STARTS from N equal rows (every iteration when I = 1, which the paper notes is
+ * parallel mini-batch SGD; otherwise the first step after prsgd_average when I divides its number) forms the
+ * new average as x - (gamma / N) sum_i G_i: one weight-gradient GEMM per tile over the minibatches of all
+ * workers, one step, N row stores (Eq. parallel-sgd-x-update summed over i, then Algorithm 1's average).
+ * Equal to update-then-average up to fp32 rounding, not bit for bit; deterministic.  0: the N stepped models are
+ * formed and summed one by one. */
+#define PRSGD_OPT_COMMON_POINT 15
 /* PRSGD_OPT_CHECK_FINITE (default 0): when 1, prsgd_sync also runs prsgd_check_finite. */
 #define PRSGD_OPT_CHECK_FINITE 9
 int prsgd_set_option(prsgd_ctx* ctx, int32_t option, int64_t value);
@@ -337,7 +355,8 @@ int prsgd_set_option(prsgd_ctx* ctx, int32_t option, int64_t value);
 #define PRSGD_KERNEL_UPDATE_AVERAGE 4  /* the same with the node average fused in                   */
 #define PRSGD_KERNEL_AVERAGE        5  /* stand-alone node average (+ broadcast)                    */
 #define PRSGD_KERNEL_MISC           6  /* broadcast of x^0, shadow refresh                          */
-#define PRSGD_KERNEL_FAMILIES       7
+#define PRSGD_KERNEL_HEAD           7  /* class layer: logits, softmax-CE gradient, step, dZ below  */
+#define PRSGD_KERNEL_FAMILIES       8
 
 /* Device time (milliseconds, from the event pairs) and launch count of one
  * kernel family since the previous call for that family; both counters are

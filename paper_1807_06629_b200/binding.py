@@ -33,8 +33,10 @@ OPT_SHARED_RESTART = 10
 OPT_FORWARD_CHAIN = 11
 OPT_WORKER_GROUPS = 12
 OPT_DX_SHARED_PAIR = 13
+OPT_HEAD_KERNEL = 14
+OPT_COMMON_POINT = 15
 ERR_DEVICE_TIMEOUT, ERR_NONFINITE = -6, -7
-KERNEL_FAMILIES = ("forward", "softmax", "dx", "update", "update_average", "average", "misc")
+KERNEL_FAMILIES = ("forward", "softmax", "dx", "update", "update_average", "average", "misc", "head")
 MAX_LAYERS = 16
 
 EXPORTS = [

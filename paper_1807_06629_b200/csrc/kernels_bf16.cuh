@@ -33,6 +33,9 @@ struct TcLayerMaps {
 
 struct TcState {
   TcLayerMaps layer[PRSGD_MAX_LAYERS];
+  CUtensorMap head_shadow;  // bf16 W_L, box {64, ceil16(d_L), 1}: tiles of tc_head_kernel (valid when head_rows > 0)
+  CUtensorMap head_master;  // fp32 W_L, box {32, ceil16(d_L), 1}
+  int head_rows = 0;
   int num_sms = 148;
   bool pool_bound = false;
 };
@@ -1928,6 +1931,11 @@ __global__ void __launch_bounds__(128) bias_average_kernel(const BiasAverageArgs
   for (int r = 0; r < a.N; ++r) p[(int64_t)r * a.m_pad] = y;
 }
 
+}  // namespace prsgd
+#include "kernels_head.cuh"
+#include "kernels_update_common.cuh"
+namespace prsgd {
+
 // Self-test of the failure path: waits on an mbarrier that nothing ever arrives on, with a short
 // limit, so that the wait expires, the status word is set and the kernel returns normally.
 __global__ void __launch_bounds__(32) wait_expiry_kernel(DeviceStatus* status, long long limit_cycles) {
@@ -1968,6 +1976,14 @@ inline int tc_create(prsgd_ctx* c, std::string* err) {
       rc = make_map3(&mp.act_in, false, c->buf.act_bk[l - 1], ldi, B, N, ldi * 2, B * ldi * 2, 64, (uint32_t)B, err);
     }
   }
+  if (rc == PRSGD_OK && c->L >= 2 && c->dims[c->L] <= 128) {      // the class layer's tiles with only as many rows as it has
+    const Layer& ly = c->layer[c->L - 1];
+    const uint64_t din = ly.d_in, dout = ly.d_out;
+    const uint32_t rows = (uint32_t)((ly.d_out + 15) / 16 * 16);
+    rc = make_map3(&st->head_shadow, false, c->shadow + ly.w_off, din, dout, N, din * 2, (uint64_t)c->m_pad * 2, 64, rows, err);
+    if (rc == PRSGD_OK) rc = make_map3(&st->head_master, true, c->params + ly.w_off, din, dout, N, din * 4, (uint64_t)c->m_pad * 4, 32, rows, err);
+    st->head_rows = (int)rows;
+  }
   if (rc != PRSGD_OK) { delete st; return rc; }
   cudaError_t e = cudaSuccess;
   const int big = (int)stream_smem_bytes(c->B);
@@ -1991,6 +2007,9 @@ inline int tc_create(prsgd_ctx* c, std::string* err) {
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_next_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdNextCfg<64, false>::smem(c->B));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_next_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdNextCfg<128, false>::smem(c->B));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_next_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdNextCfg<64, true>::smem(c->B));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_common_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCommonCfg::smem(c->B));
+  if (e == cudaSuccess && st->head_rows > 0)
+    e = cudaFuncSetAttribute(tc_head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)head_smem_bytes(c->B, st->head_rows));
   if (e != cudaSuccess) {
     *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e);
     delete st;
@@ -2069,6 +2088,35 @@ inline void tc_launch_forward(prsgd_ctx* c, int l, const DrawArgs& dr, const uin
     launch_pdl(tc_stream_kernel<TC_FWD_LINEAR>, grid, kStreamThreads, smem, c->stream, st->layer[l - 1].shadow_k, st->layer[l - 1].act_in, a);
 }
 
+// The class layer's forward GEMM, softmax-CE gradient, step and dZ of the layer below as one launch of
+// clusters (tc_head_kernel): plain SGD step, at most 128 classes, d_{L-1} = 128 x {1, 2, 4, 8}, and the
+// options that the two launches it replaces depend on left at their defaults.  One CTA per (worker, 128
+// features) runs its code once, from a cold instruction cache: that pays while all CTAs are resident at the
+// same time (one wave); with more workers the persistent kernels, whose CTAs walk several items, are faster
+// (64 workers x 8 slices: 68 us against 39 us), unless PRSGD_OPT_HEAD_KERNEL = 2 asks for it regardless.
+inline bool tc_head_applies(const prsgd_ctx* c) {
+  if (c->head_kernel == 0 || c->L < 2 || !tc_epilogues_fused(c) || c->dx_in_update != 1 || c->velocity != nullptr) return false;
+  const TcState* st = static_cast<const TcState*>(c->tc);
+  const int din = c->layer[c->L - 1].d_in;
+  if (st->head_rows == 0 || !(din == 128 || din == 256 || din == 512 || din == 1024)) return false;
+  return c->head_kernel == 2 || (int64_t)c->N * (din / 128) <= (int64_t)st->num_sms;
+}
+
+inline void tc_launch_head(prsgd_ctx* c, const DrawArgs& dr, const uint8_t* active) {
+  TcState* st = static_cast<TcState*>(c->tc);
+  const int L = c->L;
+  const Layer& ly = c->layer[L - 1];
+  HeadArgs a{};
+  a.B = c->B; a.N = c->N; a.C = ly.d_out; a.Cp = st->head_rows; a.gamma = c->gamma; a.draw = dr; a.active = active; a.status = c->status;
+  a.prefetch = (active == nullptr && c->early_loads) ? 1 : 0;
+  a.bias_rw = c->params + ly.b_off; a.bias_lo_rw = c->params + c->layer[L - 2].b_off; a.bias_stride = c->m_pad;
+  a.Y = c->Y; a.P = c->P; a.row_losses = c->losses; a.draws = c->draws;
+  a.out_bk = c->buf.delta_bk[L - 1]; a.ld_out = c->buf.ld[L - 1];
+  const unsigned cl = (unsigned)(ly.d_in / 128);
+  launch_pdl_cluster(tc_head_kernel, dim3(cl, (unsigned)c->N), dim3(kHeadThreads), head_smem_bytes(c->B, st->head_rows), c->stream, cl,
+                     st->head_shadow, st->layer[L - 1].act_in, st->head_master, a);
+}
+
 // The per-worker flags the launches being enqueued honour: Algorithm 3's mask, or the mask of a worker group.
 inline const uint8_t* worker_mask(const prsgd_ctx* c) {
   if (c->group_active != nullptr) return c->group_active;
@@ -2076,23 +2124,23 @@ inline const uint8_t* worker_mask(const prsgd_ctx* c) {
 }
 
 // forward GEMMs of layers l_first..L as one launch (tc_forward_chain_kernel)
-inline bool tc_chain_applies(const prsgd_ctx* c, int l_first) {
-  const int n_seg = c->L - l_first + 1;
+inline bool tc_chain_applies(const prsgd_ctx* c, int l_first, int l_last) {
+  const int n_seg = l_last - l_first + 1;
   return c->forward_chain != 0 && n_seg >= 2 && n_seg <= kChainMax && c->group_active == nullptr;   // (its counters serve one chain at a time)
 }
 
-inline void tc_launch_forward_chain(prsgd_ctx* c, int l_first, const DrawArgs& dr, const uint8_t* active) {
+inline void tc_launch_forward_chain(prsgd_ctx* c, int l_first, int l_last, const DrawArgs& dr, const uint8_t* active) {
   TcState* st = static_cast<TcState*>(c->tc);
   ChainMaps maps;
   ChainArgs a{};
-  a.B = c->B; a.N = c->N; a.n_seg = c->L - l_first + 1;
+  a.B = c->B; a.N = c->N; a.n_seg = l_last - l_first + 1;
   a.shared_w = tc_shared_restart(c, active) ? 1 : 0;
-  a.softmax = tc_epilogues_fused(c) ? 1 : 0;
+  a.softmax = (l_last == c->L && tc_epilogues_fused(c)) ? 1 : 0;
   a.stages = stream_stages(c->B, a.softmax != 0);
   a.draw = dr; a.active = active; a.status = c->status; a.bias_stride = c->m_pad;
   a.ready = c->chain_ready; a.done = c->chain_ready + (size_t)kChainMax * c->N;
   int items = 0;
-  for (int l = l_first; l <= c->L; ++l) {
+  for (int l = l_first; l <= l_last; ++l) {
     const Layer& ly = c->layer[l - 1];
     ChainSeg& g = a.seg[l - l_first];
     g.k_steps = (ly.d_in / 64 + 1) / 2; g.tiles_m = (ly.d_out + 127) / 128; g.M_total = ly.d_out; g.ld_out = c->buf.ld[l];
@@ -2249,6 +2297,25 @@ inline void tc_launch_update_next(prsgd_ctx* c, const DrawArgs& dr) {
   else tc_launch_update_next_tn<64, false>(c, dr);
 }
 
+// Fused update + average of layer l from a common starting point: one weight-gradient GEMM over the minibatches
+// of all workers (tc_update_common_kernel).
+inline void tc_launch_update_common(prsgd_ctx* c, int l, const DrawArgs& dr) {
+  TcState* st = static_cast<TcState*>(c->tc);
+  const Layer& ly = c->layer[l - 1];
+  UpdateCommonArgs a{};
+  a.B = c->B; a.N = c->N; a.tiles_m = (ly.d_out + 127) / 128; a.tiles_n = (ly.d_in + 63) / 64;
+  a.gamma = c->gamma; a.pool = l == 1; a.draw = dr; a.status = c->status;
+  a.prefetch = c->early_loads ? 1 : 0;
+  a.divisor = c->avg_divisor > 0.f ? c->avg_divisor : (float)c->N;
+  a.stages = UpdCommonCfg::stages(c->B);
+  const int items = a.tiles_m * a.tiles_n;
+  const int grid = items < st->num_sms ? items : st->num_sms;
+  const TcLayerMaps& mp = st->layer[l - 1];
+  a.params = c->params + ly.w_off; a.shadow = c->shadow + ly.w_off; a.m_pad = c->m_pad; a.d_in = ly.d_in; a.d_out = ly.d_out;
+  launch_pdl(tc_update_common_kernel, dim3(grid), kUpdCommonThreads, UpdCommonCfg::smem(c->B), c->stream, mp.delta_out, mp.act_in,
+             mp.master, a);
+}
+
 // Tile width: forced by PRSGD_OPT_UPDATE_TILE, else chosen per launch.  Wide tiles need fewer TMA
 // operations per byte and win when every SM has a long queue of them; narrow tiles give four
 // pipeline stages and twice as many work items, which wins on small stores and on the fused form,
@@ -2258,6 +2325,10 @@ inline void tc_launch_update(prsgd_ctx* c, int l, const DrawArgs& dr, const uint
   const Layer& ly = c->layer[l - 1];
   if (c->velocity != nullptr) {            // momentum step: 64-wide tiles (two stages of master + momentum + output)
     tc_launch_update_tn<64, true>(c, l, dr, active, fuse);
+    return;
+  }
+  if (fuse && c->common_point != 0 && tc_shared_restart(c, active)) {   // every worker starts this step from the same point
+    tc_launch_update_common(c, l, dr);
     return;
   }
   int tile = c->upd_tile;

@@ -300,12 +300,16 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging, bool more_follow) {
   const bool next_fwd = c->next_forward && more_follow && !averaging && L > 1 && tc_epilogues_fused(c);
   const bool skip_f1 = c->a1_ready;
   c->a1_ready = false;
-  if (tc_chain_applies(c, skip_f1 ? 2 : 1)) {          // every remaining layer's forward GEMM in one launch
+  // The class layer as one launch of clusters (logits, softmax-CE gradient, step of W_L, dZ_{L-1}): whenever its
+  // step is the plain one (a class layer large enough for the fused update + average keeps the separate launches).
+  const bool head = tc_head_applies(c) && !(fuse && tc_layer_fuses_average(c, L));
+  const int l_fwd_last = head ? L - 1 : L;
+  if (tc_chain_applies(c, skip_f1 ? 2 : 1, l_fwd_last)) {          // every remaining layer's forward GEMM in one launch
     prof_begin(c, PRSGD_KERNEL_FORWARD);
-    tc_launch_forward_chain(c, skip_f1 ? 2 : 1, dr, act_mask);
+    tc_launch_forward_chain(c, skip_f1 ? 2 : 1, l_fwd_last, dr, act_mask);
     LAUNCH_CHECK(c);
   } else {
-    for (int l = skip_f1 ? 2 : 1; l <= L; ++l) {
+    for (int l = skip_f1 ? 2 : 1; l <= l_fwd_last; ++l) {
       prof_begin(c, PRSGD_KERNEL_FORWARD);
       tc_launch_forward(c, l, dr, act_mask);
       LAUNCH_CHECK(c);
@@ -329,9 +333,16 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging, bool more_follow) {
   // Layers >= 2 whose update is the plain SGD step: one launch forms dZ_{l-1} and applies the step of W_l (the
   // fused update + average of an averaging iteration owns a tile across workers instead and keeps dX separate).
   const bool dx_in_upd = c->dx_in_update && tc_epilogues_fused(c);
+  if (head) {
+    prof_begin(c, PRSGD_KERNEL_HEAD);
+    tc_launch_head(c, dr, act_mask);
+    LAUNCH_CHECK(c);
+  }
   for (int l = L; l >= 1; --l) {          // dX_l reads W_l before the update of layer l overwrites it
     const bool fuse_l = fuse && tc_layer_fuses_average(c, l);
-    if (l > 1 && dx_in_upd && !fuse_l && (c->dx_in_update == 2 || tc_layer_folds_dx(c, l))) {
+    if (l == L && head) {
+      // (forward, step and dZ_{L-1} of this layer were the head launch)
+    } else if (l > 1 && dx_in_upd && !fuse_l && (c->dx_in_update == 2 || tc_layer_folds_dx(c, l))) {
       prof_begin(c, PRSGD_KERNEL_UPDATE);
       tc_launch_update_dx(c, l);
       LAUNCH_CHECK(c);
@@ -713,7 +724,7 @@ void period_key(const prsgd_ctx* c, uint64_t (&key)[13]) {
   key[7] = (uint64_t)c->average_velocity; key[8] = reinterpret_cast<uint64_t>(c->X);
   key[9] = reinterpret_cast<uint64_t>(c->Y); key[10] = (uint64_t)c->worker0; key[11] = (uint64_t)c->fused_epilogues | ((uint64_t)c->early_loads << 1) | ((uint64_t)c->next_forward << 2) | ((uint64_t)c->dx_in_update << 3);
   key[12] = (c->rows_identical ? 1u : 0u) | ((uint64_t)c->shared_restart << 1) | ((uint64_t)c->forward_chain << 2) |
-            ((uint64_t)c->worker_groups << 3) | ((uint64_t)c->dx_shared_pair << 6);   // the period's first iteration may share reads
+            ((uint64_t)c->worker_groups << 3) | ((uint64_t)c->dx_shared_pair << 6) | ((uint64_t)c->head_kernel << 7) | ((uint64_t)c->common_point << 9);   // the period's first iteration may share reads
 }
 
 // One whole averaging period (I iterations starting right after an average) as a CUDA graph: the
@@ -1119,6 +1130,12 @@ int prsgd_set_option(prsgd_ctx* c, int32_t option, int64_t value) {
   if (option == PRSGD_OPT_SHARED_RESTART) { c->shared_restart = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_FORWARD_CHAIN) { c->forward_chain = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_DX_SHARED_PAIR) { c->dx_shared_pair = value != 0; return PRSGD_OK; }
+  if (option == PRSGD_OPT_COMMON_POINT) { c->common_point = value != 0; return PRSGD_OK; }
+  if (option == PRSGD_OPT_HEAD_KERNEL) {
+    if (value < 0 || value > 2) return fail(c, PRSGD_ERR_ARG, "PRSGD_OPT_HEAD_KERNEL takes 0, 1 or 2");
+    c->head_kernel = (int)value;
+    return PRSGD_OK;
+  }
   if (option == PRSGD_OPT_WORKER_GROUPS) {
     if (value < 1 || value > kMaxGroups) return fail(c, PRSGD_ERR_ARG, "PRSGD_OPT_WORKER_GROUPS takes 1..4");
     // group g holds the contiguous workers [g N / G, (g + 1) N / G)

@@ -56,6 +56,21 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
+// The same for a grid of thread-block clusters of `cluster_x` CTAs along x (grid.x a multiple of it).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                      unsigned cluster_x, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = cluster_x; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+  cfg.attrs = attr; cfg.numAttrs = 2;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 constexpr int kMaxGroups = 4;
 constexpr int64_t kSegAlign = 32;  // every segment of a row starts at a multiple of 32 elements
 
@@ -97,6 +112,8 @@ struct prsgd_ctx {
   int average_velocity = 0;      // average the buffers together with the models
   int upd_tile = 0;              // column width of the update kernel's tile: 0 = chosen per launch, 64 or 128
   int dx_shared_pair = 1;        // 64-wide update + dX: one pair of bf16 tiles behind the stages (more stages) instead of one per stage
+  int common_point = 1;          // fused update + average from a common starting point: one GEMM over all workers' minibatches
+  int head_kernel = 1;           // the class layer's forward, softmax-CE gradient, step and dZ below it as one launch of clusters
   int dx_in_update = 1;          // layers >= 2: the update launch also forms dZ of the layer below (tensor-core path)
   int next_forward = 1;          // layer 1's update also forms a_1 of the next iteration (tensor-core path)
   bool a1_ready = false;         // a_1 of the coming iteration has already been formed by the previous update

@@ -78,20 +78,30 @@ def test_byte_model_follows_the_launch_rules():
     library counts on the GPU (125 update launches per cfg4 period, ...), and the shared restart, the folding and
     the momentum options move the bytes the way the kernels do."""
     cfg4 = synth.WORKLOADS["cfg4"]
-    f = bench.period_bytes(cfg4, 8496384)
+    assert bench.period_bytes(cfg4, 8496384)["head"][1] == 0       # 64 workers x 8 slices: more than one wave, not used
+    h = bench.period_bytes(cfg4, 8496384, head_kernel=2)   # the class layer as one launch of its own family
+    assert {k: v[1] for k, v in h.items() if v[1]} == {"forward": 65, "dx": 2, "update": 93, "update_average": 3,
+                                                         "average": 1, "misc": 1, "head": 32}
+    f = bench.period_bytes(cfg4, 8496384, head_kernel=0)
     assert {k: v[1] for k, v in f.items() if v[1]} == {"forward": 97, "dx": 2, "update": 125, "update_average": 3,
                                                          "average": 1, "misc": 1}
+    assert sum(v[0] for v in f.values()) - sum(v[0] for v in h.values()) == (
+        32 * 64 * (100 * 4 + 32 * 100 * 4 + 32 * (100 + 1024) * 2)      # no bias re-read, no fp32 logits, operands read once
+        - 63 * 100 * 1024 * 2)                             # (its first iteration reads every worker's own copy of W_L)
     plain = 64 * 8496228                                   # parameters of all workers
     per_iter = f["update"][0] / 31.25                      # 125 launches = 31 plain iterations + the class layer's 32nd
     assert 9.0 * plain < per_iter < 10.2 * plain           # ~10 B/param, minus the bf16 copy of W_1 that is not written
+    assert 9.0 * plain < h["update"][0] / 31 + h["head"][0] / 32 < 10.2 * plain
     g = bench.period_bytes(cfg4, 8496384, momentum=True)
     assert g["update"][0] > f["update"][0] + 7.5 * plain * 31 and g["update_average"][1] == 3
     c3 = synth.WORKLOADS["cfg3"].with_(I=1)
     shared, own = bench.period_bytes(c3, 4206656), bench.period_bytes(c3, 4206656, shared_restart=False)
     assert shared["forward"][0] * 5 < own["forward"][0] and shared["update_average"][0] < own["update_average"][0]
     assert own["update_average"][0] - shared["update_average"][0] == 15 * (3072 * 1024 + 1024 * 1024) * 4
-    c16 = bench.period_bytes(synth.WORKLOADS["cfg3"].with_(I=16), 4206656)
+    c16 = bench.period_bytes(synth.WORKLOADS["cfg3"].with_(I=16), 4206656, head_kernel=0)
     assert c16["forward"][1] == 33 and c16["dx"][1] == 16 and c16["update"][1] == 46
+    c16 = bench.period_bytes(synth.WORKLOADS["cfg3"].with_(I=16), 4206656)
+    assert c16["forward"][1] == 17 and c16["dx"][1] == 16 and c16["update"][1] == 30 and c16["head"][1] == 16
     assert bench.period_bytes(synth.WORKLOADS["cfg3"].with_(I=16), 4206656, forward_chain=True)["forward"][1] == 16
     f32 = bench.period_bytes(synth.WORKLOADS["cfg2"], 669728)
     assert f32["forward"][1] == 24 and f32["softmax"][1] == 8 and f32["update_average"][1] == 3
