@@ -343,6 +343,15 @@ int prsgd_get_velocity_stacked(prsgd_ctx* ctx, float* dst, int dst_on_device);
  * Equal to update-then-average up to fp32 rounding, not bit for bit; deterministic.  0: the N stepped models are
  * formed and summed one by one. */
 #define PRSGD_OPT_COMMON_POINT 15
+/* PRSGD_OPT_SPLIT_BLOCKS (default 0, tensor-core path, no worker mask): the update launch of layer 1 that also forms
+ * the next a_1 walks row blocks of 128 output features, whole blocks per CTA.  1: their column tiles are dealt out
+ * in equal runs, one per SM, whenever whole blocks would leave SMs idle or in a short last round (128 blocks on
+ * 148 SMs, 512 blocks = 3.46 rounds) and the launch is large; a row block cut by a run boundary gets its forward
+ * sum from the partial sums of its two or three CTAs, added in run order by whichever finishes last (no CTA waits
+ * for another).  2: also for small launches.  The weights are bit-identical either way; a_1 of a cut row block is
+ * summed in another order (fp32 rounding) and is deterministic.  Off by default: the launch is bound by the
+ * memory system, not by its longest CTA, and equal runs gained nothing measurable. */
+#define PRSGD_OPT_SPLIT_BLOCKS 16
 /* PRSGD_OPT_CHECK_FINITE (default 0): when 1, prsgd_sync also runs prsgd_check_finite. */
 #define PRSGD_OPT_CHECK_FINITE 9
 int prsgd_set_option(prsgd_ctx* ctx, int32_t option, int64_t value);

@@ -1143,6 +1143,50 @@ __device__ __forceinline__ void momentum_pair(uint8_t* vrow, uint32_t j, uint32_
 // The forward launch of layer 1 in the next iteration is then skipped, and W_1's bf16 shadow, which
 // only that launch reads, is not written (the host uses the ordinary update on the last iteration of
 // a call, so the shadow is valid whenever control returns to the caller).
+// The (block, first tile, end tile) segments one CTA of a block-walking kernel handles.  A block is a row block
+// of tc_update_next_kernel (its tiles = the column tiles the forward product accumulates over).  Plain form: whole
+// blocks, blockIdx.x, + gridDim.x, ...  Split form: the tiles of all blocks, in block-major order, are cut into
+// runs of `chunk` tiles, one run per CTA, so every CTA streams the same number of tiles however the block count
+// divides by the CTA count; a block cut by a run boundary is finished by whichever of its CTAs comes last
+// (see SplitArgs).
+struct BlockWalk {
+  int tn, split, nblocks, stride;
+  int64_t t, t1;
+  int rb, k0, k1;
+  __device__ BlockWalk(int tiles_per_block, int blocks, int split_, int chunk)
+      : tn(tiles_per_block), split(split_), nblocks(blocks), stride((int)gridDim.x), rb((int)blockIdx.x - (int)gridDim.x), k0(0), k1(0) {
+    t = (int64_t)blockIdx.x * chunk;
+    t1 = t + chunk;
+    const int64_t all = (int64_t)blocks * tiles_per_block;
+    if (t1 > all) t1 = all;
+  }
+  __device__ bool next() {
+    if (split) {
+      if (t >= t1) return false;
+      rb = (int)(t / tn);
+      k0 = (int)(t - (int64_t)rb * tn);
+      k1 = (int64_t)k0 + (t1 - t) < (int64_t)tn ? k0 + (int)(t1 - t) : tn;
+      t += k1 - k0;
+      return true;
+    }
+    rb += stride; k0 = 0; k1 = tn;
+    return rb < nblocks;
+  }
+  __device__ bool whole() const { return k0 == 0 && k1 == tn; }
+};
+
+// Split form: a CTA that holds only part of a block's accumulator writes it, as fp32, to a slot of its own in
+// global memory (slot 2 c for the first segment of CTA c, 2 c + 1 for a later one: a run has at most one cut
+// block at each end), raises the block's counter, and the CTA that finds the counter complete adds the parts in
+// run order, applies the block epilogue and zeroes the counter again.  Nobody waits for anybody, and the order of
+// the additions is fixed, so the result does not depend on which CTA comes last.
+struct SplitArgs {
+  int on;                    // 0: whole blocks per CTA
+  int chunk;                 // tiles per CTA
+  float* part;               // [2 * CTAs][B][128] fp32
+  unsigned int* count;       // [blocks], zero between launches
+};
+
 struct UpdateNextArgs {
   int B, N;
   int tiles_m, tiles_n;
@@ -1157,6 +1201,7 @@ struct UpdateNextArgs {
   int M_total;               // d_1
   float mu;                  // momentum form: v <- mu v + G, x <- x - gamma v
   const uint8_t* active;     // per-worker flag or nullptr: an inactive worker's row blocks are skipped
+  SplitArgs split;           // row blocks cut at run boundaries (never together with a worker mask)
 };
 
 template <int TN, bool MOM> struct UpdNextCfg {
@@ -1250,7 +1295,9 @@ __global__ void __launch_bounds__(kUpdBlkThreads, 1) tc_update_next_kernel(const
     // ---------------- loader
     uint32_t it = 0, rbi = 0;
     bool ok = true;
-    for (int rb = blockIdx.x; rb < total_rb && ok; rb += gridDim.x) {
+    BlockWalk wk(a.tiles_n, total_rb, a.split.on, a.split.chunk);
+    while (ok && wk.next()) {
+      const int rb = wk.rb;
       const int n = rb / a.tiles_m, m0 = (rb % a.tiles_m) * 128;
       if (!item_active(n)) continue;
       const int64_t t = draw_t(a.draw);
@@ -1265,7 +1312,7 @@ __global__ void __launch_bounds__(kUpdBlkThreads, 1) tc_update_next_kernel(const
         tma_load_3d(dz_u32(q) + op_box, &mapDelta, dz_full(q), m0 + 64, 0, n);
         ++rbi;
       }
-      for (int kb = 0; kb < a.tiles_n; ++kb, ++it) {
+      for (int kb = wk.k0; kb < wk.k1; ++kb, ++it) {
         const int s = it % S;
         const uint32_t ph = (it / S) & 1u;
         ok = mbar_wait(stage_empty(s), ph ^ 1u, abort_flag, a.status, 0x401);
@@ -1309,10 +1356,11 @@ __global__ void __launch_bounds__(kUpdBlkThreads, 1) tc_update_next_kernel(const
     bool ok = true;
     bool have_prev = false;
     uint32_t p_it = 0, p_rbi = 0;
-    int p_kb = 0;
-    auto forward_of = [&](uint32_t j, int kb, uint32_t rj) -> bool {
+    bool p_first = false, p_last = false;
+    // forward product of tile j; `first` / `last`: the tile opens / closes its segment of the row block
+    auto forward_of = [&](uint32_t j, bool first, bool last, uint32_t rj) -> bool {
       const int s = j % S, q = rj & 1;
-      if (kb == 0 && !mbar_wait(facc_empty(q), ((rj >> 1) & 1u) ^ 1u, abort_flag, a.status, 0x402)) return false;
+      if (first && !mbar_wait(facc_empty(q), ((rj >> 1) & 1u) ^ 1u, abort_flag, a.status, 0x402)) return false;
       if (!mbar_wait(tile_ready(s), (j / S) & 1u, abort_flag, a.status, 0x403)) return false;
       tc_fence_after();
       const uint32_t acc = tmem + kFwdCol + (uint32_t)(q * a.B);
@@ -1321,19 +1369,20 @@ __global__ void __launch_bounds__(kUpdBlkThreads, 1) tc_update_next_kernel(const
 #pragma unroll
         for (int k = 0; k < 4; ++k)
           mma_bf16(acc, smem_desc_sw128(ops_u32(s) + h * 16384u + k * 32u, 16u, 1024u),
-                   smem_desc_sw128(next_u32(s) + h * op_box + k * 32u, 16u, 1024u), idesc_fw, (kb | h | k) != 0 ? 1u : 0u);
+                   smem_desc_sw128(next_u32(s) + h * op_box + k * 32u, 16u, 1024u), idesc_fw, (!first || (h | k) != 0) ? 1u : 0u);
       }
       mma_commit(fwd_done(s));
-      if (kb == a.tiles_n - 1) mma_commit(facc_full(q));
+      if (last) mma_commit(facc_full(q));
       return true;
     };
-    for (int rb = blockIdx.x; rb < total_rb && ok; rb += gridDim.x) {
-      if (!item_active(rb / a.tiles_m)) continue;
-      for (int kb = 0; kb < a.tiles_n && ok; ++kb, ++it) {
+    BlockWalk wk(a.tiles_n, total_rb, a.split.on, a.split.chunk);
+    while (ok && wk.next()) {
+      if (!item_active(wk.rb / a.tiles_m)) continue;
+      for (int kb = wk.k0; kb < wk.k1 && ok; ++kb, ++it) {
         const int s = it % S;
         const uint32_t ph = (it / S) & 1u;
         const int dq = rbi & 1;
-        if (kb == 0) {
+        if (kb == wk.k0) {
           ok = mbar_wait(dz_full(dq), (rbi >> 1) & 1u, abort_flag, a.status, 0x40C);
           if (!ok) break;
         }
@@ -1346,22 +1395,24 @@ __global__ void __launch_bounds__(kUpdBlkThreads, 1) tc_update_next_kernel(const
           mma_bf16(tmem + (uint32_t)(s * TN), smem_desc_sw128(sa + k * 2048u, op_box, 1024u),
                    smem_desc_sw128(sb + k * 2048u, op_box, 1024u), idesc_dw, k != 0 ? 1u : 0u);
         mma_commit(acc_full(s));
-        if (kb == a.tiles_n - 1) mma_commit(dz_empty(dq));      // the block's dZ boxes are free once these products are done
-        if (have_prev) ok = forward_of(p_it, p_kb, p_rbi);
-        p_it = it; p_kb = kb; p_rbi = rbi; have_prev = true;
+        if (kb == wk.k1 - 1) mma_commit(dz_empty(dq));          // the block's dZ boxes are free once these products are done
+        if (have_prev) ok = forward_of(p_it, p_first, p_last, p_rbi);
+        p_it = it; p_first = kb == wk.k0; p_last = kb == wk.k1 - 1; p_rbi = rbi; have_prev = true;
       }
-      ++rbi;                                              // counts the row blocks actually walked
+      ++rbi;                                              // counts the segments actually walked
     }
-    if (ok && have_prev) forward_of(p_it, p_kb, p_rbi);
+    if (ok && have_prev) forward_of(p_it, p_first, p_last, p_rbi);
   } else if (warp == 2 && lane == 0) {
     // ---------------- storer: TMA stores of finished tiles; the stage goes back to the loader once the
     // forward MMAs have consumed its bf16 tile too
     uint32_t it = 0;
     bool ok = true;
-    for (int rb = blockIdx.x; rb < total_rb && ok; rb += gridDim.x) {
+    BlockWalk wk(a.tiles_n, total_rb, a.split.on, a.split.chunk);
+    while (ok && wk.next()) {
+      const int rb = wk.rb;
       const int n = rb / a.tiles_m, m0 = (rb % a.tiles_m) * 128;
       if (!item_active(n)) continue;
-      for (int kb = 0; kb < a.tiles_n; ++kb, ++it) {
+      for (int kb = wk.k0; kb < wk.k1; ++kb, ++it) {
         const int s = it % S;
         const uint32_t ph = (it / S) & 1u;
         const int n0 = kb * TN;
@@ -1390,9 +1441,10 @@ __global__ void __launch_bounds__(kUpdBlkThreads, 1) tc_update_next_kernel(const
     const uint32_t sw = (uint32_t)(r & 7);
     uint32_t it = 0;
     bool ok = true;
-    for (int rb = blockIdx.x; rb < total_rb && ok; rb += gridDim.x) {
-      if (!item_active(rb / a.tiles_m)) continue;
-      for (int kb = 0; kb < a.tiles_n; ++kb, ++it) {
+    BlockWalk wk(a.tiles_n, total_rb, a.split.on, a.split.chunk);
+    while (ok && wk.next()) {
+      if (!item_active(wk.rb / a.tiles_m)) continue;
+      for (int kb = wk.k0; kb < wk.k1; ++kb, ++it) {
         const int s = it % S;
         const uint32_t ph = (it / S) & 1u;
         ok = mbar_wait(full_w(s), ph, abort_flag, a.status, 0x408) &&
@@ -1442,7 +1494,11 @@ __global__ void __launch_bounds__(kUpdBlkThreads, 1) tc_update_next_kernel(const
     const int batches = a.B / 16;
     uint32_t rbi = 0;
     bool ok = true;
-    for (int rb = blockIdx.x; rb < total_rb && ok; rb += gridDim.x) {
+    const int etid = tid - 224;                           // 0..127 among these warps
+    volatile unsigned int* last_flag = reinterpret_cast<volatile unsigned int*>(gen + (bar0 - base) + 264);
+    BlockWalk wk(a.tiles_n, total_rb, a.split.on, a.split.chunk);
+    while (ok && wk.next()) {
+      const int rb = wk.rb;
       const int n = rb / a.tiles_m, m = (rb % a.tiles_m) * 128 + r;
       if (!item_active(n)) continue;
       const int q = rbi & 1;
@@ -1451,18 +1507,63 @@ __global__ void __launch_bounds__(kUpdBlkThreads, 1) tc_update_next_kernel(const
       ok = __all_sync(0xffffffffu, mbar_wait(facc_full(q), (rbi >> 1) & 1u, abort_flag, a.status, 0x40A));
       if (!ok) break;
       tc_fence_after();
-      for (int bi = 0; bi < batches; ++bi) {
-        uint32_t v[16];
-        tmem_ld16(tmem + lane_off + kFwdCol + (uint32_t)(q * a.B + bi * 16), v);
-        tmem_ld_wait();
-        if (valid) {
+      if (wk.whole()) {
+        for (int bi = 0; bi < batches; ++bi) {
+          uint32_t v[16];
+          tmem_ld16(tmem + lane_off + kFwdCol + (uint32_t)(q * a.B + bi * 16), v);
+          tmem_ld_wait();
+          if (valid) {
 #pragma unroll
-          for (int j = 0; j < 16; ++j)
-            a.next_out[((int64_t)n * a.B + bi * 16 + j) * a.next_ld + m] = f32_to_bf16_rn(fmaxf(__uint_as_float(v[j]) + bias, 0.f));
+            for (int j = 0; j < 16; ++j)
+              a.next_out[((int64_t)n * a.B + bi * 16 + j) * a.next_ld + m] = f32_to_bf16_rn(fmaxf(__uint_as_float(v[j]) + bias, 0.f));
+          }
         }
+        tc_fence_before();
+        mbar_arrive(facc_empty(q));
+      } else {
+        // part of a row block: this CTA's share of z_1 goes to its slot; whoever completes the block's counter
+        // adds the shares in run order and applies bias and ReLU
+        float* mine = a.split.part + ((int64_t)(2 * blockIdx.x + (rbi == 0 ? 0 : 1)) * a.B) * 128 + r;
+        for (int bi = 0; bi < batches; ++bi) {
+          uint32_t v[16];
+          tmem_ld16(tmem + lane_off + kFwdCol + (uint32_t)(q * a.B + bi * 16), v);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 16; ++j) __stcg(mine + (bi * 16 + j) * 128, __uint_as_float(v[j]));
+        }
+        tc_fence_before();
+        mbar_arrive(facc_empty(q));
+        __threadfence();
+        named_bar_sync(2, 128);
+        const int64_t tb = (int64_t)rb * a.tiles_n;          // first tile of the block in the global order
+        const int c_first = (int)(tb / a.split.chunk), c_last = (int)((tb + a.tiles_n - 1) / a.split.chunk);
+        if (etid == 0) *last_flag = atomicAdd(a.split.count + rb, 1u) == (unsigned int)(c_last - c_first) ? 1u : 0u;
+        named_bar_sync(2, 128);
+        if (*last_flag != 0u) {
+          __threadfence();
+          for (int b0 = 0; b0 < a.B; b0 += 16) {             // sixteen rows at a time: their loads are in flight together
+            float z[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) z[j] = 0.f;
+            for (int cc = c_first; cc <= c_last; ++cc) {     // CTA cc's segment of this block is its first one unless its run began earlier
+              const int slot = 2 * cc + ((int64_t)cc * a.split.chunk < tb ? 1 : 0);
+              const float* src = a.split.part + ((int64_t)slot * a.B + b0) * 128 + r;
+              float v[16];
+#pragma unroll
+              for (int j = 0; j < 16; ++j) v[j] = __ldcg(src + j * 128);
+#pragma unroll
+              for (int j = 0; j < 16; ++j) z[j] += v[j];
+            }
+            if (valid) {
+#pragma unroll
+              for (int j = 0; j < 16; ++j)
+                a.next_out[((int64_t)n * a.B + b0 + j) * a.next_ld + m] = f32_to_bf16_rn(fmaxf(z[j] + bias, 0.f));
+            }
+          }
+          if (etid == 0) a.split.count[rb] = 0u;
+        }
+        named_bar_sync(2, 128);                             // (the flag is read by all before the next block overwrites it)
       }
-      tc_fence_before();
-      mbar_arrive(facc_empty(q));
       ++rbi;
     }
   }
@@ -2262,6 +2363,30 @@ inline void tc_launch_update_dx(prsgd_ctx* c, int l) {
   else tc_launch_update_dx_m<64, false, false>(c, l);
 }
 
+// Whether a block-walking launch of `blocks` blocks of `tn` tiles runs in its split form (PRSGD_OPT_SPLIT_BLOCKS,
+// off by default), and with what run length: only without a worker mask, only when equal runs shorten the longest
+// CTA's walk by 5 % or more, and (unless the option says 2) only for launches of at least eight tiles per SM.
+// Measured: layer 1 of a 16-worker 3072-1024 net (128 row blocks on 148 SMs) 121 us split, 119 us whole; of a
+// 64-worker 1024-2048 net (3.46 rounds of blocks) within 0.5 %: the launch is bound by the memory system, which
+// the remaining CTAs of a short last round saturate just as well.
+inline SplitArgs tc_split_plan(const prsgd_ctx* c, int64_t blocks, int tn, const uint8_t* active, int* grid) {
+  const TcState* st = static_cast<const TcState*>(c->tc);
+  SplitArgs sp{};
+  sp.part = c->split_part; sp.count = c->split_count;
+  const int64_t tiles = blocks * tn;
+  const int g_whole = blocks < st->num_sms ? (int)blocks : st->num_sms;
+  *grid = g_whole;
+  if (c->split_blocks == 0 || active != nullptr || st->num_sms > kSplitMaxCtas || blocks <= 0) return sp;
+  const int g = tiles < st->num_sms ? (int)tiles : st->num_sms;
+  const int64_t chunk = (tiles + g - 1) / g;
+  const int64_t whole_walk = (blocks + g_whole - 1) / g_whole * tn;
+  const bool pays = 20 * chunk <= 19 * whole_walk && (c->split_blocks == 2 || tiles >= 8 * (int64_t)st->num_sms);
+  if (!pays) return sp;
+  sp.on = 1; sp.chunk = (int)chunk;
+  *grid = (int)((tiles + chunk - 1) / chunk);
+  return sp;
+}
+
 // Update of layer 1 that also forms a_1 of the next iteration (tc_update_next_kernel).
 template <int TN, bool MOM>
 inline void tc_launch_update_next_tn(prsgd_ctx* c, const DrawArgs& dr) {
@@ -2274,8 +2399,8 @@ inline void tc_launch_update_next_tn(prsgd_ctx* c, const DrawArgs& dr) {
   a.stages = UpdNextCfg<TN, MOM>::stages(c->B);
   a.next_out = c->buf.act_bk[1]; a.next_ld = c->buf.ld[1];
   a.bias = c->params + ly.b_off; a.bias_stride = c->m_pad; a.M_total = ly.d_out;
-  const int items = a.tiles_m * c->N;
-  const int grid = items < st->num_sms ? items : st->num_sms;
+  int grid = 1;
+  a.split = tc_split_plan(c, (int64_t)a.tiles_m * c->N, a.tiles_n, a.active, &grid);
   const TcLayerMaps& mp = st->layer[0];
   launch_pdl(tc_update_next_kernel<TN, MOM>, dim3(grid), kUpdBlkThreads, UpdNextCfg<TN, MOM>::smem(c->B), c->stream, mp.delta_out,
              mp.act_in, mp.master, MOM ? mp.velocity : mp.master, a);

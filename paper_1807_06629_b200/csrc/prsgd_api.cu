@@ -142,6 +142,15 @@ size_t carve_scratch(int N, const prsgd_model_spec* s, int64_t m_pad, prsgd_ctx*
       }
     }
   } else {
+    // split blocks of the folded update kernels: two fp32 slots of [B][128] per CTA and a counter per block
+    int wmax = 1;
+    for (int l = 0; l <= L; ++l) wmax = s->dims[l] > wmax ? s->dims[l] : wmax;
+    auto spart = take(sizeof(float) * 2 * (size_t)kSplitMaxCtas * B * 128);
+    auto scount = take(sizeof(unsigned int) * (size_t)N * ((wmax + 63) / 64));
+    if (ctx) {
+      ctx->split_part = reinterpret_cast<float*>(spart);
+      ctx->split_count = reinterpret_cast<unsigned int*>(scount);
+    }
     for (int l = 1; l <= L; ++l) {
       const int ld = (int)round_up(s->dims[l], 64);
       const size_t e = (size_t)N * B * ld;
@@ -724,7 +733,7 @@ void period_key(const prsgd_ctx* c, uint64_t (&key)[13]) {
   key[7] = (uint64_t)c->average_velocity; key[8] = reinterpret_cast<uint64_t>(c->X);
   key[9] = reinterpret_cast<uint64_t>(c->Y); key[10] = (uint64_t)c->worker0; key[11] = (uint64_t)c->fused_epilogues | ((uint64_t)c->early_loads << 1) | ((uint64_t)c->next_forward << 2) | ((uint64_t)c->dx_in_update << 3);
   key[12] = (c->rows_identical ? 1u : 0u) | ((uint64_t)c->shared_restart << 1) | ((uint64_t)c->forward_chain << 2) |
-            ((uint64_t)c->worker_groups << 3) | ((uint64_t)c->dx_shared_pair << 6) | ((uint64_t)c->head_kernel << 7) | ((uint64_t)c->common_point << 9);   // the period's first iteration may share reads
+            ((uint64_t)c->worker_groups << 3) | ((uint64_t)c->dx_shared_pair << 6) | ((uint64_t)c->head_kernel << 7) | ((uint64_t)c->common_point << 9) | ((uint64_t)c->split_blocks << 10);   // the period's first iteration may share reads
 }
 
 // One whole averaging period (I iterations starting right after an average) as a CUDA graph: the
@@ -1131,6 +1140,11 @@ int prsgd_set_option(prsgd_ctx* c, int32_t option, int64_t value) {
   if (option == PRSGD_OPT_FORWARD_CHAIN) { c->forward_chain = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_DX_SHARED_PAIR) { c->dx_shared_pair = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_COMMON_POINT) { c->common_point = value != 0; return PRSGD_OK; }
+  if (option == PRSGD_OPT_SPLIT_BLOCKS) {
+    if (value < 0 || value > 2) return fail(c, PRSGD_ERR_ARG, "PRSGD_OPT_SPLIT_BLOCKS takes 0, 1 or 2");
+    c->split_blocks = (int)value;
+    return PRSGD_OK;
+  }
   if (option == PRSGD_OPT_HEAD_KERNEL) {
     if (value < 0 || value > 2) return fail(c, PRSGD_ERR_ARG, "PRSGD_OPT_HEAD_KERNEL takes 0, 1 or 2");
     c->head_kernel = (int)value;
@@ -1199,6 +1213,11 @@ int prsgd_clear_device_error(prsgd_ctx* c) {
   CUDA_TRY(c, cudaMemsetAsync(c->status, 0, sizeof(DeviceStatus), c->stream));
   // an interrupted forward chain may have left its counters half way
   CUDA_TRY(c, cudaMemsetAsync(c->chain_ready, 0, sizeof(unsigned int) * ((size_t)kChainMax * c->N + 1), c->stream));
+  if (c->split_count != nullptr) {   // ... and an interrupted split launch the counters of its cut blocks
+    int wmax = 1;
+    for (int l = 0; l <= c->L; ++l) wmax = c->dims[l] > wmax ? c->dims[l] : wmax;
+    CUDA_TRY(c, cudaMemsetAsync(c->split_count, 0, sizeof(unsigned int) * (size_t)c->N * ((wmax + 63) / 64), c->stream));
+  }
   CUDA_TRY(c, cudaStreamSynchronize(c->stream));
   c->err.clear();
   c->rows_identical = false;     // whatever the interrupted launches left

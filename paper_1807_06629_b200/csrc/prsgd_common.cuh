@@ -72,6 +72,7 @@ inline cudaError_t launch_pdl_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 
 }
 
 constexpr int kMaxGroups = 4;
+constexpr int kSplitMaxCtas = 192;  // CTAs of a launch that may each hold two partial accumulators in global memory
 constexpr int64_t kSegAlign = 32;  // every segment of a row starts at a multiple of 32 elements
 
 inline int64_t round_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
@@ -112,6 +113,9 @@ struct prsgd_ctx {
   int average_velocity = 0;      // average the buffers together with the models
   int upd_tile = 0;              // column width of the update kernel's tile: 0 = chosen per launch, 64 or 128
   int dx_shared_pair = 1;        // 64-wide update + dX: one pair of bf16 tiles behind the stages (more stages) instead of one per stage
+  int split_blocks = 0;          // layer 1's update + next forward: row blocks cut at run boundaries so that every CTA streams the same number of tiles
+  float* split_part = nullptr;           // [2 * kSplitMaxCtas][B][128] fp32 partial accumulators
+  unsigned int* split_count = nullptr;   // a counter per block, zero between launches
   int common_point = 1;          // fused update + average from a common starting point: one GEMM over all workers' minibatches
   int head_kernel = 1;           // the class layer's forward, softmax-CE gradient, step and dZ below it as one launch of clusters
   int dx_in_update = 1;          // layers >= 2: the update launch also forms dZ of the layer below (tensor-core path)

@@ -558,6 +558,64 @@ def test_reading_the_common_restart_point_once_changes_no_bit(torch_cuda):
                     assert np.array_equal(grp[0][3], o[3])
 
 
+SPLIT_CASES = [
+    (_w("tc-split-ragged", 2, (192, 320, 100), 32, I=3), None),
+    (_w("tc-split-wide-in", 3, (448, 256, 10), 16, I=4), None),
+    (_w("tc-split-one-block", 1, (1024, 128, 10), 32, I=2), None),
+    (_w("tc-split-b64", 2, (128, 128, 100), 64, I=2), None),
+    (_w("tc-split-mom", 3, (320, 256, 10), 32, I=3), 0.9),
+]
+
+
+@pytest.mark.parametrize("w,mu", SPLIT_CASES, ids=[c[0].name for c in SPLIT_CASES])
+def test_row_blocks_cut_at_run_boundaries(torch_cuda, w, mu):
+    """Layer 1's update + next forward with its column tiles dealt out in equal runs (PRSGD_OPT_SPLIT_BLOCKS = 2
+    forces it on small shapes): a row block cut by a run boundary gets its a_1 from partial sums added in run
+    order by the last of its CTAs.  The step of an iteration does not depend on it (bit-identical weights after
+    the first iteration); later iterations start from an a_1 summed in another order, so they agree to rounding;
+    the form is deterministic (two runs, direct and replayed, same bits), works for both tile widths, and a period
+    meets the oracle's bounds."""
+    torch = torch_cuda
+    from paper_1807_06629_b200 import binding
+    X, Y, x0 = make_inputs(w)
+    x0s = np.tile(x0, (w.N, 1))
+    T = 2 * w.I + 2
+    runs = {}
+    for split, graph, tile in ((0, 0, 0), (2, 0, 0), (2, 1, 0), (2, 0, 64), (2, 0, 128), (2, 0, 0)):
+        with torch.cuda.stream(torch.cuda.Stream()):
+            p = make_ctx(w, X, Y, x0)
+            if mu is not None:
+                p.enable_momentum(mu)
+            p.set_option(binding.OPT_SPLIT_BLOCKS, split)
+            p.set_option(binding.OPT_GRAPH, graph)
+            p.set_option(binding.OPT_UPDATE_TILE, tile)
+            n0 = p.get_launch_count()
+            p.local_steps(2)
+            second = p.get_params_stacked()
+            p.local_steps(T - 2)
+            runs.setdefault((split, graph, tile), []).append(
+                (second, p.get_params_stacked(), p.get_losses(), p.get_draws().tolist(), p.get_launch_count() - n0))
+            torch.cuda.current_stream().synchronize()
+            p.close()
+    off = runs[(0, 0, 0)][0]
+    on = runs[(2, 0, 0)]
+    assert np.array_equal(on[0][1], on[1][1]) and np.array_equal(on[0][2], on[1][2])        # deterministic
+    for key in ((2, 1, 0), (2, 0, 64), (2, 0, 128)):
+        o = runs[key][0]
+        if key[2] == 0 or mu is not None:                  # (a tile width of its own cuts the blocks elsewhere)
+            assert np.array_equal(on[0][1], o[1]), key
+        assert rel_l2(o[1] - x0s, off[1] - x0s) <= 2e-2, key
+        assert o[3] == off[3] and (key[1] == 1 or o[4] == off[4])
+    # iteration 1 has no folded forward before it and iteration 2 starts from the a_1 it formed: the first step is
+    # bit-identical, the second within rounding
+    assert rel_l2(on[0][0] - x0s, off[0] - x0s) <= 5e-3, rel_l2(on[0][0] - x0s, off[0] - x0s)
+    assert np.allclose(on[0][2], off[2], rtol=5e-3, atol=1e-4)
+    want = oracle_run(w, X, Y, x0s.astype(np.float64), 0, T) if mu is None else None
+    if want is not None:
+        assert rel_l2(on[0][1], want) <= TOL_PERIOD
+        assert rel_l2(on[0][1] - x0s, want - x0s) <= TOL_UPDATE
+
+
 COMMON_CASES = [
     _w("tc-common-b32", 3, (640, 1024, 10), 32, I=1),
     _w("tc-common-b64-n5", 5, (1024, 768, 100), 64, I=1),
