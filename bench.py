@@ -229,7 +229,7 @@ def ncu_traffic_per_launch(workload: str, family: str, N: int):
 # ----------------------------------------------------------------------------- byte model
 def period_bytes(w: synth.Workload, m_pad: int, sms: int = 148, momentum: bool = False, fused_average: bool = True,
                  fused_epilogues: bool = True, next_forward: bool = True, dx_in_update=True,
-                 shared_restart: bool = True, forward_chain: bool = False, head_kernel=1) -> dict:
+                 shared_restart: bool = True, forward_chain: bool = False, head_kernel=1, head_forward: bool = False) -> dict:
     """Algorithmic HBM bytes and launch counts of ONE averaging period (prsgd_local_steps(I) from a period
     boundary) of all N workers, per kernel family: {family: [bytes, launches]}.
 
@@ -246,7 +246,9 @@ def period_bytes(w: synth.Workload, m_pad: int, sms: int = 148, momentum: bool =
     Without the fused form the stand-alone average reads and writes the whole store (8 B/word, + 2 B bf16 copy).
     The class layer (at most 128 classes, last hidden width 128..1024, plain step) is one launch of its own
     family ("head"): its forward read of the bf16 copy, its update (10 B/param) and the mask read and dZ write
-    of the layer below; a_{L-1} is read once for both products.
+    of the layer below; a_{L-1} is read once for both products.  With three or more layers (and shared memory
+    for a ring of two stages behind the class layer's tiles) the same launch also does the forward GEMM of layer
+    L - 1, whose output then stays in shared memory.
     """
     bf = w.precision == 1
     e = 2 if bf else 4
@@ -261,6 +263,9 @@ def period_bytes(w: synth.Workload, m_pad: int, sms: int = 148, momentum: bool =
     def add(name, nbytes):
         fam[name][0] += nbytes
         fam[name][1] += 1
+    cp = (d[L] + 15) // 16 * 16
+    head_fixed = (8 * cp * 128 + 4 * B * 128 + 2 * B * (cp + 1) * 4 + 768 + 1023) // 1024 * 1024
+    head_fwd_ok = head_ok and head_forward and L >= 3 and (227 * 1024 - head_fixed - 1024) // (2 * (16384 + B * 128)) >= 2
     a1_ready = False
     for j in range(1, I + 1):
         averaging = w.I > 0 and j == I
@@ -271,7 +276,8 @@ def period_bytes(w: synth.Workload, m_pad: int, sms: int = 148, momentum: bool =
         wr = 1 if (bf and shared_restart and j == 1 and w.I > 0) else N
         l_first = 2 if a1_ready else 1
         head = head_ok and not (fuse and 2 * ((d[L] + 127) // 128) * ((d[L - 1] + 63) // 64) >= sms)
-        l_last = L - 1 if head else L
+        head_fwd = head and head_fwd_ok
+        l_last = (L - 2 if head_fwd else L - 1) if head else L
         chained = bf and forward_chain and 2 <= l_last - l_first + 1 <= 8      # all layers' forward GEMMs in one launch
         for l in range(l_first, l_last + 1):
             add("forward", wr * d[l] * d[l - 1] * e + N * (d[l] * 4 + B * d[l - 1] * e + B * d[l] * (e if l < L else 4)))
@@ -280,13 +286,16 @@ def period_bytes(w: synth.Workload, m_pad: int, sms: int = 148, momentum: bool =
         a1_ready = False
         if not epi:
             add("softmax", N * B * d[L] * (4 + 4 + e))
+        small_avg = 0
         if head:
             add("head", N * (d[L] * d[L - 1] * e + B * d[L - 1] * e + (d[L] * d[L - 1] + d[L]) * upd_b + B * d[L - 1] * 2 * e))
+            if head_fwd:       # + layer L - 1's forward: its weights and input read, its output neither written nor re-read
+                fam["head"][0] += wr * d[L - 1] * d[L - 2] * e + N * (d[L - 1] * 4 + B * d[L - 2] * e) - N * B * d[L - 1] * e
         for l in range(L, 0, -1):
             wl = d[l] * d[l - 1]
             if l == L and head:
                 if bf and fuse:
-                    add("average", N * wl * 10)
+                    small_avg += N * wl * 10
                 continue
             tiles64 = ((d[l] + 127) // 128) * ((d[l - 1] + 63) // 64)
             fuse_l = fuse and (not bf or 2 * tiles64 >= sms)
@@ -304,11 +313,11 @@ def period_bytes(w: synth.Workload, m_pad: int, sms: int = 148, momentum: bool =
                     upd -= (N - wr) * wl * 4
                 add("update_average" if fuse_l else "update", upd)
             if bf and fuse and not fuse_l:
-                add("average", N * wl * 10)
+                small_avg += N * wl * 10
         if not epi and bf:
             add("misc", 0)
         if bf and fuse:
-            add("misc", 0)
+            add("misc", small_avg)        # bias segments, and the weight segments too small for the fused form, in one launch
         if averaging and not fuse:
             add("average", N * m_pad * (8 + (2 if bf else 0)))
     return fam
@@ -463,6 +472,8 @@ def measure_config(torch, w_cfg, args, dev, rank, world, scaling, steps, warmup,
                       (args.no_head_kernel, binding.OPT_HEAD_KERNEL)):
         if flag:
             p.set_option(opt, 0)
+    if args.head_forward:
+        p.set_option(binding.OPT_HEAD_FORWARD, 1)
     if args.head_kernel_always:
         p.set_option(binding.OPT_HEAD_KERNEL, 2)
     if args.fold_all_dx:
@@ -517,7 +528,8 @@ def measure_config(torch, w_cfg, args, dev, rank, world, scaling, steps, warmup,
                              fused_epilogues=not args.no_fused_epilogues, next_forward=not args.no_next_forward,
                              dx_in_update=0 if args.no_dx_in_update else (2 if args.fold_all_dx else 1),
                              shared_restart=not args.no_shared_restart, forward_chain=args.forward_chain,
-                             head_kernel=0 if args.no_head_kernel else (2 if args.head_kernel_always else 1))
+                             head_kernel=0 if args.no_head_kernel else (2 if args.head_kernel_always else 1),
+                             head_forward=args.head_forward)
     if sharded_mode:          # a shard's period ends with row sums fused into the last step; the restart is a pass of its own
         fam_model["average"] = [fam_model["average"][0] + p.m_pad * 4 + w.N * p.m_pad * (4 + (2 if w.precision == 1 else 0)),
                                 fam_model["average"][1] + 4]
@@ -605,6 +617,8 @@ def parse_args(argv=None):
                     help="one forward launch per layer instead of one launch for all layers")
     ap.add_argument("--head-kernel-always", action="store_true",
                     help="the class layer as one launch of clusters even when its CTAs need more than one wave")
+    ap.add_argument("--head-forward", action="store_true",
+                    help="the forward GEMM of layer L - 1 inside the class layer's cluster launch instead of a launch of its own")
     ap.add_argument("--no-head-kernel", action="store_true",
                     help="the class layer's forward GEMM and update as launches of their own instead of one launch of clusters")
     ap.add_argument("--no-next-forward", action="store_true",

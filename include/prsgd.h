@@ -335,6 +335,19 @@ int prsgd_get_velocity_stacked(prsgd_ctx* ctx, float* dst, int dst_on_device);
  * launches of their own.  The two forms agree to fp32 rounding of the logits (different summation order, fast
  * exponential), not bit for bit; each is deterministic. */
 #define PRSGD_OPT_HEAD_KERNEL 14
+/* PRSGD_OPT_MERGED_SMALL_AVERAGE (default 1, tensor-core path, fused averaging iterations): the weight segments of
+ * layers too small for the fused update + average (the class layer) are averaged by the launch that averages the
+ * bias segments, at the end of the iteration, instead of by a launch of their own after the layer's update.  Same
+ * arithmetic (fp32 sum in worker order, one division): same bits. */
+#define PRSGD_OPT_MERGED_SMALL_AVERAGE 18
+/* PRSGD_OPT_HEAD_FORWARD (default 0; needs the cluster launch of PRSGD_OPT_HEAD_KERNEL, at least three layers and
+ * shared memory for two pipeline stages behind the class layer's tiles): when 1, the CTAs of a worker's cluster
+ * first form the 128 features of the last hidden activation they need, a_{L-1} = relu(W_{L-1} a_{L-2} + b_{L-1}),
+ * each streaming its row tile of W_{L-1}, and keep them in shared memory: one launch fewer per iteration, and
+ * a_{L-1} is never written to global memory.  Same bits as the separate forward launch (same products in the same
+ * order).  Off by default: measured slower (the two launches overlap the second one's start-up with the first
+ * one's streaming, which one launch cannot). */
+#define PRSGD_OPT_HEAD_FORWARD 17
 /* PRSGD_OPT_COMMON_POINT (default 1, tensor-core path, plain SGD step, fused average, PRSGD_OPT_SHARED_RESTART on):
  * an averaging iteration that STARTS from N equal rows (every iteration when I = 1, which the paper notes is
  * parallel mini-batch SGD; otherwise the first step after prsgd_average when I divides its number) forms the

@@ -36,6 +36,8 @@ OPT_DX_SHARED_PAIR = 13
 OPT_HEAD_KERNEL = 14
 OPT_COMMON_POINT = 15
 OPT_SPLIT_BLOCKS = 16
+OPT_HEAD_FORWARD = 17
+OPT_MERGED_SMALL_AVERAGE = 18
 ERR_DEVICE_TIMEOUT, ERR_NONFINITE = -6, -7
 KERNEL_FAMILIES = ("forward", "softmax", "dx", "update", "update_average", "average", "misc", "head")
 MAX_LAYERS = 16

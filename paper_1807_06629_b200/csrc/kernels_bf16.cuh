@@ -1998,38 +1998,51 @@ __global__ void __launch_bounds__(128) bias_update_kernel(const BiasArgs a) {
   *bp = fmaf(-a.gamma, g, *bp);
 }
 
-// Node average of every layer's bias segment in one launch (averaging iteration of the fused form):
-// grid (ceil(max d_l / 128), L), one thread per bias entry, the same arithmetic as average_rows_kernel
-// (fp32 sum in worker order, one division), so the bits equal update-then-average.
+// Node average of every layer's bias segment in one launch (averaging iteration of the fused form), plus the
+// weight segments of the layers that are too small for the fused update + average (the class layer): grid
+// (blocks, L + weight segments), one thread per entry (grid-stride over a weight segment), the same arithmetic as
+// average_rows_kernel (fp32 sum in worker order, one division), so the bits equal update-then-average.
 struct BiasAverageArgs {
   float* params;             // the store, or the momentum buffers (same layout)
   int64_t m_pad;
-  int N;
+  int N, L;
   int64_t b_off[PRSGD_MAX_LAYERS];
   int d_out[PRSGD_MAX_LAYERS];
   const DeviceStatus* status;
   float divisor;             // N, or 1 to leave the row sum
+  int n_seg;                 // weight segments averaged in the same launch (blockIdx.y = L + k)
+  int64_t seg_off[PRSGD_MAX_LAYERS];
+  int64_t seg_len[PRSGD_MAX_LAYERS];
+  uint16_t* shadow;          // bf16 copy of the store: the averaged weight segments are written there too
 };
 
 __global__ void __launch_bounds__(128) bias_average_kernel(const BiasAverageArgs a) {
   ptx::pdl_wait();
   ptx::pdl_trigger();     // after the wait: a later launch's early loads overlap this launch only
-  const int l = blockIdx.y;
-  const int j = blockIdx.x * blockDim.x + threadIdx.x;
-  if (j >= a.d_out[l] || a.status->error != 0u) return;
-  float* p = a.params + a.b_off[l] + j;
-  float s = 0.f;
-  int i = 0;
-  for (; i + 8 <= a.N; i += 8) {
-    float v[8];
+  if (a.status->error != 0u) return;
+  const int y = blockIdx.y;
+  const int64_t off = y < a.L ? a.b_off[y] : a.seg_off[y - a.L];
+  const int64_t len = y < a.L ? (int64_t)a.d_out[y] : a.seg_len[y - a.L];
+  for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < len; j += (int64_t)gridDim.x * blockDim.x) {
+    float* p = a.params + off + j;
+    float s = 0.f;
+    int i = 0;
+    for (; i + 8 <= a.N; i += 8) {
+      float v[8];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) v[u] = p[(int64_t)(i + u) * a.m_pad];
+      for (int u = 0; u < 8; ++u) v[u] = p[(int64_t)(i + u) * a.m_pad];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) s += v[u];
+      for (int u = 0; u < 8; ++u) s += v[u];
+    }
+    for (; i < a.N; ++i) s += p[(int64_t)i * a.m_pad];
+    const float mean = __fdiv_rn(s, a.divisor);
+    for (int r = 0; r < a.N; ++r) p[(int64_t)r * a.m_pad] = mean;
+    if (y >= a.L && a.shadow != nullptr) {
+      const uint16_t h = (uint16_t)(pack_bf16x2(mean, 0.f) & 0xFFFFu);
+      uint16_t* q = a.shadow + off + j;
+      for (int r = 0; r < a.N; ++r) q[(int64_t)r * a.m_pad] = h;
+    }
   }
-  for (; i < a.N; ++i) s += p[(int64_t)i * a.m_pad];
-  const float y = __fdiv_rn(s, a.divisor);
-  for (int r = 0; r < a.N; ++r) p[(int64_t)r * a.m_pad] = y;
 }
 
 }  // namespace prsgd
@@ -2110,7 +2123,8 @@ inline int tc_create(prsgd_ctx* c, std::string* err) {
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_next_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdNextCfg<64, true>::smem(c->B));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_update_common_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UpdCommonCfg::smem(c->B));
   if (e == cudaSuccess && st->head_rows > 0)
-    e = cudaFuncSetAttribute(tc_head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)head_smem_bytes(c->B, st->head_rows));
+    e = cudaFuncSetAttribute(tc_head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)head_smem_bytes(c->B, st->head_rows, 4) > 227 * 1024
+                                 ? 227 * 1024 : (int)head_smem_bytes(c->B, st->head_rows, 4));
   if (e != cudaSuccess) {
     *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(e);
     delete st;
@@ -2203,7 +2217,19 @@ inline bool tc_head_applies(const prsgd_ctx* c) {
   return c->head_kernel == 2 || (int64_t)c->N * (din / 128) <= (int64_t)st->num_sms;
 }
 
-inline void tc_launch_head(prsgd_ctx* c, const DrawArgs& dr, const uint8_t* active) {
+// The forward GEMM of layer L - 1 inside the head launch (PRSGD_OPT_HEAD_FORWARD): at least three layers (layer
+// L - 1's input is then an activation buffer, not the data pool) and room for a ring of two or more stages behind
+// the head's own shared memory.
+inline int tc_head_forward_stages(const prsgd_ctx* c) {
+  const TcState* st = static_cast<const TcState*>(c->tc);
+  if (c->head_forward == 0 || c->L < 3 || st->head_rows == 0) return 0;
+  const int64_t room = 227 * 1024 - (int64_t)head_smem_bytes(c->B, st->head_rows, 0);
+  int stages = (int)(room / (int64_t)head_fwd_stage_bytes(c->B));
+  if (stages > 4) stages = 4;
+  return stages >= 2 ? stages : 0;
+}
+
+inline void tc_launch_head(prsgd_ctx* c, const DrawArgs& dr, const uint8_t* active, bool with_forward) {
   TcState* st = static_cast<TcState*>(c->tc);
   const int L = c->L;
   const Layer& ly = c->layer[L - 1];
@@ -2213,9 +2239,16 @@ inline void tc_launch_head(prsgd_ctx* c, const DrawArgs& dr, const uint8_t* acti
   a.bias_rw = c->params + ly.b_off; a.bias_lo_rw = c->params + c->layer[L - 2].b_off; a.bias_stride = c->m_pad;
   a.Y = c->Y; a.P = c->P; a.row_losses = c->losses; a.draws = c->draws;
   a.out_bk = c->buf.delta_bk[L - 1]; a.ld_out = c->buf.ld[L - 1];
+  if (with_forward) {
+    a.fwd = 1; a.fwd_stages = tc_head_forward_stages(c);
+    a.fwd_ksteps = (c->layer[L - 2].d_in / 64 + 1) / 2;
+    a.fwd_prefetch = (active == nullptr && c->early_loads) ? 1 : 0;
+    a.fwd_shared_w = tc_shared_restart(c, active) ? 1 : 0;
+  }
   const unsigned cl = (unsigned)(ly.d_in / 128);
-  launch_pdl_cluster(tc_head_kernel, dim3(cl, (unsigned)c->N), dim3(kHeadThreads), head_smem_bytes(c->B, st->head_rows), c->stream, cl,
-                     st->head_shadow, st->layer[L - 1].act_in, st->head_master, a);
+  const TcLayerMaps& lo = st->layer[L >= 2 ? L - 2 : 0];
+  launch_pdl_cluster(tc_head_kernel, dim3(cl, (unsigned)c->N), dim3(kHeadThreads), head_smem_bytes(c->B, st->head_rows, a.fwd_stages),
+                     c->stream, cl, st->head_shadow, st->layer[L - 1].act_in, st->head_master, lo.shadow_k, lo.act_in, a);
 }
 
 // The per-worker flags the launches being enqueued honour: Algorithm 3's mask, or the mask of a worker group.
@@ -2508,16 +2541,26 @@ inline void tc_launch_velocity_segment_average(prsgd_ctx* c, int l) {
              (const DeviceStatus*)c->status, 0.f);
 }
 
-inline void tc_launch_bias_average(prsgd_ctx* c, float* store) {
+// `with_weights`: also the weight segments of the layers that did not take the fused update + average
+inline void tc_launch_bias_average(prsgd_ctx* c, float* store, bool with_weights = false) {
   BiasAverageArgs a{};
-  a.params = store; a.m_pad = c->m_pad; a.N = c->N; a.status = c->status;
+  a.params = store; a.m_pad = c->m_pad; a.N = c->N; a.L = c->L; a.status = c->status;
   a.divisor = (store == c->params && c->avg_divisor > 0.f) ? c->avg_divisor : (float)c->N;
-  int dmax = 1;
+  int64_t longest = 1;
   for (int l = 1; l <= c->L; ++l) {
     a.b_off[l - 1] = c->layer[l - 1].b_off; a.d_out[l - 1] = c->layer[l - 1].d_out;
-    if (a.d_out[l - 1] > dmax) dmax = a.d_out[l - 1];
+    if (a.d_out[l - 1] > longest) longest = a.d_out[l - 1];
+    if (with_weights && !tc_layer_fuses_average(c, l)) {
+      a.seg_off[a.n_seg] = c->layer[l - 1].w_off;
+      a.seg_len[a.n_seg] = (int64_t)c->layer[l - 1].d_out * c->layer[l - 1].d_in;
+      if (a.seg_len[a.n_seg] > longest) longest = a.seg_len[a.n_seg];
+      ++a.n_seg;
+    }
   }
-  launch_pdl(bias_average_kernel, dim3((dmax + 127) / 128, c->L), dim3(128), 0, c->stream, a);
+  a.shadow = with_weights ? c->shadow : nullptr;
+  int64_t blocks = (longest + 127) / 128;
+  if (blocks > 1024) blocks = 1024;                  // (a long segment is walked with a grid stride)
+  launch_pdl(bias_average_kernel, dim3((unsigned)blocks, c->L + a.n_seg), dim3(128), 0, c->stream, a);
 }
 
 }  // namespace prsgd

@@ -38,6 +38,15 @@ struct HeadArgs {
   int32_t* draws;            // [N]
   uint16_t* out_bk;          // bf16 dZ_{L-1} [N][B][ld_out]
   int ld_out;
+  // Forward GEMM of layer L - 1 in the same launch (`fwd` = 1): CTA s of a worker's cluster forms the 128 features
+  // a_{L-1}[:, 128 s ..] = relu(W_{L-1}[128 s .., :] a_{L-2} + b_{L-1}) it needs, streaming its row tile of W_{L-1}
+  // through a ring of `fwd_stages` stages like tc_stream_kernel, and writes them straight into the activation
+  // tile in shared memory: a_{L-1} never goes to global memory (nothing else reads it).
+  int fwd;
+  int fwd_ksteps;            // pipeline steps: ceil(d_{L-2} / 128)
+  int fwd_stages;
+  int fwd_prefetch;          // W_{L-1}'s first tiles may be requested before the previous launch has completed
+  int fwd_shared_w;          // every worker's W_{L-1} holds the same bits: read worker 0's (one HBM read serves all)
 };
 
 constexpr int kHeadThreads = 320;     // warp 0 loads, warp 1 MMAs, warps 2..5 logits / softmax / step of W_L, warps 6..9 dZ_{L-1}
@@ -48,14 +57,21 @@ constexpr int kHeadThreads = 320;     // warp 0 loads, warp 1 MMAs, warps 2..5 l
 // The logits MMA has M = 128: it reads 128 rows (16 KB) from the start of each bf16 box; the rows past Cp are
 // whatever lies behind the box (the regions that follow are always longer than that), and their accumulator
 // lanes are never read.
-__host__ __device__ inline uint32_t head_smem_bytes(int B, int Cp) {
+__host__ __device__ inline uint32_t head_fixed_bytes(int B, int Cp) {
   const uint32_t op_box = (uint32_t)B * 128u, wbox = (uint32_t)Cp * 128u;
-  return 2u * wbox + 2u * op_box + 4u * wbox + 2u * wbox + 2u * op_box + 2u * (uint32_t)B * (uint32_t)(Cp + 1) * 4u + 512u + 256u + 1024u;
+  const uint32_t used = 2u * wbox + 2u * op_box + 4u * wbox + 2u * wbox + 2u * op_box + 2u * (uint32_t)B * (uint32_t)(Cp + 1) * 4u + 512u + 256u;
+  return (used + 1023u) & ~1023u;                        // (the forward ring behind it holds swizzled tiles)
+}
+__host__ __device__ inline uint32_t head_fwd_stage_bytes(int B) { return 2u * (16384u + (uint32_t)B * 128u); }
+__host__ __device__ inline uint32_t head_smem_bytes(int B, int Cp, int fwd_stages = 0) {
+  return head_fixed_bytes(B, Cp) + (uint32_t)fwd_stages * head_fwd_stage_bytes(B) + 1024u;
 }
 
 __global__ void __launch_bounds__(kHeadThreads, 1) tc_head_kernel(const __grid_constant__ CUtensorMap mapShadow,
                                                                   const __grid_constant__ CUtensorMap mapAct,
                                                                   const __grid_constant__ CUtensorMap mapMaster,
+                                                                  const __grid_constant__ CUtensorMap mapWlo,
+                                                                  const __grid_constant__ CUtensorMap mapActLo,
                                                                   const HeadArgs a) {
   using namespace ptx;
   extern __shared__ uint8_t smem_raw[];
@@ -69,6 +85,11 @@ __global__ void __launch_bounds__(kHeadThreads, 1) tc_head_kernel(const __grid_c
   const uint32_t o_act = 2u * wbox, o_mst = o_act + 2u * op_box, o_new = o_mst + 4u * wbox, o_dz = o_new + 2u * wbox;
   const uint32_t o_part = o_dz + 2u * op_box, o_zs = o_part + logit_bytes, o_bias = o_zs + logit_bytes, o_bar = o_bias + 512u;
   const uint32_t g1 = base + o_bar, g2 = g1 + 8u, acc1 = g1 + 16u, acc2 = g1 + 24u, acc3 = g1 + 32u;
+  const uint32_t acc0 = g1 + 40u, act_ready = g1 + 48u;  // forward of layer L - 1: product done / a_{L-1} tile written
+  auto f_full = [&](int st) { return g1 + 96u + 8u * st; };
+  auto f_empty = [&](int st) { return g1 + 160u + 8u * st; };
+  const uint32_t o_ring = head_fixed_bytes(a.B, Cp);
+  const uint32_t fstage = head_fwd_stage_bytes(a.B);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen + o_bar + 64);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + o_bar + 68);
   float* part = reinterpret_cast<float*>(gen + o_part);
@@ -84,9 +105,12 @@ __global__ void __launch_bounds__(kHeadThreads, 1) tc_head_kernel(const __grid_c
 
   if (tid == 0) {
     mbar_init(g1, 1); mbar_init(g2, 1); mbar_init(acc1, 1); mbar_init(acc2, 1); mbar_init(acc3, 1);
+    mbar_init(acc0, 1); mbar_init(act_ready, 128);
+    for (int st = 0; st < a.fwd_stages; ++st) { mbar_init(f_full(st), 1); mbar_init(f_empty(st), 1); }
     *abort_flag = *(volatile unsigned int*)&a.status->error != 0u ? 1 : 0;   // an earlier expired wait: no-op (see tc_stream_kernel)
     fence_mbar_init();
     prefetch_tensormap(&mapShadow); prefetch_tensormap(&mapAct); prefetch_tensormap(&mapMaster);
+    if (a.fwd) { prefetch_tensormap(&mapWlo); prefetch_tensormap(&mapActLo); }
   }
   if (warp == 1) { tmem_alloc(smem_u32(tmem_slot), 256u); tmem_relinquish(); }
   tc_fence_before();
@@ -96,14 +120,31 @@ __global__ void __launch_bounds__(kHeadThreads, 1) tc_head_kernel(const __grid_c
     mbar_expect_tx(g2, 4u * wbox);
 #pragma unroll 1
     for (int q = 0; q < 4; ++q) tma_load_3d(base + o_mst + q * wbox, &mapMaster, g2, k0 + 32 * q, 0, n);
-    mbar_expect_tx(g1, 2u * wbox + 2u * op_box);         // (the activation boxes follow after the dependency wait)
+    mbar_expect_tx(g1, 2u * wbox + (a.fwd ? 0u : 2u * op_box));   // (the activation boxes follow after the dependency wait)
     tma_load_3d(base, &mapShadow, g1, k0, 0, n);
     tma_load_3d(base + wbox, &mapShadow, g1, k0 + 64, 0, n);
+  };
+  // two 64-wide K blocks of this CTA's row tile of W_{L-1} (a block past the end of K is zero-filled by TMA)
+  auto load_wlo = [&](int st, int ks) {
+    const uint32_t sa = base + o_ring + (uint32_t)st * fstage;
+    const int nw = a.fwd_shared_w ? 0 : n;
+    tma_load_3d(sa, &mapWlo, f_full(st), (2 * ks) * 64, k0, nw);
+    tma_load_3d(sa + 16384u, &mapWlo, f_full(st), (2 * ks + 1) * 64, k0, nw);
   };
   // Nothing in flight writes W_L when this launch begins (the launch before it is a forward GEMM of a lower
   // layer or layer 1's update), so its tiles are requested while that launch drains.
   const bool pre = a.prefetch != 0 && *abort_flag == 0;
-  if (pre && warp == 0 && lane == 0) load_weights();
+  int fpre = 0;                                          // forward ring stages whose weight tiles are under way already
+  if (warp == 0 && lane == 0) {
+    if (a.fwd && a.fwd_prefetch != 0 && *abort_flag == 0) {
+      fpre = a.fwd_ksteps < a.fwd_stages ? a.fwd_ksteps : a.fwd_stages;
+      for (int ks = 0; ks < fpre; ++ks) {
+        mbar_expect_tx(f_full(ks), fstage);
+        load_wlo(ks, ks);
+      }
+    }
+    if (pre) load_weights();
+  }
   pdl_wait();
   pdl_trigger();
   const uint32_t tmem = *tmem_slot;
@@ -114,14 +155,52 @@ __global__ void __launch_bounds__(kHeadThreads, 1) tc_head_kernel(const __grid_c
   const int etid = tid - 64;                             // 0..127 among warps 2..5
   float blo_old = 0.f;
 
-  // ---------------- phase 1: this slice's share of the logits
+  // ---------------- phase 0 (fwd): a_{L-1}[:, slice]; phase 1: this slice's share of the logits
   if (run) {
     if (warp == 0 && lane == 0) {
       if (!pre) load_weights();
-      tma_load_3d(base + o_act, &mapAct, g1, k0, 0, n);
-      tma_load_3d(base + o_act + op_box, &mapAct, g1, k0 + 64, 0, n);
+      if (a.fwd) {
+        bool ok = true;
+#pragma unroll 1
+        for (int ks = 0; ks < a.fwd_ksteps && ok; ++ks) {
+          const int st = ks % a.fwd_stages;
+          if (ks >= fpre) {
+            ok = mbar_wait(f_empty(st), (((uint32_t)(ks / a.fwd_stages)) & 1u) ^ 1u, abort_flag, a.status, 0x606);
+            if (!ok) break;
+            mbar_expect_tx(f_full(st), fstage);
+            load_wlo(st, ks);
+          }
+          const uint32_t sb = base + o_ring + (uint32_t)st * fstage + 32768u;
+          tma_load_3d(sb, &mapActLo, f_full(st), (2 * ks) * 64, 0, n);
+          tma_load_3d(sb + op_box, &mapActLo, f_full(st), (2 * ks + 1) * 64, 0, n);
+        }
+      } else {
+        tma_load_3d(base + o_act, &mapAct, g1, k0, 0, n);
+        tma_load_3d(base + o_act + op_box, &mapAct, g1, k0 + 64, 0, n);
+      }
     } else if (warp == 1 && lane == 0) {
-      if (mbar_wait(g1, 0u, abort_flag, a.status, 0x601)) {
+      bool fok = true;
+      if (a.fwd) {
+        const uint32_t idesc0 = idesc_bf16(128, a.B, 0, 0);
+#pragma unroll 1
+        for (int ks = 0; ks < a.fwd_ksteps && fok; ++ks) {
+          const int st = ks % a.fwd_stages;
+          fok = mbar_wait(f_full(st), ((uint32_t)(ks / a.fwd_stages)) & 1u, abort_flag, a.status, 0x607);
+          if (!fok) break;
+          tc_fence_after();
+          const uint32_t sa = base + o_ring + (uint32_t)st * fstage, sb = sa + 32768u;
+#pragma unroll 1
+          for (int jk = 0; jk < 8; ++jk) {
+            const uint32_t j = (uint32_t)jk >> 2, k = (uint32_t)jk & 3u;
+            mma_bf16(tmem + kColX, smem_desc_sw128(sa + j * 16384u + k * 32u, 16u, 1024u),
+                     smem_desc_sw128(sb + j * op_box + k * 32u, 16u, 1024u), idesc0, (ks | jk) != 0 ? 1u : 0u);
+          }
+          mma_commit(f_empty(st));
+        }
+        if (fok) mma_commit(acc0);
+        fok = fok && mbar_wait(act_ready, 0u, abort_flag, a.status, 0x608);
+      }
+      if (fok && mbar_wait(g1, 0u, abort_flag, a.status, 0x601)) {
         tc_fence_after();
         const uint32_t idesc = idesc_bf16(128, a.B, 0, 0);
 #pragma unroll 1
@@ -141,6 +220,30 @@ __global__ void __launch_bounds__(kHeadThreads, 1) tc_head_kernel(const __grid_c
         const int b = task / nz, ch = nch + task % nz;
         *reinterpret_cast<uint4*>(gen + o_dz + (uint32_t)(ch >> 3) * op_box + (uint32_t)b * 128u + ((uint32_t)((ch & 7) ^ (b & 7)) << 4)) =
             make_uint4(0u, 0u, 0u, 0u);
+      }
+      if (a.fwd) {
+        // forward epilogue of the slice: bias, ReLU, bf16, written as the two {64, B} activation boxes (row b of a
+        // box = 128 bytes, 16-byte chunks swizzled by b) the products below read; thread <-> feature k0 + r
+        const float blo = a.bias_lo_rw[(int64_t)n * a.bias_stride + k0 + r];
+        const bool ok0 = __all_sync(0xffffffffu, mbar_wait(acc0, 0u, abort_flag, a.status, 0x609));
+        if (ok0) {
+          tc_fence_after();
+          uint8_t* acol = gen + o_act + (uint32_t)(r >> 6) * op_box + (uint32_t)(r & 7) * 2u;
+          const uint32_t chunk = (uint32_t)((r & 63) >> 3);
+#pragma unroll 1
+          for (int b8 = 0; b8 < a.B; b8 += 8) {
+            uint32_t v[8];
+            tmem_ld8(tmem + lane_off + kColX + (uint32_t)b8, v);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              *reinterpret_cast<uint16_t*>(acol + (uint32_t)(b8 + j) * 128u + ((chunk ^ (uint32_t)j) << 4)) =
+                  f32_to_bf16_rn(fmaxf(__uint_as_float(v[j]) + blo, 0.f));
+          }
+          tc_fence_before();
+          fence_proxy_async();
+          mbar_arrive(act_ready);
+        }
       }
       const bool ok = __all_sync(0xffffffffu, mbar_wait(acc1, 0u, abort_flag, a.status, 0x602));
       if (ok && q4 * 32 < C) {                           // (a warp whose lanes all lie beyond C holds no logits)

@@ -312,7 +312,8 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging, bool more_follow) {
   // The class layer as one launch of clusters (logits, softmax-CE gradient, step of W_L, dZ_{L-1}): whenever its
   // step is the plain one (a class layer large enough for the fused update + average keeps the separate launches).
   const bool head = tc_head_applies(c) && !(fuse && tc_layer_fuses_average(c, L));
-  const int l_fwd_last = head ? L - 1 : L;
+  const bool head_fwd = head && tc_head_forward_stages(c) > 0 && !(skip_f1 && L == 2);   // ... and the forward GEMM below it
+  const int l_fwd_last = head ? (head_fwd ? L - 2 : L - 1) : L;
   if (tc_chain_applies(c, skip_f1 ? 2 : 1, l_fwd_last)) {          // every remaining layer's forward GEMM in one launch
     prof_begin(c, PRSGD_KERNEL_FORWARD);
     tc_launch_forward_chain(c, skip_f1 ? 2 : 1, l_fwd_last, dr, act_mask);
@@ -344,7 +345,7 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging, bool more_follow) {
   const bool dx_in_upd = c->dx_in_update && tc_epilogues_fused(c);
   if (head) {
     prof_begin(c, PRSGD_KERNEL_HEAD);
-    tc_launch_head(c, dr, act_mask);
+    tc_launch_head(c, dr, act_mask, head_fwd);
     LAUNCH_CHECK(c);
   }
   for (int l = L; l >= 1; --l) {          // dX_l reads W_l before the update of layer l overwrites it
@@ -371,9 +372,11 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging, bool more_follow) {
       LAUNCH_CHECK(c);
     }
     if (fuse && !fuse_l) {
-      prof_begin(c, PRSGD_KERNEL_AVERAGE);
-      tc_launch_weight_average(c, l);
-      LAUNCH_CHECK(c);
+      if (!c->merged_small_average) {        // (else with the bias segments, in the iteration's last launch)
+        prof_begin(c, PRSGD_KERNEL_AVERAGE);
+        tc_launch_weight_average(c, l);
+        LAUNCH_CHECK(c);
+      }
       if (avg_vel) {
         prof_begin(c, PRSGD_KERNEL_AVERAGE);
         tc_launch_velocity_segment_average(c, l);
@@ -388,7 +391,7 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging, bool more_follow) {
   }
   if (fuse) {
     prof_begin(c, PRSGD_KERNEL_MISC);
-    tc_launch_bias_average(c, c->params);
+    tc_launch_bias_average(c, c->params, c->merged_small_average != 0);
     LAUNCH_CHECK(c);
     if (avg_vel) {
       prof_begin(c, PRSGD_KERNEL_MISC);
@@ -733,7 +736,7 @@ void period_key(const prsgd_ctx* c, uint64_t (&key)[13]) {
   key[7] = (uint64_t)c->average_velocity; key[8] = reinterpret_cast<uint64_t>(c->X);
   key[9] = reinterpret_cast<uint64_t>(c->Y); key[10] = (uint64_t)c->worker0; key[11] = (uint64_t)c->fused_epilogues | ((uint64_t)c->early_loads << 1) | ((uint64_t)c->next_forward << 2) | ((uint64_t)c->dx_in_update << 3);
   key[12] = (c->rows_identical ? 1u : 0u) | ((uint64_t)c->shared_restart << 1) | ((uint64_t)c->forward_chain << 2) |
-            ((uint64_t)c->worker_groups << 3) | ((uint64_t)c->dx_shared_pair << 6) | ((uint64_t)c->head_kernel << 7) | ((uint64_t)c->common_point << 9) | ((uint64_t)c->split_blocks << 10);   // the period's first iteration may share reads
+            ((uint64_t)c->worker_groups << 3) | ((uint64_t)c->dx_shared_pair << 6) | ((uint64_t)c->head_kernel << 7) | ((uint64_t)c->common_point << 9) | ((uint64_t)c->split_blocks << 10) | ((uint64_t)c->head_forward << 12) | ((uint64_t)c->merged_small_average << 13);   // the period's first iteration may share reads
 }
 
 // One whole averaging period (I iterations starting right after an average) as a CUDA graph: the
@@ -1140,6 +1143,8 @@ int prsgd_set_option(prsgd_ctx* c, int32_t option, int64_t value) {
   if (option == PRSGD_OPT_FORWARD_CHAIN) { c->forward_chain = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_DX_SHARED_PAIR) { c->dx_shared_pair = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_COMMON_POINT) { c->common_point = value != 0; return PRSGD_OK; }
+  if (option == PRSGD_OPT_HEAD_FORWARD) { c->head_forward = value != 0; return PRSGD_OK; }
+  if (option == PRSGD_OPT_MERGED_SMALL_AVERAGE) { c->merged_small_average = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_SPLIT_BLOCKS) {
     if (value < 0 || value > 2) return fail(c, PRSGD_ERR_ARG, "PRSGD_OPT_SPLIT_BLOCKS takes 0, 1 or 2");
     c->split_blocks = (int)value;

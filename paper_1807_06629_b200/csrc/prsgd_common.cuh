@@ -117,6 +117,8 @@ struct prsgd_ctx {
   float* split_part = nullptr;           // [2 * kSplitMaxCtas][B][128] fp32 partial accumulators
   unsigned int* split_count = nullptr;   // a counter per block, zero between launches
   int common_point = 1;          // fused update + average from a common starting point: one GEMM over all workers' minibatches
+  int merged_small_average = 1;  // fused averaging iteration: weight segments too small for the fused form are averaged by the bias-average launch
+  int head_forward = 0;          // the forward GEMM of layer L - 1 runs inside the class layer's cluster launch
   int head_kernel = 1;           // the class layer's forward, softmax-CE gradient, step and dZ below it as one launch of clusters
   int dx_in_update = 1;          // layers >= 2: the update launch also forms dZ of the layer below (tensor-core path)
   int next_forward = 1;          // layer 1's update also forms a_1 of the next iteration (tensor-core path)

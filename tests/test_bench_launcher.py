@@ -81,10 +81,10 @@ def test_byte_model_follows_the_launch_rules():
     assert bench.period_bytes(cfg4, 8496384)["head"][1] == 0       # 64 workers x 8 slices: more than one wave, not used
     h = bench.period_bytes(cfg4, 8496384, head_kernel=2)   # the class layer as one launch of its own family
     assert {k: v[1] for k, v in h.items() if v[1]} == {"forward": 65, "dx": 2, "update": 93, "update_average": 3,
-                                                         "average": 1, "misc": 1, "head": 32}
+                                                         "misc": 1, "head": 32}
     f = bench.period_bytes(cfg4, 8496384, head_kernel=0)
     assert {k: v[1] for k, v in f.items() if v[1]} == {"forward": 97, "dx": 2, "update": 125, "update_average": 3,
-                                                         "average": 1, "misc": 1}
+                                                         "misc": 1}            # (the class layer's segment average rides on the bias-average launch)
     assert sum(v[0] for v in f.values()) - sum(v[0] for v in h.values()) == (
         32 * 64 * (100 * 4 + 32 * 100 * 4 + 32 * (100 + 1024) * 2)      # no bias re-read, no fp32 logits, operands read once
         - 63 * 100 * 1024 * 2)                             # (its first iteration reads every worker's own copy of W_L)
@@ -102,6 +102,9 @@ def test_byte_model_follows_the_launch_rules():
     assert c16["forward"][1] == 33 and c16["dx"][1] == 16 and c16["update"][1] == 46
     c16 = bench.period_bytes(synth.WORKLOADS["cfg3"].with_(I=16), 4206656)
     assert c16["forward"][1] == 17 and c16["dx"][1] == 16 and c16["update"][1] == 30 and c16["head"][1] == 16
+    c16f = bench.period_bytes(synth.WORKLOADS["cfg3"].with_(I=16), 4206656, head_forward=True)   # ... and layer 2's forward inside the head launch
+    assert c16f["forward"][1] == 1 and c16f["head"][1] == 16
+    assert (c16["forward"][0] + c16["head"][0]) - (c16f["forward"][0] + c16f["head"][0]) == 16 * 16 * 2 * 64 * 1024 * 2
     assert bench.period_bytes(synth.WORKLOADS["cfg3"].with_(I=16), 4206656, forward_chain=True)["forward"][1] == 16
     f32 = bench.period_bytes(synth.WORKLOADS["cfg2"], 669728)
     assert f32["forward"][1] == 24 and f32["softmax"][1] == 8 and f32["update_average"][1] == 3

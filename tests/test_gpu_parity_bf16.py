@@ -280,6 +280,7 @@ def test_class_layer_in_one_launch_of_clusters(torch_cuda, w):
         with torch.cuda.stream(torch.cuda.Stream()):
             p = make_ctx(w, X, Y, x0)
             p.set_option(binding.OPT_HEAD_KERNEL, head)
+            p.set_option(binding.OPT_HEAD_FORWARD, 0)        # (the forward GEMM below it stays a launch: it has a test of its own)
             p.set_option(binding.OPT_GRAPH, graph)
             n0 = p.get_launch_count()
             p.local_steps(1)
@@ -556,6 +557,92 @@ def test_reading_the_common_restart_point_once_changes_no_bit(torch_cuda):
                 assert np.array_equal(grp[0][2], o[2])
                 if mu is not None:
                     assert np.array_equal(grp[0][3], o[3])
+
+
+def test_small_weight_segments_averaged_by_the_bias_average_launch_change_no_bit(torch_cuda):
+    """On a fused averaging iteration the weight segments too small for the fused update + average (every layer
+    of these small nets; the class layer of the large ones) are averaged by the launch that averages the bias
+    segments instead of by launches of their own: identical parameters, bf16 copies and momentum buffers over
+    several periods, direct and replayed, with and without the cluster launch, also in the row-sum form; fewer
+    launches."""
+    torch = torch_cuda
+    from paper_1807_06629_b200 import binding
+    cases = ((SMALL[1], None), (SMALL[4], None), (_w("tc-merge-I1", 3, (640, 1024, 10), 32, I=1), None),
+             (_w("tc-merge-mom", 4, (128, 256, 10), 32, I=2), 0.9))
+    for w, mu in cases:
+        X, Y, x0 = make_inputs(w)
+        outs = []
+        for merged, graph, head in ((0, 0, 1), (1, 0, 1), (1, 1, 1), (0, 0, 0), (1, 0, 0)):
+            with torch.cuda.stream(torch.cuda.Stream()):
+                p = make_ctx(w, X, Y, x0)
+                if mu is not None:
+                    p.enable_momentum(mu, average_velocity=True)
+                p.set_option(binding.OPT_MERGED_SMALL_AVERAGE, merged)
+                p.set_option(binding.OPT_GRAPH, graph)
+                p.set_option(binding.OPT_HEAD_KERNEL, head)
+                n0 = p.get_launch_count()
+                p.local_steps(3 * w.I + 1)
+                launches = p.get_launch_count() - n0
+                p.sync()
+                shadow = p.shadow.view(torch.int16).cpu().numpy().copy()
+                p.set_interval(0)
+                if mu is None:
+                    p.local_steps_sum(1)
+                outs.append((head, p.get_params_stacked(), shadow, p.get_velocity_stacked() if mu is not None else None, launches, graph))
+                torch.cuda.current_stream().synchronize()
+                p.close()
+        for head in (1, 0):
+            grp = [o for o in outs if o[0] == head]
+            for o in grp[1:]:
+                assert np.array_equal(grp[0][1], o[1]) and np.array_equal(grp[0][2], o[2]), (w.name, head)
+                if mu is not None:
+                    assert np.array_equal(grp[0][3], o[3])
+            assert grp[1][4] < grp[0][4]
+
+
+HEAD_FWD_CASES = [
+    _w("tc-tail-small", 3, (128, 256, 128, 10), 32, I=3),
+    _w("tc-tail-ragged-k", 2, (192, 320, 1024, 10), 64, I=2),
+    _w("tc-tail-b16-c100", 5, (64, 128, 512, 100), 16, I=3),
+    _w("tc-tail-deep", 2, (64, 192, 256, 256, 10), 32, I=2),
+    _w("tc-tail-I1", 4, (128, 1024, 256, 10), 32, I=1),
+]
+
+
+@pytest.mark.parametrize("w", HEAD_FWD_CASES, ids=[w.name for w in HEAD_FWD_CASES])
+def test_forward_below_the_class_layer_inside_the_cluster_launch(torch_cuda, w):
+    """The forward GEMM of layer L - 1 done by the class layer's cluster launch (every CTA forms the 128 features of
+    a_{L-1} it needs and keeps them in shared memory) against the separate forward launch: the same products in
+    the same order, so identical parameters, losses and draws over several periods, direct and replayed, with a
+    worker mask, from a common restart point (I = 1) and with the option that shares one copy of the weights
+    off; one launch fewer per iteration."""
+    torch = torch_cuda
+    from paper_1807_06629_b200 import binding
+    X, Y, x0 = make_inputs(w)
+    T = 2 * w.I + 2
+    for variant in ("plain", "mask", "no-shared-restart"):
+        outs = []
+        for fwd, graph in ((0, 0), (1, 0), (1, 1)):
+            with torch.cuda.stream(torch.cuda.Stream()):
+                p = make_ctx(w, X, Y, x0)
+                p.set_option(binding.OPT_HEAD_FORWARD, fwd)
+                p.set_option(binding.OPT_GRAPH, graph)
+                if variant == "mask":
+                    p.set_active([1 if i != 1 else 0 for i in range(w.N)])
+                if variant == "no-shared-restart":
+                    p.set_option(binding.OPT_SHARED_RESTART, 0)
+                n0 = p.get_launch_count()
+                p.local_steps(1)
+                p.local_steps(T - 1)
+                outs.append((p.get_params_stacked(), p.get_losses(), p.get_draws().tolist(), p.get_launch_count() - n0))
+                torch.cuda.current_stream().synchronize()
+                p.close()
+        keep = [i for i in range(w.N) if variant != "mask" or i != 1]
+        for o in outs[1:]:
+            assert np.array_equal(outs[0][0], o[0]), (w.name, variant)
+            assert np.array_equal(outs[0][1][keep], o[1][keep])
+            assert [outs[0][2][i] for i in keep] == [o[2][i] for i in keep]
+        assert outs[1][3] == outs[0][3] - T, (outs[0][3], outs[1][3])
 
 
 SPLIT_CASES = [
