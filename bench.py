@@ -229,7 +229,7 @@ def ncu_traffic_per_launch(workload: str, family: str, N: int):
 # ----------------------------------------------------------------------------- byte model
 def period_bytes(w: synth.Workload, m_pad: int, sms: int = 148, momentum: bool = False, fused_average: bool = True,
                  fused_epilogues: bool = True, next_forward: bool = True, dx_in_update=True,
-                 shared_restart: bool = True, forward_chain: bool = False, head_kernel=1, head_forward: bool = False) -> dict:
+                 shared_restart: bool = True, forward_chain: bool = False, head_kernel=1, head_forward: bool = False, common_point: bool = True) -> dict:
     """Algorithmic HBM bytes and launch counts of ONE averaging period (prsgd_local_steps(I) from a period
     boundary) of all N workers, per kernel family: {family: [bytes, launches]}.
 
@@ -287,6 +287,7 @@ def period_bytes(w: synth.Workload, m_pad: int, sms: int = 148, momentum: bool =
         if not epi:
             add("softmax", N * B * d[L] * (4 + 4 + e))
         small_avg = 0
+        common_layers = 0
         if head:
             add("head", N * (d[L] * d[L - 1] * e + B * d[L - 1] * e + (d[L] * d[L - 1] + d[L]) * upd_b + B * d[L - 1] * 2 * e))
             if head_fwd:       # + layer L - 1's forward: its weights and input read, its output neither written nor re-read
@@ -312,6 +313,10 @@ def period_bytes(w: synth.Workload, m_pad: int, sms: int = 148, momentum: bool =
                 if fuse_l:
                     upd -= (N - wr) * wl * 4
                 add("update_average" if fuse_l else "update", upd)
+                if fuse_l and wr == 1 and not momentum and common_point:
+                    common_layers += 1          # from a common point these layers share ONE launch after the dX launches
+                    if common_layers > 1:
+                        fam["update_average"][1] -= 1
             if bf and fuse and not fuse_l:
                 small_avg += N * wl * 10
         if not epi and bf:
@@ -469,7 +474,7 @@ def measure_config(torch, w_cfg, args, dev, rank, world, scaling, steps, warmup,
                       (args.no_fused_epilogues, binding.OPT_FUSED_EPILOGUES),
                       (args.no_shared_restart, binding.OPT_SHARED_RESTART),
                       (args.no_forward_chain, binding.OPT_FORWARD_CHAIN),
-                      (args.no_head_kernel, binding.OPT_HEAD_KERNEL)):
+                      (args.no_head_kernel, binding.OPT_HEAD_KERNEL), (args.no_common_point, binding.OPT_COMMON_POINT)):
         if flag:
             p.set_option(opt, 0)
     if args.head_forward:
@@ -529,7 +534,7 @@ def measure_config(torch, w_cfg, args, dev, rank, world, scaling, steps, warmup,
                              dx_in_update=0 if args.no_dx_in_update else (2 if args.fold_all_dx else 1),
                              shared_restart=not args.no_shared_restart, forward_chain=args.forward_chain,
                              head_kernel=0 if args.no_head_kernel else (2 if args.head_kernel_always else 1),
-                             head_forward=args.head_forward)
+                             head_forward=args.head_forward, common_point=not args.no_common_point)
     if sharded_mode:          # a shard's period ends with row sums fused into the last step; the restart is a pass of its own
         fam_model["average"] = [fam_model["average"][0] + p.m_pad * 4 + w.N * p.m_pad * (4 + (2 if w.precision == 1 else 0)),
                                 fam_model["average"][1] + 4]
@@ -617,6 +622,8 @@ def parse_args(argv=None):
                     help="one forward launch per layer instead of one launch for all layers")
     ap.add_argument("--head-kernel-always", action="store_true",
                     help="the class layer as one launch of clusters even when its CTAs need more than one wave")
+    ap.add_argument("--no-common-point", action="store_true",
+                    help="an averaging iteration that starts from N equal rows forms and sums the N stepped models one by one")
     ap.add_argument("--head-forward", action="store_true",
                     help="the forward GEMM of layer L - 1 inside the class layer's cluster launch instead of a launch of its own")
     ap.add_argument("--no-head-kernel", action="store_true",

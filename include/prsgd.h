@@ -352,7 +352,9 @@ int prsgd_get_velocity_stacked(prsgd_ctx* ctx, float* dst, int dst_on_device);
  * an averaging iteration that STARTS from N equal rows (every iteration when I = 1, which the paper notes is
  * parallel mini-batch SGD; otherwise the first step after prsgd_average when I divides its number) forms the
  * new average as x - (gamma / N) sum_i G_i: one weight-gradient GEMM per tile over the minibatches of all
- * workers, one step, N row stores (Eq. parallel-sgd-x-update summed over i, then Algorithm 1's average).
+ * workers, one step, N row stores (Eq. parallel-sgd-x-update summed over i, then Algorithm 1's average).  All
+ * such layers share one launch after the iteration's dX launches, and the tiles of its last, partly filled round
+ * are each formed by several CTAs that store a share of the rows (2: whole tiles only).
  * Equal to update-then-average up to fp32 rounding, not bit for bit; deterministic.  0: the N stepped models are
  * formed and summed one by one. */
 #define PRSGD_OPT_COMMON_POINT 15

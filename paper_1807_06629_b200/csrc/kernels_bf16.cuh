@@ -2455,23 +2455,46 @@ inline void tc_launch_update_next(prsgd_ctx* c, const DrawArgs& dr) {
   else tc_launch_update_next_tn<64, false>(c, dr);
 }
 
-// Fused update + average of layer l from a common starting point: one weight-gradient GEMM over the minibatches
-// of all workers (tc_update_common_kernel).
-inline void tc_launch_update_common(prsgd_ctx* c, int l, const DrawArgs& dr) {
+inline bool tc_layer_fuses_average(const prsgd_ctx* c, int l);
+
+// Fused update + average from a common starting point for the layers in `layers` (n of them, 1-based, any order):
+// one weight-gradient GEMM per tile over the minibatches of all workers (tc_update_common_kernel), all layers'
+// tiles in one launch, the tiles of the last partly filled round cut into row ranges.
+inline void tc_launch_update_common(prsgd_ctx* c, const int* layers, int n, const DrawArgs& dr) {
   TcState* st = static_cast<TcState*>(c->tc);
-  const Layer& ly = c->layer[l - 1];
+  CommonMaps maps;
   UpdateCommonArgs a{};
-  a.B = c->B; a.N = c->N; a.tiles_m = (ly.d_out + 127) / 128; a.tiles_n = (ly.d_in + 63) / 64;
-  a.gamma = c->gamma; a.pool = l == 1; a.draw = dr; a.status = c->status;
+  a.B = c->B; a.N = c->N; a.n_seg = n;
+  a.gamma = c->gamma; a.draw = dr; a.status = c->status;
   a.prefetch = c->early_loads ? 1 : 0;
   a.divisor = c->avg_divisor > 0.f ? c->avg_divisor : (float)c->N;
   a.stages = UpdCommonCfg::stages(c->B);
-  const int items = a.tiles_m * a.tiles_n;
-  const int grid = items < st->num_sms ? items : st->num_sms;
-  const TcLayerMaps& mp = st->layer[l - 1];
-  a.params = c->params + ly.w_off; a.shadow = c->shadow + ly.w_off; a.m_pad = c->m_pad; a.d_in = ly.d_in; a.d_out = ly.d_out;
-  launch_pdl(tc_update_common_kernel, dim3(grid), kUpdCommonThreads, UpdCommonCfg::smem(c->B), c->stream, mp.delta_out, mp.act_in,
-             mp.master, a);
+  a.m_pad = c->m_pad;
+  int tiles = 0;
+  for (int i = 0; i < n; ++i) {
+    const int l = layers[i];
+    const Layer& ly = c->layer[l - 1];
+    CommonSeg& g = a.seg[i];
+    g.tiles_n = (ly.d_in + 63) / 64; g.tile0 = tiles; g.pool = l == 1 ? 1 : 0; g.d_in = ly.d_in; g.d_out = ly.d_out;
+    g.params = c->params + ly.w_off; g.shadow = c->shadow + ly.w_off;
+    tiles += ((ly.d_out + 127) / 128) * g.tiles_n;
+    maps.delta[i] = st->layer[l - 1].delta_out; maps.act[i] = st->layer[l - 1].act_in; maps.master[i] = st->layer[l - 1].master;
+  }
+  for (int i = n; i < kCommonMax; ++i) { maps.delta[i] = maps.delta[0]; maps.act[i] = maps.act[0]; maps.master[i] = maps.master[0]; }
+  a.tiles = tiles;
+  const int grid = tiles < st->num_sms ? tiles : st->num_sms;
+  a.full_tiles = tiles / grid * grid;
+  const int rest = tiles - a.full_tiles;                       // tiles of the last, partly filled round
+  a.split = rest > 0 ? grid / rest : 1;
+  if (a.split > c->N) a.split = c->N;
+  if (a.split < 1 || c->common_point == 2) a.split = 1;        // (2: whole tiles only)
+  launch_pdl(tc_update_common_kernel, dim3(grid), kUpdCommonThreads, UpdCommonCfg::smem(c->B), c->stream, maps, a);
+}
+
+// Whether the averaging iteration being enqueued forms layer l's step from the common point in the one launch
+// that follows the dX launches.
+inline bool tc_layer_takes_common_point(const prsgd_ctx* c, int l, const uint8_t* active) {
+  return c->common_point != 0 && c->velocity == nullptr && tc_shared_restart(c, active) && tc_layer_fuses_average(c, l);
 }
 
 // Tile width: forced by PRSGD_OPT_UPDATE_TILE, else chosen per launch.  Wide tiles need fewer TMA
@@ -2483,10 +2506,6 @@ inline void tc_launch_update(prsgd_ctx* c, int l, const DrawArgs& dr, const uint
   const Layer& ly = c->layer[l - 1];
   if (c->velocity != nullptr) {            // momentum step: 64-wide tiles (two stages of master + momentum + output)
     tc_launch_update_tn<64, true>(c, l, dr, active, fuse);
-    return;
-  }
-  if (fuse && c->common_point != 0 && tc_shared_restart(c, active)) {   // every worker starts this step from the same point
-    tc_launch_update_common(c, l, dr);
     return;
   }
   int tile = c->upd_tile;

@@ -12,26 +12,47 @@
 // only stores does).  Four warps read the finished tile from shared memory into registers once and write it N
 // times with 16-byte stores, a quarter warp per 128-byte row segment; the output buffer is free again as soon
 // as it has been read, so the next tile's products and epilogue proceed under the stores.
+// One launch serves every layer that takes this form (their tiles form one list, layer by layer: all of them need
+// only the dZ and activation buffers, which are complete once the dX launches have run), and the tiles of the
+// list's last, partly filled round are cut into row ranges: with 512 tiles on 148 SMs the last round has 68
+// tiles, each then formed by two CTAs that store eight rows apiece (forming a tile is hidden under the previous
+// tile's stores; storing is what takes time).
 // The result equals update-then-average up to fp32 rounding (one rounding of the summed gradient instead of N
 // roundings of the stepped models); it is deterministic (fixed worker order inside the accumulator).
 #pragma once
 
 namespace prsgd {
 
+constexpr int kCommonMax = 8;     // layers one launch can serve
+
+struct CommonSeg {
+  int tiles_n;               // 64-column tiles of d_{l-1}
+  int tile0;                 // index of the layer's first tile in the launch's list
+  int pool;                  // layer 1: the activation operand is the drawn block of the data pool
+  int d_in, d_out;
+  float* params;             // fp32 store + offset of W_l (row stride m_pad elements)
+  uint16_t* shadow;          // bf16 copy + offset of W_l
+};
+
+struct CommonMaps {
+  CUtensorMap delta[kCommonMax];   // bf16 dZ_l, box {64, B, 1}
+  CUtensorMap act[kCommonMax];     // bf16 a_{l-1} (the data pool for layer 1), box {64, B, 1}
+  CUtensorMap master[kCommonMax];  // fp32 W_l, box {32, 128, 1}
+};
+
 struct UpdateCommonArgs {
   int B, N;
-  int tiles_m, tiles_n;      // 128-row tiles of d_l, 64-column tiles of d_{l-1}
+  int n_seg, tiles;          // layers and tiles in the list
+  int full_tiles;            // the first full_tiles tiles are stored whole (a multiple of the grid size)
+  int split;                 // each later tile is shared by `split` CTAs, which store N / split rows each
   float gamma;
-  int pool;                  // layer 1: the activation operand is the drawn block of the data pool
   DrawArgs draw;
   DeviceStatus* status;
   int prefetch;              // 1: the first master tile may be requested before the previous launch has completed
   float divisor;             // the summed models N x - gamma sum_i G_i are divided by this (N; 1 leaves the row SUM)
   int stages;
-  float* params;             // fp32 store + offset of W_l (row stride m_pad elements)
-  uint16_t* shadow;          // bf16 copy + offset of W_l
   int64_t m_pad;
-  int d_in, d_out;
+  CommonSeg seg[kCommonMax];
 };
 
 constexpr int kUpdCommonThreads = 320;   // warp 0 loader, 1 MMA, 2..5 epilogue, 6..9 row stores
@@ -48,10 +69,8 @@ struct UpdCommonCfg {
   static size_t smem(int B) { return (size_t)stages(B) * stage(B) + kBuf + 1024 + 512; }
 };
 
-__global__ void __launch_bounds__(kUpdCommonThreads, 1) tc_update_common_kernel(const __grid_constant__ CUtensorMap mapDelta,
-                                                                                const __grid_constant__ CUtensorMap mapAct,
-                                                                                const __grid_constant__ CUtensorMap mapMaster,
-                                                                                const UpdateCommonArgs a) {
+__global__ void __launch_bounds__(kUpdCommonThreads, 1) tc_update_common_kernel(const __grid_constant__ CommonMaps maps,
+                                                                                const __grid_constant__ UpdateCommonArgs a) {
   using namespace ptx;
   using Cfg = UpdCommonCfg;
   extern __shared__ uint8_t smem_raw[];
@@ -74,7 +93,20 @@ __global__ void __launch_bounds__(kUpdCommonThreads, 1) tc_update_common_kernel(
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 260);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int tiles = a.tiles_m * a.tiles_n;
+  // The items of this CTA: whole tiles blockIdx.x, + gridDim.x, ... below full_tiles, then (for the first CTAs) one
+  // tile of the last round, shared with split - 1 neighbours: item -> (tile, first row, end row).
+  const int G = (int)gridDim.x;
+  const int n_whole = a.full_tiles / G;
+  const int tail_tile = a.full_tiles + (int)blockIdx.x / a.split;
+  const int n_items_all = n_whole + (tail_tile < a.tiles ? 1 : 0);
+  auto item_tile = [&](int i) { return i < n_whole ? (int)blockIdx.x + i * G : tail_tile; };
+  auto item_rows = [&](int i, int& nb, int& ne) {
+    if (i < n_whole) { nb = 0; ne = a.N; return; }
+    const int part = (int)blockIdx.x % a.split;
+    nb = (int)((int64_t)a.N * part / a.split);
+    ne = (int)((int64_t)a.N * (part + 1) / a.split);
+  };
+  auto seg_of = [&](int tile) { int si = 0; while (si + 1 < a.n_seg && tile >= a.seg[si + 1].tile0) ++si; return si; };
 
   if (tid == 0) {
     for (int s = 0; s < S; ++s) { mbar_init(full_ops(s), 1); mbar_init(stage_empty(s), 1); }
@@ -82,53 +114,60 @@ __global__ void __launch_bounds__(kUpdCommonThreads, 1) tc_update_common_kernel(
     mbar_init(mst_full, 1); mbar_init(tile_ready, 128); mbar_init(out_free, 128);
     *abort_flag = *(volatile unsigned int*)&a.status->error != 0u ? 1 : 0;   // an earlier expired wait: no-op (see tc_stream_kernel)
     fence_mbar_init();
-    prefetch_tensormap(&mapDelta); prefetch_tensormap(&mapAct); prefetch_tensormap(&mapMaster);
+    for (int i = 0; i < a.n_seg; ++i) { prefetch_tensormap(&maps.delta[i]); prefetch_tensormap(&maps.act[i]); prefetch_tensormap(&maps.master[i]); }
   }
   if (warp == 1) { tmem_alloc(smem_u32(tmem_slot), 128u); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   // the common point is read from worker 0's row (every row holds the same bits)
-  auto load_master = [&](int m0, int n0) {
+  auto load_master = [&](int tile) {
+    const int si = seg_of(tile);
+    const int rel = tile - a.seg[si].tile0;
+    const int m0 = (rel / a.seg[si].tiles_n) * 128, n0 = (rel % a.seg[si].tiles_n) * 64;
     mbar_expect_tx(mst_full, Cfg::kMaster);
-    tma_load_3d(buf_u32, &mapMaster, mst_full, n0, m0, 0);
-    tma_load_3d(buf_u32 + 16384u, &mapMaster, mst_full, n0 + 32, m0, 0);
+    tma_load_3d(buf_u32, &maps.master[si], mst_full, n0, m0, 0);
+    tma_load_3d(buf_u32 + 16384u, &maps.master[si], mst_full, n0 + 32, m0, 0);
   };
   // The master tiles were last written an iteration ago (the launch before this one only reads bf16 copies), so
   // the first one is requested while that launch drains.
-  const bool pre = a.prefetch != 0 && *abort_flag == 0 && (int)blockIdx.x < tiles;
-  if (pre && warp == 0 && lane == 0) load_master(((int)blockIdx.x / a.tiles_n) * 128, ((int)blockIdx.x % a.tiles_n) * 64);
+  const bool pre = a.prefetch != 0 && *abort_flag == 0 && n_items_all > 0;
+  if (pre && warp == 0 && lane == 0) load_master(item_tile(0));
   pdl_wait();
   pdl_trigger();
   const uint32_t tmem = *tmem_slot;
-  const int total = *abort_flag != 0 ? 0 : tiles;
+  const int n_items = *abort_flag != 0 ? 0 : n_items_all;
 
-  // Every role walks the same tiles w = blockIdx.x, + gridDim.x, ...; tile number ti of this CTA uses accumulator
-  // ti % 2; `it` counts (tile, worker) operand stages.  (Dealing out (tile, row) pairs instead, so that every CTA
-  // stores the same number of rows, was slower: the tiles that straddle two CTAs are formed twice, and forming a
-  // tile takes almost as long as storing it.)
+  // Every role walks the same items; item number ti of this CTA uses accumulator ti % 2; `it` counts (tile, worker)
+  // operand stages.  (Dealing out (tile, row) pairs in equal runs for ALL tiles, so that every CTA stores the same
+  // number of rows, was slower: every CTA then forms one more tile than it stores, and forming a tile takes a
+  // third of the time of storing it; cutting only the tiles of the last round costs nothing, the extra tile is
+  // formed while the previous one is stored.)
   if (warp == 0 && lane == 0) {
     // ---------------- loader
     uint32_t it = 0, ti = 0;
     bool ok = true;
-    for (int w = blockIdx.x; w < total && ok; w += gridDim.x, ++ti) {
-      const int m0 = (w / a.tiles_n) * 128, n0 = (w % a.tiles_n) * 64;
+    for (; (int)ti < n_items && ok; ++ti) {
+      const int w = item_tile((int)ti);
+      const int si = seg_of(w);
+      const int rel = w - a.seg[si].tile0;
+      const int m0 = (rel / a.seg[si].tiles_n) * 128, n0 = (rel % a.seg[si].tiles_n) * 64;
       if (ti >= 1) ok = mbar_wait(out_free, (ti - 1u) & 1u, abort_flag, a.status, 0x701);   // the store warps hold the previous tile in registers
       if (!ok) break;
-      if (!(pre && ti == 0)) load_master(m0, n0);
+      if (!(pre && ti == 0)) load_master(w);
       for (int n = 0; n < a.N; ++n, ++it) {
         const int s = it % S;
         ok = mbar_wait(stage_empty(s), ((it / S) & 1u) ^ 1u, abort_flag, a.status, 0x702);
         if (!ok) break;
-        const int row0 = a.pool ? (int)draw_block(a.draw.seed, a.draw.worker0 + n, draw_t(a.draw), a.draw.n_blocks) * a.B : 0;
+        const int row0 = a.seg[si].pool ? (int)draw_block(a.draw.seed, a.draw.worker0 + n, draw_t(a.draw), a.draw.n_blocks) * a.B : 0;
         const uint32_t ops = ops_u32(s);
         mbar_expect_tx(full_ops(s), 3u * op_box);
-        tma_load_3d(ops, &mapDelta, full_ops(s), m0, 0, n);
-        tma_load_3d(ops + op_box, &mapDelta, full_ops(s), m0 + 64, 0, n);
-        tma_load_3d(ops + 2u * op_box, &mapAct, full_ops(s), n0, row0, n);
+        tma_load_3d(ops, &maps.delta[si], full_ops(s), m0, 0, n);
+        tma_load_3d(ops + op_box, &maps.delta[si], full_ops(s), m0 + 64, 0, n);
+        tma_load_3d(ops + 2u * op_box, &maps.act[si], full_ops(s), n0, row0, n);
       }
     }
-    if (total == 0 && pre) {           // the launch turned into a no-op: let the early tile land
+    if (n_items == 0 && pre) {         // the launch turned into a no-op: let the early tile land
       const long long t0 = clock64();
       while (!mbar_try_wait(mst_full, 0u) && clock64() - t0 < 200000000ll) {}
     }
@@ -138,7 +177,7 @@ __global__ void __launch_bounds__(kUpdCommonThreads, 1) tc_update_common_kernel(
     const int ksteps = a.B / 16;
     uint32_t it = 0, ti = 0;
     bool ok = true;
-    for (int w = blockIdx.x; w < total && ok; w += gridDim.x, ++ti) {
+    for (; (int)ti < n_items && ok; ++ti) {
       const int q = ti & 1;
       ok = mbar_wait(acc_empty(q), ((ti >> 1) & 1u) ^ 1u, abort_flag, a.status, 0x703);
       if (!ok) break;
@@ -165,8 +204,13 @@ __global__ void __launch_bounds__(kUpdCommonThreads, 1) tc_update_common_kernel(
     const int j = t & 7, rsub = t >> 3;                   // chunk within the box row; row = rsub + 16 i
     uint32_t ti = 0;
     bool ok = true;
-    for (int w = blockIdx.x; w < total && ok; w += gridDim.x, ++ti) {
-      const int m0 = (w / a.tiles_n) * 128, n0 = (w % a.tiles_n) * 64;
+    for (; (int)ti < n_items && ok; ++ti) {
+      const int w = item_tile((int)ti);
+      const CommonSeg& sg = a.seg[seg_of(w)];
+      const int rel = w - sg.tile0;
+      const int m0 = (rel / sg.tiles_n) * 128, n0 = (rel % sg.tiles_n) * 64;
+      int nb, ne;
+      item_rows((int)ti, nb, ne);
       ok = __all_sync(0xffffffffu, mbar_wait(tile_ready, ti & 1u, abort_flag, a.status, 0x705));
       if (!ok) break;
       const uint8_t* buf = gen;
@@ -177,13 +221,13 @@ __global__ void __launch_bounds__(kUpdCommonThreads, 1) tc_update_common_kernel(
         v[i] = *reinterpret_cast<const uint4*>(buf + (i >> 3) * 16384 + rr * 128 + ((j ^ (rr & 7)) << 4));
       }
       mbar_arrive(out_free);                              // the buffer may take the next tile's master tile
-      float* prow = a.params + (int64_t)(m0 + rsub) * a.d_in + n0 + 4 * j;
-      uint16_t* srow = a.shadow + (int64_t)(m0 + rsub) * a.d_in + n0 + 8 * j;
-      const int64_t step = 16 * (int64_t)a.d_in;          // 16 rows further down
-      for (int n = 0; n < a.N; ++n) {
+      float* prow = sg.params + (int64_t)nb * a.m_pad + (int64_t)(m0 + rsub) * sg.d_in + n0 + 4 * j;
+      uint16_t* srow = sg.shadow + (int64_t)nb * a.m_pad + (int64_t)(m0 + rsub) * sg.d_in + n0 + 8 * j;
+      const int64_t step = 16 * (int64_t)sg.d_in;         // 16 rows further down
+      for (int n = nb; n < ne; ++n) {
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-          if (m0 + rsub + 16 * i < a.d_out) {             // (rows past the layer's height do not exist)
+          if (m0 + rsub + 16 * i < sg.d_out) {            // (rows past the layer's height do not exist)
             *reinterpret_cast<uint4*>(prow + i * step) = v[i];
             *reinterpret_cast<uint4*>(prow + i * step + 32) = v[8 + i];
             *reinterpret_cast<uint4*>(srow + i * step) = v[16 + i];
@@ -204,7 +248,7 @@ __global__ void __launch_bounds__(kUpdCommonThreads, 1) tc_update_common_kernel(
     const float c1 = __fdiv_rn((float)a.N, a.divisor), c2 = __fdiv_rn(a.gamma, a.divisor);
     uint32_t ti = 0;
     bool ok = true;
-    for (int w = blockIdx.x; w < total && ok; w += gridDim.x, ++ti) {
+    for (; (int)ti < n_items && ok; ++ti) {
       const int ob = ti & 1;                              // the accumulator
       ok = mbar_wait(mst_full, ti & 1u, abort_flag, a.status, 0x706) && mbar_wait(acc_full(ob), (ti >> 1) & 1u, abort_flag, a.status, 0x707);
       ok = __all_sync(0xffffffffu, ok);

@@ -348,10 +348,18 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging, bool more_follow) {
     tc_launch_head(c, dr, act_mask, head_fwd);
     LAUNCH_CHECK(c);
   }
+  int common_layers[PRSGD_MAX_LAYERS], n_common = 0;     // layers whose averaged step is formed from the common point, in one launch at the end
   for (int l = L; l >= 1; --l) {          // dX_l reads W_l before the update of layer l overwrites it
     const bool fuse_l = fuse && tc_layer_fuses_average(c, l);
     if (l == L && head) {
       // (forward, step and dZ_{L-1} of this layer were the head launch)
+    } else if (fuse_l && n_common < kCommonMax && tc_layer_takes_common_point(c, l, act_mask)) {
+      if (l > 1) {
+        prof_begin(c, PRSGD_KERNEL_DX);
+        tc_launch_dx(c, l, dr, act_mask);
+        LAUNCH_CHECK(c);
+      }
+      common_layers[n_common++] = l;      // (needs only dZ_l and a_{l-1}, which nothing later in the iteration changes)
     } else if (l > 1 && dx_in_upd && !fuse_l && (c->dx_in_update == 2 || tc_layer_folds_dx(c, l))) {
       prof_begin(c, PRSGD_KERNEL_UPDATE);
       tc_launch_update_dx(c, l);
@@ -383,6 +391,11 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging, bool more_follow) {
         LAUNCH_CHECK(c);
       }
     }
+  }
+  if (n_common > 0) {
+    prof_begin(c, PRSGD_KERNEL_UPDATE_AVERAGE);
+    tc_launch_update_common(c, common_layers, n_common, dr);
+    LAUNCH_CHECK(c);
   }
   if (!epi) {
     prof_begin(c, PRSGD_KERNEL_MISC);
@@ -736,7 +749,9 @@ void period_key(const prsgd_ctx* c, uint64_t (&key)[13]) {
   key[7] = (uint64_t)c->average_velocity; key[8] = reinterpret_cast<uint64_t>(c->X);
   key[9] = reinterpret_cast<uint64_t>(c->Y); key[10] = (uint64_t)c->worker0; key[11] = (uint64_t)c->fused_epilogues | ((uint64_t)c->early_loads << 1) | ((uint64_t)c->next_forward << 2) | ((uint64_t)c->dx_in_update << 3);
   key[12] = (c->rows_identical ? 1u : 0u) | ((uint64_t)c->shared_restart << 1) | ((uint64_t)c->forward_chain << 2) |
-            ((uint64_t)c->worker_groups << 3) | ((uint64_t)c->dx_shared_pair << 6) | ((uint64_t)c->head_kernel << 7) | ((uint64_t)c->common_point << 9) | ((uint64_t)c->split_blocks << 10) | ((uint64_t)c->head_forward << 12) | ((uint64_t)c->merged_small_average << 13);   // the period's first iteration may share reads
+            ((uint64_t)c->worker_groups << 3) | ((uint64_t)c->dx_shared_pair << 6) | ((uint64_t)c->head_kernel << 7) |
+            ((uint64_t)c->common_point << 9) | ((uint64_t)c->split_blocks << 11) | ((uint64_t)c->head_forward << 13) |
+            ((uint64_t)c->merged_small_average << 14);      // (rows_identical: the period's first iteration may share reads)
 }
 
 // One whole averaging period (I iterations starting right after an average) as a CUDA graph: the
@@ -1142,7 +1157,11 @@ int prsgd_set_option(prsgd_ctx* c, int32_t option, int64_t value) {
   if (option == PRSGD_OPT_SHARED_RESTART) { c->shared_restart = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_FORWARD_CHAIN) { c->forward_chain = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_DX_SHARED_PAIR) { c->dx_shared_pair = value != 0; return PRSGD_OK; }
-  if (option == PRSGD_OPT_COMMON_POINT) { c->common_point = value != 0; return PRSGD_OK; }
+  if (option == PRSGD_OPT_COMMON_POINT) {
+    if (value < 0 || value > 2) return fail(c, PRSGD_ERR_ARG, "PRSGD_OPT_COMMON_POINT takes 0, 1 or 2");
+    c->common_point = (int)value;
+    return PRSGD_OK;
+  }
   if (option == PRSGD_OPT_HEAD_FORWARD) { c->head_forward = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_MERGED_SMALL_AVERAGE) { c->merged_small_average = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_SPLIT_BLOCKS) {
