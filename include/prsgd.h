@@ -335,6 +335,16 @@ int prsgd_get_velocity_stacked(prsgd_ctx* ctx, float* dst, int dst_on_device);
  * launches of their own.  The two forms agree to fp32 rounding of the logits (different summation order, fast
  * exponential), not bit for bit; each is deterministic. */
 #define PRSGD_OPT_HEAD_KERNEL 14
+/* PRSGD_OPT_TILED_WEIGHTS (default 1, tensor-core path): inside a row of the store, of the bf16 copy and of the
+ * momentum buffers the weight segment of a hidden layer whose height d_l is a multiple of 128 is kept as 128 x 64
+ * tiles, one after another (tile (r / 128, c / 64) at index (r / 128) (d_{l-1} / 64) + c / 64, row-major inside
+ * a tile), so that every tile a kernel loads or stores is one contiguous piece of memory; the class layer, layers of
+ * other heights and the fp32 path keep row-major segments.  Nothing changes at this interface: every call that
+ * takes or returns parameters (prsgd_set_params*, prsgd_get_params*, prsgd_get_average*, prsgd_get_velocity_stacked)
+ * speaks the canonical order, offsets and m_pad are the same, and prsgd_partial_sum / prsgd_assign_rows work on
+ * columns of the rows as they are (all ranks of a job use the same setting).  Changing the option re-orders the
+ * store in place (a pass over all rows).  Same bits either way. */
+#define PRSGD_OPT_TILED_WEIGHTS 19
 /* PRSGD_OPT_MERGED_SMALL_AVERAGE (default 1, tensor-core path, fused averaging iterations): the weight segments of
  * layers too small for the fused update + average (the class layer) are averaged by the launch that averages the
  * bias segments, at the end of the iteration, instead of by a launch of their own after the layer's update.  Same

@@ -162,4 +162,30 @@ __global__ void __launch_bounds__(256) refresh_shadow_kernel(const float* __rest
   reinterpret_cast<uint2*>(S)[c] = make_uint2(pack_bf16x2(v.x, v.y), pack_bf16x2(v.z, v.w));
 }
 
+// Rows of the store (or of the momentum buffers) <-> rows in canonical order (W_1 row-major, b_1, W_2, ...
+// without gaps).  A tile-major weight segment (see WTile) is permuted on the way; everything else is a copy.
+// Grid (blocks, 2 L, rows): blockIdx.y = 2 (l - 1) for W_l, + 1 for b_l.
+struct CanonArgs {
+  int L;
+  int64_t w_off[PRSGD_MAX_LAYERS], b_off[PRSGD_MAX_LAYERS];       // offsets inside a store row
+  int64_t w_pos[PRSGD_MAX_LAYERS], b_pos[PRSGD_MAX_LAYERS];       // offsets inside a canonical row
+  int d_out[PRSGD_MAX_LAYERS];
+  WTile wt[PRSGD_MAX_LAYERS];
+};
+
+__global__ void __launch_bounds__(256) canonical_copy_kernel(float* __restrict__ store, int64_t store_stride,
+                                                             float* __restrict__ lin, int64_t lin_stride,
+                                                             const CanonArgs a, int to_store) {
+  const int l = blockIdx.y >> 1, is_bias = blockIdx.y & 1;
+  float* srow = store + (int64_t)blockIdx.z * store_stride + (is_bias ? a.b_off[l] : a.w_off[l]);
+  float* lrow = lin + (int64_t)blockIdx.z * lin_stride + (is_bias ? a.b_pos[l] : a.w_pos[l]);
+  const int d_in = a.wt[l].d_in;
+  const int64_t len = is_bias ? (int64_t)a.d_out[l] : (int64_t)a.d_out[l] * d_in;
+  for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < len; j += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t o = (is_bias || !a.wt[l].tiled) ? j : wtile_offset(a.wt[l], (int)(j / d_in), (int)(j % d_in));
+    if (to_store) srow[o] = lrow[j];
+    else lrow[j] = srow[o];
+  }
+}
+
 }  // namespace prsgd

@@ -104,6 +104,7 @@ struct StreamArgs {
   float* bias_vel;           // its momentum segment, or nullptr
   float gamma, mu;
   // Softmax cross-entropy gradient in the epilogue of the last forward GEMM (needs tiles_m == 1)
+  WTile wt;                  // order of the weight segment's elements
   int prefetch;              // 1: the weight tiles may be requested before the previous launch has completed
   int shared_w;              // 1: every worker's weights hold the same bits (the launch follows a node average with
                              // nothing in between), so every item reads worker 0's tiles: one HBM read serves all N
@@ -182,10 +183,10 @@ __global__ void __launch_bounds__(kStreamThreads, 1) tc_stream_kernel(const __gr
     for (int j = 0; j < 2; ++j) {
       const int k0 = (2 * ks + j) * 64;              // a block past the end of K is zero-filled by TMA
       if (MODE == TC_DX) {
-        tma_load_3d(sa + j * kTileA, &mapW, full_bar(s), m0, k0, n);
-        tma_load_3d(sa + j * kTileA + 8192u, &mapW, full_bar(s), m0 + 64, k0, n);
+        tma_load_w(sa + j * kTileA, &mapW, full_bar(s), a.wt, m0, k0, n);
+        tma_load_w(sa + j * kTileA + 8192u, &mapW, full_bar(s), a.wt, m0 + 64, k0, n);
       } else {
-        tma_load_3d(sa + j * kTileA, &mapW, full_bar(s), k0, m0, n);
+        tma_load_w(sa + j * kTileA, &mapW, full_bar(s), a.wt, k0, m0, n);
       }
     }
   };
@@ -417,6 +418,7 @@ struct ChainSeg {
   int pool;                  // operand B rows come from the data pool at the drawn block (layer 1)
   int prefetch;              // the weight tiles may be requested before the previous launch has completed
   int item0;                 // index of the layer's first item in the list
+  WTile wt;                  // order of the weight segment's elements
   uint16_t* out_bk;          // bf16 [N][B][ld_out]
   float* out_f32;            // fp32 [N][B][ld_out] (logits without the softmax epilogue)
   const float* bias;         // params + b_off; worker stride ChainArgs::bias_stride
@@ -483,7 +485,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) tc_forward_chain_kernel(con
   auto load_weights = [&](int si, int s, int ks, int m0, int n) {
     const uint32_t sa = base + (uint32_t)s * stage_bytes;
 #pragma unroll
-    for (int j = 0; j < 2; ++j) tma_load_3d(sa + j * kTileA, &maps.w[si], full_bar(s), (2 * ks + j) * 64, m0, n);
+    for (int j = 0; j < 2; ++j) tma_load_w(sa + j * kTileA, &maps.w[si], full_bar(s), a.seg[si].wt, (2 * ks + j) * 64, m0, n);
   };
   auto load_operand = [&](int si, int s, int ks, int row0, int n) {
     const uint32_t sb = base + (uint32_t)s * stage_bytes + 2u * kTileA;
@@ -705,6 +707,7 @@ struct UpdateArgs {
   DrawArgs draw;
   const uint8_t* active;
   DeviceStatus* status;
+  WTile wt;                // order of the weight segment's elements
   int prefetch;            // 1: master tiles may be requested before the previous launch has completed
   float divisor;           // fused form: the summed models are divided by this (N; 1 leaves the local row SUM in every
                            // row, the first half of an average whose other rows live on other GPUs)
@@ -805,10 +808,10 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
     mbar_expect_tx(full_w(s), Cfg::kMaster + Cfg::kVel);
     const int nm = (FUSE && a.shared_w) ? 0 : n;
 #pragma unroll
-    for (int q = 0; q < NB32; ++q) tma_load_3d(master_u32(s) + q * 16384u, &mapMaster, full_w(s), n0 + 32 * q, m0, nm);
+    for (int q = 0; q < NB32; ++q) tma_load_w(master_u32(s) + q * 16384u, &mapMaster, full_w(s), a.wt, n0 + 32 * q, m0, nm);
     if (MOM) {
 #pragma unroll
-      for (int q = 0; q < NB32; ++q) tma_load_3d(vel_u32(s) + q * 16384u, &mapVel, full_w(s), n0 + 32 * q, m0, n);
+      for (int q = 0; q < NB32; ++q) tma_load_w(vel_u32(s) + q * 16384u, &mapVel, full_w(s), a.wt, n0 + 32 * q, m0, n);
     }
   };
   // The master (and momentum) tiles were last written an iteration ago, so those of the first items
@@ -903,13 +906,13 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
     bool ok = true;
     auto store_tile = [&](int s, int m0, int n0, int n) {
 #pragma unroll
-      for (int q = 0; q < NB32; ++q) tma_store_3d(&mapMaster, master_u32(s) + q * 16384u, n0 + 32 * q, m0, n);
+      for (int q = 0; q < NB32; ++q) tma_store_w(&mapMaster, master_u32(s) + q * 16384u, a.wt, n0 + 32 * q, m0, n);
       if (MOM) {
 #pragma unroll
-        for (int q = 0; q < NB32; ++q) tma_store_3d(&mapVel, vel_u32(s) + q * 16384u, n0 + 32 * q, m0, n);
+        for (int q = 0; q < NB32; ++q) tma_store_w(&mapVel, vel_u32(s) + q * 16384u, a.wt, n0 + 32 * q, m0, n);
       }
 #pragma unroll
-      for (int h = 0; h < NB64; ++h) tma_store_3d(&mapShadow, ops_u32(s) + h * 16384u, n0 + 64 * h, m0, n);
+      for (int h = 0; h < NB64; ++h) tma_store_w(&mapShadow, ops_u32(s) + h * 16384u, a.wt, n0 + 64 * h, m0, n);
     };
     for (int w = blockIdx.x; w < total_items && ok; w += gridDim.x) {
       const int tile = FUSE ? w : w % tiles;
@@ -933,9 +936,9 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
         // tile's operand loads for as long as the memory system takes to absorb it
         for (int n = 0; n < a.N; ++n) {
 #pragma unroll
-          for (int q = 0; q < NB32; ++q) tma_store_3d(&mapMaster, out_u32 + q * 16384u, n0 + 32 * q, m0, n);
+          for (int q = 0; q < NB32; ++q) tma_store_w(&mapMaster, out_u32 + q * 16384u, a.wt, n0 + 32 * q, m0, n);
 #pragma unroll
-          for (int h = 0; h < NB64; ++h) tma_store_3d(&mapShadow, out_u32 + Cfg::kMaster + h * 16384u, n0 + 64 * h, m0, n);
+          for (int h = 0; h < NB64; ++h) tma_store_w(&mapShadow, out_u32 + Cfg::kMaster + h * 16384u, a.wt, n0 + 64 * h, m0, n);
           tma_commit_group();
           tma_wait_group_read0();
         }
@@ -952,13 +955,13 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
           if (n == a.N - 1) {
             for (int rr = 0; rr < a.N; ++rr) {
 #pragma unroll
-              for (int q = 0; q < NB32; ++q) tma_store_3d(&mapMaster, master_u32(s) + q * 16384u, n0 + 32 * q, m0, rr);
+              for (int q = 0; q < NB32; ++q) tma_store_w(&mapMaster, master_u32(s) + q * 16384u, a.wt, n0 + 32 * q, m0, rr);
 #pragma unroll
-              for (int h = 0; h < NB64; ++h) tma_store_3d(&mapShadow, ops_u32(s) + h * 16384u, n0 + 64 * h, m0, rr);
+              for (int h = 0; h < NB64; ++h) tma_store_w(&mapShadow, ops_u32(s) + h * 16384u, a.wt, n0 + 64 * h, m0, rr);
             }
           }
 #pragma unroll
-          for (int q = 0; q < NB32; ++q) tma_store_3d(&mapVel, vel_u32(s) + q * 16384u, n0 + 32 * q, m0, n);
+          for (int q = 0; q < NB32; ++q) tma_store_w(&mapVel, vel_u32(s) + q * 16384u, a.wt, n0 + 32 * q, m0, n);
           tma_commit_group();
           tma_wait_group_read0();
           mbar_arrive(stage_empty(s));
@@ -1202,6 +1205,7 @@ struct UpdateNextArgs {
   float mu;                  // momentum form: v <- mu v + G, x <- x - gamma v
   const uint8_t* active;     // per-worker flag or nullptr: an inactive worker's row blocks are skipped
   SplitArgs split;           // row blocks cut at run boundaries (never together with a worker mask)
+  WTile wt;                  // order of the weight segment's elements
 };
 
 template <int TN, bool MOM> struct UpdNextCfg {
@@ -1327,10 +1331,10 @@ __global__ void __launch_bounds__(kUpdBlkThreads, 1) tc_update_next_kernel(const
         }
         mbar_expect_tx(full_w(s), Cfg::kMaster + Cfg::kVel);
 #pragma unroll
-        for (int q = 0; q < NB32; ++q) tma_load_3d(master_u32(s) + q * 16384u, &mapMaster, full_w(s), n0 + 32 * q, m0, n);
+        for (int q = 0; q < NB32; ++q) tma_load_w(master_u32(s) + q * 16384u, &mapMaster, full_w(s), a.wt, n0 + 32 * q, m0, n);
         if (MOM) {
 #pragma unroll
-          for (int q = 0; q < NB32; ++q) tma_load_3d(vel_u32(s) + q * 16384u, &mapVel, full_w(s), n0 + 32 * q, m0, n);
+          for (int q = 0; q < NB32; ++q) tma_load_w(vel_u32(s) + q * 16384u, &mapVel, full_w(s), a.wt, n0 + 32 * q, m0, n);
         }
       }
     }
@@ -1419,10 +1423,10 @@ __global__ void __launch_bounds__(kUpdBlkThreads, 1) tc_update_next_kernel(const
         ok = mbar_wait(tile_ready(s), ph, abort_flag, a.status, 0x406);
         if (!ok) break;
 #pragma unroll
-        for (int q = 0; q < NB32; ++q) tma_store_3d(&mapMaster, master_u32(s) + q * 16384u, n0 + 32 * q, m0, n);
+        for (int q = 0; q < NB32; ++q) tma_store_w(&mapMaster, master_u32(s) + q * 16384u, a.wt, n0 + 32 * q, m0, n);
         if (MOM) {
 #pragma unroll
-          for (int q = 0; q < NB32; ++q) tma_store_3d(&mapVel, vel_u32(s) + q * 16384u, n0 + 32 * q, m0, n);
+          for (int q = 0; q < NB32; ++q) tma_store_w(&mapVel, vel_u32(s) + q * 16384u, a.wt, n0 + 32 * q, m0, n);
         }
         tma_commit_group();
         tma_wait_group_read0();
@@ -1601,6 +1605,7 @@ struct UpdateDxArgs {
   float mu;                  // momentum form: v <- mu v + G, x <- x - gamma v
   float* bias_vel;           // momentum segment of b_{l-1}, or nullptr
   const uint8_t* active;     // per-worker flag or nullptr: an inactive worker's column blocks are skipped
+  WTile wt;                  // order of the weight segment's elements
 };
 
 // Two stage layouts.  Own pair (SP = false): every stage holds fp32 master | momentum | bf16 old | bf16 new (first
@@ -1725,10 +1730,10 @@ __global__ void __launch_bounds__(kUpdBlkThreads, 1) tc_update_dx_kernel(const _
         for (int h = 0; h < NB64; ++h) tma_load_3d(act_u32(s) + h * op_box, &mapAct, full_ops(s), n0 + 64 * h, 0, n);
         mbar_expect_tx(full_w(s), Cfg::kMaster + Cfg::kVel);
 #pragma unroll
-        for (int q = 0; q < NB32; ++q) tma_load_3d(master_u32(s) + q * 16384u, &mapMaster, full_w(s), n0 + 32 * q, m0, n);
+        for (int q = 0; q < NB32; ++q) tma_load_w(master_u32(s) + q * 16384u, &mapMaster, full_w(s), a.wt, n0 + 32 * q, m0, n);
         if (MOM) {
-          tma_load_3d(vel_u32(s), &mapVel, full_w(s), n0, m0, n);
-          tma_load_3d(vel_u32(s) + 16384u, &mapVel, full_w(s), n0 + 32, m0, n);
+          tma_load_w(vel_u32(s), &mapVel, full_w(s), a.wt, n0, m0, n);
+          tma_load_w(vel_u32(s) + 16384u, &mapVel, full_w(s), a.wt, n0 + 32, m0, n);
         }
       }
     }
@@ -1803,13 +1808,13 @@ __global__ void __launch_bounds__(kUpdBlkThreads, 1) tc_update_dx_kernel(const _
         ok = mbar_wait(tile_ready(s), ph, abort_flag, a.status, 0x506);
         if (!ok) break;
 #pragma unroll
-        for (int h = 0; h < NB64; ++h) tma_store_3d(&mapShadow, new_u32(s) + h * 16384u, n0 + 64 * h, m0, n);
+        for (int h = 0; h < NB64; ++h) tma_store_w(&mapShadow, new_u32(s) + h * 16384u, a.wt, n0 + 64 * h, m0, n);
         if (kSharedPair) tma_commit_group();              // a group of its own: the shared pair is released first
 #pragma unroll
-        for (int q = 0; q < NB32; ++q) tma_store_3d(&mapMaster, master_u32(s) + q * 16384u, n0 + 32 * q, m0, n);
+        for (int q = 0; q < NB32; ++q) tma_store_w(&mapMaster, master_u32(s) + q * 16384u, a.wt, n0 + 32 * q, m0, n);
         if (MOM) {
-          tma_store_3d(&mapVel, vel_u32(s), n0, m0, n);
-          tma_store_3d(&mapVel, vel_u32(s) + 16384u, n0 + 32, m0, n);
+          tma_store_w(&mapVel, vel_u32(s), a.wt, n0, m0, n);
+          tma_store_w(&mapVel, vel_u32(s) + 16384u, a.wt, n0 + 32, m0, n);
         }
         tma_commit_group();
         if (kSharedPair) {
@@ -2066,6 +2071,44 @@ __global__ void __launch_bounds__(32) wait_expiry_kernel(DeviceStatus* status, l
 // ---------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------
+// Order of layer l's weight segment (1-based l): tile-major for hidden layers whose height is a multiple of 128
+// (the class layer, whose tiles the head kernel loads with only as many rows as it has, stays row-major).
+inline bool tc_layer_tiled(const prsgd_ctx* c, int l) {
+  const Layer& ly = c->layer[l - 1];
+  return c->precision == PRSGD_PRECISION_BF16 && c->tiled_weights != 0 && l < c->L && ly.d_out % 128 == 0 && ly.d_in % 64 == 0;
+}
+inline WTile tc_wtile(const prsgd_ctx* c, int l) {
+  WTile t;
+  t.tiled = tc_layer_tiled(c, l) ? 1 : 0; t.tn = c->layer[l - 1].d_in / 64; t.d_in = c->layer[l - 1].d_in;
+  return t;
+}
+
+// tensor maps over a weight segment of layer l: {d_in, d_out, N} row-major, {64, tiles * 128, N} tile-major
+inline int tc_make_weight_map(const prsgd_ctx* c, CUtensorMap* m, bool fp32, const void* seg, int l, uint32_t b0, uint32_t b1, std::string* err) {
+  const Layer& ly = c->layer[l - 1];
+  const uint64_t esz = fp32 ? 4 : 2;
+  if (tc_layer_tiled(c, l)) {
+    const uint64_t tiles = (uint64_t)(ly.d_out / 128) * (uint64_t)(ly.d_in / 64);
+    return make_map3(m, fp32, seg, 64, tiles * 128, (uint64_t)c->N, 64 * esz, (uint64_t)c->m_pad * esz, b0, b1, err);
+  }
+  return make_map3(m, fp32, seg, (uint64_t)ly.d_in, (uint64_t)ly.d_out, (uint64_t)c->N, (uint64_t)ly.d_in * esz, (uint64_t)c->m_pad * esz, b0, b1, err);
+}
+
+// (re)builds the maps of all weight segments: at creation and whenever the order of the segments changes
+inline int tc_make_weight_maps(prsgd_ctx* c, std::string* err) {
+  TcState* st = static_cast<TcState*>(c->tc);
+  int rc = PRSGD_OK;
+  for (int l = 1; l <= c->L && rc == PRSGD_OK; ++l) {
+    const Layer& ly = c->layer[l - 1];
+    TcLayerMaps& mp = st->layer[l - 1];
+    rc = tc_make_weight_map(c, &mp.shadow_k, false, c->shadow + ly.w_off, l, 64, 128, err);
+    if (rc == PRSGD_OK) rc = tc_make_weight_map(c, &mp.shadow_mn, false, c->shadow + ly.w_off, l, 64, 64, err);
+    if (rc == PRSGD_OK) rc = tc_make_weight_map(c, &mp.master, true, c->params + ly.w_off, l, 32, 128, err);
+    if (rc == PRSGD_OK && c->velocity != nullptr) rc = tc_make_weight_map(c, &mp.velocity, true, c->velocity + ly.w_off, l, 32, 128, err);
+  }
+  return rc;
+}
+
 inline int tc_create(prsgd_ctx* c, std::string* err) {
   if (c->B > 64) { *err = "BF16 precision supports batch 16, 32 or 64"; return PRSGD_ERR_ALIGN; }
   TcState* st = new (std::nothrow) TcState();
@@ -2074,15 +2117,11 @@ inline int tc_create(prsgd_ctx* c, std::string* err) {
   if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device) == cudaSuccess && sms > 0) st->num_sms = sms;
   const uint64_t N = c->N, B = c->B;
   int rc = PRSGD_OK;
+  c->tc = st;
+  rc = tc_make_weight_maps(c, err);
+  c->tc = nullptr;
   for (int l = 1; l <= c->L && rc == PRSGD_OK; ++l) {
-    const Layer& ly = c->layer[l - 1];
     TcLayerMaps& mp = st->layer[l - 1];
-    const uint64_t din = ly.d_in, dout = ly.d_out;
-    const uint16_t* sh = c->shadow + ly.w_off;
-    const float* ms = c->params + ly.w_off;
-    rc = make_map3(&mp.shadow_k, false, sh, din, dout, N, din * 2, (uint64_t)c->m_pad * 2, 64, 128, err);
-    if (rc == PRSGD_OK) rc = make_map3(&mp.shadow_mn, false, sh, din, dout, N, din * 2, (uint64_t)c->m_pad * 2, 64, 64, err);
-    if (rc == PRSGD_OK) rc = make_map3(&mp.master, true, ms, din, dout, N, din * 4, (uint64_t)c->m_pad * 4, 32, 128, err);
     const uint64_t ld = c->buf.ld[l];
     if (rc == PRSGD_OK) rc = make_map3(&mp.delta_out, false, c->buf.delta_bk[l], ld, B, N, ld * 2, B * ld * 2, 64, (uint32_t)B, err);
     if (rc == PRSGD_OK && l > 1) {
@@ -2139,17 +2178,7 @@ inline void tc_destroy(prsgd_ctx* c) {
   c->tc = nullptr;
 }
 
-inline int tc_bind_velocity(prsgd_ctx* c, std::string* err) {
-  TcState* st = static_cast<TcState*>(c->tc);
-  for (int l = 1; l <= c->L; ++l) {
-    const Layer& ly = c->layer[l - 1];
-    const uint64_t din = ly.d_in, dout = ly.d_out;
-    int rc = make_map3(&st->layer[l - 1].velocity, true, c->velocity + ly.w_off, din, dout, (uint64_t)c->N, din * 4,
-                       (uint64_t)c->m_pad * 4, 32, 128, err);
-    if (rc != PRSGD_OK) return rc;
-  }
-  return PRSGD_OK;
-}
+inline int tc_bind_velocity(prsgd_ctx* c, std::string* err) { return tc_make_weight_maps(c, err); }
 
 inline int tc_bind_data(prsgd_ctx* c, std::string* err) {
   TcState* st = static_cast<TcState*>(c->tc);
@@ -2179,7 +2208,7 @@ inline void tc_launch_forward(prsgd_ctx* c, int l, const DrawArgs& dr, const uin
   const Layer& ly = c->layer[l - 1];
   StreamArgs a{};
   a.B = c->B; a.N = c->N; a.k_steps = (ly.d_in / 64 + 1) / 2; a.M_total = ly.d_out; a.tiles_m = (ly.d_out + 127) / 128;
-  a.stages = stream_stages(c->B);
+  a.stages = stream_stages(c->B); a.wt = tc_wtile(c, l);
   a.pool = l == 1; a.draw = dr; a.ld_out = c->buf.ld[l];
   a.out_bk = c->buf.act_bk[l]; a.out_f32 = c->buf.act_f32[l];
   a.bias = c->params + ly.b_off; a.bias_stride = c->m_pad;
@@ -2244,6 +2273,7 @@ inline void tc_launch_head(prsgd_ctx* c, const DrawArgs& dr, const uint8_t* acti
     a.fwd_ksteps = (c->layer[L - 2].d_in / 64 + 1) / 2;
     a.fwd_prefetch = (active == nullptr && c->early_loads) ? 1 : 0;
     a.fwd_shared_w = tc_shared_restart(c, active) ? 1 : 0;
+    a.wt_lo = tc_wtile(c, L - 1);
   }
   const unsigned cl = (unsigned)(ly.d_in / 128);
   const TcLayerMaps& lo = st->layer[L >= 2 ? L - 2 : 0];
@@ -2278,7 +2308,7 @@ inline void tc_launch_forward_chain(prsgd_ctx* c, int l_first, int l_last, const
     const Layer& ly = c->layer[l - 1];
     ChainSeg& g = a.seg[l - l_first];
     g.k_steps = (ly.d_in / 64 + 1) / 2; g.tiles_m = (ly.d_out + 127) / 128; g.M_total = ly.d_out; g.ld_out = c->buf.ld[l];
-    g.linear = l == c->L ? 1 : 0; g.pool = l == 1 ? 1 : 0;
+    g.linear = l == c->L ? 1 : 0; g.pool = l == 1 ? 1 : 0; g.wt = tc_wtile(c, l);
     // early weight loads overlap whatever launch precedes the whole forward pass: only when that launch is known
     // to leave the weights of layers >= 2 alone (the layer-1 update or a bias launch that ended the iteration before)
     g.prefetch = (l > 1 && active == nullptr && c->early_loads && c->upper_weights_quiet) ? 1 : 0;
@@ -2307,7 +2337,7 @@ inline void tc_launch_dx(prsgd_ctx* c, int l, const DrawArgs& dr, const uint8_t*
   const Layer& ly = c->layer[l - 1];
   StreamArgs a{};
   a.B = c->B; a.N = c->N; a.k_steps = (c->buf.ld[l] / 64 + 1) / 2; a.M_total = ly.d_in; a.tiles_m = (ly.d_in + 127) / 128;
-  a.stages = stream_stages(c->B);
+  a.stages = stream_stages(c->B); a.wt = tc_wtile(c, l);
   a.pool = 0; a.draw = dr; a.ld_out = c->buf.ld[l - 1];
   a.out_bk = c->buf.delta_bk[l - 1]; a.mask_src = c->buf.act_bk[l - 1];
   a.active = active; a.status = c->status;
@@ -2331,7 +2361,7 @@ inline void tc_launch_update_tn(prsgd_ctx* c, int l, const DrawArgs& dr, const u
   a.B = c->B; a.N = c->N; a.tiles_m = (ly.d_out + 127) / 128; a.tiles_n = (ly.d_in + TN - 1) / TN;
   a.gamma = c->gamma; a.mu = c->mu; a.pool = l == 1; a.draw = dr; a.active = active; a.status = c->status;
   a.prefetch = (active == nullptr && c->early_loads) ? 1 : 0;
-  a.shared_w = (fuse && tc_shared_restart(c, active)) ? 1 : 0;
+  a.shared_w = (fuse && tc_shared_restart(c, active)) ? 1 : 0; a.wt = tc_wtile(c, l);
   a.avg_vel = c->average_velocity ? 1 : 0;
   a.divisor = c->avg_divisor > 0.f ? c->avg_divisor : (float)c->N;
   const int items = a.tiles_m * a.tiles_n * (fuse ? 1 : c->N);
@@ -2368,7 +2398,7 @@ inline void tc_launch_update_dx_m(prsgd_ctx* c, int l) {
   const Layer& ly = c->layer[l - 1];
   UpdateDxArgs a{};
   a.B = c->B; a.N = c->N; a.tiles_m = (ly.d_out + 127) / 128; a.tiles_n = (ly.d_in + TN - 1) / TN;
-  a.gamma = c->gamma; a.status = c->status; a.stages = UpdDxCfg<TN, MOM, SP>::stages(c->B);
+  a.gamma = c->gamma; a.status = c->status; a.stages = UpdDxCfg<TN, MOM, SP>::stages(c->B); a.wt = tc_wtile(c, l);
   a.out_bk = c->buf.delta_bk[l - 1]; a.mask_src = c->buf.act_bk[l - 1]; a.ld_out = c->buf.ld[l - 1]; a.M_total = ly.d_in;
   a.bias_rw = c->params + c->layer[l - 2].b_off; a.bias_stride = c->m_pad;
   a.mu = c->mu; a.bias_vel = MOM ? c->velocity + c->layer[l - 2].b_off : nullptr;
@@ -2429,7 +2459,7 @@ inline void tc_launch_update_next_tn(prsgd_ctx* c, const DrawArgs& dr) {
   a.B = c->B; a.N = c->N; a.tiles_m = (ly.d_out + 127) / 128; a.tiles_n = (ly.d_in + TN - 1) / TN;
   a.gamma = c->gamma; a.mu = c->mu; a.draw = dr; a.status = c->status;
   a.active = worker_mask(c);
-  a.stages = UpdNextCfg<TN, MOM>::stages(c->B);
+  a.stages = UpdNextCfg<TN, MOM>::stages(c->B); a.wt = tc_wtile(c, 1);
   a.next_out = c->buf.act_bk[1]; a.next_ld = c->buf.ld[1];
   a.bias = c->params + ly.b_off; a.bias_stride = c->m_pad; a.M_total = ly.d_out;
   int grid = 1;
@@ -2476,7 +2506,7 @@ inline void tc_launch_update_common(prsgd_ctx* c, const int* layers, int n, cons
     const Layer& ly = c->layer[l - 1];
     CommonSeg& g = a.seg[i];
     g.tiles_n = (ly.d_in + 63) / 64; g.tile0 = tiles; g.pool = l == 1 ? 1 : 0; g.d_in = ly.d_in; g.d_out = ly.d_out;
-    g.params = c->params + ly.w_off; g.shadow = c->shadow + ly.w_off;
+    g.params = c->params + ly.w_off; g.shadow = c->shadow + ly.w_off; g.wt = tc_wtile(c, l);
     tiles += ((ly.d_out + 127) / 128) * g.tiles_n;
     maps.delta[i] = st->layer[l - 1].delta_out; maps.act[i] = st->layer[l - 1].act_in; maps.master[i] = st->layer[l - 1].master;
   }

@@ -47,6 +47,7 @@ struct HeadArgs {
   int fwd_stages;
   int fwd_prefetch;          // W_{L-1}'s first tiles may be requested before the previous launch has completed
   int fwd_shared_w;          // every worker's W_{L-1} holds the same bits: read worker 0's (one HBM read serves all)
+  WTile wt_lo;               // order of W_{L-1}'s elements
 };
 
 constexpr int kHeadThreads = 320;     // warp 0 loads, warp 1 MMAs, warps 2..5 logits / softmax / step of W_L, warps 6..9 dZ_{L-1}
@@ -128,8 +129,8 @@ __global__ void __launch_bounds__(kHeadThreads, 1) tc_head_kernel(const __grid_c
   auto load_wlo = [&](int st, int ks) {
     const uint32_t sa = base + o_ring + (uint32_t)st * fstage;
     const int nw = a.fwd_shared_w ? 0 : n;
-    tma_load_3d(sa, &mapWlo, f_full(st), (2 * ks) * 64, k0, nw);
-    tma_load_3d(sa + 16384u, &mapWlo, f_full(st), (2 * ks + 1) * 64, k0, nw);
+    tma_load_w(sa, &mapWlo, f_full(st), a.wt_lo, (2 * ks) * 64, k0, nw);
+    tma_load_w(sa + 16384u, &mapWlo, f_full(st), a.wt_lo, (2 * ks + 1) * 64, k0, nw);
   };
   // Nothing in flight writes W_L when this launch begins (the launch before it is a forward GEMM of a lower
   // layer or layer 1's update), so its tiles are requested while that launch drains.

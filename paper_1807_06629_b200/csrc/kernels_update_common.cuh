@@ -32,6 +32,7 @@ struct CommonSeg {
   int d_in, d_out;
   float* params;             // fp32 store + offset of W_l (row stride m_pad elements)
   uint16_t* shadow;          // bf16 copy + offset of W_l
+  WTile wt;                  // order of the segment's elements
 };
 
 struct CommonMaps {
@@ -126,8 +127,8 @@ __global__ void __launch_bounds__(kUpdCommonThreads, 1) tc_update_common_kernel(
     const int rel = tile - a.seg[si].tile0;
     const int m0 = (rel / a.seg[si].tiles_n) * 128, n0 = (rel % a.seg[si].tiles_n) * 64;
     mbar_expect_tx(mst_full, Cfg::kMaster);
-    tma_load_3d(buf_u32, &maps.master[si], mst_full, n0, m0, 0);
-    tma_load_3d(buf_u32 + 16384u, &maps.master[si], mst_full, n0 + 32, m0, 0);
+    tma_load_w(buf_u32, &maps.master[si], mst_full, a.seg[si].wt, n0, m0, 0);
+    tma_load_w(buf_u32 + 16384u, &maps.master[si], mst_full, a.seg[si].wt, n0 + 32, m0, 0);
   };
   // The master tiles were last written an iteration ago (the launch before this one only reads bf16 copies), so
   // the first one is requested while that launch drains.
@@ -221,9 +222,10 @@ __global__ void __launch_bounds__(kUpdCommonThreads, 1) tc_update_common_kernel(
         v[i] = *reinterpret_cast<const uint4*>(buf + (i >> 3) * 16384 + rr * 128 + ((j ^ (rr & 7)) << 4));
       }
       mbar_arrive(out_free);                              // the buffer may take the next tile's master tile
-      float* prow = sg.params + (int64_t)nb * a.m_pad + (int64_t)(m0 + rsub) * sg.d_in + n0 + 4 * j;
-      uint16_t* srow = sg.shadow + (int64_t)nb * a.m_pad + (int64_t)(m0 + rsub) * sg.d_in + n0 + 8 * j;
-      const int64_t step = 16 * (int64_t)sg.d_in;         // 16 rows further down
+      const int64_t first = wtile_offset(sg.wt, m0 + rsub, n0);       // row rsub of the tile, its first column
+      float* prow = sg.params + (int64_t)nb * a.m_pad + first + 4 * j;
+      uint16_t* srow = sg.shadow + (int64_t)nb * a.m_pad + first + 8 * j;
+      const int64_t step = 16 * (int64_t)(sg.wt.tiled ? 64 : sg.d_in);      // 16 rows further down
       for (int n = nb; n < ne; ++n) {
 #pragma unroll
         for (int i = 0; i < 8; ++i) {

@@ -117,6 +117,7 @@ size_t carve_scratch(int N, const prsgd_model_spec* s, int64_t m_pad, prsgd_ctx*
   auto losses = take(sizeof(float) * (size_t)N * B);
   auto active = take((size_t)N);
   auto stage = take(sizeof(float) * (size_t)m_pad);
+  auto canon = take(sizeof(float) * (size_t)m_pad);
   auto tdev = take(sizeof(int64_t));
   auto chain = take(sizeof(unsigned int) * ((size_t)kChainMax * N + 1));
   auto gmasks = take((size_t)kMaxGroups * N);
@@ -129,6 +130,7 @@ size_t carve_scratch(int N, const prsgd_model_spec* s, int64_t m_pad, prsgd_ctx*
     ctx->losses = reinterpret_cast<float*>(losses);
     ctx->active = active;
     ctx->stage_row = reinterpret_cast<float*>(stage);
+    ctx->canon_row = reinterpret_cast<float*>(canon);
     std::memset(&ctx->buf, 0, sizeof(ctx->buf));
   }
   if (s->precision == PRSGD_PRECISION_FP32) {
@@ -173,22 +175,57 @@ bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) %
 
 int grid1d(int64_t n, int block) { return (int)((n + block - 1) / block); }
 
-// ---- copies between the canonical (gap-free) order and the padded rows -----------------
-// rows [row0, row0 + nrows) of `store` (the parameters or the momentum buffers) <-> nrows * m floats at `lin`
-int copy_canonical(prsgd_ctx* c, float* store, float* lin, int64_t row0, int64_t nrows, bool to_store) {
+// ---- copies between the canonical (gap-free, row-major) order and the rows of the store ----------------
+CanonArgs canon_args(const prsgd_ctx* c) {
+  CanonArgs a{};
+  a.L = c->L;
   int64_t pos = 0;
   for (int l = 0; l < c->L; ++l) {
     const Layer& ly = c->layer[l];
-    const int64_t seg[2] = {(int64_t)ly.d_in * ly.d_out, (int64_t)ly.d_out};
-    const int64_t offs[2] = {ly.w_off, ly.b_off};
-    for (int k = 0; k < 2; ++k) {
-      float* st = store + row0 * c->m_pad + offs[k];
-      float* li = lin + pos;
-      if (to_store)
-        CUDA_TRY(c, cudaMemcpy2DAsync(st, c->m_pad * 4, li, c->m * 4, seg[k] * 4, nrows, cudaMemcpyDefault, c->stream));
-      else
-        CUDA_TRY(c, cudaMemcpy2DAsync(li, c->m * 4, st, c->m_pad * 4, seg[k] * 4, nrows, cudaMemcpyDefault, c->stream));
-      pos += seg[k];
+    a.w_off[l] = ly.w_off; a.b_off[l] = ly.b_off; a.d_out[l] = ly.d_out;
+    a.wt[l].tiled = 0; a.wt[l].tn = ly.d_in / 64; a.wt[l].d_in = ly.d_in;
+    if (c->precision == PRSGD_PRECISION_BF16) a.wt[l] = tc_wtile(c, l + 1);
+    a.w_pos[l] = pos; pos += (int64_t)ly.d_in * ly.d_out;
+    a.b_pos[l] = pos; pos += ly.d_out;
+  }
+  return a;
+}
+
+int launch_canonical(prsgd_ctx* c, float* store, int64_t store_stride, float* lin, int64_t lin_stride, int64_t nrows, bool to_store) {
+  const CanonArgs a = canon_args(c);
+  int64_t longest = 1;
+  for (int l = 0; l < c->L; ++l) {
+    const int64_t n = (int64_t)c->layer[l].d_in * c->layer[l].d_out;
+    if (n > longest) longest = n;
+  }
+  int64_t blocks = (longest + 255) / 256;
+  if (blocks > 2048) blocks = 2048;
+  for (int64_t r0 = 0; r0 < nrows; r0 += 32768) {          // (grid z is limited to 65535)
+    const int64_t nr = nrows - r0 < 32768 ? nrows - r0 : 32768;
+    canonical_copy_kernel<<<dim3((unsigned)blocks, 2 * c->L, (unsigned)nr), 256, 0, c->stream>>>(
+        store + r0 * store_stride, store_stride, lin + r0 * lin_stride, lin_stride, a, to_store ? 1 : 0);
+    LAUNCH_CHECK(c);
+  }
+  return PRSGD_OK;
+}
+
+// rows [row0, row0 + nrows) of `store` (the parameters or the momentum buffers) <-> nrows * m floats at `lin`;
+// host memory goes through one canonical row on the device
+int copy_canonical(prsgd_ctx* c, float* store, float* lin, int64_t row0, int64_t nrows, bool to_store, bool lin_on_device) {
+  float* rows = store + row0 * c->m_pad;
+  if (lin_on_device) return launch_canonical(c, rows, c->m_pad, lin, c->m, nrows, to_store);
+  if (c->readout_pending) {                     // (the canonical row still holds an asynchronous read-out)
+    CUDA_TRY(c, cudaStreamWaitEvent(c->stream, c->readout_event, 0));
+  }
+  for (int64_t r = 0; r < nrows; ++r) {
+    if (to_store) {
+      CUDA_TRY(c, cudaMemcpyAsync(c->canon_row, lin + r * c->m, (size_t)c->m * 4, cudaMemcpyHostToDevice, c->stream));
+      int rc = launch_canonical(c, rows + r * c->m_pad, c->m_pad, c->canon_row, c->m, 1, true);
+      if (rc != PRSGD_OK) return rc;
+    } else {
+      int rc = launch_canonical(c, rows + r * c->m_pad, c->m_pad, c->canon_row, c->m, 1, false);
+      if (rc != PRSGD_OK) return rc;
+      CUDA_TRY(c, cudaMemcpyAsync(lin + r * c->m, c->canon_row, (size_t)c->m * 4, cudaMemcpyDeviceToHost, c->stream));
     }
   }
   return PRSGD_OK;
@@ -612,11 +649,10 @@ int prsgd_swap_data(prsgd_ctx* c) {
 }
 
 int prsgd_set_params(prsgd_ctx* c, const float* src, int32_t worker, int src_on_device) {
-  (void)src_on_device;
   if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
   if (!src) return fail(c, PRSGD_ERR_ARG, "src is NULL");
   if (worker < -1 || worker >= c->N) return fail(c, PRSGD_ERR_ARG, "worker out of range");
-  int rc = copy_canonical(c, c->params, const_cast<float*>(src), worker < 0 ? 0 : worker, 1, true);
+  int rc = copy_canonical(c, c->params, const_cast<float*>(src), worker < 0 ? 0 : worker, 1, true, src_on_device != 0);
   if (rc != PRSGD_OK) return rc;
   if (worker < 0 && c->N > 1) {
     prof_begin(c, PRSGD_KERNEL_MISC);
@@ -632,7 +668,7 @@ int prsgd_set_params(prsgd_ctx* c, const float* src, int32_t worker, int src_on_
 int prsgd_set_params_stacked(prsgd_ctx* c, const float* src, int src_on_device) {
   if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
   if (!src) return fail(c, PRSGD_ERR_ARG, "src is NULL");
-  int rc = copy_canonical(c, c->params, const_cast<float*>(src), 0, c->N, true);
+  int rc = copy_canonical(c, c->params, const_cast<float*>(src), 0, c->N, true, src_on_device != 0);
   if (rc != PRSGD_OK) return rc;
   if (!src_on_device) CUDA_TRY(c, cudaStreamSynchronize(c->stream));
   c->rows_identical = c->N == 1;
@@ -641,20 +677,18 @@ int prsgd_set_params_stacked(prsgd_ctx* c, const float* src, int src_on_device) 
 }
 
 int prsgd_get_params_stacked(prsgd_ctx* c, float* dst, int dst_on_device) {
-  (void)dst_on_device;
   if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
   if (!dst) return fail(c, PRSGD_ERR_ARG, "dst is NULL");
-  int rc = copy_canonical(c, c->params, dst, 0, c->N, false);
+  int rc = copy_canonical(c, c->params, dst, 0, c->N, false, dst_on_device != 0);
   if (rc != PRSGD_OK) return rc;
   return check_device_status(c);
 }
 
 int prsgd_get_params(prsgd_ctx* c, float* dst, int32_t worker, int dst_on_device) {
-  (void)dst_on_device;
   if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
   if (!dst) return fail(c, PRSGD_ERR_ARG, "dst is NULL");
   if (worker < 0 || worker >= c->N) return fail(c, PRSGD_ERR_ARG, "worker out of range");
-  int rc = copy_canonical(c, c->params, dst, worker, 1, false);
+  int rc = copy_canonical(c, c->params, dst, worker, 1, false, dst_on_device != 0);
   if (rc != PRSGD_OK) return rc;
   return check_device_status(c);
 }
@@ -751,7 +785,7 @@ void period_key(const prsgd_ctx* c, uint64_t (&key)[13]) {
   key[12] = (c->rows_identical ? 1u : 0u) | ((uint64_t)c->shared_restart << 1) | ((uint64_t)c->forward_chain << 2) |
             ((uint64_t)c->worker_groups << 3) | ((uint64_t)c->dx_shared_pair << 6) | ((uint64_t)c->head_kernel << 7) |
             ((uint64_t)c->common_point << 9) | ((uint64_t)c->split_blocks << 11) | ((uint64_t)c->head_forward << 13) |
-            ((uint64_t)c->merged_small_average << 14);      // (rows_identical: the period's first iteration may share reads)
+            ((uint64_t)c->merged_small_average << 14) | ((uint64_t)c->tiled_weights << 15);      // (rows_identical: the period's first iteration may share reads)
 }
 
 // One whole averaging period (I iterations starting right after an average) as a CUDA graph: the
@@ -895,18 +929,13 @@ int prsgd_get_average_async(prsgd_ctx* c, float* h_dst, void* copy_stream) {
                                                                                 c->stage_row, nullptr);
     LAUNCH_CHECK(c);
   }
+  {   // the mean in canonical order, still on the training stream; one copy to the host on the caller's stream
+    int rc = launch_canonical(c, c->stage_row, c->m_pad, c->canon_row, c->m, 1, false);
+    if (rc != PRSGD_OK) return rc;
+  }
   CUDA_TRY(c, cudaEventRecord(c->mean_ready_event, c->stream));
   CUDA_TRY(c, cudaStreamWaitEvent(cs, c->mean_ready_event, 0));
-  int64_t pos = 0;
-  for (int l = 0; l < c->L; ++l) {
-    const Layer& ly = c->layer[l];
-    const int64_t seg[2] = {(int64_t)ly.d_in * ly.d_out, (int64_t)ly.d_out};
-    const int64_t offs[2] = {ly.w_off, ly.b_off};
-    for (int q = 0; q < 2; ++q) {
-      CUDA_TRY(c, cudaMemcpyAsync(h_dst + pos, c->stage_row + offs[q], seg[q] * 4, cudaMemcpyDeviceToHost, cs));
-      pos += seg[q];
-    }
-  }
+  CUDA_TRY(c, cudaMemcpyAsync(h_dst, c->canon_row, (size_t)c->m * 4, cudaMemcpyDeviceToHost, cs));
   CUDA_TRY(c, cudaEventRecord(c->readout_event, cs));
   c->readout_pending = true;
   return PRSGD_OK;
@@ -925,18 +954,13 @@ int prsgd_get_average(prsgd_ctx* c, float* dst, int dst_on_device) {
                                                                                 c->stage_row, nullptr);
     LAUNCH_CHECK(c);
   }
-  int64_t pos = 0;
-  for (int l = 0; l < c->L; ++l) {
-    const Layer& ly = c->layer[l];
-    const int64_t seg[2] = {(int64_t)ly.d_in * ly.d_out, (int64_t)ly.d_out};
-    const int64_t offs[2] = {ly.w_off, ly.b_off};
-    for (int q = 0; q < 2; ++q) {
-      CUDA_TRY(c, cudaMemcpyAsync(dst + pos, mean + offs[q], seg[q] * 4, cudaMemcpyDefault, c->stream));
-      pos += seg[q];
-    }
+  if (dst_on_device) return launch_canonical(c, const_cast<float*>(mean), c->m_pad, dst, c->m, 1, false);
+  {
+    int rc = launch_canonical(c, const_cast<float*>(mean), c->m_pad, c->canon_row, c->m, 1, false);
+    if (rc != PRSGD_OK) return rc;
   }
-  if (!dst_on_device) return check_device_status(c);
-  return PRSGD_OK;
+  CUDA_TRY(c, cudaMemcpyAsync(dst, c->canon_row, (size_t)c->m * 4, cudaMemcpyDeviceToHost, c->stream));
+  return check_device_status(c);
 }
 
 int prsgd_enable_momentum(prsgd_ctx* c, float mu, void* d_velocity, int average_velocity) {
@@ -958,11 +982,10 @@ int prsgd_enable_momentum(prsgd_ctx* c, float mu, void* d_velocity, int average_
 }
 
 int prsgd_get_velocity_stacked(prsgd_ctx* c, float* dst, int dst_on_device) {
-  (void)dst_on_device;
   if (!c) return fail(nullptr, PRSGD_ERR_ARG, "ctx is NULL");
   if (!dst) return fail(c, PRSGD_ERR_ARG, "dst is NULL");
   if (!c->velocity) return fail(c, PRSGD_ERR_STATE, "momentum is not enabled");
-  int rc = copy_canonical(c, c->velocity, dst, 0, c->N, false);   // same row layout as the store
+  int rc = copy_canonical(c, c->velocity, dst, 0, c->N, false, dst_on_device != 0);   // same row layout as the store
   if (rc != PRSGD_OK) return rc;
   return check_device_status(c);
 }
@@ -1157,6 +1180,29 @@ int prsgd_set_option(prsgd_ctx* c, int32_t option, int64_t value) {
   if (option == PRSGD_OPT_SHARED_RESTART) { c->shared_restart = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_FORWARD_CHAIN) { c->forward_chain = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_DX_SHARED_PAIR) { c->dx_shared_pair = value != 0; return PRSGD_OK; }
+  if (option == PRSGD_OPT_TILED_WEIGHTS) {
+    const int want = value != 0 ? 1 : 0;
+    if (want == c->tiled_weights || c->precision != PRSGD_PRECISION_BF16) { c->tiled_weights = want; return PRSGD_OK; }
+    // re-order the store in place: every row through the canonical order, old order out, new order in
+    CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+    if (c->readout_pending) CUDA_TRY(c, cudaStreamWaitEvent(c->stream, c->readout_event, 0));
+    float* stores[2] = {c->params, c->velocity};
+    for (int r = 0; r < c->N; ++r) {
+      for (int k = 0; k < 2; ++k) {
+        if (stores[k] == nullptr) continue;
+        c->tiled_weights = 1 - want;
+        int rc = launch_canonical(c, stores[k] + (int64_t)r * c->m_pad, c->m_pad, c->canon_row, c->m, 1, false);
+        c->tiled_weights = want;
+        if (rc == PRSGD_OK) rc = launch_canonical(c, stores[k] + (int64_t)r * c->m_pad, c->m_pad, c->canon_row, c->m, 1, true);
+        if (rc != PRSGD_OK) return rc;
+      }
+    }
+    std::string terr;
+    int trc = tc_make_weight_maps(c, &terr);
+    if (trc != PRSGD_OK) return fail(c, trc, terr);
+    c->a1_ready = false;
+    return refresh_shadow(c);
+  }
   if (option == PRSGD_OPT_COMMON_POINT) {
     if (value < 0 || value > 2) return fail(c, PRSGD_ERR_ARG, "PRSGD_OPT_COMMON_POINT takes 0, 1 or 2");
     c->common_point = (int)value;

@@ -111,6 +111,27 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t sr
                ::"l"((uint64_t)map), "r"(src), "r"(c0), "r"(c1), "r"(c2)
                : "memory");
 }
+// The same for a box of a weight segment given by its first column and row in the d_out x d_in matrix: with the
+// tile-major order (see WTile) the tensor map is {64, tiles * 128, N} and the box lies inside one 128 x 64 tile.
+// A box that starts beyond the matrix width (the zero-filled tail of a contraction) is sent out of bounds.
+__device__ __forceinline__ void wtile_xy(const WTile& t, int col, int row, int& x, int& y) {
+  if (t.tiled) {
+    x = col & 63;
+    y = col < t.d_in ? ((row >> 7) * t.tn + (col >> 6)) * 128 + (row & 127) : 0x7FFFFF00;
+  } else {
+    x = col; y = row;
+  }
+}
+__device__ __forceinline__ void tma_load_w(uint32_t dst, const CUtensorMap* map, uint32_t bar, const WTile& t, int col, int row, int n) {
+  int x, y;
+  wtile_xy(t, col, row, x, y);
+  tma_load_3d(dst, map, bar, x, y, n);
+}
+__device__ __forceinline__ void tma_store_w(const CUtensorMap* map, uint32_t src, const WTile& t, int col, int row, int n) {
+  int x, y;
+  wtile_xy(t, col, row, x, y);
+  tma_store_3d(map, src, x, y, n);
+}
 __device__ __forceinline__ void tma_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void tma_wait_group_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void tma_wait_group_read1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }

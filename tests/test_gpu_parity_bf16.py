@@ -600,6 +600,74 @@ def test_small_weight_segments_averaged_by_the_bias_average_launch_change_no_bit
             assert grp[1][4] < grp[0][4]
 
 
+TILED_CASES = [
+    _w("tc-tiled-two-layer", 3, (128, 256, 10), 32, I=2),
+    _w("tc-tiled-mixed", 2, (64, 128, 64, 10), 16, I=3),
+    _w("tc-tiled-odd-width", 3, (448, 256, 10), 16, I=2),
+    _w("tc-tiled-deep", 2, (192, 384, 256, 128, 100), 32, I=2),
+    _w("tc-tiled-I1", 3, (640, 1024, 10), 32, I=1),
+    _w("tc-tiled-b64", 2, (128, 1024, 256, 10), 64, I=2),
+]
+
+
+@pytest.mark.parametrize("w", TILED_CASES, ids=[w.name for w in TILED_CASES])
+def test_tile_major_weight_segments_change_no_bit(torch_cuda, w):
+    """Hidden layers' weight segments stored as 128 x 64 tiles (PRSGD_OPT_TILED_WEIGHTS) against row-major
+    segments: the same arithmetic on the same numbers, so every result that crosses the interface -- stacked
+    parameters, one worker's parameters, the node average (to the host, to the device, asynchronously), losses,
+    momentum buffers -- is identical, for both tile widths, the folded and the separate launches, momentum, a
+    worker mask and replayed periods; switching the order in the middle of a run changes nothing either; the bf16
+    copy equals bf16(master) element for element in whichever order the rows are."""
+    torch = torch_cuda
+    from paper_1807_06629_b200 import binding
+    X, Y, x0 = make_inputs(w)
+    T = 2 * w.I + 1
+    variants = [("plain", {}), ("tile64", {binding.OPT_UPDATE_TILE: 64}), ("tile128", {binding.OPT_UPDATE_TILE: 128}),
+                ("separate", {binding.OPT_DX_IN_UPDATE: 0, binding.OPT_NEXT_FORWARD: 0}), ("fold-all", {binding.OPT_DX_IN_UPDATE: 2}),
+                ("momentum", {}), ("mask", {}), ("head-forward", {binding.OPT_HEAD_FORWARD: 1}), ("chain", {binding.OPT_FORWARD_CHAIN: 1})]
+    for name, opts in variants:
+        outs = []
+        for tiled, graph, switch in ((0, 0, False), (1, 0, False), (1, 1, False), (0, 0, True)):
+            with torch.cuda.stream(torch.cuda.Stream()):
+                p = make_ctx(w, X, Y, x0)
+                p.set_option(binding.OPT_TILED_WEIGHTS, tiled)
+                p.set_option(binding.OPT_GRAPH, graph)
+                for k, v in opts.items():
+                    p.set_option(k, v)
+                if name == "momentum":
+                    p.enable_momentum(0.9, average_velocity=True)
+                if name == "mask":
+                    p.set_active([1 if i != 1 else 0 for i in range(w.N)])
+                p.local_steps(2)
+                if switch:
+                    p.set_option(binding.OPT_TILED_WEIGHTS, 1)          # re-orders the store (and the momentum buffers) in place
+                p.local_steps(T - 2)
+                p.sync()
+                store = p.params.cpu().numpy().reshape(w.N, p.m_pad)
+                shadow = p.shadow.view(torch.int16).cpu().numpy().view(np.uint16).reshape(w.N, p.m_pad)
+                for l in range(len(w.dims) - 1):
+                    a, n = p.layout.w_off[l], w.dims[l] * w.dims[l + 1]
+                    assert np.array_equal(shadow[:, a:a + n], synth.bf16_bits(store[:, a:a + n])), (w.name, name, l)
+                avg_dev = torch.empty(p.m, dtype=torch.float32, device="cuda")
+                p.get_average(avg_dev)
+                pinned = torch.empty(p.m, dtype=torch.float32).pin_memory()
+                side = torch.cuda.Stream()
+                p.get_average_async(pinned, side)
+                side.synchronize()
+                outs.append((p.get_params_stacked(), p.get_losses(), p.get_average(), avg_dev.cpu().numpy(), pinned.numpy().copy(),
+                             p.get_params(w.N - 1), p.get_velocity_stacked() if name == "momentum" else None))
+                torch.cuda.current_stream().synchronize()
+                p.close()
+        keep = [i for i in range(w.N) if name != "mask" or i != 1]
+        for o in outs[1:]:
+            assert np.array_equal(outs[0][0], o[0]), (w.name, name)
+            assert np.array_equal(outs[0][1][keep], o[1][keep])
+            assert np.array_equal(outs[0][2], o[2]) and np.array_equal(o[2], o[3]) and np.array_equal(o[2], o[4])
+            assert np.array_equal(outs[0][5], o[5]) and np.array_equal(o[5], o[0][w.N - 1])
+            if name == "momentum":
+                assert np.array_equal(outs[0][6], o[6])
+
+
 HEAD_FWD_CASES = [
     _w("tc-tail-small", 3, (128, 256, 128, 10), 32, I=3),
     _w("tc-tail-ragged-k", 2, (192, 320, 1024, 10), 64, I=2),
