@@ -200,9 +200,9 @@ class ClockSampler:
 # profiles/).  The update kernels stream every worker's tiles once, so traffic grows in proportion to the
 # number of workers: the record is scaled by N / workers.  Valid only while the kernels' source is unchanged.
 NCU_TRAFFIC = {
-    # profiles/tc_update_kernels_cfg4_N16.md: 556.8 MB read + 557.4 MB written by the four update launches of a plain iteration
-    ("cfg4", "update"): {"workers": 16, "bytes_per_iteration": 556.8e6 + 557.4e6, "launches_per_iteration": 4,
-                         "kernel_sha256": "5d0be5d942d5fb66dac97c8fc56e7863832c072fdc8735e2a8f10a5e3cd7ea12"},
+    # profiles/tc_update_kernels_cfg4_N16.md: 556.9 MB read + 554.7 MB written by the four update launches of a plain iteration
+    ("cfg4", "update"): {"workers": 16, "bytes_per_iteration": 556.9e6 + 554.7e6, "launches_per_iteration": 4,
+                         "kernel_sha256": "35b47287a2c2c915b5115f8603d324af592d6182b6a2e9b787368e4718c03f01"},
 }
 
 
@@ -474,7 +474,8 @@ def measure_config(torch, w_cfg, args, dev, rank, world, scaling, steps, warmup,
                       (args.no_fused_epilogues, binding.OPT_FUSED_EPILOGUES),
                       (args.no_shared_restart, binding.OPT_SHARED_RESTART),
                       (args.no_forward_chain, binding.OPT_FORWARD_CHAIN),
-                      (args.no_head_kernel, binding.OPT_HEAD_KERNEL), (args.no_common_point, binding.OPT_COMMON_POINT)):
+                      (args.no_head_kernel, binding.OPT_HEAD_KERNEL), (args.no_common_point, binding.OPT_COMMON_POINT),
+                      (args.no_tiled_weights, binding.OPT_TILED_WEIGHTS)):
         if flag:
             p.set_option(opt, 0)
     if args.head_forward:
@@ -622,6 +623,8 @@ def parse_args(argv=None):
                     help="one forward launch per layer instead of one launch for all layers")
     ap.add_argument("--head-kernel-always", action="store_true",
                     help="the class layer as one launch of clusters even when its CTAs need more than one wave")
+    ap.add_argument("--no-tiled-weights", action="store_true",
+                    help="hidden layers' weight segments row-major instead of as 128 x 64 tiles")
     ap.add_argument("--no-common-point", action="store_true",
                     help="an averaging iteration that starts from N equal rows forms and sums the N stepped models one by one")
     ap.add_argument("--head-forward", action="store_true",
