@@ -475,7 +475,7 @@ def measure_config(torch, w_cfg, args, dev, rank, world, scaling, steps, warmup,
                       (args.no_shared_restart, binding.OPT_SHARED_RESTART),
                       (args.no_forward_chain, binding.OPT_FORWARD_CHAIN),
                       (args.no_head_kernel, binding.OPT_HEAD_KERNEL), (args.no_common_point, binding.OPT_COMMON_POINT),
-                      (args.no_tiled_weights, binding.OPT_TILED_WEIGHTS)):
+                      (args.no_tiled_weights, binding.OPT_TILED_WEIGHTS), (args.no_overlap_update, binding.OPT_OVERLAP_UPDATE)):
         if flag:
             p.set_option(opt, 0)
     if args.head_forward:
@@ -623,6 +623,8 @@ def parse_args(argv=None):
                     help="one forward launch per layer instead of one launch for all layers")
     ap.add_argument("--head-kernel-always", action="store_true",
                     help="the class layer as one launch of clusters even when its CTAs need more than one wave")
+    ap.add_argument("--no-overlap-update", action="store_true",
+                    help="layer 2's update before layer 1's, each launch after the other, instead of beside it")
     ap.add_argument("--no-tiled-weights", action="store_true",
                     help="hidden layers' weight segments row-major instead of as 128 x 64 tiles")
     ap.add_argument("--no-common-point", action="store_true",

@@ -345,6 +345,13 @@ int prsgd_get_velocity_stacked(prsgd_ctx* ctx, float* dst, int dst_on_device);
  * columns of the rows as they are (all ranks of a job use the same setting).  Changing the option re-orders the
  * store in place (a pass over all rows).  Same bits either way. */
 #define PRSGD_OPT_TILED_WEIGHTS 19
+/* PRSGD_OPT_OVERLAP_UPDATE (default 1, tensor-core path, three layers or more, every worker active):
+ * on iterations whose layer-1 update also forms the next iteration's first activation (PRSGD_OPT_NEXT_FORWARD) and
+ * whose layer 2 runs dX and update as separate launches, layer 2's update is enqueued AFTER layer 1's and starts
+ * beside it: it needs nothing that launch produces, so its CTAs take the SMs that launch leaves idle (whole row
+ * blocks per CTA seldom fill the GPU) and the others as they fall free, claiming tiles from a device counter.  The
+ * next iteration's a_1 goes to a second buffer meanwhile.  Same arithmetic per tile: same bits. */
+#define PRSGD_OPT_OVERLAP_UPDATE 20
 /* PRSGD_OPT_MERGED_SMALL_AVERAGE (default 1, tensor-core path, fused averaging iterations): the weight segments of
  * layers too small for the fused update + average (the class layer) are averaged by the launch that averages the
  * bias segments, at the end of the iteration, instead of by a launch of their own after the layer's update.  Same

@@ -39,6 +39,7 @@ OPT_SPLIT_BLOCKS = 16
 OPT_HEAD_FORWARD = 17
 OPT_MERGED_SMALL_AVERAGE = 18
 OPT_TILED_WEIGHTS = 19
+OPT_OVERLAP_UPDATE = 20
 ERR_DEVICE_TIMEOUT, ERR_NONFINITE = -6, -7
 KERNEL_FAMILIES = ("forward", "softmax", "dx", "update", "update_average", "average", "misc", "head")
 MAX_LAYERS = 16

@@ -35,6 +35,7 @@ struct TcState {
   TcLayerMaps layer[PRSGD_MAX_LAYERS];
   CUtensorMap head_shadow;  // bf16 W_L, box {64, ceil16(d_L), 1}: tiles of tc_head_kernel (valid when head_rows > 0)
   CUtensorMap head_master;  // fp32 W_L, box {32, ceil16(d_L), 1}
+  CUtensorMap act1_alt;     // a_1 in its second buffer, same geometry as layer[1].act_in (valid when L >= 2)
   int head_rows = 0;
   int num_sms = 148;
   bool pool_bound = false;
@@ -115,6 +116,8 @@ struct StreamArgs {
   int ld_delta;
   float* row_losses;         // [N][B]
   int32_t* draws;            // [N]
+  unsigned int* zero_word;   // not nullptr: block 0 clears this word after its dependency wait (the item counter of an
+                             // overlapped update launched later in the iteration)
 };
 
 // Persistent: one CTA per SM walks (tile, worker) items.  Warp 0 issues TMA, warp 1 issues MMAs,
@@ -212,6 +215,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) tc_stream_kernel(const __gr
   }
   pdl_wait();            // everything above overlapped the previous kernel's tail; dependent memory is touched below
   pdl_trigger();         // only now: the next launch's early loads may overlap this launch, never an older one
+  if (a.zero_word != nullptr && blockIdx.x == 0 && tid == 0) *a.zero_word = 0u;
   const uint32_t tmem = *tmem_slot;
   const int total_items = *abort_flag != 0 ? 0 : a.tiles_m * a.N;
   auto item_active = [&](int n) { return a.active == nullptr || a.active[n] != 0; };
@@ -715,7 +719,16 @@ struct UpdateArgs {
   int shared_w;            // fused form only, 1: every worker's master tile holds the same bits (the launch follows a
                            // node average with nothing in between): all N loads of a tile read worker 0's copy, which
                            // nobody overwrites before the CTA that owns the tile has summed all N workers
+  // Overlapped form (plain step only, no worker mask): the launch just before this one does not produce anything
+  // this one reads and has passed its own dependency wait in every CTA before this one starts, so this kernel
+  // begins WITHOUT a dependency wait, beside that launch, and takes the wait before it exits (whoever waits for
+  // this launch thereby waits for both).  CTAs become resident as SMs fall free, so items are not dealt out by
+  // block index: the loader claims the next one from *next_item (zero at launch) and hands the index to the other
+  // roles through a ring in shared memory.
+  unsigned int* next_item;
 };
+
+constexpr int kUpdSchedSlots = 8;         // ring of claimed item indices (>= twice the stage count)
 
 constexpr int kUpdThreads = 224;          // warp 0 loader, 1 MMA, 2 storer, 3..6 epilogue
 // The two folded update kernels end every block of tiles (a column block's dX, a row block's next forward)
@@ -735,7 +748,7 @@ template <int TN, bool MOM> struct UpdCfg {
   __host__ __device__ static uint32_t ops_bytes(int B) { return (uint32_t)(2 + TN / 64) * (uint32_t)B * 128u; }
   __host__ __device__ static uint32_t region(int B) { return ops_bytes(B) > kOut ? ops_bytes(B) : kOut; }
   __host__ __device__ static uint32_t stage(int B) { return kMaster + kVel + region(B); }
-  static size_t smem(int B) { return (size_t)kStages * stage(B) + 1024 + 256; }
+  static size_t smem(int B) { return (size_t)kStages * stage(B) + 1024 + 384; }
 };
 
 // MOM: the local step of the paper's experiment, v <- mu v + G, x <- x - gamma v; the momentum tile
@@ -781,6 +794,10 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
   volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + (size_t)Cfg::kStages * stage_bytes + 196);
   const uint32_t out_free = bar0 + 200u;               // kOutBuf: the row stores have read the output buffer
   const uint32_t out_u32 = base + (uint32_t)S * stage_bytes;     // kOutBuf: fp32 tile, then the bf16 tile
+  constexpr uint32_t R = (uint32_t)kUpdSchedSlots;
+  auto sched_full = [&](uint32_t i) { return bar0 + 208u + 8u * i; };   // overlapped form: slot i of the ring holds an item index
+  volatile int* sched = reinterpret_cast<volatile int*>(gen + (size_t)Cfg::kStages * stage_bytes + 272);
+  const bool dyn = !FUSE && a.next_item != nullptr;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t op_box = (uint32_t)a.B * 128u;       // one {64, B} box
@@ -793,6 +810,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
       mbar_init(acc_full(s), 1); mbar_init(acc_empty(s), 128); mbar_init(tile_ready(s), 128);
     }
     mbar_init(out_free, 1);
+    for (uint32_t i = 0; i < R; ++i) mbar_init(sched_full(i), 1);
     *abort_flag = *(volatile unsigned int*)&a.status->error != 0u ? 1 : 0;   // an earlier expired wait: no-op (see tc_stream_kernel)
     fence_mbar_init();
     prefetch_tensormap(&mapDelta); prefetch_tensormap(&mapAct);
@@ -818,7 +836,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
   // are requested while the previous launch (which only reads the bf16 shadow) drains; `prefetch` is
   // set by the host when no worker mask is in use, so item k of this CTA is known without reading memory.
   uint32_t pre = 0;
-  if (warp == 0 && lane == 0 && a.prefetch != 0) {
+  if (warp == 0 && lane == 0 && a.prefetch != 0 && !dyn) {
     for (int k = 0; k < S; ++k) {
       const int w = FUSE ? (int)blockIdx.x : (int)blockIdx.x + k * (int)gridDim.x;
       const int n = FUSE ? k : w / tiles;
@@ -829,20 +847,45 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
       ++pre;
     }
   }
-  pdl_wait();            // set-up above overlapped the previous kernel's tail; dependent memory is touched below
-  pdl_trigger();         // only now: the next launch's early loads may overlap this launch, never an older one
+  if (!dyn) {
+    pdl_wait();          // set-up above overlapped the previous kernel's tail; dependent memory is touched below
+    pdl_trigger();       // only now: the next launch's early loads may overlap this launch, never an older one
+  }
   const uint32_t tmem = *tmem_slot;
   const int total_items = *abort_flag != 0 ? 0 : items_all;
 
   // Every role walks the same sequence of (tile, worker) items; `it` counts the items it has handled,
   // item `it` lives in stage it % S and TMEM columns (it % S) * TN.
   auto item_active = [&](int n) { return FUSE || a.active == nullptr || a.active[n] != 0; };
+  // Item k of this CTA's sequence (-1: the sequence has ended): dealt out by block index, or, in the overlapped
+  // form, whatever the loader claimed k-th (every role but the loader reads it from the ring).
+  auto item_of = [&](uint32_t k, bool& ok) -> int {
+    if (!dyn) {
+      const int64_t w = (int64_t)blockIdx.x + (int64_t)k * (int64_t)gridDim.x;
+      return w < (int64_t)total_items ? (int)w : -1;
+    }
+    ok = mbar_wait(sched_full(k % R), (k / R) & 1u, abort_flag, a.status, 0x20B);
+    return ok ? sched[k % R] : -1;
+  };
 
   if (warp == 0 && lane == 0) {
     // ---------------- loader
     uint32_t it = 0;
     bool ok = true;
-    for (int w = blockIdx.x; w < total_items && ok; w += gridDim.x) {
+    for (uint32_t k = 0; ok; ++k) {
+      int w;
+      if (dyn) {
+        // the stage first, the claim last: a CTA that waits for room in its ring leaves the items to the others
+        ok = mbar_wait(stage_empty(k % S), ((k / S) & 1u) ^ 1u, abort_flag, a.status, 0x201);
+        if (!ok) break;
+        w = total_items > 0 ? (int)atomicAdd(a.next_item, 1u) : -1;
+        if (w >= total_items) w = -1;
+        sched[k % R] = w;
+        mbar_arrive(sched_full(k % R));
+      } else {
+        w = item_of(k, ok);
+      }
+      if (w < 0) break;
       const int tile = FUSE ? w : w % tiles;
       const int n_begin = FUSE ? 0 : w / tiles, n_end = FUSE ? a.N : n_begin + 1;
       const int m0 = (tile / a.tiles_n) * 128, n0 = (tile % a.tiles_n) * TN;
@@ -850,7 +893,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
         if (!item_active(n)) continue;
         const int s = it % S;
         const uint32_t ph = (it / S) & 1u;
-        if (it >= pre) {                                  // (the early items already have their master tiles under way)
+        if (it >= pre && !dyn) {                          // (the early items already have their master tiles under way)
           ok = mbar_wait(stage_empty(s), ph ^ 1u, abort_flag, a.status, 0x201);
           if (!ok) break;
         }
@@ -882,7 +925,9 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
     const int ksteps = a.B / 16;
     uint32_t it = 0;
     bool ok = true;
-    for (int w = blockIdx.x; w < total_items && ok; w += gridDim.x) {
+    for (uint32_t k = 0; ok; ++k) {
+      const int w = item_of(k, ok);
+      if (w < 0) break;
       const int n_begin = FUSE ? 0 : w / tiles, n_end = FUSE ? a.N : n_begin + 1;
       for (int n = n_begin; n < n_end; ++n) {
         if (!item_active(n)) continue;
@@ -914,7 +959,9 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
 #pragma unroll
       for (int h = 0; h < NB64; ++h) tma_store_w(&mapShadow, ops_u32(s) + h * 16384u, a.wt, n0 + 64 * h, m0, n);
     };
-    for (int w = blockIdx.x; w < total_items && ok; w += gridDim.x) {
+    for (uint32_t k = 0; ok; ++k) {
+      const int w = item_of(k, ok);
+      if (w < 0) break;
       const int tile = FUSE ? w : w % tiles;
       const int m0 = (tile / a.tiles_n) * 128, n0 = (tile % a.tiles_n) * TN;
       if (!FUSE) {
@@ -999,7 +1046,10 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
     const bool vel_per_worker = FUSE && MOM && a.avg_vel == 0;      // the storer takes every worker's momentum tile
     uint32_t it = 0, tile_it = 0;
     bool ok = true;
-    for (int w = blockIdx.x; w < total_items && ok; w += gridDim.x, ++tile_it) {
+    for (uint32_t k = 0; ok; ++k, ++tile_it) {
+      const int w = item_of(k, ok);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok || w < 0) break;
       const int n_begin = FUSE ? 0 : w / tiles, n_end = FUSE ? a.N : n_begin + 1;
       float sum[NSUM], vsum[NVSUM];
       float xr[NXR];                                        // shared weights: the tile every worker starts from
@@ -1122,6 +1172,10 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
   tc_fence_before();
   __syncthreads();
   if (warp == 1) tmem_dealloc(tmem, 256u);
+  if (dyn) {             // the overlapped form: only now the launch before this one has to have completed
+    pdl_wait();
+    pdl_trigger();
+  }
 }
 
 // v <- mu v + G on two neighbouring 16-byte chunks (j, j + 1) of a 128-byte-swizzled fp32 row of the momentum
@@ -2127,6 +2181,8 @@ inline int tc_create(prsgd_ctx* c, std::string* err) {
     if (rc == PRSGD_OK && l > 1) {
       const uint64_t ldi = c->buf.ld[l - 1];
       rc = make_map3(&mp.act_in, false, c->buf.act_bk[l - 1], ldi, B, N, ldi * 2, B * ldi * 2, 64, (uint32_t)B, err);
+      if (rc == PRSGD_OK && l == 2)
+        rc = make_map3(&st->act1_alt, false, c->buf.act1_alt, ldi, B, N, ldi * 2, B * ldi * 2, 64, (uint32_t)B, err);
     }
   }
   if (rc == PRSGD_OK && c->L >= 2 && c->dims[c->L] <= 128) {      // the class layer's tiles with only as many rows as it has
@@ -2191,6 +2247,24 @@ inline int tc_bind_data(prsgd_ctx* c, std::string* err) {
 
 // The softmax cross-entropy gradient and every bias step run inside GEMM epilogues when the class
 // count fits one 128-row tile (and PRSGD_OPT_FUSED_EPILOGUES is on); otherwise as kernels of their own.
+// a_1 lives in one of two buffers (prsgd_ctx::a1_sel names the one of the current iteration); every other
+// activation has one.  tc_act_in: a_{l-1} as the operand of layer l's GEMMs; tc_act_ptr: a_l as plain memory.
+inline const CUtensorMap& tc_act_in(const prsgd_ctx* c, int l) {
+  const TcState* st = static_cast<const TcState*>(c->tc);
+  return (l == 2 && c->a1_sel != 0) ? st->act1_alt : st->layer[l - 1].act_in;
+}
+inline uint16_t* tc_act_ptr(const prsgd_ctx* c, int l) {
+  return (l == 1 && c->a1_sel != 0) ? c->buf.act1_alt : c->buf.act_bk[l];
+}
+
+// Early weight loads of the forward launch being enqueued: not right after an overlapped update, which may still
+// be writing the weights of layer 2 when that launch's CTAs start (the flag is consumed by the first launch).
+inline bool tc_forward_early_loads(prsgd_ctx* c) {
+  const bool quiet = !c->no_early_once;
+  c->no_early_once = false;
+  return c->early_loads != 0 && quiet;
+}
+
 inline bool tc_epilogues_fused(const prsgd_ctx* c) { return c->fused_epilogues != 0 && c->dims[c->L] <= 128; }
 
 // Right after a node average every worker's row holds the same bits (Algorithm 1: all workers restart from y),
@@ -2210,10 +2284,11 @@ inline void tc_launch_forward(prsgd_ctx* c, int l, const DrawArgs& dr, const uin
   a.B = c->B; a.N = c->N; a.k_steps = (ly.d_in / 64 + 1) / 2; a.M_total = ly.d_out; a.tiles_m = (ly.d_out + 127) / 128;
   a.stages = stream_stages(c->B); a.wt = tc_wtile(c, l);
   a.pool = l == 1; a.draw = dr; a.ld_out = c->buf.ld[l];
-  a.out_bk = c->buf.act_bk[l]; a.out_f32 = c->buf.act_f32[l];
+  a.out_bk = tc_act_ptr(c, l); a.out_f32 = c->buf.act_f32[l];
   a.bias = c->params + ly.b_off; a.bias_stride = c->m_pad;
   a.active = active; a.status = c->status;
-  a.prefetch = (l > 1 && active == nullptr && c->early_loads) ? 1 : 0;   // W_1 was written by the launch just before
+  const bool early = tc_forward_early_loads(c);
+  a.prefetch = (l > 1 && active == nullptr && early) ? 1 : 0;   // W_1 was written by the launch just before
   a.shared_w = tc_shared_restart(c, active) ? 1 : 0;
   const bool softmax = l == c->L && tc_epilogues_fused(c);
   if (softmax) {        // the softmax-CE gradient, the loss and the step of b_L happen in this launch's epilogue
@@ -2227,9 +2302,9 @@ inline void tc_launch_forward(prsgd_ctx* c, int l, const DrawArgs& dr, const uin
   dim3 grid(items < st->num_sms ? items : st->num_sms);
   const size_t smem = stream_smem_bytes(c->B, softmax);
   if (l < c->L)
-    launch_pdl(tc_stream_kernel<TC_FWD_RELU>, grid, kStreamThreads, smem, c->stream, st->layer[l - 1].shadow_k, st->layer[l - 1].act_in, a);
+    launch_pdl(tc_stream_kernel<TC_FWD_RELU>, grid, kStreamThreads, smem, c->stream, st->layer[l - 1].shadow_k, tc_act_in(c, l), a);
   else
-    launch_pdl(tc_stream_kernel<TC_FWD_LINEAR>, grid, kStreamThreads, smem, c->stream, st->layer[l - 1].shadow_k, st->layer[l - 1].act_in, a);
+    launch_pdl(tc_stream_kernel<TC_FWD_LINEAR>, grid, kStreamThreads, smem, c->stream, st->layer[l - 1].shadow_k, tc_act_in(c, l), a);
 }
 
 // The class layer's forward GEMM, softmax-CE gradient, step and dZ of the layer below as one launch of
@@ -2271,14 +2346,14 @@ inline void tc_launch_head(prsgd_ctx* c, const DrawArgs& dr, const uint8_t* acti
   if (with_forward) {
     a.fwd = 1; a.fwd_stages = tc_head_forward_stages(c);
     a.fwd_ksteps = (c->layer[L - 2].d_in / 64 + 1) / 2;
-    a.fwd_prefetch = (active == nullptr && c->early_loads) ? 1 : 0;
+    a.fwd_prefetch = (active == nullptr && tc_forward_early_loads(c)) ? 1 : 0;
     a.fwd_shared_w = tc_shared_restart(c, active) ? 1 : 0;
     a.wt_lo = tc_wtile(c, L - 1);
   }
   const unsigned cl = (unsigned)(ly.d_in / 128);
   const TcLayerMaps& lo = st->layer[L >= 2 ? L - 2 : 0];
   launch_pdl_cluster(tc_head_kernel, dim3(cl, (unsigned)c->N), dim3(kHeadThreads), head_smem_bytes(c->B, st->head_rows, a.fwd_stages),
-                     c->stream, cl, st->head_shadow, st->layer[L - 1].act_in, st->head_master, lo.shadow_k, lo.act_in, a);
+                     c->stream, cl, st->head_shadow, tc_act_in(c, L), st->head_master, lo.shadow_k, tc_act_in(c, L - 1), a);
 }
 
 // The per-worker flags the launches being enqueued honour: Algorithm 3's mask, or the mask of a worker group.
@@ -2304,6 +2379,7 @@ inline void tc_launch_forward_chain(prsgd_ctx* c, int l_first, int l_last, const
   a.draw = dr; a.active = active; a.status = c->status; a.bias_stride = c->m_pad;
   a.ready = c->chain_ready; a.done = c->chain_ready + (size_t)kChainMax * c->N;
   int items = 0;
+  const bool early = tc_forward_early_loads(c);
   for (int l = l_first; l <= l_last; ++l) {
     const Layer& ly = c->layer[l - 1];
     ChainSeg& g = a.seg[l - l_first];
@@ -2311,12 +2387,12 @@ inline void tc_launch_forward_chain(prsgd_ctx* c, int l_first, int l_last, const
     g.linear = l == c->L ? 1 : 0; g.pool = l == 1 ? 1 : 0; g.wt = tc_wtile(c, l);
     // early weight loads overlap whatever launch precedes the whole forward pass: only when that launch is known
     // to leave the weights of layers >= 2 alone (the layer-1 update or a bias launch that ended the iteration before)
-    g.prefetch = (l > 1 && active == nullptr && c->early_loads && c->upper_weights_quiet) ? 1 : 0;
+    g.prefetch = (l > 1 && active == nullptr && early && c->upper_weights_quiet) ? 1 : 0;
     g.item0 = items;
-    g.out_bk = c->buf.act_bk[l]; g.out_f32 = c->buf.act_f32[l]; g.bias = c->params + ly.b_off;
+    g.out_bk = tc_act_ptr(c, l); g.out_f32 = c->buf.act_f32[l]; g.bias = c->params + ly.b_off;
     items += g.tiles_m * c->N;
     maps.w[l - l_first] = st->layer[l - 1].shadow_k;
-    maps.b[l - l_first] = st->layer[l - 1].act_in;
+    maps.b[l - l_first] = tc_act_in(c, l);
   }
   for (int i = a.n_seg; i < kChainMax; ++i) { maps.w[i] = maps.w[0]; maps.b[i] = maps.b[0]; }
   a.total_items = items;
@@ -2332,15 +2408,15 @@ inline void tc_launch_forward_chain(prsgd_ctx* c, int l_first, int l_last, const
 }
 
 // dZ_{l-1} from dZ_l through W_l (l >= 2)
-inline void tc_launch_dx(prsgd_ctx* c, int l, const DrawArgs& dr, const uint8_t* active) {
+inline void tc_launch_dx(prsgd_ctx* c, int l, const DrawArgs& dr, const uint8_t* active, unsigned int* zero_word = nullptr) {
   TcState* st = static_cast<TcState*>(c->tc);
   const Layer& ly = c->layer[l - 1];
   StreamArgs a{};
   a.B = c->B; a.N = c->N; a.k_steps = (c->buf.ld[l] / 64 + 1) / 2; a.M_total = ly.d_in; a.tiles_m = (ly.d_in + 127) / 128;
   a.stages = stream_stages(c->B); a.wt = tc_wtile(c, l);
   a.pool = 0; a.draw = dr; a.ld_out = c->buf.ld[l - 1];
-  a.out_bk = c->buf.delta_bk[l - 1]; a.mask_src = c->buf.act_bk[l - 1];
-  a.active = active; a.status = c->status;
+  a.out_bk = c->buf.delta_bk[l - 1]; a.mask_src = tc_act_ptr(c, l - 1);
+  a.active = active; a.status = c->status; a.zero_word = zero_word;
   a.prefetch = (active == nullptr && c->early_loads) ? 1 : 0;
   a.shared_w = tc_shared_restart(c, active) ? 1 : 0;
   if (tc_epilogues_fused(c)) {      // the step of b_{l-1} rides on the epilogue that forms dZ_{l-1}
@@ -2354,13 +2430,14 @@ inline void tc_launch_dx(prsgd_ctx* c, int l, const DrawArgs& dr, const uint8_t*
 }
 
 template <int TN, bool MOM>
-inline void tc_launch_update_tn(prsgd_ctx* c, int l, const DrawArgs& dr, const uint8_t* active, bool fuse) {
+inline void tc_launch_update_tn(prsgd_ctx* c, int l, const DrawArgs& dr, const uint8_t* active, bool fuse, bool overlapped) {
   TcState* st = static_cast<TcState*>(c->tc);
   const Layer& ly = c->layer[l - 1];
   UpdateArgs a{};
   a.B = c->B; a.N = c->N; a.tiles_m = (ly.d_out + 127) / 128; a.tiles_n = (ly.d_in + TN - 1) / TN;
   a.gamma = c->gamma; a.mu = c->mu; a.pool = l == 1; a.draw = dr; a.active = active; a.status = c->status;
-  a.prefetch = (active == nullptr && c->early_loads) ? 1 : 0;
+  a.prefetch = (active == nullptr && c->early_loads && !overlapped) ? 1 : 0;
+  a.next_item = overlapped ? c->tile_counter : nullptr;       // (the caller has checked: plain step, no mask, not fused)
   a.shared_w = (fuse && tc_shared_restart(c, active)) ? 1 : 0; a.wt = tc_wtile(c, l);
   a.avg_vel = c->average_velocity ? 1 : 0;
   a.divisor = c->avg_divisor > 0.f ? c->avg_divisor : (float)c->N;
@@ -2370,14 +2447,14 @@ inline void tc_launch_update_tn(prsgd_ctx* c, int l, const DrawArgs& dr, const u
   const size_t smem = UpdCfg<TN, MOM>::smem(c->B);
   if constexpr (MOM) {
     if (fuse)
-      launch_pdl(tc_update_kernel<true, TN, true>, dim3(grid), kUpdThreads, smem, c->stream, mp.delta_out, mp.act_in, mp.master, mp.shadow_k, mp.velocity, a);
+      launch_pdl(tc_update_kernel<true, TN, true>, dim3(grid), kUpdThreads, smem, c->stream, mp.delta_out, tc_act_in(c, l), mp.master, mp.shadow_k, mp.velocity, a);
     else
-      launch_pdl(tc_update_kernel<false, TN, true>, dim3(grid), kUpdThreads, smem, c->stream, mp.delta_out, mp.act_in, mp.master, mp.shadow_k, mp.velocity, a);
+      launch_pdl(tc_update_kernel<false, TN, true>, dim3(grid), kUpdThreads, smem, c->stream, mp.delta_out, tc_act_in(c, l), mp.master, mp.shadow_k, mp.velocity, a);
   } else {
     if (fuse)
-      launch_pdl(tc_update_kernel<true, TN, false>, dim3(grid), kUpdThreads, smem, c->stream, mp.delta_out, mp.act_in, mp.master, mp.shadow_k, mp.master, a);
+      launch_pdl(tc_update_kernel<true, TN, false>, dim3(grid), kUpdThreads, smem, c->stream, mp.delta_out, tc_act_in(c, l), mp.master, mp.shadow_k, mp.master, a);
     else
-      launch_pdl(tc_update_kernel<false, TN, false>, dim3(grid), kUpdThreads, smem, c->stream, mp.delta_out, mp.act_in, mp.master, mp.shadow_k, mp.master, a);
+      launch_pdl(tc_update_kernel<false, TN, false>, dim3(grid), kUpdThreads, smem, c->stream, mp.delta_out, tc_act_in(c, l), mp.master, mp.shadow_k, mp.master, a);
   }
 }
 
@@ -2399,7 +2476,7 @@ inline void tc_launch_update_dx_m(prsgd_ctx* c, int l) {
   UpdateDxArgs a{};
   a.B = c->B; a.N = c->N; a.tiles_m = (ly.d_out + 127) / 128; a.tiles_n = (ly.d_in + TN - 1) / TN;
   a.gamma = c->gamma; a.status = c->status; a.stages = UpdDxCfg<TN, MOM, SP>::stages(c->B); a.wt = tc_wtile(c, l);
-  a.out_bk = c->buf.delta_bk[l - 1]; a.mask_src = c->buf.act_bk[l - 1]; a.ld_out = c->buf.ld[l - 1]; a.M_total = ly.d_in;
+  a.out_bk = c->buf.delta_bk[l - 1]; a.mask_src = tc_act_ptr(c, l - 1); a.ld_out = c->buf.ld[l - 1]; a.M_total = ly.d_in;
   a.bias_rw = c->params + c->layer[l - 2].b_off; a.bias_stride = c->m_pad;
   a.mu = c->mu; a.bias_vel = MOM ? c->velocity + c->layer[l - 2].b_off : nullptr;
   a.active = worker_mask(c);
@@ -2407,7 +2484,7 @@ inline void tc_launch_update_dx_m(prsgd_ctx* c, int l) {
   const int grid = items < st->num_sms ? items : st->num_sms;
   const TcLayerMaps& mp = st->layer[l - 1];
   launch_pdl(tc_update_dx_kernel<TN, MOM, SP>, dim3(grid), kUpdBlkThreads, UpdDxCfg<TN, MOM, SP>::smem(c->B), c->stream, mp.delta_out,
-             mp.act_in, mp.master, mp.shadow_k, MOM ? mp.velocity : mp.master, a);
+             tc_act_in(c, l), mp.master, mp.shadow_k, MOM ? mp.velocity : mp.master, a);
 }
 
 // 128-wide column blocks when every SM has a long queue of them and the operand boxes leave room for two
@@ -2452,7 +2529,7 @@ inline SplitArgs tc_split_plan(const prsgd_ctx* c, int64_t blocks, int tn, const
 
 // Update of layer 1 that also forms a_1 of the next iteration (tc_update_next_kernel).
 template <int TN, bool MOM>
-inline void tc_launch_update_next_tn(prsgd_ctx* c, const DrawArgs& dr) {
+inline void tc_launch_update_next_tn(prsgd_ctx* c, const DrawArgs& dr, bool other_a1) {
   TcState* st = static_cast<TcState*>(c->tc);
   const Layer& ly = c->layer[0];
   UpdateNextArgs a{};
@@ -2460,7 +2537,9 @@ inline void tc_launch_update_next_tn(prsgd_ctx* c, const DrawArgs& dr) {
   a.gamma = c->gamma; a.mu = c->mu; a.draw = dr; a.status = c->status;
   a.active = worker_mask(c);
   a.stages = UpdNextCfg<TN, MOM>::stages(c->B); a.wt = tc_wtile(c, 1);
-  a.next_out = c->buf.act_bk[1]; a.next_ld = c->buf.ld[1];
+  // (other_a1: something launched after this still reads the current a_1, so the next one goes to the other buffer)
+  a.next_out = other_a1 ? (c->a1_sel != 0 ? c->buf.act_bk[1] : c->buf.act1_alt) : tc_act_ptr(c, 1);
+  a.next_ld = c->buf.ld[1];
   a.bias = c->params + ly.b_off; a.bias_stride = c->m_pad; a.M_total = ly.d_out;
   int grid = 1;
   a.split = tc_split_plan(c, (int64_t)a.tiles_m * c->N, a.tiles_n, a.active, &grid);
@@ -2469,11 +2548,11 @@ inline void tc_launch_update_next_tn(prsgd_ctx* c, const DrawArgs& dr) {
              mp.act_in, mp.master, MOM ? mp.velocity : mp.master, a);
 }
 
-inline void tc_launch_update_next(prsgd_ctx* c, const DrawArgs& dr) {
+inline void tc_launch_update_next(prsgd_ctx* c, const DrawArgs& dr, bool other_a1 = false) {
   const TcState* st = static_cast<const TcState*>(c->tc);
   const Layer& ly = c->layer[0];
   if (c->velocity != nullptr) {            // momentum step: 64-wide tiles (two stages of master + momentum tiles)
-    tc_launch_update_next_tn<64, true>(c, dr);
+    tc_launch_update_next_tn<64, true>(c, dr, other_a1);
     return;
   }
   int tile = c->upd_tile;
@@ -2481,8 +2560,8 @@ inline void tc_launch_update_next(prsgd_ctx* c, const DrawArgs& dr) {
     const int64_t tiles128 = (int64_t)((ly.d_out + 127) / 128) * ((ly.d_in + 127) / 128);
     tile = (c->B <= 32 && tiles128 * c->N >= 32 * (int64_t)st->num_sms) ? 128 : 64;
   }
-  if (tile == 128 && UpdNextCfg<128, false>::stages(c->B) >= 2) tc_launch_update_next_tn<128, false>(c, dr);
-  else tc_launch_update_next_tn<64, false>(c, dr);
+  if (tile == 128 && UpdNextCfg<128, false>::stages(c->B) >= 2) tc_launch_update_next_tn<128, false>(c, dr, other_a1);
+  else tc_launch_update_next_tn<64, false>(c, dr, other_a1);
 }
 
 inline bool tc_layer_fuses_average(const prsgd_ctx* c, int l);
@@ -2508,7 +2587,7 @@ inline void tc_launch_update_common(prsgd_ctx* c, const int* layers, int n, cons
     g.tiles_n = (ly.d_in + 63) / 64; g.tile0 = tiles; g.pool = l == 1 ? 1 : 0; g.d_in = ly.d_in; g.d_out = ly.d_out;
     g.params = c->params + ly.w_off; g.shadow = c->shadow + ly.w_off; g.wt = tc_wtile(c, l);
     tiles += ((ly.d_out + 127) / 128) * g.tiles_n;
-    maps.delta[i] = st->layer[l - 1].delta_out; maps.act[i] = st->layer[l - 1].act_in; maps.master[i] = st->layer[l - 1].master;
+    maps.delta[i] = st->layer[l - 1].delta_out; maps.act[i] = tc_act_in(c, l); maps.master[i] = st->layer[l - 1].master;
   }
   for (int i = n; i < kCommonMax; ++i) { maps.delta[i] = maps.delta[0]; maps.act[i] = maps.act[0]; maps.master[i] = maps.master[0]; }
   a.tiles = tiles;
@@ -2531,11 +2610,11 @@ inline bool tc_layer_takes_common_point(const prsgd_ctx* c, int l, const uint8_t
 // operations per byte and win when every SM has a long queue of them; narrow tiles give four
 // pipeline stages and twice as many work items, which wins on small stores and on the fused form,
 // where a launch has only one item per tile.
-inline void tc_launch_update(prsgd_ctx* c, int l, const DrawArgs& dr, const uint8_t* active, bool fuse) {
+inline void tc_launch_update(prsgd_ctx* c, int l, const DrawArgs& dr, const uint8_t* active, bool fuse, bool overlapped = false) {
   const TcState* st = static_cast<const TcState*>(c->tc);
   const Layer& ly = c->layer[l - 1];
   if (c->velocity != nullptr) {            // momentum step: 64-wide tiles (two stages of master + momentum + output)
-    tc_launch_update_tn<64, true>(c, l, dr, active, fuse);
+    tc_launch_update_tn<64, true>(c, l, dr, active, fuse, overlapped);
     return;
   }
   int tile = c->upd_tile;
@@ -2544,8 +2623,8 @@ inline void tc_launch_update(prsgd_ctx* c, int l, const DrawArgs& dr, const uint
     if (fuse) tile = 2 * tiles128 >= 3 * (int64_t)st->num_sms ? 128 : 64;
     else tile = (c->B <= 32 && tiles128 * c->N >= 32 * (int64_t)st->num_sms) ? 128 : 64;
   }
-  if (tile == 128) tc_launch_update_tn<128, false>(c, l, dr, active, fuse);
-  else tc_launch_update_tn<64, false>(c, l, dr, active, fuse);
+  if (tile == 128) tc_launch_update_tn<128, false>(c, l, dr, active, fuse, overlapped);
+  else tc_launch_update_tn<64, false>(c, l, dr, active, fuse, overlapped);
 }
 
 // Bias step of all layers (after the last dZ has been formed).  On an averaging iteration it is followed

@@ -41,6 +41,16 @@ int fail(prsgd_ctx* ctx, int code, const std::string& msg) {
     prof_end(ctx);                                                                             \
   } while (0)
 
+// The same for a launch whose timing interval stays open: the next launch overlaps it and is timed with it.
+#define LAUNCH_CHECK_OPEN(ctx)                                                                 \
+  do {                                                                                         \
+    cudaError_t e__ = cudaGetLastError();                                                      \
+    if (e__ != cudaSuccess)                                                                    \
+      return fail((ctx), PRSGD_ERR_CUDA, std::string("kernel launch: ") + cudaGetErrorString(e__)); \
+    (ctx)->launches++;                                                                         \
+    (ctx)->open_launches++;                                                                    \
+  } while (0)
+
 // Optional per-kernel timing: an event pair around every launch of a family.
 void prof_begin(prsgd_ctx* c, int kind) {
   if (!c->profile) return;
@@ -53,13 +63,13 @@ void prof_begin(prsgd_ctx* c, int kind) {
     if (cudaEventCreate(&b) != cudaSuccess) { cudaEventDestroy(a); return; }
   }
   cudaEventRecord(a, c->stream);
-  c->open_kind = kind; c->open_a = a; c->open_b = b;
+  c->open_kind = kind; c->open_a = a; c->open_b = b; c->open_launches = 0;
 }
 
 void prof_end(prsgd_ctx* c) {
   if (!c->profile || c->open_kind < 0) return;
   cudaEventRecord(c->open_b, c->stream);
-  c->pending.push_back({c->open_kind, c->open_a, c->open_b});
+  c->pending.push_back({c->open_kind, c->open_a, c->open_b, c->open_launches + 1});
   c->open_kind = -1;
 }
 
@@ -149,9 +159,12 @@ size_t carve_scratch(int N, const prsgd_model_spec* s, int64_t m_pad, prsgd_ctx*
     for (int l = 0; l <= L; ++l) wmax = s->dims[l] > wmax ? s->dims[l] : wmax;
     auto spart = take(sizeof(float) * 2 * (size_t)kSplitMaxCtas * B * 128);
     auto scount = take(sizeof(unsigned int) * (size_t)N * ((wmax + 63) / 64));
+    auto tcount = take(sizeof(unsigned int));
+    auto a1alt = take(L > 1 ? 2 * (size_t)N * B * (size_t)round_up(s->dims[1], 64) : 0);
     if (ctx) {
       ctx->split_part = reinterpret_cast<float*>(spart);
       ctx->split_count = reinterpret_cast<unsigned int*>(scount);
+      ctx->tile_counter = reinterpret_cast<unsigned int*>(tcount);
     }
     for (int l = 1; l <= L; ++l) {
       const int ld = (int)round_up(s->dims[l], 64);
@@ -167,6 +180,7 @@ size_t carve_scratch(int N, const prsgd_model_spec* s, int64_t m_pad, prsgd_ctx*
         ctx->buf.delta_bk[l] = reinterpret_cast<uint16_t*>(dbk);
       }
     }
+    if (ctx) ctx->buf.act1_alt = L > 1 ? reinterpret_cast<uint16_t*>(a1alt) : nullptr;
   }
   return off;
 }
@@ -346,6 +360,7 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging, bool more_follow) {
   const bool next_fwd = c->next_forward && more_follow && !averaging && L > 1 && tc_epilogues_fused(c);
   const bool skip_f1 = c->a1_ready;
   c->a1_ready = false;
+  if (!skip_f1) c->a1_sel = 0;          // this iteration's first forward launch writes a_1: into the first buffer
   // The class layer as one launch of clusters (logits, softmax-CE gradient, step of W_L, dZ_{L-1}): whenever its
   // step is the plain one (a class layer large enough for the fused update + average keeps the separate launches).
   const bool head = tc_head_applies(c) && !(fuse && tc_layer_fuses_average(c, L));
@@ -385,6 +400,10 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging, bool more_follow) {
     tc_launch_head(c, dr, act_mask, head_fwd);
     LAUNCH_CHECK(c);
   }
+  // (every worker active, layer 2 on separate dX and update launches, layer 1's launch the folded one)
+  const bool overlap = c->overlap_update != 0 && next_fwd && L >= 3 && act_mask == nullptr &&
+                       !(dx_in_upd && (c->dx_in_update == 2 || tc_layer_folds_dx(c, 2)));
+  bool deferred = false;
   int common_layers[PRSGD_MAX_LAYERS], n_common = 0;     // layers whose averaged step is formed from the common point, in one launch at the end
   for (int l = L; l >= 1; --l) {          // dX_l reads W_l before the update of layer l overwrites it
     const bool fuse_l = fuse && tc_layer_fuses_average(c, l);
@@ -402,19 +421,32 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging, bool more_follow) {
       tc_launch_update_dx(c, l);
       LAUNCH_CHECK(c);
     } else {
+      // Layer 2's plain update waits for nothing that layer 1's launch produces, and that launch (whole row blocks
+      // per CTA) often leaves SMs idle: layer 2's update is enqueued after it, in the form that starts beside it.
+      const bool defer = l == 2 && overlap;
       if (l > 1) {
         prof_begin(c, PRSGD_KERNEL_DX);
-        tc_launch_dx(c, l, dr, act_mask);
+        tc_launch_dx(c, l, dr, act_mask, defer ? c->tile_counter : nullptr);
         LAUNCH_CHECK(c);
       }
-      prof_begin(c, fuse_l ? PRSGD_KERNEL_UPDATE_AVERAGE : PRSGD_KERNEL_UPDATE);
-      if (l == 1 && next_fwd) {
-        tc_launch_update_next(c, dr);
-        c->a1_ready = true;
+      if (defer) {
+        deferred = true;
       } else {
-        tc_launch_update(c, l, dr, act_mask, fuse_l);
+        prof_begin(c, fuse_l ? PRSGD_KERNEL_UPDATE_AVERAGE : PRSGD_KERNEL_UPDATE);
+        if (l == 1 && next_fwd) {
+          tc_launch_update_next(c, dr, deferred);         // (deferred: a_1 of iteration t + 1 goes to the other buffer)
+          c->a1_ready = true;
+          if (deferred) {
+            LAUNCH_CHECK_OPEN(c);
+            tc_launch_update(c, 2, dr, act_mask, false, true);     // still reads this iteration's a_1
+            c->a1_sel ^= 1;
+            c->no_early_once = true;
+          }
+        } else {
+          tc_launch_update(c, l, dr, act_mask, fuse_l);
+        }
+        LAUNCH_CHECK(c);
       }
-      LAUNCH_CHECK(c);
     }
     if (fuse && !fuse_l) {
       if (!c->merged_small_average) {        // (else with the bias segments, in the iteration's last launch)
@@ -449,8 +481,9 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging, bool more_follow) {
       LAUNCH_CHECK(c);
     }
   }
-  // the iteration ends with layer 1's update (or a bias launch after it): nothing in flight writes W_2..W_L
-  c->upper_weights_quiet = true;
+  // the iteration ends with layer 1's update (or a bias launch after it): nothing in flight writes W_2..W_L,
+  // unless layer 2's update was enqueued last
+  c->upper_weights_quiet = !deferred;
   return PRSGD_OK;
 }
 
@@ -785,7 +818,7 @@ void period_key(const prsgd_ctx* c, uint64_t (&key)[13]) {
   key[12] = (c->rows_identical ? 1u : 0u) | ((uint64_t)c->shared_restart << 1) | ((uint64_t)c->forward_chain << 2) |
             ((uint64_t)c->worker_groups << 3) | ((uint64_t)c->dx_shared_pair << 6) | ((uint64_t)c->head_kernel << 7) |
             ((uint64_t)c->common_point << 9) | ((uint64_t)c->split_blocks << 11) | ((uint64_t)c->head_forward << 13) |
-            ((uint64_t)c->merged_small_average << 14) | ((uint64_t)c->tiled_weights << 15);      // (rows_identical: the period's first iteration may share reads)
+            ((uint64_t)c->merged_small_average << 14) | ((uint64_t)c->tiled_weights << 15) | ((uint64_t)c->overlap_update << 16);      // (rows_identical: the period's first iteration may share reads)
 }
 
 // One whole averaging period (I iterations starting right after an average) as a CUDA graph: the
@@ -1209,6 +1242,7 @@ int prsgd_set_option(prsgd_ctx* c, int32_t option, int64_t value) {
     return PRSGD_OK;
   }
   if (option == PRSGD_OPT_HEAD_FORWARD) { c->head_forward = value != 0; return PRSGD_OK; }
+  if (option == PRSGD_OPT_OVERLAP_UPDATE) { c->overlap_update = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_MERGED_SMALL_AVERAGE) { c->merged_small_average = value != 0; return PRSGD_OK; }
   if (option == PRSGD_OPT_SPLIT_BLOCKS) {
     if (value < 0 || value > 2) return fail(c, PRSGD_ERR_ARG, "PRSGD_OPT_SPLIT_BLOCKS takes 0, 1 or 2");
@@ -1256,7 +1290,7 @@ int prsgd_get_profile(prsgd_ctx* c, int32_t family, double* ms_total, int64_t* l
     CUDA_TRY(c, cudaStreamSynchronize(c->stream));
     for (auto& p : c->pending) {
       float ms = 0.f;
-      if (cudaEventElapsedTime(&ms, p.a, p.b) == cudaSuccess) { c->prof_ms[p.kind] += ms; c->prof_count[p.kind]++; }
+      if (cudaEventElapsedTime(&ms, p.a, p.b) == cudaSuccess) { c->prof_ms[p.kind] += ms; c->prof_count[p.kind] += p.launches; }
       c->event_pool.push_back(p.a);
       c->event_pool.push_back(p.b);
     }

@@ -106,6 +106,7 @@ struct Buffers {
   // bf16 path: activations and deltas, batch-major rows [N][B][ld] with the leading dimension padded to 64
   uint16_t* act_bk[PRSGD_MAX_LAYERS + 1];
   uint16_t* delta_bk[PRSGD_MAX_LAYERS + 1];
+  uint16_t* act1_alt;                       // second buffer for a_1 (same shape as act_bk[1]), see prsgd_ctx::overlap_update
   int ld[PRSGD_MAX_LAYERS + 1];             // padded feature count of layer l's output
 };
 
@@ -141,6 +142,14 @@ struct prsgd_ctx {
   int dx_in_update = 1;          // layers >= 2: the update launch also forms dZ of the layer below (tensor-core path)
   int next_forward = 1;          // layer 1's update also forms a_1 of the next iteration (tensor-core path)
   bool a1_ready = false;         // a_1 of the coming iteration has already been formed by the previous update
+  // Layer 2's plain update launched AFTER layer 1's update + next forward and without a dependency wait at its
+  // start, so that its CTAs fill the SMs that launch leaves idle and take over the others as they drain (tiles are
+  // claimed from a device counter).  a_1 of the next iteration then goes to the other one of two buffers, because
+  // layer 2's update still reads this iteration's a_1 meanwhile.
+  int overlap_update = 1;
+  int a1_sel = 0;                        // which of the two a_1 buffers holds (or will receive) the current iteration's a_1
+  bool no_early_once = false;            // the next forward launch follows an overlapped update that writes W_2: no early weight loads
+  unsigned int* tile_counter = nullptr;  // the overlapped update's next unclaimed item; zeroed by the dX launch before it
   int early_loads = 1;           // tensor-core kernels request tiles nobody is writing before their dependency wait
   int fused_epilogues = 1;       // softmax-CE gradient and bias steps inside the GEMM epilogues (tensor-core path)
   int shared_restart = 1;        // the iteration after a node average reads worker 0's weights for every worker
@@ -207,9 +216,10 @@ struct prsgd_ctx {
   std::vector<PeriodGraph> graphs;
 
   // optional per-kernel timing (PRSGD_OPT_PROFILE)
-  struct Timed { int kind; cudaEvent_t a, b; };
+  struct Timed { int kind; cudaEvent_t a, b; int launches; };
   bool profile = false;
   int open_kind = -1;
+  int open_launches = 0;         // launches enqueued inside the open interval so far
   cudaEvent_t open_a = nullptr, open_b = nullptr;
   std::vector<Timed> pending;
   std::vector<cudaEvent_t> event_pool;
