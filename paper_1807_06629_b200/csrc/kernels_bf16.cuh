@@ -726,6 +726,10 @@ struct UpdateArgs {
   // block index: the loader claims the next one from *next_item (zero at launch) and hands the index to the other
   // roles through a ring in shared memory.
   unsigned int* next_item;
+  // 1: the same start and end (no dependency wait until just before the exit) with items dealt out by block index:
+  // for a launch enqueued right after a small one that it does not depend on (the averages of the bias segments),
+  // whose CTAs have all passed their own dependency wait before this one starts.
+  int late;
 };
 
 constexpr int kUpdSchedSlots = 8;         // ring of claimed item indices (>= twice the stage count)
@@ -798,6 +802,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
   auto sched_full = [&](uint32_t i) { return bar0 + 208u + 8u * i; };   // overlapped form: slot i of the ring holds an item index
   volatile int* sched = reinterpret_cast<volatile int*>(gen + (size_t)Cfg::kStages * stage_bytes + 272);
   const bool dyn = !FUSE && a.next_item != nullptr;
+  const bool late = dyn || a.late != 0;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t op_box = (uint32_t)a.B * 128u;       // one {64, B} box
@@ -847,7 +852,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
       ++pre;
     }
   }
-  if (!dyn) {
+  if (!late) {
     pdl_wait();          // set-up above overlapped the previous kernel's tail; dependent memory is touched below
     pdl_trigger();       // only now: the next launch's early loads may overlap this launch, never an older one
   }
@@ -1172,7 +1177,7 @@ __global__ void __launch_bounds__(kUpdThreads, 1) tc_update_kernel(const __grid_
   tc_fence_before();
   __syncthreads();
   if (warp == 1) tmem_dealloc(tmem, 256u);
-  if (dyn) {             // the overlapped form: only now the launch before this one has to have completed
+  if (late) {            // the overlapped forms: only now the launch before this one has to have completed
     pdl_wait();
     pdl_trigger();
   }
@@ -2430,14 +2435,15 @@ inline void tc_launch_dx(prsgd_ctx* c, int l, const DrawArgs& dr, const uint8_t*
 }
 
 template <int TN, bool MOM>
-inline void tc_launch_update_tn(prsgd_ctx* c, int l, const DrawArgs& dr, const uint8_t* active, bool fuse, bool overlapped) {
+inline void tc_launch_update_tn(prsgd_ctx* c, int l, const DrawArgs& dr, const uint8_t* active, bool fuse, bool overlapped, bool late) {
   TcState* st = static_cast<TcState*>(c->tc);
   const Layer& ly = c->layer[l - 1];
   UpdateArgs a{};
   a.B = c->B; a.N = c->N; a.tiles_m = (ly.d_out + 127) / 128; a.tiles_n = (ly.d_in + TN - 1) / TN;
   a.gamma = c->gamma; a.mu = c->mu; a.pool = l == 1; a.draw = dr; a.active = active; a.status = c->status;
   a.prefetch = (active == nullptr && c->early_loads && !overlapped) ? 1 : 0;
-  a.next_item = overlapped ? c->tile_counter : nullptr;       // (the caller has checked: plain step, no mask, not fused)
+  a.next_item = overlapped ? c->tile_counter : nullptr;       // (the caller has checked: no mask, not fused)
+  a.late = late ? 1 : 0;
   a.shared_w = (fuse && tc_shared_restart(c, active)) ? 1 : 0; a.wt = tc_wtile(c, l);
   a.avg_vel = c->average_velocity ? 1 : 0;
   a.divisor = c->avg_divisor > 0.f ? c->avg_divisor : (float)c->N;
@@ -2569,13 +2575,13 @@ inline bool tc_layer_fuses_average(const prsgd_ctx* c, int l);
 // Fused update + average from a common starting point for the layers in `layers` (n of them, 1-based, any order):
 // one weight-gradient GEMM per tile over the minibatches of all workers (tc_update_common_kernel), all layers'
 // tiles in one launch, the tiles of the last partly filled round cut into row ranges.
-inline void tc_launch_update_common(prsgd_ctx* c, const int* layers, int n, const DrawArgs& dr) {
+inline void tc_launch_update_common(prsgd_ctx* c, const int* layers, int n, const DrawArgs& dr, bool late = false) {
   TcState* st = static_cast<TcState*>(c->tc);
   CommonMaps maps;
   UpdateCommonArgs a{};
   a.B = c->B; a.N = c->N; a.n_seg = n;
   a.gamma = c->gamma; a.draw = dr; a.status = c->status;
-  a.prefetch = c->early_loads ? 1 : 0;
+  a.prefetch = c->early_loads ? 1 : 0; a.late = late ? 1 : 0;
   a.divisor = c->avg_divisor > 0.f ? c->avg_divisor : (float)c->N;
   a.stages = UpdCommonCfg::stages(c->B);
   a.m_pad = c->m_pad;
@@ -2610,11 +2616,12 @@ inline bool tc_layer_takes_common_point(const prsgd_ctx* c, int l, const uint8_t
 // operations per byte and win when every SM has a long queue of them; narrow tiles give four
 // pipeline stages and twice as many work items, which wins on small stores and on the fused form,
 // where a launch has only one item per tile.
-inline void tc_launch_update(prsgd_ctx* c, int l, const DrawArgs& dr, const uint8_t* active, bool fuse, bool overlapped = false) {
+inline void tc_launch_update(prsgd_ctx* c, int l, const DrawArgs& dr, const uint8_t* active, bool fuse, bool overlapped = false,
+                             bool late = false) {
   const TcState* st = static_cast<const TcState*>(c->tc);
   const Layer& ly = c->layer[l - 1];
   if (c->velocity != nullptr) {            // momentum step: 64-wide tiles (two stages of master + momentum + output)
-    tc_launch_update_tn<64, true>(c, l, dr, active, fuse, overlapped);
+    tc_launch_update_tn<64, true>(c, l, dr, active, fuse, overlapped, late);
     return;
   }
   int tile = c->upd_tile;
@@ -2623,8 +2630,8 @@ inline void tc_launch_update(prsgd_ctx* c, int l, const DrawArgs& dr, const uint
     if (fuse) tile = 2 * tiles128 >= 3 * (int64_t)st->num_sms ? 128 : 64;
     else tile = (c->B <= 32 && tiles128 * c->N >= 32 * (int64_t)st->num_sms) ? 128 : 64;
   }
-  if (tile == 128) tc_launch_update_tn<128, false>(c, l, dr, active, fuse, overlapped);
-  else tc_launch_update_tn<64, false>(c, l, dr, active, fuse, overlapped);
+  if (tile == 128) tc_launch_update_tn<128, false>(c, l, dr, active, fuse, overlapped, late);
+  else tc_launch_update_tn<64, false>(c, l, dr, active, fuse, overlapped, late);
 }
 
 // Bias step of all layers (after the last dZ has been formed).  On an averaging iteration it is followed

@@ -50,6 +50,7 @@ struct UpdateCommonArgs {
   DrawArgs draw;
   DeviceStatus* status;
   int prefetch;              // 1: the first master tile may be requested before the previous launch has completed
+  int late;                  // 1: no dependency wait at the start, one before the exit (see UpdateArgs::late)
   float divisor;             // the summed models N x - gamma sum_i G_i are divided by this (N; 1 leaves the row SUM)
   int stages;
   int64_t m_pad;
@@ -134,8 +135,10 @@ __global__ void __launch_bounds__(kUpdCommonThreads, 1) tc_update_common_kernel(
   // the first one is requested while that launch drains.
   const bool pre = a.prefetch != 0 && *abort_flag == 0 && n_items_all > 0;
   if (pre && warp == 0 && lane == 0) load_master(item_tile(0));
-  pdl_wait();
-  pdl_trigger();
+  if (a.late == 0) {
+    pdl_wait();
+    pdl_trigger();
+  }
   const uint32_t tmem = *tmem_slot;
   const int n_items = *abort_flag != 0 ? 0 : n_items_all;
 
@@ -286,6 +289,10 @@ __global__ void __launch_bounds__(kUpdCommonThreads, 1) tc_update_common_kernel(
   tc_fence_before();
   __syncthreads();
   if (warp == 1) tmem_dealloc(tmem, 128u);
+  if (a.late != 0) {
+    pdl_wait();
+    pdl_trigger();
+  }
 }
 
 }  // namespace prsgd

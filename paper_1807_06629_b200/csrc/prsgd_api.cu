@@ -404,6 +404,22 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging, bool more_follow) {
   const bool overlap = c->overlap_update != 0 && next_fwd && L >= 3 && act_mask == nullptr &&
                        !(dx_in_upd && (c->dx_in_update == 2 || tc_layer_folds_dx(c, 2)));
   bool deferred = false;
+  // Fused averaging iteration: the averages of the bias segments (and of the small weight segments) need every bias
+  // step, i.e. every dX launch, but not layer 1's fused update + average, the iteration's last big launch.  They are
+  // enqueued just before it and that launch starts beside them instead of being followed by them.
+  const bool small_first = c->overlap_update != 0 && fuse && epi && L >= 2 && act_mask == nullptr && tc_layer_fuses_average(c, 1);
+  bool small_done = false;
+  auto small_averages = [&]() -> int {
+    prof_begin(c, PRSGD_KERNEL_MISC);
+    tc_launch_bias_average(c, c->params, c->merged_small_average != 0);
+    LAUNCH_CHECK(c);
+    if (avg_vel) {
+      prof_begin(c, PRSGD_KERNEL_MISC);
+      tc_launch_bias_average(c, c->velocity);
+      LAUNCH_CHECK(c);
+    }
+    return PRSGD_OK;
+  };
   int common_layers[PRSGD_MAX_LAYERS], n_common = 0;     // layers whose averaged step is formed from the common point, in one launch at the end
   for (int l = L; l >= 1; --l) {          // dX_l reads W_l before the update of layer l overwrites it
     const bool fuse_l = fuse && tc_layer_fuses_average(c, l);
@@ -432,6 +448,12 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging, bool more_follow) {
       if (defer) {
         deferred = true;
       } else {
+        bool late = false;
+        if (l == 1 && small_first && fuse_l && n_common == 0) {   // (with layers waiting for the common-point launch: before that one)
+          const int rc = small_averages();
+          if (rc != PRSGD_OK) return rc;
+          small_done = late = true;
+        }
         prof_begin(c, fuse_l ? PRSGD_KERNEL_UPDATE_AVERAGE : PRSGD_KERNEL_UPDATE);
         if (l == 1 && next_fwd) {
           tc_launch_update_next(c, dr, deferred);         // (deferred: a_1 of iteration t + 1 goes to the other buffer)
@@ -443,7 +465,7 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging, bool more_follow) {
             c->no_early_once = true;
           }
         } else {
-          tc_launch_update(c, l, dr, act_mask, fuse_l);
+          tc_launch_update(c, l, dr, act_mask, fuse_l, false, late);
         }
         LAUNCH_CHECK(c);
       }
@@ -462,8 +484,14 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging, bool more_follow) {
     }
   }
   if (n_common > 0) {
+    bool late = false;
+    if (small_first && !small_done) {
+      const int rc = small_averages();
+      if (rc != PRSGD_OK) return rc;
+      small_done = late = true;
+    }
     prof_begin(c, PRSGD_KERNEL_UPDATE_AVERAGE);
-    tc_launch_update_common(c, common_layers, n_common, dr);
+    tc_launch_update_common(c, common_layers, n_common, dr, late);
     LAUNCH_CHECK(c);
   }
   if (!epi) {
@@ -471,19 +499,13 @@ int step_bf16(prsgd_ctx* c, int64_t t, bool averaging, bool more_follow) {
     tc_launch_bias(c, act_mask);
     LAUNCH_CHECK(c);
   }
-  if (fuse) {
-    prof_begin(c, PRSGD_KERNEL_MISC);
-    tc_launch_bias_average(c, c->params, c->merged_small_average != 0);
-    LAUNCH_CHECK(c);
-    if (avg_vel) {
-      prof_begin(c, PRSGD_KERNEL_MISC);
-      tc_launch_bias_average(c, c->velocity);
-      LAUNCH_CHECK(c);
-    }
+  if (fuse && !small_done) {
+    const int rc = small_averages();
+    if (rc != PRSGD_OK) return rc;
   }
-  // the iteration ends with layer 1's update (or a bias launch after it): nothing in flight writes W_2..W_L,
-  // unless layer 2's update was enqueued last
-  c->upper_weights_quiet = !deferred;
+  // a plain iteration ends with layer 1's update: nothing in flight writes W_2..W_L, unless layer 2's update was
+  // enqueued last; a fused averaging iteration ends with launches that write them
+  c->upper_weights_quiet = !deferred && !fuse;
   return PRSGD_OK;
 }
 

@@ -673,13 +673,15 @@ OVERLAP_CASES = [
     _w("tc-overlap-b64", 2, (192, 1024, 256, 10), 64, I=4),
     _w("tc-overlap-deep", 2, (64, 256, 384, 256, 100), 16, I=2),
     _w("tc-overlap-many", 20, (256, 1024, 512, 10), 32, I=5),
+    _w("tc-overlap-I1", 4, (128, 1024, 256, 10), 32, I=1),
 ]
 
 
 @pytest.mark.parametrize("w", OVERLAP_CASES, ids=[w.name for w in OVERLAP_CASES])
 def test_second_layers_update_beside_the_first_layers_changes_no_bit(torch_cuda, w):
     """Layer 2's update enqueued after layer 1's update + next forward and started beside it, tiles claimed from a
-    device counter, the next a_1 in a second buffer (PRSGD_OPT_OVERLAP_UPDATE), against the launches one after the
+    device counter, the next a_1 in a second buffer, and on fused averaging iterations the last big launch started
+    beside the averages of the small segments (PRSGD_OPT_OVERLAP_UPDATE), against the launches one after the
     other: every tile is formed from the same numbers in the same order, so parameters, bf16 copy, losses and node
     average are identical; with direct launches and replayed periods, both tile widths, the momentum step, calls
     that end inside a period, and more row blocks than SMs."""
@@ -687,7 +689,8 @@ def test_second_layers_update_beside_the_first_layers_changes_no_bit(torch_cuda,
     from paper_1807_06629_b200 import binding
     X, Y, x0 = make_inputs(w)
     T = 2 * w.I + 2
-    for name, opts in (("plain", {}), ("tile128", {binding.OPT_UPDATE_TILE: 128}), ("no-head", {binding.OPT_HEAD_KERNEL: 0}), ("momentum", {})):
+    for name, opts in (("plain", {}), ("tile128", {binding.OPT_UPDATE_TILE: 128}), ("no-head", {binding.OPT_HEAD_KERNEL: 0}), ("momentum", {}),
+                       ("momentum-averaged", {})):
         outs = []
         for overlap, graph in ((0, 0), (1, 0), (1, 1)):
             with torch.cuda.stream(torch.cuda.Stream()):
@@ -696,8 +699,8 @@ def test_second_layers_update_beside_the_first_layers_changes_no_bit(torch_cuda,
                 p.set_option(binding.OPT_GRAPH, graph)
                 for k, v in opts.items():
                     p.set_option(k, v)
-                if name == "momentum":
-                    p.enable_momentum(0.9)
+                if name.startswith("momentum"):
+                    p.enable_momentum(0.9, average_velocity=name.endswith("averaged"))
                 n0 = p.get_launch_count()
                 p.local_steps(w.I + 1)           # ends inside the second period
                 mid = p.get_params_stacked()
@@ -709,14 +712,14 @@ def test_second_layers_update_beside_the_first_layers_changes_no_bit(torch_cuda,
                     a, n = p.layout.w_off[l], w.dims[l] * w.dims[l + 1]
                     assert np.array_equal(shadow[:, a:a + n], synth.bf16_bits(store[:, a:a + n])), (w.name, name, l)
                 outs.append((p.get_params_stacked(), mid, p.get_losses(), p.get_average(), p.get_launch_count() - n0,
-                             p.get_velocity_stacked() if name == "momentum" else None))
+                             p.get_velocity_stacked() if name.startswith("momentum") else None))
                 torch.cuda.current_stream().synchronize()
                 p.close()
         for o in outs[1:]:
             assert np.array_equal(outs[0][0], o[0]), (w.name, name)
             assert np.array_equal(outs[0][1], o[1]), (w.name, name)
             assert np.array_equal(outs[0][2], o[2]) and np.array_equal(outs[0][3], o[3])
-            if name == "momentum":
+            if name.startswith("momentum"):
                 assert np.array_equal(outs[0][5], o[5])
         assert outs[0][4] == outs[1][4]
 
