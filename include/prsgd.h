@@ -92,8 +92,9 @@ typedef struct {
 int prsgd_layout(const prsgd_model_spec* spec, prsgd_layout_t* out);
 
 /* Bytes the caller must provide: params = N*m_pad*4; shadow = N*m_pad*2 for
- * BF16 precision, else 0; scratch = activations, deltas, logits, losses, the
- * draw table, one m_pad-float staging row and the status words.  Host only. */
+ * BF16 precision, else 0; scratch = activations (the first layer's twice for BF16
+ * precision), deltas, logits, losses, the draw table, two m_pad-float rows (staging,
+ * canonical order), counters and the status words.  Host only. */
 int prsgd_workspace_bytes(int32_t N, const prsgd_model_spec* spec,
                           size_t* params_bytes, size_t* shadow_bytes, size_t* scratch_bytes);
 
