@@ -901,11 +901,16 @@ int prsgd_local_steps(prsgd_ctx* c, int64_t k) {
     if (c->use_graph && !c->profile && c->I > 0 && k >= c->I && (c->t % c->I) == 0) {
       prsgd_ctx::PeriodGraph* g = get_period_graph(c);
       if (g != nullptr) {
-        counter_set_kernel<<<1, 1, 0, c->stream>>>(c->t_dev, c->t);
-        CUDA_TRY(c, cudaGetLastError());
+        if (c->t_dev_after != c->t) {                  // (a replayed period leaves the counter at the next period's start)
+          counter_set_kernel<<<1, 1, 0, c->stream>>>(c->t_dev, c->t);
+          CUDA_TRY(c, cudaGetLastError());
+          c->launches += 1;
+        }
+        c->t_dev_after = -1;
         CUDA_TRY(c, cudaGraphLaunch(g->exec, c->stream));
+        c->t_dev_after = c->t + c->I;
         c->rows_identical = true;                      // a period ends with the node average
-        c->launches += g->launches + 1;
+        c->launches += g->launches;
         c->t += c->I;
         k -= c->I;
         continue;

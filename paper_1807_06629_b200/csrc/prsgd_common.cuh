@@ -213,6 +213,7 @@ struct prsgd_ctx {
   int use_graph = 1;
   bool capturing = false;
   int64_t* t_dev = nullptr;      // device copy of t at the start of the period being replayed
+  int64_t t_dev_after = -1;      // what that counter will hold once the enqueued work has run (-1: not known)
   std::vector<PeriodGraph> graphs;
 
   // optional per-kernel timing (PRSGD_OPT_PROFILE)

@@ -1214,9 +1214,10 @@ def test_graph_replay_of_whole_periods_is_bit_identical(torch_cuda):
         assert np.array_equal(outs[0][0], outs[1][0])
         assert outs[0][1] == outs[1][1] and outs[0][2] == outs[1][2] == 6 * w.I + 1
         assert np.array_equal(outs[0][3], outs[1][3])
-        # same kernels, plus one counter-set launch per replayed period (three, then one after the new setting:
-        # the second request first walks to the period boundary with direct launches)
-        assert outs[1][4] == outs[0][4] + 4
+        # same kernels, plus one counter-set launch per run of replayed periods (a replay leaves the device counter
+        # at the next period's start): one before the three periods, one after the new setting, whose request first
+        # walks to the period boundary with direct launches
+        assert outs[1][4] == outs[0][4] + 2
 
 
 def test_expired_wait_is_reported_and_the_context_recovers(torch_cuda):
