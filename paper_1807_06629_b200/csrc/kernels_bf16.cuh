@@ -2502,7 +2502,10 @@ inline void tc_launch_update_dx(prsgd_ctx* c, int l) {
   int tile = c->upd_tile;
   if (tile == 0) {
     const int64_t blocks128 = (int64_t)((ly.d_in + 127) / 128) * c->N;
-    tile = (blocks128 >= 4 * (int64_t)st->num_sms && ly.d_out > 128) ? 128 : 64;
+    // (a layer of one row tile, the class layer, has one tile per block: the wide form halves the number of blocks,
+    // and with them the block epilogues that set its pace)
+    tile = (blocks128 >= 4 * (int64_t)st->num_sms && ly.d_out > 128) ||
+           (ly.d_out <= 128 && c->B <= 32 && blocks128 >= 2 * (int64_t)st->num_sms) ? 128 : 64;
   }
   if (tile == 128 && UpdDxCfg<128, false>::stages(c->B) >= 2) tc_launch_update_dx_m<128, false>(c, l);
   else if (c->dx_shared_pair) tc_launch_update_dx_m<64, false, true>(c, l);      // more stages (see UpdDxCfg)
@@ -2627,7 +2630,8 @@ inline void tc_launch_update(prsgd_ctx* c, int l, const DrawArgs& dr, const uint
   int tile = c->upd_tile;
   if (tile == 0) {
     const int64_t tiles128 = (int64_t)((ly.d_out + 127) / 128) * ((ly.d_in + 127) / 128);
-    if (fuse) tile = 2 * tiles128 >= 3 * (int64_t)st->num_sms ? 128 : 64;
+    // (fused form: a CTA owns a tile across all workers; wide tiles once one round of them nearly fills the GPU)
+    if (fuse) tile = (2 * tiles128 >= 3 * (int64_t)st->num_sms || (c->B <= 32 && 5 * tiles128 >= 4 * (int64_t)st->num_sms)) ? 128 : 64;
     else tile = (c->B <= 32 && tiles128 * c->N >= 32 * (int64_t)st->num_sms) ? 128 : 64;
   }
   if (tile == 128) tc_launch_update_tn<128, false>(c, l, dr, active, fuse, overlapped, late);
