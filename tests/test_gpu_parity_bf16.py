@@ -724,6 +724,32 @@ def test_second_layers_update_beside_the_first_layers_changes_no_bit(torch_cuda,
         assert outs[0][4] == outs[1][4]
 
 
+@pytest.mark.parametrize("I,T", [(16, 40), (1, 12), (3, 20)])
+def test_overlapped_launches_at_full_size_change_no_bit(torch_cuda, I, T):
+    """The 16-worker 3072-1024-1024-10 configuration as the benchmark runs it (replayed periods, 128 row-block CTAs
+    of layer 1's launch beside the claimed tiles of layer 2's update, the last big launch of an averaging iteration
+    beside the small averages) against the launches one after the other: identical parameters and losses, also
+    across calls that end inside a period and an odd number of iterations per period."""
+    torch = torch_cuda
+    from paper_1807_06629_b200 import binding
+    w = synth.WORKLOADS["cfg3"].with_(pool_samples=256, I=I)
+    X, Y, x0 = make_inputs(w)
+    outs = []
+    for overlap, graph in ((0, 0), (1, 1), (1, 0)):
+        with torch.cuda.stream(torch.cuda.Stream()):
+            p = make_ctx(w, X, Y, x0)
+            p.set_option(binding.OPT_OVERLAP_UPDATE, overlap)
+            p.set_option(binding.OPT_GRAPH, graph)
+            p.local_steps(5)
+            p.local_steps(T - 5)
+            p.sync()
+            outs.append((p.params.cpu().numpy().copy(), p.get_losses().copy()))
+            torch.cuda.current_stream().synchronize()
+            p.close()
+    for o in outs[1:]:
+        assert np.array_equal(outs[0][0], o[0]) and np.array_equal(outs[0][1], o[1])
+
+
 HEAD_FWD_CASES = [
     _w("tc-tail-small", 3, (128, 256, 128, 10), 32, I=3),
     _w("tc-tail-ragged-k", 2, (192, 320, 1024, 10), 64, I=2),
